@@ -1,0 +1,187 @@
+"""Oracle decode loops: greedy (Section 2), blockwise parallel decoding in
+its two-call form (Section 3) and in its merged form (Section 4).  Test
+infrastructure only (see the package docstring).
+
+Every loop is written against an ``invoke(dec_inputs, n_new)`` callable -- one
+*model invocation*: given decoder inputs u_0..u_t (u_0 the start token,
+u_t = y_t) it returns, for each of the last ``n_new`` positions, the argmax
+token of each of the k models p_1..p_k: an integer table [n_new][k].  Entry
+[r][i-1] for the position holding u_t is argmax p_i(y_{t+i} | y_<=t, x).
+Tests drive the loops with hand-made tables; ``TransformerScorer`` supplies
+the real model.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Callable, List, Optional, Sequence
+
+import numpy as np
+
+from .model import DecoderCache, OracleModel, argmax_lowest, decoder_full, encode, head_logits
+
+START_ID = 0
+
+
+@dataclass
+class DecodeResult:
+    ids: List[int]
+    khats: List[int] = field(default_factory=list)   # accepted block size per iteration
+    invocations: int = 0
+
+    @property
+    def iterations(self) -> int:
+        return len(self.khats)
+
+    @property
+    def mean_block(self) -> float:
+        """Mean accepted block size: tokens per decoding iteration (the
+        priming invocation is not an iteration)."""
+        return len(self.ids) / max(1, len(self.khats))
+
+
+# --------------------------------------------------------------------------- acceptance
+
+def accept_exact(proposal: int, row_p1: Sequence[int]) -> bool:
+    """Section 3, Verify: the proposal must equal the base model's argmax."""
+    return proposal == row_p1[0]
+
+
+def verify_prefix(block: Sequence[int], p1_of: Callable[[int], Sequence[int]],
+                  accept: Callable[[int, Sequence[int]], bool] = accept_exact) -> int:
+    """Largest khat such that proposal i is accepted for all 1 <= i <= khat.
+
+    ``block[i-1]`` is the proposal for y_{j+i}; ``p1_of(i)`` gives what the
+    acceptance test needs about p_1(y_{j+i} | y_<=j+i-1): a sequence whose first
+    entry is its argmax.  Proposal 1 is p_1's own argmax on the same prefix, so
+    khat >= 1 without testing it.
+    """
+    khat = 1
+    while khat < len(block) and accept(block[khat], p1_of(khat + 1)):
+        khat += 1
+    return khat
+
+
+def clip_termination(block: Sequence[int], khat: int, j: int, n_max: int, eos: int):
+    """Fixed-length termination clips the accepted count to the tokens still
+    wanted; with an end-of-sequence id the block is cut after the first
+    accepted EOS.  Returns (khat, finished)."""
+    khat = min(khat, n_max - j)
+    finished = (j + khat >= n_max)
+    if eos >= 0:
+        for i in range(khat):
+            if block[i] == eos:
+                return i + 1, True
+    return khat, finished
+
+
+# --------------------------------------------------------------------------- loops
+
+def greedy(invoke, n_max: int, eos: int = -1) -> DecodeResult:
+    """Section 2: extend with argmax p_1 one token at a time."""
+    res = DecodeResult(ids=[])
+    inputs = [START_ID]
+    while len(res.ids) < n_max:
+        tok = int(invoke(inputs, 1)[0][0])
+        res.invocations += 1
+        res.ids.append(tok)
+        res.khats.append(1)
+        inputs.append(tok)
+        if eos >= 0 and tok == eos:
+            break
+    return res
+
+
+TailFn = Callable[[int, int], Sequence[int]]   # (j accepted so far, iteration index) -> proposals 2..k
+
+
+def blockwise_twocall(invoke, k: int, n_max: int, eos: int = -1,
+                      tail_fn: Optional[TailFn] = None, accept=accept_exact) -> DecodeResult:
+    """Section 3 literally: a Predict invocation on the accepted prefix, then a
+    Verify invocation on prefix + block; two invocations per iteration."""
+    res = DecodeResult(ids=[])
+    inputs = [START_ID]
+    while True:
+        j = len(res.ids)
+        block = [int(t) for t in invoke(inputs, 1)[0][:k]]                 # Predict
+        if tail_fn is not None:
+            block[1:] = [int(t) for t in tail_fn(j, res.iterations)]
+        table = invoke(inputs + block, k)                                  # Verify
+        res.invocations += 2
+        # p_1 for y_{j+i} is conditioned on y_<=j+i-1, i.e. sits at the position of proposal i-1
+        khat = verify_prefix(block, lambda i: [table[i - 2][0]], accept)
+        khat, finished = clip_termination(block, khat, j, n_max, eos)
+        res.ids += block[:khat]
+        res.khats.append(khat)
+        inputs += block[:khat]
+        if finished:
+            return res
+
+
+def blockwise_merged(invoke, k: int, n_max: int, eos: int = -1,
+                     tail_fn: Optional[TailFn] = None, accept=accept_exact) -> DecodeResult:
+    """Section 4: the combined model returns all k heads at all k block
+    positions, so the row of the last accepted position is the next Predict;
+    one priming invocation, then one invocation per iteration."""
+    res = DecodeResult(ids=[])
+    inputs = [START_ID]
+    block = [int(t) for t in invoke(inputs, 1)[0][:k]]                     # priming pass
+    res.invocations = 1
+    while True:
+        j = len(res.ids)
+        if tail_fn is not None:
+            block[1:] = [int(t) for t in tail_fn(j, res.iterations)]
+        table = invoke(inputs + block, k)
+        res.invocations += 1
+        khat = verify_prefix(block, lambda i: [table[i - 2][0]], accept)
+        khat, finished = clip_termination(block, khat, j, n_max, eos)
+        res.ids += block[:khat]
+        res.khats.append(khat)
+        inputs += block[:khat]
+        if finished:
+            return res
+        block = [int(t) for t in table[khat - 1][:k]]                      # reuse row khat
+
+
+# --------------------------------------------------------------------------- the real model
+
+class TransformerScorer:
+    """``invoke`` backed by the oracle Transformer for one source row.
+
+    cached=False recomputes the whole decoder over the prefix at every call
+    (the plain definition); cached=True keeps self-attention K/V of accepted
+    positions and only runs the new ones.  ``last_logits`` / ``last_hidden``
+    hold the [n_new, k, V] logits and [n_new, d] decoder outputs of the latest
+    call."""
+
+    def __init__(self, m: OracleModel, src_ids, src_len: Optional[int] = None, k: Optional[int] = None,
+                 cached: bool = False, capacity: int = 0):
+        self.m = m
+        self.k = m.k_model if k is None else k
+        self.src_len = len(src_ids) if src_len is None else int(src_len)
+        self.memory = encode(m, src_ids, self.src_len)
+        self.cached = cached
+        self.cache = DecoderCache(m, self.memory, self.src_len, capacity) if cached else None
+        self.inputs_seen: List[int] = []
+        self.last_logits = None
+        self.last_hidden = None
+
+    def logits(self, dec_inputs: Sequence[int], n_new: int) -> np.ndarray:
+        if not self.cached:
+            h = decoder_full(self.m, self.memory, self.src_len, dec_inputs)[-n_new:]
+        else:
+            keep = len(dec_inputs) - n_new
+            c = self.cache
+            # positions already run and now part of the accepted prefix become live
+            if keep < c.length or list(dec_inputs[:c.length]) != self.inputs_seen[:c.length]:
+                raise ValueError("cache does not hold this prefix")
+            if list(dec_inputs[c.length:keep]) != self.inputs_seen[c.length:keep]:
+                raise ValueError("prefix extends beyond what the last pass computed")
+            c.commit(keep - c.length)
+            h = c.extend(dec_inputs[keep:])
+            self.inputs_seen = list(dec_inputs)
+        self.last_hidden = h
+        self.last_logits = head_logits(self.m, h, self.k)
+        return self.last_logits
+
+    def __call__(self, dec_inputs: Sequence[int], n_new: int) -> np.ndarray:
+        return argmax_lowest(self.logits(dec_inputs, n_new))
