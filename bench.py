@@ -1,0 +1,347 @@
+#!/usr/bin/env python
+"""Benchmark of the blockwise-parallel-decoding hot path on B200.
+
+One *step* is one complete decode of the headline workload (big model,
+d_model 1024, k = 8, batch 1, 128 tokens) under controlled acceptance: every
+merged score-and-propose iteration runs the decoder pass over the k block
+positions, the k heads, the fused vocabulary top-1, verification and the cache
+commit.  `value` is decoded tokens/s with everything resident on the device;
+`e2e` goes through the public calls with host buffers (source ids in, token ids
+out, encoder included).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from bpd_inputs import WORKLOADS, forced_tail, geometric_schedule, make_source, make_weights  # noqa: E402
+
+METRIC = "decoded tokens/s at batch 1 (d=1024, k=8)"
+HEADLINE = "C3"
+MEAN_ACCEPT = 5.0            # geometric mean of the controlled-acceptance schedule for the headline line
+NOMINAL_HBM_GBS = 8000.0
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def iteration_bytes(cfg, k, batch, mean_T, mean_S):
+    """Bytes one merged iteration must move: every weight once, the cache once."""
+    e = cfg.elem_bytes
+    d, f, V, L, fh, km = cfg.d_model, cfg.d_ff, cfg.vocab, cfg.n_dec, cfg.d_hidden, cfg.k_model
+    layers = L * (4 * d * d + 2 * d * d + 2 * d * f)
+    w1 = d * km * fh if cfg.head_layout == 0 else d * k * fh
+    w2 = k * d * km * fh if cfg.head_layout == 0 else k * d * fh
+    return e * (layers + w1 + w2 + V * d) + batch * L * 2 * e * d * (mean_T + mean_S), e * w2
+
+
+def build_plan(w, greedy_ids, k, mean):
+    plan = np.zeros((w.batch, w.n_decode, k - 1), dtype=np.int32)
+    khats = []
+    for b in range(w.batch):
+        G, R = geometric_schedule(w.accept_seed * 1000 + b, mean, w.n_decode + 1)
+        for j in range(w.n_decode):
+            plan[b, j] = forced_tail(greedy_ids[b], j, k, int(G[j]), int(R[j]), w.cfg.vocab)
+        j = 0
+        while j < w.n_decode:
+            kh = min(k, int(G[j]), w.n_decode - j)
+            khats.append(kh)
+            j += kh
+    return plan, khats
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle samples while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            self.proc.terminate()
+            self.proc.wait()
+            self.t.join(timeout=2)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[1])); mx.append(float(r[2]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------- oracle legs (CPU)
+
+def oracle_sample(w, blob, src, src_len, k, mean, n_tokens, repeats=1):
+    """Time the oracle's merged blockwise decode (cached forward) on the first
+    ``n_tokens`` tokens of row 0.  Returns (tokens/s, seconds per decode, threads)."""
+    from oracle.decode import TransformerScorer, blockwise_merged, greedy
+    from oracle.model import parse_blob
+    om = parse_blob(blob)
+    row = src[0, :src_len[0]]
+    g = np.array(greedy(TransformerScorer(om, row, k=1, cached=True, capacity=n_tokens + 4), n_tokens).ids)
+    G, R = geometric_schedule(w.accept_seed * 1000, mean, n_tokens + 1)
+    times = []
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        sc = TransformerScorer(om, row, k=k, cached=True, capacity=n_tokens + 2 * k + 2)
+        res = blockwise_merged(sc, k, n_tokens,
+                               tail_fn=lambda j, it: forced_tail(g, j, k, int(G[j]), int(R[j]), w.cfg.vocab))
+        times.append(time.perf_counter() - t0)
+        assert res.ids == list(g)
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    return n_tokens / float(np.mean(times)), times, threads
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = WORKLOADS[HEADLINE]
+    k = w.cfg.k_model
+    blob = make_weights(w.cfg, w.weight_seed, w.sigma)
+    src, src_len = make_source(w)
+    n_tokens = 12
+    tps, times, threads = oracle_sample(w, blob, src, src_len, k, MEAN_ACCEPT, n_tokens,
+                                        repeats=args.steps + args.warmup)
+    timed = times[args.warmup:]
+    value = n_tokens / float(np.mean(timed))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * float(np.mean(timed)),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{HEADLINE}: big enc-dec 6+6, d_model 1024, k=8, batch 1 "
+                               f"(oracle sample: first {n_tokens} tokens, controlled acceptance mean {MEAN_ACCEPT})"},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+                         "sample": f"first {n_tokens} of {w.n_decode} tokens per step"},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- GPU arm
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_1811_03115_b200.build import build_library
+    build_library()
+    import paper_1811_03115_b200 as bpd
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+
+    w = WORKLOADS[HEADLINE]
+    cfg, k, N = w.cfg, w.cfg.k_model, w.n_decode
+    blob = make_weights(cfg, w.weight_seed, w.sigma)
+    src, src_len = make_source(w)
+    model = bpd.Model(blob, dev)
+    sess = bpd.Session(model, w.batch, w.max_src, N)
+    sess.bpd_encode(src, src_len)
+    g_ids, _, g_st = sess.bpd_decode_greedy(N)
+    plan, khats = build_plan(w, g_ids, k, MEAN_ACCEPT)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed_decodes(n_steps, mode):
+        """Device-resident: state rewound on the device, results left on the device."""
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        ev0.record()
+        for _ in range(n_steps):
+            sess.bpd_rewind()
+            if mode == "greedy":
+                sess.bpd_decode_greedy(N, fetch=False)
+            else:
+                sess.bpd_decode_blockwise(k, N, fetch=False)
+        ev1.record()
+        barrier()
+        return ev0.elapsed_time(ev1) / n_steps      # ms per decode
+
+    def max_over_ranks(ms):
+        if world > 1:
+            t = torch.tensor([ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            return float(t.item())
+        return ms
+
+    # ---- headline: controlled acceptance, device resident
+    sess.bpd_encode(src, src_len)
+    sess.bpd_set_forced_plan(plan, k)
+    timed_decodes(args.warmup, "block")
+    launches0 = bpd.bpd_kernel_launches()
+    with ClockSampler(local) as clocks:
+        ms_step = max_over_ranks(timed_decodes(args.steps, "block"))
+    launches = bpd.bpd_kernel_launches() - launches0
+    ids, _, st = sess.bpd_fetch_output(N)
+    assert np.array_equal(ids, g_ids), "controlled-acceptance decode differs from greedy"
+    assert st.row_iterations == len(khats)
+    iters = st.iterations
+    us_iter = 1e3 * ms_step / iters
+    value = world * w.batch * N / (ms_step * 1e-3)
+
+    # ---- per-phase timing of the same decode (events inside the pass), for the roofline of the dominant kernel
+    sess.bpd_profile(True)
+    timed_decodes(max(1, min(args.steps, 5)), "block")
+    phases = [sess.bpd_profile_read(p) for p in range(4)]
+    sess.bpd_profile(False)
+    peak, peak_kind = _peaks()
+    mean_T = 1 + N / 2.0
+    it_bytes, w2_bytes = iteration_bytes(cfg, k, w.batch, mean_T, float(src_len.mean()))
+    n_w2, ms_w2 = phases[2]
+    # the priming pass evaluates the same k heads on one row: same weight bytes per launch
+    w2_us = 1e3 * ms_w2 / max(1, n_w2)
+    achieved = w2_bytes / (w2_us * 1e-6) / 1e9
+    roofline = {"bound": "hbm", "kernel": "head output layers (k*d_model x k*d_hidden weights, + residual)",
+                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "peak_kind": f"of {peak_kind}", "traffic": None,
+                "bytes_per_launch": w2_bytes, "us_per_launch": w2_us, "launches_timed": n_w2}
+    phase_us = {name: (1e3 * ms / max(1, n)) for name, (n, ms) in
+                zip(["layers", "head_hidden", "head_output", "vocab_top1"], phases)}
+
+    # ---- other modes (context): greedy, free-running blockwise, mean-2 acceptance
+    extra = {}
+    if rank == 0 and not args.quick:
+        sess.bpd_encode(src, src_len)
+        timed_decodes(1, "greedy")
+        ms_g = timed_decodes(max(1, args.steps // 2), "greedy")
+        extra["greedy"] = {"tokens_per_s": N / (ms_g * 1e-3), "us_per_pass": 1e3 * ms_g / N}
+        sess.bpd_encode(src, src_len)
+        timed_decodes(1, "block")
+        ms_f = timed_decodes(max(1, args.steps // 2), "block")
+        _, _, st_f = sess.bpd_fetch_output(N)
+        extra["blockwise_free"] = {"tokens_per_s": N / (ms_f * 1e-3), "us_per_iteration": 1e3 * ms_f / st_f.iterations,
+                                   "mean_block": st_f.mean_block}
+        plan2, kh2 = build_plan(w, g_ids, k, 2.0)
+        sess.bpd_encode(src, src_len)
+        sess.bpd_set_forced_plan(plan2, k)
+        timed_decodes(1, "block")
+        ms_2 = timed_decodes(max(1, args.steps // 2), "block")
+        extra["controlled_mean2"] = {"tokens_per_s": N / (ms_2 * 1e-3), "us_per_iteration": 1e3 * ms_2 / len(kh2),
+                                     "mean_block": N / len(kh2)}
+
+    # ---- end to end through the public calls with host buffers
+    sess.bpd_encode(src, src_len)
+    e2e_times = []
+    for i in range(args.warmup + args.steps):
+        barrier()
+        t0 = time.perf_counter()
+        sess.bpd_encode(src, src_len)                 # H2D of the source ids + encoder
+        sess.bpd_set_forced_plan(plan, k)             # H2D of the acceptance plan
+        out_ids, out_len, _ = sess.bpd_decode_blockwise(k, N)   # D2H of the token ids
+        torch.cuda.synchronize()
+        e2e_times.append(time.perf_counter() - t0)
+    e2e_ms = max_over_ranks(1e3 * float(np.mean(e2e_times[args.warmup:])))
+    h2d = src.nbytes + src_len.nbytes + plan.nbytes
+    d2h = w.batch * N * 4 + w.batch * 4 + (3 + 17) * 8
+
+    if rank != 0:
+        return
+    # ---- oracle on the host cores, bounded sample
+    cpu = None
+    if not args.no_cpu:
+        n_tok = 12
+        tps, times, threads = oracle_sample(w, blob, src, src_len, k, MEAN_ACCEPT, n_tok, repeats=2)
+        cpu = {"value": tps, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+               "sample": f"first {n_tok} of {N} tokens, 2 decodes, {np.mean(times):.1f} s each"}
+    line = {
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{HEADLINE}: big enc-dec 6+6, d_model 1024, 16 heads, FFN 4096, vocab 32768, "
+                               f"k=8 dense heads, batch 1, source 40 ids, decode {N} tokens, controlled acceptance "
+                               f"(geometric mean {MEAN_ACCEPT}, mean accepted block {N / len(khats):.2f})",
+                   "l2": "weights (847 MB per iteration) exceed L2; no flush needed",
+                   "replicas": world},
+        "us_per_iteration": us_iter, "iterations_per_step": iters,
+        "iteration_hbm_gbs": it_bytes / (us_iter * 1e-6) / 1e9,
+        "iteration_frac_of_8tbs": it_bytes / (us_iter * 1e-6) / 1e9 / NOMINAL_HBM_GBS,
+        "iteration_frac_of_measured": it_bytes / (us_iter * 1e-6) / 1e9 / peak,
+        "phase_us": phase_us, "modes": extra,
+        "clocks": clocks.summary(),
+        "e2e": {"value": world * w.batch * N / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--quick", action="store_true", help="skip the context modes")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the oracle leg")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,786 @@
+// C ABI of the blockwise-parallel-decoding library: blob parsing, buffer
+// planning, the encoder, the decoder pass and the decode loops.
+#include <math.h>
+#include <string.h>
+
+#include <algorithm>
+#include <atomic>
+#include <new>
+
+#include "host.hpp"
+#include "kernels_simt.cuh"
+
+namespace bpd {
+
+thread_local char g_err[512] = "";
+
+int fail(int code, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  return code;
+}
+
+static inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// ------------------------------------------------------------------ blob
+static const char kMagic[8] = {'B', 'P', 'D', 'W', '0', '0', '0', '1'};
+
+int parse_blob(const void* blob, size_t n, ParsedBlob* out) {
+  if (!blob) return fail(BPD_E_INVALID, "blob is null");
+  if (n < 128) return fail(BPD_E_FORMAT, "blob shorter than its header (%zu bytes)", n);
+  const unsigned char* p = static_cast<const unsigned char*>(blob);
+  if (memcmp(p, kMagic, 8) != 0) return fail(BPD_E_FORMAT, "bad magic");
+  int32_t f[12];
+  memcpy(f, p + 8, sizeof(f));
+  float eps;
+  memcpy(&eps, p + 56, 4);
+  int32_t n_tensors;
+  memcpy(&n_tensors, p + 60, 4);
+  uint64_t dir_off, data_off, total;
+  memcpy(&dir_off, p + 64, 8);
+  memcpy(&data_off, p + 72, 8);
+  memcpy(&total, p + 80, 8);
+  if (f[0] != 1) return fail(BPD_E_FORMAT, "unsupported blob version %d", f[0]);
+  if (total != n) return fail(BPD_E_FORMAT, "blob size %zu does not match header %llu", n, (unsigned long long)total);
+  Config& c = out->cfg;
+  c.dtype = f[1]; c.n_enc = f[2]; c.n_dec = f[3]; c.d = f[4]; c.H = f[5]; c.d_ff = f[6]; c.V = f[7];
+  c.k_model = f[8]; c.d_hidden = f[9]; c.head_layout = f[10]; c.p1_identity = f[11]; c.eps = eps;
+  if (c.dtype != 0 && c.dtype != 1) return fail(BPD_E_FORMAT, "unknown dtype %d", c.dtype);
+  if (c.n_enc < 1 || c.n_dec < 1 || c.n_enc > 64 || c.n_dec > 64) return fail(BPD_E_FORMAT, "bad layer counts");
+  if (c.d < 8 || c.d % 8 || c.H < 1 || c.d % c.H) return fail(BPD_E_FORMAT, "bad d_model/heads %d/%d", c.d, c.H);
+  const int dh = c.d / c.H;
+  if (dh % 8 || dh > 128) return fail(BPD_E_UNSUPPORTED, "head width %d (need a multiple of 8, at most 128)", dh);
+  if (c.d > kArgmaxMaxD) return fail(BPD_E_UNSUPPORTED, "d_model %d above %d", c.d, kArgmaxMaxD);
+  if (c.d_ff < 8 || c.d_ff % 8 || c.d_hidden < 8 || c.d_hidden % 8) return fail(BPD_E_FORMAT, "bad FFN widths");
+  if (c.V < 2) return fail(BPD_E_FORMAT, "bad vocabulary size %d", c.V);
+  if (c.k_model < 1 || c.k_model > kMaxK) return fail(BPD_E_UNSUPPORTED, "k_model %d outside 1..%d", c.k_model, kMaxK);
+  if (c.head_layout != 0 && c.head_layout != 1) return fail(BPD_E_FORMAT, "unknown head layout %d", c.head_layout);
+  if (!(eps > 0.f)) return fail(BPD_E_FORMAT, "bad layer-norm eps");
+  if (n_tensors < 1 || dir_off != 128 || dir_off + 96ull * n_tensors > n || data_off > n)
+    return fail(BPD_E_FORMAT, "bad directory");
+  for (int t = 0; t < n_tensors; ++t) {
+    const unsigned char* e = p + dir_off + 96ull * t;
+    char name[65];
+    memcpy(name, e, 64);
+    name[64] = 0;
+    TensorEntry te;
+    memcpy(&te.ndim, e + 64, 4);
+    memcpy(te.dims, e + 68, 12);
+    memcpy(&te.offset, e + 80, 8);
+    memcpy(&te.nbytes, e + 88, 8);
+    if (te.ndim < 1 || te.ndim > 3) return fail(BPD_E_FORMAT, "tensor %s: bad rank", name);
+    uint64_t cnt = 1;
+    for (int i = 0; i < te.ndim; ++i) {
+      if (te.dims[i] < 1) return fail(BPD_E_FORMAT, "tensor %s: bad dimension", name);
+      cnt *= (uint64_t)te.dims[i];
+    }
+    if (cnt * c.elem() != te.nbytes || te.offset % 256 || te.offset < data_off || te.offset + te.nbytes > n)
+      return fail(BPD_E_FORMAT, "tensor %s: bad extent", name);
+    out->t[name] = te;
+  }
+  out->total = total;
+  return BPD_OK;
+}
+
+static int find(const ParsedBlob& pb, char* base, const std::string& name, std::initializer_list<int> shape,
+                const void** out) {
+  auto it = pb.t.find(name);
+  if (it == pb.t.end()) return fail(BPD_E_FORMAT, "tensor %s missing", name.c_str());
+  const TensorEntry& te = it->second;
+  if (te.ndim != (int)shape.size()) return fail(BPD_E_FORMAT, "tensor %s: rank %d", name.c_str(), te.ndim);
+  int i = 0;
+  for (int s : shape)
+    if (te.dims[i++] != s) return fail(BPD_E_FORMAT, "tensor %s: dimension %d is %d, want %d", name.c_str(), i - 1, te.dims[i - 1], s);
+  *out = base + te.offset;
+  return BPD_OK;
+}
+
+// ------------------------------------------------------------------ session planning
+struct Arena {
+  size_t off = 0;
+  char* base = nullptr;
+  template <typename T> T* take(size_t count) {
+    off = align_up(off);
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += count * sizeof(T);
+    return p;
+  }
+  void* take_bytes(size_t n) { return take<char>(n); }
+};
+
+static int pages_per_row(const Config& c, int max_tgt) { return ceil_div(max_tgt + 1 + c.k_model, kPage); }
+
+// Lays the session out; with base == nullptr only measures.
+static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, char* base, bpd_session* s) {
+  Arena a;
+  a.base = base;
+  const size_t ea = c.elem();
+  const size_t Rmax = (size_t)B * c.k_model, E = (size_t)B * max_src, Rall = std::max(Rmax, E);
+  const size_t R2 = Rmax * c.k_model;
+  const int ppr = pages_per_row(c, max_tgt);
+  const size_t d = c.d;
+  float* x = a.take<float>(Rall * d);
+  float* h_f32 = a.take<float>(Rmax * d);
+  void* xn = a.take_bytes(Rall * d * ea);
+  void* qbuf = a.take_bytes(std::max(E * 3 * d, Rmax * d) * ea);
+  void* attn = a.take_bytes(Rall * d * ea);
+  void* ffh = a.take_bytes(Rall * c.d_ff * ea);
+  void* u = a.take_bytes(Rmax * c.k_model * c.d_hidden * ea);
+  void* o = a.take_bytes(R2 * d * ea);
+  std::vector<void*> crosskv(c.n_dec), kc(c.n_dec), vc(c.n_dec);
+  for (int l = 0; l < c.n_dec; ++l) crosskv[l] = a.take_bytes(E * 2 * d * ea);
+  for (int l = 0; l < c.n_dec; ++l) {
+    kc[l] = a.take_bytes((size_t)B * ppr * kPage * d * ea);
+    vc[l] = a.take_bytes((size_t)B * ppr * kPage * d * ea);
+  }
+  int* page_table = a.take<int>((size_t)B * ppr);
+  RowState st;
+  st.len = a.take<int>(B); st.j = a.take<int>(B); st.finished = a.take<int>(B); st.src_len = a.take<int>(B);
+  st.block = a.take<int>((size_t)B * kMaxK); st.cur_block = a.take<int>((size_t)B * kMaxK);
+  st.khat = a.take<int>(B);
+  st.table = a.take<int>((size_t)B * kMaxK * kMaxK);
+  st.out_ids = a.take<int>((size_t)B * max_tgt);
+  st.all_done = a.take<int>(1); st.error = a.take<int>(1);
+  st.stats = a.take<long long>(3 + kMaxK + 1);
+  st.page_table = page_table; st.pages_per_row = ppr; st.max_tgt = max_tgt;
+  int* src_dev = a.take<int>(E);
+  int* tail_dev = a.take<int>((size_t)B * kMaxK);
+  int* plan_dev = a.take<int>((size_t)B * max_tgt * (kMaxK - 1));
+  const size_t tiles = ceil_div(c.V, kVocTile);
+  float* part_val = a.take<float>(tiles * R2);
+  int* part_idx = a.take<int>(tiles * R2);
+  unsigned* counters = a.take<unsigned>(ceil_div((int)R2, kRC) + 1);
+  if (s) {
+    s->x = x; s->h_f32 = h_f32; s->xn = xn; s->qbuf = qbuf; s->attn = attn; s->ffh = ffh; s->u = u; s->o = o;
+    s->crosskv = crosskv; s->kcache = kc; s->vcache = vc; s->st = st; s->src_dev = src_dev;
+    s->tail_dev = tail_dev; s->plan_dev = plan_dev; s->part_val = part_val; s->part_idx = part_idx;
+    s->counters = counters; s->ppr = ppr;
+  }
+  return align_up(a.off);
+}
+
+static size_t weight_bytes_for(const ParsedBlob& pb) { return align_up(pb.total) + align_up(pb.cfg.d / 2 * sizeof(double)); }
+
+// ------------------------------------------------------------------ launches
+static std::atomic<long long> g_launches{0};
+template <typename WT, typename AT, int EPI>
+static void launch_linear(const LinearParams& p, int zcount, cudaStream_t st) {
+  dim3 grid(ceil_div(p.N, kLinWarps * kFPW), ceil_div(p.rows, kRC), zcount);
+  linear_kernel<WT, AT, EPI><<<grid, kLinWarps * 32, 0, st>>>(p);
+  ++g_launches;
+}
+
+static LinearParams lin(const void* x, long long ldx, const void* w, int K, int N, const void* bias, int rows,
+                        void* y, long long ldy, int relu, const int* all_done) {
+  LinearParams p;
+  memset(&p, 0, sizeof(p));
+  p.x = x; p.ldx = ldx; p.w = w; p.ldw = K; p.bias = bias; p.rows = rows; p.K = K; p.N = N;
+  p.relu = relu; p.y = y; p.ldy = ldy; p.all_done = all_done;
+  return p;
+}
+
+template <typename WT, typename AT>
+static void launch_ln(const float* x, const void* g, const void* b, void* y, float* y32, int rows, int d, float eps,
+                      const int* all_done, cudaStream_t st) {
+  LnParams p{x, g, b, y, y32, rows, d, eps, all_done};
+  layernorm_kernel<WT, AT><<<ceil_div(rows, 4), 128, 0, st>>>(p);
+  ++g_launches;
+}
+
+template <typename WT, typename AT>
+static void launch_vocab_argmax(const void* x, const void* w, int rows, int d, int V, float* part_val, int* part_idx,
+                                unsigned* counters, int* out_idx, float* out_val, float* logits, const int* all_done,
+                                cudaStream_t st) {
+  ArgmaxParams p{x, (long long)d, w, rows, d, V, part_val, part_idx, counters, out_idx, out_val, logits, all_done};
+  dim3 grid(ceil_div(V, kVocTile), ceil_div(rows, kRC));
+  vocab_argmax_kernel<WT, AT><<<grid, kLinWarps * 32, (size_t)kRC * d * sizeof(float), st>>>(p);
+  ++g_launches;
+}
+
+// Optional per-phase timing: pairs of events around a phase of the pass, on the session's stream.
+static void prof_mark(bpd_session* s, int slot, int end) {
+  if (!s->profiling) return;
+  cudaEvent_t ev;
+  if (cudaEventCreate(&ev) != cudaSuccess) return;
+  cudaEventRecord(ev, s->stream);
+  (end ? s->prof_end : s->prof_begin)[slot].push_back(ev);
+}
+
+static void prof_clear(bpd_session* s) {
+  for (int i = 0; i < kProfSlots; ++i) {
+    for (cudaEvent_t e : s->prof_begin[i]) cudaEventDestroy(e);
+    for (cudaEvent_t e : s->prof_end[i]) cudaEventDestroy(e);
+    s->prof_begin[i].clear();
+    s->prof_end[i].clear();
+  }
+}
+
+// ------------------------------------------------------------------ encoder
+template <typename WT, typename AT>
+static int run_encoder(bpd_session* s) {
+  const bpd_model* m = s->m;
+  const Config& c = m->cfg;
+  cudaStream_t st = s->stream;
+  const int E = s->B * s->max_src, d = c.d;
+  EmbedParams ep;
+  memset(&ep, 0, sizeof(ep));
+  ep.table = m->src_embed; ep.inv_freq = m->inv_freq; ep.x = s->x; ep.rows = E; ep.rows_per_b = s->max_src;
+  ep.d = d; ep.vocab = c.V; ep.st = s->st; ep.src = s->src_dev;
+  embed_kernel<WT><<<E, 128, 0, st>>>(ep);
+  ++g_launches;
+  for (int l = 0; l < c.n_enc; ++l) {
+    const EncLayer& L = m->enc[l];
+    launch_ln<WT, AT>(s->x, L.ln1g, L.ln1b, s->xn, nullptr, E, d, c.eps, nullptr, st);
+    launch_linear<WT, AT, kEpiStoreAct>(lin(s->xn, d, L.wqkv, d, 3 * d, nullptr, E, s->qbuf, 3 * d, 0, nullptr), 1, st);
+    AttnParams ap;
+    memset(&ap, 0, sizeof(ap));
+    ap.q = s->qbuf; ap.ldq = 3 * d; ap.out = s->attn; ap.ldo = d; ap.rows = E; ap.rows_per_b = s->max_src;
+    ap.H = c.H; ap.dh = d / c.H; ap.causal = 0; ap.limit_b = s->st.src_len;
+    ap.k = static_cast<AT*>(s->qbuf) + d; ap.v = static_cast<AT*>(s->qbuf) + 2 * d;
+    ap.ldkv = 3 * d; ap.bstride = (long long)s->max_src * 3 * d; ap.paged = 0; ap.st = s->st;
+    ap.scale = 1.0f / sqrtf((float)ap.dh);
+    attention_kernel<AT><<<ceil_div(E * c.H, 4), 128, 0, st>>>(ap);
+    ++g_launches;
+    LinearParams po = lin(s->attn, d, L.wo, d, d, nullptr, E, s->x, d, 0, nullptr);
+    launch_linear<WT, AT, kEpiResidual>(po, 1, st);
+    launch_ln<WT, AT>(s->x, L.ln2g, L.ln2b, s->xn, nullptr, E, d, c.eps, nullptr, st);
+    launch_linear<WT, AT, kEpiStoreAct>(lin(s->xn, d, L.w1, d, c.d_ff, L.b1, E, s->ffh, c.d_ff, 1, nullptr), 1, st);
+    launch_linear<WT, AT, kEpiResidual>(lin(s->ffh, c.d_ff, L.w2, c.d_ff, d, L.b2, E, s->x, d, 0, nullptr), 1, st);
+  }
+  launch_ln<WT, AT>(s->x, m->enc_lnf_g, m->enc_lnf_b, s->xn, nullptr, E, d, c.eps, nullptr, st);
+  for (int l = 0; l < c.n_dec; ++l)
+    launch_linear<WT, AT, kEpiStoreAct>(lin(s->xn, d, m->dec[l].cwkv, d, 2 * d, nullptr, E, s->crosskv[l], 2 * d, 0, nullptr), 1, st);
+  BPD_CUDA(cudaGetLastError());
+  return BPD_OK;
+}
+
+// ------------------------------------------------------------------ one decoder pass + heads + top-1 + verify
+struct PassArgs {
+  int mode;          // PassMode
+  int kcur;          // positions scored per row
+  int kh;            // heads evaluated per position
+  int knext;         // width of the block selected for the next pass
+  const int* forced; // device, or null
+  int forced_rows, kforced;
+  int max_new, eos;
+  float* logits_dump;   // device [B*kcur*kh, V] or null
+};
+
+template <typename WT, typename AT>
+static int run_pass(bpd_session* s, const PassArgs& a) {
+  const bpd_model* m = s->m;
+  const Config& c = m->cfg;
+  cudaStream_t st = s->stream;
+  const int d = c.d, R = s->B * a.kcur, R2 = R * a.kh;
+  const int* done = s->st.all_done;
+  EmbedParams ep;
+  memset(&ep, 0, sizeof(ep));
+  ep.table = m->tgt_embed; ep.inv_freq = m->inv_freq; ep.x = s->x; ep.rows = R; ep.rows_per_b = a.kcur;
+  ep.d = d; ep.vocab = c.V; ep.st = s->st; ep.forced = a.forced; ep.forced_rows = a.forced_rows;
+  ep.kforced = a.kforced; ep.src = nullptr; ep.all_done = done;
+  prof_mark(s, kProfLayers, 0);
+  embed_kernel<WT><<<R, 128, 0, st>>>(ep);
+  ++g_launches;
+  for (int l = 0; l < c.n_dec; ++l) {
+    const DecLayer& L = m->dec[l];
+    // self-attention over the cache plus the causal part of the block
+    launch_ln<WT, AT>(s->x, L.ln1g, L.ln1b, s->xn, nullptr, R, d, c.eps, done, st);
+    LinearParams pq = lin(s->xn, d, L.wqkv, d, 3 * d, nullptr, R, s->qbuf, d, 0, done);
+    pq.d = d; pq.kcache = s->kcache[l]; pq.vcache = s->vcache[l]; pq.st = s->st; pq.rows_per_b = a.kcur;
+    launch_linear<WT, AT, kEpiQkv>(pq, 1, st);
+    AttnParams ap;
+    memset(&ap, 0, sizeof(ap));
+    ap.q = s->qbuf; ap.ldq = d; ap.out = s->attn; ap.ldo = d; ap.rows = R; ap.rows_per_b = a.kcur;
+    ap.H = c.H; ap.dh = d / c.H; ap.causal = 1; ap.k = s->kcache[l]; ap.v = s->vcache[l]; ap.ldkv = d;
+    ap.paged = 1; ap.st = s->st; ap.scale = 1.0f / sqrtf((float)ap.dh); ap.all_done = done;
+    attention_kernel<AT><<<ceil_div(R * c.H, 4), 128, 0, st>>>(ap);
+    ++g_launches;
+    launch_linear<WT, AT, kEpiResidual>(lin(s->attn, d, L.wo, d, d, nullptr, R, s->x, d, 0, done), 1, st);
+    // cross-attention over the encoder memory
+    launch_ln<WT, AT>(s->x, L.ln2g, L.ln2b, s->xn, nullptr, R, d, c.eps, done, st);
+    launch_linear<WT, AT, kEpiStoreAct>(lin(s->xn, d, L.cwq, d, d, nullptr, R, s->qbuf, d, 0, done), 1, st);
+    ap.causal = 0; ap.limit_b = s->st.src_len; ap.k = s->crosskv[l]; ap.v = static_cast<AT*>(s->crosskv[l]) + d;
+    ap.ldkv = 2 * d; ap.bstride = (long long)s->max_src * 2 * d; ap.paged = 0;
+    attention_kernel<AT><<<ceil_div(R * c.H, 4), 128, 0, st>>>(ap);
+    ++g_launches;
+    launch_linear<WT, AT, kEpiResidual>(lin(s->attn, d, L.cwo, d, d, nullptr, R, s->x, d, 0, done), 1, st);
+    // feed-forward
+    launch_ln<WT, AT>(s->x, L.ln3g, L.ln3b, s->xn, nullptr, R, d, c.eps, done, st);
+    launch_linear<WT, AT, kEpiStoreAct>(lin(s->xn, d, L.w1, d, c.d_ff, L.b1, R, s->ffh, c.d_ff, 1, done), 1, st);
+    launch_linear<WT, AT, kEpiResidual>(lin(s->ffh, c.d_ff, L.w2, c.d_ff, d, L.b2, R, s->x, d, 0, done), 1, st);
+  }
+  launch_ln<WT, AT>(s->x, m->dec_lnf_g, m->dec_lnf_b, s->xn, s->h_f32, R, d, c.eps, done, st);
+  prof_mark(s, kProfLayers, 1);
+  // proposal heads: hidden layer, k output layers with a residual from the decoder output
+  const int fh = c.d_hidden;
+  const long long ldu = (long long)c.k_model * fh;
+  const int hid = (c.head_layout == 0) ? c.k_model * fh : a.kh * fh;
+  prof_mark(s, kProfHeadW1, 0);
+  launch_linear<WT, AT, kEpiStoreAct>(lin(s->xn, d, m->head_w1, d, hid, m->head_b1, R, s->u, ldu, 1, done), 1, st);
+  prof_mark(s, kProfHeadW1, 1);
+  prof_mark(s, kProfHeadW2, 0);
+  if (c.head_layout == 0) {
+    LinearParams ph = lin(s->u, ldu, m->head_w2, c.k_model * fh, a.kh * d, m->head_b2, R, s->o, (long long)a.kh * d, 0, done);
+    ph.h = s->h_f32; ph.d = d; ph.head_identity = c.p1_identity;
+    launch_linear<WT, AT, kEpiHeadOut>(ph, 1, st);
+  } else {
+    LinearParams ph = lin(s->u, ldu, m->head_w2, fh, d, m->head_b2, R, s->o, (long long)a.kh * d, 0, done);
+    ph.xz = fh; ph.wz = (long long)d * fh; ph.bz = d; ph.yz = d;
+    ph.h = s->h_f32; ph.d = d; ph.head_identity = c.p1_identity;
+    launch_linear<WT, AT, kEpiHeadOut>(ph, a.kh, st);
+  }
+  prof_mark(s, kProfHeadW2, 1);
+  // shared vocabulary projection with a fused top-1: table[b][r][i]
+  prof_mark(s, kProfVocab, 0);
+  launch_vocab_argmax<WT, AT>(s->o, m->out_proj, R2, d, c.V, s->part_val, s->part_idx, s->counters, s->st.table,
+                              nullptr, a.logits_dump, done, st);
+  prof_mark(s, kProfVocab, 1);
+  VerifyParams vp{s->st, s->B, a.kcur, a.kh, a.knext, a.mode, a.max_new, a.eos};
+  verify_commit_kernel<<<1, 32 * ceil_div(s->B, 32), 0, st>>>(vp);
+  ++g_launches;
+  BPD_CUDA(cudaGetLastError());
+  s->invocations += 1;
+  return BPD_OK;
+}
+
+static int dispatch_pass(bpd_session* s, const PassArgs& a) {
+  return s->m->cfg.dtype == 0 ? run_pass<float, float>(s, a) : run_pass<bf16, bf16>(s, a);
+}
+
+static int check_device_error(bpd_session* s) {
+  int err = 0;
+  BPD_CUDA(cudaMemcpyAsync(&s->pinned[64], s->st.error, sizeof(int), cudaMemcpyDeviceToHost, s->stream));
+  BPD_CUDA(cudaStreamSynchronize(s->stream));
+  err = s->pinned[64];
+  if (err == 1) return fail(BPD_E_INVALID, "a token id outside the vocabulary reached the decoder");
+  if (err != 0) return fail(BPD_E_CUDA, "device-side error word %d", err);
+  return BPD_OK;
+}
+
+static int fetch(bpd_session* s, int max_new, int32_t* out_ids, int32_t* out_len, bpd_stats* stats, float ms) {
+  const int B = s->B;
+  std::vector<int> ids, jj(B);
+  std::vector<long long> sv(3 + kMaxK + 1);
+  if (out_ids) {
+    ids.resize((size_t)B * s->max_tgt);
+    BPD_CUDA(cudaMemcpyAsync(ids.data(), s->st.out_ids, ids.size() * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
+  }
+  BPD_CUDA(cudaMemcpyAsync(jj.data(), s->st.j, B * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
+  BPD_CUDA(cudaMemcpyAsync(sv.data(), s->st.stats, sv.size() * sizeof(long long), cudaMemcpyDeviceToHost, s->stream));
+  BPD_CUDA(cudaStreamSynchronize(s->stream));
+  for (int b = 0; b < B; ++b) {
+    const int n = std::min(jj[b], max_new);
+    if (out_len) out_len[b] = n;
+    if (out_ids) {
+      for (int t = 0; t < max_new; ++t) out_ids[(size_t)b * max_new + t] = (t < n) ? ids[(size_t)b * s->max_tgt + t] : -1;
+    }
+  }
+  if (stats) {
+    memset(stats, 0, sizeof(*stats));
+    stats->row_iterations = sv[0]; stats->tokens = sv[1]; stats->iterations = sv[2];
+    for (int i = 0; i <= kMaxK; ++i) stats->khat_hist[i] = sv[3 + i];
+    stats->invocations = s->invocations;
+    stats->device_ms = ms;
+  }
+  return BPD_OK;
+}
+
+}  // namespace bpd
+
+using namespace bpd;
+
+// =================================================================== C ABI
+extern "C" {
+
+const char* bpd_last_error(void) { return g_err; }
+
+int bpd_query_sizes(const void* blob, size_t blob_bytes, int batch, int max_src, int max_tgt, size_t* weight_bytes,
+                    size_t* session_bytes) {
+  ParsedBlob pb;
+  int rc = parse_blob(blob, blob_bytes, &pb);
+  if (rc) return rc;
+  if (batch < 1 || batch > 1024 || max_src < 1 || max_tgt < 1) return fail(BPD_E_INVALID, "batch/max_src/max_tgt out of range");
+  if (weight_bytes) *weight_bytes = weight_bytes_for(pb);
+  if (session_bytes) *session_bytes = plan_session(pb.cfg, batch, max_src, max_tgt, nullptr, nullptr);
+  return BPD_OK;
+}
+
+int bpd_session_bytes(const bpd_model* model, int batch, int max_src, int max_tgt, size_t* session_bytes) {
+  if (!model || !session_bytes) return fail(BPD_E_INVALID, "null argument");
+  if (batch < 1 || batch > 1024 || max_src < 1 || max_tgt < 1) return fail(BPD_E_INVALID, "batch/max_src/max_tgt out of range");
+  *session_bytes = plan_session(model->cfg, batch, max_src, max_tgt, nullptr, nullptr);
+  return BPD_OK;
+}
+
+int bpd_load_weights(const void* blob, size_t blob_bytes, void* dev_weight_buf, size_t dev_bytes, void* cuda_stream,
+                     bpd_model** out) {
+  if (!out) return fail(BPD_E_INVALID, "out is null");
+  *out = nullptr;
+  ParsedBlob pb;
+  int rc = parse_blob(blob, blob_bytes, &pb);
+  if (rc) return rc;
+  if (!dev_weight_buf) return fail(BPD_E_INVALID, "device weight buffer is null");
+  if ((uintptr_t)dev_weight_buf % 256) return fail(BPD_E_INVALID, "device weight buffer is not 256-byte aligned");
+  if (dev_bytes < weight_bytes_for(pb)) return fail(BPD_E_NOMEM, "device weight buffer has %zu bytes, need %zu", dev_bytes, weight_bytes_for(pb));
+  bpd_model* m = new (std::nothrow) bpd_model();
+  if (!m) return fail(BPD_E_NOMEM, "host allocation failed");
+  const Config& c = pb.cfg;
+  m->cfg = c; m->base = static_cast<char*>(dev_weight_buf); m->bytes = dev_bytes; m->stream = (cudaStream_t)cuda_stream;
+  char* B = m->base;
+  const int d = c.d, f = c.d_ff, V = c.V, k = c.k_model, fh = c.d_hidden;
+#define T(name, out, ...) if ((rc = find(pb, B, name, {__VA_ARGS__}, &(out)))) { delete m; return rc; }
+  T("src_embed", m->src_embed, V, d) T("tgt_embed", m->tgt_embed, V, d) T("out_proj", m->out_proj, V, d)
+  m->enc.resize(c.n_enc); m->dec.resize(c.n_dec);
+  for (int l = 0; l < c.n_enc; ++l) {
+    const std::string p = "enc." + std::to_string(l);
+    EncLayer& L = m->enc[l];
+    T(p + ".ln1.g", L.ln1g, d) T(p + ".ln1.b", L.ln1b, d) T(p + ".attn.wqkv", L.wqkv, 3 * d, d) T(p + ".attn.wo", L.wo, d, d)
+    T(p + ".ln2.g", L.ln2g, d) T(p + ".ln2.b", L.ln2b, d)
+    T(p + ".ffn.w1", L.w1, f, d) T(p + ".ffn.b1", L.b1, f) T(p + ".ffn.w2", L.w2, d, f) T(p + ".ffn.b2", L.b2, d)
+  }
+  T("enc.lnf.g", m->enc_lnf_g, d) T("enc.lnf.b", m->enc_lnf_b, d)
+  for (int l = 0; l < c.n_dec; ++l) {
+    const std::string p = "dec." + std::to_string(l);
+    DecLayer& L = m->dec[l];
+    T(p + ".ln1.g", L.ln1g, d) T(p + ".ln1.b", L.ln1b, d) T(p + ".self.wqkv", L.wqkv, 3 * d, d) T(p + ".self.wo", L.wo, d, d)
+    T(p + ".ln2.g", L.ln2g, d) T(p + ".ln2.b", L.ln2b, d)
+    T(p + ".cross.wq", L.cwq, d, d) T(p + ".cross.wkv", L.cwkv, 2 * d, d) T(p + ".cross.wo", L.cwo, d, d)
+    T(p + ".ln3.g", L.ln3g, d) T(p + ".ln3.b", L.ln3b, d)
+    T(p + ".ffn.w1", L.w1, f, d) T(p + ".ffn.b1", L.b1, f) T(p + ".ffn.w2", L.w2, d, f) T(p + ".ffn.b2", L.b2, d)
+  }
+  T("dec.lnf.g", m->dec_lnf_g, d) T("dec.lnf.b", m->dec_lnf_b, d)
+  T("head.w1", m->head_w1, k * fh, d) T("head.b1", m->head_b1, k * fh)
+  if (c.head_layout == 0) { T("head.w2", m->head_w2, k * d, k * fh) } else { T("head.w2", m->head_w2, k, d, fh) }
+  T("head.b2", m->head_b2, k * d)
+#undef T
+  std::vector<double> invf(d / 2);
+  for (int i = 0; i < d / 2; ++i) invf[i] = pow(10000.0, -2.0 * i / d);
+  double* invf_dev = reinterpret_cast<double*>(m->base + align_up(pb.total));
+  m->inv_freq = invf_dev;
+  cudaError_t e = cudaMemcpyAsync(m->base, blob, pb.total, cudaMemcpyHostToDevice, m->stream);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(invf_dev, invf.data(), invf.size() * sizeof(double), cudaMemcpyHostToDevice, m->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(m->stream);
+  if (e != cudaSuccess) { delete m; return fail(BPD_E_CUDA, "weight upload failed: %s", cudaGetErrorString(e)); }
+  *out = m;
+  return BPD_OK;
+}
+
+int bpd_model_destroy(bpd_model* m) {
+  delete m;
+  return BPD_OK;
+}
+
+int bpd_session_create(const bpd_model* model, int batch, int max_src, int max_tgt, void* dev_session_buf,
+                       size_t dev_bytes, void* cuda_stream, bpd_session** out) {
+  if (!out) return fail(BPD_E_INVALID, "out is null");
+  *out = nullptr;
+  if (!model || !dev_session_buf) return fail(BPD_E_INVALID, "model or session buffer is null");
+  if (batch < 1 || batch > 1024 || max_src < 1 || max_tgt < 1) return fail(BPD_E_INVALID, "batch/max_src/max_tgt out of range");
+  if ((uintptr_t)dev_session_buf % 256) return fail(BPD_E_INVALID, "session buffer is not 256-byte aligned");
+  const size_t need = plan_session(model->cfg, batch, max_src, max_tgt, nullptr, nullptr);
+  if (dev_bytes < need) return fail(BPD_E_NOMEM, "session buffer has %zu bytes, need %zu", dev_bytes, need);
+  bpd_session* s = new (std::nothrow) bpd_session();
+  if (!s) return fail(BPD_E_NOMEM, "host allocation failed");
+  s->m = model; s->B = batch; s->max_src = max_src; s->max_tgt = max_tgt;
+  s->base = static_cast<char*>(dev_session_buf); s->bytes = dev_bytes; s->stream = (cudaStream_t)cuda_stream;
+  s->profiling = 0;
+  s->phase = kPhaseCreated; s->plan_len = 0; s->plan_k = 0; s->invocations = 0; s->pinned = nullptr;
+  plan_session(model->cfg, batch, max_src, max_tgt, s->base, s);
+  // page table: row b's p-th page is physical page p*B + b (rows interleaved in the pool)
+  std::vector<int> pt((size_t)batch * s->ppr);
+  for (int b = 0; b < batch; ++b)
+    for (int p = 0; p < s->ppr; ++p) pt[(size_t)b * s->ppr + p] = p * batch + b;
+  cudaError_t e = cudaMallocHost(reinterpret_cast<void**>(&s->pinned), (256 + (size_t)batch * kMaxK) * sizeof(int));
+  for (int i = 0; i < 8 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&s->ev_flag[i], cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreate(&s->ev0);
+  if (e == cudaSuccess) e = cudaEventCreate(&s->ev1);
+  if (e == cudaSuccess) e = cudaMemsetAsync(s->base, 0, need, s->stream);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(const_cast<int*>(s->st.page_table), pt.data(), pt.size() * sizeof(int), cudaMemcpyHostToDevice, s->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s->stream);
+  if (e != cudaSuccess) {
+    delete s;
+    return fail(BPD_E_CUDA, "session set-up failed: %s", cudaGetErrorString(e));
+  }
+  *out = s;
+  return BPD_OK;
+}
+
+int bpd_session_destroy(bpd_session* s) {
+  if (!s) return BPD_OK;
+  cudaStreamSynchronize(s->stream);
+  prof_clear(s);
+  if (s->pinned) cudaFreeHost(s->pinned);
+  for (int i = 0; i < 8; ++i) cudaEventDestroy(s->ev_flag[i]);
+  cudaEventDestroy(s->ev0);
+  cudaEventDestroy(s->ev1);
+  delete s;
+  return BPD_OK;
+}
+
+int bpd_encode(bpd_session* s, const int32_t* src_ids, const int32_t* src_len) {
+  if (!s || !src_ids || !src_len) return fail(BPD_E_INVALID, "null argument");
+  const Config& c = s->m->cfg;
+  const int B = s->B, S = s->max_src;
+  std::vector<int> ids((size_t)B * S, 0), lens(B);
+  for (int b = 0; b < B; ++b) {
+    if (src_len[b] < 1 || src_len[b] > S) return fail(BPD_E_SHAPE, "src_len[%d] = %d outside 1..%d", b, src_len[b], S);
+    lens[b] = src_len[b];
+    for (int t = 0; t < src_len[b]; ++t) {
+      const int id = src_ids[(size_t)b * S + t];
+      if (id < 0 || id >= c.V) return fail(BPD_E_INVALID, "source id %d at row %d position %d outside the vocabulary", id, b, t);
+      ids[(size_t)b * S + t] = id;
+    }
+  }
+  // staging through pinned memory keeps the copies asynchronous and ordered on the stream
+  BPD_CUDA(cudaStreamSynchronize(s->stream));
+  BPD_CUDA(cudaMemcpyAsync(s->src_dev, ids.data(), ids.size() * sizeof(int), cudaMemcpyHostToDevice, s->stream));
+  BPD_CUDA(cudaMemcpyAsync(s->tail_dev, lens.data(), B * sizeof(int), cudaMemcpyHostToDevice, s->stream));
+  ResetParams rp{s->st, B, s->ppr, s->tail_dev};
+  reset_rows_kernel<<<1, 32 * ceil_div(B, 32), 0, s->stream>>>(rp);
+  ++g_launches;
+  BPD_CUDA(cudaStreamSynchronize(s->stream));   // host vectors go out of scope
+  int rc = (c.dtype == 0) ? run_encoder<float, float>(s) : run_encoder<bf16, bf16>(s);
+  if (rc) return rc;
+  s->phase = kPhaseEncoded; s->plan_len = 0; s->plan_k = 0; s->invocations = 0;
+  return BPD_OK;
+}
+
+int bpd_rewind(bpd_session* s) {
+  if (!s) return fail(BPD_E_INVALID, "session is null");
+  if (s->phase < kPhaseEncoded) return fail(BPD_E_STATE, "nothing encoded yet");
+  ResetParams rp{s->st, s->B, s->ppr, s->st.src_len};
+  reset_rows_kernel<<<1, 32 * ceil_div(s->B, 32), 0, s->stream>>>(rp);
+  ++g_launches;
+  BPD_CUDA(cudaGetLastError());
+  s->phase = kPhaseEncoded; s->invocations = 0;
+  return BPD_OK;
+}
+
+long long bpd_kernel_launches(void) { return g_launches.load(); }
+
+int bpd_profile(bpd_session* s, int enable) {
+  if (!s) return fail(BPD_E_INVALID, "session is null");
+  BPD_CUDA(cudaStreamSynchronize(s->stream));
+  prof_clear(s);
+  s->profiling = enable ? 1 : 0;
+  return BPD_OK;
+}
+
+int bpd_profile_read(bpd_session* s, int phase, int64_t* launches, double* total_ms) {
+  if (!s || !launches || !total_ms) return fail(BPD_E_INVALID, "null argument");
+  if (phase < 0 || phase >= kProfSlots) return fail(BPD_E_INVALID, "phase %d outside 0..%d", phase, kProfSlots - 1);
+  BPD_CUDA(cudaStreamSynchronize(s->stream));
+  const size_t n = std::min(s->prof_begin[phase].size(), s->prof_end[phase].size());
+  double sum = 0;
+  for (size_t i = 0; i < n; ++i) {
+    float ms = 0.f;
+    BPD_CUDA(cudaEventElapsedTime(&ms, s->prof_begin[phase][i], s->prof_end[phase][i]));
+    sum += ms;
+  }
+  *launches = (int64_t)n;
+  *total_ms = sum;
+  return BPD_OK;
+}
+
+int bpd_set_forced_plan(bpd_session* s, const int32_t* plan, int plan_len, int k) {
+  if (!s) return fail(BPD_E_INVALID, "session is null");
+  if (!plan) { s->plan_len = 0; s->plan_k = 0; return BPD_OK; }
+  if (k < 2 || k > s->m->cfg.k_model) return fail(BPD_E_INVALID, "k = %d outside 2..%d", k, s->m->cfg.k_model);
+  if (plan_len < 1 || plan_len > s->max_tgt) return fail(BPD_E_SHAPE, "plan_len = %d outside 1..%d", plan_len, s->max_tgt);
+  const size_t n = (size_t)s->B * plan_len * (k - 1);
+  for (size_t i = 0; i < n; ++i)
+    if (plan[i] < 0 || plan[i] >= s->m->cfg.V) return fail(BPD_E_INVALID, "plan entry %zu = %d outside the vocabulary", i, plan[i]);
+  BPD_CUDA(cudaMemcpyAsync(s->plan_dev, plan, n * sizeof(int), cudaMemcpyHostToDevice, s->stream));
+  BPD_CUDA(cudaStreamSynchronize(s->stream));
+  s->plan_len = plan_len; s->plan_k = k;
+  return BPD_OK;
+}
+
+static int check_decode_args(bpd_session* s, int max_new, int eos) {
+  if (!s) return fail(BPD_E_INVALID, "session is null");
+  if (max_new < 1 || max_new > s->max_tgt) return fail(BPD_E_SHAPE, "max_new = %d outside 1..%d", max_new, s->max_tgt);
+  if (eos < -1 || eos >= s->m->cfg.V) return fail(BPD_E_INVALID, "eos_id = %d outside the vocabulary", eos);
+  return BPD_OK;
+}
+
+// Launch passes until the device reports every row finished.  The flag of pass
+// t is read back asynchronously and looked at two passes later, so the host
+// never stalls the stream; passes issued after the end return at once.
+static int decode_loop(bpd_session* s, const PassArgs& a, int max_passes) {
+  for (int it = 0; it < max_passes; ++it) {
+    if (it >= 2) {
+      BPD_CUDA(cudaEventSynchronize(s->ev_flag[(it - 2) % 8]));
+      if (s->pinned[(it - 2) % 8]) break;
+    }
+    int rc = dispatch_pass(s, a);
+    if (rc) return rc;
+    BPD_CUDA(cudaMemcpyAsync(&s->pinned[it % 8], s->st.all_done, sizeof(int), cudaMemcpyDeviceToHost, s->stream));
+    BPD_CUDA(cudaEventRecord(s->ev_flag[it % 8], s->stream));
+  }
+  return BPD_OK;
+}
+
+static int finish_decode(bpd_session* s, int max_new, int32_t* out_ids, int32_t* out_len, bpd_stats* stats) {
+  BPD_CUDA(cudaEventRecord(s->ev1, s->stream));
+  if (!out_ids && !out_len && !stats) return BPD_OK;
+  BPD_CUDA(cudaEventSynchronize(s->ev1));
+  float ms = 0.f;
+  BPD_CUDA(cudaEventElapsedTime(&ms, s->ev0, s->ev1));
+  int rc = check_device_error(s);
+  if (rc) return rc;
+  return fetch(s, max_new, out_ids, out_len, stats, ms);
+}
+
+int bpd_decode_greedy(bpd_session* s, int max_new, int32_t eos_id, int32_t* out_ids, int32_t* out_len, bpd_stats* stats) {
+  int rc = check_decode_args(s, max_new, eos_id);
+  if (rc) return rc;
+  if (s->phase != kPhaseEncoded) return fail(BPD_E_STATE, "bpd_decode_greedy needs a freshly encoded session");
+  s->phase = kPhaseGreedy;
+  BPD_CUDA(cudaEventRecord(s->ev0, s->stream));
+  PassArgs a{kModeGreedy, 1, 1, 1, nullptr, 0, 0, max_new, eos_id, nullptr};
+  rc = decode_loop(s, a, max_new);
+  if (rc) return rc;
+  return finish_decode(s, max_new, out_ids, out_len, stats);
+}
+
+int bpd_decode_blockwise(bpd_session* s, int k, int accept_mode, int max_new, int32_t eos_id, int32_t* out_ids,
+                         int32_t* out_len, bpd_stats* stats) {
+  int rc = check_decode_args(s, max_new, eos_id);
+  if (rc) return rc;
+  if (k < 1 || k > s->m->cfg.k_model) return fail(BPD_E_INVALID, "k = %d outside 1..%d", k, s->m->cfg.k_model);
+  if (accept_mode != BPD_ACCEPT_EXACT) return fail(BPD_E_UNSUPPORTED, "acceptance mode %d", accept_mode);
+  if (s->phase != kPhaseEncoded) return fail(BPD_E_STATE, "bpd_decode_blockwise needs a freshly encoded session");
+  if (s->plan_len && s->plan_k != k) return fail(BPD_E_SHAPE, "forced plan was installed for k = %d", s->plan_k);
+  s->phase = kPhaseBlockwise;
+  BPD_CUDA(cudaEventRecord(s->ev0, s->stream));
+  PassArgs prime{kModePrime, 1, k, k, nullptr, 0, 0, max_new, eos_id, nullptr};
+  rc = dispatch_pass(s, prime);
+  if (rc) return rc;
+  PassArgs a{kModeBlock, k, k, k, s->plan_len ? s->plan_dev : nullptr, s->plan_len, k, max_new, eos_id, nullptr};
+  rc = decode_loop(s, a, max_new);
+  if (rc) return rc;
+  return finish_decode(s, max_new, out_ids, out_len, stats);
+}
+
+int bpd_iteration(bpd_session* s, int k, int accept_mode, int max_new, int32_t eos_id, const int32_t* forced_tail,
+                  bpd_iter_out* out) {
+  int rc = check_decode_args(s, max_new, eos_id);
+  if (rc) return rc;
+  if (k < 1 || k > s->m->cfg.k_model) return fail(BPD_E_INVALID, "k = %d outside 1..%d", k, s->m->cfg.k_model);
+  if (accept_mode != BPD_ACCEPT_EXACT) return fail(BPD_E_UNSUPPORTED, "acceptance mode %d", accept_mode);
+  if (s->phase != kPhaseEncoded && s->phase != kPhaseBlockwise) return fail(BPD_E_STATE, "bpd_iteration needs an encoded session that is not decoding greedily");
+  const int B = s->B, V = s->m->cfg.V;
+  if (forced_tail && k > 1) {
+    for (int i = 0; i < B * (k - 1); ++i)
+      if (forced_tail[i] < 0 || forced_tail[i] >= V) return fail(BPD_E_INVALID, "forced_tail[%d] = %d outside the vocabulary", i, forced_tail[i]);
+  }
+  if (s->phase == kPhaseEncoded) {
+    PassArgs prime{kModePrime, 1, k, k, nullptr, 0, 0, max_new, eos_id, nullptr};
+    rc = dispatch_pass(s, prime);
+    if (rc) return rc;
+    s->phase = kPhaseBlockwise;
+  }
+  PassArgs a{kModeBlock, k, k, k, nullptr, 0, 0, max_new, eos_id, out ? out->logits_dev : nullptr};
+  if (forced_tail && k > 1) {
+    BPD_CUDA(cudaStreamSynchronize(s->stream));   // the staging slots may still be in flight
+    memcpy(&s->pinned[128], forced_tail, sizeof(int) * B * (k - 1));
+    BPD_CUDA(cudaMemcpyAsync(s->tail_dev, &s->pinned[128], sizeof(int) * B * (k - 1), cudaMemcpyHostToDevice, s->stream));
+    a.forced = s->tail_dev; a.forced_rows = 1; a.kforced = k;
+  } else if (s->plan_len) {
+    if (s->plan_k != k) return fail(BPD_E_SHAPE, "forced plan was installed for k = %d", s->plan_k);
+    a.forced = s->plan_dev; a.forced_rows = s->plan_len; a.kforced = k;
+  }
+  rc = dispatch_pass(s, a);
+  if (rc) return rc;
+  if (!out) return BPD_OK;
+  if (out->hidden_dev)
+    BPD_CUDA(cudaMemcpyAsync(out->hidden_dev, s->h_f32, sizeof(float) * B * k * s->m->cfg.d, cudaMemcpyDeviceToDevice, s->stream));
+  std::vector<int> khat(B), table((size_t)B * k * k), blk((size_t)B * kMaxK), cur((size_t)B * kMaxK);
+  BPD_CUDA(cudaMemcpyAsync(khat.data(), s->st.khat, B * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
+  BPD_CUDA(cudaMemcpyAsync(table.data(), s->st.table, table.size() * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
+  BPD_CUDA(cudaMemcpyAsync(blk.data(), s->st.block, blk.size() * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
+  BPD_CUDA(cudaMemcpyAsync(cur.data(), s->st.cur_block, cur.size() * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
+  BPD_CUDA(cudaStreamSynchronize(s->stream));
+  rc = check_device_error(s);
+  if (rc) return rc;
+  for (int b = 0; b < B; ++b) {
+    if (out->khat) out->khat[b] = khat[b];
+    for (int i = 0; i < k; ++i) {
+      if (out->accepted) out->accepted[b * k + i] = (i < khat[b]) ? cur[b * kMaxK + i] : -1;
+      if (out->next_block) out->next_block[b * k + i] = blk[b * kMaxK + i];
+      if (out->block) out->block[b * k + i] = cur[b * kMaxK + i];
+    }
+  }
+  if (out->table) memcpy(out->table, table.data(), table.size() * sizeof(int));
+  return BPD_OK;
+}
+
+int bpd_fetch_output(bpd_session* s, int max_new, int32_t* out_ids, int32_t* out_len, bpd_stats* stats) {
+  if (!s) return fail(BPD_E_INVALID, "session is null");
+  if (max_new < 1 || max_new > s->max_tgt) return fail(BPD_E_SHAPE, "max_new = %d outside 1..%d", max_new, s->max_tgt);
+  if (s->phase < kPhaseEncoded) return fail(BPD_E_STATE, "nothing encoded yet");
+  float ms = 0.f;
+  if (s->phase != kPhaseEncoded) {
+    BPD_CUDA(cudaEventSynchronize(s->ev1));
+    BPD_CUDA(cudaEventElapsedTime(&ms, s->ev0, s->ev1));
+  }
+  int rc = check_device_error(s);
+  if (rc) return rc;
+  return fetch(s, max_new, out_ids, out_len, stats, ms);
+}
+
+// ------------------------------------------------------------------ single operators
+size_t bpd_op_vocab_argmax_scratch_bytes(int rows, int d, int vocab, int dtype) {
+  (void)d; (void)dtype;
+  if (rows < 1 || vocab < 1) return 0;
+  const size_t tiles = ceil_div(vocab, kVocTile);
+  return align_up(tiles * rows * sizeof(float)) + align_up(tiles * rows * sizeof(int)) +
+         align_up((ceil_div(rows, kRC) + 1) * sizeof(unsigned));
+}
+
+int bpd_op_vocab_argmax(const void* x, const void* w, int rows, int d, int vocab, int dtype, void* scratch,
+                        size_t scratch_bytes, int32_t* out_idx, float* out_val, void* cuda_stream) {
+  if (!x || !w || !scratch || !out_idx) return fail(BPD_E_INVALID, "null argument");
+  if (rows < 1 || vocab < 1 || d < 8 || d % 8 || d > kArgmaxMaxD) return fail(BPD_E_SHAPE, "rows/d/vocab out of range (d must be a multiple of 8, at most %d)", kArgmaxMaxD);
+  if (dtype != 0 && dtype != 1) return fail(BPD_E_INVALID, "unknown dtype %d", dtype);
+  if ((uintptr_t)x % 16 || (uintptr_t)w % 16 || (uintptr_t)scratch % 256) return fail(BPD_E_INVALID, "misaligned pointer");
+  if (scratch_bytes < bpd_op_vocab_argmax_scratch_bytes(rows, d, vocab, dtype)) return fail(BPD_E_NOMEM, "scratch too small");
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const size_t tiles = ceil_div(vocab, kVocTile);
+  char* p = static_cast<char*>(scratch);
+  float* pv = reinterpret_cast<float*>(p);
+  p += align_up(tiles * rows * sizeof(float));
+  int* pi = reinterpret_cast<int*>(p);
+  p += align_up(tiles * rows * sizeof(int));
+  unsigned* cnt = reinterpret_cast<unsigned*>(p);
+  BPD_CUDA(cudaMemsetAsync(cnt, 0, (ceil_div(rows, kRC) + 1) * sizeof(unsigned), st));
+  if (dtype == 0) launch_vocab_argmax<float, float>(x, w, rows, d, vocab, pv, pi, cnt, out_idx, out_val, nullptr, nullptr, st);
+  else launch_vocab_argmax<bf16, bf16>(x, w, rows, d, vocab, pv, pi, cnt, out_idx, out_val, nullptr, nullptr, st);
+  BPD_CUDA(cudaGetLastError());
+  return BPD_OK;
+}
+
+size_t bpd_op_linear_scratch_bytes(int rows, int in_f, int out_f, int dtype) {
+  (void)rows; (void)in_f; (void)out_f; (void)dtype;
+  return 256;
+}
+
+int bpd_op_linear(const void* x, const void* w, const void* bias, int rows, int in_f, int out_f, int dtype, int relu,
+                  void* scratch, size_t scratch_bytes, float* y, void* cuda_stream) {
+  (void)scratch; (void)scratch_bytes;
+  if (!x || !w || !y) return fail(BPD_E_INVALID, "null argument");
+  if (rows < 1 || out_f < 1 || in_f < 8 || in_f % 8) return fail(BPD_E_SHAPE, "rows/in_f/out_f out of range (in_f must be a multiple of 8)");
+  if (dtype != 0 && dtype != 1) return fail(BPD_E_INVALID, "unknown dtype %d", dtype);
+  if ((uintptr_t)x % 16 || (uintptr_t)w % 16) return fail(BPD_E_INVALID, "misaligned pointer");
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  LinearParams p = lin(x, in_f, w, in_f, out_f, bias, rows, y, out_f, relu, nullptr);
+  if (dtype == 0) launch_linear<float, float, kEpiStoreF32>(p, 1, st);
+  else launch_linear<bf16, bf16, kEpiStoreF32>(p, 1, st);
+  BPD_CUDA(cudaGetLastError());
+  return BPD_OK;
+}
+
+}  // extern "C"

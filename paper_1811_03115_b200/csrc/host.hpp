@@ -1,0 +1,99 @@
+// Host-side structures behind the opaque handles of bpd.h.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdarg.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include <map>
+#include <string>
+#include <vector>
+
+#include "../../include/bpd.h"
+#include "common.cuh"
+
+namespace bpd {
+
+extern thread_local char g_err[512];
+int fail(int code, const char* fmt, ...);
+
+#define BPD_CUDA(expr)                                                                   \
+  do {                                                                                   \
+    cudaError_t e__ = (expr);                                                            \
+    if (e__ != cudaSuccess)                                                              \
+      return bpd::fail(BPD_E_CUDA, "%s failed: %s (%s:%d)", #expr, cudaGetErrorString(e__), \
+                       __FILE__, __LINE__);                                              \
+  } while (0)
+
+struct Config {
+  int dtype, n_enc, n_dec, d, H, d_ff, V, k_model, d_hidden, head_layout, p1_identity;
+  float eps;
+  int elem() const { return dtype == 0 ? 4 : 2; }
+};
+
+struct TensorEntry {
+  int ndim;
+  int dims[3];
+  uint64_t offset, nbytes;
+};
+
+struct ParsedBlob {
+  Config cfg;
+  std::map<std::string, TensorEntry> t;
+  uint64_t total;
+};
+int parse_blob(const void* blob, size_t n, ParsedBlob* out);
+
+struct EncLayer {
+  const void *ln1g, *ln1b, *wqkv, *wo, *ln2g, *ln2b, *w1, *b1, *w2, *b2;
+};
+struct DecLayer {
+  const void *ln1g, *ln1b, *wqkv, *wo, *ln2g, *ln2b, *cwq, *cwkv, *cwo, *ln3g, *ln3b, *w1, *b1, *w2, *b2;
+};
+
+}  // namespace bpd
+
+struct bpd_model {
+  bpd::Config cfg;
+  char* base;            // device weight buffer
+  size_t bytes;
+  cudaStream_t stream;
+  const void *src_embed, *tgt_embed, *out_proj;
+  std::vector<bpd::EncLayer> enc;
+  std::vector<bpd::DecLayer> dec;
+  const void *enc_lnf_g, *enc_lnf_b, *dec_lnf_g, *dec_lnf_b;
+  const void *head_w1, *head_b1, *head_w2, *head_b2;
+  const double* inv_freq;   // device [d/2]
+};
+
+enum ProfSlot { kProfLayers = 0, kProfHeadW1 = 1, kProfHeadW2 = 2, kProfVocab = 3, kProfSlots = 4 };
+
+enum SessionPhase { kPhaseCreated = 0, kPhaseEncoded = 1, kPhaseBlockwise = 2, kPhaseGreedy = 3 };
+
+struct bpd_session {
+  const bpd_model* m;
+  int B, max_src, max_tgt, ppr;
+  char* base;
+  size_t bytes;
+  cudaStream_t stream;
+  int phase;
+  // activations
+  float *x, *h_f32;
+  void *xn, *qbuf, *attn, *ffh, *u, *o;
+  std::vector<void*> crosskv, kcache, vcache;
+  // integers
+  bpd::RowState st;
+  int *src_dev, *tail_dev, *plan_dev;
+  int plan_len, plan_k;    // 0 when no plan installed
+  // vocabulary top-1 workspace
+  float* part_val;
+  int* part_idx;
+  unsigned* counters;
+  // host side
+  int* pinned;             // pinned ring of all_done flags + staging
+  cudaEvent_t ev_flag[8];
+  cudaEvent_t ev0, ev1;
+  int64_t invocations;
+  int profiling;
+  std::vector<cudaEvent_t> prof_begin[kProfSlots], prof_end[kProfSlots];
+};

@@ -1,0 +1,516 @@
+// CUDA-core kernels of the decoding pass: embedding, layer norm, skinny
+// projections with fused epilogues, attention over the paged cache, the
+// vocabulary projection with a fused top-1, and verify/accept/commit.
+// Every reduction has a fixed order that does not depend on how many rows a
+// launch carries, so a position scored alone (greedy) and the same position
+// scored inside a block give bit-identical results.
+#pragma once
+#include "common.cuh"
+
+namespace bpd {
+
+// ------------------------------------------------------------------ embedding (decoder and encoder)
+struct EmbedParams {
+  const void* table;       // [V, d] weight dtype
+  const double* inv_freq;  // [d/2] 10000^(-2i/d)
+  float* x;                // [rows, d] residual stream
+  int rows, rows_per_b, d, vocab;
+  // decoder: token = block[b][i] (or a forced proposal), position = len[b] + i
+  RowState st;
+  const int* forced;       // [B][forced_rows][kforced-1] or null
+  int forced_rows;         // 1: one tail per row; >1: indexed by tokens emitted so far
+  int kforced;
+  // encoder: token = src[b][s], position = s
+  const int* src;          // [B][rows_per_b] or null (decoder mode)
+  const int* all_done;
+};
+
+template <typename WT>
+__global__ void embed_kernel(EmbedParams p) {
+  if (p.all_done && *p.all_done) return;
+  const int r = blockIdx.x;
+  const int b = r / p.rows_per_b, i = r % p.rows_per_b;
+  int tok, pos;
+  if (p.src) {
+    tok = p.src[r];
+    pos = i;
+  } else {
+    tok = p.st.block[b * kMaxK + i];
+    if (p.forced && i >= 1 && i < p.kforced) {
+      const int jb = p.st.j[b];
+      if (p.forced_rows == 1)
+        tok = p.forced[(size_t)b * (p.kforced - 1) + (i - 1)];
+      else if (jb < p.forced_rows)
+        tok = p.forced[((size_t)b * p.forced_rows + jb) * (p.kforced - 1) + (i - 1)];
+    }
+    pos = p.st.len[b] + i;
+    if (threadIdx.x == 0) p.st.cur_block[b * kMaxK + i] = tok;
+  }
+  if (tok < 0 || tok >= p.vocab) {   // never index outside the table; report instead
+    if (threadIdx.x == 0) atomicCAS(p.st.error, 0, 1);
+    tok = 0;
+  }
+  const WT* row = reinterpret_cast<const WT*>(p.table) + (size_t)tok * p.d;
+  const float scale = sqrtf((float)p.d);
+  for (int c = threadIdx.x; c < p.d; c += blockDim.x) {
+    const double ang = (double)pos * p.inv_freq[c >> 1];
+    const float pe = (float)((c & 1) ? cos(ang) : sin(ang));
+    p.x[(size_t)r * p.d + c] = to_f(row[c]) * scale + pe;
+  }
+}
+
+// ------------------------------------------------------------------ layer norm (one warp per row)
+struct LnParams {
+  const float* x;   // [rows, d]
+  const void* g;    // [d] weight dtype
+  const void* b;
+  void* y;          // [rows, d] activation dtype
+  float* y_f32;     // optional fp32 copy
+  int rows, d;
+  float eps;
+  const int* all_done;
+};
+
+template <typename WT, typename AT>
+__global__ void __launch_bounds__(128) layernorm_kernel(LnParams p) {
+  if (p.all_done && *p.all_done) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r = blockIdx.x * 4 + warp;
+  if (r >= p.rows) return;
+  const float* x = p.x + (size_t)r * p.d;
+  float s = 0.f;
+  for (int c = lane; c < p.d; c += 32) s += x[c];
+  const float mean = warp_sum(s) / (float)p.d;
+  float v = 0.f;
+  for (int c = lane; c < p.d; c += 32) { const float t = x[c] - mean; v += t * t; }
+  const float rstd = rsqrtf(warp_sum(v) / (float)p.d + p.eps);
+  const WT* g = reinterpret_cast<const WT*>(p.g);
+  const WT* bb = reinterpret_cast<const WT*>(p.b);
+  AT* y = reinterpret_cast<AT*>(p.y) + (size_t)r * p.d;
+  for (int c = lane; c < p.d; c += 32) {
+    const float o = (x[c] - mean) * rstd * to_f(g[c]) + to_f(bb[c]);
+    y[c] = from_f<AT>(o);
+    if (p.y_f32) p.y_f32[(size_t)r * p.d + c] = o;
+  }
+}
+
+// ------------------------------------------------------------------ skinny projection y = x W^T (+ epilogue)
+enum Epilogue {
+  kEpiStoreAct = 0,  // y_act[r][n] = act(v + bias)
+  kEpiStoreF32 = 1,  // y_f32[r][n] = act(v + bias)
+  kEpiResidual = 2,  // x_f32[r][n] += v + bias
+  kEpiQkv = 3,       // n < d: q[r][n]; else key / value into the paged cache at position len[b] + i
+  kEpiHeadOut = 4    // o[r][n] = v + bias + h[r][n mod d]   (residual to each of the k outputs)
+};
+
+struct LinearParams {
+  const void* x; long long ldx;   // activations [rows, K]
+  const void* w; long long ldw;   // weights [N, K]
+  const void* bias;               // [N] or null
+  int rows, K, N;
+  long long xz, wz, bz, yz;       // element offsets per blockIdx.z
+  int relu;
+  void* y; long long ldy;
+  const float* h; int d;          // kEpiHeadOut: residual source; kEpiQkv: model width
+  int head_identity;              // kEpiHeadOut: first d outputs are h itself
+  void* kcache; void* vcache;     // kEpiQkv
+  RowState st; int rows_per_b;
+  const int* all_done;
+};
+
+constexpr int kRC = 8;      // rows per CTA pass
+constexpr int kFPW = 4;     // output features per warp
+constexpr int kKT = 512;    // K tile staged in shared memory
+constexpr int kLinWarps = 8;
+
+template <typename WT, typename AT, int EPI>
+__device__ __forceinline__ void linear_epilogue(const LinearParams& p, int z, int r, int n, float v) {
+  if (p.bias) v += to_f(reinterpret_cast<const WT*>(p.bias)[z * p.bz + n]);
+  if (p.relu) v = fmaxf(v, 0.f);
+  if (EPI == kEpiStoreAct) {
+    reinterpret_cast<AT*>(p.y)[z * p.yz + (long long)r * p.ldy + n] = from_f<AT>(v);
+  } else if (EPI == kEpiStoreF32) {
+    reinterpret_cast<float*>(p.y)[z * p.yz + (long long)r * p.ldy + n] = v;
+  } else if (EPI == kEpiResidual) {
+    reinterpret_cast<float*>(p.y)[(long long)r * p.ldy + n] += v;
+  } else if (EPI == kEpiHeadOut) {
+    const int c = n % p.d;
+    const float hv = p.h[(size_t)r * p.d + c];
+    const int nz = z * (int)(p.yz) + n;   // output column within the row of k*d
+    v = (p.head_identity && nz < p.d) ? hv : v + hv;
+    reinterpret_cast<AT*>(p.y)[z * p.yz + (long long)r * p.ldy + n] = from_f<AT>(v);
+  } else if (EPI == kEpiQkv) {
+    const int d = p.d;
+    if (n < d) {
+      reinterpret_cast<AT*>(p.y)[(long long)r * p.ldy + n] = from_f<AT>(v);
+    } else {
+      const int b = r / p.rows_per_b, i = r % p.rows_per_b;
+      const int pos = p.st.len[b] + i;
+      const int page = p.st.page_table[b * p.st.pages_per_row + pos / kPage];
+      const size_t slot = ((size_t)page * kPage + (pos % kPage)) * d;
+      if (n < 2 * d) reinterpret_cast<AT*>(p.kcache)[slot + (n - d)] = from_f<AT>(v);
+      else reinterpret_cast<AT*>(p.vcache)[slot + (n - 2 * d)] = from_f<AT>(v);
+    }
+  }
+}
+
+// One warp owns kFPW output features and kRC rows; its lanes split K, each
+// accumulating in increasing-k order, then a butterfly sum.  The order depends
+// only on K, never on the number of rows.
+template <typename WT, typename AT, int EPI>
+__global__ void __launch_bounds__(kLinWarps * 32) linear_kernel(LinearParams p) {
+  if (p.all_done && *p.all_done) return;
+  __shared__ __align__(16) float xs[kRC][kKT];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int z = blockIdx.z;
+  const AT* X = reinterpret_cast<const AT*>(p.x) + z * p.xz;
+  const WT* W = reinterpret_cast<const WT*>(p.w) + z * p.wz;
+  const int r0 = blockIdx.y * kRC;
+  const int nr = min(kRC, p.rows - r0);
+  const int n0 = blockIdx.x * (kLinWarps * kFPW) + warp * kFPW;
+  float acc[kFPW][kRC];
+#pragma unroll
+  for (int f = 0; f < kFPW; ++f)
+#pragma unroll
+    for (int r = 0; r < kRC; ++r) acc[f][r] = 0.f;
+
+  for (int kt = 0; kt < p.K; kt += kKT) {
+    __syncthreads();
+    for (int v = threadIdx.x; v < kRC * kKT / 8; v += kLinWarps * 32) {
+      const int r = v / (kKT / 8), kk = (v % (kKT / 8)) * 8;
+      float t[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      if (r < nr && kt + kk < p.K) load8(X + (long long)(r0 + r) * p.ldx + kt + kk, t);
+      *reinterpret_cast<float4*>(&xs[r][kk]) = make_float4(t[0], t[1], t[2], t[3]);
+      *reinterpret_cast<float4*>(&xs[r][kk + 4]) = make_float4(t[4], t[5], t[6], t[7]);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int c = 0; c < kKT / 256; ++c) {
+      const int kk = c * 256 + lane * 8;
+      if (kt + kk < p.K) {
+        float wv[kFPW][8];
+#pragma unroll
+        for (int f = 0; f < kFPW; ++f) {
+          if (n0 + f < p.N) {
+            load8_stream(W + (long long)(n0 + f) * p.ldw + kt + kk, wv[f]);
+          } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) wv[f][e] = 0.f;
+          }
+        }
+#pragma unroll
+        for (int r = 0; r < kRC; ++r) {
+          const float4 a = *reinterpret_cast<const float4*>(&xs[r][kk]);
+          const float4 b = *reinterpret_cast<const float4*>(&xs[r][kk + 4]);
+          const float xv[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+          for (int f = 0; f < kFPW; ++f)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[f][r] = fmaf(wv[f][e], xv[e], acc[f][r]);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int f = 0; f < kFPW; ++f)
+#pragma unroll
+    for (int r = 0; r < kRC; ++r) {
+      const float v = warp_sum(acc[f][r]);
+      if (lane == f * kRC + r && r < nr && n0 + f < p.N) linear_epilogue<WT, AT, EPI>(p, z, r0 + r, n0 + f, v);
+    }
+}
+
+// ------------------------------------------------------------------ attention (one warp per (row, head))
+struct AttnParams {
+  const void* q; long long ldq;    // query of row r, head h at q + r*ldq + h*dh
+  void* out; long long ldo;
+  int rows, rows_per_b, H, dh;
+  int causal;                      // 1: keys 0 .. len[b]+i ; 0: keys 0 .. limit_b[b]-1
+  const int* limit_b;
+  const void* k; const void* v;    // linear: row s of batch b at base + b*bstride + s*ldkv ; paged: page pool
+  long long ldkv, bstride;
+  int paged;
+  RowState st;
+  float scale;
+  const int* all_done;
+};
+
+// Keys are taken in chunks of 32 absolute positions, lane = key; running
+// max / sum are merged chunk by chunk in position order (fixed order).
+template <typename AT>
+__global__ void __launch_bounds__(128) attention_kernel(AttnParams p) {
+  if (p.all_done && *p.all_done) return;
+  __shared__ float qs[4][128];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int item = blockIdx.x * 4 + warp;
+  if (item >= p.rows * p.H) return;
+  const int r = item / p.H, h = item % p.H;
+  const int b = r / p.rows_per_b, i = r % p.rows_per_b;
+  const int dh = p.dh;
+  const int limit = p.causal ? (p.st.len[b] + i + 1) : p.limit_b[b];
+  const AT* q = reinterpret_cast<const AT*>(p.q) + (long long)r * p.ldq + h * dh;
+  for (int c = lane; c < dh; c += 32) qs[warp][c] = to_f(q[c]) * p.scale;
+  __syncwarp();
+  const AT* K = reinterpret_cast<const AT*>(p.k);
+  const AT* V = reinterpret_cast<const AT*>(p.v);
+  const int* pt = p.st.page_table + b * p.st.pages_per_row;
+  auto row_off = [&](int pos) -> size_t {
+    if (p.paged) return ((size_t)pt[pos / kPage] * kPage + (pos % kPage)) * p.ldkv + h * dh;
+    return (size_t)b * p.bstride + (size_t)pos * p.ldkv + h * dh;
+  };
+  float m_run = -INFINITY, l_run = 0.f;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};   // output dims lane, lane+32, lane+64, lane+96
+  for (int c0 = 0; c0 < limit; c0 += 32) {
+    const int pos = c0 + lane;
+    float s = -INFINITY;
+    if (pos < limit) {
+      const AT* kr = K + row_off(pos);
+      float dot = 0.f;
+      for (int c = 0; c < dh; c += 8) {
+        float kv[8];
+        load8(kr + c, kv);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) dot = fmaf(qs[warp][c + e], kv[e], dot);
+      }
+      s = dot;
+    }
+    const float m_new = fmaxf(m_run, warp_max(s));
+    const float corr = expf(m_run - m_new);      // exp(-inf) = 0 on the first chunk
+    const float pj = (pos < limit) ? expf(s - m_new) : 0.f;
+    l_run = l_run * corr + warp_sum(pj);
+#pragma unroll
+    for (int t = 0; t < 4; ++t) acc[t] *= corr;
+    const int nk = min(32, limit - c0);
+    for (int jj = 0; jj < nk; ++jj) {
+      const float pw = __shfl_sync(0xffffffffu, pj, jj);
+      const AT* vr = V + row_off(c0 + jj);
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        const int c = lane + 32 * t;
+        if (c < dh) acc[t] = fmaf(pw, to_f(vr[c]), acc[t]);
+      }
+    }
+    m_run = m_new;
+  }
+  AT* o = reinterpret_cast<AT*>(p.out) + (long long)r * p.ldo + h * dh;
+  const float inv = 1.f / l_run;
+#pragma unroll
+  for (int t = 0; t < 4; ++t) {
+    const int c = lane + 32 * t;
+    if (c < dh) o[c] = from_f<AT>(acc[t] * inv);
+  }
+}
+
+// ------------------------------------------------------------------ vocabulary projection + top-1
+struct ArgmaxParams {
+  const void* x; long long ldx;   // [rows, d] activations
+  const void* w;                  // [V, d]
+  int rows, d, V;
+  float* part_val; int* part_idx; // [tiles][rows] workspace
+  unsigned* counters;             // [row chunks], zero between launches
+  int* out_idx; float* out_val;   // [rows]
+  float* logits;                  // optional dump [rows, V]
+  const int* all_done;
+};
+constexpr int kVocTile = 256;     // vocabulary rows per CTA
+constexpr int kArgmaxMaxD = 1024;
+
+template <typename WT, typename AT>
+__global__ void __launch_bounds__(kLinWarps * 32) vocab_argmax_kernel(ArgmaxParams p) {
+  if (p.all_done && *p.all_done) return;
+  extern __shared__ __align__(16) float xs_dyn[];   // [kRC][d]
+  __shared__ float sv[kLinWarps][kRC];
+  __shared__ int si[kLinWarps][kRC];
+  __shared__ unsigned ticket;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r0 = blockIdx.y * kRC;
+  const int nr = min(kRC, p.rows - r0);
+  const int d = p.d;
+  const AT* X = reinterpret_cast<const AT*>(p.x);
+  const WT* W = reinterpret_cast<const WT*>(p.w);
+  for (int v = threadIdx.x; v < kRC * d / 8; v += kLinWarps * 32) {
+    const int r = v / (d / 8), kk = (v % (d / 8)) * 8;
+    float t[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    if (r < nr) load8(X + (long long)(r0 + r) * p.ldx + kk, t);
+    *reinterpret_cast<float4*>(&xs_dyn[r * d + kk]) = make_float4(t[0], t[1], t[2], t[3]);
+    *reinterpret_cast<float4*>(&xs_dyn[r * d + kk + 4]) = make_float4(t[4], t[5], t[6], t[7]);
+  }
+  __syncthreads();
+  float bv[kRC];
+  int bi[kRC];
+#pragma unroll
+  for (int r = 0; r < kRC; ++r) { bv[r] = -INFINITY; bi[r] = 0x7fffffff; }
+  const int tile0 = blockIdx.x * kVocTile;
+  for (int g = 0; g < kVocTile / (kLinWarps * kFPW); ++g) {
+    const int n0 = tile0 + g * (kLinWarps * kFPW) + warp * kFPW;   // ascending over g for a given warp
+    if (n0 >= p.V) break;
+    float acc[kFPW][kRC];
+#pragma unroll
+    for (int f = 0; f < kFPW; ++f)
+#pragma unroll
+      for (int r = 0; r < kRC; ++r) acc[f][r] = 0.f;
+    for (int kk = lane * 8; kk < d; kk += 256) {
+      float wv[kFPW][8];
+#pragma unroll
+      for (int f = 0; f < kFPW; ++f) {
+        if (n0 + f < p.V) {
+          load8_stream(W + (size_t)(n0 + f) * d + kk, wv[f]);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) wv[f][e] = 0.f;
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < kRC; ++r) {
+        const float4 a = *reinterpret_cast<const float4*>(&xs_dyn[r * d + kk]);
+        const float4 b = *reinterpret_cast<const float4*>(&xs_dyn[r * d + kk + 4]);
+        const float xv[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int f = 0; f < kFPW; ++f)
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc[f][r] = fmaf(wv[f][e], xv[e], acc[f][r]);
+      }
+    }
+#pragma unroll
+    for (int f = 0; f < kFPW; ++f)
+#pragma unroll
+      for (int r = 0; r < kRC; ++r) {
+        const float v = warp_sum(acc[f][r]);
+        if (n0 + f < p.V) {
+          if (better(v, n0 + f, bv[r], bi[r])) { bv[r] = v; bi[r] = n0 + f; }
+          if (p.logits && lane == f * kRC + r && r < nr) p.logits[(size_t)(r0 + r) * p.V + n0 + f] = v;
+        }
+      }
+  }
+  if (lane == 0) {
+#pragma unroll
+    for (int r = 0; r < kRC; ++r) { sv[warp][r] = bv[r]; si[warp][r] = bi[r]; }
+  }
+  __syncthreads();
+  if (threadIdx.x < nr) {
+    const int r = threadIdx.x;
+    float v = sv[0][r];
+    int ix = si[0][r];
+    for (int w2 = 1; w2 < kLinWarps; ++w2)
+      if (better(sv[w2][r], si[w2][r], v, ix)) { v = sv[w2][r]; ix = si[w2][r]; }
+    p.part_val[(size_t)blockIdx.x * p.rows + r0 + r] = v;
+    p.part_idx[(size_t)blockIdx.x * p.rows + r0 + r] = ix;
+  }
+  // The CTA that finishes last for this row chunk merges all tiles (no waiting on anyone).
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) ticket = atomicAdd(&p.counters[blockIdx.y], 1u);
+  __syncthreads();
+  if (ticket != gridDim.x - 1) return;
+  __threadfence();
+  for (int r = warp; r < nr; r += kLinWarps) {
+    float v = -INFINITY;
+    int ix = 0x7fffffff;
+    for (int t = lane; t < (int)gridDim.x; t += 32) {
+      const float tv = __ldcg(&p.part_val[(size_t)t * p.rows + r0 + r]);
+      const int ti = __ldcg(&p.part_idx[(size_t)t * p.rows + r0 + r]);
+      if (better(tv, ti, v, ix)) { v = tv; ix = ti; }
+    }
+    warp_argmax(v, ix);
+    if (lane == 0) {
+      p.out_idx[r0 + r] = ix;
+      if (p.out_val) p.out_val[r0 + r] = v;
+    }
+  }
+  if (threadIdx.x == 0) p.counters[blockIdx.y] = 0;
+}
+
+// ------------------------------------------------------------------ verify / accept / commit / select next
+struct VerifyParams {
+  RowState st;
+  int B, kcur, kh, knext;   // positions scored per row, heads per position, width of the next block
+  int mode;
+  int max_new, eos;
+};
+
+__global__ void verify_commit_kernel(VerifyParams p) {
+  if (*p.st.all_done) return;
+  __shared__ int any_open;
+  if (threadIdx.x == 0) any_open = 0;
+  __syncthreads();
+  const int b = threadIdx.x;
+  if (b < p.B) {
+    int* blk = p.st.block + b * kMaxK;
+    const int* cur = p.st.cur_block + b * kMaxK;
+    const int* A = p.st.table + (size_t)b * p.kcur * p.kh;
+    if (p.st.finished[b]) {
+      p.st.khat[b] = 0;
+    } else if (p.mode == kModePrime) {
+      // start token becomes part of the prefix; its row of predictions is the first block
+      p.st.len[b] += 1;
+      p.st.khat[b] = 0;
+      for (int i = 0; i < p.knext; ++i) blk[i] = A[i];
+      atomicOr(&any_open, 1);
+    } else if (p.mode == kModeGreedy) {
+      const int tok = A[0];
+      const int j = p.st.j[b];
+      p.st.out_ids[(size_t)b * p.st.max_tgt + j] = tok;
+      p.st.j[b] = j + 1;
+      p.st.len[b] += 1;
+      p.st.khat[b] = 1;
+      blk[0] = tok;
+      const int fin = (j + 1 >= p.max_new) || (p.eos >= 0 && tok == p.eos);
+      p.st.finished[b] = fin;
+      if (!fin) atomicOr(&any_open, 1);
+      atomicAdd((unsigned long long*)&p.st.stats[0], 1ull);
+      atomicAdd((unsigned long long*)&p.st.stats[1], 1ull);
+      atomicAdd((unsigned long long*)&p.st.stats[3 + 1], 1ull);
+    } else {
+      // longest prefix of the block that the base model would have produced itself:
+      // proposal i+1 is checked against head 1 at the position of proposal i
+      int khat = 1;
+      while (khat < p.kcur && cur[khat] == A[(khat - 1) * p.kh]) ++khat;
+      const int j = p.st.j[b];
+      khat = min(khat, p.max_new - j);
+      int fin = (j + khat >= p.max_new);
+      if (p.eos >= 0) {
+        for (int i = 0; i < khat; ++i)
+          if (cur[i] == p.eos) { khat = i + 1; fin = 1; break; }
+      }
+      for (int i = 0; i < khat; ++i) p.st.out_ids[(size_t)b * p.st.max_tgt + j + i] = cur[i];
+      p.st.j[b] = j + khat;
+      p.st.len[b] += khat;      // keys/values of rejected positions stay behind the length and get overwritten
+      p.st.khat[b] = khat;
+      for (int i = 0; i < p.knext; ++i) blk[i] = A[(khat - 1) * p.kh + i];
+      p.st.finished[b] = fin;
+      if (!fin) atomicOr(&any_open, 1);
+      atomicAdd((unsigned long long*)&p.st.stats[0], 1ull);
+      atomicAdd((unsigned long long*)&p.st.stats[1], (unsigned long long)khat);
+      atomicAdd((unsigned long long*)&p.st.stats[3 + khat], 1ull);
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    if (p.mode != kModePrime) p.st.stats[2] += 1;
+    if (!any_open) *p.st.all_done = 1;
+  }
+}
+
+struct ResetParams {
+  RowState st;
+  int B, ppr;
+  const int* src_len;
+};
+__global__ void reset_rows_kernel(ResetParams p) {
+  const int b = threadIdx.x;
+  if (b < p.B) {
+    p.st.len[b] = 0;
+    p.st.j[b] = 0;
+    p.st.finished[b] = 0;
+    p.st.khat[b] = 0;
+    p.st.src_len[b] = p.src_len[b];
+    for (int i = 0; i < kMaxK; ++i) { p.st.block[b * kMaxK + i] = 0; p.st.cur_block[b * kMaxK + i] = 0; }
+  }
+  if (threadIdx.x == 0) {
+    *p.st.all_done = 0;
+    *p.st.error = 0;
+    for (int i = 0; i < 3 + kMaxK + 1; ++i) p.st.stats[i] = 0;
+  }
+}
+
+}  // namespace bpd

@@ -1,0 +1,285 @@
+"""GPU parity: the CUDA library against the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+
+from bpd_inputs import (DTYPE_BF16, DTYPE_F32, HEAD_BLOCKDIAG, HEAD_DENSE, WORKLOADS, ModelConfig, Workload,
+                        forced_tail, geometric_schedule, make_source, make_weights)
+
+pytestmark = pytest.mark.gpu
+
+MINI = Workload("mini", ModelConfig(2, 2, 128, 2, 256, 1000, 4, 256, dtype=DTYPE_BF16), 0.05,
+                11, 12, 13, batch=1, src_lo=9, src_hi=9, n_decode=24)
+MINI_BLOCK = MINI.with_layout(HEAD_BLOCKDIAG)
+MINI_BATCH = Workload("mini3", MINI.cfg, 0.05, 11, 22, 23, batch=3, src_lo=3, src_hi=11, n_decode=20)
+MINI_F32 = Workload("minif", ModelConfig(1, 2, 96, 6, 200, 333, 3, 136, dtype=DTYPE_F32), 0.1,
+                    31, 32, 33, batch=2, src_lo=2, src_hi=7, n_decode=15)
+
+
+@pytest.fixture(scope="module")
+def bpd():
+    import paper_1811_03115_b200 as pkg
+    return pkg
+
+
+def _setup(bpd, w, extra_tgt=0):
+    from oracle.model import parse_blob
+    blob = make_weights(w.cfg, w.weight_seed, w.sigma)
+    model = bpd.Model(blob)
+    src, src_len = make_source(w)
+    return blob, model, src, src_len, parse_blob(blob)
+
+
+def _tail_fn(w, greedy_ids, k, mean):
+    sched = [geometric_schedule(w.accept_seed * 1000 + b, mean, w.n_decode + 1) for b in range(w.batch)]
+
+    def fn(b, j, it):
+        G, R = sched[b]
+        jj = min(j, w.n_decode)
+        return forced_tail(greedy_ids[b], jj, k, int(G[jj]), int(R[jj]), w.cfg.vocab)
+    return fn, sched
+
+
+def _plan(w, greedy_ids, k, mean):
+    fn, sched = _tail_fn(w, greedy_ids, k, mean)
+    plan = np.zeros((w.batch, w.n_decode, k - 1), dtype=np.int32)
+    for b in range(w.batch):
+        for j in range(w.n_decode):
+            plan[b, j] = fn(b, j, 0)
+    return plan, sched
+
+
+def _expected_khats(sched_b, k, n):
+    G, _ = sched_b
+    j, out = 0, []
+    while j < n:
+        kh = min(k, int(G[j]), n - j)
+        out.append(kh)
+        j += kh
+    return out
+
+
+# ---------------------------------------------------------------- single operators
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("rows,in_f,out_f", [(1, 64, 50), (8, 1024, 3072), (13, 520, 77), (64, 256, 129)])
+def test_op_linear_matches_definition(bpd, dtype, rows, in_f, out_f):
+    import torch
+    g = torch.Generator().manual_seed(rows * 1000 + in_f)
+    td = torch.float32 if dtype == "f32" else torch.bfloat16
+    x = (torch.randn(rows, in_f, generator=g)).to(td)
+    w = (torch.randn(out_f, in_f, generator=g) * 0.05).to(td)
+    b = (torch.randn(out_f, generator=g) * 0.1).to(td)
+    want = x.double().numpy() @ w.double().numpy().T + b.double().numpy()
+    y = bpd.bpd_op_linear(x.cuda(), w.cuda(), b.cuda(), relu=False).cpu().numpy()
+    np.testing.assert_allclose(y, want, atol=2e-4 * np.sqrt(in_f / 64))
+    y = bpd.bpd_op_linear(x.cuda(), w.cuda(), None, relu=True).cpu().numpy()
+    np.testing.assert_allclose(y, np.maximum(want - b.double().numpy(), 0), atol=2e-4 * np.sqrt(in_f / 64))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("rows,d,vocab", [(1, 64, 5), (16, 512, 1000), (64, 1024, 32768), (9, 128, 257)])
+def test_op_vocab_argmax_matches_definition(bpd, dtype, rows, d, vocab):
+    import torch
+    from oracle.model import argmax_lowest
+    g = torch.Generator().manual_seed(rows + d + vocab)
+    td = torch.float32 if dtype == "f32" else torch.bfloat16
+    x = torch.randn(rows, d, generator=g).to(td)
+    w = (torch.randn(vocab, d, generator=g) * 0.02).to(td)
+    if vocab > 8:
+        w[7] = w[3]                      # an exact tie: the lower id must win if it is the maximum
+        x[0] = (w[3].float() * 50).to(td)
+    logits = x.double().numpy() @ w.double().numpy().T
+    idx, val = bpd.bpd_op_vocab_argmax(x.cuda(), w.cuda(), want_val=True)
+    idx, val = idx.cpu().numpy(), val.cpu().numpy()
+    want = argmax_lowest(logits)
+    best = logits.max(-1)
+    for r in range(rows):
+        second = np.partition(logits[r], -2)[-2] if vocab > 1 else -np.inf
+        if best[r] - second > 1e-3:
+            assert idx[r] == want[r]
+        assert abs(logits[r, idx[r]] - best[r]) <= 1e-3
+        assert abs(val[r] - best[r]) <= 1e-3
+    if vocab > 8:
+        assert idx[0] == 3
+    # a second call on the same scratch-free path gives the same answer (counters were reset)
+    idx2 = bpd.bpd_op_vocab_argmax(x.cuda(), w.cuda()).cpu().numpy()
+    assert np.array_equal(idx, idx2)
+
+
+# ---------------------------------------------------------------- whole path, small models
+
+@pytest.mark.parametrize("w", [WORKLOADS["C1"], MINI, MINI_BLOCK, MINI_BATCH, MINI_F32], ids=lambda w: w.name)
+def test_greedy_blockwise_and_lockstep(bpd, w):
+    from harness import lockstep
+    blob, model, src, src_len, om = _setup(bpd, w)
+    k, N = w.cfg.k_model, w.n_decode
+    s = bpd.Session(model, w.batch, w.max_src, N)
+    # greedy, then blockwise: identical ids (the guarantee of Section 3), on the GPU alone
+    s.bpd_encode(src, src_len)
+    g_ids, g_len, g_st = s.bpd_decode_greedy(N)
+    assert np.all(g_len == N) and g_st.tokens == N * w.batch and g_st.invocations == N
+    for kk in sorted({1, 2, k}):
+        s.bpd_encode(src, src_len)
+        b_ids, b_len, b_st = s.bpd_decode_blockwise(kk, N)
+        assert np.array_equal(b_ids, g_ids), f"k={kk}: blockwise differs from greedy"
+        assert b_st.tokens == N * w.batch and b_st.invocations == b_st.iterations + 1
+        assert sum(c * n for c, n in enumerate(b_st.khat_hist)) == N * w.batch
+        if kk == 1:
+            assert b_st.iterations == N
+    # controlled acceptance through the device-resident plan: khat is known in advance
+    for mean in (2.0, 5.0):
+        plan, sched = _plan(w, g_ids, k, mean)
+        s.bpd_encode(src, src_len)
+        s.bpd_set_forced_plan(plan, k)
+        p_ids, _, p_st = s.bpd_decode_blockwise(k, N)
+        assert np.array_equal(p_ids, g_ids)
+        want = [_expected_khats(sched[b], k, N) for b in range(w.batch)]
+        hist = np.zeros(17, dtype=np.int64)
+        for row in want:
+            for kh in row:
+                hist[kh] += 1
+        assert list(hist) == list(p_st.khat_hist)
+        assert p_st.iterations == max(len(r) for r in want)
+        assert p_st.row_iterations == sum(len(r) for r in want)
+    # lock-step against the oracle: free-running, then with forced tails
+    rep = lockstep(s, om, src, src_len, k, N, max_iters=N)
+    for b in range(w.batch):
+        assert rep.emitted[b] == list(g_ids[b]), "lock-step output differs from the GPU's greedy decode"
+    if w.cfg.dtype == DTYPE_F32:
+        assert rep.adopted == 0
+    fn, sched = _tail_fn(w, g_ids, k, 2.0)
+    rep2 = lockstep(s, om, src, src_len, k, N, max_iters=N, tail_fn=fn)
+    for b in range(w.batch):
+        assert [r[b] for r in rep2.khats if r[b] > 0] == _expected_khats(sched[b], k, N)
+    s.close()
+    model.close()
+
+
+def test_c1_ids_equal_oracle_greedy(bpd):
+    """fp32 weights: the GPU's greedy and blockwise ids are the oracle's greedy ids."""
+    from oracle.decode import TransformerScorer, blockwise_merged, greedy
+    w = WORKLOADS["C1"]
+    blob, model, src, src_len, om = _setup(bpd, w)
+    s = bpd.Session(model, 1, w.max_src, w.n_decode)
+    s.bpd_encode(src, src_len)
+    ids, _, _ = s.bpd_decode_blockwise(4, w.n_decode)
+    sc = TransformerScorer(om, src[0, :src_len[0]], cached=True, capacity=w.n_decode + 12)
+    want = greedy(sc, w.n_decode)
+    assert list(ids[0]) == want.ids
+    ob = blockwise_merged(TransformerScorer(om, src[0, :src_len[0]], cached=True, capacity=w.n_decode + 12),
+                          4, w.n_decode)
+    s.bpd_encode(src, src_len)
+    _, _, st = s.bpd_decode_blockwise(4, w.n_decode)
+    assert st.iterations == ob.iterations and st.invocations == ob.invocations
+    s.close()
+    model.close()
+
+
+def test_eos_terminates_inside_a_block(bpd):
+    w = MINI
+    blob, model, src, src_len, om = _setup(bpd, w)
+    N, k = w.n_decode, 4
+    s = bpd.Session(model, 1, w.max_src, N)
+    s.bpd_encode(src, src_len)
+    g_ids, _, _ = s.bpd_decode_greedy(N)
+    eos_at = 6
+    eos = int(g_ids[0, eos_at])
+    first = list(g_ids[0]).index(eos)
+    plan = np.zeros((1, N, k - 1), dtype=np.int32)
+    for j in range(N):
+        plan[0, j] = forced_tail(g_ids[0], j, k, k, 0, w.cfg.vocab)     # always-right proposals
+    s.bpd_encode(src, src_len)
+    s.bpd_set_forced_plan(plan, k)
+    ids, ln, st = s.bpd_decode_blockwise(k, N, eos_id=eos)
+    assert ln[0] == first + 1 and list(ids[0, :first + 1]) == list(g_ids[0, :first + 1])
+    assert np.all(ids[0, first + 1:] == -1)
+    assert st.iterations == -(-(first + 1) // k)
+    s.bpd_encode(src, src_len)
+    ids2, ln2, _ = s.bpd_decode_greedy(N, eos_id=eos)
+    assert ln2[0] == first + 1 and np.array_equal(ids2, ids)
+    s.close()
+    model.close()
+
+
+def test_state_and_argument_errors(bpd):
+    w = MINI
+    blob, model, src, src_len, _ = _setup(bpd, w)
+    s = bpd.Session(model, 1, w.max_src, 16)
+    with pytest.raises(bpd.BpdError) as e:
+        s.bpd_decode_greedy(8)
+    assert e.value.status == -5
+    s.bpd_encode(src, src_len)
+    with pytest.raises(bpd.BpdError) as e:
+        s.bpd_decode_blockwise(5, 8)          # k above k_model
+    assert e.value.status == -1
+    with pytest.raises(bpd.BpdError) as e:
+        s.bpd_decode_greedy(17)               # above max_tgt
+    assert e.value.status == -2
+    bad = src.copy()
+    bad[0, 0] = w.cfg.vocab
+    with pytest.raises(bpd.BpdError) as e:
+        s.bpd_encode(bad, src_len)
+    assert e.value.status == -1
+    s.bpd_encode(src, src_len)
+    s.bpd_decode_greedy(8)
+    with pytest.raises(bpd.BpdError) as e:
+        s.bpd_iteration(4, 8)                 # greedy session cannot continue blockwise
+    assert e.value.status == -5
+    s.close()
+    model.close()
+
+
+# ---------------------------------------------------------------- paper-sized configurations
+
+def _full_size(bpd, name, iters, rows=None, layout=HEAD_DENSE, mean=2.0, free_iters=2):
+    from harness import lockstep
+    w = WORKLOADS[name].with_layout(layout)
+    blob, model, src, src_len, om = _setup(bpd, w)
+    del blob
+    k, N = w.cfg.k_model, w.n_decode
+    s = bpd.Session(model, w.batch, w.max_src, N)
+    s.bpd_encode(src, src_len)
+    g_ids, _, _ = s.bpd_decode_greedy(N)
+    s.bpd_encode(src, src_len)
+    b_ids, _, b_st = s.bpd_decode_blockwise(k, N)
+    assert np.array_equal(b_ids, g_ids)
+    plan, sched = _plan(w, g_ids, k, mean)
+    s.bpd_encode(src, src_len)
+    s.bpd_set_forced_plan(plan, k)
+    p_ids, _, p_st = s.bpd_decode_blockwise(k, N)
+    assert np.array_equal(p_ids, g_ids)
+    want = [_expected_khats(sched[b], k, N) for b in range(w.batch)]
+    assert p_st.row_iterations == sum(len(r) for r in want)
+    assert p_st.iterations == max(len(r) for r in want)
+    rep = lockstep(s, om, src, src_len, k, N, max_iters=free_iters, rows=rows)
+    fn, _ = _tail_fn(w, g_ids, k, mean)
+    rep2 = lockstep(s, om, src, src_len, k, N, max_iters=iters, tail_fn=fn, rows=rows)
+    for b in (rows if rows is not None else range(w.batch)):
+        got = [r[i] for r in rep2.khats for i, bb in enumerate(rows if rows is not None else range(w.batch)) if bb == b]
+        assert got == want[b][:len(got)]
+    s.close()
+    model.close()
+    return rep, rep2
+
+
+def test_c2_base_model(bpd):
+    _full_size(bpd, "C2", iters=6)
+
+
+def test_c2_base_model_blockdiag(bpd):
+    _full_size(bpd, "C2", iters=3, layout=HEAD_BLOCKDIAG)
+
+
+def test_c3_big_model(bpd):
+    _full_size(bpd, "C3", iters=3, mean=5.0, free_iters=1)
+
+
+def test_c5_super_resolution_shape(bpd):
+    _full_size(bpd, "C5", iters=3, mean=5.0, free_iters=1)
+
+
+def test_c4_batch32_ragged(bpd):
+    w = WORKLOADS["C4"]
+    _, src_len = make_source(w)
+    rows = sorted({int(np.argmin(src_len)), int(np.argmax(src_len)), 0, w.batch - 1})
+    _full_size(bpd, "C4", iters=2, rows=rows, mean=2.0, free_iters=1)
