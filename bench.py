@@ -150,7 +150,7 @@ def run_reference(args):
     k = w.cfg.k_model
     blob = make_weights(w.cfg, w.weight_seed, w.sigma)
     src, src_len = make_source(w)
-    n_tokens = 12
+    n_tokens = 32
     tps, times, threads = oracle_sample(w, blob, src, src_len, k, MEAN_ACCEPT, n_tokens,
                                         repeats=args.steps + args.warmup)
     timed = times[args.warmup:]
@@ -298,7 +298,7 @@ def run_gpu(args):
     # ---- oracle on the host cores, bounded sample
     cpu = None
     if not args.no_cpu:
-        n_tok = 12
+        n_tok = N
         tps, times, threads = oracle_sample(w, blob, src, src_len, k, MEAN_ACCEPT, n_tok, repeats=2)
         cpu = {"value": tps, "unit": "tokens/s", "cores": threads, "kind": "oracle",
                "sample": f"first {n_tok} of {N} tokens, 2 decodes, {np.mean(times):.1f} s each"}

@@ -117,7 +117,8 @@ static int pages_per_row(const Config& c, int max_tgt) { return ceil_div(max_tgt
 static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, char* base, bpd_session* s) {
   Arena a;
   a.base = base;
-  const size_t ea = c.elem();
+  const size_t ea = sizeof(float);   // activations stay fp32 between kernels; only weights and the cache are narrow
+  const size_t ec = c.elem();
   const size_t Rmax = (size_t)B * c.k_model, E = (size_t)B * max_src, Rall = std::max(Rmax, E);
   const size_t R2 = Rmax * c.k_model;
   const int ppr = pages_per_row(c, max_tgt);
@@ -133,8 +134,8 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
   std::vector<void*> crosskv(c.n_dec), kc(c.n_dec), vc(c.n_dec);
   for (int l = 0; l < c.n_dec; ++l) crosskv[l] = a.take_bytes(E * 2 * d * ea);
   for (int l = 0; l < c.n_dec; ++l) {
-    kc[l] = a.take_bytes((size_t)B * ppr * kPage * d * ea);
-    vc[l] = a.take_bytes((size_t)B * ppr * kPage * d * ea);
+    kc[l] = a.take_bytes((size_t)B * ppr * kPage * d * ec);
+    vc[l] = a.take_bytes((size_t)B * ppr * kPage * d * ec);
   }
   int* page_table = a.take<int>((size_t)B * ppr);
   RowState st;
@@ -144,7 +145,7 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
   st.table = a.take<int>((size_t)B * kMaxK * kMaxK);
   st.out_ids = a.take<int>((size_t)B * max_tgt);
   st.all_done = a.take<int>(1); st.error = a.take<int>(1);
-  st.stats = a.take<long long>(3 + kMaxK + 1);
+  st.stats = a.take<long long>(4 + kMaxK + 1);
   st.page_table = page_table; st.pages_per_row = ppr; st.max_tgt = max_tgt;
   int* src_dev = a.take<int>(E);
   int* tail_dev = a.take<int>((size_t)B * kMaxK);
@@ -219,7 +220,7 @@ static void prof_clear(bpd_session* s) {
 }
 
 // ------------------------------------------------------------------ encoder
-template <typename WT, typename AT>
+template <typename WT>
 static int run_encoder(bpd_session* s) {
   const bpd_model* m = s->m;
   const Config& c = m->cfg;
@@ -233,26 +234,26 @@ static int run_encoder(bpd_session* s) {
   ++g_launches;
   for (int l = 0; l < c.n_enc; ++l) {
     const EncLayer& L = m->enc[l];
-    launch_ln<WT, AT>(s->x, L.ln1g, L.ln1b, s->xn, nullptr, E, d, c.eps, nullptr, st);
-    launch_linear<WT, AT, kEpiStoreAct>(lin(s->xn, d, L.wqkv, d, 3 * d, nullptr, E, s->qbuf, 3 * d, 0, nullptr), 1, st);
+    launch_ln<WT, float>(s->x, L.ln1g, L.ln1b, s->xn, nullptr, E, d, c.eps, nullptr, st);
+    launch_linear<WT, float, kEpiStoreAct>(lin(s->xn, d, L.wqkv, d, 3 * d, nullptr, E, s->qbuf, 3 * d, 0, nullptr), 1, st);
     AttnParams ap;
     memset(&ap, 0, sizeof(ap));
     ap.q = s->qbuf; ap.ldq = 3 * d; ap.out = s->attn; ap.ldo = d; ap.rows = E; ap.rows_per_b = s->max_src;
     ap.H = c.H; ap.dh = d / c.H; ap.causal = 0; ap.limit_b = s->st.src_len;
-    ap.k = static_cast<AT*>(s->qbuf) + d; ap.v = static_cast<AT*>(s->qbuf) + 2 * d;
+    ap.k = static_cast<float*>(s->qbuf) + d; ap.v = static_cast<float*>(s->qbuf) + 2 * d;
     ap.ldkv = 3 * d; ap.bstride = (long long)s->max_src * 3 * d; ap.paged = 0; ap.st = s->st;
     ap.scale = 1.0f / sqrtf((float)ap.dh);
-    attention_kernel<AT><<<ceil_div(E * c.H, 4), 128, 0, st>>>(ap);
+    attention_kernel<float, float><<<ceil_div(E * c.H, 4), 128, 0, st>>>(ap);
     ++g_launches;
     LinearParams po = lin(s->attn, d, L.wo, d, d, nullptr, E, s->x, d, 0, nullptr);
-    launch_linear<WT, AT, kEpiResidual>(po, 1, st);
-    launch_ln<WT, AT>(s->x, L.ln2g, L.ln2b, s->xn, nullptr, E, d, c.eps, nullptr, st);
-    launch_linear<WT, AT, kEpiStoreAct>(lin(s->xn, d, L.w1, d, c.d_ff, L.b1, E, s->ffh, c.d_ff, 1, nullptr), 1, st);
-    launch_linear<WT, AT, kEpiResidual>(lin(s->ffh, c.d_ff, L.w2, c.d_ff, d, L.b2, E, s->x, d, 0, nullptr), 1, st);
+    launch_linear<WT, float, kEpiResidual>(po, 1, st);
+    launch_ln<WT, float>(s->x, L.ln2g, L.ln2b, s->xn, nullptr, E, d, c.eps, nullptr, st);
+    launch_linear<WT, float, kEpiStoreAct>(lin(s->xn, d, L.w1, d, c.d_ff, L.b1, E, s->ffh, c.d_ff, 1, nullptr), 1, st);
+    launch_linear<WT, float, kEpiResidual>(lin(s->ffh, c.d_ff, L.w2, c.d_ff, d, L.b2, E, s->x, d, 0, nullptr), 1, st);
   }
-  launch_ln<WT, AT>(s->x, m->enc_lnf_g, m->enc_lnf_b, s->xn, nullptr, E, d, c.eps, nullptr, st);
+  launch_ln<WT, float>(s->x, m->enc_lnf_g, m->enc_lnf_b, s->xn, nullptr, E, d, c.eps, nullptr, st);
   for (int l = 0; l < c.n_dec; ++l)
-    launch_linear<WT, AT, kEpiStoreAct>(lin(s->xn, d, m->dec[l].cwkv, d, 2 * d, nullptr, E, s->crosskv[l], 2 * d, 0, nullptr), 1, st);
+    launch_linear<WT, float, kEpiStoreAct>(lin(s->xn, d, m->dec[l].cwkv, d, 2 * d, nullptr, E, s->crosskv[l], 2 * d, 0, nullptr), 1, st);
   BPD_CUDA(cudaGetLastError());
   return BPD_OK;
 }
@@ -269,7 +270,7 @@ struct PassArgs {
   float* logits_dump;   // device [B*kcur*kh, V] or null
 };
 
-template <typename WT, typename AT>
+template <typename WT>
 static int run_pass(bpd_session* s, const PassArgs& a) {
   const bpd_model* m = s->m;
   const Config& c = m->cfg;
@@ -287,55 +288,55 @@ static int run_pass(bpd_session* s, const PassArgs& a) {
   for (int l = 0; l < c.n_dec; ++l) {
     const DecLayer& L = m->dec[l];
     // self-attention over the cache plus the causal part of the block
-    launch_ln<WT, AT>(s->x, L.ln1g, L.ln1b, s->xn, nullptr, R, d, c.eps, done, st);
+    launch_ln<WT, float>(s->x, L.ln1g, L.ln1b, s->xn, nullptr, R, d, c.eps, done, st);
     LinearParams pq = lin(s->xn, d, L.wqkv, d, 3 * d, nullptr, R, s->qbuf, d, 0, done);
     pq.d = d; pq.kcache = s->kcache[l]; pq.vcache = s->vcache[l]; pq.st = s->st; pq.rows_per_b = a.kcur;
-    launch_linear<WT, AT, kEpiQkv>(pq, 1, st);
+    launch_linear<WT, float, kEpiQkv>(pq, 1, st);
     AttnParams ap;
     memset(&ap, 0, sizeof(ap));
     ap.q = s->qbuf; ap.ldq = d; ap.out = s->attn; ap.ldo = d; ap.rows = R; ap.rows_per_b = a.kcur;
     ap.H = c.H; ap.dh = d / c.H; ap.causal = 1; ap.k = s->kcache[l]; ap.v = s->vcache[l]; ap.ldkv = d;
     ap.paged = 1; ap.st = s->st; ap.scale = 1.0f / sqrtf((float)ap.dh); ap.all_done = done;
-    attention_kernel<AT><<<ceil_div(R * c.H, 4), 128, 0, st>>>(ap);
+    attention_kernel<float, WT><<<ceil_div(R * c.H, 4), 128, 0, st>>>(ap);
     ++g_launches;
-    launch_linear<WT, AT, kEpiResidual>(lin(s->attn, d, L.wo, d, d, nullptr, R, s->x, d, 0, done), 1, st);
+    launch_linear<WT, float, kEpiResidual>(lin(s->attn, d, L.wo, d, d, nullptr, R, s->x, d, 0, done), 1, st);
     // cross-attention over the encoder memory
-    launch_ln<WT, AT>(s->x, L.ln2g, L.ln2b, s->xn, nullptr, R, d, c.eps, done, st);
-    launch_linear<WT, AT, kEpiStoreAct>(lin(s->xn, d, L.cwq, d, d, nullptr, R, s->qbuf, d, 0, done), 1, st);
-    ap.causal = 0; ap.limit_b = s->st.src_len; ap.k = s->crosskv[l]; ap.v = static_cast<AT*>(s->crosskv[l]) + d;
+    launch_ln<WT, float>(s->x, L.ln2g, L.ln2b, s->xn, nullptr, R, d, c.eps, done, st);
+    launch_linear<WT, float, kEpiStoreAct>(lin(s->xn, d, L.cwq, d, d, nullptr, R, s->qbuf, d, 0, done), 1, st);
+    ap.causal = 0; ap.limit_b = s->st.src_len; ap.k = s->crosskv[l]; ap.v = static_cast<float*>(s->crosskv[l]) + d;
     ap.ldkv = 2 * d; ap.bstride = (long long)s->max_src * 2 * d; ap.paged = 0;
-    attention_kernel<AT><<<ceil_div(R * c.H, 4), 128, 0, st>>>(ap);
+    attention_kernel<float, float><<<ceil_div(R * c.H, 4), 128, 0, st>>>(ap);
     ++g_launches;
-    launch_linear<WT, AT, kEpiResidual>(lin(s->attn, d, L.cwo, d, d, nullptr, R, s->x, d, 0, done), 1, st);
+    launch_linear<WT, float, kEpiResidual>(lin(s->attn, d, L.cwo, d, d, nullptr, R, s->x, d, 0, done), 1, st);
     // feed-forward
-    launch_ln<WT, AT>(s->x, L.ln3g, L.ln3b, s->xn, nullptr, R, d, c.eps, done, st);
-    launch_linear<WT, AT, kEpiStoreAct>(lin(s->xn, d, L.w1, d, c.d_ff, L.b1, R, s->ffh, c.d_ff, 1, done), 1, st);
-    launch_linear<WT, AT, kEpiResidual>(lin(s->ffh, c.d_ff, L.w2, c.d_ff, d, L.b2, R, s->x, d, 0, done), 1, st);
+    launch_ln<WT, float>(s->x, L.ln3g, L.ln3b, s->xn, nullptr, R, d, c.eps, done, st);
+    launch_linear<WT, float, kEpiStoreAct>(lin(s->xn, d, L.w1, d, c.d_ff, L.b1, R, s->ffh, c.d_ff, 1, done), 1, st);
+    launch_linear<WT, float, kEpiResidual>(lin(s->ffh, c.d_ff, L.w2, c.d_ff, d, L.b2, R, s->x, d, 0, done), 1, st);
   }
-  launch_ln<WT, AT>(s->x, m->dec_lnf_g, m->dec_lnf_b, s->xn, s->h_f32, R, d, c.eps, done, st);
+  launch_ln<WT, float>(s->x, m->dec_lnf_g, m->dec_lnf_b, s->xn, s->h_f32, R, d, c.eps, done, st);
   prof_mark(s, kProfLayers, 1);
   // proposal heads: hidden layer, k output layers with a residual from the decoder output
   const int fh = c.d_hidden;
   const long long ldu = (long long)c.k_model * fh;
   const int hid = (c.head_layout == 0) ? c.k_model * fh : a.kh * fh;
   prof_mark(s, kProfHeadW1, 0);
-  launch_linear<WT, AT, kEpiStoreAct>(lin(s->xn, d, m->head_w1, d, hid, m->head_b1, R, s->u, ldu, 1, done), 1, st);
+  launch_linear<WT, float, kEpiStoreAct>(lin(s->xn, d, m->head_w1, d, hid, m->head_b1, R, s->u, ldu, 1, done), 1, st);
   prof_mark(s, kProfHeadW1, 1);
   prof_mark(s, kProfHeadW2, 0);
   if (c.head_layout == 0) {
     LinearParams ph = lin(s->u, ldu, m->head_w2, c.k_model * fh, a.kh * d, m->head_b2, R, s->o, (long long)a.kh * d, 0, done);
     ph.h = s->h_f32; ph.d = d; ph.head_identity = c.p1_identity;
-    launch_linear<WT, AT, kEpiHeadOut>(ph, 1, st);
+    launch_linear<WT, float, kEpiHeadOut>(ph, 1, st);
   } else {
     LinearParams ph = lin(s->u, ldu, m->head_w2, fh, d, m->head_b2, R, s->o, (long long)a.kh * d, 0, done);
     ph.xz = fh; ph.wz = (long long)d * fh; ph.bz = d; ph.yz = d;
     ph.h = s->h_f32; ph.d = d; ph.head_identity = c.p1_identity;
-    launch_linear<WT, AT, kEpiHeadOut>(ph, a.kh, st);
+    launch_linear<WT, float, kEpiHeadOut>(ph, a.kh, st);
   }
   prof_mark(s, kProfHeadW2, 1);
   // shared vocabulary projection with a fused top-1: table[b][r][i]
   prof_mark(s, kProfVocab, 0);
-  launch_vocab_argmax<WT, AT>(s->o, m->out_proj, R2, d, c.V, s->part_val, s->part_idx, s->counters, s->st.table,
+  launch_vocab_argmax<WT, float>(s->o, m->out_proj, R2, d, c.V, s->part_val, s->part_idx, s->counters, s->st.table,
                               nullptr, a.logits_dump, done, st);
   prof_mark(s, kProfVocab, 1);
   VerifyParams vp{s->st, s->B, a.kcur, a.kh, a.knext, a.mode, a.max_new, a.eos};
@@ -347,7 +348,7 @@ static int run_pass(bpd_session* s, const PassArgs& a) {
 }
 
 static int dispatch_pass(bpd_session* s, const PassArgs& a) {
-  return s->m->cfg.dtype == 0 ? run_pass<float, float>(s, a) : run_pass<bf16, bf16>(s, a);
+  return s->m->cfg.dtype == 0 ? run_pass<float>(s, a) : run_pass<bf16>(s, a);
 }
 
 static int check_device_error(bpd_session* s) {
@@ -363,7 +364,7 @@ static int check_device_error(bpd_session* s) {
 static int fetch(bpd_session* s, int max_new, int32_t* out_ids, int32_t* out_len, bpd_stats* stats, float ms) {
   const int B = s->B;
   std::vector<int> ids, jj(B);
-  std::vector<long long> sv(3 + kMaxK + 1);
+  std::vector<long long> sv(4 + kMaxK + 1);
   if (out_ids) {
     ids.resize((size_t)B * s->max_tgt);
     BPD_CUDA(cudaMemcpyAsync(ids.data(), s->st.out_ids, ids.size() * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
@@ -381,8 +382,8 @@ static int fetch(bpd_session* s, int max_new, int32_t* out_ids, int32_t* out_len
   if (stats) {
     memset(stats, 0, sizeof(*stats));
     stats->row_iterations = sv[0]; stats->tokens = sv[1]; stats->iterations = sv[2];
-    for (int i = 0; i <= kMaxK; ++i) stats->khat_hist[i] = sv[3 + i];
-    stats->invocations = s->invocations;
+    for (int i = 0; i <= kMaxK; ++i) stats->khat_hist[i] = sv[4 + i];
+    stats->invocations = sv[2] + sv[3];   // passes that did work (passes issued after the end return at once)
     stats->device_ms = ms;
   }
   return BPD_OK;
@@ -542,7 +543,7 @@ int bpd_encode(bpd_session* s, const int32_t* src_ids, const int32_t* src_len) {
   reset_rows_kernel<<<1, 32 * ceil_div(B, 32), 0, s->stream>>>(rp);
   ++g_launches;
   BPD_CUDA(cudaStreamSynchronize(s->stream));   // host vectors go out of scope
-  int rc = (c.dtype == 0) ? run_encoder<float, float>(s) : run_encoder<bf16, bf16>(s);
+  int rc = (c.dtype == 0) ? run_encoder<float>(s) : run_encoder<bf16>(s);
   if (rc) return rc;
   s->phase = kPhaseEncoded; s->plan_len = 0; s->plan_k = 0; s->invocations = 0;
   return BPD_OK;

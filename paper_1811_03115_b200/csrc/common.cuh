@@ -86,7 +86,7 @@ struct RowState {
   int* out_ids;    // [B][max_tgt]
   int* all_done;   // [1]
   int* error;      // [1] first device-side error code
-  long long* stats;  // [0] row_iterations, [1] tokens, [2] iterations, [3..3+kMaxK] khat histogram
+  long long* stats;  // [0] row_iterations, [1] tokens, [2] iterations, [3] priming passes, [4..4+kMaxK] khat histogram
   const int* page_table;  // [B][pages_per_row]
   int pages_per_row;
   int max_tgt;

@@ -148,8 +148,9 @@ __device__ __forceinline__ void linear_epilogue(const LinearParams& p, int z, in
       const int pos = p.st.len[b] + i;
       const int page = p.st.page_table[b * p.st.pages_per_row + pos / kPage];
       const size_t slot = ((size_t)page * kPage + (pos % kPage)) * d;
-      if (n < 2 * d) reinterpret_cast<AT*>(p.kcache)[slot + (n - d)] = from_f<AT>(v);
-      else reinterpret_cast<AT*>(p.vcache)[slot + (n - 2 * d)] = from_f<AT>(v);
+      // the cache is stored in the weights' element type
+      if (n < 2 * d) reinterpret_cast<WT*>(p.kcache)[slot + (n - d)] = from_f<WT>(v);
+      else reinterpret_cast<WT*>(p.vcache)[slot + (n - 2 * d)] = from_f<WT>(v);
     }
   }
 }
@@ -237,7 +238,7 @@ struct AttnParams {
 
 // Keys are taken in chunks of 32 absolute positions, lane = key; running
 // max / sum are merged chunk by chunk in position order (fixed order).
-template <typename AT>
+template <typename QT, typename CT>
 __global__ void __launch_bounds__(128) attention_kernel(AttnParams p) {
   if (p.all_done && *p.all_done) return;
   __shared__ float qs[4][128];
@@ -248,11 +249,11 @@ __global__ void __launch_bounds__(128) attention_kernel(AttnParams p) {
   const int b = r / p.rows_per_b, i = r % p.rows_per_b;
   const int dh = p.dh;
   const int limit = p.causal ? (p.st.len[b] + i + 1) : p.limit_b[b];
-  const AT* q = reinterpret_cast<const AT*>(p.q) + (long long)r * p.ldq + h * dh;
+  const QT* q = reinterpret_cast<const QT*>(p.q) + (long long)r * p.ldq + h * dh;
   for (int c = lane; c < dh; c += 32) qs[warp][c] = to_f(q[c]) * p.scale;
   __syncwarp();
-  const AT* K = reinterpret_cast<const AT*>(p.k);
-  const AT* V = reinterpret_cast<const AT*>(p.v);
+  const CT* K = reinterpret_cast<const CT*>(p.k);
+  const CT* V = reinterpret_cast<const CT*>(p.v);
   const int* pt = p.st.page_table + b * p.st.pages_per_row;
   auto row_off = [&](int pos) -> size_t {
     if (p.paged) return ((size_t)pt[pos / kPage] * kPage + (pos % kPage)) * p.ldkv + h * dh;
@@ -264,7 +265,7 @@ __global__ void __launch_bounds__(128) attention_kernel(AttnParams p) {
     const int pos = c0 + lane;
     float s = -INFINITY;
     if (pos < limit) {
-      const AT* kr = K + row_off(pos);
+      const CT* kr = K + row_off(pos);
       float dot = 0.f;
       for (int c = 0; c < dh; c += 8) {
         float kv[8];
@@ -283,7 +284,7 @@ __global__ void __launch_bounds__(128) attention_kernel(AttnParams p) {
     const int nk = min(32, limit - c0);
     for (int jj = 0; jj < nk; ++jj) {
       const float pw = __shfl_sync(0xffffffffu, pj, jj);
-      const AT* vr = V + row_off(c0 + jj);
+      const CT* vr = V + row_off(c0 + jj);
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
         const int c = lane + 32 * t;
@@ -292,12 +293,12 @@ __global__ void __launch_bounds__(128) attention_kernel(AttnParams p) {
     }
     m_run = m_new;
   }
-  AT* o = reinterpret_cast<AT*>(p.out) + (long long)r * p.ldo + h * dh;
+  QT* o = reinterpret_cast<QT*>(p.out) + (long long)r * p.ldo + h * dh;
   const float inv = 1.f / l_run;
 #pragma unroll
   for (int t = 0; t < 4; ++t) {
     const int c = lane + 32 * t;
-    if (c < dh) o[c] = from_f<AT>(acc[t] * inv);
+    if (c < dh) o[c] = from_f<QT>(acc[t] * inv);
   }
 }
 
@@ -459,7 +460,7 @@ __global__ void verify_commit_kernel(VerifyParams p) {
       if (!fin) atomicOr(&any_open, 1);
       atomicAdd((unsigned long long*)&p.st.stats[0], 1ull);
       atomicAdd((unsigned long long*)&p.st.stats[1], 1ull);
-      atomicAdd((unsigned long long*)&p.st.stats[3 + 1], 1ull);
+      atomicAdd((unsigned long long*)&p.st.stats[4 + 1], 1ull);
     } else {
       // longest prefix of the block that the base model would have produced itself:
       // proposal i+1 is checked against head 1 at the position of proposal i
@@ -481,12 +482,12 @@ __global__ void verify_commit_kernel(VerifyParams p) {
       if (!fin) atomicOr(&any_open, 1);
       atomicAdd((unsigned long long*)&p.st.stats[0], 1ull);
       atomicAdd((unsigned long long*)&p.st.stats[1], (unsigned long long)khat);
-      atomicAdd((unsigned long long*)&p.st.stats[3 + khat], 1ull);
+      atomicAdd((unsigned long long*)&p.st.stats[4 + khat], 1ull);
     }
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    if (p.mode != kModePrime) p.st.stats[2] += 1;
+    p.st.stats[p.mode == kModePrime ? 3 : 2] += 1;
     if (!any_open) *p.st.all_done = 1;
   }
 }
@@ -509,7 +510,7 @@ __global__ void reset_rows_kernel(ResetParams p) {
   if (threadIdx.x == 0) {
     *p.st.all_done = 0;
     *p.st.error = 0;
-    for (int i = 0; i < 3 + kMaxK + 1; ++i) p.st.stats[i] = 0;
+    for (int i = 0; i < 4 + kMaxK + 1; ++i) p.st.stats[i] = 0;
   }
 }
 
