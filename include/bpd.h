@@ -186,6 +186,25 @@ int bpd_op_vocab_argmax(const void* x, const void* w, int rows, int d, int vocab
                         void* scratch, size_t scratch_bytes, int32_t* out_idx, float* out_val,
                         void* cuda_stream);
 
+/* The same top-1 for callers that cannot hand over a workspace and must not
+ * trigger a device allocation: code running under a framework that has already
+ * claimed the whole GPU for its own pool, a serving loop that cannot afford the
+ * device-wide synchronisation an allocation may cause, or a plug-in callback
+ * that is only allowed to enqueue work.  (The paper has no counterpart; this is
+ * a deployment convenience.)  The cross-CTA reduction workspace is a fixed
+ * 512 KiB array inside the library image, resident on every GPU that loads the
+ * library until the process exits.  Limits: rows <= 256, vocab <= 65536,
+ * d <= 1024 and a multiple of 8; larger sizes return BPD_E_NOMEM and leave the
+ * outputs untouched.  Arguments as bpd_op_vocab_argmax, minus the scratch.
+ * The call performs no cudaMalloc/cudaFree and uses no allocating library.
+ * The first call on each device looks the array's device address up (with that
+ * device current); make that first call outside any stream capture.  All calls
+ * share the one array: the call clears the arrival counters it needs, but two
+ * calls whose kernels may overlap on the GPU (different streams, or different
+ * host threads) race on it -- keep them on one stream or serialise them. */
+int bpd_op_vocab_argmax_noalloc(const void* x, const void* w, int rows, int d, int vocab, int dtype,
+                                int32_t* out_idx, float* out_val, void* cuda_stream);
+
 /* y[r][n] = act(sum_c x[r][c] * w[n][c] + bias[n]); the projection used by every
  * layer.  x: device [rows, in_f] `dtype`; w: device [out_f, in_f] `dtype`; bias:
  * device [out_f] `dtype` or NULL; y: device [rows, out_f] float32; relu != 0

@@ -6,7 +6,7 @@
 build module can be imported before the library exists).  There is no CPU
 fallback: touching any binding name without a built library raises.
 """
-_BINDING_NAMES = ("BpdError", "Model", "Session", "Stats", "bpd_op_linear", "bpd_op_vocab_argmax",
+_BINDING_NAMES = ("BpdError", "Model", "Session", "Stats", "bpd_op_linear", "bpd_op_vocab_argmax", "bpd_op_vocab_argmax_noalloc",
                   "bpd_kernel_launches", "bpd_query_sizes", "lib", "EXPORTED")
 
 

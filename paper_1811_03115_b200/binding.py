@@ -65,6 +65,7 @@ _SIGS = {
     "bpd_fetch_output": (_i, [_vp, _i, _vp, _vp, C.POINTER(bpd_stats)]),
     "bpd_op_vocab_argmax_scratch_bytes": (_sz, [_i, _i, _i, _i]),
     "bpd_op_vocab_argmax": (_i, [_vp, _vp, _i, _i, _i, _i, _vp, _sz, _vp, _vp, _vp]),
+    "bpd_op_vocab_argmax_noalloc": (_i, [_vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp]),
     "bpd_op_linear_scratch_bytes": (_sz, [_i, _i, _i, _i]),
     "bpd_op_linear": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _sz, _vp, _vp]),
 }
@@ -265,6 +266,19 @@ def bpd_op_vocab_argmax(x, w, want_val: bool = False):
     _check(lib.bpd_op_vocab_argmax(x.data_ptr(), w.data_ptr(), rows, d, vocab, dtype, scratch.data_ptr(), nbytes,
                                    idx.data_ptr(), None if val is None else val.data_ptr(), _stream()))
     return (idx, val) if want_val else idx
+
+
+def bpd_op_vocab_argmax_noalloc(x, w, out_idx, out_val=None):
+    """Top-1 of x w^T using the library's built-in workspace: nothing is allocated
+    here or in the library, the caller passes the outputs (int32 [rows] and,
+    optionally, float32 [rows] CUDA tensors).  For callers that cannot allocate:
+    see include/bpd.h for the limits and the sharing rule."""
+    import torch
+    rows, d = x.shape
+    dtype = 0 if x.dtype == torch.float32 else 1
+    _check(lib.bpd_op_vocab_argmax_noalloc(x.data_ptr(), w.data_ptr(), rows, d, w.shape[0], dtype,
+                                           out_idx.data_ptr(), None if out_val is None else out_val.data_ptr(),
+                                           _stream()))
 
 
 def bpd_op_linear(x, w, bias=None, relu: bool = False):

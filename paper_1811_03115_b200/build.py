@@ -8,7 +8,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB_PATH = os.path.join(HERE, "libbpd.so")
-SOURCES = ["bpd.cu"]
+SOURCES = ["bpd.cu", "noalloc.cu"]
 
 
 def _nvcc() -> str:

@@ -429,7 +429,7 @@ struct VerifyParams {
   int max_new, eos;
 };
 
-__global__ void verify_commit_kernel(VerifyParams p) {
+static __global__ void verify_commit_kernel(VerifyParams p) {
   if (*p.st.all_done) return;
   __shared__ int any_open;
   if (threadIdx.x == 0) any_open = 0;
@@ -497,7 +497,7 @@ struct ResetParams {
   int B, ppr;
   const int* src_len;
 };
-__global__ void reset_rows_kernel(ResetParams p) {
+static __global__ void reset_rows_kernel(ResetParams p) {
   const int b = threadIdx.x;
   if (b < p.B) {
     p.st.len[b] = 0;
