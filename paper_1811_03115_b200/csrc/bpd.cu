@@ -1,6 +1,7 @@
 // C ABI of the blockwise-parallel-decoding library: blob parsing, buffer
 // planning, the encoder, the decoder pass and the decode loops.
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -9,6 +10,7 @@
 
 #include "host.hpp"
 #include "kernels_simt.cuh"
+#include "tc_host.hpp"
 
 namespace bpd {
 
@@ -150,15 +152,40 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
   int* src_dev = a.take<int>(E);
   int* tail_dev = a.take<int>((size_t)B * kMaxK);
   int* plan_dev = a.take<int>((size_t)B * max_tgt * (kMaxK - 1));
-  const size_t tiles = ceil_div(c.V, kVocTile);
+  const size_t tiles = std::max(ceil_div(c.V, kVocTile), ceil_div(c.V, tc::kBM));
   float* part_val = a.take<float>(tiles * R2);
   int* part_idx = a.take<int>(tiles * R2);
   unsigned* counters = a.take<unsigned>(ceil_div((int)R2, kRC) + 1);
+  // split-K workspace of the tensor-core projections: the largest any launch of this session can need
+  size_t ws = 0, ncnt = 1;
+  if (c.dtype == 1) {
+    auto need = [&](int N, int K, size_t T, int z) {
+      ws = std::max(ws, tc::ws_floats(N, K, (int)T, z));
+      ncnt = std::max(ncnt, tc::counters_needed(N, (int)T, z));
+    };
+    const int dd = c.d, ff = c.d_ff, fh = c.d_hidden, km = c.k_model;
+    for (size_t T : {Rmax, E}) {
+      need(3 * dd, dd, T, 1); need(dd, dd, T, 1); need(ff, dd, T, 1); need(dd, ff, T, 1); need(2 * dd, dd, T, 1);
+    }
+    for (int kh = 1; kh <= km; ++kh) {
+      need(kh * fh, dd, Rmax, 1); need(km * fh, dd, Rmax, 1);
+      need(kh * dd, km * fh, Rmax, 1);
+      need(dd, fh, Rmax, kh);
+    }
+    need(c.V, dd, R2, 1);
+  }
+  float* tc_ws = a.take<float>(ws);
+  unsigned* tc_counters = a.take<unsigned>(ncnt);
+  unsigned* tc_done = a.take<unsigned>(1);
   if (s) {
     s->x = x; s->h_f32 = h_f32; s->xn = xn; s->qbuf = qbuf; s->attn = attn; s->ffh = ffh; s->u = u; s->o = o;
     s->crosskv = crosskv; s->kcache = kc; s->vcache = vc; s->st = st; s->src_dev = src_dev;
     s->tail_dev = tail_dev; s->plan_dev = plan_dev; s->part_val = part_val; s->part_idx = part_idx;
-    s->counters = counters; s->ppr = ppr;
+    s->counters = counters; s->ppr = ppr; s->part_elems = tiles * R2;
+    s->tc_ws = tc_ws; s->tc_ws_floats = ws; s->tc_counters = tc_counters; s->tc_n_counters = ncnt; s->tc_done = tc_done;
+    s->pl_xn = (long long)(Rall * d); s->pl_attn = (long long)(Rall * d); s->pl_ffh = (long long)(Rall * c.d_ff);
+    s->pl_u = (long long)(Rmax * c.k_model * c.d_hidden); s->pl_o = (long long)(R2 * d);
+    s->rows_all = (int)Rall; s->rows_dec = (int)Rmax; s->rows_head = (int)R2;
   }
   return align_up(a.off);
 }
@@ -185,8 +212,8 @@ static LinearParams lin(const void* x, long long ldx, const void* w, int K, int 
 
 template <typename WT, typename AT>
 static void launch_ln(const float* x, const void* g, const void* b, void* y, float* y32, int rows, int d, float eps,
-                      const int* all_done, cudaStream_t st) {
-  LnParams p{x, g, b, y, y32, rows, d, eps, all_done};
+                      const int* all_done, cudaStream_t st, long long plane = 0) {
+  LnParams p{x, g, b, y, plane, y32, rows, d, eps, all_done};
   layernorm_kernel<WT, AT><<<ceil_div(rows, 4), 128, 0, st>>>(p);
   ++g_launches;
 }
@@ -347,7 +374,170 @@ static int run_pass(bpd_session* s, const PassArgs& a) {
   return BPD_OK;
 }
 
+// ------------------------------------------------------------------ tensor-core path (bf16 models)
+static tc::Scratch tc_scratch(bpd_session* s) {
+  tc::Scratch sc;
+  sc.ws = s->tc_ws; sc.ws_floats = s->tc_ws_floats; sc.tile_counters = s->tc_counters; sc.n_counters = s->tc_n_counters;
+  sc.done_counter = s->tc_done; sc.part_val = s->part_val; sc.part_idx = s->part_idx; sc.part_elems = s->part_elems;
+  sc.error = s->st.error;
+  return sc;
+}
+
+static tc::TcParams tc_params(const void* bias, int relu, const int* all_done) {
+  tc::TcParams p;
+  memset(&p, 0, sizeof(p));
+  p.bias = static_cast<const bf16*>(bias); p.relu = relu; p.all_done = all_done;
+  return p;
+}
+
+#define BPD_TRY(expr) do { int rc__ = (expr); if (rc__) return rc__; } while (0)
+
+static int run_encoder_tc(bpd_session* s) {
+  const bpd_model* m = s->m;
+  const Config& c = m->cfg;
+  cudaStream_t st = s->stream;
+  const int E = s->B * s->max_src, d = c.d, f = c.d_ff;
+  const tc::Scratch sc = tc_scratch(s);
+  EmbedParams ep;
+  memset(&ep, 0, sizeof(ep));
+  ep.table = m->src_embed; ep.inv_freq = m->inv_freq; ep.x = s->x; ep.rows = E; ep.rows_per_b = s->max_src;
+  ep.d = d; ep.vocab = c.V; ep.st = s->st; ep.src = s->src_dev;
+  embed_kernel<bf16><<<E, 128, 0, st>>>(ep);
+  ++g_launches;
+  const tc::Operands xn{nullptr, 0, s->xn, s->pl_xn, d, s->rows_all, d};
+  const tc::Operands at{nullptr, 0, s->attn, s->pl_attn, d, s->rows_all, d};
+  const tc::Operands fh{nullptr, 0, s->ffh, s->pl_ffh, f, s->rows_all, f};
+  auto with_w = [](tc::Operands o, const void* w, int rows) { o.w = w; o.w_rows = rows; return o; };
+  for (int l = 0; l < c.n_enc; ++l) {
+    const EncLayer& L = m->enc[l];
+    launch_ln<bf16, float>(s->x, L.ln1g, L.ln1b, s->xn, nullptr, E, d, c.eps, nullptr, st, s->pl_xn);
+    tc::TcParams pq = tc_params(nullptr, 0, nullptr);
+    pq.out_f32 = static_cast<float*>(s->qbuf); pq.ldo = 3 * d;
+    BPD_TRY(tc::launch<tc::kTcF32>(with_w(xn, L.wqkv, 3 * d), 3 * d, d, E, pq, sc, st)); ++g_launches;
+    AttnParams ap;
+    memset(&ap, 0, sizeof(ap));
+    ap.q = s->qbuf; ap.ldq = 3 * d; ap.out = s->attn; ap.ldo = d; ap.out_plane = s->pl_attn; ap.rows = E;
+    ap.rows_per_b = s->max_src; ap.H = c.H; ap.dh = d / c.H; ap.causal = 0; ap.limit_b = s->st.src_len;
+    ap.k = static_cast<float*>(s->qbuf) + d; ap.v = static_cast<float*>(s->qbuf) + 2 * d;
+    ap.ldkv = 3 * d; ap.bstride = (long long)s->max_src * 3 * d; ap.paged = 0; ap.st = s->st;
+    ap.scale = 1.0f / sqrtf((float)ap.dh);
+    attention_kernel<float, float><<<ceil_div(E * c.H, 4), 128, 0, st>>>(ap);
+    ++g_launches;
+    tc::TcParams po = tc_params(nullptr, 0, nullptr);
+    po.out_f32 = s->x; po.ldo = d;
+    BPD_TRY(tc::launch<tc::kTcResidual>(with_w(at, L.wo, d), d, d, E, po, sc, st)); ++g_launches;
+    launch_ln<bf16, float>(s->x, L.ln2g, L.ln2b, s->xn, nullptr, E, d, c.eps, nullptr, st, s->pl_xn);
+    tc::TcParams p1 = tc_params(L.b1, 1, nullptr);
+    p1.out_hi = static_cast<bf16*>(s->ffh); p1.plane = s->pl_ffh; p1.ldo = f;
+    BPD_TRY(tc::launch<tc::kTcPlanes>(with_w(xn, L.w1, f), f, d, E, p1, sc, st)); ++g_launches;
+    tc::TcParams p2 = tc_params(L.b2, 0, nullptr);
+    p2.out_f32 = s->x; p2.ldo = d;
+    BPD_TRY(tc::launch<tc::kTcResidual>(with_w(fh, L.w2, d), d, f, E, p2, sc, st)); ++g_launches;
+  }
+  launch_ln<bf16, float>(s->x, m->enc_lnf_g, m->enc_lnf_b, s->xn, nullptr, E, d, c.eps, nullptr, st, s->pl_xn);
+  for (int l = 0; l < c.n_dec; ++l) {
+    tc::TcParams pk = tc_params(nullptr, 0, nullptr);
+    pk.out_f32 = static_cast<float*>(s->crosskv[l]); pk.ldo = 2 * d;
+    BPD_TRY(tc::launch<tc::kTcF32>(with_w(xn, m->dec[l].cwkv, 2 * d), 2 * d, d, E, pk, sc, st)); ++g_launches;
+  }
+  BPD_CUDA(cudaGetLastError());
+  return BPD_OK;
+}
+
+static int run_pass_tc(bpd_session* s, const PassArgs& a) {
+  const bpd_model* m = s->m;
+  const Config& c = m->cfg;
+  cudaStream_t st = s->stream;
+  const int d = c.d, f = c.d_ff, R = s->B * a.kcur, R2 = R * a.kh;
+  const int* done = s->st.all_done;
+  const tc::Scratch sc = tc_scratch(s);
+  prof_mark(s, kProfLayers, 0);
+  EmbedParams ep;
+  memset(&ep, 0, sizeof(ep));
+  ep.table = m->tgt_embed; ep.inv_freq = m->inv_freq; ep.x = s->x; ep.rows = R; ep.rows_per_b = a.kcur;
+  ep.d = d; ep.vocab = c.V; ep.st = s->st; ep.forced = a.forced; ep.forced_rows = a.forced_rows;
+  ep.kforced = a.kforced; ep.src = nullptr; ep.all_done = done;
+  embed_kernel<bf16><<<R, 128, 0, st>>>(ep);
+  ++g_launches;
+  const tc::Operands xn{nullptr, 0, s->xn, s->pl_xn, d, s->rows_all, d};
+  const tc::Operands at{nullptr, 0, s->attn, s->pl_attn, d, s->rows_all, d};
+  const tc::Operands fx{nullptr, 0, s->ffh, s->pl_ffh, f, s->rows_all, f};
+  auto with_w = [](tc::Operands o, const void* w, int rows) { o.w = w; o.w_rows = rows; return o; };
+  for (int l = 0; l < c.n_dec; ++l) {
+    const DecLayer& L = m->dec[l];
+    launch_ln<bf16, float>(s->x, L.ln1g, L.ln1b, s->xn, nullptr, R, d, c.eps, done, st, s->pl_xn);
+    tc::TcParams pq = tc_params(nullptr, 0, done);
+    pq.out_f32 = static_cast<float*>(s->qbuf); pq.ldo = d; pq.d = d;
+    pq.kcache = static_cast<bf16*>(s->kcache[l]); pq.vcache = static_cast<bf16*>(s->vcache[l]);
+    pq.st = s->st; pq.rows_per_b = a.kcur;
+    BPD_TRY(tc::launch<tc::kTcQkv>(with_w(xn, L.wqkv, 3 * d), 3 * d, d, R, pq, sc, st)); ++g_launches;
+    AttnParams ap;
+    memset(&ap, 0, sizeof(ap));
+    ap.q = s->qbuf; ap.ldq = d; ap.out = s->attn; ap.ldo = d; ap.out_plane = s->pl_attn; ap.rows = R;
+    ap.rows_per_b = a.kcur; ap.H = c.H; ap.dh = d / c.H; ap.causal = 1; ap.k = s->kcache[l]; ap.v = s->vcache[l];
+    ap.ldkv = d; ap.paged = 1; ap.st = s->st; ap.scale = 1.0f / sqrtf((float)ap.dh); ap.all_done = done;
+    attention_kernel<float, bf16><<<ceil_div(R * c.H, 4), 128, 0, st>>>(ap);
+    ++g_launches;
+    tc::TcParams po = tc_params(nullptr, 0, done);
+    po.out_f32 = s->x; po.ldo = d;
+    BPD_TRY(tc::launch<tc::kTcResidual>(with_w(at, L.wo, d), d, d, R, po, sc, st)); ++g_launches;
+    launch_ln<bf16, float>(s->x, L.ln2g, L.ln2b, s->xn, nullptr, R, d, c.eps, done, st, s->pl_xn);
+    tc::TcParams pc = tc_params(nullptr, 0, done);
+    pc.out_f32 = static_cast<float*>(s->qbuf); pc.ldo = d;
+    BPD_TRY(tc::launch<tc::kTcF32>(with_w(xn, L.cwq, d), d, d, R, pc, sc, st)); ++g_launches;
+    ap.causal = 0; ap.limit_b = s->st.src_len; ap.k = s->crosskv[l]; ap.v = static_cast<float*>(s->crosskv[l]) + d;
+    ap.ldkv = 2 * d; ap.bstride = (long long)s->max_src * 2 * d; ap.paged = 0;
+    attention_kernel<float, float><<<ceil_div(R * c.H, 4), 128, 0, st>>>(ap);
+    ++g_launches;
+    BPD_TRY(tc::launch<tc::kTcResidual>(with_w(at, L.cwo, d), d, d, R, po, sc, st)); ++g_launches;
+    launch_ln<bf16, float>(s->x, L.ln3g, L.ln3b, s->xn, nullptr, R, d, c.eps, done, st, s->pl_xn);
+    tc::TcParams p1 = tc_params(L.b1, 1, done);
+    p1.out_hi = static_cast<bf16*>(s->ffh); p1.plane = s->pl_ffh; p1.ldo = f;
+    BPD_TRY(tc::launch<tc::kTcPlanes>(with_w(xn, L.w1, f), f, d, R, p1, sc, st)); ++g_launches;
+    tc::TcParams p2 = tc_params(L.b2, 0, done);
+    p2.out_f32 = s->x; p2.ldo = d;
+    BPD_TRY(tc::launch<tc::kTcResidual>(with_w(fx, L.w2, d), d, f, R, p2, sc, st)); ++g_launches;
+  }
+  launch_ln<bf16, float>(s->x, m->dec_lnf_g, m->dec_lnf_b, s->xn, s->h_f32, R, d, c.eps, done, st, s->pl_xn);
+  prof_mark(s, kProfLayers, 1);
+  // proposal heads
+  const int fhd = c.d_hidden, km = c.k_model;
+  const int ldu = km * fhd;
+  const int hid = (c.head_layout == 0) ? km * fhd : a.kh * fhd;
+  prof_mark(s, kProfHeadW1, 0);
+  tc::TcParams pu = tc_params(m->head_b1, 1, done);
+  pu.out_hi = static_cast<bf16*>(s->u); pu.plane = s->pl_u; pu.ldo = ldu;
+  BPD_TRY(tc::launch<tc::kTcPlanes>(with_w(xn, m->head_w1, km * fhd), hid, d, R, pu, sc, st)); ++g_launches;
+  prof_mark(s, kProfHeadW1, 1);
+  prof_mark(s, kProfHeadW2, 0);
+  tc::Operands uo{m->head_w2, km * d, s->u, s->pl_u, ldu, s->rows_dec, ldu};
+  tc::TcParams ph = tc_params(m->head_b2, 0, done);
+  ph.out_hi = static_cast<bf16*>(s->o); ph.plane = s->pl_o; ph.ldo = (long long)a.kh * d;
+  ph.h = s->h_f32; ph.d = d; ph.head_identity = c.p1_identity;
+  if (c.head_layout == 0) {
+    BPD_TRY(tc::launch<tc::kTcHeadOut>(uo, a.kh * d, km * fhd, R, ph, sc, st));
+  } else {
+    ph.zofs_n = d;
+    BPD_TRY(tc::launch<tc::kTcHeadOut>(uo, d, fhd, R, ph, sc, st, a.kh, d, fhd));
+  }
+  ++g_launches;
+  prof_mark(s, kProfHeadW2, 1);
+  prof_mark(s, kProfVocab, 0);
+  tc::Operands oo{m->out_proj, c.V, s->o, s->pl_o, d, s->rows_head, d};
+  tc::TcParams pv = tc_params(nullptr, 0, done);
+  pv.out_idx = s->st.table; pv.logits = a.logits_dump;
+  BPD_TRY(tc::launch<tc::kTcArgmax>(oo, c.V, d, R2, pv, sc, st)); ++g_launches;
+  prof_mark(s, kProfVocab, 1);
+  VerifyParams vp{s->st, s->B, a.kcur, a.kh, a.knext, a.mode, a.max_new, a.eos};
+  verify_commit_kernel<<<1, 32 * ceil_div(s->B, 32), 0, st>>>(vp);
+  ++g_launches;
+  BPD_CUDA(cudaGetLastError());
+  s->invocations += 1;
+  return BPD_OK;
+}
+
 static int dispatch_pass(bpd_session* s, const PassArgs& a) {
+  if (s->tc) return run_pass_tc(s, a);
   return s->m->cfg.dtype == 0 ? run_pass<float>(s, a) : run_pass<bf16>(s, a);
 }
 
@@ -357,6 +547,7 @@ static int check_device_error(bpd_session* s) {
   BPD_CUDA(cudaStreamSynchronize(s->stream));
   err = s->pinned[64];
   if (err == 1) return fail(BPD_E_INVALID, "a token id outside the vocabulary reached the decoder");
+  if (err >= 101 && err <= 103) return fail(BPD_E_TIMEOUT, "a bounded wait inside the projection kernel expired (code %d)", err);
   if (err != 0) return fail(BPD_E_CUDA, "device-side error word %d", err);
   return BPD_OK;
 }
@@ -488,6 +679,7 @@ int bpd_session_create(const bpd_model* model, int batch, int max_src, int max_t
   s->m = model; s->B = batch; s->max_src = max_src; s->max_tgt = max_tgt;
   s->base = static_cast<char*>(dev_session_buf); s->bytes = dev_bytes; s->stream = (cudaStream_t)cuda_stream;
   s->profiling = 0;
+  s->tc = (model->cfg.dtype == 1 && !getenv("BPD_DISABLE_TC")) ? 1 : 0;
   s->phase = kPhaseCreated; s->plan_len = 0; s->plan_k = 0; s->invocations = 0; s->pinned = nullptr;
   plan_session(model->cfg, batch, max_src, max_tgt, s->base, s);
   // page table: row b's p-th page is physical page p*B + b (rows interleaved in the pool)
@@ -543,7 +735,7 @@ int bpd_encode(bpd_session* s, const int32_t* src_ids, const int32_t* src_len) {
   reset_rows_kernel<<<1, 32 * ceil_div(B, 32), 0, s->stream>>>(rp);
   ++g_launches;
   BPD_CUDA(cudaStreamSynchronize(s->stream));   // host vectors go out of scope
-  int rc = (c.dtype == 0) ? run_encoder<float>(s) : run_encoder<bf16>(s);
+  int rc = s->tc ? run_encoder_tc(s) : ((c.dtype == 0) ? run_encoder<float>(s) : run_encoder<bf16>(s));
   if (rc) return rc;
   s->phase = kPhaseEncoded; s->plan_len = 0; s->plan_k = 0; s->invocations = 0;
   return BPD_OK;
@@ -734,9 +926,42 @@ int bpd_fetch_output(bpd_session* s, int max_new, int32_t* out_ids, int32_t* out
 }
 
 // ------------------------------------------------------------------ single operators
+// Scratch layout of the bf16 (tensor-core) operators: a zero "lo" plane for the caller's single-plane bf16
+// activations, the split-K workspace, tile counters, the top-1 merge counter and partials, an error word.
+struct OpScratch {
+  size_t zero_off, ws_off, cnt_off, done_off, pv_off, pi_off, err_off, total;
+  size_t ws_floats, n_counters, part_elems;
+};
+static OpScratch op_scratch_layout(int rows, int in_f, int out_f) {
+  OpScratch o;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + bytes); return at; };
+  o.ws_floats = tc::ws_floats(out_f, in_f, rows, 1);
+  o.n_counters = tc::counters_needed(out_f, rows, 1);
+  o.part_elems = (size_t)ceil_div(out_f, tc::kBM) * rows;
+  o.zero_off = take((size_t)rows * in_f * sizeof(bf16));
+  o.ws_off = take(o.ws_floats * sizeof(float));
+  o.cnt_off = take(o.n_counters * sizeof(unsigned));
+  o.done_off = take(sizeof(unsigned));
+  o.pv_off = take(o.part_elems * sizeof(float));
+  o.pi_off = take(o.part_elems * sizeof(int));
+  o.err_off = take(sizeof(int));
+  o.total = off;
+  return o;
+}
+static bool op_use_tc(int dtype) { return dtype == 1 && !getenv("BPD_DISABLE_TC"); }
+
+static int op_tc_finish(char* scratch, const OpScratch& L, cudaStream_t st) {
+  int err = 0;
+  BPD_CUDA(cudaMemcpyAsync(&err, scratch + L.err_off, sizeof(int), cudaMemcpyDeviceToHost, st));
+  BPD_CUDA(cudaStreamSynchronize(st));
+  if (err) return fail(BPD_E_TIMEOUT, "a bounded wait inside the projection kernel expired (code %d)", err);
+  return BPD_OK;
+}
+
 size_t bpd_op_vocab_argmax_scratch_bytes(int rows, int d, int vocab, int dtype) {
-  (void)d; (void)dtype;
-  if (rows < 1 || vocab < 1) return 0;
+  if (rows < 1 || vocab < 1 || d < 1) return 0;
+  if (op_use_tc(dtype)) return op_scratch_layout(rows, d, vocab).total;
   const size_t tiles = ceil_div(vocab, kVocTile);
   return align_up(tiles * rows * sizeof(float)) + align_up(tiles * rows * sizeof(int)) +
          align_up((ceil_div(rows, kRC) + 1) * sizeof(unsigned));
@@ -750,8 +975,24 @@ int bpd_op_vocab_argmax(const void* x, const void* w, int rows, int d, int vocab
   if ((uintptr_t)x % 16 || (uintptr_t)w % 16 || (uintptr_t)scratch % 256) return fail(BPD_E_INVALID, "misaligned pointer");
   if (scratch_bytes < bpd_op_vocab_argmax_scratch_bytes(rows, d, vocab, dtype)) return fail(BPD_E_NOMEM, "scratch too small");
   cudaStream_t st = (cudaStream_t)cuda_stream;
-  const size_t tiles = ceil_div(vocab, kVocTile);
   char* p = static_cast<char*>(scratch);
+  if (op_use_tc(dtype)) {
+    const OpScratch L = op_scratch_layout(rows, d, vocab);
+    BPD_CUDA(cudaMemsetAsync(p, 0, L.total, st));
+    tc::Scratch sc{reinterpret_cast<float*>(p + L.ws_off), L.ws_floats, reinterpret_cast<unsigned*>(p + L.cnt_off),
+                   L.n_counters, reinterpret_cast<unsigned*>(p + L.done_off), reinterpret_cast<float*>(p + L.pv_off),
+                   reinterpret_cast<int*>(p + L.pi_off), L.part_elems, reinterpret_cast<int*>(p + L.err_off)};
+    const long long plane = (reinterpret_cast<const bf16*>(p + L.zero_off) - static_cast<const bf16*>(x));
+    tc::Operands op{w, vocab, x, plane, d, rows, d};
+    tc::TcParams tp;
+    memset(&tp, 0, sizeof(tp));
+    tp.out_idx = out_idx; tp.out_val = out_val;
+    int rc = tc::launch<tc::kTcArgmax>(op, vocab, d, rows, tp, sc, st);
+    if (rc) return rc;
+    ++g_launches;
+    return op_tc_finish(p, L, st);
+  }
+  const size_t tiles = ceil_div(vocab, kVocTile);
   float* pv = reinterpret_cast<float*>(p);
   p += align_up(tiles * rows * sizeof(float));
   int* pi = reinterpret_cast<int*>(p);
@@ -765,18 +1006,37 @@ int bpd_op_vocab_argmax(const void* x, const void* w, int rows, int d, int vocab
 }
 
 size_t bpd_op_linear_scratch_bytes(int rows, int in_f, int out_f, int dtype) {
-  (void)rows; (void)in_f; (void)out_f; (void)dtype;
+  if (rows < 1 || in_f < 1 || out_f < 1) return 0;
+  if (op_use_tc(dtype)) return op_scratch_layout(rows, in_f, out_f).total;
   return 256;
 }
 
 int bpd_op_linear(const void* x, const void* w, const void* bias, int rows, int in_f, int out_f, int dtype, int relu,
                   void* scratch, size_t scratch_bytes, float* y, void* cuda_stream) {
-  (void)scratch; (void)scratch_bytes;
   if (!x || !w || !y) return fail(BPD_E_INVALID, "null argument");
   if (rows < 1 || out_f < 1 || in_f < 8 || in_f % 8) return fail(BPD_E_SHAPE, "rows/in_f/out_f out of range (in_f must be a multiple of 8)");
   if (dtype != 0 && dtype != 1) return fail(BPD_E_INVALID, "unknown dtype %d", dtype);
   if ((uintptr_t)x % 16 || (uintptr_t)w % 16) return fail(BPD_E_INVALID, "misaligned pointer");
   cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (op_use_tc(dtype)) {
+    if (!scratch || (uintptr_t)scratch % 256) return fail(BPD_E_INVALID, "scratch is null or misaligned");
+    const OpScratch L = op_scratch_layout(rows, in_f, out_f);
+    if (scratch_bytes < L.total) return fail(BPD_E_NOMEM, "scratch too small");
+    char* p = static_cast<char*>(scratch);
+    BPD_CUDA(cudaMemsetAsync(p, 0, L.total, st));
+    tc::Scratch sc{reinterpret_cast<float*>(p + L.ws_off), L.ws_floats, reinterpret_cast<unsigned*>(p + L.cnt_off),
+                   L.n_counters, reinterpret_cast<unsigned*>(p + L.done_off), reinterpret_cast<float*>(p + L.pv_off),
+                   reinterpret_cast<int*>(p + L.pi_off), L.part_elems, reinterpret_cast<int*>(p + L.err_off)};
+    const long long plane = (reinterpret_cast<const bf16*>(p + L.zero_off) - static_cast<const bf16*>(x));
+    tc::Operands op{w, out_f, x, plane, in_f, rows, in_f};
+    tc::TcParams tp;
+    memset(&tp, 0, sizeof(tp));
+    tp.bias = static_cast<const bf16*>(bias); tp.relu = relu; tp.out_f32 = y; tp.ldo = out_f;
+    int rc = tc::launch<tc::kTcF32>(op, out_f, in_f, rows, tp, sc, st);
+    if (rc) return rc;
+    ++g_launches;
+    return op_tc_finish(p, L, st);
+  }
   LinearParams p = lin(x, in_f, w, in_f, out_f, bias, rows, y, out_f, relu, nullptr);
   if (dtype == 0) launch_linear<float, float, kEpiStoreF32>(p, 1, st);
   else launch_linear<bf16, bf16, kEpiStoreF32>(p, 1, st);

@@ -1,0 +1,412 @@
+// Weight-streaming projection on the 5th-generation tensor cores (sm_100a):
+//   y[t][n] = sum_c x[t][c] * w[n][c]        t < T tokens (few), n < N features (many)
+// The weight matrix is the MMA's M operand (128 features per tile), the tokens are
+// its N operand.  Weights (bf16, [N, K] row-major) and activations (two bf16
+// planes hi + lo that together carry an fp32 value, [rows, K] row-major) are
+// brought into 128-byte-swizzled shared memory by TMA; one elected thread issues
+// tcgen05.mma with the fp32 accumulator in tensor memory; four warps read it
+// back with tcgen05.ld and run the fused epilogue.  K can be split over CTAs
+// (grid.y): partial tiles go to a workspace and the CTA that arrives last for a
+// tile adds them in split order, so the summation order is fixed by (N, K) alone.
+//
+// Every wait on an mbarrier is bounded; on expiry the CTA records an error code,
+// skips its remaining work, waits (bounded) for copies in flight, frees its
+// tensor memory and returns.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace bpd {
+namespace tc {
+
+constexpr int kBM = 128;          // features per tile (MMA M)
+constexpr int kBK = 64;           // K elements per pipeline stage (128 bytes of bf16: one swizzle row)
+constexpr int kStages = 4;
+constexpr int kThreads = 192;     // warp 0: TMA, warp 1: MMA + tensor-memory allocation, warps 2-5: epilogue
+constexpr int kMaxBN = 128;       // tokens per CTA (MMA N), a multiple of 16
+constexpr unsigned long long kSpinCycles = 2000000000ull;   // about a second
+
+enum TcEpilogue {
+  kTcPlanes = 0,    // out planes (hi, lo) = split(act(v + bias))
+  kTcF32 = 1,       // out fp32 = act(v + bias)
+  kTcResidual = 2,  // x fp32 += v + bias
+  kTcQkv = 3,       // n < d: q fp32; else key / value (bf16) into the paged cache
+  kTcHeadOut = 4,   // out planes = split(v + bias + h[t][n mod d])
+  kTcArgmax = 5     // per-token top-1 over all features (two-level merge), optional logits dump
+};
+
+struct TcParams {
+  int T, N, K;                 // tokens in this launch, features, reduction length
+  int bn;                      // MMA N: T rounded up to 16 (per token tile)
+  int splits;                  // grid.y
+  int chunks_per_split;        // K chunks (of kBK) each split owns
+  const bf16* bias;            // [N] or null
+  int relu;
+  // outputs
+  bf16* out_hi; long long plane; long long ldo;   // planes: lo plane = hi + plane
+  float* out_f32;              // kTcF32 / kTcResidual / kTcQkv(q): [T, ldo]
+  const float* h; int d;       // kTcHeadOut residual; kTcQkv model width
+  int head_identity;
+  int zofs_n;                  // column offset of this z-slice inside the output row (block-diagonal heads)
+  bf16* kcache; bf16* vcache;  // kTcQkv
+  RowState st; int rows_per_b;
+  // split-K workspace
+  float* ws;                   // [z][tile][split][bn][128]
+  unsigned* tile_counters;     // [z][tiles]
+  // top-1
+  float* part_val; int* part_idx;   // [tiles][T]
+  unsigned* done_counter;           // [1]
+  int* out_idx; float* out_val; float* logits;
+  int* error;                  // device error word
+  const int* all_done;
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok;
+}
+// Bounded wait: false if the phase did not complete within about a second.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if ((unsigned long long)(clock64() - t0) > kSpinCycles) return false;
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 16 consecutive fp32 columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory operand descriptor: K-major rows of 128 bytes, 128-byte swizzle,
+// 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3ffff) >> 4);          // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                           // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;                 // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                           // descriptor version
+  d |= (uint64_t)2 << 61;                           // layout: 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128.
+__device__ __forceinline__ uint32_t instr_desc_bf16(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+}
+
+__device__ __forceinline__ void split_bf16(float v, bf16& hi, bf16& lo) {
+  hi = __float2bfloat16_rn(v);
+  lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+
+// Shared-memory footprint of one CTA.
+__host__ __device__ inline size_t stage_bytes(int bn) { return (size_t)kBM * 128 + 2 * (size_t)bn * 128; }
+__host__ __device__ inline size_t smem_bytes(int bn) { return kStages * stage_bytes(bn) + 1024 /*alignment*/ + 256; }
+
+// ---------------------------------------------------------------- final epilogue for one (feature, token)
+template <int EPI>
+__device__ __forceinline__ void tc_store(const TcParams& p, int z, int t, int n, float v) {
+  if (p.bias) v += __bfloat162float(p.bias[n + p.zofs_n * z]);
+  if (p.relu) v = fmaxf(v, 0.f);
+  if (EPI == kTcPlanes) {
+    bf16 hi, lo;
+    split_bf16(v, hi, lo);
+    const long long o = (long long)t * p.ldo + n + (long long)p.zofs_n * z;
+    p.out_hi[o] = hi;
+    p.out_hi[o + p.plane] = lo;
+  } else if (EPI == kTcF32) {
+    p.out_f32[(long long)t * p.ldo + n] = v;
+  } else if (EPI == kTcResidual) {
+    p.out_f32[(long long)t * p.ldo + n] += v;
+  } else if (EPI == kTcHeadOut) {
+    const int nz = n + p.zofs_n * z;
+    const float hv = p.h[(size_t)t * p.d + (n % p.d)];
+    v = (p.head_identity && nz < p.d) ? hv : v + hv;
+    bf16 hi, lo;
+    split_bf16(v, hi, lo);
+    const long long o = (long long)t * p.ldo + nz;
+    p.out_hi[o] = hi;
+    p.out_hi[o + p.plane] = lo;
+  } else if (EPI == kTcQkv) {
+    const int d = p.d;
+    if (n < d) {
+      p.out_f32[(long long)t * p.ldo + n] = v;
+    } else {
+      const int b = t / p.rows_per_b, i = t % p.rows_per_b;
+      const int pos = p.st.len[b] + i;
+      const int page = p.st.page_table[b * p.st.pages_per_row + pos / kPage];
+      const size_t slot = ((size_t)page * kPage + (pos % kPage)) * d;
+      if (n < 2 * d) p.kcache[slot + (n - d)] = __float2bfloat16_rn(v);
+      else p.vcache[slot + (n - 2 * d)] = __float2bfloat16_rn(v);
+    }
+  }
+}
+
+// ---------------------------------------------------------------- the kernel
+// grid = (feature tiles, K splits, z), z = token tile * zslices + slice (slices: block-diagonal heads).
+// tmA: weights [N, K]; tmBh / tmBl: activation planes [rows, K]; box = (64, 128) and (64, bn).
+template <int EPI>
+__global__ void __launch_bounds__(kThreads)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmBh,
+               const __grid_constant__ CUtensorMap tmBl, TcParams p, int zslices, int a_rows_per_slice,
+               int b_cols_per_slice) {
+  if (p.all_done && *p.all_done) return;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;      // swizzled tiles need 1024-byte alignment
+  uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
+  const int bn = p.bn;
+  const uint32_t stage_sz = (uint32_t)stage_bytes(bn);
+  const uint32_t bars = base + kStages * stage_sz;                   // full[kStages], empty[kStages], accum
+  volatile uint32_t* ctl = reinterpret_cast<volatile uint32_t*>(gen_base + kStages * stage_sz + 128);
+  // ctl[0] = tensor-memory base, ctl[1] = "this CTA reduces the tile", ctl[2] = "this CTA merges the top-1",
+  // ctl[3] = "the accumulator arrived"
+  __shared__ float s_val[4][kMaxBN];
+  __shared__ int s_idx[4][kMaxBN];
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tile = blockIdx.x, split = blockIdx.y;
+  const int ttile = blockIdx.z / zslices, slice = blockIdx.z % zslices;
+  const int t0 = ttile * bn;
+  const int nt = min(bn, p.T - t0);                                  // live tokens in this tile
+  const int total_chunks = (p.K + kBK - 1) / kBK;
+  const int c0 = split * p.chunks_per_split;
+  const int c1 = min(total_chunks, c0 + p.chunks_per_split);
+  const int nchunks = max(0, c1 - c0);
+  const uint32_t ncols = bn <= 32 ? 32u : (bn <= 64 ? 64u : 128u);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(bars + 8 * s, 1);
+      mbar_init(bars + 8 * (kStages + s), 1);
+    }
+    mbar_init(bars + 8 * 2 * kStages, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    ctl[1] = 0;
+    ctl[2] = 0;
+  }
+  if (warp == 1) tmem_alloc(base + kStages * stage_sz + 128, ncols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = ctl[0];
+  bool ok = true;
+
+  if (warp == 0 && lane == 0) {
+    // ---------------- TMA producer
+    const int a_row = slice * a_rows_per_slice + tile * kBM;
+    int issued = 0;
+    for (int it = 0; it < nchunks; ++it) {
+      const int s = it % kStages;
+      const uint32_t ph = (it / kStages) & 1;
+      if (!mbar_wait(bars + 8 * (kStages + s), ph ^ 1)) { ok = false; break; }
+      issued = it + 1;
+      const uint32_t full = bars + 8 * s;
+      const uint32_t sa = base + s * stage_sz;
+      mbar_expect_tx(full, stage_sz);
+      const int kx = (c0 + it) * kBK;
+      tma_load_2d(sa, &tmA, full, kx, a_row);
+      tma_load_2d(sa + kBM * 128, &tmBh, full, slice * b_cols_per_slice + kx, t0);
+      tma_load_2d(sa + kBM * 128 + bn * 128, &tmBl, full, slice * b_cols_per_slice + kx, t0);
+    }
+    if (!ok) {
+      atomicCAS(p.error, 0, 101);
+      // give the copies already issued a bounded chance to land before this CTA's shared memory goes away
+      for (int it = max(0, issued - kStages); it < issued; ++it) mbar_wait(bars + 8 * (it % kStages), (it / kStages) & 1);
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---------------- MMA issuer
+    const uint32_t idesc = instr_desc_bf16(bn);
+    for (int it = 0; it < nchunks; ++it) {
+      const int s = it % kStages;
+      const uint32_t ph = (it / kStages) & 1;
+      if (!mbar_wait(bars + 8 * s, ph)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t sa = base + s * stage_sz;
+#pragma unroll
+      for (int kk = 0; kk < kBK / 16; ++kk) {
+        const uint64_t ad = smem_desc_sw128(sa + kk * 32);
+        const uint64_t bh = smem_desc_sw128(sa + kBM * 128 + kk * 32);
+        const uint64_t bl = smem_desc_sw128(sa + kBM * 128 + bn * 128 + kk * 32);
+        umma_f16(tmem, ad, bh, idesc, (it > 0 || kk > 0) ? 1u : 0u);
+        umma_f16(tmem, ad, bl, idesc, 1u);
+      }
+      umma_commit(bars + 8 * (kStages + s));       // frees the stage once these MMAs have read it
+    }
+    umma_commit(bars + 8 * 2 * kStages);            // accumulator complete
+    if (!ok) atomicCAS(p.error, 0, 102);
+  } else if (warp >= 2) {
+    // ---------------- epilogue: thread = one feature row, registers = tokens
+    const int q = warp & 3;                          // tensor-memory lane quarter this warp may read
+    const int row = q * 32 + lane;
+    const int n = tile * kBM + row;                  // feature index within the slice
+    const int et = threadIdx.x - 64;                 // 0..127
+    // one thread waits for the accumulator; the other 127 learn the outcome through the named barrier
+    if (et == 0) {
+      bool done = true;
+      if (nchunks > 0) done = mbar_wait(bars + 8 * 2 * kStages, 0);
+      if (!done) atomicCAS(p.error, 0, 103);
+      ctl[3] = done ? 1u : 0u;
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    ok = (ctl[3] != 0);
+    tc_fence_after();
+    const int ntiles = gridDim.x;
+    const bool direct = (p.splits == 1);
+    float* wsz = p.ws + ((size_t)blockIdx.z * ntiles + tile) * p.splits * (size_t)bn * kBM;
+    if (ok) {
+      if (direct) {
+        for (int cb = 0; cb < bn; cb += 16) {
+          float v[16];
+          tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + cb, v);
+          if (EPI != kTcArgmax) {
+#pragma unroll
+            for (int c = 0; c < 16; ++c)
+              if (cb + c < nt && n < p.N) tc_store<EPI>(p, slice, t0 + cb + c, n, v[c]);
+          } else {
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+              float x = (n < p.N) ? v[c] : -INFINITY;
+              int ix = (n < p.N) ? n : 0x7fffffff;
+              if (p.logits && cb + c < nt && n < p.N) p.logits[(size_t)(t0 + cb + c) * p.N + n] = x;
+              warp_argmax(x, ix);
+              if (lane == 0) { s_val[q][cb + c] = x; s_idx[q][cb + c] = ix; }
+            }
+          }
+        }
+      } else {
+        // partial tile -> workspace [split][token][128], coalesced over features
+        for (int cb = 0; cb < bn; cb += 16) {
+          float v[16];
+          if (nchunks > 0) tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + cb, v);
+          else {
+#pragma unroll
+            for (int c = 0; c < 16; ++c) v[c] = 0.f;
+          }
+#pragma unroll
+          for (int c = 0; c < 16; ++c)
+            if (cb + c < nt) wsz[((size_t)split * bn + cb + c) * kBM + row] = v[c];
+        }
+        __threadfence();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (et == 0) {
+          const unsigned prev = atomicAdd(&p.tile_counters[(size_t)blockIdx.z * ntiles + tile], 1u);
+          ctl[1] = (prev == (unsigned)p.splits - 1) ? 1u : 0u;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (ctl[1]) {
+          __threadfence();
+          for (int c = 0; c < nt; ++c) {
+            float acc = 0.f;
+            for (int s = 0; s < p.splits; ++s) acc += __ldcg(&wsz[((size_t)s * bn + c) * kBM + row]);
+            if (EPI != kTcArgmax) {
+              if (n < p.N) tc_store<EPI>(p, slice, t0 + c, n, acc);
+            } else {
+              float x = (n < p.N) ? acc : -INFINITY;
+              int ix = (n < p.N) ? n : 0x7fffffff;
+              if (p.logits && n < p.N) p.logits[(size_t)(t0 + c) * p.N + n] = x;
+              warp_argmax(x, ix);
+              if (lane == 0) { s_val[q][c] = x; s_idx[q][c] = ix; }
+            }
+          }
+          if (et == 0) p.tile_counters[(size_t)blockIdx.z * ntiles + tile] = 0;   // ready for the next launch
+        }
+      }
+      if (EPI == kTcArgmax && (direct || ctl[1])) {
+        // tile-level (value, index) per token, then the CTA that completes the last tile merges all tiles
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (et < nt) {
+          float x = s_val[0][et];
+          int ix = s_idx[0][et];
+#pragma unroll
+          for (int w = 1; w < 4; ++w)
+            if (better(s_val[w][et], s_idx[w][et], x, ix)) { x = s_val[w][et]; ix = s_idx[w][et]; }
+          p.part_val[(size_t)tile * p.T + t0 + et] = x;
+          p.part_idx[(size_t)tile * p.T + t0 + et] = ix;
+        }
+        __threadfence();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (et == 0) {
+          const unsigned prev = atomicAdd(p.done_counter, 1u);
+          ctl[2] = (prev == (unsigned)(ntiles * (gridDim.z / zslices)) - 1) ? 1u : 0u;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (ctl[2]) {
+          __threadfence();
+          for (int t = warp - 2; t < p.T; t += 4) {
+            float x = -INFINITY;
+            int ix = 0x7fffffff;
+            for (int tl = lane; tl < ntiles; tl += 32) {
+              const float tv = __ldcg(&p.part_val[(size_t)tl * p.T + t]);
+              const int ti = __ldcg(&p.part_idx[(size_t)tl * p.T + t]);
+              if (better(tv, ti, x, ix)) { x = tv; ix = ti; }
+            }
+            warp_argmax(x, ix);
+            if (lane == 0) {
+              p.out_idx[t] = ix;
+              if (p.out_val) p.out_val[t] = x;
+            }
+          }
+          if (et == 0) *p.done_counter = 0;
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, ncols);
+  }
+}
+
+}  // namespace tc
+}  // namespace bpd

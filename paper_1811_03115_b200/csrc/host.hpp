@@ -88,7 +88,15 @@ struct bpd_session {
   // vocabulary top-1 workspace
   float* part_val;
   int* part_idx;
+  size_t part_elems;
   unsigned* counters;
+  // tensor-core path (bf16 models): activations feeding a projection are two bf16 planes (hi + lo)
+  int tc;
+  long long pl_xn, pl_attn, pl_ffh, pl_u, pl_o;   // elements between the planes of each buffer
+  int rows_all, rows_dec, rows_head;              // allocated rows of xn/attn/ffh, of u, of o
+  float* tc_ws; size_t tc_ws_floats;
+  unsigned* tc_counters; size_t tc_n_counters;
+  unsigned* tc_done;
   // host side
   int* pinned;             // pinned ring of all_done flags + staging
   cudaEvent_t ev_flag[8];

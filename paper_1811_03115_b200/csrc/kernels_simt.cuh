@@ -64,7 +64,8 @@ struct LnParams {
   const float* x;   // [rows, d]
   const void* g;    // [d] weight dtype
   const void* b;
-  void* y;          // [rows, d] activation dtype
+  void* y;          // [rows, d] activation dtype, or two bf16 planes (hi, lo) when plane > 0
+  long long plane;  // elements between the hi and the lo plane; 0 = single array
   float* y_f32;     // optional fp32 copy
   int rows, d;
   float eps;
@@ -89,7 +90,14 @@ __global__ void __launch_bounds__(128) layernorm_kernel(LnParams p) {
   AT* y = reinterpret_cast<AT*>(p.y) + (size_t)r * p.d;
   for (int c = lane; c < p.d; c += 32) {
     const float o = (x[c] - mean) * rstd * to_f(g[c]) + to_f(bb[c]);
-    y[c] = from_f<AT>(o);
+    if (p.plane) {
+      bf16* yp = reinterpret_cast<bf16*>(p.y) + (size_t)r * p.d + c;
+      const bf16 hi = __float2bfloat16_rn(o);
+      yp[0] = hi;
+      yp[p.plane] = __float2bfloat16_rn(o - __bfloat162float(hi));
+    } else {
+      y[c] = from_f<AT>(o);
+    }
     if (p.y_f32) p.y_f32[(size_t)r * p.d + c] = o;
   }
 }
@@ -225,6 +233,7 @@ __global__ void __launch_bounds__(kLinWarps * 32) linear_kernel(LinearParams p) 
 struct AttnParams {
   const void* q; long long ldq;    // query of row r, head h at q + r*ldq + h*dh
   void* out; long long ldo;
+  long long out_plane;             // > 0: output as two bf16 planes (hi, lo) this many elements apart
   int rows, rows_per_b, H, dh;
   int causal;                      // 1: keys 0 .. len[b]+i ; 0: keys 0 .. limit_b[b]-1
   const int* limit_b;
@@ -298,7 +307,17 @@ __global__ void __launch_bounds__(128) attention_kernel(AttnParams p) {
 #pragma unroll
   for (int t = 0; t < 4; ++t) {
     const int c = lane + 32 * t;
-    if (c < dh) o[c] = from_f<QT>(acc[t] * inv);
+    if (c < dh) {
+      const float ov = acc[t] * inv;
+      if (p.out_plane) {
+        bf16* op = reinterpret_cast<bf16*>(p.out) + (long long)r * p.ldo + h * dh + c;
+        const bf16 hi = __float2bfloat16_rn(ov);
+        op[0] = hi;
+        op[p.out_plane] = __float2bfloat16_rn(ov - __bfloat162float(hi));
+      } else {
+        o[c] = from_f<QT>(ov);
+      }
+    }
   }
 }
 

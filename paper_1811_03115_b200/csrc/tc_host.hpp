@@ -1,0 +1,144 @@
+// Host side of the tensor-core projection: TMA tensor maps, K-split planning and launches.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <map>
+#include <mutex>
+#include <tuple>
+
+#include "gemm_tc.cuh"
+#include "host.hpp"
+
+namespace bpd {
+namespace tc {
+
+// Resident CTA slots the planner aims to fill: 2 CTAs on each of the 148 SMs of a B200.
+constexpr int kSlots = 296;
+constexpr int kMinChunksPerSplit = 2;
+
+struct Plan {
+  int tiles, chunks, splits, chunks_per_split;
+};
+// Depends on (N, K) only -- never on the number of tokens -- so that a position
+// scored alone and the same position scored inside a block add up in the same order.
+inline Plan plan_splits(int N, int K) {
+  Plan pl;
+  pl.tiles = (N + kBM - 1) / kBM;
+  pl.chunks = (K + kBK - 1) / kBK;
+  int splits = std::max(1, std::min(pl.chunks / kMinChunksPerSplit, kSlots / pl.tiles));
+  pl.chunks_per_split = (pl.chunks + splits - 1) / splits;
+  pl.splits = (pl.chunks + pl.chunks_per_split - 1) / pl.chunks_per_split;
+  return pl;
+}
+inline int token_tiles(int T) { return (T + kMaxBN - 1) / kMaxBN; }
+inline int token_bn(int T) {
+  const int per = (T + token_tiles(T) - 1) / token_tiles(T);
+  return std::max(16, (per + 15) / 16 * 16);
+}
+// fp32 elements of split-K workspace a launch with these sizes needs.
+inline size_t ws_floats(int N, int K, int T, int zslices) {
+  const Plan pl = plan_splits(N, K);
+  if (pl.splits == 1) return 0;
+  return (size_t)token_tiles(T) * zslices * pl.tiles * pl.splits * token_bn(T) * kBM;
+}
+inline size_t counters_needed(int N, int T, int zslices) {
+  return (size_t)token_tiles(T) * zslices * ((N + kBM - 1) / kBM);
+}
+
+struct Scratch {
+  float* ws; size_t ws_floats;
+  unsigned* tile_counters; size_t n_counters;
+  unsigned* done_counter;
+  float* part_val; int* part_idx; size_t part_elems;
+  int* error;
+};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline int get_encode_fn(EncodeTiledFn* out) {
+  static EncodeTiledFn fn = nullptr;
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q);
+    if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !p)
+      return fail(BPD_E_CUDA, "cuTensorMapEncodeTiled is not available: %s", cudaGetErrorString(e));
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  *out = fn;
+  return BPD_OK;
+}
+
+// bf16 matrix [rows, cols] with `ld` elements between rows; boxes of (64 columns, box_rows rows), 128-byte swizzle.
+inline int make_map(const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows, CUtensorMap* out) {
+  typedef std::tuple<const void*, uint64_t, uint64_t, uint64_t, uint32_t> Key;
+  static std::map<Key, CUtensorMap> cache;
+  static std::mutex mu;
+  const Key key(ptr, rows, cols, ld, box_rows);
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = cache.find(key);
+    if (it != cache.end()) { *out = it->second; return BPD_OK; }
+  }
+  if ((uintptr_t)ptr % 16 || (ld * 2) % 16) return fail(BPD_E_INVALID, "tensor-map operand is not 16-byte aligned");
+  if (box_rows < 1 || box_rows > 256) return fail(BPD_E_INVALID, "tensor-map box of %u rows", box_rows);
+  EncodeTiledFn enc;
+  int rc = get_encode_fn(&enc);
+  if (rc) return rc;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {ld * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)kBK, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(BPD_E_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+  std::lock_guard<std::mutex> lock(mu);
+  cache[key] = *out;
+  return BPD_OK;
+}
+
+struct Operands {
+  const void* w; int w_rows;            // weights [w_rows, K] (all slices stacked)
+  const void* x; long long x_plane;     // activation planes: hi at x, lo at x + x_plane (elements)
+  long long ldx; int x_rows; int x_cols;  // allocated rows, total columns per row
+};
+
+template <int EPI>
+int launch(const Operands& op, int N, int K, int T, TcParams p, const Scratch& sc, cudaStream_t st, int zslices = 1,
+           int a_rows_per_slice = 0, int b_cols_per_slice = 0) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    BPD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(kMaxBN)));
+    attr_set = true;
+  }
+  const Plan pl = plan_splits(N, K);
+  const int ttiles = token_tiles(T), bn = token_bn(T);
+  const size_t need_ws = ws_floats(N, K, T, zslices), need_cnt = counters_needed(N, T, zslices);
+  if (need_ws > sc.ws_floats || need_cnt > sc.n_counters)
+    return fail(BPD_E_NOMEM, "split-K workspace too small (%zu floats, %zu counters needed)", need_ws, need_cnt);
+  if (EPI == kTcArgmax && (size_t)pl.tiles * T > sc.part_elems) return fail(BPD_E_NOMEM, "top-1 workspace too small");
+  CUtensorMap ma, mh, ml;
+  int rc = make_map(op.w, (uint64_t)op.w_rows, (uint64_t)K, (uint64_t)K, kBM, &ma);
+  if (rc) return rc;
+  rc = make_map(op.x, (uint64_t)op.x_rows, (uint64_t)op.x_cols, (uint64_t)op.ldx, (uint32_t)bn, &mh);
+  if (rc) return rc;
+  rc = make_map(static_cast<const bf16*>(op.x) + op.x_plane, (uint64_t)op.x_rows, (uint64_t)op.x_cols, (uint64_t)op.ldx,
+                (uint32_t)bn, &ml);
+  if (rc) return rc;
+  p.T = T; p.N = N; p.K = K; p.bn = bn; p.splits = pl.splits; p.chunks_per_split = pl.chunks_per_split;
+  p.ws = sc.ws; p.tile_counters = sc.tile_counters; p.done_counter = sc.done_counter;
+  p.part_val = sc.part_val; p.part_idx = sc.part_idx; p.error = sc.error;
+  dim3 grid(pl.tiles, pl.splits, ttiles * zslices);
+  gemm_tc_kernel<EPI><<<grid, kThreads, smem_bytes(bn), st>>>(ma, mh, ml, p, zslices, a_rows_per_slice, b_cols_per_slice);
+  BPD_CUDA(cudaGetLastError());
+  return BPD_OK;
+}
+
+}  // namespace tc
+}  // namespace bpd
