@@ -205,14 +205,14 @@ def run_gpu(args):
         """Device-resident: state rewound on the device, results left on the device."""
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
-        ev0.record()
+        ev0.record(sess.stream)
         for _ in range(n_steps):
             sess.bpd_rewind()
             if mode == "greedy":
                 sess.bpd_decode_greedy(N, fetch=False)
             else:
                 sess.bpd_decode_blockwise(k, N, fetch=False)
-        ev1.record()
+        ev1.record(sess.stream)
         barrier()
         return ev0.elapsed_time(ev1) / n_steps      # ms per decode
 

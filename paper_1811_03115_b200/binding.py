@@ -153,9 +153,13 @@ class Session:
         sb = nb.value
         with torch.cuda.device(model.device):
             self.buf = torch.empty(sb, dtype=torch.uint8, device=model.device)
+            # a stream of its own: the library replays each decoder pass as a CUDA graph, which the
+            # default stream cannot capture.  Time it with events recorded on ``self.stream``.
+            self.stream = torch.cuda.Stream(device=model.device)
+            self.stream.wait_stream(torch.cuda.current_stream())
             self.handle = _vp(0)
             _check(lib.bpd_session_create(model.handle, batch, max_src, max_tgt, self.buf.data_ptr(), sb,
-                                          _stream(), C.byref(self.handle)))
+                                          self.stream.cuda_stream, C.byref(self.handle)))
         self.session_bytes = sb
 
     def close(self):

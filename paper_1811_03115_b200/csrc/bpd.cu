@@ -139,6 +139,8 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
     kc[l] = a.take_bytes((size_t)B * ppr * kPage * d * ec);
     vc[l] = a.take_bytes((size_t)B * ppr * kPage * d * ec);
   }
+  const size_t npos = std::max<size_t>(max_src, (size_t)max_tgt + 1 + c.k_model);
+  float* pe = a.take<float>(npos * d);
   int* page_table = a.take<int>((size_t)B * ppr);
   RowState st;
   st.len = a.take<int>(B); st.j = a.take<int>(B); st.finished = a.take<int>(B); st.src_len = a.take<int>(B);
@@ -181,7 +183,7 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
     s->x = x; s->h_f32 = h_f32; s->xn = xn; s->qbuf = qbuf; s->attn = attn; s->ffh = ffh; s->u = u; s->o = o;
     s->crosskv = crosskv; s->kcache = kc; s->vcache = vc; s->st = st; s->src_dev = src_dev;
     s->tail_dev = tail_dev; s->plan_dev = plan_dev; s->part_val = part_val; s->part_idx = part_idx;
-    s->counters = counters; s->ppr = ppr; s->part_elems = tiles * R2;
+    s->counters = counters; s->ppr = ppr; s->part_elems = tiles * R2; s->pe = pe; s->npos = (int)npos;
     s->tc_ws = tc_ws; s->tc_ws_floats = ws; s->tc_counters = tc_counters; s->tc_n_counters = ncnt; s->tc_done = tc_done;
     s->pl_xn = (long long)(Rall * d); s->pl_attn = (long long)(Rall * d); s->pl_ffh = (long long)(Rall * c.d_ff);
     s->pl_u = (long long)(Rmax * c.k_model * c.d_hidden); s->pl_o = (long long)(R2 * d);
@@ -190,7 +192,7 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
   return align_up(a.off);
 }
 
-static size_t weight_bytes_for(const ParsedBlob& pb) { return align_up(pb.total) + align_up(pb.cfg.d / 2 * sizeof(double)); }
+static size_t weight_bytes_for(const ParsedBlob& pb) { return align_up(pb.total); }
 
 // ------------------------------------------------------------------ launches
 static std::atomic<long long> g_launches{0};
@@ -255,7 +257,7 @@ static int run_encoder(bpd_session* s) {
   const int E = s->B * s->max_src, d = c.d;
   EmbedParams ep;
   memset(&ep, 0, sizeof(ep));
-  ep.table = m->src_embed; ep.inv_freq = m->inv_freq; ep.x = s->x; ep.rows = E; ep.rows_per_b = s->max_src;
+  ep.table = m->src_embed; ep.pe = s->pe; ep.npos = s->npos; ep.x = s->x; ep.rows = E; ep.rows_per_b = s->max_src;
   ep.d = d; ep.vocab = c.V; ep.st = s->st; ep.src = s->src_dev;
   embed_kernel<WT><<<E, 128, 0, st>>>(ep);
   ++g_launches;
@@ -270,7 +272,7 @@ static int run_encoder(bpd_session* s) {
     ap.k = static_cast<float*>(s->qbuf) + d; ap.v = static_cast<float*>(s->qbuf) + 2 * d;
     ap.ldkv = 3 * d; ap.bstride = (long long)s->max_src * 3 * d; ap.paged = 0; ap.st = s->st;
     ap.scale = 1.0f / sqrtf((float)ap.dh);
-    attention_kernel<float, float><<<ceil_div(E * c.H, 4), 128, 0, st>>>(ap);
+    launch_attention<float, float>(ap, st);
     ++g_launches;
     LinearParams po = lin(s->attn, d, L.wo, d, d, nullptr, E, s->x, d, 0, nullptr);
     launch_linear<WT, float, kEpiResidual>(po, 1, st);
@@ -306,7 +308,7 @@ static int run_pass(bpd_session* s, const PassArgs& a) {
   const int* done = s->st.all_done;
   EmbedParams ep;
   memset(&ep, 0, sizeof(ep));
-  ep.table = m->tgt_embed; ep.inv_freq = m->inv_freq; ep.x = s->x; ep.rows = R; ep.rows_per_b = a.kcur;
+  ep.table = m->tgt_embed; ep.pe = s->pe; ep.npos = s->npos; ep.x = s->x; ep.rows = R; ep.rows_per_b = a.kcur;
   ep.d = d; ep.vocab = c.V; ep.st = s->st; ep.forced = a.forced; ep.forced_rows = a.forced_rows;
   ep.kforced = a.kforced; ep.src = nullptr; ep.all_done = done;
   prof_mark(s, kProfLayers, 0);
@@ -324,7 +326,7 @@ static int run_pass(bpd_session* s, const PassArgs& a) {
     ap.q = s->qbuf; ap.ldq = d; ap.out = s->attn; ap.ldo = d; ap.rows = R; ap.rows_per_b = a.kcur;
     ap.H = c.H; ap.dh = d / c.H; ap.causal = 1; ap.k = s->kcache[l]; ap.v = s->vcache[l]; ap.ldkv = d;
     ap.paged = 1; ap.st = s->st; ap.scale = 1.0f / sqrtf((float)ap.dh); ap.all_done = done;
-    attention_kernel<float, WT><<<ceil_div(R * c.H, 4), 128, 0, st>>>(ap);
+    launch_attention<float, WT>(ap, st);
     ++g_launches;
     launch_linear<WT, float, kEpiResidual>(lin(s->attn, d, L.wo, d, d, nullptr, R, s->x, d, 0, done), 1, st);
     // cross-attention over the encoder memory
@@ -332,7 +334,7 @@ static int run_pass(bpd_session* s, const PassArgs& a) {
     launch_linear<WT, float, kEpiStoreAct>(lin(s->xn, d, L.cwq, d, d, nullptr, R, s->qbuf, d, 0, done), 1, st);
     ap.causal = 0; ap.limit_b = s->st.src_len; ap.k = s->crosskv[l]; ap.v = static_cast<float*>(s->crosskv[l]) + d;
     ap.ldkv = 2 * d; ap.bstride = (long long)s->max_src * 2 * d; ap.paged = 0;
-    attention_kernel<float, float><<<ceil_div(R * c.H, 4), 128, 0, st>>>(ap);
+    launch_attention<float, float>(ap, st);
     ++g_launches;
     launch_linear<WT, float, kEpiResidual>(lin(s->attn, d, L.cwo, d, d, nullptr, R, s->x, d, 0, done), 1, st);
     // feed-forward
@@ -400,7 +402,7 @@ static int run_encoder_tc(bpd_session* s) {
   const tc::Scratch sc = tc_scratch(s);
   EmbedParams ep;
   memset(&ep, 0, sizeof(ep));
-  ep.table = m->src_embed; ep.inv_freq = m->inv_freq; ep.x = s->x; ep.rows = E; ep.rows_per_b = s->max_src;
+  ep.table = m->src_embed; ep.pe = s->pe; ep.npos = s->npos; ep.x = s->x; ep.rows = E; ep.rows_per_b = s->max_src;
   ep.d = d; ep.vocab = c.V; ep.st = s->st; ep.src = s->src_dev;
   embed_kernel<bf16><<<E, 128, 0, st>>>(ep);
   ++g_launches;
@@ -421,7 +423,7 @@ static int run_encoder_tc(bpd_session* s) {
     ap.k = static_cast<float*>(s->qbuf) + d; ap.v = static_cast<float*>(s->qbuf) + 2 * d;
     ap.ldkv = 3 * d; ap.bstride = (long long)s->max_src * 3 * d; ap.paged = 0; ap.st = s->st;
     ap.scale = 1.0f / sqrtf((float)ap.dh);
-    attention_kernel<float, float><<<ceil_div(E * c.H, 4), 128, 0, st>>>(ap);
+    launch_attention<float, float>(ap, st);
     ++g_launches;
     tc::TcParams po = tc_params(nullptr, 0, nullptr);
     po.out_f32 = s->x; po.ldo = d;
@@ -454,7 +456,7 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   prof_mark(s, kProfLayers, 0);
   EmbedParams ep;
   memset(&ep, 0, sizeof(ep));
-  ep.table = m->tgt_embed; ep.inv_freq = m->inv_freq; ep.x = s->x; ep.rows = R; ep.rows_per_b = a.kcur;
+  ep.table = m->tgt_embed; ep.pe = s->pe; ep.npos = s->npos; ep.x = s->x; ep.rows = R; ep.rows_per_b = a.kcur;
   ep.d = d; ep.vocab = c.V; ep.st = s->st; ep.forced = a.forced; ep.forced_rows = a.forced_rows;
   ep.kforced = a.kforced; ep.src = nullptr; ep.all_done = done;
   embed_kernel<bf16><<<R, 128, 0, st>>>(ep);
@@ -476,7 +478,7 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
     ap.q = s->qbuf; ap.ldq = d; ap.out = s->attn; ap.ldo = d; ap.out_plane = s->pl_attn; ap.rows = R;
     ap.rows_per_b = a.kcur; ap.H = c.H; ap.dh = d / c.H; ap.causal = 1; ap.k = s->kcache[l]; ap.v = s->vcache[l];
     ap.ldkv = d; ap.paged = 1; ap.st = s->st; ap.scale = 1.0f / sqrtf((float)ap.dh); ap.all_done = done;
-    attention_kernel<float, bf16><<<ceil_div(R * c.H, 4), 128, 0, st>>>(ap);
+    launch_attention<float, bf16>(ap, st);
     ++g_launches;
     tc::TcParams po = tc_params(nullptr, 0, done);
     po.out_f32 = s->x; po.ldo = d;
@@ -487,7 +489,7 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
     BPD_TRY(tc::launch<tc::kTcF32>(with_w(xn, L.cwq, d), d, d, R, pc, sc, st)); ++g_launches;
     ap.causal = 0; ap.limit_b = s->st.src_len; ap.k = s->crosskv[l]; ap.v = static_cast<float*>(s->crosskv[l]) + d;
     ap.ldkv = 2 * d; ap.bstride = (long long)s->max_src * 2 * d; ap.paged = 0;
-    attention_kernel<float, float><<<ceil_div(R * c.H, 4), 128, 0, st>>>(ap);
+    launch_attention<float, float>(ap, st);
     ++g_launches;
     BPD_TRY(tc::launch<tc::kTcResidual>(with_w(at, L.cwo, d), d, d, R, po, sc, st)); ++g_launches;
     launch_ln<bf16, float>(s->x, L.ln3g, L.ln3b, s->xn, nullptr, R, d, c.eps, done, st, s->pl_xn);
@@ -536,9 +538,42 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   return BPD_OK;
 }
 
-static int dispatch_pass(bpd_session* s, const PassArgs& a) {
+static int dispatch_eager(bpd_session* s, const PassArgs& a) {
   if (s->tc) return run_pass_tc(s, a);
   return s->m->cfg.dtype == 0 ? run_pass<float>(s, a) : run_pass<bf16>(s, a);
+}
+
+// A pass is a fixed sequence of launches for given arguments: the first use runs it eagerly (which also
+// creates tensor maps and sets kernel attributes), the second captures it into a CUDA graph, later uses replay it.
+static int dispatch_pass(bpd_session* s, const PassArgs& a) {
+  if (s->profiling || !s->use_graphs || a.logits_dump) return dispatch_eager(s, a);
+  const GraphKey key(a.mode, a.kcur, a.kh, a.knext, (const void*)a.forced, a.forced_rows, a.kforced, a.max_new, a.eos,
+                     (const void*)a.logits_dump);
+  GraphEntry& ge = s->graphs[key];
+  if (ge.exec) {
+    BPD_CUDA(cudaGraphLaunch(ge.exec, s->stream));
+    g_launches += ge.launches;
+    s->invocations += 1;
+    return BPD_OK;
+  }
+  if (ge.uses++ == 0) return dispatch_eager(s, a);
+  const long long before = g_launches.load();
+  BPD_CUDA(cudaStreamBeginCapture(s->stream, cudaStreamCaptureModeThreadLocal));
+  const int rc = dispatch_eager(s, a);
+  cudaGraph_t graph = nullptr;
+  const cudaError_t e = cudaStreamEndCapture(s->stream, &graph);
+  if (rc) { if (graph) cudaGraphDestroy(graph); return rc; }
+  if (e != cudaSuccess || !graph) return fail(BPD_E_CUDA, "stream capture of the decoder pass failed: %s", cudaGetErrorString(e));
+  ge.launches = g_launches.load() - before;
+  s->invocations -= 1;                       // the captured call only recorded the work
+  g_launches -= ge.launches;
+  const cudaError_t e2 = cudaGraphInstantiate(&ge.exec, graph, 0);
+  cudaGraphDestroy(graph);
+  if (e2 != cudaSuccess) { ge.exec = nullptr; return fail(BPD_E_CUDA, "cudaGraphInstantiate failed: %s", cudaGetErrorString(e2)); }
+  BPD_CUDA(cudaGraphLaunch(ge.exec, s->stream));
+  g_launches += ge.launches;
+  s->invocations += 1;
+  return BPD_OK;
 }
 
 static int check_device_error(bpd_session* s) {
@@ -648,12 +683,7 @@ int bpd_load_weights(const void* blob, size_t blob_bytes, void* dev_weight_buf, 
   if (c.head_layout == 0) { T("head.w2", m->head_w2, k * d, k * fh) } else { T("head.w2", m->head_w2, k, d, fh) }
   T("head.b2", m->head_b2, k * d)
 #undef T
-  std::vector<double> invf(d / 2);
-  for (int i = 0; i < d / 2; ++i) invf[i] = pow(10000.0, -2.0 * i / d);
-  double* invf_dev = reinterpret_cast<double*>(m->base + align_up(pb.total));
-  m->inv_freq = invf_dev;
   cudaError_t e = cudaMemcpyAsync(m->base, blob, pb.total, cudaMemcpyHostToDevice, m->stream);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(invf_dev, invf.data(), invf.size() * sizeof(double), cudaMemcpyHostToDevice, m->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(m->stream);
   if (e != cudaSuccess) { delete m; return fail(BPD_E_CUDA, "weight upload failed: %s", cudaGetErrorString(e)); }
   *out = m;
@@ -680,18 +710,30 @@ int bpd_session_create(const bpd_model* model, int batch, int max_src, int max_t
   s->base = static_cast<char*>(dev_session_buf); s->bytes = dev_bytes; s->stream = (cudaStream_t)cuda_stream;
   s->profiling = 0;
   s->tc = (model->cfg.dtype == 1 && !getenv("BPD_DISABLE_TC")) ? 1 : 0;
+  // the default streams cannot be captured: graphs need a stream of the caller's own
+  const bool own_stream = s->stream != nullptr && s->stream != cudaStreamLegacy && s->stream != cudaStreamPerThread;
+  s->use_graphs = (own_stream && !getenv("BPD_DISABLE_GRAPHS")) ? 1 : 0;
   s->phase = kPhaseCreated; s->plan_len = 0; s->plan_k = 0; s->invocations = 0; s->pinned = nullptr;
   plan_session(model->cfg, batch, max_src, max_tgt, s->base, s);
   // page table: row b's p-th page is physical page p*B + b (rows interleaved in the pool)
   std::vector<int> pt((size_t)batch * s->ppr);
   for (int b = 0; b < batch; ++b)
     for (int p = 0; p < s->ppr; ++p) pt[(size_t)b * s->ppr + p] = p * batch + b;
+  // sinusoidal positions: PE(p, 2i) = sin(p / 10000^(2i/d)), PE(p, 2i+1) = cos(same), evaluated in double
+  std::vector<float> pe((size_t)s->npos * model->cfg.d);
+  for (int pos = 0; pos < s->npos; ++pos)
+    for (int i = 0; i < model->cfg.d / 2; ++i) {
+      const double ang = (double)pos / pow(10000.0, 2.0 * i / model->cfg.d);
+      pe[(size_t)pos * model->cfg.d + 2 * i] = (float)sin(ang);
+      pe[(size_t)pos * model->cfg.d + 2 * i + 1] = (float)cos(ang);
+    }
   cudaError_t e = cudaMallocHost(reinterpret_cast<void**>(&s->pinned), (256 + (size_t)batch * kMaxK) * sizeof(int));
   for (int i = 0; i < 8 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&s->ev_flag[i], cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreate(&s->ev0);
   if (e == cudaSuccess) e = cudaEventCreate(&s->ev1);
   if (e == cudaSuccess) e = cudaMemsetAsync(s->base, 0, need, s->stream);
   if (e == cudaSuccess) e = cudaMemcpyAsync(const_cast<int*>(s->st.page_table), pt.data(), pt.size() * sizeof(int), cudaMemcpyHostToDevice, s->stream);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(s->pe, pe.data(), pe.size() * sizeof(float), cudaMemcpyHostToDevice, s->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s->stream);
   if (e != cudaSuccess) {
     delete s;
@@ -705,6 +747,8 @@ int bpd_session_destroy(bpd_session* s) {
   if (!s) return BPD_OK;
   cudaStreamSynchronize(s->stream);
   prof_clear(s);
+  for (auto& kv : s->graphs)
+    if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
   if (s->pinned) cudaFreeHost(s->pinned);
   for (int i = 0; i < 8; ++i) cudaEventDestroy(s->ev_flag[i]);
   cudaEventDestroy(s->ev0);

@@ -344,17 +344,36 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (ctl[1]) {
           __threadfence();
-          for (int c = 0; c < nt; ++c) {
-            float acc = 0.f;
-            for (int s = 0; s < p.splits; ++s) acc += __ldcg(&wsz[((size_t)s * bn + c) * kBM + row]);
-            if (EPI != kTcArgmax) {
-              if (n < p.N) tc_store<EPI>(p, slice, t0 + c, n, acc);
-            } else {
-              float x = (n < p.N) ? acc : -INFINITY;
-              int ix = (n < p.N) ? n : 0x7fffffff;
-              if (p.logits && n < p.N) p.logits[(size_t)(t0 + c) * p.N + n] = x;
-              warp_argmax(x, ix);
-              if (lane == 0) { s_val[q][c] = x; s_idx[q][c] = ix; }
+          // splits are added in split order; the loads of four splits x eight tokens are issued together
+          for (int cg = 0; cg < nt; cg += 8) {
+            float acc[8];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) acc[c] = 0.f;
+            for (int s0 = 0; s0 < p.splits; s0 += 4) {
+              float v[4][8];
+#pragma unroll
+              for (int ss = 0; ss < 4; ++ss)
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                  v[ss][c] = (s0 + ss < p.splits && cg + c < nt)
+                                 ? __ldcg(&wsz[((size_t)(s0 + ss) * bn + cg + c) * kBM + row]) : 0.f;
+#pragma unroll
+              for (int ss = 0; ss < 4; ++ss)
+#pragma unroll
+                for (int c = 0; c < 8; ++c) acc[c] += v[ss][c];
+            }
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              if (cg + c >= nt) break;
+              if (EPI != kTcArgmax) {
+                if (n < p.N) tc_store<EPI>(p, slice, t0 + cg + c, n, acc[c]);
+              } else {
+                float x = (n < p.N) ? acc[c] : -INFINITY;
+                int ix = (n < p.N) ? n : 0x7fffffff;
+                if (p.logits && n < p.N) p.logits[(size_t)(t0 + cg + c) * p.N + n] = x;
+                warp_argmax(x, ix);
+                if (lane == 0) { s_val[q][cg + c] = x; s_idx[q][cg + c] = ix; }
+              }
             }
           }
           if (et == 0) p.tile_counters[(size_t)blockIdx.z * ntiles + tile] = 0;   // ready for the next launch

@@ -7,6 +7,7 @@
 
 #include <map>
 #include <string>
+#include <tuple>
 #include <vector>
 
 #include "../../include/bpd.h"
@@ -63,7 +64,13 @@ struct bpd_model {
   std::vector<bpd::DecLayer> dec;
   const void *enc_lnf_g, *enc_lnf_b, *dec_lnf_g, *dec_lnf_b;
   const void *head_w1, *head_b1, *head_w2, *head_b2;
-  const double* inv_freq;   // device [d/2]
+};
+
+typedef std::tuple<int, int, int, int, const void*, int, int, int, int, const void*> GraphKey;
+struct GraphEntry {
+  int uses = 0;
+  long long launches = 0;
+  cudaGraphExec_t exec = nullptr;
 };
 
 enum ProfSlot { kProfLayers = 0, kProfHeadW1 = 1, kProfHeadW2 = 2, kProfVocab = 3, kProfSlots = 4 };
@@ -78,7 +85,8 @@ struct bpd_session {
   cudaStream_t stream;
   int phase;
   // activations
-  float *x, *h_f32;
+  float *x, *h_f32, *pe;
+  int npos;
   void *xn, *qbuf, *attn, *ffh, *u, *o;
   std::vector<void*> crosskv, kcache, vcache;
   // integers
@@ -103,5 +111,7 @@ struct bpd_session {
   cudaEvent_t ev0, ev1;
   int64_t invocations;
   int profiling;
+  int use_graphs;
+  std::map<GraphKey, GraphEntry> graphs;
   std::vector<cudaEvent_t> prof_begin[kProfSlots], prof_end[kProfSlots];
 };

@@ -12,7 +12,8 @@ namespace bpd {
 // ------------------------------------------------------------------ embedding (decoder and encoder)
 struct EmbedParams {
   const void* table;       // [V, d] weight dtype
-  const double* inv_freq;  // [d/2] 10000^(-2i/d)
+  const float* pe;         // [npos, d] sinusoidal position signal, tabulated on the host in double precision
+  int npos;
   float* x;                // [rows, d] residual stream
   int rows, rows_per_b, d, vocab;
   // decoder: token = block[b][i] (or a forced proposal), position = len[b] + i
@@ -46,16 +47,21 @@ __global__ void embed_kernel(EmbedParams p) {
     pos = p.st.len[b] + i;
     if (threadIdx.x == 0) p.st.cur_block[b * kMaxK + i] = tok;
   }
-  if (tok < 0 || tok >= p.vocab) {   // never index outside the table; report instead
+  if (tok < 0 || tok >= p.vocab || pos >= p.npos) {   // never index outside the tables; report instead
     if (threadIdx.x == 0) atomicCAS(p.st.error, 0, 1);
     tok = 0;
+    pos = 0;
   }
   const WT* row = reinterpret_cast<const WT*>(p.table) + (size_t)tok * p.d;
+  const float* pe = p.pe + (size_t)pos * p.d;
   const float scale = sqrtf((float)p.d);
-  for (int c = threadIdx.x; c < p.d; c += blockDim.x) {
-    const double ang = (double)pos * p.inv_freq[c >> 1];
-    const float pe = (float)((c & 1) ? cos(ang) : sin(ang));
-    p.x[(size_t)r * p.d + c] = to_f(row[c]) * scale + pe;
+  for (int c = threadIdx.x * 8; c < p.d; c += blockDim.x * 8) {
+    float w[8], e[8];
+    load8(row + c, w);
+    load8(pe + c, e);
+    float4* out = reinterpret_cast<float4*>(p.x + (size_t)r * p.d + c);
+    out[0] = make_float4(w[0] * scale + e[0], w[1] * scale + e[1], w[2] * scale + e[2], w[3] * scale + e[3]);
+    out[1] = make_float4(w[4] * scale + e[4], w[5] * scale + e[5], w[6] * scale + e[6], w[7] * scale + e[7]);
   }
 }
 
@@ -72,33 +78,62 @@ struct LnParams {
   const int* all_done;
 };
 
+constexpr int kLnMaxD = 1024;   // the row is held in registers: 8 float4 per lane
+
 template <typename WT, typename AT>
 __global__ void __launch_bounds__(128) layernorm_kernel(LnParams p) {
   if (p.all_done && *p.all_done) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = blockIdx.x * 4 + warp;
   if (r >= p.rows) return;
-  const float* x = p.x + (size_t)r * p.d;
+  const float4* x4 = reinterpret_cast<const float4*>(p.x + (size_t)r * p.d);
+  const int nv = p.d >> 2;                 // float4 per row (d is a multiple of 8)
+  float4 v[kLnMaxD / 128];
   float s = 0.f;
-  for (int c = lane; c < p.d; c += 32) s += x[c];
+#pragma unroll
+  for (int i = 0; i < kLnMaxD / 128; ++i) {
+    const int idx = i * 32 + lane;
+    v[i] = (idx < nv) ? x4[idx] : make_float4(0.f, 0.f, 0.f, 0.f);
+    s += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+  }
   const float mean = warp_sum(s) / (float)p.d;
-  float v = 0.f;
-  for (int c = lane; c < p.d; c += 32) { const float t = x[c] - mean; v += t * t; }
-  const float rstd = rsqrtf(warp_sum(v) / (float)p.d + p.eps);
+  float q = 0.f;
+#pragma unroll
+  for (int i = 0; i < kLnMaxD / 128; ++i) {
+    if (i * 32 + lane < nv) {
+      const float a = v[i].x - mean, b = v[i].y - mean, c = v[i].z - mean, d = v[i].w - mean;
+      q += (a * a + b * b) + (c * c + d * d);
+    }
+  }
+  const float rstd = rsqrtf(warp_sum(q) / (float)p.d + p.eps);
   const WT* g = reinterpret_cast<const WT*>(p.g);
   const WT* bb = reinterpret_cast<const WT*>(p.b);
-  AT* y = reinterpret_cast<AT*>(p.y) + (size_t)r * p.d;
-  for (int c = lane; c < p.d; c += 32) {
-    const float o = (x[c] - mean) * rstd * to_f(g[c]) + to_f(bb[c]);
-    if (p.plane) {
-      bf16* yp = reinterpret_cast<bf16*>(p.y) + (size_t)r * p.d + c;
-      const bf16 hi = __float2bfloat16_rn(o);
-      yp[0] = hi;
-      yp[p.plane] = __float2bfloat16_rn(o - __bfloat162float(hi));
-    } else {
-      y[c] = from_f<AT>(o);
+#pragma unroll
+  for (int i = 0; i < kLnMaxD / 128; ++i) {
+    const int idx = i * 32 + lane;
+    if (idx < nv) {
+      const int c = idx * 4;
+      const float in[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+      float o[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) o[e] = (in[e] - mean) * rstd * to_f(g[c + e]) + to_f(bb[c + e]);
+      if (p.plane) {
+        bf16* yp = reinterpret_cast<bf16*>(p.y) + (size_t)r * p.d + c;
+        bf16 hi[4], lo[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          hi[e] = __float2bfloat16_rn(o[e]);
+          lo[e] = __float2bfloat16_rn(o[e] - __bfloat162float(hi[e]));
+        }
+        *reinterpret_cast<uint2*>(yp) = *reinterpret_cast<const uint2*>(hi);
+        *reinterpret_cast<uint2*>(yp + p.plane) = *reinterpret_cast<const uint2*>(lo);
+      } else {
+        AT* y = reinterpret_cast<AT*>(p.y) + (size_t)r * p.d + c;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) y[e] = from_f<AT>(o[e]);
+      }
+      if (p.y_f32) *reinterpret_cast<float4*>(p.y_f32 + (size_t)r * p.d + c) = make_float4(o[0], o[1], o[2], o[3]);
     }
-    if (p.y_f32) p.y_f32[(size_t)r * p.d + c] = o;
   }
 }
 
@@ -318,6 +353,142 @@ __global__ void __launch_bounds__(128) attention_kernel(AttnParams p) {
         o[c] = from_f<QT>(ov);
       }
     }
+  }
+}
+
+// Attention with the keys of one (row, head) spread over the 8 warps of a CTA: warp w takes the 32-key
+// chunks w, w+8, ... in increasing position order, then the 8 partial (max, sum, output) states are
+// merged in warp order.  The partition depends only on key positions, so the result for a position does
+// not depend on how many rows the launch carries.  DH = head width (16, 32, 64 or 128).
+constexpr int kAttnWarps = 8;
+
+template <int N> __device__ __forceinline__ void load_n(const float* p, float (&o)[N]) {
+#pragma unroll
+  for (int i = 0; i < N; ++i) o[i] = p[i];
+}
+template <> __device__ __forceinline__ void load_n<2>(const float* p, float (&o)[2]) {
+  const float2 v = *reinterpret_cast<const float2*>(p); o[0] = v.x; o[1] = v.y;
+}
+template <> __device__ __forceinline__ void load_n<4>(const float* p, float (&o)[4]) {
+  const float4 v = *reinterpret_cast<const float4*>(p); o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w;
+}
+template <int N> __device__ __forceinline__ void load_n(const bf16* p, float (&o)[N]) {
+#pragma unroll
+  for (int i = 0; i < N; ++i) o[i] = __bfloat162float(p[i]);
+}
+template <> __device__ __forceinline__ void load_n<2>(const bf16* p, float (&o)[2]) {
+  const uint32_t v = *reinterpret_cast<const uint32_t*>(p);
+  o[0] = __uint_as_float(v << 16); o[1] = __uint_as_float(v & 0xffff0000u);
+}
+template <> __device__ __forceinline__ void load_n<4>(const bf16* p, float (&o)[4]) {
+  const uint2 v = *reinterpret_cast<const uint2*>(p);
+  o[0] = __uint_as_float(v.x << 16); o[1] = __uint_as_float(v.x & 0xffff0000u);
+  o[2] = __uint_as_float(v.y << 16); o[3] = __uint_as_float(v.y & 0xffff0000u);
+}
+
+template <typename QT, typename CT, int DH>
+__global__ void __launch_bounds__(kAttnWarps * 32) attention_split_kernel(AttnParams p) {
+  if (p.all_done && *p.all_done) return;
+  constexpr int DPL = (DH >= 32) ? DH / 32 : 1;       // output dims per lane (contiguous)
+  __shared__ float s_q[DH];
+  __shared__ float s_m[kAttnWarps], s_l[kAttnWarps];
+  __shared__ float s_acc[kAttnWarps][DH];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int item = blockIdx.x;
+  const int r = item / p.H, h = item % p.H;
+  const int b = r / p.rows_per_b, i = r % p.rows_per_b;
+  const int limit = p.causal ? (p.st.len[b] + i + 1) : p.limit_b[b];
+  const QT* q = reinterpret_cast<const QT*>(p.q) + (long long)r * p.ldq + h * DH;
+  if (threadIdx.x < DH) s_q[threadIdx.x] = to_f(q[threadIdx.x]) * p.scale;
+  __syncthreads();
+  const CT* K = reinterpret_cast<const CT*>(p.k);
+  const CT* V = reinterpret_cast<const CT*>(p.v);
+  const int* pt = p.st.page_table + b * p.st.pages_per_row;
+  float m_run = -INFINITY, l_run = 0.f;
+  float acc[DPL];
+#pragma unroll
+  for (int t = 0; t < DPL; ++t) acc[t] = 0.f;
+  const int nchunks = (limit + 31) >> 5;
+  const bool owns = (DH >= 32) || (lane < DH);
+  const int dim0 = (DH >= 32) ? lane * DPL : lane;
+  for (int ch = warp; ch < nchunks; ch += kAttnWarps) {
+    const int c0 = ch << 5;
+    // a 32-key chunk never straddles a 64-position page
+    const size_t base = p.paged ? ((size_t)pt[c0 / kPage] * kPage + (c0 % kPage)) * p.ldkv + h * DH
+                                : (size_t)b * p.bstride + (size_t)c0 * p.ldkv + h * DH;
+    const int nk = min(32, limit - c0);
+    float sc = -INFINITY;
+    if (lane < nk) {
+      const CT* kr = K + base + (size_t)lane * p.ldkv;
+      float dot = 0.f;
+#pragma unroll
+      for (int c = 0; c < DH; c += 8) {
+        float kv[8];
+        load8(kr + c, kv);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) dot = fmaf(s_q[c + e], kv[e], dot);
+      }
+      sc = dot;
+    }
+    const float m_new = fmaxf(m_run, warp_max(sc));
+    const float corr = expf(m_run - m_new);
+    const float pj = (lane < nk) ? expf(sc - m_new) : 0.f;
+    l_run = l_run * corr + warp_sum(pj);
+#pragma unroll
+    for (int t = 0; t < DPL; ++t) acc[t] *= corr;
+    const CT* vb = V + base + dim0;
+#pragma unroll 8
+    for (int jj = 0; jj < nk; ++jj) {
+      const float pw = __shfl_sync(0xffffffffu, pj, jj);
+      if (owns) {
+        float vv[DPL];
+        load_n<DPL>(vb + (size_t)jj * p.ldkv, vv);
+#pragma unroll
+        for (int t = 0; t < DPL; ++t) acc[t] = fmaf(pw, vv[t], acc[t]);
+      }
+    }
+    m_run = m_new;
+  }
+  if (lane == 0) { s_m[warp] = m_run; s_l[warp] = l_run; }
+  if (owns) {
+#pragma unroll
+    for (int t = 0; t < DPL; ++t) s_acc[warp][dim0 + t] = acc[t];
+  }
+  __syncthreads();
+  if (threadIdx.x < DH) {
+    const int c = threadIdx.x;
+    float M = s_m[0];
+#pragma unroll
+    for (int w = 1; w < kAttnWarps; ++w) M = fmaxf(M, s_m[w]);
+    float num = 0.f, den = 0.f;
+#pragma unroll
+    for (int w = 0; w < kAttnWarps; ++w) {
+      const float e = expf(s_m[w] - M);          // warps without keys hold -inf: weight 0
+      num = fmaf(e, s_acc[w][c], num);
+      den = fmaf(e, s_l[w], den);
+    }
+    const float ov = num / den;
+    if (p.out_plane) {
+      bf16* op = reinterpret_cast<bf16*>(p.out) + (long long)r * p.ldo + h * DH + c;
+      const bf16 hi = __float2bfloat16_rn(ov);
+      op[0] = hi;
+      op[p.out_plane] = __float2bfloat16_rn(ov - __bfloat162float(hi));
+    } else {
+      reinterpret_cast<QT*>(p.out)[(long long)r * p.ldo + h * DH + c] = from_f<QT>(ov);
+    }
+  }
+}
+
+// Picks the split kernel for the common head widths, the generic one-warp kernel otherwise.
+template <typename QT, typename CT>
+static void launch_attention(const AttnParams& p, cudaStream_t st) {
+  const int items = p.rows * p.H;
+  switch (p.dh) {
+    case 16: attention_split_kernel<QT, CT, 16><<<items, kAttnWarps * 32, 0, st>>>(p); break;
+    case 32: attention_split_kernel<QT, CT, 32><<<items, kAttnWarps * 32, 0, st>>>(p); break;
+    case 64: attention_split_kernel<QT, CT, 64><<<items, kAttnWarps * 32, 0, st>>>(p); break;
+    case 128: attention_split_kernel<QT, CT, 128><<<items, kAttnWarps * 32, 0, st>>>(p); break;
+    default: attention_kernel<QT, CT><<<(items + 3) / 4, 128, 0, st>>>(p); break;
   }
 }
 
