@@ -33,15 +33,27 @@ METRIC = "decoded tokens/s at batch 1 (d=1024, k=8)"
 HEADLINE = "C3"
 MEAN_ACCEPT = 5.0            # geometric mean of the controlled-acceptance schedule for the headline line
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu capture
+# summarised under profiles/ (None until a capture of the current kernel exists)
+TRAFFIC = {"C3": 538183424 + 3915264}     # profiles/head_output_gemm_tc_c3.txt
 
 
 def _peaks():
+    """(HBM GB/s, sustained bf16 TFLOP/s, kind) from the driver-written measurement, else the machine's fallback."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as fh:
             p = json.load(fh)
-        return float(p["hbm_gbs"]), "measured"
-    return 6650.0, "fallback"
+        return float(p["hbm_gbs"]), float(p.get("bf16_tflops_sustained", 1400.0)), "measured"
+    return 6650.0, 1400.0, "fallback"
+
+
+DESCRIPTIONS = {
+    "C2": "C2: base enc-dec 6+6, d_model 512, 8 heads, FFN 2048, vocab 32768, k=4 dense heads, batch 1, source 32 ids",
+    "C3": "C3: big enc-dec 6+6, d_model 1024, 16 heads, FFN 4096, vocab 32768, k=8 dense heads, batch 1, source 40 ids",
+    "C4": "C4: big enc-dec 6+6, d_model 1024, k=10 dense heads, batch 32, source lengths uniform in [10,80]",
+    "C5": "C5: super-resolution shape, 6+6, d_model 512, vocab 256, k=10 dense heads, batch 1, 192 source ids",
+}
 
 
 def iteration_bytes(cfg, k, batch, mean_T, mean_S):
@@ -186,7 +198,7 @@ def run_gpu(args):
     torch.cuda.set_device(local)
     dev = f"cuda:{local}"
 
-    w = WORKLOADS[HEADLINE]
+    w = WORKLOADS[args.workload]
     cfg, k, N = w.cfg, w.cfg.k_model, w.n_decode
     blob = make_weights(cfg, w.weight_seed, w.sigma)
     src, src_len = make_source(w)
@@ -242,20 +254,37 @@ def run_gpu(args):
     sess.bpd_profile(True)
     timed_decodes(max(1, min(args.steps, 5)), "block")
     phases = [sess.bpd_profile_read(p) for p in range(4)]
-    sess.bpd_profile(False)
-    peak, peak_kind = _peaks()
+    peak, peak_tf, peak_kind = _peaks()
     mean_T = 1 + N / 2.0
     it_bytes, w2_bytes = iteration_bytes(cfg, k, w.batch, mean_T, float(src_len.mean()))
     n_w2, ms_w2 = phases[2]
-    # the priming pass evaluates the same k heads on one row: same weight bytes per launch
+    # the priming pass evaluates the same k heads on one row per sequence: same weight bytes per launch
     w2_us = 1e3 * ms_w2 / max(1, n_w2)
-    achieved = w2_bytes / (w2_us * 1e-6) / 1e9
-    roofline = {"bound": "hbm", "kernel": "head output layers (k*d_model x k*d_hidden weights, + residual)",
-                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "peak_kind": f"of {peak_kind}", "traffic": None,
-                "bytes_per_launch": w2_bytes, "us_per_launch": w2_us, "launches_timed": n_w2}
+    if w.batch < 16:
+        achieved = w2_bytes / (w2_us * 1e-6) / 1e9
+        roofline = {"bound": "hbm", "kernel": "head output layers (k*d_model x k*d_hidden weights, + residual)",
+                    "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                    "peak_kind": f"of {peak_kind}", "traffic": TRAFFIC.get(args.workload),
+                    "bytes_per_launch": w2_bytes, "us_per_launch": w2_us, "launches_timed": n_w2}
+    else:
+        # batched: the same kernel is a dense contraction; flops of the iterations (the one priming launch
+        # per decode has 1/k of the rows and is left in the average)
+        flops = 2.0 * (w.batch * k) * (w2_bytes / cfg.elem_bytes)
+        achieved = flops / (w2_us * 1e-6) / 1e12
+        roofline = {"bound": "tensor", "kernel": "head output layers (k*d_model x k*d_hidden weights, + residual)",
+                    "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf,
+                    "peak_kind": f"of {peak_kind} (sustained bf16)", "traffic": None,
+                    "flops_per_launch": flops, "us_per_launch": w2_us, "launches_timed": n_w2}
     phase_us = {name: (1e3 * ms / max(1, n)) for name, (n, ms) in
                 zip(["layers", "head_hidden", "head_output", "vocab_top1"], phases)}
+    kernel_names = ["embed", "layer_norm", "qkv", "self_attn", "o_proj", "cross_q", "cross_attn", "cross_o",
+                    "ffn1", "ffn2", "verify"]
+    kernel_us = {}
+    for i, name in enumerate(kernel_names):
+        n, ms = sess.bpd_profile_read(4 + i)
+        if n:
+            kernel_us[name] = {"launches_per_pass": n / max(1, phases[0][0]), "us_per_launch": 1e3 * ms / n}
+    sess.bpd_profile(False)
 
     # ---- other modes (context): greedy, free-running blockwise, mean-2 acceptance
     extra = {}
@@ -263,20 +292,23 @@ def run_gpu(args):
         sess.bpd_encode(src, src_len)
         timed_decodes(1, "greedy")
         ms_g = timed_decodes(max(1, args.steps // 2), "greedy")
-        extra["greedy"] = {"tokens_per_s": N / (ms_g * 1e-3), "us_per_pass": 1e3 * ms_g / N}
+        extra["greedy"] = {"tokens_per_s": w.batch * N / (ms_g * 1e-3), "us_per_pass": 1e3 * ms_g / N}
         sess.bpd_encode(src, src_len)
         timed_decodes(1, "block")
         ms_f = timed_decodes(max(1, args.steps // 2), "block")
         _, _, st_f = sess.bpd_fetch_output(N)
-        extra["blockwise_free"] = {"tokens_per_s": N / (ms_f * 1e-3), "us_per_iteration": 1e3 * ms_f / st_f.iterations,
+        extra["blockwise_free"] = {"tokens_per_s": w.batch * N / (ms_f * 1e-3),
+                                   "us_per_iteration": 1e3 * ms_f / st_f.iterations,
                                    "mean_block": st_f.mean_block}
         plan2, kh2 = build_plan(w, g_ids, k, 2.0)
         sess.bpd_encode(src, src_len)
         sess.bpd_set_forced_plan(plan2, k)
         timed_decodes(1, "block")
         ms_2 = timed_decodes(max(1, args.steps // 2), "block")
-        extra["controlled_mean2"] = {"tokens_per_s": N / (ms_2 * 1e-3), "us_per_iteration": 1e3 * ms_2 / len(kh2),
-                                     "mean_block": N / len(kh2)}
+        _, _, st_2 = sess.bpd_fetch_output(N)
+        extra["controlled_mean2"] = {"tokens_per_s": w.batch * N / (ms_2 * 1e-3),
+                                     "us_per_iteration": 1e3 * ms_2 / st_2.iterations,
+                                     "mean_block": w.batch * N / len(kh2)}
 
     # ---- end to end through the public calls with host buffers
     sess.bpd_encode(src, src_len)
@@ -303,19 +335,20 @@ def run_gpu(args):
         cpu = {"value": tps, "unit": "tokens/s", "cores": threads, "kind": "oracle",
                "sample": f"first {n_tok} of {N} tokens, 2 decodes, {np.mean(times):.1f} s each"}
     line = {
-        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+        "metric": METRIC if args.workload == HEADLINE else f"decoded tokens/s ({args.workload})",
+        "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"{HEADLINE}: big enc-dec 6+6, d_model 1024, 16 heads, FFN 4096, vocab 32768, "
-                               f"k=8 dense heads, batch 1, source 40 ids, decode {N} tokens, controlled acceptance "
-                               f"(geometric mean {MEAN_ACCEPT}, mean accepted block {N / len(khats):.2f})",
-                   "l2": "weights (847 MB per iteration) exceed L2; no flush needed",
+        "config": {"workload": f"{DESCRIPTIONS[args.workload]}, decode {N} tokens, controlled acceptance "
+                               f"(geometric mean {MEAN_ACCEPT}, mean accepted block {w.batch * N / len(khats):.2f})",
+                   "l2": f"weights streamed per iteration ({it_bytes / 1e6:.0f} MB) "
+                         + ("exceed L2; no flush needed" if it_bytes > 126e6 else "fit in L2: numbers are L2-warm"),
                    "replicas": world},
         "us_per_iteration": us_iter, "iterations_per_step": iters,
         "iteration_hbm_gbs": it_bytes / (us_iter * 1e-6) / 1e9,
         "iteration_frac_of_8tbs": it_bytes / (us_iter * 1e-6) / 1e9 / NOMINAL_HBM_GBS,
         "iteration_frac_of_measured": it_bytes / (us_iter * 1e-6) / 1e9 / peak,
-        "phase_us": phase_us, "modes": extra,
+        "phase_us": phase_us, "kernel_us_eager": kernel_us, "modes": extra,
         "clocks": clocks.summary(),
         "e2e": {"value": world * w.batch * N / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
@@ -334,6 +367,7 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=HEADLINE, choices=sorted(DESCRIPTIONS), help="configuration to time")
     ap.add_argument("--quick", action="store_true", help="skip the context modes")
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle leg")
     args = ap.parse_args()

@@ -168,7 +168,11 @@ long long bpd_kernel_launches(void);
  * the session's stream; bpd_profile(s, 0) stops.  bpd_profile_read returns how
  * many times `phase` ran and the summed device time.  Phases: 0 = embedding,
  * decoder layers and final norm; 1 = head hidden layer; 2 = head output layers
- * (+ residual); 3 = vocabulary projection with top-1. */
+ * (+ residual); 3 = vocabulary projection with top-1; for bf16 models also the
+ * individual kernels inside phase 0: 4 = embedding, 5 = layer norms, 6 = QKV
+ * projection, 7 = self-attention, 8 = output projection, 9 = cross-attention
+ * query projection, 10 = cross-attention, 11 = cross-attention output
+ * projection, 12 / 13 = feed-forward layers 1 / 2, 14 = verify and commit. */
 int bpd_profile(bpd_session* s, int enable);
 int bpd_profile_read(bpd_session* s, int phase, int64_t* launches, double* total_ms);
 

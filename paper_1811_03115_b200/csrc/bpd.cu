@@ -214,9 +214,9 @@ static LinearParams lin(const void* x, long long ldx, const void* w, int K, int 
 
 template <typename WT, typename AT>
 static void launch_ln(const float* x, const void* g, const void* b, void* y, float* y32, int rows, int d, float eps,
-                      const int* all_done, cudaStream_t st, long long plane = 0) {
+                      const int* all_done, cudaStream_t st, long long plane = 0, bool pdl = false) {
   LnParams p{x, g, b, y, plane, y32, rows, d, eps, all_done};
-  layernorm_kernel<WT, AT><<<ceil_div(rows, 4), 128, 0, st>>>(p);
+  launch_k(layernorm_kernel<WT, AT>, dim3(ceil_div(rows, 4)), dim3(128), 0, st, pdl, p);
   ++g_launches;
 }
 
@@ -446,6 +446,7 @@ static int run_encoder_tc(bpd_session* s) {
   return BPD_OK;
 }
 
+#define PROF(slot, ...) do { prof_mark(s, slot, 0); __VA_ARGS__; prof_mark(s, slot, 1); } while (0)
 static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   const bpd_model* m = s->m;
   const Config& c = m->cfg;
@@ -453,13 +454,14 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   const int d = c.d, f = c.d_ff, R = s->B * a.kcur, R2 = R * a.kh;
   const int* done = s->st.all_done;
   const tc::Scratch sc = tc_scratch(s);
+  const bool pdl = s->use_pdl != 0;   // every kernel after the first may overlap its predecessor's tail
   prof_mark(s, kProfLayers, 0);
   EmbedParams ep;
   memset(&ep, 0, sizeof(ep));
   ep.table = m->tgt_embed; ep.pe = s->pe; ep.npos = s->npos; ep.x = s->x; ep.rows = R; ep.rows_per_b = a.kcur;
   ep.d = d; ep.vocab = c.V; ep.st = s->st; ep.forced = a.forced; ep.forced_rows = a.forced_rows;
   ep.kforced = a.kforced; ep.src = nullptr; ep.all_done = done;
-  embed_kernel<bf16><<<R, 128, 0, st>>>(ep);
+  PROF(kProfEmbed, embed_kernel<bf16><<<R, 128, 0, st>>>(ep););
   ++g_launches;
   const tc::Operands xn{nullptr, 0, s->xn, s->pl_xn, d, s->rows_all, d};
   const tc::Operands at{nullptr, 0, s->attn, s->pl_attn, d, s->rows_all, d};
@@ -467,40 +469,40 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   auto with_w = [](tc::Operands o, const void* w, int rows) { o.w = w; o.w_rows = rows; return o; };
   for (int l = 0; l < c.n_dec; ++l) {
     const DecLayer& L = m->dec[l];
-    launch_ln<bf16, float>(s->x, L.ln1g, L.ln1b, s->xn, nullptr, R, d, c.eps, done, st, s->pl_xn);
+    PROF(kProfLn, launch_ln<bf16, float>(s->x, L.ln1g, L.ln1b, s->xn, nullptr, R, d, c.eps, done, st, s->pl_xn, pdl););
     tc::TcParams pq = tc_params(nullptr, 0, done);
     pq.out_f32 = static_cast<float*>(s->qbuf); pq.ldo = d; pq.d = d;
     pq.kcache = static_cast<bf16*>(s->kcache[l]); pq.vcache = static_cast<bf16*>(s->vcache[l]);
     pq.st = s->st; pq.rows_per_b = a.kcur;
-    BPD_TRY(tc::launch<tc::kTcQkv>(with_w(xn, L.wqkv, 3 * d), 3 * d, d, R, pq, sc, st)); ++g_launches;
+    PROF(kProfQkv, BPD_TRY(tc::launch<tc::kTcQkv>(with_w(xn, L.wqkv, 3 * d), 3 * d, d, R, pq, sc, st, 1, 0, 0, pdl)); ++g_launches);
     AttnParams ap;
     memset(&ap, 0, sizeof(ap));
     ap.q = s->qbuf; ap.ldq = d; ap.out = s->attn; ap.ldo = d; ap.out_plane = s->pl_attn; ap.rows = R;
     ap.rows_per_b = a.kcur; ap.H = c.H; ap.dh = d / c.H; ap.causal = 1; ap.k = s->kcache[l]; ap.v = s->vcache[l];
     ap.ldkv = d; ap.paged = 1; ap.st = s->st; ap.scale = 1.0f / sqrtf((float)ap.dh); ap.all_done = done;
-    launch_attention<float, bf16>(ap, st);
+    PROF(kProfSelfAttn, launch_attention<float, bf16>(ap, st, pdl););
     ++g_launches;
     tc::TcParams po = tc_params(nullptr, 0, done);
     po.out_f32 = s->x; po.ldo = d;
-    BPD_TRY(tc::launch<tc::kTcResidual>(with_w(at, L.wo, d), d, d, R, po, sc, st)); ++g_launches;
-    launch_ln<bf16, float>(s->x, L.ln2g, L.ln2b, s->xn, nullptr, R, d, c.eps, done, st, s->pl_xn);
+    PROF(kProfOproj, BPD_TRY(tc::launch<tc::kTcResidual>(with_w(at, L.wo, d), d, d, R, po, sc, st, 1, 0, 0, pdl)); ++g_launches);
+    PROF(kProfLn, launch_ln<bf16, float>(s->x, L.ln2g, L.ln2b, s->xn, nullptr, R, d, c.eps, done, st, s->pl_xn, pdl););
     tc::TcParams pc = tc_params(nullptr, 0, done);
     pc.out_f32 = static_cast<float*>(s->qbuf); pc.ldo = d;
-    BPD_TRY(tc::launch<tc::kTcF32>(with_w(xn, L.cwq, d), d, d, R, pc, sc, st)); ++g_launches;
+    PROF(kProfCrossQ, BPD_TRY(tc::launch<tc::kTcF32>(with_w(xn, L.cwq, d), d, d, R, pc, sc, st, 1, 0, 0, pdl)); ++g_launches);
     ap.causal = 0; ap.limit_b = s->st.src_len; ap.k = s->crosskv[l]; ap.v = static_cast<float*>(s->crosskv[l]) + d;
     ap.ldkv = 2 * d; ap.bstride = (long long)s->max_src * 2 * d; ap.paged = 0;
-    launch_attention<float, float>(ap, st);
+    PROF(kProfCrossAttn, launch_attention<float, float>(ap, st, pdl););
     ++g_launches;
-    BPD_TRY(tc::launch<tc::kTcResidual>(with_w(at, L.cwo, d), d, d, R, po, sc, st)); ++g_launches;
-    launch_ln<bf16, float>(s->x, L.ln3g, L.ln3b, s->xn, nullptr, R, d, c.eps, done, st, s->pl_xn);
+    PROF(kProfCrossO, BPD_TRY(tc::launch<tc::kTcResidual>(with_w(at, L.cwo, d), d, d, R, po, sc, st, 1, 0, 0, pdl)); ++g_launches);
+    PROF(kProfLn, launch_ln<bf16, float>(s->x, L.ln3g, L.ln3b, s->xn, nullptr, R, d, c.eps, done, st, s->pl_xn, pdl););
     tc::TcParams p1 = tc_params(L.b1, 1, done);
     p1.out_hi = static_cast<bf16*>(s->ffh); p1.plane = s->pl_ffh; p1.ldo = f;
-    BPD_TRY(tc::launch<tc::kTcPlanes>(with_w(xn, L.w1, f), f, d, R, p1, sc, st)); ++g_launches;
+    PROF(kProfFfn1, BPD_TRY(tc::launch<tc::kTcPlanes>(with_w(xn, L.w1, f), f, d, R, p1, sc, st, 1, 0, 0, pdl)); ++g_launches);
     tc::TcParams p2 = tc_params(L.b2, 0, done);
     p2.out_f32 = s->x; p2.ldo = d;
-    BPD_TRY(tc::launch<tc::kTcResidual>(with_w(fx, L.w2, d), d, f, R, p2, sc, st)); ++g_launches;
+    PROF(kProfFfn2, BPD_TRY(tc::launch<tc::kTcResidual>(with_w(fx, L.w2, d), d, f, R, p2, sc, st, 1, 0, 0, pdl)); ++g_launches);
   }
-  launch_ln<bf16, float>(s->x, m->dec_lnf_g, m->dec_lnf_b, s->xn, s->h_f32, R, d, c.eps, done, st, s->pl_xn);
+  PROF(kProfLn, launch_ln<bf16, float>(s->x, m->dec_lnf_g, m->dec_lnf_b, s->xn, s->h_f32, R, d, c.eps, done, st, s->pl_xn, pdl););
   prof_mark(s, kProfLayers, 1);
   // proposal heads
   const int fhd = c.d_hidden, km = c.k_model;
@@ -509,7 +511,7 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   prof_mark(s, kProfHeadW1, 0);
   tc::TcParams pu = tc_params(m->head_b1, 1, done);
   pu.out_hi = static_cast<bf16*>(s->u); pu.plane = s->pl_u; pu.ldo = ldu;
-  BPD_TRY(tc::launch<tc::kTcPlanes>(with_w(xn, m->head_w1, km * fhd), hid, d, R, pu, sc, st)); ++g_launches;
+  BPD_TRY(tc::launch<tc::kTcPlanes>(with_w(xn, m->head_w1, km * fhd), hid, d, R, pu, sc, st, 1, 0, 0, pdl)); ++g_launches;
   prof_mark(s, kProfHeadW1, 1);
   prof_mark(s, kProfHeadW2, 0);
   tc::Operands uo{m->head_w2, km * d, s->u, s->pl_u, ldu, s->rows_dec, ldu};
@@ -517,10 +519,10 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   ph.out_hi = static_cast<bf16*>(s->o); ph.plane = s->pl_o; ph.ldo = (long long)a.kh * d;
   ph.h = s->h_f32; ph.d = d; ph.head_identity = c.p1_identity;
   if (c.head_layout == 0) {
-    BPD_TRY(tc::launch<tc::kTcHeadOut>(uo, a.kh * d, km * fhd, R, ph, sc, st));
+    BPD_TRY(tc::launch<tc::kTcHeadOut>(uo, a.kh * d, km * fhd, R, ph, sc, st, 1, 0, 0, pdl));
   } else {
     ph.zofs_n = d;
-    BPD_TRY(tc::launch<tc::kTcHeadOut>(uo, d, fhd, R, ph, sc, st, a.kh, d, fhd));
+    BPD_TRY(tc::launch<tc::kTcHeadOut>(uo, d, fhd, R, ph, sc, st, a.kh, d, fhd, pdl));
   }
   ++g_launches;
   prof_mark(s, kProfHeadW2, 1);
@@ -528,16 +530,17 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   tc::Operands oo{m->out_proj, c.V, s->o, s->pl_o, d, s->rows_head, d};
   tc::TcParams pv = tc_params(nullptr, 0, done);
   pv.out_idx = s->st.table; pv.logits = a.logits_dump;
-  BPD_TRY(tc::launch<tc::kTcArgmax>(oo, c.V, d, R2, pv, sc, st)); ++g_launches;
+  BPD_TRY(tc::launch<tc::kTcArgmax>(oo, c.V, d, R2, pv, sc, st, 1, 0, 0, pdl)); ++g_launches;
   prof_mark(s, kProfVocab, 1);
   VerifyParams vp{s->st, s->B, a.kcur, a.kh, a.knext, a.mode, a.max_new, a.eos};
-  verify_commit_kernel<<<1, 32 * ceil_div(s->B, 32), 0, st>>>(vp);
+  PROF(kProfVerify, launch_k(verify_commit_kernel, dim3(1), dim3(32 * ceil_div(s->B, 32)), 0, st, pdl, vp););
   ++g_launches;
   BPD_CUDA(cudaGetLastError());
   s->invocations += 1;
   return BPD_OK;
 }
 
+#undef PROF
 static int dispatch_eager(bpd_session* s, const PassArgs& a) {
   if (s->tc) return run_pass_tc(s, a);
   return s->m->cfg.dtype == 0 ? run_pass<float>(s, a) : run_pass<bf16>(s, a);
@@ -713,6 +716,7 @@ int bpd_session_create(const bpd_model* model, int batch, int max_src, int max_t
   // the default streams cannot be captured: graphs need a stream of the caller's own
   const bool own_stream = s->stream != nullptr && s->stream != cudaStreamLegacy && s->stream != cudaStreamPerThread;
   s->use_graphs = (own_stream && !getenv("BPD_DISABLE_GRAPHS")) ? 1 : 0;
+  s->use_pdl = getenv("BPD_DISABLE_PDL") ? 0 : 1;
   s->phase = kPhaseCreated; s->plan_len = 0; s->plan_k = 0; s->invocations = 0; s->pinned = nullptr;
   plan_session(model->cfg, batch, max_src, max_tgt, s->base, s);
   // page table: row b's p-th page is physical page p*B + b (rows interleaved in the pool)

@@ -73,6 +73,12 @@ __device__ __forceinline__ void warp_argmax(float& v, int& i) {
   }
 }
 
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may start while
+// its predecessor still runs.  launch_dependents lets the successor start early; wait blocks until the
+// predecessor grids have completed and their writes are visible.  Both are no-ops without the attribute.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Per-row decode state living in the session buffer (device memory).
 struct RowState {
   int* len;        // [B] committed decoder inputs (cache length)

@@ -199,7 +199,7 @@ __global__ void __launch_bounds__(kThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmBh,
                const __grid_constant__ CUtensorMap tmBl, TcParams p, int zslices, int a_rows_per_slice,
                int b_cols_per_slice) {
-  if (p.all_done && *p.all_done) return;
+  pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;      // swizzled tiles need 1024-byte alignment
   uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
@@ -241,10 +241,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   bool ok = true;
 
   if (warp == 0 && lane == 0) {
-    // ---------------- TMA producer
+    // ---------------- TMA producer.  Weights do not depend on the preceding kernel: the first stages'
+    // weight tiles are requested before waiting for it; activations only after.
     const int a_row = slice * a_rows_per_slice + tile * kBM;
-    int issued = 0;
-    for (int it = 0; it < nchunks; ++it) {
+    const int npre = min(nchunks, kStages);
+    for (int it = 0; it < npre; ++it) {
+      mbar_expect_tx(bars + 8 * it, stage_sz);
+      tma_load_2d(base + it * stage_sz, &tmA, bars + 8 * it, (c0 + it) * kBK, a_row);
+    }
+    pdl_wait();
+    const bool skip = p.all_done && *p.all_done;
+    for (int it = 0; it < npre; ++it) {
+      const uint32_t sa = base + it * stage_sz;
+      const int kx = slice * b_cols_per_slice + (c0 + it) * kBK;
+      tma_load_2d(sa + kBM * 128, &tmBh, bars + 8 * it, kx, t0);
+      tma_load_2d(sa + kBM * 128 + bn * 128, &tmBl, bars + 8 * it, kx, t0);
+    }
+    int issued = npre;
+    for (int it = npre; it < nchunks && !skip; ++it) {
       const int s = it % kStages;
       const uint32_t ph = (it / kStages) & 1;
       if (!mbar_wait(bars + 8 * (kStages + s), ph ^ 1)) { ok = false; break; }
@@ -257,15 +271,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       tma_load_2d(sa + kBM * 128, &tmBh, full, slice * b_cols_per_slice + kx, t0);
       tma_load_2d(sa + kBM * 128 + bn * 128, &tmBl, full, slice * b_cols_per_slice + kx, t0);
     }
-    if (!ok) {
-      atomicCAS(p.error, 0, 101);
-      // give the copies already issued a bounded chance to land before this CTA's shared memory goes away
+    if (!ok) atomicCAS(p.error, 0, 101);
+    if (!ok || skip) {
+      // nobody will consume what is in flight: give it a bounded chance to land before shared memory goes away
       for (int it = max(0, issued - kStages); it < issued; ++it) mbar_wait(bars + 8 * (it % kStages), (it / kStages) & 1);
     }
   } else if (warp == 1 && lane == 0) {
     // ---------------- MMA issuer
     const uint32_t idesc = instr_desc_bf16(bn);
-    for (int it = 0; it < nchunks; ++it) {
+    pdl_wait();
+    const bool skip = p.all_done && *p.all_done;
+    for (int it = 0; it < nchunks && !skip; ++it) {
       const int s = it % kStages;
       const uint32_t ph = (it / kStages) & 1;
       if (!mbar_wait(bars + 8 * s, ph)) { ok = false; break; }
@@ -281,7 +297,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
       umma_commit(bars + 8 * (kStages + s));       // frees the stage once these MMAs have read it
     }
-    umma_commit(bars + 8 * 2 * kStages);            // accumulator complete
+    if (!skip) umma_commit(bars + 8 * 2 * kStages);            // accumulator complete
     if (!ok) atomicCAS(p.error, 0, 102);
   } else if (warp >= 2) {
     // ---------------- epilogue: thread = one feature row, registers = tokens
@@ -289,11 +305,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int row = q * 32 + lane;
     const int n = tile * kBM + row;                  // feature index within the slice
     const int et = threadIdx.x - 64;                 // 0..127
+    pdl_wait();
+    const bool skip = p.all_done && *p.all_done;     // same value in every thread: the flag is stable by now
     // one thread waits for the accumulator; the other 127 learn the outcome through the named barrier
     if (et == 0) {
-      bool done = true;
-      if (nchunks > 0) done = mbar_wait(bars + 8 * 2 * kStages, 0);
-      if (!done) atomicCAS(p.error, 0, 103);
+      bool done = !skip;
+      if (nchunks > 0 && !skip) done = mbar_wait(bars + 8 * 2 * kStages, 0);
+      if (!done && !skip) atomicCAS(p.error, 0, 103);
       ctl[3] = done ? 1u : 0u;
     }
     asm volatile("bar.sync 1, 128;" ::: "memory");

@@ -4,6 +4,7 @@
 #include <stdarg.h>
 #include <stdint.h>
 #include <stdio.h>
+#include <string.h>
 
 #include <map>
 #include <string>
@@ -25,6 +26,23 @@ int fail(int code, const char* fmt, ...);
       return bpd::fail(BPD_E_CUDA, "%s failed: %s (%s:%d)", #expr, cudaGetErrorString(e__), \
                        __FILE__, __LINE__);                                              \
   } while (0)
+
+// Launch with (pdl = true) or without the programmatic-stream-serialization attribute: with it the kernel
+// may begin while its predecessor in the stream is still running (it must call pdl_wait() on the device
+// before touching anything the predecessor produces).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
+                            Args&&... args) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
 
 struct Config {
   int dtype, n_enc, n_dec, d, H, d_ff, V, k_model, d_hidden, head_layout, p1_identity;
@@ -73,7 +91,9 @@ struct GraphEntry {
   cudaGraphExec_t exec = nullptr;
 };
 
-enum ProfSlot { kProfLayers = 0, kProfHeadW1 = 1, kProfHeadW2 = 2, kProfVocab = 3, kProfSlots = 4 };
+enum ProfSlot { kProfLayers = 0, kProfHeadW1 = 1, kProfHeadW2 = 2, kProfVocab = 3,
+                kProfEmbed = 4, kProfLn = 5, kProfQkv = 6, kProfSelfAttn = 7, kProfOproj = 8, kProfCrossQ = 9,
+                kProfCrossAttn = 10, kProfCrossO = 11, kProfFfn1 = 12, kProfFfn2 = 13, kProfVerify = 14, kProfSlots = 15 };
 
 enum SessionPhase { kPhaseCreated = 0, kPhaseEncoded = 1, kPhaseBlockwise = 2, kPhaseGreedy = 3 };
 
@@ -112,6 +132,7 @@ struct bpd_session {
   int64_t invocations;
   int profiling;
   int use_graphs;
+  int use_pdl;
   std::map<GraphKey, GraphEntry> graphs;
   std::vector<cudaEvent_t> prof_begin[kProfSlots], prof_end[kProfSlots];
 };

@@ -6,6 +6,7 @@
 // scored inside a block give bit-identical results.
 #pragma once
 #include "common.cuh"
+#include "host.hpp"
 
 namespace bpd {
 
@@ -28,6 +29,8 @@ struct EmbedParams {
 
 template <typename WT>
 __global__ void embed_kernel(EmbedParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
   if (p.all_done && *p.all_done) return;
   const int r = blockIdx.x;
   const int b = r / p.rows_per_b, i = r % p.rows_per_b;
@@ -82,6 +85,8 @@ constexpr int kLnMaxD = 1024;   // the row is held in registers: 8 float4 per la
 
 template <typename WT, typename AT>
 __global__ void __launch_bounds__(128) layernorm_kernel(LnParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
   if (p.all_done && *p.all_done) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = blockIdx.x * 4 + warp;
@@ -203,6 +208,8 @@ __device__ __forceinline__ void linear_epilogue(const LinearParams& p, int z, in
 // only on K, never on the number of rows.
 template <typename WT, typename AT, int EPI>
 __global__ void __launch_bounds__(kLinWarps * 32) linear_kernel(LinearParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
   if (p.all_done && *p.all_done) return;
   __shared__ __align__(16) float xs[kRC][kKT];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -284,6 +291,8 @@ struct AttnParams {
 // max / sum are merged chunk by chunk in position order (fixed order).
 template <typename QT, typename CT>
 __global__ void __launch_bounds__(128) attention_kernel(AttnParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
   if (p.all_done && *p.all_done) return;
   __shared__ float qs[4][128];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -388,6 +397,8 @@ template <> __device__ __forceinline__ void load_n<4>(const bf16* p, float (&o)[
 
 template <typename QT, typename CT, int DH>
 __global__ void __launch_bounds__(kAttnWarps * 32) attention_split_kernel(AttnParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
   if (p.all_done && *p.all_done) return;
   constexpr int DPL = (DH >= 32) ? DH / 32 : 1;       // output dims per lane (contiguous)
   __shared__ float s_q[DH];
@@ -481,14 +492,15 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_split_kernel(AttnPa
 
 // Picks the split kernel for the common head widths, the generic one-warp kernel otherwise.
 template <typename QT, typename CT>
-static void launch_attention(const AttnParams& p, cudaStream_t st) {
+static void launch_attention(const AttnParams& p, cudaStream_t st, bool pdl = false) {
   const int items = p.rows * p.H;
+  const dim3 g(items), b(kAttnWarps * 32);
   switch (p.dh) {
-    case 16: attention_split_kernel<QT, CT, 16><<<items, kAttnWarps * 32, 0, st>>>(p); break;
-    case 32: attention_split_kernel<QT, CT, 32><<<items, kAttnWarps * 32, 0, st>>>(p); break;
-    case 64: attention_split_kernel<QT, CT, 64><<<items, kAttnWarps * 32, 0, st>>>(p); break;
-    case 128: attention_split_kernel<QT, CT, 128><<<items, kAttnWarps * 32, 0, st>>>(p); break;
-    default: attention_kernel<QT, CT><<<(items + 3) / 4, 128, 0, st>>>(p); break;
+    case 16: launch_k(attention_split_kernel<QT, CT, 16>, g, b, 0, st, pdl, p); break;
+    case 32: launch_k(attention_split_kernel<QT, CT, 32>, g, b, 0, st, pdl, p); break;
+    case 64: launch_k(attention_split_kernel<QT, CT, 64>, g, b, 0, st, pdl, p); break;
+    case 128: launch_k(attention_split_kernel<QT, CT, 128>, g, b, 0, st, pdl, p); break;
+    default: launch_k(attention_kernel<QT, CT>, dim3((items + 3) / 4), dim3(128), 0, st, pdl, p); break;
   }
 }
 
@@ -508,6 +520,8 @@ constexpr int kArgmaxMaxD = 1024;
 
 template <typename WT, typename AT>
 __global__ void __launch_bounds__(kLinWarps * 32) vocab_argmax_kernel(ArgmaxParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
   if (p.all_done && *p.all_done) return;
   extern __shared__ __align__(16) float xs_dyn[];   // [kRC][d]
   __shared__ float sv[kLinWarps][kRC];
@@ -620,6 +634,8 @@ struct VerifyParams {
 };
 
 static __global__ void verify_commit_kernel(VerifyParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
   if (*p.st.all_done) return;
   __shared__ int any_open;
   if (threadIdx.x == 0) any_open = 0;

@@ -111,7 +111,7 @@ struct Operands {
 
 template <int EPI>
 int launch(const Operands& op, int N, int K, int T, TcParams p, const Scratch& sc, cudaStream_t st, int zslices = 1,
-           int a_rows_per_slice = 0, int b_cols_per_slice = 0) {
+           int a_rows_per_slice = 0, int b_cols_per_slice = 0, bool pdl = false) {
   static bool attr_set = false;
   if (!attr_set) {
     BPD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(kMaxBN)));
@@ -135,8 +135,8 @@ int launch(const Operands& op, int N, int K, int T, TcParams p, const Scratch& s
   p.ws = sc.ws; p.tile_counters = sc.tile_counters; p.done_counter = sc.done_counter;
   p.part_val = sc.part_val; p.part_idx = sc.part_idx; p.error = sc.error;
   dim3 grid(pl.tiles, pl.splits, ttiles * zslices);
-  gemm_tc_kernel<EPI><<<grid, kThreads, smem_bytes(bn), st>>>(ma, mh, ml, p, zslices, a_rows_per_slice, b_cols_per_slice);
-  BPD_CUDA(cudaGetLastError());
+  BPD_CUDA(launch_k(gemm_tc_kernel<EPI>, grid, dim3(kThreads), smem_bytes(bn), st, pdl, ma, mh, ml, p, zslices,
+                    a_rows_per_slice, b_cols_per_slice));
   return BPD_OK;
 }
 
