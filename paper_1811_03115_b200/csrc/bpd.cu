@@ -179,12 +179,13 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
   float* tc_ws = a.take<float>(ws);
   unsigned* tc_counters = a.take<unsigned>(ncnt);
   unsigned* tc_done = a.take<unsigned>(1);
+  unsigned long long* tc_best = a.take<unsigned long long>(R2);
   if (s) {
     s->x = x; s->h_f32 = h_f32; s->xn = xn; s->qbuf = qbuf; s->attn = attn; s->ffh = ffh; s->u = u; s->o = o;
     s->crosskv = crosskv; s->kcache = kc; s->vcache = vc; s->st = st; s->src_dev = src_dev;
     s->tail_dev = tail_dev; s->plan_dev = plan_dev; s->part_val = part_val; s->part_idx = part_idx;
     s->counters = counters; s->ppr = ppr; s->part_elems = tiles * R2; s->pe = pe; s->npos = (int)npos;
-    s->tc_ws = tc_ws; s->tc_ws_floats = ws; s->tc_counters = tc_counters; s->tc_n_counters = ncnt; s->tc_done = tc_done;
+    s->tc_ws = tc_ws; s->tc_ws_floats = ws; s->tc_counters = tc_counters; s->tc_n_counters = ncnt; s->tc_done = tc_done; s->tc_best = tc_best; s->tc_best_elems = R2;
     s->pl_xn = (long long)(Rall * d); s->pl_attn = (long long)(Rall * d); s->pl_ffh = (long long)(Rall * c.d_ff);
     s->pl_u = (long long)(Rmax * c.k_model * c.d_hidden); s->pl_o = (long long)(R2 * d);
     s->rows_all = (int)Rall; s->rows_dec = (int)Rmax; s->rows_head = (int)R2;
@@ -192,7 +193,8 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
   return align_up(a.off);
 }
 
-static size_t weight_bytes_for(const ParsedBlob& pb) { return align_up(pb.total); }
+static size_t fold_floats(const Config& c) { return c.dtype == 1 ? (size_t)c.n_dec * 2 * (3 * c.d + c.d + c.d_ff) : 0; }
+static size_t weight_bytes_for(const ParsedBlob& pb) { return align_up(pb.total) + align_up(fold_floats(pb.cfg) * sizeof(float)); }
 
 // ------------------------------------------------------------------ launches
 static std::atomic<long long> g_launches{0};
@@ -380,7 +382,7 @@ static int run_pass(bpd_session* s, const PassArgs& a) {
 static tc::Scratch tc_scratch(bpd_session* s) {
   tc::Scratch sc;
   sc.ws = s->tc_ws; sc.ws_floats = s->tc_ws_floats; sc.tile_counters = s->tc_counters; sc.n_counters = s->tc_n_counters;
-  sc.done_counter = s->tc_done; sc.part_val = s->part_val; sc.part_idx = s->part_idx; sc.part_elems = s->part_elems;
+  sc.done_counter = s->tc_done; sc.best = s->tc_best; sc.best_elems = s->tc_best_elems;
   sc.error = s->st.error;
   return sc;
 }
@@ -454,13 +456,15 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   const int d = c.d, f = c.d_ff, R = s->B * a.kcur, R2 = R * a.kh;
   const int* done = s->st.all_done;
   const tc::Scratch sc = tc_scratch(s);
-  const bool pdl = s->use_pdl != 0;   // every kernel after the first may overlap its predecessor's tail
+  const bool pdl = s->use_pdl != 0;
+  const bool fold = s->fold_ln != 0;   // every kernel after the first may overlap its predecessor's tail
   prof_mark(s, kProfLayers, 0);
   EmbedParams ep;
   memset(&ep, 0, sizeof(ep));
   ep.table = m->tgt_embed; ep.pe = s->pe; ep.npos = s->npos; ep.x = s->x; ep.rows = R; ep.rows_per_b = a.kcur;
   ep.d = d; ep.vocab = c.V; ep.st = s->st; ep.forced = a.forced; ep.forced_rows = a.forced_rows;
   ep.kforced = a.kforced; ep.src = nullptr; ep.all_done = done;
+  if (fold) { ep.gain = static_cast<const bf16*>(m->dec[0].ln1g); ep.xg_hi = static_cast<bf16*>(s->xn); ep.xg_plane = s->pl_xn; }
   PROF(kProfEmbed, embed_kernel<bf16><<<R, 128, 0, st>>>(ep););
   ++g_launches;
   const tc::Operands xn{nullptr, 0, s->xn, s->pl_xn, d, s->rows_all, d};
@@ -469,11 +473,12 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   auto with_w = [](tc::Operands o, const void* w, int rows) { o.w = w; o.w_rows = rows; return o; };
   for (int l = 0; l < c.n_dec; ++l) {
     const DecLayer& L = m->dec[l];
-    PROF(kProfLn, launch_ln<bf16, float>(s->x, L.ln1g, L.ln1b, s->xn, nullptr, R, d, c.eps, done, st, s->pl_xn, pdl););
+    if (!fold) PROF(kProfLn, launch_ln<bf16, float>(s->x, L.ln1g, L.ln1b, s->xn, nullptr, R, d, c.eps, done, st, s->pl_xn, pdl););
     tc::TcParams pq = tc_params(nullptr, 0, done);
     pq.out_f32 = static_cast<float*>(s->qbuf); pq.ldo = d; pq.d = d;
     pq.kcache = static_cast<bf16*>(s->kcache[l]); pq.vcache = static_cast<bf16*>(s->vcache[l]);
     pq.st = s->st; pq.rows_per_b = a.kcur;
+    if (fold) { pq.ln_x = s->x; pq.ln_d = d; pq.ln_eps = c.eps; pq.ln_s = L.s_qkv; pq.ln_c = L.c_qkv; }
     PROF(kProfQkv, BPD_TRY(tc::launch<tc::kTcQkv>(with_w(xn, L.wqkv, 3 * d), 3 * d, d, R, pq, sc, st, 1, 0, 0, pdl)); ++g_launches);
     AttnParams ap;
     memset(&ap, 0, sizeof(ap));
@@ -484,22 +489,27 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
     ++g_launches;
     tc::TcParams po = tc_params(nullptr, 0, done);
     po.out_f32 = s->x; po.ldo = d;
+    if (fold) { po.g_next = static_cast<const bf16*>(L.ln2g); po.xg_hi = static_cast<bf16*>(s->xn); po.xg_plane = s->pl_xn; }
     PROF(kProfOproj, BPD_TRY(tc::launch<tc::kTcResidual>(with_w(at, L.wo, d), d, d, R, po, sc, st, 1, 0, 0, pdl)); ++g_launches);
-    PROF(kProfLn, launch_ln<bf16, float>(s->x, L.ln2g, L.ln2b, s->xn, nullptr, R, d, c.eps, done, st, s->pl_xn, pdl););
+    if (!fold) PROF(kProfLn, launch_ln<bf16, float>(s->x, L.ln2g, L.ln2b, s->xn, nullptr, R, d, c.eps, done, st, s->pl_xn, pdl););
     tc::TcParams pc = tc_params(nullptr, 0, done);
     pc.out_f32 = static_cast<float*>(s->qbuf); pc.ldo = d;
+    if (fold) { pc.ln_x = s->x; pc.ln_d = d; pc.ln_eps = c.eps; pc.ln_s = L.s_cq; pc.ln_c = L.c_cq; }
     PROF(kProfCrossQ, BPD_TRY(tc::launch<tc::kTcF32>(with_w(xn, L.cwq, d), d, d, R, pc, sc, st, 1, 0, 0, pdl)); ++g_launches);
     ap.causal = 0; ap.limit_b = s->st.src_len; ap.k = s->crosskv[l]; ap.v = static_cast<float*>(s->crosskv[l]) + d;
     ap.ldkv = 2 * d; ap.bstride = (long long)s->max_src * 2 * d; ap.paged = 0;
     PROF(kProfCrossAttn, launch_attention<float, float>(ap, st, pdl););
     ++g_launches;
+    if (fold) po.g_next = static_cast<const bf16*>(L.ln3g);
     PROF(kProfCrossO, BPD_TRY(tc::launch<tc::kTcResidual>(with_w(at, L.cwo, d), d, d, R, po, sc, st, 1, 0, 0, pdl)); ++g_launches);
-    PROF(kProfLn, launch_ln<bf16, float>(s->x, L.ln3g, L.ln3b, s->xn, nullptr, R, d, c.eps, done, st, s->pl_xn, pdl););
+    if (!fold) PROF(kProfLn, launch_ln<bf16, float>(s->x, L.ln3g, L.ln3b, s->xn, nullptr, R, d, c.eps, done, st, s->pl_xn, pdl););
     tc::TcParams p1 = tc_params(L.b1, 1, done);
     p1.out_hi = static_cast<bf16*>(s->ffh); p1.plane = s->pl_ffh; p1.ldo = f;
+    if (fold) { p1.ln_x = s->x; p1.ln_d = d; p1.ln_eps = c.eps; p1.ln_s = L.s_f1; p1.ln_c = L.c_f1; }
     PROF(kProfFfn1, BPD_TRY(tc::launch<tc::kTcPlanes>(with_w(xn, L.w1, f), f, d, R, p1, sc, st, 1, 0, 0, pdl)); ++g_launches);
     tc::TcParams p2 = tc_params(L.b2, 0, done);
     p2.out_f32 = s->x; p2.ldo = d;
+    if (fold && l + 1 < c.n_dec) { p2.g_next = static_cast<const bf16*>(m->dec[l + 1].ln1g); p2.xg_hi = static_cast<bf16*>(s->xn); p2.xg_plane = s->pl_xn; }
     PROF(kProfFfn2, BPD_TRY(tc::launch<tc::kTcResidual>(with_w(fx, L.w2, d), d, f, R, p2, sc, st, 1, 0, 0, pdl)); ++g_launches);
   }
   PROF(kProfLn, launch_ln<bf16, float>(s->x, m->dec_lnf_g, m->dec_lnf_b, s->xn, s->h_f32, R, d, c.eps, done, st, s->pl_xn, pdl););
@@ -687,6 +697,23 @@ int bpd_load_weights(const void* blob, size_t blob_bytes, void* dev_weight_buf, 
   T("head.b2", m->head_b2, k * d)
 #undef T
   cudaError_t e = cudaMemcpyAsync(m->base, blob, pb.total, cudaMemcpyHostToDevice, m->stream);
+  if (c.dtype == 1 && e == cudaSuccess) {
+    float* fp = reinterpret_cast<float*>(m->base + align_up(pb.total));
+    auto fold = [&](const void* w, const void* g, const void* b, const void* bias, int N, float** s_out, float** c_out) {
+      *s_out = fp; fp += N;
+      *c_out = fp; fp += N;
+      FoldParams p{static_cast<const bf16*>(w), static_cast<const bf16*>(g), static_cast<const bf16*>(b),
+                   static_cast<const bf16*>(bias), *s_out, *c_out, N, d};
+      fold_ln_kernel<<<ceil_div(N, 4), 128, 0, m->stream>>>(p);
+    };
+    for (int l = 0; l < c.n_dec; ++l) {
+      DecLayer& L = m->dec[l];
+      fold(L.wqkv, L.ln1g, L.ln1b, nullptr, 3 * d, &L.s_qkv, &L.c_qkv);
+      fold(L.cwq, L.ln2g, L.ln2b, nullptr, d, &L.s_cq, &L.c_cq);
+      fold(L.w1, L.ln3g, L.ln3b, L.b1, f, &L.s_f1, &L.c_f1);
+    }
+    e = cudaGetLastError();
+  }
   if (e == cudaSuccess) e = cudaStreamSynchronize(m->stream);
   if (e != cudaSuccess) { delete m; return fail(BPD_E_CUDA, "weight upload failed: %s", cudaGetErrorString(e)); }
   *out = m;
@@ -717,6 +744,8 @@ int bpd_session_create(const bpd_model* model, int batch, int max_src, int max_t
   const bool own_stream = s->stream != nullptr && s->stream != cudaStreamLegacy && s->stream != cudaStreamPerThread;
   s->use_graphs = (own_stream && !getenv("BPD_DISABLE_GRAPHS")) ? 1 : 0;
   s->use_pdl = getenv("BPD_DISABLE_PDL") ? 0 : 1;
+  // with at most 16 rows per pass every projection CTA can afford the row statistics itself
+  s->fold_ln = (s->tc && batch * model->cfg.k_model <= 16 && !getenv("BPD_DISABLE_FOLD")) ? 1 : 0;
   s->phase = kPhaseCreated; s->plan_len = 0; s->plan_k = 0; s->invocations = 0; s->pinned = nullptr;
   plan_session(model->cfg, batch, max_src, max_tgt, s->base, s);
   // page table: row b's p-th page is physical page p*B + b (rows interleaved in the pool)
@@ -986,13 +1015,13 @@ static OpScratch op_scratch_layout(int rows, int in_f, int out_f) {
   auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + bytes); return at; };
   o.ws_floats = tc::ws_floats(out_f, in_f, rows, 1);
   o.n_counters = tc::counters_needed(out_f, rows, 1);
-  o.part_elems = (size_t)ceil_div(out_f, tc::kBM) * rows;
+  o.part_elems = (size_t)rows;
   o.zero_off = take((size_t)rows * in_f * sizeof(bf16));
   o.ws_off = take(o.ws_floats * sizeof(float));
   o.cnt_off = take(o.n_counters * sizeof(unsigned));
   o.done_off = take(sizeof(unsigned));
-  o.pv_off = take(o.part_elems * sizeof(float));
-  o.pi_off = take(o.part_elems * sizeof(int));
+  o.pv_off = take(o.part_elems * sizeof(unsigned long long));
+  o.pi_off = o.pv_off;
   o.err_off = take(sizeof(int));
   o.total = off;
   return o;
@@ -1028,8 +1057,8 @@ int bpd_op_vocab_argmax(const void* x, const void* w, int rows, int d, int vocab
     const OpScratch L = op_scratch_layout(rows, d, vocab);
     BPD_CUDA(cudaMemsetAsync(p, 0, L.total, st));
     tc::Scratch sc{reinterpret_cast<float*>(p + L.ws_off), L.ws_floats, reinterpret_cast<unsigned*>(p + L.cnt_off),
-                   L.n_counters, reinterpret_cast<unsigned*>(p + L.done_off), reinterpret_cast<float*>(p + L.pv_off),
-                   reinterpret_cast<int*>(p + L.pi_off), L.part_elems, reinterpret_cast<int*>(p + L.err_off)};
+                   L.n_counters, reinterpret_cast<unsigned*>(p + L.done_off),
+                   reinterpret_cast<unsigned long long*>(p + L.pv_off), L.part_elems, reinterpret_cast<int*>(p + L.err_off)};
     const long long plane = (reinterpret_cast<const bf16*>(p + L.zero_off) - static_cast<const bf16*>(x));
     tc::Operands op{w, vocab, x, plane, d, rows, d};
     tc::TcParams tp;
@@ -1073,8 +1102,8 @@ int bpd_op_linear(const void* x, const void* w, const void* bias, int rows, int 
     char* p = static_cast<char*>(scratch);
     BPD_CUDA(cudaMemsetAsync(p, 0, L.total, st));
     tc::Scratch sc{reinterpret_cast<float*>(p + L.ws_off), L.ws_floats, reinterpret_cast<unsigned*>(p + L.cnt_off),
-                   L.n_counters, reinterpret_cast<unsigned*>(p + L.done_off), reinterpret_cast<float*>(p + L.pv_off),
-                   reinterpret_cast<int*>(p + L.pi_off), L.part_elems, reinterpret_cast<int*>(p + L.err_off)};
+                   L.n_counters, reinterpret_cast<unsigned*>(p + L.done_off),
+                   reinterpret_cast<unsigned long long*>(p + L.pv_off), L.part_elems, reinterpret_cast<int*>(p + L.err_off)};
     const long long plane = (reinterpret_cast<const bf16*>(p + L.zero_off) - static_cast<const bf16*>(x));
     tc::Operands op{w, out_f, x, plane, in_f, rows, in_f};
     tc::TcParams tp;

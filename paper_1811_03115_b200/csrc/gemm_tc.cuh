@@ -22,7 +22,7 @@ namespace tc {
 
 constexpr int kBM = 128;          // features per tile (MMA M)
 constexpr int kBK = 64;           // K elements per pipeline stage (128 bytes of bf16: one swizzle row)
-constexpr int kStages = 4;
+constexpr int kMaxStages = 4;     // pipeline depth is chosen per launch (2..4) so that two CTAs fit on an SM when possible
 constexpr int kThreads = 192;     // warp 0: TMA, warp 1: MMA + tensor-memory allocation, warps 2-5: epilogue
 constexpr int kMaxBN = 128;       // tokens per CTA (MMA N), a multiple of 16
 constexpr unsigned long long kSpinCycles = 2000000000ull;   // about a second
@@ -55,9 +55,15 @@ struct TcParams {
   float* ws;                   // [z][tile][split][bn][128]
   unsigned* tile_counters;     // [z][tiles]
   // top-1
-  float* part_val; int* part_idx;   // [tiles][T]
+  unsigned long long* best;         // [T] packed (orderable value, ~index), zero between launches
   unsigned* done_counter;           // [1]
   int* out_idx; float* out_val; float* logits;
+  // layer norm folded into the projection: the activation planes hold x * gain (not normalised); the
+  // epilogue finishes y = rstd * (acc - mean * ln_s[n]) + ln_c[n] with per-token statistics of ln_x
+  const float* ln_x; int ln_d; float ln_eps;   // residual stream [rows, ln_d] fp32, or null
+  const float* ln_s; const float* ln_c;        // [N]: sum_c gain_c w[n][c]  and  sum_c shift_c w[n][c] + bias[n]
+  // kTcResidual: also write planes of the updated stream times the next layer norm's gain
+  const bf16* g_next; bf16* xg_hi; long long xg_plane;
   int* error;                  // device error word
   const int* all_done;
 };
@@ -143,6 +149,18 @@ __device__ __forceinline__ uint32_t instr_desc_bf16(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
 }
 
+// (value, index) packed so that an unsigned 64-bit max picks the larger value and, among equal values, the
+// lower index.  Zero is below every real entry.
+__device__ __forceinline__ unsigned long long pack_best(float v, int idx) {
+  const unsigned b = __float_as_uint(v);
+  const unsigned ord = (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+  return ((unsigned long long)ord << 32) | (unsigned long long)(0xffffffffu - (unsigned)idx);
+}
+__device__ __forceinline__ float unpack_value(unsigned long long key) {
+  const unsigned ord = (unsigned)(key >> 32);
+  return __uint_as_float((ord & 0x80000000u) ? (ord & 0x7fffffffu) : ~ord);
+}
+
 __device__ __forceinline__ void split_bf16(float v, bf16& hi, bf16& lo) {
   hi = __float2bfloat16_rn(v);
   lo = __float2bfloat16_rn(v - __bfloat162float(hi));
@@ -150,12 +168,14 @@ __device__ __forceinline__ void split_bf16(float v, bf16& hi, bf16& lo) {
 
 // Shared-memory footprint of one CTA.
 __host__ __device__ inline size_t stage_bytes(int bn) { return (size_t)kBM * 128 + 2 * (size_t)bn * 128; }
-__host__ __device__ inline size_t smem_bytes(int bn) { return kStages * stage_bytes(bn) + 1024 /*alignment*/ + 256; }
+__host__ __device__ inline int stages_for(int bn) { return bn <= 32 ? 4 : (bn <= 64 ? 3 : 4); }
+__host__ __device__ inline size_t smem_bytes(int bn) { return stages_for(bn) * stage_bytes(bn) + 1024 /*alignment*/ + 256; }
 
 // ---------------------------------------------------------------- final epilogue for one (feature, token)
 template <int EPI>
-__device__ __forceinline__ void tc_store(const TcParams& p, int z, int t, int n, float v) {
-  if (p.bias) v += __bfloat162float(p.bias[n + p.zofs_n * z]);
+__device__ __forceinline__ void tc_store(const TcParams& p, int z, int t, int n, float v, float mean, float rstd) {
+  if (p.ln_x) v = rstd * (v - mean * p.ln_s[n]) + p.ln_c[n];
+  else if (p.bias) v += __bfloat162float(p.bias[n + p.zofs_n * z]);
   if (p.relu) v = fmaxf(v, 0.f);
   if (EPI == kTcPlanes) {
     bf16 hi, lo;
@@ -166,7 +186,14 @@ __device__ __forceinline__ void tc_store(const TcParams& p, int z, int t, int n,
   } else if (EPI == kTcF32) {
     p.out_f32[(long long)t * p.ldo + n] = v;
   } else if (EPI == kTcResidual) {
-    p.out_f32[(long long)t * p.ldo + n] += v;
+    const float xnew = p.out_f32[(long long)t * p.ldo + n] + v;
+    p.out_f32[(long long)t * p.ldo + n] = xnew;
+    if (p.g_next) {
+      bf16 hi, lo;
+      split_bf16(xnew * __bfloat162float(p.g_next[n]), hi, lo);
+      p.xg_hi[(long long)t * p.ldo + n] = hi;
+      p.xg_hi[(long long)t * p.ldo + n + p.xg_plane] = lo;
+    }
   } else if (EPI == kTcHeadOut) {
     const int nz = n + p.zofs_n * z;
     const float hv = p.h[(size_t)t * p.d + (n % p.d)];
@@ -204,6 +231,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;      // swizzled tiles need 1024-byte alignment
   uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
   const int bn = p.bn;
+  const int kStages = stages_for(bn);
   const uint32_t stage_sz = (uint32_t)stage_bytes(bn);
   const uint32_t bars = base + kStages * stage_sz;                   // full[kStages], empty[kStages], accum
   volatile uint32_t* ctl = reinterpret_cast<volatile uint32_t*>(gen_base + kStages * stage_sz + 128);
@@ -211,6 +239,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   // ctl[3] = "the accumulator arrived"
   __shared__ float s_val[4][kMaxBN];
   __shared__ int s_idx[4][kMaxBN];
+  __shared__ float s_mean[16], s_rstd[16];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = blockIdx.x, split = blockIdx.y;
@@ -307,6 +336,33 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int et = threadIdx.x - 64;                 // 0..127
     pdl_wait();
     const bool skip = p.all_done && *p.all_done;     // same value in every thread: the flag is stable by now
+    if (p.ln_x && !skip) {
+      // per-token mean and 1/std of the residual stream, computed while the main loop runs: 8 threads per
+      // token (at most 16 tokens per tile in this mode), two passes, fixed order
+      const int tr = et >> 3, part = et & 7;
+      const int trc = min(tr, nt - 1);               // threads beyond the live tokens shadow the last one
+      const float4* xr = reinterpret_cast<const float4*>(p.ln_x + (size_t)(t0 + trc) * p.ln_d);
+      const int nv = p.ln_d >> 2;
+      float sum = 0.f;
+#pragma unroll 8
+      for (int i = part; i < nv; i += 8) { const float4 a = xr[i]; sum += (a.x + a.y) + (a.z + a.w); }
+      sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+      const float mean = sum / (float)p.ln_d;
+      float sq = 0.f;
+#pragma unroll 8
+      for (int i = part; i < nv; i += 8) {
+        const float4 a = xr[i];
+        const float d0 = a.x - mean, d1 = a.y - mean, d2 = a.z - mean, d3 = a.w - mean;
+        sq += (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
+      }
+      sq += __shfl_xor_sync(0xffffffffu, sq, 1);
+      sq += __shfl_xor_sync(0xffffffffu, sq, 2);
+      sq += __shfl_xor_sync(0xffffffffu, sq, 4);
+      const float rstd = rsqrtf(sq / (float)p.ln_d + p.ln_eps);
+      if (part == 0 && tr < nt) { s_mean[tr] = mean; s_rstd[tr] = rstd; }
+    }
     // one thread waits for the accumulator; the other 127 learn the outcome through the named barrier
     if (et == 0) {
       bool done = !skip;
@@ -328,7 +384,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (EPI != kTcArgmax) {
 #pragma unroll
             for (int c = 0; c < 16; ++c)
-              if (cb + c < nt && n < p.N) tc_store<EPI>(p, slice, t0 + cb + c, n, v[c]);
+              if (cb + c < nt && n < p.N) tc_store<EPI>(p, slice, t0 + cb + c, n, v[c], s_mean[(cb + c) & 15], s_rstd[(cb + c) & 15]);
           } else {
 #pragma unroll
             for (int c = 0; c < 16; ++c) {
@@ -384,7 +440,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int c = 0; c < 8; ++c) {
               if (cg + c >= nt) break;
               if (EPI != kTcArgmax) {
-                if (n < p.N) tc_store<EPI>(p, slice, t0 + cg + c, n, acc[c]);
+                if (n < p.N) tc_store<EPI>(p, slice, t0 + cg + c, n, acc[c], s_mean[(cg + c) & 15], s_rstd[(cg + c) & 15]);
               } else {
                 float x = (n < p.N) ? acc[c] : -INFINITY;
                 int ix = (n < p.N) ? n : 0x7fffffff;
@@ -406,8 +462,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
           for (int w = 1; w < 4; ++w)
             if (better(s_val[w][et], s_idx[w][et], x, ix)) { x = s_val[w][et]; ix = s_idx[w][et]; }
-          p.part_val[(size_t)tile * p.T + t0 + et] = x;
-          p.part_idx[(size_t)tile * p.T + t0 + et] = ix;
+          // one 64-bit atomic max per (tile, token): larger value wins, equal values go to the lower index;
+          // max is order independent, so the result does not depend on which tile arrives first
+          atomicMax(&p.best[t0 + et], pack_best(x, ix));
         }
         __threadfence();
         asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -418,19 +475,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (ctl[2]) {
           __threadfence();
-          for (int t = warp - 2; t < p.T; t += 4) {
-            float x = -INFINITY;
-            int ix = 0x7fffffff;
-            for (int tl = lane; tl < ntiles; tl += 32) {
-              const float tv = __ldcg(&p.part_val[(size_t)tl * p.T + t]);
-              const int ti = __ldcg(&p.part_idx[(size_t)tl * p.T + t]);
-              if (better(tv, ti, x, ix)) { x = tv; ix = ti; }
-            }
-            warp_argmax(x, ix);
-            if (lane == 0) {
-              p.out_idx[t] = ix;
-              if (p.out_val) p.out_val[t] = x;
-            }
+          for (int t = et; t < p.T; t += 128) {
+            const unsigned long long key = __ldcg(&p.best[t]);
+            p.out_idx[t] = (int)(0xffffffffu - (unsigned)(key & 0xffffffffull));
+            if (p.out_val) p.out_val[t] = unpack_value(key);
+            p.best[t] = 0ull;                       // ready for the next launch
           }
           if (et == 0) *p.done_counter = 0;
         }

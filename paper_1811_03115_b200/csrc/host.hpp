@@ -68,6 +68,8 @@ struct EncLayer {
 };
 struct DecLayer {
   const void *ln1g, *ln1b, *wqkv, *wo, *ln2g, *ln2b, *cwq, *cwkv, *cwo, *ln3g, *ln3b, *w1, *b1, *w2, *b2;
+  // layer norms folded into the projections that follow them (bf16 models): per-feature s and c vectors
+  float *s_qkv, *c_qkv, *s_cq, *c_cq, *s_f1, *c_f1;
 };
 
 }  // namespace bpd
@@ -125,6 +127,7 @@ struct bpd_session {
   float* tc_ws; size_t tc_ws_floats;
   unsigned* tc_counters; size_t tc_n_counters;
   unsigned* tc_done;
+  unsigned long long* tc_best; size_t tc_best_elems;
   // host side
   int* pinned;             // pinned ring of all_done flags + staging
   cudaEvent_t ev_flag[8];
@@ -133,6 +136,7 @@ struct bpd_session {
   int profiling;
   int use_graphs;
   int use_pdl;
+  int fold_ln;             // decoder layer norms are folded into the projections (few rows only)
   std::map<GraphKey, GraphEntry> graphs;
   std::vector<cudaEvent_t> prof_begin[kProfSlots], prof_end[kProfSlots];
 };

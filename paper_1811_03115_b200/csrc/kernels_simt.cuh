@@ -24,6 +24,8 @@ struct EmbedParams {
   int kforced;
   // encoder: token = src[b][s], position = s
   const int* src;          // [B][rows_per_b] or null (decoder mode)
+  const bf16* gain;        // optional: also write planes (hi, lo) of x * gain for a projection with a folded layer norm
+  bf16* xg_hi; long long xg_plane;
   const int* all_done;
 };
 
@@ -63,8 +65,57 @@ __global__ void embed_kernel(EmbedParams p) {
     load8(row + c, w);
     load8(pe + c, e);
     float4* out = reinterpret_cast<float4*>(p.x + (size_t)r * p.d + c);
-    out[0] = make_float4(w[0] * scale + e[0], w[1] * scale + e[1], w[2] * scale + e[2], w[3] * scale + e[3]);
-    out[1] = make_float4(w[4] * scale + e[4], w[5] * scale + e[5], w[6] * scale + e[6], w[7] * scale + e[7]);
+    float v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = w[i] * scale + e[i];
+    out[0] = make_float4(v[0], v[1], v[2], v[3]);
+    out[1] = make_float4(v[4], v[5], v[6], v[7]);
+    if (p.gain) {
+      float g[8];
+      load8(p.gain + c, g);
+      bf16 hi[8], lo[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float xg = v[i] * g[i];
+        hi[i] = __float2bfloat16_rn(xg);
+        lo[i] = __float2bfloat16_rn(xg - __bfloat162float(hi[i]));
+      }
+      bf16* dst = p.xg_hi + (size_t)r * p.d + c;
+      *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(hi);
+      *reinterpret_cast<uint4*>(dst + p.xg_plane) = *reinterpret_cast<const uint4*>(lo);
+    }
+  }
+}
+
+// ------------------------------------------------------------------ folding a layer norm into the projection after it
+// LN(x) w^T = rstd * (x*gain) w^T - rstd * mean * s + c   with   s[n] = sum_c gain[c] w[n][c],
+// c[n] = sum_c shift[c] w[n][c] + bias[n].  One warp per output feature, accumulated in double (load time only).
+struct FoldParams {
+  const bf16* w; const bf16* gain; const bf16* shift; const bf16* bias;
+  float* s; float* c;
+  int N, K;
+};
+static __global__ void __launch_bounds__(128) fold_ln_kernel(FoldParams p) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n = blockIdx.x * 4 + warp;
+  if (n >= p.N) return;
+  double ss = 0.0, cc = 0.0;
+  for (int k = lane * 8; k < p.K; k += 256) {
+    float w[8], g[8], b[8];
+    load8(p.w + (size_t)n * p.K + k, w);
+    load8(p.gain + k, g);
+    load8(p.shift + k, b);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) { ss += (double)g[e] * (double)w[e]; cc += (double)b[e] * (double)w[e]; }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    cc += __shfl_xor_sync(0xffffffffu, cc, o);
+  }
+  if (lane == 0) {
+    p.s[n] = (float)ss;
+    p.c[n] = (float)(cc + (p.bias ? (double)__bfloat162float(p.bias[n]) : 0.0));
   }
 }
 

@@ -50,7 +50,7 @@ struct Scratch {
   float* ws; size_t ws_floats;
   unsigned* tile_counters; size_t n_counters;
   unsigned* done_counter;
-  float* part_val; int* part_idx; size_t part_elems;
+  unsigned long long* best; size_t best_elems;
   int* error;
 };
 
@@ -114,7 +114,7 @@ int launch(const Operands& op, int N, int K, int T, TcParams p, const Scratch& s
            int a_rows_per_slice = 0, int b_cols_per_slice = 0, bool pdl = false) {
   static bool attr_set = false;
   if (!attr_set) {
-    BPD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(kMaxBN)));
+    BPD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)std::max(smem_bytes(kMaxBN), smem_bytes(64))));
     attr_set = true;
   }
   const Plan pl = plan_splits(N, K);
@@ -122,7 +122,7 @@ int launch(const Operands& op, int N, int K, int T, TcParams p, const Scratch& s
   const size_t need_ws = ws_floats(N, K, T, zslices), need_cnt = counters_needed(N, T, zslices);
   if (need_ws > sc.ws_floats || need_cnt > sc.n_counters)
     return fail(BPD_E_NOMEM, "split-K workspace too small (%zu floats, %zu counters needed)", need_ws, need_cnt);
-  if (EPI == kTcArgmax && (size_t)pl.tiles * T > sc.part_elems) return fail(BPD_E_NOMEM, "top-1 workspace too small");
+  if (EPI == kTcArgmax && (size_t)T > sc.best_elems) return fail(BPD_E_NOMEM, "top-1 workspace too small");
   CUtensorMap ma, mh, ml;
   int rc = make_map(op.w, (uint64_t)op.w_rows, (uint64_t)K, (uint64_t)K, kBM, &ma);
   if (rc) return rc;
@@ -133,7 +133,7 @@ int launch(const Operands& op, int N, int K, int T, TcParams p, const Scratch& s
   if (rc) return rc;
   p.T = T; p.N = N; p.K = K; p.bn = bn; p.splits = pl.splits; p.chunks_per_split = pl.chunks_per_split;
   p.ws = sc.ws; p.tile_counters = sc.tile_counters; p.done_counter = sc.done_counter;
-  p.part_val = sc.part_val; p.part_idx = sc.part_idx; p.error = sc.error;
+  p.best = sc.best; p.error = sc.error;
   dim3 grid(pl.tiles, pl.splits, ttiles * zslices);
   BPD_CUDA(launch_k(gemm_tc_kernel<EPI>, grid, dim3(kThreads), smem_bytes(bn), st, pdl, ma, mh, ml, p, zslices,
                     a_rows_per_slice, b_cols_per_slice));
