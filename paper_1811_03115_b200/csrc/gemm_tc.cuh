@@ -161,6 +161,14 @@ __device__ __forceinline__ float unpack_value(unsigned long long key) {
   return __uint_as_float((ord & 0x80000000u) ? (ord & 0x7fffffffu) : ~ord);
 }
 
+// Arrival on a device-wide counter with release (our earlier writes, and those of the CTA's other threads
+// ordered before us by the barrier, become visible) and acquire (we see what earlier arrivals released).
+__device__ __forceinline__ unsigned atom_add_acq_rel(unsigned* addr, unsigned v) {
+  unsigned old;
+  asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(addr), "r"(v) : "memory");
+  return old;
+}
+
 __device__ __forceinline__ void split_bf16(float v, bf16& hi, bf16& lo) {
   hi = __float2bfloat16_rn(v);
   lo = __float2bfloat16_rn(v - __bfloat162float(hi));
@@ -172,48 +180,73 @@ __host__ __device__ inline int stages_for(int bn) { return bn <= 32 ? 4 : (bn <=
 __host__ __device__ inline size_t smem_bytes(int bn) { return stages_for(bn) * stage_bytes(bn) + 1024 /*alignment*/ + 256; }
 
 // ---------------------------------------------------------------- final epilogue for one (feature, token)
+// Finishes up to 8 tokens of one feature.  Everything that has to be read (old residual values, the head
+// residual, cache slots) is fetched for all tokens first, so the loads overlap instead of queueing behind
+// the stores of the previous token.
 template <int EPI>
-__device__ __forceinline__ void tc_store(const TcParams& p, int z, int t, int n, float v, float mean, float rstd) {
-  if (p.ln_x) v = rstd * (v - mean * p.ln_s[n]) + p.ln_c[n];
-  else if (p.bias) v += __bfloat162float(p.bias[n + p.zofs_n * z]);
-  if (p.relu) v = fmaxf(v, 0.f);
-  if (EPI == kTcPlanes) {
-    bf16 hi, lo;
-    split_bf16(v, hi, lo);
-    const long long o = (long long)t * p.ldo + n + (long long)p.zofs_n * z;
-    p.out_hi[o] = hi;
-    p.out_hi[o + p.plane] = lo;
-  } else if (EPI == kTcF32) {
-    p.out_f32[(long long)t * p.ldo + n] = v;
-  } else if (EPI == kTcResidual) {
-    const float xnew = p.out_f32[(long long)t * p.ldo + n] + v;
-    p.out_f32[(long long)t * p.ldo + n] = xnew;
-    if (p.g_next) {
-      bf16 hi, lo;
-      split_bf16(xnew * __bfloat162float(p.g_next[n]), hi, lo);
-      p.xg_hi[(long long)t * p.ldo + n] = hi;
-      p.xg_hi[(long long)t * p.ldo + n + p.xg_plane] = lo;
+__device__ __forceinline__ void tc_store8(const TcParams& p, int z, int t_first, int ntok, int n, const float (&vin)[8],
+                                          const float* s_mean, const float* s_rstd, int stat0) {
+  float lns = 0.f, lnc = 0.f, bias = 0.f, gnext = 0.f;
+  if (p.ln_x) { lns = p.ln_s[n]; lnc = p.ln_c[n]; }
+  else if (p.bias) bias = __bfloat162float(p.bias[n + p.zofs_n * z]);
+  if (EPI == kTcResidual && p.g_next) gnext = __bfloat162float(p.g_next[n]);
+  float pre[8];
+  size_t slot[8];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    pre[c] = 0.f;
+    slot[c] = 0;
+    if (c < ntok) {
+      const int t = t_first + c;
+      if (EPI == kTcResidual) pre[c] = p.out_f32[(long long)t * p.ldo + n];
+      if (EPI == kTcHeadOut) pre[c] = p.h[(size_t)t * p.d + (n % p.d)];
+      if (EPI == kTcQkv && n >= p.d) {
+        const int b = t / p.rows_per_b, i = t % p.rows_per_b;
+        const int pos = p.st.len[b] + i;
+        const int page = p.st.page_table[b * p.st.pages_per_row + pos / kPage];
+        slot[c] = ((size_t)page * kPage + (pos % kPage)) * p.d;
+      }
     }
-  } else if (EPI == kTcHeadOut) {
-    const int nz = n + p.zofs_n * z;
-    const float hv = p.h[(size_t)t * p.d + (n % p.d)];
-    v = (p.head_identity && nz < p.d) ? hv : v + hv;
-    bf16 hi, lo;
-    split_bf16(v, hi, lo);
-    const long long o = (long long)t * p.ldo + nz;
-    p.out_hi[o] = hi;
-    p.out_hi[o + p.plane] = lo;
-  } else if (EPI == kTcQkv) {
-    const int d = p.d;
-    if (n < d) {
-      p.out_f32[(long long)t * p.ldo + n] = v;
-    } else {
-      const int b = t / p.rows_per_b, i = t % p.rows_per_b;
-      const int pos = p.st.len[b] + i;
-      const int page = p.st.page_table[b * p.st.pages_per_row + pos / kPage];
-      const size_t slot = ((size_t)page * kPage + (pos % kPage)) * d;
-      if (n < 2 * d) p.kcache[slot + (n - d)] = __float2bfloat16_rn(v);
-      else p.vcache[slot + (n - 2 * d)] = __float2bfloat16_rn(v);
+  }
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    if (c < ntok) {
+      const int t = t_first + c;
+      float v = vin[c];
+      if (p.ln_x) v = s_rstd[(stat0 + c) & 15] * (v - s_mean[(stat0 + c) & 15] * lns) + lnc;
+      else v += bias;
+      if (p.relu) v = fmaxf(v, 0.f);
+      if (EPI == kTcPlanes) {
+        bf16 hi, lo;
+        split_bf16(v, hi, lo);
+        const long long o = (long long)t * p.ldo + n + (long long)p.zofs_n * z;
+        p.out_hi[o] = hi;
+        p.out_hi[o + p.plane] = lo;
+      } else if (EPI == kTcF32) {
+        p.out_f32[(long long)t * p.ldo + n] = v;
+      } else if (EPI == kTcResidual) {
+        const float xnew = pre[c] + v;
+        p.out_f32[(long long)t * p.ldo + n] = xnew;
+        if (p.g_next) {
+          bf16 hi, lo;
+          split_bf16(xnew * gnext, hi, lo);
+          p.xg_hi[(long long)t * p.ldo + n] = hi;
+          p.xg_hi[(long long)t * p.ldo + n + p.xg_plane] = lo;
+        }
+      } else if (EPI == kTcHeadOut) {
+        const int nz = n + p.zofs_n * z;
+        v = (p.head_identity && nz < p.d) ? pre[c] : v + pre[c];
+        bf16 hi, lo;
+        split_bf16(v, hi, lo);
+        const long long o = (long long)t * p.ldo + nz;
+        p.out_hi[o] = hi;
+        p.out_hi[o + p.plane] = lo;
+      } else if (EPI == kTcQkv) {
+        const int d = p.d;
+        if (n < d) p.out_f32[(long long)t * p.ldo + n] = v;
+        else if (n < 2 * d) p.kcache[slot[c] + (n - d)] = __float2bfloat16_rn(v);
+        else p.vcache[slot[c] + (n - 2 * d)] = __float2bfloat16_rn(v);
+      }
     }
   }
 }
@@ -382,9 +415,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           float v[16];
           tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + cb, v);
           if (EPI != kTcArgmax) {
-#pragma unroll
-            for (int c = 0; c < 16; ++c)
-              if (cb + c < nt && n < p.N) tc_store<EPI>(p, slice, t0 + cb + c, n, v[c], s_mean[(cb + c) & 15], s_rstd[(cb + c) & 15]);
+            if (n < p.N) {
+              const float lo8[8] = {v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]};
+              const float hi8[8] = {v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15]};
+              tc_store8<EPI>(p, slice, t0 + cb, min(8, nt - cb), n, lo8, s_mean, s_rstd, cb);
+              tc_store8<EPI>(p, slice, t0 + cb + 8, min(8, nt - cb - 8), n, hi8, s_mean, s_rstd, cb + 8);
+            }
           } else {
 #pragma unroll
             for (int c = 0; c < 16; ++c) {
@@ -409,39 +445,37 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int c = 0; c < 16; ++c)
             if (cb + c < nt) wsz[((size_t)split * bn + cb + c) * kBM + row] = v[c];
         }
-        __threadfence();
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (et == 0) {
-          const unsigned prev = atomicAdd(&p.tile_counters[(size_t)blockIdx.z * ntiles + tile], 1u);
+          const unsigned prev = atom_add_acq_rel(&p.tile_counters[(size_t)blockIdx.z * ntiles + tile], 1u);
           ctl[1] = (prev == (unsigned)p.splits - 1) ? 1u : 0u;
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (ctl[1]) {
-          __threadfence();
-          // splits are added in split order; the loads of four splits x eight tokens are issued together
+          // splits are added in split order; the loads of eight splits x eight tokens are issued together
           for (int cg = 0; cg < nt; cg += 8) {
             float acc[8];
 #pragma unroll
             for (int c = 0; c < 8; ++c) acc[c] = 0.f;
-            for (int s0 = 0; s0 < p.splits; s0 += 4) {
-              float v[4][8];
+            for (int s0 = 0; s0 < p.splits; s0 += 8) {
+              float v[8][8];
 #pragma unroll
-              for (int ss = 0; ss < 4; ++ss)
+              for (int ss = 0; ss < 8; ++ss)
 #pragma unroll
                 for (int c = 0; c < 8; ++c)
                   v[ss][c] = (s0 + ss < p.splits && cg + c < nt)
                                  ? __ldcg(&wsz[((size_t)(s0 + ss) * bn + cg + c) * kBM + row]) : 0.f;
 #pragma unroll
-              for (int ss = 0; ss < 4; ++ss)
+              for (int ss = 0; ss < 8; ++ss)
 #pragma unroll
                 for (int c = 0; c < 8; ++c) acc[c] += v[ss][c];
             }
+            if (EPI != kTcArgmax) {
+              if (n < p.N) tc_store8<EPI>(p, slice, t0 + cg, min(8, nt - cg), n, acc, s_mean, s_rstd, cg);
+            } else {
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-              if (cg + c >= nt) break;
-              if (EPI != kTcArgmax) {
-                if (n < p.N) tc_store<EPI>(p, slice, t0 + cg + c, n, acc[c], s_mean[(cg + c) & 15], s_rstd[(cg + c) & 15]);
-              } else {
+              for (int c = 0; c < 8; ++c) {
+                if (cg + c >= nt) break;
                 float x = (n < p.N) ? acc[c] : -INFINITY;
                 int ix = (n < p.N) ? n : 0x7fffffff;
                 if (p.logits && n < p.N) p.logits[(size_t)(t0 + cg + c) * p.N + n] = x;
@@ -466,15 +500,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           // max is order independent, so the result does not depend on which tile arrives first
           atomicMax(&p.best[t0 + et], pack_best(x, ix));
         }
-        __threadfence();
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (et == 0) {
-          const unsigned prev = atomicAdd(p.done_counter, 1u);
+          const unsigned prev = atom_add_acq_rel(p.done_counter, 1u);
           ctl[2] = (prev == (unsigned)(ntiles * (gridDim.z / zslices)) - 1) ? 1u : 0u;
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (ctl[2]) {
-          __threadfence();
           for (int t = et; t < p.T; t += 128) {
             const unsigned long long key = __ldcg(&p.best[t]);
             p.out_idx[t] = (int)(0xffffffffu - (unsigned)(key & 0xffffffffull));
