@@ -41,24 +41,73 @@ class DecodeResult:
 
 # --------------------------------------------------------------------------- acceptance
 
-def accept_exact(proposal: int, row_p1: Sequence[int]) -> bool:
+class P1View:
+    """What the Verify substep may ask about p_1 at one position: its argmax and,
+    when the logits are known, the rank of any token (number of tokens that beat
+    it; larger logit wins, equal logits go to the lower id)."""
+
+    def __init__(self, argmax: Optional[int] = None, logits: Optional[np.ndarray] = None):
+        self.logits = None if logits is None else np.asarray(logits)
+        self._argmax = int(np.argmax(self.logits)) if argmax is None else int(argmax)
+
+    @property
+    def argmax(self) -> int:
+        return self._argmax
+
+    def rank(self, token: int) -> int:
+        if self.logits is None:
+            return 0 if token == self._argmax else 1 << 30
+        lg = self.logits
+        return int(np.sum(lg > lg[token]) + np.sum(lg[:token] == lg[token]))
+
+
+def _view(x) -> "P1View":
+    return x if isinstance(x, P1View) else P1View(argmax=x[0])
+
+
+def accept_exact(proposal: int, p1) -> bool:
     """Section 3, Verify: the proposal must equal the base model's argmax."""
-    return proposal == row_p1[0]
+    return proposal == _view(p1).argmax
+
+
+def accept_topn(n: int):
+    """Section 5.1: the proposal must lie within the n highest-scoring tokens of p_1."""
+    return lambda proposal, p1: _view(p1).rank(proposal) < n
+
+
+def accept_distance(eps: int):
+    """Section 5.2 with d(u, v) = |u - v| (intensities): the proposal must be within
+    eps of p_1's argmax."""
+    return lambda proposal, p1: abs(int(proposal) - _view(p1).argmax) <= eps
 
 
 def verify_prefix(block: Sequence[int], p1_of: Callable[[int], Sequence[int]],
-                  accept: Callable[[int, Sequence[int]], bool] = accept_exact) -> int:
+                  accept: Callable[[int, Sequence[int]], bool] = accept_exact, min_block: int = 1) -> int:
     """Largest khat such that proposal i is accepted for all 1 <= i <= khat.
 
     ``block[i-1]`` is the proposal for y_{j+i}; ``p1_of(i)`` gives what the
-    acceptance test needs about p_1(y_{j+i} | y_<=j+i-1): a sequence whose first
-    entry is its argmax.  Proposal 1 is p_1's own argmax on the same prefix, so
-    khat >= 1 without testing it.
+    acceptance test needs about p_1(y_{j+i} | y_<=j+i-1): a P1View, or a sequence
+    whose first entry is its argmax.  Proposal 1 is p_1's own argmax on the same
+    prefix, so khat >= 1 without testing it.  ``min_block`` (Section 5.3) forces at
+    least that many proposals to be taken.  Whatever the criterion, the token kept
+    is the proposal (Section 3, Accept), not p_1's argmax.
     """
     khat = 1
-    while khat < len(block) and accept(block[khat], p1_of(khat + 1)):
+    while khat < len(block) and (khat < min_block or accept(block[khat], p1_of(khat + 1))):
         khat += 1
     return khat
+
+
+def p1_views(invoke, table) -> Callable[[int], "P1View"]:
+    """p_1 for y_{j+i} sits at the position of proposal i-1 (row i-2 of the table).
+    Uses the scorer's logits when it keeps them, the argmax ids otherwise."""
+    logits = getattr(invoke, "last_logits", None)
+
+    def of(i: int) -> P1View:
+        if logits is not None:
+            return P1View(argmax=int(table[i - 2][0]), logits=logits[i - 2, 0])
+        return P1View(argmax=int(table[i - 2][0]))
+    return of
 
 
 def clip_termination(block: Sequence[int], khat: int, j: int, n_max: int, eos: int):
@@ -95,7 +144,7 @@ TailFn = Callable[[int, int], Sequence[int]]   # (j accepted so far, iteration i
 
 
 def blockwise_twocall(invoke, k: int, n_max: int, eos: int = -1,
-                      tail_fn: Optional[TailFn] = None, accept=accept_exact) -> DecodeResult:
+                      tail_fn: Optional[TailFn] = None, accept=accept_exact, min_block: int = 1) -> DecodeResult:
     """Section 3 literally: a Predict invocation on the accepted prefix, then a
     Verify invocation on prefix + block; two invocations per iteration."""
     res = DecodeResult(ids=[])
@@ -108,7 +157,7 @@ def blockwise_twocall(invoke, k: int, n_max: int, eos: int = -1,
         table = invoke(inputs + block, k)                                  # Verify
         res.invocations += 2
         # p_1 for y_{j+i} is conditioned on y_<=j+i-1, i.e. sits at the position of proposal i-1
-        khat = verify_prefix(block, lambda i: [table[i - 2][0]], accept)
+        khat = verify_prefix(block, p1_views(invoke, table), accept, min_block)
         khat, finished = clip_termination(block, khat, j, n_max, eos)
         res.ids += block[:khat]
         res.khats.append(khat)
@@ -118,7 +167,7 @@ def blockwise_twocall(invoke, k: int, n_max: int, eos: int = -1,
 
 
 def blockwise_merged(invoke, k: int, n_max: int, eos: int = -1,
-                     tail_fn: Optional[TailFn] = None, accept=accept_exact) -> DecodeResult:
+                     tail_fn: Optional[TailFn] = None, accept=accept_exact, min_block: int = 1) -> DecodeResult:
     """Section 4: the combined model returns all k heads at all k block
     positions, so the row of the last accepted position is the next Predict;
     one priming invocation, then one invocation per iteration."""
@@ -132,7 +181,7 @@ def blockwise_merged(invoke, k: int, n_max: int, eos: int = -1,
             block[1:] = [int(t) for t in tail_fn(j, res.iterations)]
         table = invoke(inputs + block, k)
         res.invocations += 1
-        khat = verify_prefix(block, lambda i: [table[i - 2][0]], accept)
+        khat = verify_prefix(block, p1_views(invoke, table), accept, min_block)
         khat, finished = clip_termination(block, khat, j, n_max, eos)
         res.ids += block[:khat]
         res.khats.append(khat)
