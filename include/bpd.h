@@ -51,10 +51,16 @@ typedef enum {
 typedef struct bpd_model bpd_model;     /* opaque: parsed config + device weight pointers  */
 typedef struct bpd_session bpd_session; /* opaque: B rows of decode state in device memory */
 
-/* Acceptance criteria for the Verify substep. */
+/* Acceptance criteria for the Verify substep (the accept_mode argument).
+ * Whatever the criterion, the token that is kept is the proposal (Section 3,
+ * Accept).  BPD_ACCEPT_MIN_BLOCK(l) may be OR-ed in: at least l proposals are
+ * taken per iteration regardless of the criterion (Section 5.3). */
 enum {
-  BPD_ACCEPT_EXACT = 0     /* Section 3: proposal == argmax p_1 */
+  BPD_ACCEPT_EXACT = 0     /* Section 3: proposal == argmax p_1; the output equals greedy decoding */
 };
+#define BPD_ACCEPT_TOPN(n)       ((1 << 8) | ((n) & 0xff))    /* Section 5.1: proposal among the n best of p_1, 1 <= n <= 255 */
+#define BPD_ACCEPT_DISTANCE(eps) ((2 << 8) | ((eps) & 0xff))  /* Section 5.2: |proposal - argmax p_1| <= eps (intensities)  */
+#define BPD_ACCEPT_MIN_BLOCK(l)  (((l) & 0xff) << 16)         /* Section 5.3: 1 <= l <= k                                   */
 
 #define BPD_MAX_K 16       /* largest block size / number of proposal heads */
 

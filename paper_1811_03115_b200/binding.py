@@ -75,6 +75,18 @@ for _name, (_res, _args) in _SIGS.items():
 EXPORTED = tuple(_SIGS)
 
 
+def BPD_ACCEPT_TOPN(n: int) -> int:
+    return (1 << 8) | (n & 0xff)
+
+
+def BPD_ACCEPT_DISTANCE(eps: int) -> int:
+    return (2 << 8) | (eps & 0xff)
+
+
+def BPD_ACCEPT_MIN_BLOCK(l: int) -> int:
+    return (l & 0xff) << 16
+
+
 def _check(rc: int) -> None:
     if rc != BPD_OK:
         raise BpdError(rc, lib.bpd_last_error().decode(errors="replace"))

@@ -151,6 +151,8 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
   st.all_done = a.take<int>(1); st.error = a.take<int>(1);
   st.stats = a.take<long long>(4 + kMaxK + 1);
   st.page_table = page_table; st.pages_per_row = ppr; st.max_tgt = max_tgt;
+  RankState rank;
+  rank.thr = a.take<float>(Rmax); rank.tok = a.take<int>(Rmax); rank.cnt = a.take<int>(Rmax);
   int* src_dev = a.take<int>(E);
   int* tail_dev = a.take<int>((size_t)B * kMaxK);
   int* plan_dev = a.take<int>((size_t)B * max_tgt * (kMaxK - 1));
@@ -184,6 +186,7 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
     s->x = x; s->h_f32 = h_f32; s->xn = xn; s->qbuf = qbuf; s->attn = attn; s->ffh = ffh; s->u = u; s->o = o;
     s->crosskv = crosskv; s->kcache = kc; s->vcache = vc; s->st = st; s->src_dev = src_dev;
     s->tail_dev = tail_dev; s->plan_dev = plan_dev; s->part_val = part_val; s->part_idx = part_idx;
+    s->rank = rank;
     s->counters = counters; s->ppr = ppr; s->part_elems = tiles * R2; s->pe = pe; s->npos = (int)npos;
     s->tc_ws = tc_ws; s->tc_ws_floats = ws; s->tc_counters = tc_counters; s->tc_n_counters = ncnt; s->tc_done = tc_done; s->tc_best = tc_best; s->tc_best_elems = R2;
     s->pl_xn = (long long)(Rall * d); s->pl_attn = (long long)(Rall * d); s->pl_ffh = (long long)(Rall * c.d_ff);
@@ -225,8 +228,9 @@ static void launch_ln(const float* x, const void* g, const void* b, void* y, flo
 template <typename WT, typename AT>
 static void launch_vocab_argmax(const void* x, const void* w, int rows, int d, int V, float* part_val, int* part_idx,
                                 unsigned* counters, int* out_idx, float* out_val, float* logits, const int* all_done,
-                                cudaStream_t st) {
+                                cudaStream_t st, const RankState* rank = nullptr, int rank_kh = 1) {
   ArgmaxParams p{x, (long long)d, w, rows, d, V, part_val, part_idx, counters, out_idx, out_val, logits, all_done};
+  if (rank) { p.rank = *rank; p.rank_kh = rank_kh; }
   dim3 grid(ceil_div(V, kVocTile), ceil_div(rows, kRC));
   vocab_argmax_kernel<WT, AT><<<grid, kLinWarps * 32, (size_t)kRC * d * sizeof(float), st>>>(p);
   ++g_launches;
@@ -299,7 +303,32 @@ struct PassArgs {
   int forced_rows, kforced;
   int max_new, eos;
   float* logits_dump;   // device [B*kcur*kh, V] or null
+  int accept_kind = kAcceptExact;   // Verify criterion, its parameter (n or eps), forced minimum block size
+  int accept_param = 0;
+  int min_block = 1;
 };
+
+// accept_mode of the public calls: bits 0-7 parameter, bits 8-15 criterion, bits 16-23 minimum block size
+static int decode_accept(int accept_mode, int k, PassArgs* a) {
+  const int param = accept_mode & 0xff, kind = (accept_mode >> 8) & 0xff, minb = (accept_mode >> 16) & 0xff;
+  if (accept_mode < 0 || (accept_mode >> 24)) return fail(BPD_E_INVALID, "acceptance mode 0x%x", accept_mode);
+  if (kind == kAcceptExact) {
+    if (param) return fail(BPD_E_INVALID, "exact acceptance takes no parameter");
+  } else if (kind == kAcceptTopN) {
+    if (param < 1) return fail(BPD_E_INVALID, "top-n acceptance needs n >= 1");
+  } else if (kind != kAcceptDistance) {
+    return fail(BPD_E_UNSUPPORTED, "acceptance criterion %d", kind);
+  }
+  if (minb > k) return fail(BPD_E_INVALID, "minimum block size %d above k = %d", minb, k);
+  a->accept_kind = kind; a->accept_param = param; a->min_block = std::max(1, minb);
+  return BPD_OK;
+}
+
+static VerifyParams verify_params(bpd_session* s, const PassArgs& a) {
+  VerifyParams vp{s->st, s->B, a.kcur, a.kh, a.knext, a.mode, a.max_new, a.eos, a.accept_kind, a.accept_param, a.min_block, s->rank};
+  return vp;
+}
+static bool wants_rank(const PassArgs& a) { return a.mode == kModeBlock && a.accept_kind == kAcceptTopN && a.kcur > 1; }
 
 template <typename WT>
 static int run_pass(bpd_session* s, const PassArgs& a) {
@@ -367,10 +396,15 @@ static int run_pass(bpd_session* s, const PassArgs& a) {
   prof_mark(s, kProfHeadW2, 1);
   // shared vocabulary projection with a fused top-1: table[b][r][i]
   prof_mark(s, kProfVocab, 0);
+  if (wants_rank(a)) {
+    ProposalLogitParams pl{s->o, 0, m->out_proj, s->st, s->rank, s->B, a.kcur, a.kh, d, done};
+    proposal_logit_kernel<WT><<<ceil_div(R, 4), 128, 0, st>>>(pl);
+    ++g_launches;
+  }
   launch_vocab_argmax<WT, float>(s->o, m->out_proj, R2, d, c.V, s->part_val, s->part_idx, s->counters, s->st.table,
-                              nullptr, a.logits_dump, done, st);
+                              nullptr, a.logits_dump, done, st, wants_rank(a) ? &s->rank : nullptr, a.kh);
   prof_mark(s, kProfVocab, 1);
-  VerifyParams vp{s->st, s->B, a.kcur, a.kh, a.knext, a.mode, a.max_new, a.eos};
+  VerifyParams vp = verify_params(s, a);
   verify_commit_kernel<<<1, 32 * ceil_div(s->B, 32), 0, st>>>(vp);
   ++g_launches;
   BPD_CUDA(cudaGetLastError());
@@ -540,9 +574,15 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   tc::Operands oo{m->out_proj, c.V, s->o, s->pl_o, d, s->rows_head, d};
   tc::TcParams pv = tc_params(nullptr, 0, done);
   pv.out_idx = s->st.table; pv.logits = a.logits_dump;
+  if (wants_rank(a)) {
+    ProposalLogitParams pl{s->o, s->pl_o, m->out_proj, s->st, s->rank, s->B, a.kcur, a.kh, d, done};
+    launch_k(proposal_logit_kernel<bf16>, dim3(ceil_div(R, 4)), dim3(128), 0, st, pdl, pl);
+    ++g_launches;
+    pv.rank = s->rank; pv.rank_kh = a.kh;
+  }
   BPD_TRY(tc::launch<tc::kTcArgmax>(oo, c.V, d, R2, pv, sc, st, 1, 0, 0, pdl)); ++g_launches;
   prof_mark(s, kProfVocab, 1);
-  VerifyParams vp{s->st, s->B, a.kcur, a.kh, a.knext, a.mode, a.max_new, a.eos};
+  VerifyParams vp = verify_params(s, a);
   PROF(kProfVerify, launch_k(verify_commit_kernel, dim3(1), dim3(32 * ceil_div(s->B, 32)), 0, st, pdl, vp););
   ++g_launches;
   BPD_CUDA(cudaGetLastError());
@@ -561,7 +601,7 @@ static int dispatch_eager(bpd_session* s, const PassArgs& a) {
 static int dispatch_pass(bpd_session* s, const PassArgs& a) {
   if (s->profiling || !s->use_graphs || a.logits_dump) return dispatch_eager(s, a);
   const GraphKey key(a.mode, a.kcur, a.kh, a.knext, (const void*)a.forced, a.forced_rows, a.kforced, a.max_new, a.eos,
-                     (const void*)a.logits_dump);
+                     (const void*)a.logits_dump, (a.accept_kind << 16) | (a.accept_param << 8) | a.min_block);
   GraphEntry& ge = s->graphs[key];
   if (ge.exec) {
     BPD_CUDA(cudaGraphLaunch(ge.exec, s->stream));
@@ -921,7 +961,8 @@ int bpd_decode_blockwise(bpd_session* s, int k, int accept_mode, int max_new, in
   int rc = check_decode_args(s, max_new, eos_id);
   if (rc) return rc;
   if (k < 1 || k > s->m->cfg.k_model) return fail(BPD_E_INVALID, "k = %d outside 1..%d", k, s->m->cfg.k_model);
-  if (accept_mode != BPD_ACCEPT_EXACT) return fail(BPD_E_UNSUPPORTED, "acceptance mode %d", accept_mode);
+  PassArgs acc{};
+  if ((rc = decode_accept(accept_mode, k, &acc))) return rc;
   if (s->phase != kPhaseEncoded) return fail(BPD_E_STATE, "bpd_decode_blockwise needs a freshly encoded session");
   if (s->plan_len && s->plan_k != k) return fail(BPD_E_SHAPE, "forced plan was installed for k = %d", s->plan_k);
   s->phase = kPhaseBlockwise;
@@ -929,7 +970,8 @@ int bpd_decode_blockwise(bpd_session* s, int k, int accept_mode, int max_new, in
   PassArgs prime{kModePrime, 1, k, k, nullptr, 0, 0, max_new, eos_id, nullptr};
   rc = dispatch_pass(s, prime);
   if (rc) return rc;
-  PassArgs a{kModeBlock, k, k, k, s->plan_len ? s->plan_dev : nullptr, s->plan_len, k, max_new, eos_id, nullptr};
+  PassArgs a{kModeBlock, k, k, k, s->plan_len ? s->plan_dev : nullptr, s->plan_len, k, max_new, eos_id, nullptr,
+             acc.accept_kind, acc.accept_param, acc.min_block};
   rc = decode_loop(s, a, max_new);
   if (rc) return rc;
   return finish_decode(s, max_new, out_ids, out_len, stats);
@@ -940,7 +982,8 @@ int bpd_iteration(bpd_session* s, int k, int accept_mode, int max_new, int32_t e
   int rc = check_decode_args(s, max_new, eos_id);
   if (rc) return rc;
   if (k < 1 || k > s->m->cfg.k_model) return fail(BPD_E_INVALID, "k = %d outside 1..%d", k, s->m->cfg.k_model);
-  if (accept_mode != BPD_ACCEPT_EXACT) return fail(BPD_E_UNSUPPORTED, "acceptance mode %d", accept_mode);
+  PassArgs acc{};
+  if ((rc = decode_accept(accept_mode, k, &acc))) return rc;
   if (s->phase != kPhaseEncoded && s->phase != kPhaseBlockwise) return fail(BPD_E_STATE, "bpd_iteration needs an encoded session that is not decoding greedily");
   const int B = s->B, V = s->m->cfg.V;
   if (forced_tail && k > 1) {
@@ -953,7 +996,8 @@ int bpd_iteration(bpd_session* s, int k, int accept_mode, int max_new, int32_t e
     if (rc) return rc;
     s->phase = kPhaseBlockwise;
   }
-  PassArgs a{kModeBlock, k, k, k, nullptr, 0, 0, max_new, eos_id, out ? out->logits_dev : nullptr};
+  PassArgs a{kModeBlock, k, k, k, nullptr, 0, 0, max_new, eos_id, out ? out->logits_dev : nullptr,
+             acc.accept_kind, acc.accept_param, acc.min_block};
   if (forced_tail && k > 1) {
     BPD_CUDA(cudaStreamSynchronize(s->stream));   // the staging slots may still be in flight
     memcpy(&s->pinned[128], forced_tail, sizeof(int) * B * (k - 1));

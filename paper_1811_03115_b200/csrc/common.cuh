@@ -100,4 +100,15 @@ struct RowState {
 
 enum PassMode { kModePrime = 0, kModeBlock = 1, kModeGreedy = 2 };
 
+// Acceptance criteria of the Verify substep (values match the public header).
+enum AcceptKind { kAcceptExact = 0, kAcceptTopN = 1, kAcceptDistance = 2 };
+
+// Top-n acceptance asks how many vocabulary entries beat each proposal under p_1 at the position before it.
+// Position pr = row * kcur + r (r-th block position) holds proposal r+1's token, its own logit and the count.
+struct RankState {
+  float* thr;   // [B*kcur] logit of the proposal under p_1 at position pr
+  int* tok;     // [B*kcur] the proposal's token id, -1 where there is none (last position of a block)
+  int* cnt;     // [B*kcur] entries that beat it (filled by the vocabulary projection)
+};
+
 }  // namespace bpd

@@ -58,6 +58,7 @@ struct TcParams {
   unsigned long long* best;         // [T] packed (orderable value, ~index), zero between launches
   unsigned* done_counter;           // [1]
   int* out_idx; float* out_val; float* logits;
+  RankState rank; int rank_kh;      // top-n acceptance: count entries beating each proposal (rank.cnt null = off)
   // layer norm folded into the projection: the activation planes hold x * gain (not normalised); the
   // epilogue finishes y = rstd * (acc - mean * ln_s[n]) + ln_c[n] with per-token statistics of ln_x
   const float* ln_x; int ln_d; float ln_eps;   // residual stream [rows, ln_d] fp32, or null
@@ -167,6 +168,15 @@ __device__ __forceinline__ unsigned atom_add_acq_rel(unsigned* addr, unsigned v)
   unsigned old;
   asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(addr), "r"(v) : "memory");
   return old;
+}
+
+// Top-n acceptance: among this warp's 32 features, how many beat the proposal that follows token t's position.
+__device__ __forceinline__ void count_beats(const TcParams& p, int t, int n, float x, int lane) {
+  if (!p.rank.cnt || t >= p.T || (t % p.rank_kh) != 0) return;   // uniform over the warp
+  const int pr = t / p.rank_kh, tok = p.rank.tok[pr];
+  const bool beat = tok >= 0 && n < p.N && n != tok && better(x, n, p.rank.thr[pr], tok);
+  const unsigned m = __ballot_sync(0xffffffffu, beat);
+  if (lane == 0 && m) atomicAdd(&p.rank.cnt[pr], __popc(m));
 }
 
 __device__ __forceinline__ void split_bf16(float v, bf16& hi, bf16& lo) {
@@ -427,6 +437,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               float x = (n < p.N) ? v[c] : -INFINITY;
               int ix = (n < p.N) ? n : 0x7fffffff;
               if (p.logits && cb + c < nt && n < p.N) p.logits[(size_t)(t0 + cb + c) * p.N + n] = x;
+              if (cb + c < nt) count_beats(p, t0 + cb + c, n, x, lane);
               warp_argmax(x, ix);
               if (lane == 0) { s_val[q][cb + c] = x; s_idx[q][cb + c] = ix; }
             }
@@ -479,6 +490,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 float x = (n < p.N) ? acc[c] : -INFINITY;
                 int ix = (n < p.N) ? n : 0x7fffffff;
                 if (p.logits && n < p.N) p.logits[(size_t)(t0 + cg + c) * p.N + n] = x;
+                count_beats(p, t0 + cg + c, n, x, lane);
                 warp_argmax(x, ix);
                 if (lane == 0) { s_val[q][cg + c] = x; s_idx[q][cg + c] = ix; }
               }

@@ -86,7 +86,7 @@ struct bpd_model {
   const void *head_w1, *head_b1, *head_w2, *head_b2;
 };
 
-typedef std::tuple<int, int, int, int, const void*, int, int, int, int, const void*> GraphKey;
+typedef std::tuple<int, int, int, int, const void*, int, int, int, int, const void*, int> GraphKey;
 struct GraphEntry {
   int uses = 0;
   long long launches = 0;
@@ -113,6 +113,7 @@ struct bpd_session {
   std::vector<void*> crosskv, kcache, vcache;
   // integers
   bpd::RowState st;
+  bpd::RankState rank;
   int *src_dev, *tail_dev, *plan_dev;
   int plan_len, plan_k;    // 0 when no plan installed
   // vocabulary top-1 workspace

@@ -555,6 +555,52 @@ static void launch_attention(const AttnParams& p, cudaStream_t st, bool pdl = fa
   }
 }
 
+// ------------------------------------------------------------------ logit of each proposal under p_1 (top-n acceptance)
+struct ProposalLogitParams {
+  const void* o; long long o_plane;   // head outputs [B*kcur*kh, d]: activation dtype, or bf16 planes when o_plane > 0
+  const void* w;                      // [V, d]
+  RowState st;
+  RankState rank;
+  int B, kcur, kh, d;
+  const int* all_done;
+};
+// One warp per block position: thr = o[position, head 1] . w[proposal after it].
+template <typename WT>
+__global__ void __launch_bounds__(128) proposal_logit_kernel(ProposalLogitParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
+  if (p.all_done && *p.all_done) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int pr = blockIdx.x * 4 + warp;
+  if (pr >= p.B * p.kcur) return;
+  const int b = pr / p.kcur, r = pr % p.kcur;
+  int tok = -1;
+  float thr = 0.f;
+  if (r + 1 < p.kcur) {
+    tok = p.st.cur_block[b * kMaxK + r + 1];
+    const WT* wr = reinterpret_cast<const WT*>(p.w) + (size_t)tok * p.d;
+    const size_t row = (size_t)pr * p.kh * p.d;
+    float acc = 0.f;
+    for (int c = lane * 8; c < p.d; c += 256) {
+      float wv[8], ov[8];
+      load8(wr + c, wv);
+      if (p.o_plane) {
+        float lo[8];
+        load8(reinterpret_cast<const bf16*>(p.o) + row + c, ov);
+        load8(reinterpret_cast<const bf16*>(p.o) + row + c + p.o_plane, lo);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) ov[e] += lo[e];
+      } else {
+        load8(reinterpret_cast<const float*>(p.o) + row + c, ov);
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc = fmaf(wv[e], ov[e], acc);
+    }
+    thr = warp_sum(acc);
+  }
+  if (lane == 0) { p.rank.tok[pr] = tok; p.rank.thr[pr] = thr; p.rank.cnt[pr] = 0; }
+}
+
 // ------------------------------------------------------------------ vocabulary projection + top-1
 struct ArgmaxParams {
   const void* x; long long ldx;   // [rows, d] activations
@@ -565,6 +611,7 @@ struct ArgmaxParams {
   int* out_idx; float* out_val;   // [rows]
   float* logits;                  // optional dump [rows, V]
   const int* all_done;
+  RankState rank; int rank_kh;    // top-n acceptance: count entries beating each proposal (rank.cnt null = off)
 };
 constexpr int kVocTile = 256;     // vocabulary rows per CTA
 constexpr int kArgmaxMaxD = 1024;
@@ -633,6 +680,10 @@ __global__ void __launch_bounds__(kLinWarps * 32) vocab_argmax_kernel(ArgmaxPara
       for (int r = 0; r < kRC; ++r) {
         const float v = warp_sum(acc[f][r]);
         if (n0 + f < p.V) {
+          if (p.rank.cnt && lane == 0 && r < nr && (r0 + r) % p.rank_kh == 0) {
+            const int pr = (r0 + r) / p.rank_kh, tok = p.rank.tok[pr];
+            if (tok >= 0 && tok != n0 + f && better(v, n0 + f, p.rank.thr[pr], tok)) atomicAdd(&p.rank.cnt[pr], 1);
+          }
           if (better(v, n0 + f, bv[r], bi[r])) { bv[r] = v; bi[r] = n0 + f; }
           if (p.logits && lane == f * kRC + r && r < nr) p.logits[(size_t)(r0 + r) * p.V + n0 + f] = v;
         }
@@ -682,6 +733,8 @@ struct VerifyParams {
   int B, kcur, kh, knext;   // positions scored per row, heads per position, width of the next block
   int mode;
   int max_new, eos;
+  int accept_kind, accept_param, min_block;   // exact / top-n (n) / distance (eps); forced minimum block size
+  RankState rank;                             // top-n only
 };
 
 static __global__ void verify_commit_kernel(VerifyParams p) {
@@ -722,7 +775,15 @@ static __global__ void verify_commit_kernel(VerifyParams p) {
       // longest prefix of the block that the base model would have produced itself:
       // proposal i+1 is checked against head 1 at the position of proposal i
       int khat = 1;
-      while (khat < p.kcur && cur[khat] == A[(khat - 1) * p.kh]) ++khat;
+      while (khat < p.kcur) {
+        const int top1 = A[(khat - 1) * p.kh];
+        bool okay;
+        if (p.accept_kind == kAcceptTopN) okay = p.rank.cnt[b * p.kcur + khat - 1] < p.accept_param;
+        else if (p.accept_kind == kAcceptDistance) okay = abs(cur[khat] - top1) <= p.accept_param;
+        else okay = (cur[khat] == top1);
+        if (!okay && khat >= p.min_block) break;
+        ++khat;
+      }
       const int j = p.st.j[b];
       khat = min(khat, p.max_new - j);
       int fin = (j + khat >= p.max_new);

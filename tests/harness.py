@@ -61,14 +61,54 @@ def _reconcile(gpu_ids: np.ndarray, logits: np.ndarray, rep: LockstepReport, wha
     return out.reshape(gpu_ids.shape)
 
 
+def _decision(kind, param, proposal: int, top: int, row: np.ndarray):
+    """Oracle's accept decision for one proposal and how far (in logits) it is from flipping."""
+    if kind == "exact":
+        return proposal == top, np.inf
+    if kind == "distance":
+        return abs(proposal - top) <= param, np.inf          # integers once the argmax is agreed
+    # top-n: rank under (logit desc, id asc); the boundary is between the n-th and the (n+1)-th entry
+    order = sorted(range(row.size), key=lambda v: (-row[v], v))
+    rank = order.index(proposal)
+    if rank < param:
+        other = row[order[param]] if param < row.size else -np.inf
+        return True, row[proposal] - other
+    return False, row[order[param - 1]] - row[proposal]
+
+
+def near_miss_tail(scorer_factory, inputs: List[int], p1: int, k: int, it: int, kind: str, vocab: int) -> np.ndarray:
+    """Proposals 2..k that sit around the acceptance boundary: each is chosen from the
+    oracle's p_1 at the position before it -- a cycling rank (top-n tests) or a cycling
+    offset from the argmax (distance tests)."""
+    ranks = [1, 0, 2, 3, 0, 1, 2, 0]
+    offsets = [1, -2, 0, 3, 2, -1, 0, -3]
+    seq = list(inputs) + [int(p1)]
+    tail = []
+    sc = scorer_factory()
+    for i in range(2, k + 1):
+        row = sc.logits(seq, 1)[0, 0]
+        order = sorted(range(row.size), key=lambda v: (-row[v], v))
+        if kind == "distance":
+            tok = min(max(order[0] + offsets[(it + i) % len(offsets)], 0), vocab - 1)
+        else:
+            tok = order[ranks[(it + i) % len(ranks)]]
+        tail.append(tok)
+        seq.append(tok)
+    return np.array(tail, dtype=np.int32)
+
+
 def lockstep(sess, om: OracleModel, src: np.ndarray, src_len: np.ndarray, k: int, n_max: int,
              max_iters: int, tail_fn: Optional[Callable[[int, int, int], np.ndarray]] = None,
              eos: int = -1, rows: Optional[List[int]] = None, check_values: bool = True,
-             tol: float = TOL) -> LockstepReport:
+             tol: float = TOL, accept=("exact", 0), accept_mode: int = 0, min_block: int = 1,
+             near_miss: bool = False) -> LockstepReport:
     """Drive ``sess`` (a freshly created binding Session) and the oracle together.
 
     tail_fn(row, j, iteration) -> proposals 2..k for that row, or None.
     rows: batch rows the oracle follows (default: all).
+    accept / accept_mode / min_block: the Verify criterion as the oracle names it and as
+    the C ABI encodes it.  near_miss: build the forced tails from the oracle's own p_1 so
+    that they straddle the acceptance boundary.
     """
     B = sess.B
     rows = list(range(B)) if rows is None else rows
@@ -84,12 +124,20 @@ def lockstep(sess, om: OracleModel, src: np.ndarray, src_len: np.ndarray, k: int
     j_all = np.zeros(B, dtype=np.int64)
     for it in range(max_iters):
         tails = None
-        if tail_fn is not None and k > 1:
+        if near_miss and k > 1:
+            tails = np.zeros((B, k - 1), dtype=np.int32)
+            for b in rows:
+                if done[b]:
+                    continue
+                p1 = int(np.argmax(prime_logits[b][0])) if it == 0 else blocks[b][0]
+                tails[b] = near_miss_tail(lambda: TransformerScorer(om, src[b, :src_len[b]], k=1), inputs[b], p1, k, it,
+                                          accept[0], om.V)
+        elif tail_fn is not None and k > 1:
             tails = np.zeros((B, k - 1), dtype=np.int32)
             for b in range(B):
                 tails[b] = tail_fn(b, int(j_all[b]), it)
         res = sess.bpd_iteration(k, n_max, eos_id=eos, forced_tail=tails, want_logits=check_values,
-                                 want_hidden=check_values)
+                                 want_hidden=check_values, accept_mode=accept_mode)
         if check_values:
             g_logits = res["logits"].cpu().numpy()
             g_hidden = res["hidden"].cpu().numpy()
@@ -118,7 +166,23 @@ def lockstep(sess, om: OracleModel, src: np.ndarray, src_len: np.ndarray, k: int
                 assert lerr <= tol, f"row {b} iteration {it}: logits differ by {lerr}"
             table = _reconcile(res["table"][b], lg, rep, f"row {b} iteration {it}")
             j = len(emitted[b])
-            khat = verify_prefix(blocks[b], lambda i: [table[i - 2][0]])
+            # walk the block as Section 3's Verify does; where the oracle's decision is within MARGIN of
+            # flipping, follow the GPU (its accepted count tells its decision for every proposal it reached)
+            kg = int(res["khat"][b])
+            khat = 1
+            while khat < k:
+                d, m = _decision(accept[0], accept[1], blocks[b][khat], int(table[khat - 1][0]), lg[khat - 1, 0])
+                d = d or khat < min_block
+                cut = khat >= n_max - j or (eos >= 0 and eos in blocks[b][:khat])   # the GPU stopped for another reason
+                g = True if kg > khat else (False if (kg == khat and not cut) else None)
+                if g is not None and g != d:
+                    assert m < MARGIN, (f"row {b} iteration {it}: proposal {khat + 1} GPU {'accepts' if g else 'rejects'}, "
+                                        f"oracle disagrees at margin {m:.4f}")
+                    rep.adopted += 1
+                    d = g
+                if not d:
+                    break
+                khat += 1
             khat, fin = clip_termination(blocks[b], khat, j, n_max, eos)
             assert khat == int(res["khat"][b]), f"row {b} iteration {it}: khat {res['khat'][b]} != oracle {khat}"
             acc = blocks[b][:khat]

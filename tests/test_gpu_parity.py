@@ -283,3 +283,68 @@ def test_c4_batch32_ragged(bpd):
     _, src_len = make_source(w)
     rows = sorted({int(np.argmin(src_len)), int(np.argmax(src_len)), 0, w.batch - 1})
     _full_size(bpd, "C4", iters=2, rows=rows, mean=2.0, free_iters=1)
+
+
+# ---------------------------------------------------------------- approximate acceptance (Section 5)
+
+@pytest.mark.parametrize("accept", [("topn", 2), ("topn", 3), ("distance", 2)], ids=lambda a: f"{a[0]}{a[1]}")
+@pytest.mark.parametrize("w", [WORKLOADS["C1"], MINI, MINI_BATCH], ids=lambda w: w.name)
+def test_approximate_acceptance_lockstep(bpd, w, accept):
+    """Top-n and distance acceptance against the oracle, with forced proposals that straddle the
+    acceptance boundary (taken from the oracle's own p_1 ranking)."""
+    from harness import lockstep
+    blob, model, src, src_len, om = _setup(bpd, w)
+    k, N = w.cfg.k_model, w.n_decode
+    mode = bpd.BPD_ACCEPT_TOPN(accept[1]) if accept[0] == "topn" else bpd.BPD_ACCEPT_DISTANCE(accept[1])
+    s = bpd.Session(model, w.batch, w.max_src, N)
+    rep = lockstep(s, om, src, src_len, k, N, max_iters=N, accept=accept, accept_mode=mode, near_miss=True)
+    flat = [kh for row in rep.khats for kh in row if kh > 0]
+    assert max(flat) > 1 and min(flat) < k, "the forced tails should produce both acceptances and rejections"
+    for b in range(w.batch):
+        assert len(rep.emitted[b]) == N
+    s.close()
+    model.close()
+
+
+def test_acceptance_modes_that_reduce_to_exact_and_minimum_block(bpd):
+    w = MINI
+    blob, model, src, src_len, om = _setup(bpd, w)
+    k, N = w.cfg.k_model, w.n_decode
+    s = bpd.Session(model, 1, w.max_src, N)
+    s.bpd_encode(src, src_len)
+    g_ids, _, _ = s.bpd_decode_greedy(N)
+    for mode in (bpd.BPD_ACCEPT_TOPN(1), bpd.BPD_ACCEPT_DISTANCE(0), bpd.BPD_ACCEPT_MIN_BLOCK(1)):
+        s.bpd_encode(src, src_len)
+        ids, _, st = s.bpd_decode_blockwise(k, N, accept_mode=mode)
+        assert np.array_equal(ids, g_ids)
+    # the whole vocabulary as "top n" (n = 255 is the largest the encoding carries): free-running heads on
+    # random weights are then accepted far more often than under exact matching
+    s.bpd_encode(src, src_len)
+    _, _, st_exact = s.bpd_decode_blockwise(k, N)
+    s.bpd_encode(src, src_len)
+    _, _, st_top = s.bpd_decode_blockwise(k, N, accept_mode=bpd.BPD_ACCEPT_TOPN(255))
+    assert st_top.iterations < st_exact.iterations and st_top.tokens == N
+    # minimum block size k = fixed-size blocks (Section 5.3): ceil(N / k) iterations whatever the heads say
+    s.bpd_encode(src, src_len)
+    ids, ln, st = s.bpd_decode_blockwise(k, N, accept_mode=bpd.BPD_ACCEPT_MIN_BLOCK(k))
+    assert st.iterations == -(-N // k) and ln[0] == N and st.khat_hist[k] == N // k
+    with pytest.raises(bpd.BpdError):
+        s.bpd_encode(src, src_len)
+        s.bpd_decode_blockwise(k, N, accept_mode=bpd.BPD_ACCEPT_MIN_BLOCK(k + 1))
+    with pytest.raises(bpd.BpdError):
+        s.bpd_decode_blockwise(k, N, accept_mode=3 << 8)
+    s.close()
+    model.close()
+
+
+def test_minimum_block_lockstep(bpd):
+    from harness import lockstep
+    w = MINI_F32
+    blob, model, src, src_len, om = _setup(bpd, w)
+    k, N = w.cfg.k_model, w.n_decode
+    s = bpd.Session(model, w.batch, w.max_src, N)
+    rep = lockstep(s, om, src, src_len, k, N, max_iters=N, accept=("topn", 2), near_miss=True, min_block=2,
+                   accept_mode=bpd.BPD_ACCEPT_TOPN(2) | bpd.BPD_ACCEPT_MIN_BLOCK(2))
+    assert all(kh >= 2 or kh == 0 for row in rep.khats[:-1] for kh in row)
+    s.close()
+    model.close()
