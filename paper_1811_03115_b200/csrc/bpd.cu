@@ -115,6 +115,12 @@ struct Arena {
 
 static int pages_per_row(const Config& c, int max_tgt) { return ceil_div(max_tgt + 1 + c.k_model, kPage); }
 
+// Sessions whose widest pass has more than 64 rows plan their projections for full token tiles.
+static int session_wide_ttiles(const Config& c, int B) {
+  const int rmax = B * c.k_model;
+  return rmax > 64 ? tc::token_tiles(rmax) : 0;
+}
+
 // Lays the session out; with base == nullptr only measures.
 static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, char* base, bpd_session* s) {
   Arena a;
@@ -151,6 +157,10 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
   st.all_done = a.take<int>(1); st.error = a.take<int>(1);
   st.stats = a.take<long long>(4 + kMaxK + 1);
   st.page_table = page_table; st.pages_per_row = ppr; st.max_tgt = max_tgt;
+  void* u2 = a.take_bytes((size_t)B * c.k_model * c.d_hidden * ea);
+  float* h2 = a.take<float>((size_t)B * d);
+  int* table2 = a.take<int>((size_t)B * kMaxK);
+  int* table_full = a.take<int>((size_t)B * kMaxK * kMaxK);
   RankState rank;
   rank.thr = a.take<float>(Rmax); rank.tok = a.take<int>(Rmax); rank.cnt = a.take<int>(Rmax);
   int* src_dev = a.take<int>(E);
@@ -163,8 +173,9 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
   // split-K workspace of the tensor-core projections: the largest any launch of this session can need
   size_t ws = 0, ncnt = 1;
   if (c.dtype == 1) {
+    const int wide = session_wide_ttiles(c, B);
     auto need = [&](int N, int K, size_t T, int z) {
-      ws = std::max(ws, tc::ws_floats(N, K, (int)T, z));
+      ws = std::max(ws, tc::ws_floats(N, K, (int)T, z, wide));
       ncnt = std::max(ncnt, tc::counters_needed(N, (int)T, z));
     };
     const int dd = c.d, ff = c.d_ff, fh = c.d_hidden, km = c.k_model;
@@ -187,6 +198,7 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
     s->crosskv = crosskv; s->kcache = kc; s->vcache = vc; s->st = st; s->src_dev = src_dev;
     s->tail_dev = tail_dev; s->plan_dev = plan_dev; s->part_val = part_val; s->part_idx = part_idx;
     s->rank = rank;
+    s->u2 = u2; s->pl_u2 = (long long)B * c.k_model * c.d_hidden; s->h2 = h2; s->table2 = table2; s->table_full = table_full;
     s->counters = counters; s->ppr = ppr; s->part_elems = tiles * R2; s->pe = pe; s->npos = (int)npos;
     s->tc_ws = tc_ws; s->tc_ws_floats = ws; s->tc_counters = tc_counters; s->tc_n_counters = ncnt; s->tc_done = tc_done; s->tc_best = tc_best; s->tc_best_elems = R2;
     s->pl_xn = (long long)(Rall * d); s->pl_attn = (long long)(Rall * d); s->pl_ffh = (long long)(Rall * c.d_ff);
@@ -277,7 +289,7 @@ static int run_encoder(bpd_session* s) {
     ap.H = c.H; ap.dh = d / c.H; ap.causal = 0; ap.limit_b = s->st.src_len;
     ap.k = static_cast<float*>(s->qbuf) + d; ap.v = static_cast<float*>(s->qbuf) + 2 * d;
     ap.ldkv = 3 * d; ap.bstride = (long long)s->max_src * 3 * d; ap.paged = 0; ap.st = s->st;
-    ap.scale = 1.0f / sqrtf((float)ap.dh);
+    ap.scale = 1.0f / sqrtf((float)ap.dh); ap.by_rows = (s->B >= 8) ? 1 : 0;
     launch_attention<float, float>(ap, st);
     ++g_launches;
     LinearParams po = lin(s->attn, d, L.wo, d, d, nullptr, E, s->x, d, 0, nullptr);
@@ -328,6 +340,9 @@ static VerifyParams verify_params(bpd_session* s, const PassArgs& a) {
   VerifyParams vp{s->st, s->B, a.kcur, a.kh, a.knext, a.mode, a.max_new, a.eos, a.accept_kind, a.accept_param, a.min_block, s->rank};
   return vp;
 }
+static bool pass_is_lazy(const bpd_session* s, const PassArgs& a) {
+  return s->tc && s->lazy_heads && a.mode == kModeBlock && a.kcur > 1 && !a.logits_dump;
+}
 static bool wants_rank(const PassArgs& a) { return a.mode == kModeBlock && a.accept_kind == kAcceptTopN && a.kcur > 1; }
 
 template <typename WT>
@@ -356,7 +371,7 @@ static int run_pass(bpd_session* s, const PassArgs& a) {
     memset(&ap, 0, sizeof(ap));
     ap.q = s->qbuf; ap.ldq = d; ap.out = s->attn; ap.ldo = d; ap.rows = R; ap.rows_per_b = a.kcur;
     ap.H = c.H; ap.dh = d / c.H; ap.causal = 1; ap.k = s->kcache[l]; ap.v = s->vcache[l]; ap.ldkv = d;
-    ap.paged = 1; ap.st = s->st; ap.scale = 1.0f / sqrtf((float)ap.dh); ap.all_done = done;
+    ap.paged = 1; ap.st = s->st; ap.scale = 1.0f / sqrtf((float)ap.dh); ap.by_rows = (s->B >= 8) ? 1 : 0; ap.all_done = done;
     launch_attention<float, WT>(ap, st);
     ++g_launches;
     launch_linear<WT, float, kEpiResidual>(lin(s->attn, d, L.wo, d, d, nullptr, R, s->x, d, 0, done), 1, st);
@@ -418,6 +433,7 @@ static tc::Scratch tc_scratch(bpd_session* s) {
   sc.ws = s->tc_ws; sc.ws_floats = s->tc_ws_floats; sc.tile_counters = s->tc_counters; sc.n_counters = s->tc_n_counters;
   sc.done_counter = s->tc_done; sc.best = s->tc_best; sc.best_elems = s->tc_best_elems;
   sc.error = s->st.error;
+  sc.wide_ttiles = session_wide_ttiles(s->m->cfg, s->B);
   return sc;
 }
 
@@ -458,7 +474,7 @@ static int run_encoder_tc(bpd_session* s) {
     ap.rows_per_b = s->max_src; ap.H = c.H; ap.dh = d / c.H; ap.causal = 0; ap.limit_b = s->st.src_len;
     ap.k = static_cast<float*>(s->qbuf) + d; ap.v = static_cast<float*>(s->qbuf) + 2 * d;
     ap.ldkv = 3 * d; ap.bstride = (long long)s->max_src * 3 * d; ap.paged = 0; ap.st = s->st;
-    ap.scale = 1.0f / sqrtf((float)ap.dh);
+    ap.scale = 1.0f / sqrtf((float)ap.dh); ap.by_rows = (s->B >= 8) ? 1 : 0;
     launch_attention<float, float>(ap, st);
     ++g_launches;
     tc::TcParams po = tc_params(nullptr, 0, nullptr);
@@ -487,7 +503,7 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   const bpd_model* m = s->m;
   const Config& c = m->cfg;
   cudaStream_t st = s->stream;
-  const int d = c.d, f = c.d_ff, R = s->B * a.kcur, R2 = R * a.kh;
+  const int d = c.d, f = c.d_ff, R = s->B * a.kcur;
   const int* done = s->st.all_done;
   const tc::Scratch sc = tc_scratch(s);
   const bool pdl = s->use_pdl != 0;
@@ -518,7 +534,7 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
     memset(&ap, 0, sizeof(ap));
     ap.q = s->qbuf; ap.ldq = d; ap.out = s->attn; ap.ldo = d; ap.out_plane = s->pl_attn; ap.rows = R;
     ap.rows_per_b = a.kcur; ap.H = c.H; ap.dh = d / c.H; ap.causal = 1; ap.k = s->kcache[l]; ap.v = s->vcache[l];
-    ap.ldkv = d; ap.paged = 1; ap.st = s->st; ap.scale = 1.0f / sqrtf((float)ap.dh); ap.all_done = done;
+    ap.ldkv = d; ap.paged = 1; ap.st = s->st; ap.scale = 1.0f / sqrtf((float)ap.dh); ap.by_rows = (s->B >= 8) ? 1 : 0; ap.all_done = done;
     PROF(kProfSelfAttn, launch_attention<float, bf16>(ap, st, pdl););
     ++g_launches;
     tc::TcParams po = tc_params(nullptr, 0, done);
@@ -555,32 +571,63 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   prof_mark(s, kProfHeadW1, 0);
   tc::TcParams pu = tc_params(m->head_b1, 1, done);
   pu.out_hi = static_cast<bf16*>(s->u); pu.plane = s->pl_u; pu.ldo = ldu;
-  BPD_TRY(tc::launch<tc::kTcPlanes>(with_w(xn, m->head_w1, km * fhd), hid, d, R, pu, sc, st, 1, 0, 0, pdl)); ++g_launches;
+  BPD_TRY(tc::launch<tc::kTcPlanes>(with_w(xn, m->head_w1, km * fhd), hid, d, R, pu, sc, st, 1, 0, 0, pdl, km * fhd)); ++g_launches;
   prof_mark(s, kProfHeadW1, 1);
   prof_mark(s, kProfHeadW2, 0);
-  tc::Operands uo{m->head_w2, km * d, s->u, s->pl_u, ldu, s->rows_dec, ldu};
-  tc::TcParams ph = tc_params(m->head_b2, 0, done);
-  ph.out_hi = static_cast<bf16*>(s->o); ph.plane = s->pl_o; ph.ldo = (long long)a.kh * d;
-  ph.h = s->h_f32; ph.d = d; ph.head_identity = c.p1_identity;
-  if (c.head_layout == 0) {
-    BPD_TRY(tc::launch<tc::kTcHeadOut>(uo, a.kh * d, km * fhd, R, ph, sc, st, 1, 0, 0, pdl));
-  } else {
-    ph.zofs_n = d;
-    BPD_TRY(tc::launch<tc::kTcHeadOut>(uo, d, fhd, R, ph, sc, st, a.kh, d, fhd, pdl));
+  // output layers + shared vocabulary projection with a fused top-1 for T rows and kh heads
+  auto heads = [&](const void* u_planes, long long u_plane, int u_rows, const float* hres, int T, int kh, int* table_out,
+                   bool rank, float* logits) -> int {
+    tc::Operands uo{m->head_w2, km * d, u_planes, u_plane, ldu, u_rows, ldu};
+    tc::TcParams ph = tc_params(m->head_b2, 0, done);
+    ph.out_hi = static_cast<bf16*>(s->o); ph.plane = s->pl_o; ph.ldo = (long long)kh * d;
+    ph.h = hres; ph.d = d; ph.head_identity = c.p1_identity;
+    if (c.head_layout == 0) {
+      BPD_TRY(tc::launch<tc::kTcHeadOut>(uo, kh * d, km * fhd, T, ph, sc, st, 1, 0, 0, pdl, km * d));
+    } else {
+      ph.zofs_n = d;
+      BPD_TRY(tc::launch<tc::kTcHeadOut>(uo, d, fhd, T, ph, sc, st, kh, d, fhd, pdl));
+    }
+    ++g_launches;
+    tc::Operands oo{m->out_proj, c.V, s->o, s->pl_o, d, s->rows_head, d};
+    tc::TcParams pv = tc_params(nullptr, 0, done);
+    pv.out_idx = table_out; pv.logits = logits;
+    if (rank) {
+      ProposalLogitParams pl{s->o, s->pl_o, m->out_proj, s->st, s->rank, s->B, a.kcur, kh, d, done};
+      launch_k(proposal_logit_kernel<bf16>, dim3(ceil_div(R, 4)), dim3(128), 0, st, pdl, pl);
+      ++g_launches;
+      pv.rank = s->rank; pv.rank_kh = kh;
+    }
+    BPD_TRY(tc::launch<tc::kTcArgmax>(oo, c.V, d, T * kh, pv, sc, st, 1, 0, 0, pdl)); ++g_launches;
+    return BPD_OK;
+  };
+  const bool lazy = pass_is_lazy(s, a);
+  if (lazy) {
+    // stage 1: p_1 at every block position, verification and commit
+    BPD_TRY(heads(s->u, s->pl_u, s->rows_dec, s->h_f32, R, 1, s->st.table, wants_rank(a), nullptr));
+    prof_mark(s, kProfHeadW2, 1);
+    prof_mark(s, kProfVocab, 0);
+    PassArgs a1 = a;
+    a1.kh = 1; a1.knext = 1;
+    VerifyParams v1 = verify_params(s, a1);
+    launch_k(verify_commit_kernel, dim3(1), dim3(32 * ceil_div(s->B, 32)), 0, st, pdl, v1);
+    ++g_launches;
+    // stage 2: all heads at the last accepted position of every row
+    GatherParams gp{static_cast<const bf16*>(s->u), s->pl_u, ldu, static_cast<bf16*>(s->u2), s->pl_u2, s->h_f32, s->h2, d,
+                    s->st, s->B, a.kcur, done};
+    launch_k(gather_selected_kernel, dim3(s->B), dim3(256), 0, st, pdl, gp);
+    ++g_launches;
+    BPD_TRY(heads(s->u2, s->pl_u2, s->B, s->h2, s->B, a.kh, s->table2, false, nullptr));
+    SelectParams sp{s->st, s->st.table, s->table2, s->table_full, s->B, a.kcur, a.kh, a.knext, done};
+    launch_k(select_next_kernel, dim3(1), dim3(32 * ceil_div(s->B, 32)), 0, st, pdl, sp);
+    ++g_launches;
+    prof_mark(s, kProfVocab, 1);
+    BPD_CUDA(cudaGetLastError());
+    s->invocations += 1;
+    return BPD_OK;
   }
-  ++g_launches;
+  BPD_TRY(heads(s->u, s->pl_u, s->rows_dec, s->h_f32, R, a.kh, s->st.table, wants_rank(a), a.logits_dump));
   prof_mark(s, kProfHeadW2, 1);
   prof_mark(s, kProfVocab, 0);
-  tc::Operands oo{m->out_proj, c.V, s->o, s->pl_o, d, s->rows_head, d};
-  tc::TcParams pv = tc_params(nullptr, 0, done);
-  pv.out_idx = s->st.table; pv.logits = a.logits_dump;
-  if (wants_rank(a)) {
-    ProposalLogitParams pl{s->o, s->pl_o, m->out_proj, s->st, s->rank, s->B, a.kcur, a.kh, d, done};
-    launch_k(proposal_logit_kernel<bf16>, dim3(ceil_div(R, 4)), dim3(128), 0, st, pdl, pl);
-    ++g_launches;
-    pv.rank = s->rank; pv.rank_kh = a.kh;
-  }
-  BPD_TRY(tc::launch<tc::kTcArgmax>(oo, c.V, d, R2, pv, sc, st, 1, 0, 0, pdl)); ++g_launches;
   prof_mark(s, kProfVocab, 1);
   VerifyParams vp = verify_params(s, a);
   PROF(kProfVerify, launch_k(verify_commit_kernel, dim3(1), dim3(32 * ceil_div(s->B, 32)), 0, st, pdl, vp););
@@ -599,6 +646,7 @@ static int dispatch_eager(bpd_session* s, const PassArgs& a) {
 // A pass is a fixed sequence of launches for given arguments: the first use runs it eagerly (which also
 // creates tensor maps and sets kernel attributes), the second captures it into a CUDA graph, later uses replay it.
 static int dispatch_pass(bpd_session* s, const PassArgs& a) {
+  s->last_pass_lazy = pass_is_lazy(s, a) ? 1 : 0;
   if (s->profiling || !s->use_graphs || a.logits_dump) return dispatch_eager(s, a);
   const GraphKey key(a.mode, a.kcur, a.kh, a.knext, (const void*)a.forced, a.forced_rows, a.kforced, a.max_new, a.eos,
                      (const void*)a.logits_dump, (a.accept_kind << 16) | (a.accept_param << 8) | a.min_block);
@@ -785,6 +833,9 @@ int bpd_session_create(const bpd_model* model, int batch, int max_src, int max_t
   s->use_graphs = (own_stream && !getenv("BPD_DISABLE_GRAPHS")) ? 1 : 0;
   s->use_pdl = getenv("BPD_DISABLE_PDL") ? 0 : 1;
   // with at most 16 rows per pass every projection CTA can afford the row statistics itself
+  const char* lz = getenv("BPD_LAZY_HEADS");
+  s->lazy_heads = s->tc && (lz ? atoi(lz) != 0 : batch * model->cfg.k_model >= 64);
+  s->last_pass_lazy = 0;
   s->fold_ln = (s->tc && batch * model->cfg.k_model <= 16 && !getenv("BPD_DISABLE_FOLD")) ? 1 : 0;
   s->phase = kPhaseCreated; s->plan_len = 0; s->plan_k = 0; s->invocations = 0; s->pinned = nullptr;
   plan_session(model->cfg, batch, max_src, max_tgt, s->base, s);
@@ -1014,7 +1065,8 @@ int bpd_iteration(bpd_session* s, int k, int accept_mode, int max_new, int32_t e
     BPD_CUDA(cudaMemcpyAsync(out->hidden_dev, s->h_f32, sizeof(float) * B * k * s->m->cfg.d, cudaMemcpyDeviceToDevice, s->stream));
   std::vector<int> khat(B), table((size_t)B * k * k), blk((size_t)B * kMaxK), cur((size_t)B * kMaxK);
   BPD_CUDA(cudaMemcpyAsync(khat.data(), s->st.khat, B * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
-  BPD_CUDA(cudaMemcpyAsync(table.data(), s->st.table, table.size() * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
+  BPD_CUDA(cudaMemcpyAsync(table.data(), s->last_pass_lazy ? s->table_full : s->st.table, table.size() * sizeof(int),
+                           cudaMemcpyDeviceToHost, s->stream));
   BPD_CUDA(cudaMemcpyAsync(blk.data(), s->st.block, blk.size() * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
   BPD_CUDA(cudaMemcpyAsync(cur.data(), s->st.cur_block, cur.size() * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
   BPD_CUDA(cudaStreamSynchronize(s->stream));
@@ -1102,7 +1154,7 @@ int bpd_op_vocab_argmax(const void* x, const void* w, int rows, int d, int vocab
     BPD_CUDA(cudaMemsetAsync(p, 0, L.total, st));
     tc::Scratch sc{reinterpret_cast<float*>(p + L.ws_off), L.ws_floats, reinterpret_cast<unsigned*>(p + L.cnt_off),
                    L.n_counters, reinterpret_cast<unsigned*>(p + L.done_off),
-                   reinterpret_cast<unsigned long long*>(p + L.pv_off), L.part_elems, reinterpret_cast<int*>(p + L.err_off)};
+                   reinterpret_cast<unsigned long long*>(p + L.pv_off), L.part_elems, reinterpret_cast<int*>(p + L.err_off), 0};
     const long long plane = (reinterpret_cast<const bf16*>(p + L.zero_off) - static_cast<const bf16*>(x));
     tc::Operands op{w, vocab, x, plane, d, rows, d};
     tc::TcParams tp;
@@ -1147,7 +1199,7 @@ int bpd_op_linear(const void* x, const void* w, const void* bias, int rows, int 
     BPD_CUDA(cudaMemsetAsync(p, 0, L.total, st));
     tc::Scratch sc{reinterpret_cast<float*>(p + L.ws_off), L.ws_floats, reinterpret_cast<unsigned*>(p + L.cnt_off),
                    L.n_counters, reinterpret_cast<unsigned*>(p + L.done_off),
-                   reinterpret_cast<unsigned long long*>(p + L.pv_off), L.part_elems, reinterpret_cast<int*>(p + L.err_off)};
+                   reinterpret_cast<unsigned long long*>(p + L.pv_off), L.part_elems, reinterpret_cast<int*>(p + L.err_off), 0};
     const long long plane = (reinterpret_cast<const bf16*>(p + L.zero_off) - static_cast<const bf16*>(x));
     tc::Operands op{w, out_f, x, plane, in_f, rows, in_f};
     tc::TcParams tp;

@@ -137,6 +137,9 @@ struct bpd_session {
   int profiling;
   int use_graphs;
   int use_pdl;
+  int lazy_heads;          // two-stage head evaluation (p_1 everywhere, all heads only at the accepted position)
+  int last_pass_lazy;
+  void* u2; long long pl_u2; float* h2; int *table2, *table_full;
   int fold_ln;             // decoder layer norms are folded into the projections (few rows only)
   std::map<GraphKey, GraphEntry> graphs;
   std::vector<cudaEvent_t> prof_begin[kProfSlots], prof_end[kProfSlots];

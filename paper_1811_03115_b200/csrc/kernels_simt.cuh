@@ -328,6 +328,7 @@ struct AttnParams {
   void* out; long long ldo;
   long long out_plane;             // > 0: output as two bf16 planes (hi, lo) this many elements apart
   int rows, rows_per_b, H, dh;
+  int by_rows;                     // 1: one CTA per (sequence, head) instead of per (row, head)
   int causal;                      // 1: keys 0 .. len[b]+i ; 0: keys 0 .. limit_b[b]-1
   const int* limit_b;
   const void* k; const void* v;    // linear: row s of batch b at base + b*bstride + s*ldkv ; paged: page pool
@@ -541,11 +542,104 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_split_kernel(AttnPa
   }
 }
 
+// Attention for sessions with many rows: one CTA per (sequence, head), one warp per query row (rows beyond
+// 8 wrap around).  A warp walks the 32-key chunks of its row in position order with a running max / sum, so
+// the order again depends only on key positions; the rows of a sequence share its keys through L1/L2.
+template <typename QT, typename CT, int DH>
+__global__ void __launch_bounds__(kAttnWarps * 32) attention_rows_kernel(AttnParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
+  if (p.all_done && *p.all_done) return;
+  constexpr int DPL = (DH >= 32) ? DH / 32 : 1;
+  __shared__ float s_q[kAttnWarps][DH];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b = blockIdx.x / p.H, h = blockIdx.x % p.H;
+  const CT* K = reinterpret_cast<const CT*>(p.k);
+  const CT* V = reinterpret_cast<const CT*>(p.v);
+  const int* pt = p.st.page_table + b * p.st.pages_per_row;
+  const bool owns = (DH >= 32) || (lane < DH);
+  const int dim0 = (DH >= 32) ? lane * DPL : lane;
+  for (int i = warp; i < p.rows_per_b; i += kAttnWarps) {
+    const int r = b * p.rows_per_b + i;
+    const int limit = p.causal ? (p.st.len[b] + i + 1) : p.limit_b[b];
+    const QT* q = reinterpret_cast<const QT*>(p.q) + (long long)r * p.ldq + h * DH;
+    __syncwarp();
+    for (int c = lane; c < DH; c += 32) s_q[warp][c] = to_f(q[c]) * p.scale;
+    __syncwarp();
+    float m_run = -INFINITY, l_run = 0.f;
+    float acc[DPL];
+#pragma unroll
+    for (int t = 0; t < DPL; ++t) acc[t] = 0.f;
+    for (int c0 = 0; c0 < limit; c0 += 32) {
+      const size_t base = p.paged ? ((size_t)pt[c0 / kPage] * kPage + (c0 % kPage)) * p.ldkv + h * DH
+                                  : (size_t)b * p.bstride + (size_t)c0 * p.ldkv + h * DH;
+      const int nk = min(32, limit - c0);
+      float sc = -INFINITY;
+      if (lane < nk) {
+        const CT* kr = K + base + (size_t)lane * p.ldkv;
+        float dot = 0.f;
+#pragma unroll
+        for (int c = 0; c < DH; c += 8) {
+          float kv[8];
+          load8(kr + c, kv);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) dot = fmaf(s_q[warp][c + e], kv[e], dot);
+        }
+        sc = dot;
+      }
+      const float m_new = fmaxf(m_run, warp_max(sc));
+      const float corr = expf(m_run - m_new);
+      const float pj = (lane < nk) ? expf(sc - m_new) : 0.f;
+      l_run = l_run * corr + warp_sum(pj);
+#pragma unroll
+      for (int t = 0; t < DPL; ++t) acc[t] *= corr;
+      const CT* vb = V + base + dim0;
+#pragma unroll 8
+      for (int jj = 0; jj < nk; ++jj) {
+        const float pw = __shfl_sync(0xffffffffu, pj, jj);
+        if (owns) {
+          float vv[DPL];
+          load_n<DPL>(vb + (size_t)jj * p.ldkv, vv);
+#pragma unroll
+          for (int t = 0; t < DPL; ++t) acc[t] = fmaf(pw, vv[t], acc[t]);
+        }
+      }
+      m_run = m_new;
+    }
+    if (owns) {
+      const float inv = 1.f / l_run;
+#pragma unroll
+      for (int t = 0; t < DPL; ++t) {
+        const float ov = acc[t] * inv;
+        const long long o = (long long)r * p.ldo + h * DH + dim0 + t;
+        if (p.out_plane) {
+          bf16* op = reinterpret_cast<bf16*>(p.out) + o;
+          const bf16 hi = __float2bfloat16_rn(ov);
+          op[0] = hi;
+          op[p.out_plane] = __float2bfloat16_rn(ov - __bfloat162float(hi));
+        } else {
+          reinterpret_cast<QT*>(p.out)[o] = from_f<QT>(ov);
+        }
+      }
+    }
+  }
+}
+
 // Picks the split kernel for the common head widths, the generic one-warp kernel otherwise.
 template <typename QT, typename CT>
 static void launch_attention(const AttnParams& p, cudaStream_t st, bool pdl = false) {
   const int items = p.rows * p.H;
   const dim3 g(items), b(kAttnWarps * 32);
+  if (p.by_rows) {   // many sequences: a CTA per (sequence, head); a property of the session, not of the pass
+    const dim3 gr((p.rows / p.rows_per_b) * p.H);
+    switch (p.dh) {
+      case 16: launch_k(attention_rows_kernel<QT, CT, 16>, gr, b, 0, st, pdl, p); return;
+      case 32: launch_k(attention_rows_kernel<QT, CT, 32>, gr, b, 0, st, pdl, p); return;
+      case 64: launch_k(attention_rows_kernel<QT, CT, 64>, gr, b, 0, st, pdl, p); return;
+      case 128: launch_k(attention_rows_kernel<QT, CT, 128>, gr, b, 0, st, pdl, p); return;
+      default: break;
+    }
+  }
   switch (p.dh) {
     case 16: launch_k(attention_split_kernel<QT, CT, 16>, g, b, 0, st, pdl, p); break;
     case 32: launch_k(attention_split_kernel<QT, CT, 32>, g, b, 0, st, pdl, p); break;
@@ -808,6 +902,57 @@ static __global__ void verify_commit_kernel(VerifyParams p) {
     p.st.stats[p.mode == kModePrime ? 3 : 2] += 1;
     if (!any_open) *p.st.all_done = 1;
   }
+}
+
+// ------------------------------------------------------------------ lazy heads (two-stage evaluation)
+// Stage 1 scores p_1 at every block position and verifies; stage 2 evaluates all k heads only at the last
+// accepted position of each row.  These two small kernels move the selected rows into a compact buffer and
+// then assemble the next block and the (partly filled) k x k table.
+struct GatherParams {
+  const bf16* u; long long pl_u; long long ldu;   // head hidden activations, planes [rows, ldu]
+  bf16* u2; long long pl_u2;                      // compact planes [B, ldu]
+  const float* h; float* h2; int d;               // decoder outputs [rows, d] -> [B, d]
+  RowState st;
+  int B, kcur;
+  const int* all_done;
+};
+static __global__ void __launch_bounds__(256) gather_selected_kernel(GatherParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
+  if (p.all_done && *p.all_done) return;
+  const int b = blockIdx.x;
+  const int row = b * p.kcur + max(p.st.khat[b], 1) - 1;     // last accepted position (first one for idle rows)
+  const uint4* s_hi = reinterpret_cast<const uint4*>(p.u + (size_t)row * p.ldu);
+  const uint4* s_lo = reinterpret_cast<const uint4*>(p.u + (size_t)row * p.ldu + p.pl_u);
+  uint4* d_hi = reinterpret_cast<uint4*>(p.u2 + (size_t)b * p.ldu);
+  uint4* d_lo = reinterpret_cast<uint4*>(p.u2 + (size_t)b * p.ldu + p.pl_u2);
+  for (int i = threadIdx.x; i < p.ldu / 8; i += blockDim.x) { d_hi[i] = s_hi[i]; d_lo[i] = s_lo[i]; }
+  for (int c = threadIdx.x; c < p.d; c += blockDim.x) p.h2[(size_t)b * p.d + c] = p.h[(size_t)row * p.d + c];
+}
+
+struct SelectParams {
+  RowState st;
+  const int* table1;   // [B, kcur]      p_1 at every block position
+  const int* table2;   // [B, kh]        all heads at the selected position
+  int* table_full;     // [B, kcur, kh]  what is known of the k x k table, -1 elsewhere
+  int B, kcur, kh, knext;
+  const int* all_done;
+};
+static __global__ void select_next_kernel(SelectParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
+  // When the decode ended in this very pass, stage 2 did not run: the table still reports p_1, the rest is unknown.
+  const bool ended = p.all_done && *p.all_done;
+  const int b = threadIdx.x;
+  if (b >= p.B) return;
+  const int khat = p.st.khat[b];
+  const int sel = max(khat, 1) - 1;
+  int* full = p.table_full + (size_t)b * p.kcur * p.kh;
+  for (int r = 0; r < p.kcur; ++r)
+    for (int i = 0; i < p.kh; ++i)
+      full[r * p.kh + i] = (i == 0) ? p.table1[b * p.kcur + r] : ((r == sel && !ended) ? p.table2[b * p.kh + i] : -1);
+  if (khat > 0 && !ended)
+    for (int i = 1; i < p.knext; ++i) p.st.block[b * kMaxK + i] = p.table2[b * p.kh + i];
 }
 
 struct ResetParams {

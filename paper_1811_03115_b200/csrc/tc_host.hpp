@@ -22,11 +22,17 @@ struct Plan {
 };
 // Depends on (N, K) only -- never on the number of tokens -- so that a position
 // scored alone and the same position scored inside a block add up in the same order.
-inline Plan plan_splits(int N, int K) {
+// wide_ttiles: 0 for sessions whose passes carry few rows (one token tile, two CTAs per SM, split K finely);
+// otherwise the number of token tiles of the session's widest pass: those launches already have tiles x
+// token tiles CTAs of 128 tokens each (one per SM), so K is split only as far as that leaves SMs idle.
+// It is a property of the session, so greedy and blockwise passes of one session still agree.
+inline Plan plan_splits(int N, int K, int wide_ttiles = 0) {
   Plan pl;
   pl.tiles = (N + kBM - 1) / kBM;
   pl.chunks = (K + kBK - 1) / kBK;
-  int splits = std::max(1, std::min(pl.chunks / kMinChunksPerSplit, kSlots / pl.tiles));
+  int splits;
+  if (wide_ttiles > 0) splits = std::max(1, std::min(pl.chunks / 8, (kSlots / 2) / (pl.tiles * wide_ttiles)));
+  else splits = std::max(1, std::min(pl.chunks / kMinChunksPerSplit, kSlots / pl.tiles));
   pl.chunks_per_split = (pl.chunks + splits - 1) / splits;
   pl.splits = (pl.chunks + pl.chunks_per_split - 1) / pl.chunks_per_split;
   return pl;
@@ -37,8 +43,8 @@ inline int token_bn(int T) {
   return std::max(16, (per + 15) / 16 * 16);
 }
 // fp32 elements of split-K workspace a launch with these sizes needs.
-inline size_t ws_floats(int N, int K, int T, int zslices) {
-  const Plan pl = plan_splits(N, K);
+inline size_t ws_floats(int N, int K, int T, int zslices, int wide_ttiles = 0) {
+  const Plan pl = plan_splits(N, K, wide_ttiles);
   if (pl.splits == 1) return 0;
   return (size_t)token_tiles(T) * zslices * pl.tiles * pl.splits * token_bn(T) * kBM;
 }
@@ -52,6 +58,7 @@ struct Scratch {
   unsigned* done_counter;
   unsigned long long* best; size_t best_elems;
   int* error;
+  int wide_ttiles;   // see plan_splits
 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -111,15 +118,19 @@ struct Operands {
 
 template <int EPI>
 int launch(const Operands& op, int N, int K, int T, TcParams p, const Scratch& sc, cudaStream_t st, int zslices = 1,
-           int a_rows_per_slice = 0, int b_cols_per_slice = 0, bool pdl = false) {
+           int a_rows_per_slice = 0, int b_cols_per_slice = 0, bool pdl = false, int plan_n = 0) {
   static bool attr_set = false;
   if (!attr_set) {
     BPD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)std::max(smem_bytes(kMaxBN), smem_bytes(64))));
     attr_set = true;
   }
-  const Plan pl = plan_splits(N, K);
+  // plan_n: the feature count the K split is planned for.  A launch that computes only the first features of a
+  // matrix (fewer heads) passes the full count so that every feature is summed in the same order either way.
+  Plan pl = plan_splits(plan_n > 0 ? plan_n : N, K, sc.wide_ttiles);
+  pl.tiles = (N + kBM - 1) / kBM;
   const int ttiles = token_tiles(T), bn = token_bn(T);
-  const size_t need_ws = ws_floats(N, K, T, zslices), need_cnt = counters_needed(N, T, zslices);
+  const size_t need_ws = pl.splits == 1 ? 0 : (size_t)ttiles * zslices * pl.tiles * pl.splits * bn * kBM;
+  const size_t need_cnt = counters_needed(N, T, zslices);
   if (need_ws > sc.ws_floats || need_cnt > sc.n_counters)
     return fail(BPD_E_NOMEM, "split-K workspace too small (%zu floats, %zu counters needed)", need_ws, need_cnt);
   if (EPI == kTcArgmax && (size_t)T > sc.best_elems) return fail(BPD_E_NOMEM, "top-1 workspace too small");

@@ -348,3 +348,39 @@ def test_minimum_block_lockstep(bpd):
     assert all(kh >= 2 or kh == 0 for row in rep.khats[:-1] for kh in row)
     s.close()
     model.close()
+
+
+# ---------------------------------------------------------------- lazy (two-stage) head evaluation
+
+@pytest.mark.parametrize("w", [MINI, MINI_BLOCK, MINI_BATCH], ids=lambda w: w.name)
+def test_lazy_heads_give_the_same_decode(bpd, w, monkeypatch):
+    """p_1 at every position first, all heads only at the accepted position: same ids, same accepted
+    block sizes, same next blocks as the one-stage evaluation and as the oracle."""
+    from harness import lockstep
+    blob, model, src, src_len, om = _setup(bpd, w)
+    k, N = w.cfg.k_model, w.n_decode
+    s0 = bpd.Session(model, w.batch, w.max_src, N)
+    s0.bpd_encode(src, src_len)
+    g_ids, _, _ = s0.bpd_decode_greedy(N)
+    plan, sched = _plan(w, g_ids, k, 2.0)
+    s0.bpd_encode(src, src_len)
+    s0.bpd_set_forced_plan(plan, k)
+    _, _, st0 = s0.bpd_decode_blockwise(k, N)
+    s0.close()
+    monkeypatch.setenv("BPD_LAZY_HEADS", "1")
+    s = bpd.Session(model, w.batch, w.max_src, N)
+    s.bpd_encode(src, src_len)
+    ids, _, _ = s.bpd_decode_blockwise(k, N)
+    assert np.array_equal(ids, g_ids)
+    s.bpd_encode(src, src_len)
+    s.bpd_set_forced_plan(plan, k)
+    ids, _, st = s.bpd_decode_blockwise(k, N)
+    assert np.array_equal(ids, g_ids) and st.khat_hist == st0.khat_hist and st.iterations == st0.iterations
+    rep = lockstep(s, om, src, src_len, k, N, max_iters=N, check_values=False)
+    for b in range(w.batch):
+        assert rep.emitted[b] == list(g_ids[b])
+    rep = lockstep(s, om, src, src_len, k, N, max_iters=N, check_values=False, accept=("topn", 2),
+                   accept_mode=bpd.BPD_ACCEPT_TOPN(2), near_miss=True)
+    assert max(kh for row in rep.khats for kh in row) > 1
+    s.close()
+    model.close()
