@@ -573,10 +573,10 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   pu.out_hi = static_cast<bf16*>(s->u); pu.plane = s->pl_u; pu.ldo = ldu;
   BPD_TRY(tc::launch<tc::kTcPlanes>(with_w(xn, m->head_w1, km * fhd), hid, d, R, pu, sc, st, 1, 0, 0, pdl, km * fhd)); ++g_launches;
   prof_mark(s, kProfHeadW1, 1);
-  prof_mark(s, kProfHeadW2, 0);
   // output layers + shared vocabulary projection with a fused top-1 for T rows and kh heads
   auto heads = [&](const void* u_planes, long long u_plane, int u_rows, const float* hres, int T, int kh, int* table_out,
                    bool rank, float* logits) -> int {
+    prof_mark(s, kProfHeadW2, 0);
     tc::Operands uo{m->head_w2, km * d, u_planes, u_plane, ldu, u_rows, ldu};
     tc::TcParams ph = tc_params(m->head_b2, 0, done);
     ph.out_hi = static_cast<bf16*>(s->o); ph.plane = s->pl_o; ph.ldo = (long long)kh * d;
@@ -588,6 +588,8 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
       BPD_TRY(tc::launch<tc::kTcHeadOut>(uo, d, fhd, T, ph, sc, st, kh, d, fhd, pdl));
     }
     ++g_launches;
+    prof_mark(s, kProfHeadW2, 1);
+    prof_mark(s, kProfVocab, 0);
     tc::Operands oo{m->out_proj, c.V, s->o, s->pl_o, d, s->rows_head, d};
     tc::TcParams pv = tc_params(nullptr, 0, done);
     pv.out_idx = table_out; pv.logits = logits;
@@ -598,14 +600,13 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
       pv.rank = s->rank; pv.rank_kh = kh;
     }
     BPD_TRY(tc::launch<tc::kTcArgmax>(oo, c.V, d, T * kh, pv, sc, st, 1, 0, 0, pdl)); ++g_launches;
+    prof_mark(s, kProfVocab, 1);
     return BPD_OK;
   };
   const bool lazy = pass_is_lazy(s, a);
   if (lazy) {
     // stage 1: p_1 at every block position, verification and commit
     BPD_TRY(heads(s->u, s->pl_u, s->rows_dec, s->h_f32, R, 1, s->st.table, wants_rank(a), nullptr));
-    prof_mark(s, kProfHeadW2, 1);
-    prof_mark(s, kProfVocab, 0);
     PassArgs a1 = a;
     a1.kh = 1; a1.knext = 1;
     VerifyParams v1 = verify_params(s, a1);
@@ -620,15 +621,11 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
     SelectParams sp{s->st, s->st.table, s->table2, s->table_full, s->B, a.kcur, a.kh, a.knext, done};
     launch_k(select_next_kernel, dim3(1), dim3(32 * ceil_div(s->B, 32)), 0, st, pdl, sp);
     ++g_launches;
-    prof_mark(s, kProfVocab, 1);
     BPD_CUDA(cudaGetLastError());
     s->invocations += 1;
     return BPD_OK;
   }
   BPD_TRY(heads(s->u, s->pl_u, s->rows_dec, s->h_f32, R, a.kh, s->st.table, wants_rank(a), a.logits_dump));
-  prof_mark(s, kProfHeadW2, 1);
-  prof_mark(s, kProfVocab, 0);
-  prof_mark(s, kProfVocab, 1);
   VerifyParams vp = verify_params(s, a);
   PROF(kProfVerify, launch_k(verify_commit_kernel, dim3(1), dim3(32 * ceil_div(s->B, 32)), 0, st, pdl, vp););
   ++g_launches;

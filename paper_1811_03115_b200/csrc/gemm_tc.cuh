@@ -195,27 +195,21 @@ __host__ __device__ inline size_t smem_bytes(int bn) { return stages_for(bn) * s
 // the stores of the previous token.
 template <int EPI>
 __device__ __forceinline__ void tc_store8(const TcParams& p, int z, int t_first, int ntok, int n, const float (&vin)[8],
-                                          const float* s_mean, const float* s_rstd, int stat0) {
+                                          const float* s_mean, const float* s_rstd, int stat0,
+                                          const unsigned long long* s_slot) {
   float lns = 0.f, lnc = 0.f, bias = 0.f, gnext = 0.f;
   if (p.ln_x) { lns = p.ln_s[n]; lnc = p.ln_c[n]; }
   else if (p.bias) bias = __bfloat162float(p.bias[n + p.zofs_n * z]);
   if (EPI == kTcResidual && p.g_next) gnext = __bfloat162float(p.g_next[n]);
   float pre[8];
-  size_t slot[8];
+  const bool need_old = (EPI == kTcResidual) && p.g_next != nullptr;   // otherwise the add is a fire-and-forget reduction
 #pragma unroll
   for (int c = 0; c < 8; ++c) {
     pre[c] = 0.f;
-    slot[c] = 0;
     if (c < ntok) {
       const int t = t_first + c;
-      if (EPI == kTcResidual) pre[c] = p.out_f32[(long long)t * p.ldo + n];
-      if (EPI == kTcHeadOut) pre[c] = p.h[(size_t)t * p.d + (n % p.d)];
-      if (EPI == kTcQkv && n >= p.d) {
-        const int b = t / p.rows_per_b, i = t % p.rows_per_b;
-        const int pos = p.st.len[b] + i;
-        const int page = p.st.page_table[b * p.st.pages_per_row + pos / kPage];
-        slot[c] = ((size_t)page * kPage + (pos % kPage)) * p.d;
-      }
+      if (need_old) pre[c] = p.out_f32[(long long)t * p.ldo + n];
+      if (EPI == kTcHeadOut) pre[c] = __ldg(&p.h[(size_t)t * p.d + (n % p.d)]);
     }
   }
 #pragma unroll
@@ -235,6 +229,10 @@ __device__ __forceinline__ void tc_store8(const TcParams& p, int z, int t_first,
       } else if (EPI == kTcF32) {
         p.out_f32[(long long)t * p.ldo + n] = v;
       } else if (EPI == kTcResidual) {
+        if (!need_old) {
+          atomicAdd(&p.out_f32[(long long)t * p.ldo + n], v);   // single writer per element: just x += v without a read
+          continue;
+        }
         const float xnew = pre[c] + v;
         p.out_f32[(long long)t * p.ldo + n] = xnew;
         if (p.g_next) {
@@ -254,8 +252,8 @@ __device__ __forceinline__ void tc_store8(const TcParams& p, int z, int t_first,
       } else if (EPI == kTcQkv) {
         const int d = p.d;
         if (n < d) p.out_f32[(long long)t * p.ldo + n] = v;
-        else if (n < 2 * d) p.kcache[slot[c] + (n - d)] = __float2bfloat16_rn(v);
-        else p.vcache[slot[c] + (n - 2 * d)] = __float2bfloat16_rn(v);
+        else if (n < 2 * d) p.kcache[s_slot[stat0 + c] + (n - d)] = __float2bfloat16_rn(v);
+        else p.vcache[s_slot[stat0 + c] + (n - 2 * d)] = __float2bfloat16_rn(v);
       }
     }
   }
@@ -283,6 +281,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __shared__ float s_val[4][kMaxBN];
   __shared__ int s_idx[4][kMaxBN];
   __shared__ float s_mean[16], s_rstd[16];
+  __shared__ unsigned long long s_slot[kMaxBN];   // kTcQkv: cache slot (element offset) of every token of the tile
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = blockIdx.x, split = blockIdx.y;
@@ -379,6 +378,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int et = threadIdx.x - 64;                 // 0..127
     pdl_wait();
     const bool skip = p.all_done && *p.all_done;     // same value in every thread: the flag is stable by now
+    if (EPI == kTcQkv && !skip && et < nt) {
+      const int t = t0 + et;
+      const int b = t / p.rows_per_b, i = t % p.rows_per_b;
+      const int pos = p.st.len[b] + i;
+      const int page = p.st.page_table[b * p.st.pages_per_row + pos / kPage];
+      s_slot[et] = ((unsigned long long)page * kPage + (pos % kPage)) * p.d;
+    }
     if (p.ln_x && !skip) {
       // per-token mean and 1/std of the residual stream, computed while the main loop runs: 8 threads per
       // token (at most 16 tokens per tile in this mode), two passes, fixed order
@@ -428,8 +434,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (n < p.N) {
               const float lo8[8] = {v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]};
               const float hi8[8] = {v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15]};
-              tc_store8<EPI>(p, slice, t0 + cb, min(8, nt - cb), n, lo8, s_mean, s_rstd, cb);
-              tc_store8<EPI>(p, slice, t0 + cb + 8, min(8, nt - cb - 8), n, hi8, s_mean, s_rstd, cb + 8);
+              tc_store8<EPI>(p, slice, t0 + cb, min(8, nt - cb), n, lo8, s_mean, s_rstd, cb, s_slot);
+              tc_store8<EPI>(p, slice, t0 + cb + 8, min(8, nt - cb - 8), n, hi8, s_mean, s_rstd, cb + 8, s_slot);
             }
           } else {
 #pragma unroll
@@ -482,7 +488,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 for (int c = 0; c < 8; ++c) acc[c] += v[ss][c];
             }
             if (EPI != kTcArgmax) {
-              if (n < p.N) tc_store8<EPI>(p, slice, t0 + cg, min(8, nt - cg), n, acc, s_mean, s_rstd, cg);
+              if (n < p.N) tc_store8<EPI>(p, slice, t0 + cg, min(8, nt - cg), n, acc, s_mean, s_rstd, cg, s_slot);
             } else {
 #pragma unroll
               for (int c = 0; c < 8; ++c) {
