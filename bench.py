@@ -66,6 +66,23 @@ def iteration_bytes(cfg, k, batch, mean_T, mean_S):
     return e * (layers + w1 + w2 + V * d) + batch * L * 2 * e * d * (mean_T + mean_S), e * w2
 
 
+def max_over_ranks(ms: float, device=None) -> float:
+    """Slowest rank's time (every rank must call it); identity without a process group."""
+    import torch
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        t = torch.tensor([ms], device=device or "cpu", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+    return ms
+
+
+def whole_job_tokens_per_s(tokens_per_rank: int, world: int, ms_step: float) -> float:
+    """Replicas only: every rank decodes its own copy of the workload, no data-path collective;
+    the job's throughput is all ranks' tokens over the slowest rank's time."""
+    return world * tokens_per_rank / (ms_step * 1e-3)
+
+
 def build_plan(w, greedy_ids, k, mean):
     plan = np.zeros((w.batch, w.n_decode, k - 1), dtype=np.int32)
     khats = []
@@ -228,27 +245,20 @@ def run_gpu(args):
         barrier()
         return ev0.elapsed_time(ev1) / n_steps      # ms per decode
 
-    def max_over_ranks(ms):
-        if world > 1:
-            t = torch.tensor([ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            return float(t.item())
-        return ms
-
     # ---- headline: controlled acceptance, device resident
     sess.bpd_encode(src, src_len)
     sess.bpd_set_forced_plan(plan, k)
     timed_decodes(args.warmup, "block")
     launches0 = bpd.bpd_kernel_launches()
     with ClockSampler(local) as clocks:
-        ms_step = max_over_ranks(timed_decodes(args.steps, "block"))
+        ms_step = max_over_ranks(timed_decodes(args.steps, "block"), dev)
     launches = bpd.bpd_kernel_launches() - launches0
     ids, _, st = sess.bpd_fetch_output(N)
     assert np.array_equal(ids, g_ids), "controlled-acceptance decode differs from greedy"
     assert st.row_iterations == len(khats)
     iters = st.iterations
     us_iter = 1e3 * ms_step / iters
-    value = world * w.batch * N / (ms_step * 1e-3)
+    value = whole_job_tokens_per_s(w.batch * N, world, ms_step)
 
     # ---- per-phase timing of the same decode (events inside the pass), for the roofline of the dominant kernel
     sess.bpd_profile(True)
@@ -321,7 +331,7 @@ def run_gpu(args):
         out_ids, out_len, _ = sess.bpd_decode_blockwise(k, N)   # D2H of the token ids
         torch.cuda.synchronize()
         e2e_times.append(time.perf_counter() - t0)
-    e2e_ms = max_over_ranks(1e3 * float(np.mean(e2e_times[args.warmup:])))
+    e2e_ms = max_over_ranks(1e3 * float(np.mean(e2e_times[args.warmup:])), dev)
     h2d = src.nbytes + src_len.nbytes + plan.nbytes
     d2h = w.batch * N * 4 + w.batch * 4 + (3 + 17) * 8
 
@@ -350,7 +360,7 @@ def run_gpu(args):
         "iteration_frac_of_measured": it_bytes / (us_iter * 1e-6) / 1e9 / peak,
         "phase_us": phase_us, "kernel_us_eager": kernel_us, "modes": extra,
         "clocks": clocks.summary(),
-        "e2e": {"value": world * w.batch * N / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
+        "e2e": {"value": whole_job_tokens_per_s(w.batch * N, world, e2e_ms), "unit": "tokens/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
         "gpu_launches": int(launches),
         "roofline": roofline,
