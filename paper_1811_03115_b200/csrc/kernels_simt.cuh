@@ -625,6 +625,107 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_rows_kernel(AttnPar
   }
 }
 
+// Same job for blocks of at most 16 query rows per sequence (the decoder's passes): the CTA stages each
+// 32-key chunk of K and V in shared memory once (coalesced), every warp then serves its one or two query rows
+// from there.  Per row the chunks are folded in position order with a running max / sum.
+template <typename QT, typename CT, int DH>
+__global__ void __launch_bounds__(kAttnWarps * 32) attention_seq_kernel(AttnParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
+  if (p.all_done && *p.all_done) return;
+  constexpr int DPL = (DH >= 32) ? DH / 32 : 1;
+  constexpr int RPW = 2;                                  // rows per warp: 8 warps x 2 = 16 rows
+  __shared__ float s_q[kAttnWarps * RPW][DH];
+  __shared__ float s_k[32][DH + 1];
+  __shared__ float s_v[32][DH];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b = blockIdx.x / p.H, h = blockIdx.x % p.H;
+  const CT* K = reinterpret_cast<const CT*>(p.k);
+  const CT* V = reinterpret_cast<const CT*>(p.v);
+  const int* pt = p.st.page_table + b * p.st.pages_per_row;
+  const bool owns = (DH >= 32) || (lane < DH);
+  const int dim0 = (DH >= 32) ? lane * DPL : lane;
+  const int nrows = p.rows_per_b;
+  const int base_limit = p.causal ? p.st.len[b] + 1 : p.limit_b[b];
+  const int limit_max = p.causal ? base_limit + nrows - 1 : base_limit;
+  for (int idx = threadIdx.x; idx < nrows * DH; idx += blockDim.x) {
+    const int i = idx / DH, c = idx % DH;
+    s_q[i][c] = to_f(reinterpret_cast<const QT*>(p.q)[(long long)(b * nrows + i) * p.ldq + h * DH + c]) * p.scale;
+  }
+  float m_run[RPW], l_run[RPW], acc[RPW][DPL];
+#pragma unroll
+  for (int r = 0; r < RPW; ++r) {
+    m_run[r] = -INFINITY; l_run[r] = 0.f;
+#pragma unroll
+    for (int t = 0; t < DPL; ++t) acc[r][t] = 0.f;
+  }
+  for (int c0 = 0; c0 < limit_max; c0 += 32) {
+    const size_t base = p.paged ? ((size_t)pt[c0 / kPage] * kPage + (c0 % kPage)) * p.ldkv + h * DH
+                                : (size_t)b * p.bstride + (size_t)c0 * p.ldkv + h * DH;
+    const int nk = min(32, limit_max - c0);
+    __syncthreads();                                       // the previous chunk is no longer needed
+    for (int v8 = threadIdx.x; v8 < 32 * DH / 8; v8 += blockDim.x) {
+      const int j = v8 / (DH / 8), c = (v8 % (DH / 8)) * 8;
+      float kv[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, vv[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      if (j < nk) {
+        load8(K + base + (size_t)j * p.ldkv + c, kv);
+        load8(V + base + (size_t)j * p.ldkv + c, vv);
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) { s_k[j][c + e] = kv[e]; s_v[j][c + e] = vv[e]; }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < RPW; ++r) {
+      const int i = warp + r * kAttnWarps;
+      if (i >= nrows) continue;                            // uniform over the warp
+      const int limit = p.causal ? base_limit + i : base_limit;
+      const int live = min(32, limit - c0);                // keys of this chunk the row may see
+      if (live <= 0) continue;
+      float sc = -INFINITY;
+      if (lane < live) {
+        float dot = 0.f;
+#pragma unroll
+        for (int c = 0; c < DH; ++c) dot = fmaf(s_q[i][c], s_k[lane][c], dot);
+        sc = dot;
+      }
+      const float m_new = fmaxf(m_run[r], warp_max(sc));
+      const float corr = expf(m_run[r] - m_new);
+      const float pj = (lane < live) ? expf(sc - m_new) : 0.f;
+      l_run[r] = l_run[r] * corr + warp_sum(pj);
+#pragma unroll
+      for (int t = 0; t < DPL; ++t) acc[r][t] *= corr;
+      for (int jj = 0; jj < live; ++jj) {
+        const float pw = __shfl_sync(0xffffffffu, pj, jj);
+        if (owns) {
+#pragma unroll
+          for (int t = 0; t < DPL; ++t) acc[r][t] = fmaf(pw, s_v[jj][dim0 + t], acc[r][t]);
+        }
+      }
+      m_run[r] = m_new;
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < RPW; ++r) {
+    const int i = warp + r * kAttnWarps;
+    if (i >= nrows || !owns) continue;
+    const float inv = 1.f / l_run[r];
+#pragma unroll
+    for (int t = 0; t < DPL; ++t) {
+      const float ov = acc[r][t] * inv;
+      const long long o = (long long)(b * nrows + i) * p.ldo + h * DH + dim0 + t;
+      if (p.out_plane) {
+        bf16* op = reinterpret_cast<bf16*>(p.out) + o;
+        const bf16 hi = __float2bfloat16_rn(ov);
+        op[0] = hi;
+        op[p.out_plane] = __float2bfloat16_rn(ov - __bfloat162float(hi));
+      } else {
+        reinterpret_cast<QT*>(p.out)[o] = from_f<QT>(ov);
+      }
+    }
+  }
+}
+
 // Picks the split kernel for the common head widths, the generic one-warp kernel otherwise.
 template <typename QT, typename CT>
 static void launch_attention(const AttnParams& p, cudaStream_t st, bool pdl = false) {
@@ -632,6 +733,14 @@ static void launch_attention(const AttnParams& p, cudaStream_t st, bool pdl = fa
   const dim3 g(items), b(kAttnWarps * 32);
   if (p.by_rows) {   // many sequences: a CTA per (sequence, head); a property of the session, not of the pass
     const dim3 gr((p.rows / p.rows_per_b) * p.H);
+    if (p.rows_per_b <= 16) {
+      switch (p.dh) {
+        case 16: launch_k(attention_seq_kernel<QT, CT, 16>, gr, b, 0, st, pdl, p); return;
+        case 32: launch_k(attention_seq_kernel<QT, CT, 32>, gr, b, 0, st, pdl, p); return;
+        case 64: launch_k(attention_seq_kernel<QT, CT, 64>, gr, b, 0, st, pdl, p); return;
+        default: break;
+      }
+    }
     switch (p.dh) {
       case 16: launch_k(attention_rows_kernel<QT, CT, 16>, gr, b, 0, st, pdl, p); return;
       case 32: launch_k(attention_rows_kernel<QT, CT, 32>, gr, b, 0, st, pdl, p); return;
