@@ -277,14 +277,19 @@ def run_gpu(args):
                     "peak_kind": f"of {peak_kind}", "traffic": TRAFFIC.get(args.workload),
                     "bytes_per_launch": w2_bytes, "us_per_launch": w2_us, "launches_timed": n_w2}
     else:
-        # batched: the same kernel is a dense contraction; flops of the iterations (the one priming launch
-        # per decode has 1/k of the rows and is left in the average)
-        flops = 2.0 * (w.batch * k) * (w2_bytes / cfg.elem_bytes)
-        achieved = flops / (w2_us * 1e-6) / 1e12
-        roofline = {"bound": "tensor", "kernel": "head output layers (k*d_model x k*d_hidden weights, + residual)",
+        # batched: the same kernel is a dense contraction.  Sessions this wide evaluate the heads lazily: one launch
+        # for head 1 at all batch*k positions, one for all k heads at the accepted position of each row; the
+        # algorithmic flops are those of the two launches, the time is what the pair takes per pass (the priming
+        # pass, one launch on batch rows, is left in the average)
+        kf = cfg.k_model * cfg.d_hidden
+        flops = 2.0 * (w.batch * k) * cfg.d_model * kf + 2.0 * w.batch * (k * cfg.d_model) * kf
+        n_pass = max(1, phases[0][0])
+        pair_us = 1e3 * ms_w2 / n_pass
+        achieved = flops / (pair_us * 1e-6) / 1e12
+        roofline = {"bound": "tensor", "kernel": "head output layers, both lazy stages (k*d_model x k*d_hidden weights)",
                     "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf,
                     "peak_kind": f"of {peak_kind} (sustained bf16)", "traffic": None,
-                    "flops_per_launch": flops, "us_per_launch": w2_us, "launches_timed": n_w2}
+                    "flops_per_pass": flops, "us_per_pass": pair_us, "launches_timed": n_w2}
     phase_us = {name: (1e3 * ms / max(1, n)) for name, (n, ms) in
                 zip(["layers", "head_hidden", "head_output", "vocab_top1"], phases)}
     kernel_names = ["embed", "layer_norm", "qkv", "self_attn", "o_proj", "cross_q", "cross_attn", "cross_o",
