@@ -37,19 +37,32 @@ inline Plan plan_splits(int N, int K, int wide_ttiles = 0) {
   pl.splits = (pl.chunks + pl.chunks_per_split - 1) / pl.chunks_per_split;
   return pl;
 }
-inline int token_tiles(int T) { return (T + kMaxBN - 1) / kMaxBN; }
-inline int token_bn(int T) {
-  const int per = (T + token_tiles(T) - 1) / token_tiles(T);
+// Token tiling of a launch: as few tiles of at most 128 tokens as possible, but -- in sessions with many rows --
+// more, narrower ones (not below 32 tokens) while the launch would otherwise leave SMs without a CTA.  The tile
+// width only changes the MMA's N; every output element is still the same sum in the same order.
+inline int token_tiles(int T, int ctas_per_ttile = 0) {
+  int tt = (T + kMaxBN - 1) / kMaxBN;
+  if (ctas_per_ttile > 0) {
+    const int want = (kSlots / 2 + ctas_per_ttile - 1) / ctas_per_ttile;
+    tt = std::max(tt, std::min(want, (T + 31) / 32));
+  }
+  return std::max(1, tt);
+}
+inline int token_bn(int T, int ttiles) {
+  const int per = (T + ttiles - 1) / ttiles;
   return std::max(16, (per + 15) / 16 * 16);
 }
+inline int token_bn(int T) { return token_bn(T, token_tiles(T)); }
+inline int max_token_tiles(int T) { return std::max(token_tiles(T), (T + 31) / 32); }
 // fp32 elements of split-K workspace a launch with these sizes needs.
 inline size_t ws_floats(int N, int K, int T, int zslices, int wide_ttiles = 0) {
   const Plan pl = plan_splits(N, K, wide_ttiles);
   if (pl.splits == 1) return 0;
-  return (size_t)token_tiles(T) * zslices * pl.tiles * pl.splits * token_bn(T) * kBM;
+  // upper bound over every token tiling the launch may pick: tiles * bn <= T + 16 per tile
+  return (size_t)zslices * pl.tiles * pl.splits * ((size_t)T + 16 * max_token_tiles(T)) * kBM;
 }
 inline size_t counters_needed(int N, int T, int zslices) {
-  return (size_t)token_tiles(T) * zslices * ((N + kBM - 1) / kBM);
+  return (size_t)max_token_tiles(T) * zslices * ((N + kBM - 1) / kBM);
 }
 
 struct Scratch {
@@ -128,9 +141,9 @@ int launch(const Operands& op, int N, int K, int T, TcParams p, const Scratch& s
   // matrix (fewer heads) passes the full count so that every feature is summed in the same order either way.
   Plan pl = plan_splits(plan_n > 0 ? plan_n : N, K, sc.wide_ttiles);
   pl.tiles = (N + kBM - 1) / kBM;
-  const int ttiles = token_tiles(T), bn = token_bn(T);
+  const int ttiles = token_tiles(T, sc.wide_ttiles ? pl.tiles * pl.splits * zslices : 0), bn = token_bn(T, ttiles);
   const size_t need_ws = pl.splits == 1 ? 0 : (size_t)ttiles * zslices * pl.tiles * pl.splits * bn * kBM;
-  const size_t need_cnt = counters_needed(N, T, zslices);
+  const size_t need_cnt = (size_t)ttiles * zslices * pl.tiles;
   if (need_ws > sc.ws_floats || need_cnt > sc.n_counters)
     return fail(BPD_E_NOMEM, "split-K workspace too small (%zu floats, %zu counters needed)", need_ws, need_cnt);
   if (EPI == kTcArgmax && (size_t)T > sc.best_elems) return fail(BPD_E_NOMEM, "top-1 workspace too small");
