@@ -7,7 +7,7 @@ build module can be imported before the library exists).  There is no CPU
 fallback: touching any binding name without a built library raises.
 """
 _BINDING_NAMES = ("BpdError", "Model", "Session", "Stats", "bpd_op_linear", "bpd_op_vocab_argmax", "bpd_op_vocab_argmax_noalloc",
-                  "bpd_kernel_launches", "BPD_ACCEPT_TOPN", "BPD_ACCEPT_DISTANCE", "BPD_ACCEPT_MIN_BLOCK", "bpd_query_sizes", "lib", "EXPORTED")
+                  "bpd_kernel_launches", "bpd_debug_wait_timeout", "BPD_ACCEPT_TOPN", "BPD_ACCEPT_DISTANCE", "BPD_ACCEPT_MIN_BLOCK", "bpd_query_sizes", "lib", "EXPORTED")
 
 
 def __getattr__(name):

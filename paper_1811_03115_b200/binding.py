@@ -63,6 +63,7 @@ _SIGS = {
     "bpd_profile": (_i, [_vp, _i]),
     "bpd_profile_read": (_i, [_vp, _i, C.POINTER(C.c_int64), C.POINTER(C.c_double)]),
     "bpd_fetch_output": (_i, [_vp, _i, _vp, _vp, C.POINTER(bpd_stats)]),
+    "bpd_debug_wait_timeout": (_i, [_vp, _i, _vp]),
     "bpd_op_vocab_argmax_scratch_bytes": (_sz, [_i, _i, _i, _i]),
     "bpd_op_vocab_argmax": (_i, [_vp, _vp, _i, _i, _i, _i, _vp, _sz, _vp, _vp, _vp]),
     "bpd_op_vocab_argmax_noalloc": (_i, [_vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp]),
@@ -263,6 +264,13 @@ class Session:
     @property
     def d_model(self) -> int:
         return int(np.frombuffer(self.model.blob_header[24:28], np.int32)[0])
+
+
+def bpd_debug_wait_timeout(limit_us: int = 2000) -> int:
+    """Runs the bounded-wait self test and returns the status code (BPD_E_TIMEOUT = -7 is the expected outcome)."""
+    import torch
+    word = torch.zeros(1, dtype=torch.int32, device="cuda")
+    return int(lib.bpd_debug_wait_timeout(word.data_ptr(), limit_us, _stream()))
 
 
 def bpd_kernel_launches() -> int:

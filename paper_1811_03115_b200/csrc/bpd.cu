@@ -1095,6 +1095,24 @@ int bpd_fetch_output(bpd_session* s, int max_new, int32_t* out_ids, int32_t* out
   return fetch(s, max_new, out_ids, out_len, stats, ms);
 }
 
+// ------------------------------------------------------------------ self test of the bounded waits
+int bpd_debug_wait_timeout(int32_t* dev_word, int limit_us, void* cuda_stream) {
+  if (!dev_word) return fail(BPD_E_INVALID, "device word is null");
+  if (limit_us < 1 || limit_us > 2000000) return fail(BPD_E_INVALID, "limit_us = %d outside 1..2000000", limit_us);
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  int khz = 0, dev = 0;
+  BPD_CUDA(cudaGetDevice(&dev));
+  BPD_CUDA(cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, dev));
+  BPD_CUDA(cudaMemsetAsync(dev_word, 0, sizeof(int), st));
+  tc::wait_probe_kernel<<<1, 32, 0, st>>>(dev_word, (unsigned long long)limit_us * (unsigned long long)khz / 1000ull);
+  ++g_launches;
+  int word = 0;
+  BPD_CUDA(cudaMemcpyAsync(&word, dev_word, sizeof(int), cudaMemcpyDeviceToHost, st));
+  BPD_CUDA(cudaStreamSynchronize(st));
+  if (word) return fail(BPD_E_TIMEOUT, "a bounded wait inside the probe kernel expired (code %d), as it should", word);
+  return BPD_OK;
+}
+
 // ------------------------------------------------------------------ single operators
 // Scratch layout of the bf16 (tensor-core) operators: a zero "lo" plane for the caller's single-plane bf16
 // activations, the split-K workspace, tile counters, the top-1 merge counter and partials, an error word.

@@ -88,14 +88,14 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
   return ok;
 }
 // Bounded wait: false if the phase did not complete within about a second.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_cycles = kSpinCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
-    if ((unsigned long long)(clock64() - t0) > kSpinCycles) return false;
+    if ((unsigned long long)(clock64() - t0) > limit_cycles) return false;
   }
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
@@ -256,6 +256,19 @@ __device__ __forceinline__ void tc_store8(const TcParams& p, int z, int t_first,
         else p.vcache[s_slot[stat0 + c] + (n - 2 * d)] = __float2bfloat16_rn(v);
       }
     }
+  }
+}
+
+// ---------------------------------------------------------------- bounded-wait self test
+// One CTA waits on an mbarrier that nothing ever arrives on, gives up after `limit_cycles`, records the same
+// error code the projection kernel would and returns normally: the context stays usable.
+static __global__ void wait_probe_kernel(int* error, unsigned long long limit_cycles) {
+  __shared__ __align__(8) unsigned long long bar;
+  const uint32_t b = smem_u32(&bar);
+  if (threadIdx.x == 0) {
+    mbar_init(b, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (!mbar_wait(b, 0, limit_cycles)) atomicCAS(error, 0, 103);
   }
 }
 

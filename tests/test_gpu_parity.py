@@ -384,3 +384,15 @@ def test_lazy_heads_give_the_same_decode(bpd, w, monkeypatch):
     assert max(kh for row in rep.khats for kh in row) > 1
     s.close()
     model.close()
+
+
+def test_bounded_wait_expires_and_the_context_survives(bpd):
+    """Failure detection without a fault: a wait on a barrier nobody signals gives up after its limit,
+    the call reports BPD_E_TIMEOUT and the same process keeps computing correctly afterwards."""
+    import torch
+    assert bpd.bpd_debug_wait_timeout(2000) == -7
+    assert "expired" in bpd.lib.bpd_last_error().decode()
+    x = torch.randn(4, 64).cuda()
+    w = torch.randn(10, 64).cuda()
+    y = bpd.bpd_op_linear(x, w).cpu()
+    assert torch.allclose(y, x.cpu() @ w.cpu().T, atol=1e-4)
