@@ -272,6 +272,194 @@ static __global__ void wait_probe_kernel(int* error, unsigned long long limit_cy
   }
 }
 
+// ---------------------------------------------------------------- epilogue of one (tile, split) unit
+// Shared by the one-shot projection kernel and the persistent layer kernel.  Called by the four epilogue warps
+// (128 threads, named barrier 1).
+struct EpiShared {
+  float (*s_val)[kMaxBN]; int (*s_idx)[kMaxBN];
+  float* s_mean; float* s_rstd;
+  unsigned long long* s_slot;
+  volatile uint32_t* ctl;       // [1] reduces the tile, [2] merges the top-1, [3] accumulator arrived
+};
+struct EpiUnit {
+  uint32_t tmem, acc_bar, acc_parity;
+  int tile, split, slice, zidx, ntiles, zcount, t0, nt, bn, nchunks;
+  bool skip;
+};
+template <int EPI>
+__device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& sh, const EpiUnit& u, int warp, int lane) {
+  float (*s_val)[kMaxBN] = sh.s_val;
+  int (*s_idx)[kMaxBN] = sh.s_idx;
+  float* s_mean = sh.s_mean;
+  float* s_rstd = sh.s_rstd;
+  unsigned long long* s_slot = sh.s_slot;
+  volatile uint32_t* ctl = sh.ctl;
+  const uint32_t tmem = u.tmem;
+  const int tile = u.tile, split = u.split, slice = u.slice, t0 = u.t0, nt = u.nt, bn = u.bn, nchunks = u.nchunks;
+  const bool skip = u.skip;
+  const int q = warp & 3;                          // tensor-memory lane quarter this warp may read
+  const int row = q * 32 + lane;
+  const int n = tile * kBM + row;                  // feature index within the slice
+  const int et = threadIdx.x - 64;                 // 0..127
+  if (EPI == kTcQkv && !skip && et < nt) {
+    const int t = t0 + et;
+    const int b = t / p.rows_per_b, i = t % p.rows_per_b;
+    const int pos = p.st.len[b] + i;
+    const int page = p.st.page_table[b * p.st.pages_per_row + pos / kPage];
+    s_slot[et] = ((unsigned long long)page * kPage + (pos % kPage)) * p.d;
+  }
+  if (p.ln_x && !skip) {
+    // per-token mean and 1/std of the residual stream, computed while the main loop runs: 8 threads per
+    // token (at most 16 tokens per tile in this mode), two passes, fixed order
+    const int tr = et >> 3, part = et & 7;
+    const int trc = min(tr, nt - 1);               // threads beyond the live tokens shadow the last one
+    const float4* xr = reinterpret_cast<const float4*>(p.ln_x + (size_t)(t0 + trc) * p.ln_d);
+    const int nv = p.ln_d >> 2;
+    float sum = 0.f;
+#pragma unroll 8
+    for (int i = part; i < nv; i += 8) { const float4 a = xr[i]; sum += (a.x + a.y) + (a.z + a.w); }
+    sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+    sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+    sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+    const float mean = sum / (float)p.ln_d;
+    float sq = 0.f;
+#pragma unroll 8
+    for (int i = part; i < nv; i += 8) {
+      const float4 a = xr[i];
+      const float d0 = a.x - mean, d1 = a.y - mean, d2 = a.z - mean, d3 = a.w - mean;
+      sq += (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
+    }
+    sq += __shfl_xor_sync(0xffffffffu, sq, 1);
+    sq += __shfl_xor_sync(0xffffffffu, sq, 2);
+    sq += __shfl_xor_sync(0xffffffffu, sq, 4);
+    const float rstd = rsqrtf(sq / (float)p.ln_d + p.ln_eps);
+    if (part == 0 && tr < nt) { s_mean[tr] = mean; s_rstd[tr] = rstd; }
+  }
+  // one thread waits for the accumulator; the other 127 learn the outcome through the named barrier
+  if (et == 0) {
+    bool done = !skip;
+    if (nchunks > 0 && !skip) done = mbar_wait(u.acc_bar, u.acc_parity);
+    if (!done && !skip) atomicCAS(p.error, 0, 103);
+    ctl[3] = done ? 1u : 0u;
+  }
+  asm volatile("bar.sync 1, 128;" ::: "memory");
+  const bool ok = (ctl[3] != 0);
+  tc_fence_after();
+  const int ntiles = u.ntiles;
+  const bool direct = (p.splits == 1);
+  float* wsz = p.ws + ((size_t)u.zidx * ntiles + tile) * p.splits * (size_t)bn * kBM;
+  if (ok) {
+    if (direct) {
+      for (int cb = 0; cb < bn; cb += 16) {
+        float v[16];
+        tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + cb, v);
+        if (EPI != kTcArgmax) {
+          if (n < p.N) {
+            const float lo8[8] = {v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]};
+            const float hi8[8] = {v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15]};
+            tc_store8<EPI>(p, slice, t0 + cb, min(8, nt - cb), n, lo8, s_mean, s_rstd, cb, s_slot);
+            tc_store8<EPI>(p, slice, t0 + cb + 8, min(8, nt - cb - 8), n, hi8, s_mean, s_rstd, cb + 8, s_slot);
+          }
+        } else {
+#pragma unroll
+          for (int c = 0; c < 16; ++c) {
+            float x = (n < p.N) ? v[c] : -INFINITY;
+            int ix = (n < p.N) ? n : 0x7fffffff;
+            if (p.logits && cb + c < nt && n < p.N) p.logits[(size_t)(t0 + cb + c) * p.N + n] = x;
+            if (cb + c < nt) count_beats(p, t0 + cb + c, n, x, lane);
+            warp_argmax(x, ix);
+            if (lane == 0) { s_val[q][cb + c] = x; s_idx[q][cb + c] = ix; }
+          }
+        }
+      }
+    } else {
+      // partial tile -> workspace [split][token][128], coalesced over features
+      for (int cb = 0; cb < bn; cb += 16) {
+        float v[16];
+        if (nchunks > 0) tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + cb, v);
+        else {
+#pragma unroll
+          for (int c = 0; c < 16; ++c) v[c] = 0.f;
+        }
+#pragma unroll
+        for (int c = 0; c < 16; ++c)
+          if (cb + c < nt) wsz[((size_t)split * bn + cb + c) * kBM + row] = v[c];
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (et == 0) {
+        const unsigned prev = atom_add_acq_rel(&p.tile_counters[(size_t)u.zidx * ntiles + tile], 1u);
+        ctl[1] = (prev == (unsigned)p.splits - 1) ? 1u : 0u;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (ctl[1]) {
+        // splits are added in split order; the loads of eight splits x eight tokens are issued together
+        for (int cg = 0; cg < nt; cg += 8) {
+          float acc[8];
+#pragma unroll
+          for (int c = 0; c < 8; ++c) acc[c] = 0.f;
+          for (int s0 = 0; s0 < p.splits; s0 += 8) {
+            float v[8][8];
+#pragma unroll
+            for (int ss = 0; ss < 8; ++ss)
+#pragma unroll
+              for (int c = 0; c < 8; ++c)
+                v[ss][c] = (s0 + ss < p.splits && cg + c < nt)
+                               ? __ldcg(&wsz[((size_t)(s0 + ss) * bn + cg + c) * kBM + row]) : 0.f;
+#pragma unroll
+            for (int ss = 0; ss < 8; ++ss)
+#pragma unroll
+              for (int c = 0; c < 8; ++c) acc[c] += v[ss][c];
+          }
+          if (EPI != kTcArgmax) {
+            if (n < p.N) tc_store8<EPI>(p, slice, t0 + cg, min(8, nt - cg), n, acc, s_mean, s_rstd, cg, s_slot);
+          } else {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              if (cg + c >= nt) break;
+              float x = (n < p.N) ? acc[c] : -INFINITY;
+              int ix = (n < p.N) ? n : 0x7fffffff;
+              if (p.logits && n < p.N) p.logits[(size_t)(t0 + cg + c) * p.N + n] = x;
+              count_beats(p, t0 + cg + c, n, x, lane);
+              warp_argmax(x, ix);
+              if (lane == 0) { s_val[q][cg + c] = x; s_idx[q][cg + c] = ix; }
+            }
+          }
+        }
+        if (et == 0) p.tile_counters[(size_t)u.zidx * ntiles + tile] = 0;   // ready for the next launch
+      }
+    }
+    if (EPI == kTcArgmax && (direct || ctl[1])) {
+      // tile-level (value, index) per token, then the CTA that completes the last tile merges all tiles
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (et < nt) {
+        float x = s_val[0][et];
+        int ix = s_idx[0][et];
+#pragma unroll
+        for (int w = 1; w < 4; ++w)
+          if (better(s_val[w][et], s_idx[w][et], x, ix)) { x = s_val[w][et]; ix = s_idx[w][et]; }
+        // one 64-bit atomic max per (tile, token): larger value wins, equal values go to the lower index;
+        // max is order independent, so the result does not depend on which tile arrives first
+        atomicMax(&p.best[t0 + et], pack_best(x, ix));
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (et == 0) {
+        const unsigned prev = atom_add_acq_rel(p.done_counter, 1u);
+        ctl[2] = (prev == (unsigned)(ntiles * u.zcount) - 1) ? 1u : 0u;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (ctl[2]) {
+        for (int t = et; t < p.T; t += 128) {
+          const unsigned long long key = __ldcg(&p.best[t]);
+          p.out_idx[t] = (int)(0xffffffffu - (unsigned)(key & 0xffffffffull));
+          if (p.out_val) p.out_val[t] = unpack_value(key);
+          p.best[t] = 0ull;                       // ready for the next launch
+        }
+        if (et == 0) *p.done_counter = 0;
+      }
+    }
+  }
+}
+
 // ---------------------------------------------------------------- the kernel
 // grid = (feature tiles, K splits, z), z = token tile * zslices + slice (slices: block-diagonal heads).
 // tmA: weights [N, K]; tmBh / tmBl: activation planes [rows, K]; box = (64, 128) and (64, bn).
@@ -385,169 +573,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (!ok) atomicCAS(p.error, 0, 102);
   } else if (warp >= 2) {
     // ---------------- epilogue: thread = one feature row, registers = tokens
-    const int q = warp & 3;                          // tensor-memory lane quarter this warp may read
-    const int row = q * 32 + lane;
-    const int n = tile * kBM + row;                  // feature index within the slice
-    const int et = threadIdx.x - 64;                 // 0..127
     pdl_wait();
-    const bool skip = p.all_done && *p.all_done;     // same value in every thread: the flag is stable by now
-    if (EPI == kTcQkv && !skip && et < nt) {
-      const int t = t0 + et;
-      const int b = t / p.rows_per_b, i = t % p.rows_per_b;
-      const int pos = p.st.len[b] + i;
-      const int page = p.st.page_table[b * p.st.pages_per_row + pos / kPage];
-      s_slot[et] = ((unsigned long long)page * kPage + (pos % kPage)) * p.d;
-    }
-    if (p.ln_x && !skip) {
-      // per-token mean and 1/std of the residual stream, computed while the main loop runs: 8 threads per
-      // token (at most 16 tokens per tile in this mode), two passes, fixed order
-      const int tr = et >> 3, part = et & 7;
-      const int trc = min(tr, nt - 1);               // threads beyond the live tokens shadow the last one
-      const float4* xr = reinterpret_cast<const float4*>(p.ln_x + (size_t)(t0 + trc) * p.ln_d);
-      const int nv = p.ln_d >> 2;
-      float sum = 0.f;
-#pragma unroll 8
-      for (int i = part; i < nv; i += 8) { const float4 a = xr[i]; sum += (a.x + a.y) + (a.z + a.w); }
-      sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-      sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-      sum += __shfl_xor_sync(0xffffffffu, sum, 4);
-      const float mean = sum / (float)p.ln_d;
-      float sq = 0.f;
-#pragma unroll 8
-      for (int i = part; i < nv; i += 8) {
-        const float4 a = xr[i];
-        const float d0 = a.x - mean, d1 = a.y - mean, d2 = a.z - mean, d3 = a.w - mean;
-        sq += (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
-      }
-      sq += __shfl_xor_sync(0xffffffffu, sq, 1);
-      sq += __shfl_xor_sync(0xffffffffu, sq, 2);
-      sq += __shfl_xor_sync(0xffffffffu, sq, 4);
-      const float rstd = rsqrtf(sq / (float)p.ln_d + p.ln_eps);
-      if (part == 0 && tr < nt) { s_mean[tr] = mean; s_rstd[tr] = rstd; }
-    }
-    // one thread waits for the accumulator; the other 127 learn the outcome through the named barrier
-    if (et == 0) {
-      bool done = !skip;
-      if (nchunks > 0 && !skip) done = mbar_wait(bars + 8 * 2 * kStages, 0);
-      if (!done && !skip) atomicCAS(p.error, 0, 103);
-      ctl[3] = done ? 1u : 0u;
-    }
-    asm volatile("bar.sync 1, 128;" ::: "memory");
-    ok = (ctl[3] != 0);
-    tc_fence_after();
-    const int ntiles = gridDim.x;
-    const bool direct = (p.splits == 1);
-    float* wsz = p.ws + ((size_t)blockIdx.z * ntiles + tile) * p.splits * (size_t)bn * kBM;
-    if (ok) {
-      if (direct) {
-        for (int cb = 0; cb < bn; cb += 16) {
-          float v[16];
-          tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + cb, v);
-          if (EPI != kTcArgmax) {
-            if (n < p.N) {
-              const float lo8[8] = {v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]};
-              const float hi8[8] = {v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15]};
-              tc_store8<EPI>(p, slice, t0 + cb, min(8, nt - cb), n, lo8, s_mean, s_rstd, cb, s_slot);
-              tc_store8<EPI>(p, slice, t0 + cb + 8, min(8, nt - cb - 8), n, hi8, s_mean, s_rstd, cb + 8, s_slot);
-            }
-          } else {
-#pragma unroll
-            for (int c = 0; c < 16; ++c) {
-              float x = (n < p.N) ? v[c] : -INFINITY;
-              int ix = (n < p.N) ? n : 0x7fffffff;
-              if (p.logits && cb + c < nt && n < p.N) p.logits[(size_t)(t0 + cb + c) * p.N + n] = x;
-              if (cb + c < nt) count_beats(p, t0 + cb + c, n, x, lane);
-              warp_argmax(x, ix);
-              if (lane == 0) { s_val[q][cb + c] = x; s_idx[q][cb + c] = ix; }
-            }
-          }
-        }
-      } else {
-        // partial tile -> workspace [split][token][128], coalesced over features
-        for (int cb = 0; cb < bn; cb += 16) {
-          float v[16];
-          if (nchunks > 0) tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + cb, v);
-          else {
-#pragma unroll
-            for (int c = 0; c < 16; ++c) v[c] = 0.f;
-          }
-#pragma unroll
-          for (int c = 0; c < 16; ++c)
-            if (cb + c < nt) wsz[((size_t)split * bn + cb + c) * kBM + row] = v[c];
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (et == 0) {
-          const unsigned prev = atom_add_acq_rel(&p.tile_counters[(size_t)blockIdx.z * ntiles + tile], 1u);
-          ctl[1] = (prev == (unsigned)p.splits - 1) ? 1u : 0u;
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (ctl[1]) {
-          // splits are added in split order; the loads of eight splits x eight tokens are issued together
-          for (int cg = 0; cg < nt; cg += 8) {
-            float acc[8];
-#pragma unroll
-            for (int c = 0; c < 8; ++c) acc[c] = 0.f;
-            for (int s0 = 0; s0 < p.splits; s0 += 8) {
-              float v[8][8];
-#pragma unroll
-              for (int ss = 0; ss < 8; ++ss)
-#pragma unroll
-                for (int c = 0; c < 8; ++c)
-                  v[ss][c] = (s0 + ss < p.splits && cg + c < nt)
-                                 ? __ldcg(&wsz[((size_t)(s0 + ss) * bn + cg + c) * kBM + row]) : 0.f;
-#pragma unroll
-              for (int ss = 0; ss < 8; ++ss)
-#pragma unroll
-                for (int c = 0; c < 8; ++c) acc[c] += v[ss][c];
-            }
-            if (EPI != kTcArgmax) {
-              if (n < p.N) tc_store8<EPI>(p, slice, t0 + cg, min(8, nt - cg), n, acc, s_mean, s_rstd, cg, s_slot);
-            } else {
-#pragma unroll
-              for (int c = 0; c < 8; ++c) {
-                if (cg + c >= nt) break;
-                float x = (n < p.N) ? acc[c] : -INFINITY;
-                int ix = (n < p.N) ? n : 0x7fffffff;
-                if (p.logits && n < p.N) p.logits[(size_t)(t0 + cg + c) * p.N + n] = x;
-                count_beats(p, t0 + cg + c, n, x, lane);
-                warp_argmax(x, ix);
-                if (lane == 0) { s_val[q][cg + c] = x; s_idx[q][cg + c] = ix; }
-              }
-            }
-          }
-          if (et == 0) p.tile_counters[(size_t)blockIdx.z * ntiles + tile] = 0;   // ready for the next launch
-        }
-      }
-      if (EPI == kTcArgmax && (direct || ctl[1])) {
-        // tile-level (value, index) per token, then the CTA that completes the last tile merges all tiles
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (et < nt) {
-          float x = s_val[0][et];
-          int ix = s_idx[0][et];
-#pragma unroll
-          for (int w = 1; w < 4; ++w)
-            if (better(s_val[w][et], s_idx[w][et], x, ix)) { x = s_val[w][et]; ix = s_idx[w][et]; }
-          // one 64-bit atomic max per (tile, token): larger value wins, equal values go to the lower index;
-          // max is order independent, so the result does not depend on which tile arrives first
-          atomicMax(&p.best[t0 + et], pack_best(x, ix));
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (et == 0) {
-          const unsigned prev = atom_add_acq_rel(p.done_counter, 1u);
-          ctl[2] = (prev == (unsigned)(ntiles * (gridDim.z / zslices)) - 1) ? 1u : 0u;
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (ctl[2]) {
-          for (int t = et; t < p.T; t += 128) {
-            const unsigned long long key = __ldcg(&p.best[t]);
-            p.out_idx[t] = (int)(0xffffffffu - (unsigned)(key & 0xffffffffull));
-            if (p.out_val) p.out_val[t] = unpack_value(key);
-            p.best[t] = 0ull;                       // ready for the next launch
-          }
-          if (et == 0) *p.done_counter = 0;
-        }
-      }
-    }
+    const EpiShared sh{s_val, s_idx, s_mean, s_rstd, s_slot, ctl};
+    const EpiUnit u{tmem, bars + 8 * 2 * kStages, 0u, tile, split, slice, (int)blockIdx.z, (int)gridDim.x,
+                    (int)gridDim.z / zslices, t0, nt, bn, nchunks, p.all_done && *p.all_done};
+    tc_epilogue<EPI>(p, sh, u, warp, lane);
   }
   tc_fence_before();
   __syncthreads();
