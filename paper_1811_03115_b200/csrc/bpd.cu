@@ -11,6 +11,7 @@
 #include "host.hpp"
 #include "kernels_simt.cuh"
 #include "tc_host.hpp"
+#include "fused_layer.cuh"
 
 namespace bpd {
 
@@ -193,7 +194,13 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
   unsigned* tc_counters = a.take<unsigned>(ncnt);
   unsigned* tc_done = a.take<unsigned>(1);
   unsigned long long* tc_best = a.take<unsigned long long>(R2);
+  // fused decoder layers (few rows per pass): per-head / per-cluster shares of the output projections, slice counters
+  const bool fused_ok = c.dtype == 1 && fused::supported(c.d, c.H, c.d_ff, (int)Rmax);
+  const size_t fused_parts = std::max<size_t>(c.H, c.d_ff / (fused::kC * fused::kHS));
+  float* fused_ws = a.take<float>(fused_ok ? fused_parts * Rmax * d : 0);
+  unsigned* fused_counters = a.take<unsigned>(fused::kC);
   if (s) {
+    s->fused_ws = fused_ws; s->fused_counters = fused_counters;
     s->x = x; s->h_f32 = h_f32; s->xn = xn; s->qbuf = qbuf; s->attn = attn; s->ffh = ffh; s->u = u; s->o = o;
     s->crosskv = crosskv; s->kcache = kc; s->vcache = vc; s->st = st; s->src_dev = src_dev;
     s->tail_dev = tail_dev; s->plan_dev = plan_dev; s->part_val = part_val; s->part_idx = part_idx;
@@ -498,6 +505,86 @@ static int run_encoder_tc(bpd_session* s) {
   return BPD_OK;
 }
 
+// ------------------------------------------------------------------ fused decoder layers (few rows per pass)
+template <typename P>
+static int fused_attr(void (*kernel)(P), size_t smem) {
+  BPD_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  return BPD_OK;
+}
+
+// Embedding, then three launches per decoder layer (self-attention block, cross-attention block, feed-forward
+// block); leaves the residual stream in s->x like the kernel-per-projection path.
+static int run_layers_fused(bpd_session* s, const PassArgs& a) {
+  const bpd_model* m = s->m;
+  const Config& c = m->cfg;
+  cudaStream_t st = s->stream;
+  const int d = c.d, R = s->B * a.kcur;
+  const int* done = s->st.all_done;
+  const bool pdl = s->use_pdl != 0;
+  const int nt = (R + 7) / 8;
+  const size_t smem_self = fused::attn_layout<true>(d, nt).total, smem_cross = fused::attn_layout<false>(d, nt).total;
+  const size_t smem_ffn = fused::ffn_layout(d, nt).total;
+  // the opt-in shared-memory limit of each kernel grows with the widest model seen so far
+  static size_t attr_max[3][3] = {{0, 0, 0}, {0, 0, 0}, {0, 0, 0}};
+  if (smem_self > attr_max[nt][0] || smem_cross > attr_max[nt][1] || smem_ffn > attr_max[nt][2]) {
+    if (nt == 1) {
+      BPD_TRY(fused_attr(fused::attn_block_kernel<true, 1>, smem_self));
+      BPD_TRY(fused_attr(fused::attn_block_kernel<false, 1>, smem_cross));
+      BPD_TRY(fused_attr(fused::ffn_block_kernel<1>, smem_ffn));
+    } else {
+      BPD_TRY(fused_attr(fused::attn_block_kernel<true, 2>, smem_self));
+      BPD_TRY(fused_attr(fused::attn_block_kernel<false, 2>, smem_cross));
+      BPD_TRY(fused_attr(fused::ffn_block_kernel<2>, smem_ffn));
+    }
+    attr_max[nt][0] = smem_self; attr_max[nt][1] = smem_cross; attr_max[nt][2] = smem_ffn;
+  }
+  EmbedParams ep;
+  memset(&ep, 0, sizeof(ep));
+  ep.table = m->tgt_embed; ep.pe = s->pe; ep.npos = s->npos; ep.x = s->x; ep.rows = R; ep.rows_per_b = a.kcur;
+  ep.d = d; ep.vocab = c.V; ep.st = s->st; ep.forced = a.forced; ep.forced_rows = a.forced_rows;
+  ep.kforced = a.kforced; ep.src = nullptr; ep.all_done = done;
+  embed_kernel<bf16><<<R, 128, 0, st>>>(ep);
+  ++g_launches;
+  const dim3 block(fused::kThreads), grid_attn(fused::kC, c.H), grid_ffn(fused::kC, c.d_ff / (fused::kC * fused::kHS));
+  for (int l = 0; l < c.n_dec; ++l) {
+    const DecLayer& L = m->dec[l];
+    fused::AttnBlockParams ps;
+    memset(&ps, 0, sizeof(ps));
+    ps.x = s->x; ps.gain = static_cast<const bf16*>(L.ln1g); ps.fold_s = L.s_qkv; ps.fold_c = L.c_qkv;
+    ps.w_in = static_cast<const bf16*>(L.wqkv); ps.w_out = static_cast<const bf16*>(L.wo);
+    ps.d = d; ps.H = c.H; ps.R = R; ps.rows_per_b = a.kcur; ps.eps = c.eps;
+    ps.kcache = static_cast<bf16*>(s->kcache[l]); ps.vcache = static_cast<bf16*>(s->vcache[l]);
+    ps.attn.rows = R; ps.attn.rows_per_b = a.kcur; ps.attn.H = c.H; ps.attn.dh = fused::kDH; ps.attn.causal = 1;
+    ps.attn.k = s->kcache[l]; ps.attn.v = s->vcache[l]; ps.attn.ldkv = d; ps.attn.paged = 1; ps.attn.st = s->st;
+    ps.attn.scale = 1.0f / sqrtf((float)fused::kDH);
+    ps.ws = s->fused_ws; ps.counters = s->fused_counters; ps.all_done = done;
+    fused::AttnBlockParams pc = ps;
+    pc.gain = static_cast<const bf16*>(L.ln2g); pc.fold_s = L.s_cq; pc.fold_c = L.c_cq;
+    pc.w_in = static_cast<const bf16*>(L.cwq); pc.w_out = static_cast<const bf16*>(L.cwo);
+    pc.kcache = nullptr; pc.vcache = nullptr;
+    pc.attn.causal = 0; pc.attn.limit_b = s->st.src_len; pc.attn.k = s->crosskv[l];
+    pc.attn.v = static_cast<float*>(s->crosskv[l]) + d; pc.attn.ldkv = 2 * d;
+    pc.attn.bstride = (long long)s->max_src * 2 * d; pc.attn.paged = 0;
+    fused::FfnBlockParams pf;
+    memset(&pf, 0, sizeof(pf));
+    pf.x = s->x; pf.gain = static_cast<const bf16*>(L.ln3g); pf.fold_s = L.s_f1; pf.fold_c = L.c_f1;
+    pf.w1 = static_cast<const bf16*>(L.w1); pf.w2 = static_cast<const bf16*>(L.w2); pf.b2 = static_cast<const bf16*>(L.b2);
+    pf.d = d; pf.ff = c.d_ff; pf.R = R; pf.NJ = (int)grid_ffn.y; pf.eps = c.eps;
+    pf.ws = s->fused_ws; pf.counters = s->fused_counters; pf.all_done = done;
+    if (nt == 1) {
+      BPD_CUDA(launch_k(fused::attn_block_kernel<true, 1>, grid_attn, block, smem_self, st, pdl, ps));
+      BPD_CUDA(launch_k(fused::attn_block_kernel<false, 1>, grid_attn, block, smem_cross, st, pdl, pc));
+      BPD_CUDA(launch_k(fused::ffn_block_kernel<1>, grid_ffn, block, smem_ffn, st, pdl, pf));
+    } else {
+      BPD_CUDA(launch_k(fused::attn_block_kernel<true, 2>, grid_attn, block, smem_self, st, pdl, ps));
+      BPD_CUDA(launch_k(fused::attn_block_kernel<false, 2>, grid_attn, block, smem_cross, st, pdl, pc));
+      BPD_CUDA(launch_k(fused::ffn_block_kernel<2>, grid_ffn, block, smem_ffn, st, pdl, pf));
+    }
+    g_launches += 3;
+  }
+  return BPD_OK;
+}
+
 #define PROF(slot, ...) do { prof_mark(s, slot, 0); __VA_ARGS__; prof_mark(s, slot, 1); } while (0)
 static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   const bpd_model* m = s->m;
@@ -508,7 +595,11 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   const tc::Scratch sc = tc_scratch(s);
   const bool pdl = s->use_pdl != 0;
   const bool fold = s->fold_ln != 0;   // every kernel after the first may overlap its predecessor's tail
+  const tc::Operands xn{nullptr, 0, s->xn, s->pl_xn, d, s->rows_all, d};
+  auto with_w = [](tc::Operands o, const void* w, int rows) { o.w = w; o.w_rows = rows; return o; };
   prof_mark(s, kProfLayers, 0);
+  if (s->fused) BPD_TRY(run_layers_fused(s, a));
+  else {
   EmbedParams ep;
   memset(&ep, 0, sizeof(ep));
   ep.table = m->tgt_embed; ep.pe = s->pe; ep.npos = s->npos; ep.x = s->x; ep.rows = R; ep.rows_per_b = a.kcur;
@@ -517,10 +608,8 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   if (fold) { ep.gain = static_cast<const bf16*>(m->dec[0].ln1g); ep.xg_hi = static_cast<bf16*>(s->xn); ep.xg_plane = s->pl_xn; }
   PROF(kProfEmbed, embed_kernel<bf16><<<R, 128, 0, st>>>(ep););
   ++g_launches;
-  const tc::Operands xn{nullptr, 0, s->xn, s->pl_xn, d, s->rows_all, d};
   const tc::Operands at{nullptr, 0, s->attn, s->pl_attn, d, s->rows_all, d};
   const tc::Operands fx{nullptr, 0, s->ffh, s->pl_ffh, f, s->rows_all, f};
-  auto with_w = [](tc::Operands o, const void* w, int rows) { o.w = w; o.w_rows = rows; return o; };
   for (int l = 0; l < c.n_dec; ++l) {
     const DecLayer& L = m->dec[l];
     if (!fold) PROF(kProfLn, launch_ln<bf16, float>(s->x, L.ln1g, L.ln1b, s->xn, nullptr, R, d, c.eps, done, st, s->pl_xn, pdl););
@@ -561,6 +650,7 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
     p2.out_f32 = s->x; p2.ldo = d;
     if (fold && l + 1 < c.n_dec) { p2.g_next = static_cast<const bf16*>(m->dec[l + 1].ln1g); p2.xg_hi = static_cast<bf16*>(s->xn); p2.xg_plane = s->pl_xn; }
     PROF(kProfFfn2, BPD_TRY(tc::launch<tc::kTcResidual>(with_w(fx, L.w2, d), d, f, R, p2, sc, st, 1, 0, 0, pdl)); ++g_launches);
+  }
   }
   PROF(kProfLn, launch_ln<bf16, float>(s->x, m->dec_lnf_g, m->dec_lnf_b, s->xn, s->h_f32, R, d, c.eps, done, st, s->pl_xn, pdl););
   prof_mark(s, kProfLayers, 1);
@@ -834,6 +924,8 @@ int bpd_session_create(const bpd_model* model, int batch, int max_src, int max_t
   s->lazy_heads = s->tc && (lz ? atoi(lz) != 0 : batch * model->cfg.k_model >= 64);
   s->last_pass_lazy = 0;
   s->fold_ln = (s->tc && batch * model->cfg.k_model <= 16 && !getenv("BPD_DISABLE_FOLD")) ? 1 : 0;
+  s->fused = (s->tc && fused::supported(model->cfg.d, model->cfg.H, model->cfg.d_ff, batch * model->cfg.k_model) &&
+              !getenv("BPD_DISABLE_FUSED")) ? 1 : 0;
   s->phase = kPhaseCreated; s->plan_len = 0; s->plan_k = 0; s->invocations = 0; s->pinned = nullptr;
   plan_session(model->cfg, batch, max_src, max_tgt, s->base, s);
   // page table: row b's p-th page is physical page p*B + b (rows interleaved in the pool)

@@ -33,6 +33,22 @@ __device__ __forceinline__ void load8(const float* p, float (&out)[8]) {
   out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
   out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
 }
+// Same, read from L2 (data another SM may have written earlier in the same launch must not come from L1).
+__device__ __forceinline__ void load8_cg(const bf16* p, float (&out)[8]) {
+  uint4 raw = __ldcg(reinterpret_cast<const uint4*>(p));
+  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    out[2 * i] = __uint_as_float(w[i] << 16);
+    out[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
+__device__ __forceinline__ void load8_cg(const float* p, float (&out)[8]) {
+  float4 a = __ldcg(reinterpret_cast<const float4*>(p));
+  float4 b = __ldcg(reinterpret_cast<const float4*>(p + 4));
+  out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
+  out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
+}
 // Same, bypassing L1 (weights are streamed once).
 __device__ __forceinline__ void load8_stream(const bf16* p, float (&out)[8]) {
   uint4 raw = __ldcs(reinterpret_cast<const uint4*>(p));

@@ -1,0 +1,548 @@
+// Decoder layers for sessions with few rows per pass (batch 1, at most 16 rows): three launches per layer
+// instead of eight.
+//
+// With so few rows a decoder layer is a chain of eight small dependent steps, and the time goes to what separates
+// them (launch, a trip to L2 and back, a device-wide join), not to the 29 MB of weights.  Most of those joins are
+// not needed: a head's attention only needs that head's 3 x 64 query/key/value features, and the output
+// projection is a sum over heads.  So
+//
+//   attn_block_kernel<SELF>   layer norm -> Q,K,V of one head -> cache write -> attention -> that head's share of
+//                             the output projection -> sum over heads + residual
+//   attn_block_kernel<CROSS>  layer norm -> Q of one head -> attention over the encoder keys -> same tail
+//   ffn_block_kernel          layer norm -> 32 hidden units (ReLU) -> their share of the second projection ->
+//                             sum over all hidden slices + bias + residual
+//
+// One thread-block cluster of kC CTAs works on a head (or on kC hidden slices); inside it the reduction length
+// is split over the CTAs and partial sums travel through distributed shared memory, always added in rank
+// order.  Across clusters the partial outputs go through a small workspace and the last cluster to arrive adds
+// them in cluster order, so every element is the same sum in the same order however many rows a pass carries.
+// Weights are static: every CTA starts copying its slice into shared memory before it waits for the previous
+// launch (programmatic dependent launch), which takes HBM latency off the chain.
+//
+// The products are tiny (at most 16 columns), so they run on mma.sync (m16n8k16, bf16 in, fp32 out) straight
+// from shared memory; activations are two bf16 planes (hi + lo) as everywhere else on the tensor-core path.
+#pragma once
+#include <cooperative_groups.h>
+
+#include "gemm_tc.cuh"
+#include "kernels_simt.cuh"
+
+namespace bpd {
+namespace fused {
+
+namespace cg = cooperative_groups;
+
+constexpr int kC = 8;            // CTAs per cluster
+constexpr int kThreads = 256;
+constexpr int kWarps = 8;
+constexpr int kDH = 64;          // head width this path is built for
+constexpr int kHS = 32;          // hidden units per CTA in the feed-forward block
+constexpr int kMaxRows = 16;
+
+// Row stride (bytes) of a shared-memory matrix whose rows hold `row_bytes` (a multiple of 64): congruent to 64
+// mod 128, so that the 16-byte fragment loads of eight lanes (two rows x four quarters) cover all 32 banks once.
+__host__ __device__ inline int padded(int row_bytes) { return (row_bytes % 128 == 0) ? row_bytes + 64 : row_bytes; }
+
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(tc::smem_u32(smem)), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+// Cluster barrier in two halves (all threads of the CTA execute both).  The first pair of a kernel only makes
+// sure that every CTA of the cluster is running before anybody writes into its shared memory.
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// v = hi + lo with hi, lo bf16 (as 16-bit patterns).
+__device__ __forceinline__ void split_bits(float v, uint32_t& hi, uint32_t& lo) {
+  bf16 h, l;
+  tc::split_bf16(v, h, l);
+  hi = __bfloat16_as_ushort(h);
+  lo = __bfloat16_as_ushort(l);
+}
+
+// acc[nt] += W(16 rows x K) * X(K x 8 tokens of tile nt), X = hi + lo planes.
+// w: first of 16 weight rows in shared memory (row-major, sw bytes apart); xh / xl: planes, one row per token (sx
+// bytes apart).  K is a multiple of 32.  The contraction index is permuted inside each group of 32 so that a
+// lane's fragments are 16 contiguous bytes: lane (g, t) takes k = 8t..8t+7 of rows g and g+8 and of token g, and
+// uses them as slots {2t, 2t+1, 2t+8, 2t+9} of two successive MMAs -- the same permutation on both operands.
+// acc[nt][0..3] = (row g, token 2t), (row g, token 2t+1), (row g+8, token 2t), (row g+8, token 2t+1).
+template <int NT>
+__device__ __forceinline__ void mma_rows16(float (&acc)[NT][4], const uint8_t* w, int sw, const uint8_t* xh, const uint8_t* xl,
+                                           int sx, int K, int lane) {
+  const int g = lane >> 2, t = lane & 3;
+  const uint8_t* w0 = w + g * sw + t * 16;
+  const uint8_t* w1 = w0 + 8 * sw;
+  for (int k0 = 0; k0 < K; k0 += 32) {
+    const uint4 a = *reinterpret_cast<const uint4*>(w0 + k0 * 2);
+    const uint4 b = *reinterpret_cast<const uint4*>(w1 + k0 * 2);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const uint4 h = *reinterpret_cast<const uint4*>(xh + (nt * 8 + g) * sx + t * 16 + k0 * 2);
+      const uint4 l = *reinterpret_cast<const uint4*>(xl + (nt * 8 + g) * sx + t * 16 + k0 * 2);
+      mma_bf16(acc[nt], a.x, b.x, a.y, b.y, h.x, h.y);
+      mma_bf16(acc[nt], a.x, b.x, a.y, b.y, l.x, l.y);
+      mma_bf16(acc[nt], a.z, b.z, a.w, b.w, h.z, h.w);
+      mma_bf16(acc[nt], a.z, b.z, a.w, b.w, l.z, l.w);
+    }
+  }
+}
+
+// Rows of the residual stream: per-token mean and 1/std (all columns) and the planes of x * gain for columns
+// [k_lo, k_lo + ks).  One warp per token (tokens w, w+8), every lane a fixed share of the row, one pass: each lane
+// sums its share about its own first element, then the 32 partial (count, mean, M2) triples are merged pairwise
+// in a fixed order.  Rows come from L2: another launch wrote them.
+__device__ __forceinline__ void rows_stats_planes(const float* x, const bf16* gain, int R, int d, float eps, int k_lo, int ks,
+                                                  uint8_t* xh, uint8_t* xl, int sx, float* s_mean, float* s_rstd) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nv = d >> 2;
+  for (int tk = warp; tk < R; tk += kWarps) {
+    const float4* xr = reinterpret_cast<const float4*>(x + (size_t)tk * d);
+    float cnt = 0.f, mu = 0.f, m2 = 0.f;
+    if (lane < nv) {
+      const float shift = __ldcg(&xr[lane]).x;
+      float a1 = 0.f, a2 = 0.f;
+      int n = 0;
+#pragma unroll 8
+      for (int i = lane; i < nv; i += 32) {
+        const float4 a = __ldcg(&xr[i]);
+        const float d0 = a.x - shift, d1 = a.y - shift, d2 = a.z - shift, d3 = a.w - shift;
+        a1 += (d0 + d1) + (d2 + d3);
+        a2 += (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
+        n += 4;
+        const int col = i * 4 - k_lo;
+        if (col >= 0 && col < ks) {
+          const uint2 gw = *reinterpret_cast<const uint2*>(gain + i * 4);
+          const float v[4] = {a.x * __uint_as_float(gw.x << 16), a.y * __uint_as_float(gw.x & 0xffff0000u),
+                              a.z * __uint_as_float(gw.y << 16), a.w * __uint_as_float(gw.y & 0xffff0000u)};
+          uint32_t hi[4], lo[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) split_bits(v[e], hi[e], lo[e]);
+          *reinterpret_cast<uint2*>(xh + tk * sx + col * 2) = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
+          *reinterpret_cast<uint2*>(xl + tk * sx + col * 2) = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
+        }
+      }
+      cnt = (float)n;
+      mu = shift + a1 / (float)n;
+      m2 = a2 - a1 * a1 / (float)n;
+    }
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const float cb = __shfl_xor_sync(0xffffffffu, cnt, off);
+      const float mb = __shfl_xor_sync(0xffffffffu, mu, off);
+      const float qb = __shfl_xor_sync(0xffffffffu, m2, off);
+      // the lower lane of a pair is "a" on both sides, so both lanes evaluate the same expression
+      const bool low = (lane & off) == 0;
+      const float ca = low ? cnt : cb, ma = low ? mu : mb, qa = low ? m2 : qb;
+      const float c2 = low ? cb : cnt, mc = low ? mb : mu, q2 = low ? qb : m2;
+      const float n = ca + c2;
+      if (n > 0.f) {
+        const float delta = mc - ma;
+        mu = ma + delta * (c2 / n);
+        m2 = qa + q2 + delta * delta * (ca * c2 / n);
+      }
+      cnt = n;
+    }
+    if (lane == 0) {
+      s_mean[tk] = mu;
+      s_rstd[tk] = rsqrtf(fmaxf(m2, 0.f) / (float)d + eps);
+    }
+  }
+}
+
+// Sum over `np` partial outputs + residual (+ bias) for the feature slice [col0, col0 + width) of all R rows, by
+// the CTA that completed the slice: x[t][f] += bias[f] + ws[0][t][f] + ws[1][t][f] + ... in that order.
+__device__ __forceinline__ void merge_slice(float* x, const float* ws, const bf16* bias, int np, int R, int d, int col0, int width) {
+  const int w4 = width >> 2;
+  for (int idx = threadIdx.x; idx < R * w4; idx += kThreads) {
+    const int t = idx / w4, col = col0 + (idx % w4) * 4;
+    float4 acc = __ldcg(reinterpret_cast<const float4*>(x + (size_t)t * d + col));
+    if (bias) {
+      const uint2 bw = *reinterpret_cast<const uint2*>(bias + col);
+      acc.x += __uint_as_float(bw.x << 16); acc.y += __uint_as_float(bw.x & 0xffff0000u);
+      acc.z += __uint_as_float(bw.y << 16); acc.w += __uint_as_float(bw.y & 0xffff0000u);
+    }
+    const float4* wp = reinterpret_cast<const float4*>(ws + (size_t)t * d + col);
+    const size_t step = (size_t)R * d / 4;
+#pragma unroll 8
+    for (int p = 0; p < np; ++p) {
+      const float4 v = __ldcg(wp + p * step);
+      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    *reinterpret_cast<float4*>(x + (size_t)t * d + col) = acc;
+  }
+}
+
+// ------------------------------------------------------------------ attention block (self or cross)
+struct AttnBlockParams {
+  float* x;                       // residual stream [R, d], updated in place
+  const bf16* gain;               // layer-norm gain [d]
+  const float* fold_s;            // layer norm folded into the input projection: y = rstd (acc - mean s[n]) + c[n]
+  const float* fold_c;
+  const bf16* w_in;               // [3d, d] (self: Q, K, V stacked) or [d, d] (cross: Q)
+  const bf16* w_out;              // [d, d]
+  int d, H, R, rows_per_b;
+  float eps;
+  bf16* kcache; bf16* vcache;     // self: paged cache of this layer, new rows are written here
+  AttnParams attn;                // keys / values, paging, lengths, scale (q and out are not used)
+  float* ws;                      // [H][R][d] per-head shares of the output projection
+  unsigned* counters;             // [kC], zero between launches
+  const int* all_done;
+};
+
+struct AttnLayout {
+  int s_in, s_out, s_x;           // row strides (bytes)
+  int w_in, w_out, xh, xl, oh, ol, part, q, mean, rstd, attn, flag, total;   // offsets (bytes)
+  int zero_begin, zero_end;       // planes that must start at zero
+};
+template <bool SELF>
+__host__ __device__ inline AttnLayout attn_layout(int d, int NT) {
+  AttnLayout L;
+  const int ks = d / kC, rows_in = SELF ? 3 * kDH : kDH;
+  L.s_in = padded(ks * 2); L.s_out = padded(kDH * 2); L.s_x = padded(ks * 2);
+  int off = 0;
+  L.w_in = off; off += rows_in * L.s_in;
+  L.w_out = off; off += (d / kC) * L.s_out;
+  L.zero_begin = off;
+  L.xh = off; off += NT * 8 * L.s_x;
+  L.xl = off; off += NT * 8 * L.s_x;
+  L.oh = off; off += NT * 8 * L.s_out;
+  L.ol = off; off += NT * 8 * L.s_out;
+  L.zero_end = off;
+  L.part = off; off += kC * NT * rows_in * 4;
+  L.q = off; off += NT * kDH * 4;
+  L.mean = off; off += kMaxRows * 4;
+  L.rstd = off; off += kMaxRows * 4;
+  L.attn = off; off += (int)((sizeof(AttnSmem<kDH, kWarps>) + 15) / 16 * 16);
+  L.flag = off; off += 16;
+  L.total = off;
+  return L;
+}
+
+template <bool SELF, int NT>
+__global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_block_kernel(AttnBlockParams p) {
+  extern __shared__ __align__(16) uint8_t fsm[];
+  cg::cluster_group cluster = cg::this_cluster();
+  const int c = (int)cluster.block_rank(), h = blockIdx.y;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, t4 = lane & 3;
+  const int d = p.d, ks = d / kC, slice = d / kC;
+  constexpr int ROWS_IN = SELF ? 3 * kDH : kDH;
+  const AttnLayout L = attn_layout<SELF>(d, NT);
+  uint8_t* w_in_s = fsm + L.w_in;
+  uint8_t* w_out_s = fsm + L.w_out;
+  uint8_t* xh_s = fsm + L.xh;
+  uint8_t* xl_s = fsm + L.xl;
+  uint8_t* oh_s = fsm + L.oh;
+  uint8_t* ol_s = fsm + L.ol;
+  float* part_s = reinterpret_cast<float*>(fsm + L.part);
+  float* q_s = reinterpret_cast<float*>(fsm + L.q);
+  float* s_mean = reinterpret_cast<float*>(fsm + L.mean);
+  float* s_rstd = reinterpret_cast<float*>(fsm + L.rstd);
+  AttnSmem<kDH, kWarps>& sm = *reinterpret_cast<AttnSmem<kDH, kWarps>*>(fsm + L.attn);
+  volatile int* flag = reinterpret_cast<volatile int*>(fsm + L.flag);
+
+  pdl_launch_dependents();
+  // This CTA's weights -- ROWS_IN rows x ks columns of the input projection, `slice` rows x 64 columns of the
+  // output projection -- do not depend on the previous launch: start copying them now.
+  {
+    const int cpr = ks * 2 / 16;
+    for (int idx = tid; idx < ROWS_IN * cpr; idx += kThreads) {
+      const int row = idx / cpr, c16 = idx % cpr;
+      const int grow = (row / kDH) * d + h * kDH + (row % kDH);
+      cp_async16(w_in_s + row * L.s_in + c16 * 16, p.w_in + (size_t)grow * d + c * ks + c16 * 8);
+    }
+    for (int idx = tid; idx < slice * 8; idx += kThreads) {
+      const int row = idx >> 3, c16 = idx & 7;
+      cp_async16(w_out_s + row * L.s_out + c16 * 16, p.w_out + (size_t)(c * slice + row) * d + h * kDH + c16 * 8);
+    }
+    cp_async_commit();
+  }
+  for (int i = L.zero_begin / 16 + tid; i < L.zero_end / 16; i += kThreads) reinterpret_cast<uint4*>(fsm)[i] = make_uint4(0, 0, 0, 0);
+  pdl_wait();
+  if (p.all_done && *p.all_done) {      // the same answer in every CTA: nobody reaches a cluster barrier
+    cp_async_wait_all();
+    return;
+  }
+  cluster_arrive();
+  __syncthreads();
+  rows_stats_planes(p.x, p.gain, p.R, d, p.eps, c * ks, ks, xh_s, xl_s, L.s_x, s_mean, s_rstd);
+  cp_async_wait_all();
+  __syncthreads();
+  cluster_wait();
+
+  // ---- input projection over this CTA's part of the reduction; token t's partial goes to rank t % kC
+  for (int mt = warp; mt < ROWS_IN / 16; mt += kWarps) {
+    float acc[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+    mma_rows16<NT>(acc, w_in_s + mt * 16 * L.s_in, L.s_in, xh_s, xl_s, L.s_x, ks, lane);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int row = mt * 16 + g + ((e & 2) ? 8 : 0), token = nt * 8 + 2 * t4 + (e & 1);
+        if (token < p.R) {
+          float* remote = cluster.map_shared_rank(part_s, token % kC);
+          remote[(c * NT + token / kC) * ROWS_IN + row] = acc[nt][e];
+        }
+      }
+  }
+  cluster.sync();
+
+  // ---- this rank's tokens: add the partials in rank order, finish the layer norm, write keys / values
+  for (int slot = 0; slot < NT; ++slot) {
+    const int token = slot * kC + c;
+    if (token < p.R && tid < ROWS_IN) {
+      float a = 0.f;
+#pragma unroll
+      for (int src = 0; src < kC; ++src) a += part_s[(src * NT + slot) * ROWS_IN + tid];
+      const int sect = tid / kDH, f = tid % kDH;
+      const int n = sect * d + h * kDH + f;
+      const float y = s_rstd[token] * (a - s_mean[token] * p.fold_s[n]) + p.fold_c[n];
+      if (sect == 0) {
+        q_s[slot * kDH + f] = y * p.attn.scale;
+      } else {
+        const int b = token / p.rows_per_b, i = token % p.rows_per_b;
+        const int pos = p.attn.st.len[b] + i;
+        const int page = p.attn.st.page_table[b * p.attn.st.pages_per_row + pos / kPage];
+        const size_t at = ((size_t)page * kPage + (pos % kPage)) * d + h * kDH + f;
+        (sect == 1 ? p.kcache : p.vcache)[at] = __float2bfloat16_rn(y);
+      }
+    }
+  }
+  if (SELF) {
+    __threadfence();
+    cluster.sync();                      // the block's new keys and values are in the cache for every rank's rows
+  } else {
+    __syncthreads();
+  }
+
+  // ---- attention of this rank's rows; the result goes to every rank as planes
+  for (int slot = 0; slot < NT; ++slot) {
+    const int token = slot * kC + c;
+    if (token < p.R) {                   // uniform over the CTA
+      if (tid < kDH) sm.q[tid] = q_s[slot * kDH + tid];
+      __syncthreads();
+      const int b = token / p.rows_per_b, i = token % p.rows_per_b;
+      const int limit = p.attn.causal ? (p.attn.st.len[b] + i + 1) : p.attn.limit_b[b];
+      float ov;
+      if (SELF) ov = attention_head<bf16, kDH, kWarps, true>(p.attn, b, h, limit, sm);
+      else ov = attention_head<float, kDH, kWarps, false>(p.attn, b, h, limit, sm);
+      if (tid < kDH) {
+        uint32_t hi, lo;
+        split_bits(ov, hi, lo);
+#pragma unroll
+        for (int dst = 0; dst < kC; ++dst) {
+          reinterpret_cast<unsigned short*>(cluster.map_shared_rank(oh_s, dst) + token * L.s_out)[tid] = (unsigned short)hi;
+          reinterpret_cast<unsigned short*>(cluster.map_shared_rank(ol_s, dst) + token * L.s_out)[tid] = (unsigned short)lo;
+        }
+      }
+      __syncthreads();
+    }
+  }
+  cluster.sync();
+
+  // ---- this head's share of the output projection for the features of slice c
+  float* wsh = p.ws + (size_t)h * p.R * d;
+  for (int mt = warp; mt < slice / 16; mt += kWarps) {
+    float acc[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+    mma_rows16<NT>(acc, w_out_s + mt * 16 * L.s_out, L.s_out, oh_s, ol_s, L.s_out, kDH, lane);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int row = mt * 16 + g + ((e & 2) ? 8 : 0), token = nt * 8 + 2 * t4 + (e & 1);
+        if (token < p.R) wsh[(size_t)token * d + c * slice + row] = acc[nt][e];
+      }
+  }
+  __syncthreads();
+  if (tid == 0) *flag = (tc::atom_add_acq_rel(&p.counters[c], 1u) == (unsigned)p.H - 1) ? 1 : 0;
+  __syncthreads();
+  if (*flag) {                           // last head to arrive at this slice: heads are added in head order
+    merge_slice(p.x, p.ws, nullptr, p.H, p.R, d, c * slice, slice);
+    if (tid == 0) p.counters[c] = 0;
+  }
+}
+
+// ------------------------------------------------------------------ feed-forward block
+struct FfnBlockParams {
+  float* x;                       // residual stream [R, d], updated in place
+  const bf16* gain;
+  const float* fold_s;            // layer norm folded into the first projection (c also holds its bias)
+  const float* fold_c;
+  const bf16* w1;                 // [ff, d]
+  const bf16* w2;                 // [d, ff]
+  const bf16* b2;                 // [d]
+  int d, ff, R, NJ;               // NJ clusters, each kC * kHS hidden units
+  float eps;
+  float* ws;                      // [NJ][R][d] per-cluster shares of the second projection
+  unsigned* counters;             // [kC], zero between launches
+  const int* all_done;
+};
+
+struct FfnLayout {
+  int s1, s2, s_x, s_h;
+  int w1, w2, xh, xl, hh, hl, part1, mean, rstd, flag, total;   // part2 shares the bytes of w1
+  int zero_begin, zero_end;
+};
+__host__ __device__ inline FfnLayout ffn_layout(int d, int NT) {
+  FfnLayout L;
+  const int ks = d / kC, slice = d / kC;
+  L.s1 = padded(ks * 2); L.s2 = padded(kHS * 2); L.s_x = padded(ks * 2); L.s_h = padded(kHS * 2);
+  int off = 0;
+  const int w1_bytes = kC * kHS * L.s1, part2_bytes = kC * slice * NT * 8 * 4;
+  L.w1 = off; off += (w1_bytes > part2_bytes ? w1_bytes : part2_bytes);
+  L.w2 = off; off += d * L.s2;
+  L.zero_begin = off;
+  L.xh = off; off += NT * 8 * L.s_x;
+  L.xl = off; off += NT * 8 * L.s_x;
+  L.hh = off; off += NT * 8 * L.s_h;
+  L.hl = off; off += NT * 8 * L.s_h;
+  L.zero_end = off;
+  L.part1 = off; off += kC * kHS * NT * 8 * 4;
+  L.mean = off; off += kMaxRows * 4;
+  L.rstd = off; off += kMaxRows * 4;
+  L.flag = off; off += 16;
+  L.total = off;
+  return L;
+}
+
+template <int NT>
+__global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 1) ffn_block_kernel(FfnBlockParams p) {
+  extern __shared__ __align__(16) uint8_t fsm[];
+  cg::cluster_group cluster = cg::this_cluster();
+  const int c = (int)cluster.block_rank(), j = blockIdx.y;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, t4 = lane & 3;
+  const int d = p.d, ks = d / kC, slice = d / kC;
+  const int hid_cluster = j * kC * kHS, hid0 = hid_cluster + c * kHS;
+  const FfnLayout L = ffn_layout(d, NT);
+  uint8_t* w1_s = fsm + L.w1;
+  float* part2_s = reinterpret_cast<float*>(fsm + L.w1);
+  uint8_t* w2_s = fsm + L.w2;
+  uint8_t* xh_s = fsm + L.xh;
+  uint8_t* xl_s = fsm + L.xl;
+  uint8_t* hh_s = fsm + L.hh;
+  uint8_t* hl_s = fsm + L.hl;
+  float* part1_s = reinterpret_cast<float*>(fsm + L.part1);
+  float* s_mean = reinterpret_cast<float*>(fsm + L.mean);
+  float* s_rstd = reinterpret_cast<float*>(fsm + L.rstd);
+  volatile int* flag = reinterpret_cast<volatile int*>(fsm + L.flag);
+
+  pdl_launch_dependents();
+  // Static weights of this CTA: the cluster's kC * kHS rows of the first projection restricted to this rank's ks
+  // columns, and this rank's kHS columns of the second projection (all d rows).
+  {
+    const int cpr = ks * 2 / 16;
+    for (int idx = tid; idx < kC * kHS * cpr; idx += kThreads) {
+      const int row = idx / cpr, c16 = idx % cpr;
+      cp_async16(w1_s + row * L.s1 + c16 * 16, p.w1 + (size_t)(hid_cluster + row) * d + c * ks + c16 * 8);
+    }
+    constexpr int cpr2 = kHS * 2 / 16;
+    for (int idx = tid; idx < d * cpr2; idx += kThreads) {
+      const int row = idx / cpr2, c16 = idx % cpr2;
+      cp_async16(w2_s + row * L.s2 + c16 * 16, p.w2 + (size_t)row * p.ff + hid0 + c16 * 8);
+    }
+    cp_async_commit();
+  }
+  for (int i = L.zero_begin / 16 + tid; i < L.zero_end / 16; i += kThreads) reinterpret_cast<uint4*>(fsm)[i] = make_uint4(0, 0, 0, 0);
+  pdl_wait();
+  if (p.all_done && *p.all_done) {
+    cp_async_wait_all();
+    return;
+  }
+  cluster_arrive();
+  __syncthreads();
+  rows_stats_planes(p.x, p.gain, p.R, d, p.eps, c * ks, ks, xh_s, xl_s, L.s_x, s_mean, s_rstd);
+  cp_async_wait_all();
+  __syncthreads();
+  cluster_wait();
+
+  // ---- first projection of the cluster's hidden units over this rank's columns; unit f belongs to rank f / kHS
+  for (int mt = warp; mt < kC * kHS / 16; mt += kWarps) {
+    float acc[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+    mma_rows16<NT>(acc, w1_s + mt * 16 * L.s1, L.s1, xh_s, xl_s, L.s_x, ks, lane);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int f = mt * 16 + g + ((e & 2) ? 8 : 0), token = nt * 8 + 2 * t4 + (e & 1);
+        if (token < p.R) {
+          float* remote = cluster.map_shared_rank(part1_s, f / kHS);
+          remote[(c * kHS + f % kHS) * (NT * 8) + token] = acc[nt][e];
+        }
+      }
+  }
+  cluster.sync();            // from here on nobody reads its w1 slice any more: part2 may overwrite it
+
+  // ---- this rank's hidden units: partials in rank order, layer norm, bias, ReLU, planes
+  for (int idx = tid; idx < kHS * p.R; idx += kThreads) {
+    const int f = idx % kHS, token = idx / kHS;
+    float a = 0.f;
+#pragma unroll
+    for (int src = 0; src < kC; ++src) a += part1_s[(src * kHS + f) * (NT * 8) + token];
+    const int n = hid0 + f;
+    const float y = fmaxf(s_rstd[token] * (a - s_mean[token] * p.fold_s[n]) + p.fold_c[n], 0.f);
+    uint32_t hi, lo;
+    split_bits(y, hi, lo);
+    reinterpret_cast<unsigned short*>(hh_s + token * L.s_h)[f] = (unsigned short)hi;
+    reinterpret_cast<unsigned short*>(hl_s + token * L.s_h)[f] = (unsigned short)lo;
+  }
+  __syncthreads();
+
+  // ---- second projection restricted to these kHS hidden units, all d features; feature n belongs to rank n / slice
+  for (int mt = warp; mt < d / 16; mt += kWarps) {
+    float acc[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+    mma_rows16<NT>(acc, w2_s + mt * 16 * L.s2, L.s2, hh_s, hl_s, L.s_h, kHS, lane);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int n = mt * 16 + g + ((e & 2) ? 8 : 0), token = nt * 8 + 2 * t4 + (e & 1);
+        if (token < p.R) {
+          float* remote = cluster.map_shared_rank(part2_s, n / slice);
+          remote[(c * slice + n % slice) * (NT * 8) + token] = acc[nt][e];
+        }
+      }
+  }
+  cluster.sync();
+
+  // ---- the cluster's share of this rank's feature slice, then the sum over clusters by the last one to arrive
+  float* wsj = p.ws + (size_t)j * p.R * d;
+  for (int idx = tid; idx < slice * p.R; idx += kThreads) {
+    const int f = idx % slice, token = idx / slice;
+    float a = 0.f;
+#pragma unroll
+    for (int src = 0; src < kC; ++src) a += part2_s[(src * slice + f) * (NT * 8) + token];
+    wsj[(size_t)token * d + c * slice + f] = a;
+  }
+  __syncthreads();
+  if (tid == 0) *flag = (tc::atom_add_acq_rel(&p.counters[c], 1u) == (unsigned)p.NJ - 1) ? 1 : 0;
+  __syncthreads();
+  if (*flag) {
+    merge_slice(p.x, p.ws, p.b2, p.NJ, p.R, d, c * slice, slice);
+    if (tid == 0) p.counters[c] = 0;
+  }
+}
+
+// Shapes this path is built for.
+__host__ inline bool supported(int d, int H, int ff, int rows) {
+  return H > 0 && d == H * kDH && d % (kC * 32) == 0 && ff % (kC * kHS) == 0 && rows >= 1 && rows <= kMaxRows;
+}
+
+}  // namespace fused
+}  // namespace bpd

@@ -141,6 +141,9 @@ struct bpd_session {
   int last_pass_lazy;
   void* u2; long long pl_u2; float* h2; int *table2, *table_full;
   int fold_ln;             // decoder layer norms are folded into the projections (few rows only)
+  int fused;               // decoder layers as three launches each (clusters; at most 16 rows per pass)
+  float* fused_ws;
+  unsigned* fused_counters;
   std::map<GraphKey, GraphEntry> graphs;
   std::vector<cudaEvent_t> prof_begin[kProfSlots], prof_end[kProfSlots];
 };

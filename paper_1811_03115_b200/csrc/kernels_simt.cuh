@@ -29,12 +29,9 @@ struct EmbedParams {
   const int* all_done;
 };
 
+// One row of the embedding (all threads of the CTA).
 template <typename WT>
-__global__ void embed_kernel(EmbedParams p) {
-  pdl_launch_dependents();
-  pdl_wait();
-  if (p.all_done && *p.all_done) return;
-  const int r = blockIdx.x;
+__device__ __forceinline__ void embed_row(const EmbedParams& p, int r) {
   const int b = r / p.rows_per_b, i = r % p.rows_per_b;
   int tok, pos;
   if (p.src) {
@@ -85,6 +82,14 @@ __global__ void embed_kernel(EmbedParams p) {
       *reinterpret_cast<uint4*>(dst + p.xg_plane) = *reinterpret_cast<const uint4*>(lo);
     }
   }
+}
+
+template <typename WT>
+__global__ void embed_kernel(EmbedParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
+  if (p.all_done && *p.all_done) return;
+  embed_row<WT>(p, blockIdx.x);
 }
 
 // ------------------------------------------------------------------ folding a layer norm into the projection after it
@@ -447,23 +452,44 @@ template <> __device__ __forceinline__ void load_n<4>(const bf16* p, float (&o)[
   o[2] = __uint_as_float(v.y << 16); o[3] = __uint_as_float(v.y & 0xffff0000u);
 }
 
-template <typename QT, typename CT, int DH>
-__global__ void __launch_bounds__(kAttnWarps * 32) attention_split_kernel(AttnParams p) {
-  pdl_launch_dependents();
-  pdl_wait();
-  if (p.all_done && *p.all_done) return;
+template <int DH, int NW> struct AttnSmem {
+  float q[DH];
+  float m[NW], l[NW];
+  float acc[NW][DH];
+};
+// Variants of load_n that read from L2 (see COHERENT below).
+template <int N> __device__ __forceinline__ void load_n_cg(const float* p, float (&o)[N]) {
+#pragma unroll
+  for (int i = 0; i < N; ++i) o[i] = __ldcg(p + i);
+}
+template <> __device__ __forceinline__ void load_n_cg<2>(const float* p, float (&o)[2]) {
+  const float2 v = __ldcg(reinterpret_cast<const float2*>(p)); o[0] = v.x; o[1] = v.y;
+}
+template <> __device__ __forceinline__ void load_n_cg<4>(const float* p, float (&o)[4]) {
+  const float4 v = __ldcg(reinterpret_cast<const float4*>(p)); o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w;
+}
+template <int N> __device__ __forceinline__ void load_n_cg(const bf16* p, float (&o)[N]) {
+#pragma unroll
+  for (int i = 0; i < N; ++i) o[i] = __uint_as_float((uint32_t)__ldcg(reinterpret_cast<const unsigned short*>(p + i)) << 16);
+}
+template <> __device__ __forceinline__ void load_n_cg<2>(const bf16* p, float (&o)[2]) {
+  const uint32_t v = __ldcg(reinterpret_cast<const uint32_t*>(p));
+  o[0] = __uint_as_float(v << 16); o[1] = __uint_as_float(v & 0xffff0000u);
+}
+template <> __device__ __forceinline__ void load_n_cg<4>(const bf16* p, float (&o)[4]) {
+  const uint2 v = __ldcg(reinterpret_cast<const uint2*>(p));
+  o[0] = __uint_as_float(v.x << 16); o[1] = __uint_as_float(v.x & 0xffff0000u);
+  o[2] = __uint_as_float(v.y << 16); o[3] = __uint_as_float(v.y & 0xffff0000u);
+}
+
+// Attention of one query row and one head by a CTA of NW warps (see the comment above).  sm.q holds the scaled
+// query and a __syncthreads() lies between its writes and this call.  Threads c < DH return output element c.
+// COHERENT: keys and values may have been written by other SMs earlier in the same launch, so they are read
+// from L2 rather than through L1.
+template <typename CT, int DH, int NW, bool COHERENT>
+__device__ __forceinline__ float attention_head(const AttnParams& p, int b, int h, int limit, AttnSmem<DH, NW>& sm) {
   constexpr int DPL = (DH >= 32) ? DH / 32 : 1;       // output dims per lane (contiguous)
-  __shared__ float s_q[DH];
-  __shared__ float s_m[kAttnWarps], s_l[kAttnWarps];
-  __shared__ float s_acc[kAttnWarps][DH];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int item = blockIdx.x;
-  const int r = item / p.H, h = item % p.H;
-  const int b = r / p.rows_per_b, i = r % p.rows_per_b;
-  const int limit = p.causal ? (p.st.len[b] + i + 1) : p.limit_b[b];
-  const QT* q = reinterpret_cast<const QT*>(p.q) + (long long)r * p.ldq + h * DH;
-  if (threadIdx.x < DH) s_q[threadIdx.x] = to_f(q[threadIdx.x]) * p.scale;
-  __syncthreads();
   const CT* K = reinterpret_cast<const CT*>(p.k);
   const CT* V = reinterpret_cast<const CT*>(p.v);
   const int* pt = p.st.page_table + b * p.st.pages_per_row;
@@ -474,7 +500,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_split_kernel(AttnPa
   const int nchunks = (limit + 31) >> 5;
   const bool owns = (DH >= 32) || (lane < DH);
   const int dim0 = (DH >= 32) ? lane * DPL : lane;
-  for (int ch = warp; ch < nchunks; ch += kAttnWarps) {
+  for (int ch = warp; ch < nchunks; ch += NW) {
     const int c0 = ch << 5;
     // a 32-key chunk never straddles a 64-position page
     const size_t base = p.paged ? ((size_t)pt[c0 / kPage] * kPage + (c0 % kPage)) * p.ldkv + h * DH
@@ -487,9 +513,9 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_split_kernel(AttnPa
 #pragma unroll
       for (int c = 0; c < DH; c += 8) {
         float kv[8];
-        load8(kr + c, kv);
+        if (COHERENT) load8_cg(kr + c, kv); else load8(kr + c, kv);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) dot = fmaf(s_q[c + e], kv[e], dot);
+        for (int e = 0; e < 8; ++e) dot = fmaf(sm.q[c + e], kv[e], dot);
       }
       sc = dot;
     }
@@ -505,32 +531,49 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_split_kernel(AttnPa
       const float pw = __shfl_sync(0xffffffffu, pj, jj);
       if (owns) {
         float vv[DPL];
-        load_n<DPL>(vb + (size_t)jj * p.ldkv, vv);
+        if (COHERENT) load_n_cg<DPL>(vb + (size_t)jj * p.ldkv, vv); else load_n<DPL>(vb + (size_t)jj * p.ldkv, vv);
 #pragma unroll
         for (int t = 0; t < DPL; ++t) acc[t] = fmaf(pw, vv[t], acc[t]);
       }
     }
     m_run = m_new;
   }
-  if (lane == 0) { s_m[warp] = m_run; s_l[warp] = l_run; }
+  if (lane == 0) { sm.m[warp] = m_run; sm.l[warp] = l_run; }
   if (owns) {
 #pragma unroll
-    for (int t = 0; t < DPL; ++t) s_acc[warp][dim0 + t] = acc[t];
+    for (int t = 0; t < DPL; ++t) sm.acc[warp][dim0 + t] = acc[t];
   }
   __syncthreads();
+  float ov = 0.f;
   if (threadIdx.x < DH) {
     const int c = threadIdx.x;
-    float M = s_m[0];
+    float M = sm.m[0];
 #pragma unroll
-    for (int w = 1; w < kAttnWarps; ++w) M = fmaxf(M, s_m[w]);
+    for (int w = 1; w < NW; ++w) M = fmaxf(M, sm.m[w]);
     float num = 0.f, den = 0.f;
 #pragma unroll
-    for (int w = 0; w < kAttnWarps; ++w) {
-      const float e = expf(s_m[w] - M);          // warps without keys hold -inf: weight 0
-      num = fmaf(e, s_acc[w][c], num);
-      den = fmaf(e, s_l[w], den);
+    for (int w = 0; w < NW; ++w) {
+      const float e = expf(sm.m[w] - M);          // warps without keys hold -inf: weight 0
+      num = fmaf(e, sm.acc[w][c], num);
+      den = fmaf(e, sm.l[w], den);
     }
-    const float ov = num / den;
+    ov = num / den;
+  }
+  return ov;
+}
+
+// One (row, head) item of a launch: query from p.q, output to p.out; callers separate items with __syncthreads().
+template <typename QT, typename CT, int DH, int NW>
+__device__ __forceinline__ void attention_item(const AttnParams& p, int item, AttnSmem<DH, NW>& sm) {
+  const int r = item / p.H, h = item % p.H;
+  const int b = r / p.rows_per_b, i = r % p.rows_per_b;
+  const int limit = p.causal ? (p.st.len[b] + i + 1) : p.limit_b[b];
+  const QT* q = reinterpret_cast<const QT*>(p.q) + (long long)r * p.ldq + h * DH;
+  if (threadIdx.x < DH) sm.q[threadIdx.x] = to_f(q[threadIdx.x]) * p.scale;
+  __syncthreads();
+  const float ov = attention_head<CT, DH, NW, false>(p, b, h, limit, sm);
+  if (threadIdx.x < DH) {
+    const int c = threadIdx.x;
     if (p.out_plane) {
       bf16* op = reinterpret_cast<bf16*>(p.out) + (long long)r * p.ldo + h * DH + c;
       const bf16 hi = __float2bfloat16_rn(ov);
@@ -540,6 +583,15 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_split_kernel(AttnPa
       reinterpret_cast<QT*>(p.out)[(long long)r * p.ldo + h * DH + c] = from_f<QT>(ov);
     }
   }
+}
+
+template <typename QT, typename CT, int DH>
+__global__ void __launch_bounds__(kAttnWarps * 32) attention_split_kernel(AttnParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
+  if (p.all_done && *p.all_done) return;
+  __shared__ AttnSmem<DH, kAttnWarps> sm;
+  attention_item<QT, CT, DH, kAttnWarps>(p, blockIdx.x, sm);
 }
 
 // Attention for sessions with many rows: one CTA per (sequence, head), one warp per query row (rows beyond

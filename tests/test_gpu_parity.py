@@ -11,6 +11,10 @@ MINI = Workload("mini", ModelConfig(2, 2, 128, 2, 256, 1000, 4, 256, dtype=DTYPE
                 11, 12, 13, batch=1, src_lo=9, src_hi=9, n_decode=24)
 MINI_BLOCK = MINI.with_layout(HEAD_BLOCKDIAG)
 MINI_BATCH = Workload("mini3", MINI.cfg, 0.05, 11, 22, 23, batch=3, src_lo=3, src_hi=11, n_decode=20)
+# shapes the three-launches-per-layer decoder path takes (head width 64, d_model a multiple of 256)
+MIDI = Workload("midi", ModelConfig(2, 2, 256, 4, 512, 1000, 4, 256, dtype=DTYPE_BF16), 0.05,
+                41, 42, 43, batch=1, src_lo=9, src_hi=9, n_decode=24)
+MIDI_BATCH = Workload("midi3", MIDI.cfg, 0.05, 41, 52, 53, batch=3, src_lo=3, src_hi=11, n_decode=20)
 MINI_F32 = Workload("minif", ModelConfig(1, 2, 96, 6, 200, 333, 3, 136, dtype=DTYPE_F32), 0.1,
                     31, 32, 33, batch=2, src_lo=2, src_hi=7, n_decode=15)
 
@@ -108,7 +112,8 @@ def test_op_vocab_argmax_matches_definition(bpd, dtype, rows, d, vocab):
 
 # ---------------------------------------------------------------- whole path, small models
 
-@pytest.mark.parametrize("w", [WORKLOADS["C1"], MINI, MINI_BLOCK, MINI_BATCH, MINI_F32], ids=lambda w: w.name)
+@pytest.mark.parametrize("w", [WORKLOADS["C1"], MINI, MINI_BLOCK, MINI_BATCH, MINI_F32, MIDI, MIDI_BATCH],
+                         ids=lambda w: w.name)
 def test_greedy_blockwise_and_lockstep(bpd, w):
     from harness import lockstep
     blob, model, src, src_len, om = _setup(bpd, w)
@@ -384,6 +389,32 @@ def test_lazy_heads_give_the_same_decode(bpd, w, monkeypatch):
     assert max(kh for row in rep.khats for kh in row) > 1
     s.close()
     model.close()
+
+@pytest.mark.parametrize("w", [MIDI, MIDI_BATCH], ids=lambda w: w.name)
+def test_fused_layers_agree_with_kernel_per_projection(bpd, w, monkeypatch):
+    """Sessions with few rows run each decoder layer as three launches (one cluster per head / per group of hidden
+    units).  The sums are split differently from the kernel-per-projection path, so the two agree to fp32
+    rounding of bf16-weight products, far inside the oracle tolerance."""
+    blob, model, src, src_len, om = _setup(bpd, w)
+    k, N = w.cfg.k_model, w.n_decode
+
+    def run():
+        s = bpd.Session(model, w.batch, w.max_src, N)
+        s.bpd_encode(src, src_len)
+        steps = []
+        for _ in range(4):
+            r = s.bpd_iteration(k, N, want_logits=True, want_hidden=True)
+            steps.append((r["hidden"].cpu().numpy().copy(), r["logits"].cpu().numpy().copy()))
+        s.close()
+        return steps
+
+    a_steps = run()
+    monkeypatch.setenv("BPD_DISABLE_FUSED", "1")
+    b_steps = run()
+    for (ha, la), (hb, lb) in zip(a_steps, b_steps):
+        assert np.abs(ha - hb).max() <= 2e-3 and np.abs(la - lb).max() <= 2e-3
+    model.close()
+
 
 
 def test_bounded_wait_expires_and_the_context_survives(bpd):
