@@ -9,7 +9,7 @@
 //   attn_block_kernel<SELF>   layer norm -> Q,K,V of one head -> cache write -> attention -> that head's share of
 //                             the output projection -> sum over heads + residual
 //   attn_block_kernel<CROSS>  layer norm -> Q of one head -> attention over the encoder keys -> same tail
-//   ffn_block_kernel          layer norm -> 32 hidden units (ReLU) -> their share of the second projection ->
+//   ffn_block_kernel          layer norm -> 16 hidden units (ReLU) -> their share of the second projection ->
 //                             sum over all hidden slices + bias + residual
 //
 // One thread-block cluster of kC CTAs works on a head (or on kC hidden slices); inside it the reduction length
@@ -36,7 +36,7 @@ constexpr int kC = 8;            // CTAs per cluster
 constexpr int kThreads = 256;
 constexpr int kWarps = 8;
 constexpr int kDH = 64;          // head width this path is built for
-constexpr int kHS = 32;          // hidden units per CTA in the feed-forward block
+constexpr int kHS = 16;          // hidden units per CTA in the feed-forward block
 constexpr int kMaxRows = 16;
 
 // Row stride (bytes) of a shared-memory matrix whose rows hold `row_bytes` (a multiple of 64): congruent to 64
@@ -98,37 +98,50 @@ __device__ __forceinline__ void mma_rows16(float (&acc)[NT][4], const uint8_t* w
 // Rows of the residual stream: per-token mean and 1/std (all columns) and the planes of x * gain for columns
 // [k_lo, k_lo + ks).  One warp per token (tokens w, w+8), every lane a fixed share of the row, one pass: each lane
 // sums its share about its own first element, then the 32 partial (count, mean, M2) triples are merged pairwise
-// in a fixed order.  Rows come from L2: another launch wrote them.
-__device__ __forceinline__ void rows_stats_planes(const float* x, const bf16* gain, int R, int d, float eps, int k_lo, int ks,
-                                                  uint8_t* xh, uint8_t* xl, int sx, float* s_mean, float* s_rstd) {
+// in a fixed order.  Rows come from L2 (another launch wrote them), eight loads per lane in flight.
+__device__ __forceinline__ void rows_stats_planes(const float* __restrict__ x, const bf16* __restrict__ gain, int R, int d,
+                                                  float eps, int k_lo, int ks, uint8_t* __restrict__ xh,
+                                                  uint8_t* __restrict__ xl, int sx, float* s_mean, float* s_rstd) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nv = d >> 2;
+  constexpr int kBatch = 8;
   for (int tk = warp; tk < R; tk += kWarps) {
     const float4* xr = reinterpret_cast<const float4*>(x + (size_t)tk * d);
-    float cnt = 0.f, mu = 0.f, m2 = 0.f;
-    if (lane < nv) {
-      const float shift = __ldcg(&xr[lane]).x;
-      float a1 = 0.f, a2 = 0.f;
-      int n = 0;
-#pragma unroll 8
-      for (int i = lane; i < nv; i += 32) {
-        const float4 a = __ldcg(&xr[i]);
-        const float d0 = a.x - shift, d1 = a.y - shift, d2 = a.z - shift, d3 = a.w - shift;
-        a1 += (d0 + d1) + (d2 + d3);
-        a2 += (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
-        n += 4;
-        const int col = i * 4 - k_lo;
-        if (col >= 0 && col < ks) {
-          const uint2 gw = *reinterpret_cast<const uint2*>(gain + i * 4);
-          const float v[4] = {a.x * __uint_as_float(gw.x << 16), a.y * __uint_as_float(gw.x & 0xffff0000u),
-                              a.z * __uint_as_float(gw.y << 16), a.w * __uint_as_float(gw.y & 0xffff0000u)};
-          uint32_t hi[4], lo[4];
+    float shift = 0.f, a1 = 0.f, a2 = 0.f;
+    int n = 0;
+    for (int i0 = lane; i0 < nv; i0 += 32 * kBatch) {
+      float4 buf[kBatch];
+      uint2 gw[kBatch];
 #pragma unroll
-          for (int e = 0; e < 4; ++e) split_bits(v[e], hi[e], lo[e]);
-          *reinterpret_cast<uint2*>(xh + tk * sx + col * 2) = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
-          *reinterpret_cast<uint2*>(xl + tk * sx + col * 2) = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
+      for (int u = 0; u < kBatch; ++u) {
+        const int i = i0 + 32 * u, col = i * 4 - k_lo;
+        buf[u] = (i < nv) ? __ldcg(&xr[i]) : make_float4(0.f, 0.f, 0.f, 0.f);
+        gw[u] = (i < nv && col >= 0 && col < ks) ? *reinterpret_cast<const uint2*>(gain + i * 4) : make_uint2(0u, 0u);
+      }
+      if (i0 == lane) shift = buf[0].x;
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) {
+        const int i = i0 + 32 * u, col = i * 4 - k_lo;
+        if (i < nv) {
+          const float4 a = buf[u];
+          const float d0 = a.x - shift, d1 = a.y - shift, d2 = a.z - shift, d3 = a.w - shift;
+          a1 += (d0 + d1) + (d2 + d3);
+          a2 += (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
+          n += 4;
+          if (col >= 0 && col < ks) {
+            const float v[4] = {a.x * __uint_as_float(gw[u].x << 16), a.y * __uint_as_float(gw[u].x & 0xffff0000u),
+                                a.z * __uint_as_float(gw[u].y << 16), a.w * __uint_as_float(gw[u].y & 0xffff0000u)};
+            uint32_t hi[4], lo[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) split_bits(v[e], hi[e], lo[e]);
+            *reinterpret_cast<uint2*>(xh + tk * sx + col * 2) = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
+            *reinterpret_cast<uint2*>(xl + tk * sx + col * 2) = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
+          }
         }
       }
+    }
+    float cnt = 0.f, mu = 0.f, m2 = 0.f;
+    if (n > 0) {
       cnt = (float)n;
       mu = shift + a1 / (float)n;
       m2 = a2 - a1 * a1 / (float)n;
@@ -142,13 +155,13 @@ __device__ __forceinline__ void rows_stats_planes(const float* x, const bf16* ga
       const bool low = (lane & off) == 0;
       const float ca = low ? cnt : cb, ma = low ? mu : mb, qa = low ? m2 : qb;
       const float c2 = low ? cb : cnt, mc = low ? mb : mu, q2 = low ? qb : m2;
-      const float n = ca + c2;
-      if (n > 0.f) {
+      const float nn = ca + c2;
+      if (nn > 0.f) {
         const float delta = mc - ma;
-        mu = ma + delta * (c2 / n);
-        m2 = qa + q2 + delta * delta * (ca * c2 / n);
+        mu = ma + delta * (c2 / nn);
+        m2 = qa + q2 + delta * delta * (ca * c2 / nn);
       }
-      cnt = n;
+      cnt = nn;
     }
     if (lane == 0) {
       s_mean[tk] = mu;
@@ -249,6 +262,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
   AttnSmem<kDH, kWarps>& sm = *reinterpret_cast<AttnSmem<kDH, kWarps>*>(fsm + L.attn);
   volatile int* flag = reinterpret_cast<volatile int*>(fsm + L.flag);
 
+  // TRACE 0
   pdl_launch_dependents();
   // This CTA's weights -- ROWS_IN rows x ks columns of the input projection, `slice` rows x 64 columns of the
   // output projection -- do not depend on the previous launch: start copying them now.
@@ -266,7 +280,9 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
     cp_async_commit();
   }
   for (int i = L.zero_begin / 16 + tid; i < L.zero_end / 16; i += kThreads) reinterpret_cast<uint4*>(fsm)[i] = make_uint4(0, 0, 0, 0);
+  // TRACE 1
   pdl_wait();
+  // TRACE 2
   if (p.all_done && *p.all_done) {      // the same answer in every CTA: nobody reaches a cluster barrier
     cp_async_wait_all();
     return;
@@ -274,9 +290,11 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
   cluster_arrive();
   __syncthreads();
   rows_stats_planes(p.x, p.gain, p.R, d, p.eps, c * ks, ks, xh_s, xl_s, L.s_x, s_mean, s_rstd);
+  // TRACE 3
   cp_async_wait_all();
   __syncthreads();
   cluster_wait();
+  // TRACE 4
 
   // ---- input projection over this CTA's part of the reduction; token t's partial goes to rank t % kC
   for (int mt = warp; mt < ROWS_IN / 16; mt += kWarps) {
@@ -295,7 +313,9 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
         }
       }
   }
+  // TRACE 5
   cluster.sync();
+  // TRACE 6
 
   // ---- this rank's tokens: add the partials in rank order, finish the layer norm, write keys / values
   for (int slot = 0; slot < NT; ++slot) {
@@ -325,6 +345,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
     __syncthreads();
   }
 
+  // TRACE 7
   // ---- attention of this rank's rows; the result goes to every rank as planes
   for (int slot = 0; slot < NT; ++slot) {
     const int token = slot * kC + c;
@@ -348,7 +369,9 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
       __syncthreads();
     }
   }
+  // TRACE 8
   cluster.sync();
+  // TRACE 9
 
   // ---- this head's share of the output projection for the features of slice c
   float* wsh = p.ws + (size_t)h * p.R * d;
@@ -366,8 +389,10 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
       }
   }
   __syncthreads();
+  // TRACE 10
   if (tid == 0) *flag = (tc::atom_add_acq_rel(&p.counters[c], 1u) == (unsigned)p.H - 1) ? 1 : 0;
   __syncthreads();
+  // TRACE 11
   if (*flag) {                           // last head to arrive at this slice: heads are added in head order
     merge_slice(p.x, p.ws, nullptr, p.H, p.R, d, c * slice, slice);
     if (tid == 0) p.counters[c] = 0;
@@ -390,18 +415,35 @@ struct FfnBlockParams {
   const int* all_done;
 };
 
+// acc[nt] += W(16 rows x 16) * X(16 x 8 tokens of tile nt): the 16-wide version of mma_rows16 (lane (g, t) takes
+// k = 4t..4t+3, eight contiguous bytes, as slots {2t, 2t+1, 2t+8, 2t+9}).
+template <int NT>
+__device__ __forceinline__ void mma_rows16_k16(float (&acc)[NT][4], const uint8_t* w, int sw, const uint8_t* xh,
+                                               const uint8_t* xl, int sx, int lane) {
+  const int g = lane >> 2, t = lane & 3;
+  const uint2 a = *reinterpret_cast<const uint2*>(w + g * sw + t * 8);
+  const uint2 b = *reinterpret_cast<const uint2*>(w + (g + 8) * sw + t * 8);
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    const uint2 h = *reinterpret_cast<const uint2*>(xh + (nt * 8 + g) * sx + t * 8);
+    const uint2 l = *reinterpret_cast<const uint2*>(xl + (nt * 8 + g) * sx + t * 8);
+    mma_bf16(acc[nt], a.x, b.x, a.y, b.y, h.x, h.y);
+    mma_bf16(acc[nt], a.x, b.x, a.y, b.y, l.x, l.y);
+  }
+}
+
 struct FfnLayout {
-  int s1, s2, s_x, s_h;
-  int w1, w2, xh, xl, hh, hl, part1, mean, rstd, flag, total;   // part2 shares the bytes of w1
+  int s1, s2, s_x, s_h, s_p;      // row strides: bytes, except s_p (floats between the tokens of the partial output)
+  int w1, w2, xh, xl, hh, hl, part1, mean, rstd, flag, total;   // the partial output shares the bytes of w1
   int zero_begin, zero_end;
 };
 __host__ __device__ inline FfnLayout ffn_layout(int d, int NT) {
   FfnLayout L;
-  const int ks = d / kC, slice = d / kC;
-  L.s1 = padded(ks * 2); L.s2 = padded(kHS * 2); L.s_x = padded(ks * 2); L.s_h = padded(kHS * 2);
+  const int ks = d / kC;
+  L.s1 = padded(ks * 2); L.s2 = kHS * 2; L.s_x = padded(ks * 2); L.s_h = kHS * 2; L.s_p = d + 4;
   int off = 0;
-  const int w1_bytes = kC * kHS * L.s1, part2_bytes = kC * slice * NT * 8 * 4;
-  L.w1 = off; off += (w1_bytes > part2_bytes ? w1_bytes : part2_bytes);
+  const int w1_bytes = kC * kHS * L.s1, out_bytes = NT * 8 * L.s_p * 4;
+  L.w1 = off; off += (w1_bytes > out_bytes ? w1_bytes : out_bytes);
   L.w2 = off; off += d * L.s2;
   L.zero_begin = off;
   L.xh = off; off += NT * 8 * L.s_x;
@@ -418,7 +460,7 @@ __host__ __device__ inline FfnLayout ffn_layout(int d, int NT) {
 }
 
 template <int NT>
-__global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 1) ffn_block_kernel(FfnBlockParams p) {
+__global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) ffn_block_kernel(FfnBlockParams p) {
   extern __shared__ __align__(16) uint8_t fsm[];
   cg::cluster_group cluster = cg::this_cluster();
   const int c = (int)cluster.block_rank(), j = blockIdx.y;
@@ -428,7 +470,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 1) ffn_bl
   const int hid_cluster = j * kC * kHS, hid0 = hid_cluster + c * kHS;
   const FfnLayout L = ffn_layout(d, NT);
   uint8_t* w1_s = fsm + L.w1;
-  float* part2_s = reinterpret_cast<float*>(fsm + L.w1);
+  float* out_s = reinterpret_cast<float*>(fsm + L.w1);
   uint8_t* w2_s = fsm + L.w2;
   uint8_t* xh_s = fsm + L.xh;
   uint8_t* xl_s = fsm + L.xl;
@@ -439,6 +481,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 1) ffn_bl
   float* s_rstd = reinterpret_cast<float*>(fsm + L.rstd);
   volatile int* flag = reinterpret_cast<volatile int*>(fsm + L.flag);
 
+  // TRACE 0
   pdl_launch_dependents();
   // Static weights of this CTA: the cluster's kC * kHS rows of the first projection restricted to this rank's ks
   // columns, and this rank's kHS columns of the second projection (all d rows).
@@ -456,7 +499,9 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 1) ffn_bl
     cp_async_commit();
   }
   for (int i = L.zero_begin / 16 + tid; i < L.zero_end / 16; i += kThreads) reinterpret_cast<uint4*>(fsm)[i] = make_uint4(0, 0, 0, 0);
+  // TRACE 1
   pdl_wait();
+  // TRACE 2
   if (p.all_done && *p.all_done) {
     cp_async_wait_all();
     return;
@@ -464,9 +509,11 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 1) ffn_bl
   cluster_arrive();
   __syncthreads();
   rows_stats_planes(p.x, p.gain, p.R, d, p.eps, c * ks, ks, xh_s, xl_s, L.s_x, s_mean, s_rstd);
+  // TRACE 3
   cp_async_wait_all();
   __syncthreads();
   cluster_wait();
+  // TRACE 4
 
   // ---- first projection of the cluster's hidden units over this rank's columns; unit f belongs to rank f / kHS
   for (int mt = warp; mt < kC * kHS / 16; mt += kWarps) {
@@ -485,7 +532,9 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 1) ffn_bl
         }
       }
   }
-  cluster.sync();            // from here on nobody reads its w1 slice any more: part2 may overwrite it
+  // TRACE 5
+  cluster.sync();
+  // TRACE 6
 
   // ---- this rank's hidden units: partials in rank order, layer norm, bias, ReLU, planes
   for (int idx = tid; idx < kHS * p.R; idx += kThreads) {
@@ -501,42 +550,51 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 1) ffn_bl
     reinterpret_cast<unsigned short*>(hl_s + token * L.s_h)[f] = (unsigned short)lo;
   }
   __syncthreads();
+  // TRACE 7
 
-  // ---- second projection restricted to these kHS hidden units, all d features; feature n belongs to rank n / slice
+  // ---- second projection restricted to these kHS hidden units, all d features, kept in this CTA's shared memory
+  // (over the bytes of the first projection's weights, which this CTA no longer reads)
   for (int mt = warp; mt < d / 16; mt += kWarps) {
     float acc[NT][4];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
-    mma_rows16<NT>(acc, w2_s + mt * 16 * L.s2, L.s2, hh_s, hl_s, L.s_h, kHS, lane);
+    mma_rows16_k16<NT>(acc, w2_s + mt * 16 * L.s2, L.s2, hh_s, hl_s, L.s_h, lane);
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const int n = mt * 16 + g + ((e & 2) ? 8 : 0), token = nt * 8 + 2 * t4 + (e & 1);
-        if (token < p.R) {
-          float* remote = cluster.map_shared_rank(part2_s, n / slice);
-          remote[(c * slice + n % slice) * (NT * 8) + token] = acc[nt][e];
-        }
+        out_s[token * L.s_p + n] = acc[nt][e];
       }
   }
+  // TRACE 8
   cluster.sync();
+  // TRACE 9
 
-  // ---- the cluster's share of this rank's feature slice, then the sum over clusters by the last one to arrive
+  // ---- rank c collects feature slice c from all eight ranks (in rank order): the cluster's share of the output
   float* wsj = p.ws + (size_t)j * p.R * d;
-  for (int idx = tid; idx < slice * p.R; idx += kThreads) {
-    const int f = idx % slice, token = idx / slice;
-    float a = 0.f;
+  const int s4 = slice >> 2;
+  for (int idx = tid; idx < s4 * p.R; idx += kThreads) {
+    const int f4 = idx % s4, token = idx / s4;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-    for (int src = 0; src < kC; ++src) a += part2_s[(src * slice + f) * (NT * 8) + token];
-    wsj[(size_t)token * d + c * slice + f] = a;
+    for (int src = 0; src < kC; ++src) {
+      const float4 v = *reinterpret_cast<const float4*>(cluster.map_shared_rank(out_s, src) + token * L.s_p + c * slice + f4 * 4);
+      a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+    }
+    *reinterpret_cast<float4*>(wsj + (size_t)token * d + c * slice + f4 * 4) = a;
   }
+  cluster_arrive();          // this CTA has read what it needs from the others
   __syncthreads();
+  // TRACE 10
   if (tid == 0) *flag = (tc::atom_add_acq_rel(&p.counters[c], 1u) == (unsigned)p.NJ - 1) ? 1 : 0;
   __syncthreads();
-  if (*flag) {
+  // TRACE 11
+  if (*flag) {               // last cluster to arrive at this slice: clusters are added in cluster order
     merge_slice(p.x, p.ws, p.b2, p.NJ, p.R, d, c * slice, slice);
     if (tid == 0) p.counters[c] = 0;
   }
+  cluster_wait();            // nobody leaves while another rank may still read its shared memory
 }
 
 // Shapes this path is built for.

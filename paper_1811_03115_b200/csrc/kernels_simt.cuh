@@ -526,14 +526,27 @@ __device__ __forceinline__ float attention_head(const AttnParams& p, int b, int 
 #pragma unroll
     for (int t = 0; t < DPL; ++t) acc[t] *= corr;
     const CT* vb = V + base + dim0;
-#pragma unroll 8
-    for (int jj = 0; jj < nk; ++jj) {
-      const float pw = __shfl_sync(0xffffffffu, pj, jj);
-      if (owns) {
-        float vv[DPL];
-        if (COHERENT) load_n_cg<DPL>(vb + (size_t)jj * p.ldkv, vv); else load_n<DPL>(vb + (size_t)jj * p.ldkv, vv);
+    // value rows are fetched 16 at a time so that their loads overlap; rows beyond the chunk's last key repeat
+    // it with weight 0 (pj is 0 in those lanes), which leaves the sum unchanged
 #pragma unroll
-        for (int t = 0; t < DPL; ++t) acc[t] = fmaf(pw, vv[t], acc[t]);
+    for (int j0 = 0; j0 < 32; j0 += 16) {
+      if (j0 < nk) {
+        float vv[16][DPL];
+        if (owns) {
+#pragma unroll
+          for (int jj = 0; jj < 16; ++jj) {
+            const int jc = min(j0 + jj, nk - 1);
+            if (COHERENT) load_n_cg<DPL>(vb + (size_t)jc * p.ldkv, vv[jj]); else load_n<DPL>(vb + (size_t)jc * p.ldkv, vv[jj]);
+          }
+        }
+#pragma unroll
+        for (int jj = 0; jj < 16; ++jj) {
+          const float pw = __shfl_sync(0xffffffffu, pj, j0 + jj);
+          if (owns) {
+#pragma unroll
+            for (int t = 0; t < DPL; ++t) acc[t] = fmaf(pw, vv[jj][t], acc[t]);
+          }
+        }
       }
     }
     m_run = m_new;
