@@ -522,7 +522,7 @@ static int run_layers_fused(bpd_session* s, const PassArgs& a) {
   const int* done = s->st.all_done;
   const bool pdl = s->use_pdl != 0;
   const int nt = (R + 7) / 8;
-  const size_t smem_self = fused::attn_layout<true>(d, nt).total, smem_cross = fused::attn_layout<false>(d, nt).total;
+  const size_t smem_self = fused::attn_layout<true>(d, nt, s->B * s->ppr).total, smem_cross = fused::attn_layout<false>(d, nt, 0).total;
   const size_t smem_ffn = fused::ffn_layout(d, nt).total;
   // the opt-in shared-memory limit of each kernel grows with the widest model seen so far
   static size_t attr_max[3][3] = {{0, 0, 0}, {0, 0, 0}, {0, 0, 0}};

@@ -174,20 +174,28 @@ __device__ __forceinline__ void rows_stats_planes(const float* __restrict__ x, c
 // the CTA that completed the slice: x[t][f] += bias[f] + ws[0][t][f] + ws[1][t][f] + ... in that order.
 __device__ __forceinline__ void merge_slice(float* x, const float* ws, const bf16* bias, int np, int R, int d, int col0, int width) {
   const int w4 = width >> 2;
+  constexpr int kBatch = 16;
   for (int idx = threadIdx.x; idx < R * w4; idx += kThreads) {
     const int t = idx / w4, col = col0 + (idx % w4) * 4;
     float4 acc = __ldcg(reinterpret_cast<const float4*>(x + (size_t)t * d + col));
-    if (bias) {
-      const uint2 bw = *reinterpret_cast<const uint2*>(bias + col);
-      acc.x += __uint_as_float(bw.x << 16); acc.y += __uint_as_float(bw.x & 0xffff0000u);
-      acc.z += __uint_as_float(bw.y << 16); acc.w += __uint_as_float(bw.y & 0xffff0000u);
-    }
+    uint2 bw = make_uint2(0u, 0u);
+    if (bias) bw = *reinterpret_cast<const uint2*>(bias + col);
     const float4* wp = reinterpret_cast<const float4*>(ws + (size_t)t * d + col);
     const size_t step = (size_t)R * d / 4;
-#pragma unroll 8
-    for (int p = 0; p < np; ++p) {
-      const float4 v = __ldcg(wp + p * step);
-      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    float4 v[kBatch];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) v[u] = (u < np) ? __ldcg(wp + u * step) : make_float4(0.f, 0.f, 0.f, 0.f);
+    acc.x += __uint_as_float(bw.x << 16); acc.y += __uint_as_float(bw.x & 0xffff0000u);
+    acc.z += __uint_as_float(bw.y << 16); acc.w += __uint_as_float(bw.y & 0xffff0000u);
+    for (int p0 = 0; p0 < np; p0 += kBatch) {
+      if (p0 > 0) {
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) v[u] = (p0 + u < np) ? __ldcg(wp + (p0 + u) * step) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) {
+        if (p0 + u < np) { acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w; }
+      }
     }
     *reinterpret_cast<float4*>(x + (size_t)t * d + col) = acc;
   }
@@ -212,11 +220,11 @@ struct AttnBlockParams {
 
 struct AttnLayout {
   int s_in, s_out, s_x;           // row strides (bytes)
-  int w_in, w_out, xh, xl, oh, ol, part, q, mean, rstd, attn, flag, total;   // offsets (bytes)
+  int w_in, w_out, xh, xl, oh, ol, part, q, mean, rstd, attn, flag, len, pt, total;   // offsets (bytes)
   int zero_begin, zero_end;       // planes that must start at zero
 };
 template <bool SELF>
-__host__ __device__ inline AttnLayout attn_layout(int d, int NT) {
+__host__ __device__ inline AttnLayout attn_layout(int d, int NT, int pt_ints) {
   AttnLayout L;
   const int ks = d / kC, rows_in = SELF ? 3 * kDH : kDH;
   L.s_in = padded(ks * 2); L.s_out = padded(kDH * 2); L.s_x = padded(ks * 2);
@@ -235,6 +243,8 @@ __host__ __device__ inline AttnLayout attn_layout(int d, int NT) {
   L.rstd = off; off += kMaxRows * 4;
   L.attn = off; off += (int)((sizeof(AttnSmem<kDH, kWarps>) + 15) / 16 * 16);
   L.flag = off; off += 16;
+  L.len = off; off += kMaxRows * 4;
+  L.pt = off; off += (pt_ints * 4 + 15) / 16 * 16;
   L.total = off;
   return L;
 }
@@ -248,7 +258,9 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
   const int g = lane >> 2, t4 = lane & 3;
   const int d = p.d, ks = d / kC, slice = d / kC;
   constexpr int ROWS_IN = SELF ? 3 * kDH : kDH;
-  const AttnLayout L = attn_layout<SELF>(d, NT);
+  const int nb = p.R / p.rows_per_b;                                   // sequences in this pass
+  const int pt_ints = SELF ? nb * p.attn.st.pages_per_row : 0;
+  const AttnLayout L = attn_layout<SELF>(d, NT, pt_ints);
   uint8_t* w_in_s = fsm + L.w_in;
   uint8_t* w_out_s = fsm + L.w_out;
   uint8_t* xh_s = fsm + L.xh;
@@ -261,11 +273,14 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
   float* s_rstd = reinterpret_cast<float*>(fsm + L.rstd);
   AttnSmem<kDH, kWarps>& sm = *reinterpret_cast<AttnSmem<kDH, kWarps>*>(fsm + L.attn);
   volatile int* flag = reinterpret_cast<volatile int*>(fsm + L.flag);
+  int* s_len = reinterpret_cast<int*>(fsm + L.len);    // per sequence: tokens in the cache (self) or source length (cross)
+  int* s_pt = reinterpret_cast<int*>(fsm + L.pt);      // self: the sequences' page-table rows
 
   // TRACE 0
   pdl_launch_dependents();
-  // This CTA's weights -- ROWS_IN rows x ks columns of the input projection, `slice` rows x 64 columns of the
-  // output projection -- do not depend on the previous launch: start copying them now.
+  cluster_arrive();
+  // Everything that does not depend on the previous launch starts now.  This CTA's weights: ROWS_IN rows x ks
+  // columns of the input projection, `slice` rows x 64 columns of the output projection.
   {
     const int cpr = ks * 2 / 16;
     for (int idx = tid; idx < ROWS_IN * cpr; idx += kThreads) {
@@ -280,20 +295,30 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
     cp_async_commit();
   }
   for (int i = L.zero_begin / 16 + tid; i < L.zero_end / 16; i += kThreads) reinterpret_cast<uint4*>(fsm)[i] = make_uint4(0, 0, 0, 0);
+  // the folded layer-norm vectors of the feature this thread finishes, page tables, source lengths: all static
+  float fs = 0.f, fc = 0.f;
+  if (tid < ROWS_IN) {
+    const int n = (tid / kDH) * d + h * kDH + (tid % kDH);
+    fs = p.fold_s[n];
+    fc = p.fold_c[n];
+  }
+  if (SELF) {
+    for (int i = tid; i < pt_ints; i += kThreads) s_pt[i] = p.attn.st.page_table[i];
+  } else if (tid < nb) {
+    s_len[tid] = p.attn.limit_b[tid];
+  }
+  __syncthreads();
   // TRACE 1
   pdl_wait();
   // TRACE 2
-  if (p.all_done && *p.all_done) {      // the same answer in every CTA: nobody reaches a cluster barrier
-    cp_async_wait_all();
-    return;
-  }
-  cluster_arrive();
-  __syncthreads();
+  const int ended = p.all_done ? *p.all_done : 0;      // the same answer in every CTA
+  if (SELF && tid < nb) s_len[tid] = p.attn.st.len[tid];
   rows_stats_planes(p.x, p.gain, p.R, d, p.eps, c * ks, ks, xh_s, xl_s, L.s_x, s_mean, s_rstd);
   // TRACE 3
   cp_async_wait_all();
   __syncthreads();
-  cluster_wait();
+  cluster_wait();                                      // every CTA of the cluster is running: its shared memory may be written
+  if (ended) return;
   // TRACE 4
 
   // ---- input projection over this CTA's part of the reduction; token t's partial goes to rank t % kC
@@ -325,14 +350,13 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
 #pragma unroll
       for (int src = 0; src < kC; ++src) a += part_s[(src * NT + slot) * ROWS_IN + tid];
       const int sect = tid / kDH, f = tid % kDH;
-      const int n = sect * d + h * kDH + f;
-      const float y = s_rstd[token] * (a - s_mean[token] * p.fold_s[n]) + p.fold_c[n];
+      const float y = s_rstd[token] * (a - s_mean[token] * fs) + fc;
       if (sect == 0) {
         q_s[slot * kDH + f] = y * p.attn.scale;
       } else {
         const int b = token / p.rows_per_b, i = token % p.rows_per_b;
-        const int pos = p.attn.st.len[b] + i;
-        const int page = p.attn.st.page_table[b * p.attn.st.pages_per_row + pos / kPage];
+        const int pos = s_len[b] + i;
+        const int page = s_pt[b * p.attn.st.pages_per_row + pos / kPage];
         const size_t at = ((size_t)page * kPage + (pos % kPage)) * d + h * kDH + f;
         (sect == 1 ? p.kcache : p.vcache)[at] = __float2bfloat16_rn(y);
       }
@@ -347,16 +371,18 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
 
   // TRACE 7
   // ---- attention of this rank's rows; the result goes to every rank as planes
+  AttnParams ap = p.attn;
+  if (SELF) ap.st.page_table = s_pt;
   for (int slot = 0; slot < NT; ++slot) {
     const int token = slot * kC + c;
     if (token < p.R) {                   // uniform over the CTA
       if (tid < kDH) sm.q[tid] = q_s[slot * kDH + tid];
       __syncthreads();
       const int b = token / p.rows_per_b, i = token % p.rows_per_b;
-      const int limit = p.attn.causal ? (p.attn.st.len[b] + i + 1) : p.attn.limit_b[b];
+      const int limit = SELF ? (s_len[b] + i + 1) : s_len[b];
       float ov;
-      if (SELF) ov = attention_head<bf16, kDH, kWarps, true>(p.attn, b, h, limit, sm);
-      else ov = attention_head<float, kDH, kWarps, false>(p.attn, b, h, limit, sm);
+      if (SELF) ov = attention_head<bf16, kDH, kWarps, true>(ap, b, h, limit, sm);
+      else ov = attention_head<float, kDH, kWarps, false>(ap, b, h, limit, sm);
       if (tid < kDH) {
         uint32_t hi, lo;
         split_bits(ov, hi, lo);
@@ -483,6 +509,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) ffn_bl
 
   // TRACE 0
   pdl_launch_dependents();
+  cluster_arrive();
   // Static weights of this CTA: the cluster's kC * kHS rows of the first projection restricted to this rank's ks
   // columns, and this rank's kHS columns of the second projection (all d rows).
   {
@@ -499,20 +526,19 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) ffn_bl
     cp_async_commit();
   }
   for (int i = L.zero_begin / 16 + tid; i < L.zero_end / 16; i += kThreads) reinterpret_cast<uint4*>(fsm)[i] = make_uint4(0, 0, 0, 0);
+  // folded layer-norm vectors of the hidden unit this thread finishes (kHS * R <= 256 items, one per thread)
+  const float fs = p.fold_s[hid0 + tid % kHS], fc = p.fold_c[hid0 + tid % kHS];
+  __syncthreads();
   // TRACE 1
   pdl_wait();
   // TRACE 2
-  if (p.all_done && *p.all_done) {
-    cp_async_wait_all();
-    return;
-  }
-  cluster_arrive();
-  __syncthreads();
+  const int ended = p.all_done ? *p.all_done : 0;      // the same answer in every CTA
   rows_stats_planes(p.x, p.gain, p.R, d, p.eps, c * ks, ks, xh_s, xl_s, L.s_x, s_mean, s_rstd);
   // TRACE 3
   cp_async_wait_all();
   __syncthreads();
   cluster_wait();
+  if (ended) return;
   // TRACE 4
 
   // ---- first projection of the cluster's hidden units over this rank's columns; unit f belongs to rank f / kHS
@@ -542,8 +568,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) ffn_bl
     float a = 0.f;
 #pragma unroll
     for (int src = 0; src < kC; ++src) a += part1_s[(src * kHS + f) * (NT * 8) + token];
-    const int n = hid0 + f;
-    const float y = fmaxf(s_rstd[token] * (a - s_mean[token] * p.fold_s[n]) + p.fold_c[n], 0.f);
+    const float y = fmaxf(s_rstd[token] * (a - s_mean[token] * fs) + fc, 0.f);     // idx == tid: f == tid % kHS
     uint32_t hi, lo;
     split_bits(y, hi, lo);
     reinterpret_cast<unsigned short*>(hh_s + token * L.s_h)[f] = (unsigned short)hi;
@@ -576,12 +601,13 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) ffn_bl
   const int s4 = slice >> 2;
   for (int idx = tid; idx < s4 * p.R; idx += kThreads) {
     const int f4 = idx % s4, token = idx / s4;
+    float4 v[kC];
+#pragma unroll
+    for (int src = 0; src < kC; ++src)
+      v[src] = *reinterpret_cast<const float4*>(cluster.map_shared_rank(out_s, src) + token * L.s_p + c * slice + f4 * 4);
     float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-    for (int src = 0; src < kC; ++src) {
-      const float4 v = *reinterpret_cast<const float4*>(cluster.map_shared_rank(out_s, src) + token * L.s_p + c * slice + f4 * 4);
-      a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
-    }
+    for (int src = 0; src < kC; ++src) { a.x += v[src].x; a.y += v[src].y; a.z += v[src].z; a.w += v[src].w; }
     *reinterpret_cast<float4*>(wsj + (size_t)token * d + c * slice + f4 * 4) = a;
   }
   cluster_arrive();          // this CTA has read what it needs from the others
