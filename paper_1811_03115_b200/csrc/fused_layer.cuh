@@ -95,77 +95,87 @@ __device__ __forceinline__ void mma_rows16(float (&acc)[NT][4], const uint8_t* w
   }
 }
 
-// Rows of the residual stream: per-token mean and 1/std (all columns) and the planes of x * gain for columns
-// [k_lo, k_lo + ks).  One warp per token (tokens w, w+8), every lane a fixed share of the row, one pass: each lane
-// sums its share about its own first element, then the 32 partial (count, mean, M2) triples are merged pairwise
-// in a fixed order.  Rows come from L2 (another launch wrote them), eight loads per lane in flight.
-__device__ __forceinline__ void rows_stats_planes(const float* __restrict__ x, const bf16* __restrict__ gain, int R, int d,
-                                                  float eps, int k_lo, int ks, uint8_t* __restrict__ xh,
-                                                  uint8_t* __restrict__ xl, int sx, float* s_mean, float* s_rstd) {
+// Per-token mean and 1/std of the rows of the residual stream.  One warp per token (tokens w, w+8), every lane
+// the same fixed share of the row (d is a multiple of 128), one pass: each lane sums its share about its own
+// first element, then the 32 partial (mean, M2) pairs -- all over equally many elements -- are merged pairwise in
+// a fixed order: mean = (mean_a + mean_b) / 2, M2 = M2_a + M2_b + (mean_b - mean_a)^2 * n / 2 with n elements on
+// each side.  Rows come from L2 (another launch wrote them), eight loads per lane in flight.
+__device__ __forceinline__ void rows_stats(const float* __restrict__ x, int R, int d, float eps, float* s_mean, float* s_rstd) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nv = d >> 2;
   constexpr int kBatch = 8;
+  const float per_lane = (float)(d >> 5), inv_per_lane = 1.0f / per_lane;
   for (int tk = warp; tk < R; tk += kWarps) {
     const float4* xr = reinterpret_cast<const float4*>(x + (size_t)tk * d);
     float shift = 0.f, a1 = 0.f, a2 = 0.f;
-    int n = 0;
     for (int i0 = lane; i0 < nv; i0 += 32 * kBatch) {
       float4 buf[kBatch];
-      uint2 gw[kBatch];
 #pragma unroll
-      for (int u = 0; u < kBatch; ++u) {
-        const int i = i0 + 32 * u, col = i * 4 - k_lo;
-        buf[u] = (i < nv) ? __ldcg(&xr[i]) : make_float4(0.f, 0.f, 0.f, 0.f);
-        gw[u] = (i < nv && col >= 0 && col < ks) ? *reinterpret_cast<const uint2*>(gain + i * 4) : make_uint2(0u, 0u);
-      }
+      for (int u = 0; u < kBatch; ++u) buf[u] = (i0 + 32 * u < nv) ? __ldcg(&xr[i0 + 32 * u]) : make_float4(0.f, 0.f, 0.f, 0.f);
       if (i0 == lane) shift = buf[0].x;
 #pragma unroll
       for (int u = 0; u < kBatch; ++u) {
-        const int i = i0 + 32 * u, col = i * 4 - k_lo;
-        if (i < nv) {
+        if (i0 + 32 * u < nv) {
           const float4 a = buf[u];
           const float d0 = a.x - shift, d1 = a.y - shift, d2 = a.z - shift, d3 = a.w - shift;
           a1 += (d0 + d1) + (d2 + d3);
           a2 += (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
-          n += 4;
-          if (col >= 0 && col < ks) {
-            const float v[4] = {a.x * __uint_as_float(gw[u].x << 16), a.y * __uint_as_float(gw[u].x & 0xffff0000u),
-                                a.z * __uint_as_float(gw[u].y << 16), a.w * __uint_as_float(gw[u].y & 0xffff0000u)};
-            uint32_t hi[4], lo[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) split_bits(v[e], hi[e], lo[e]);
-            *reinterpret_cast<uint2*>(xh + tk * sx + col * 2) = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
-            *reinterpret_cast<uint2*>(xl + tk * sx + col * 2) = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
-          }
         }
       }
     }
-    float cnt = 0.f, mu = 0.f, m2 = 0.f;
-    if (n > 0) {
-      cnt = (float)n;
-      mu = shift + a1 / (float)n;
-      m2 = a2 - a1 * a1 / (float)n;
-    }
+    float mu = shift + a1 * inv_per_lane;
+    float m2 = a2 - a1 * a1 * inv_per_lane;
+    float half_n = 0.5f * per_lane;                  // half the elements behind each side of the next merge
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
-      const float cb = __shfl_xor_sync(0xffffffffu, cnt, off);
       const float mb = __shfl_xor_sync(0xffffffffu, mu, off);
       const float qb = __shfl_xor_sync(0xffffffffu, m2, off);
-      // the lower lane of a pair is "a" on both sides, so both lanes evaluate the same expression
-      const bool low = (lane & off) == 0;
-      const float ca = low ? cnt : cb, ma = low ? mu : mb, qa = low ? m2 : qb;
-      const float c2 = low ? cb : cnt, mc = low ? mb : mu, q2 = low ? qb : m2;
-      const float nn = ca + c2;
-      if (nn > 0.f) {
-        const float delta = mc - ma;
-        mu = ma + delta * (c2 / nn);
-        m2 = qa + q2 + delta * delta * (ca * c2 / nn);
-      }
-      cnt = nn;
+      const float delta = mb - mu;
+      m2 = (m2 + qb) + delta * delta * half_n;       // symmetric in the two lanes: both hold the same result
+      mu = 0.5f * (mu + mb);
+      half_n *= 2.f;
     }
     if (lane == 0) {
       s_mean[tk] = mu;
       s_rstd[tk] = rsqrtf(fmaxf(m2, 0.f) / (float)d + eps);
+    }
+  }
+}
+
+// Planes (hi, lo) of x * gain for columns [k_lo, k_lo + ks) of all R rows: item idx = (row, group of four columns),
+// thread t takes items t and t + kThreads (R * ks / 4 <= 512).  The gain words are static and fetched ahead
+// (planes_gain, before the wait on the previous launch), the rows are fetched by planes_fetch right after it.
+__device__ __forceinline__ void planes_gain(const bf16* __restrict__ gain, int R, int k_lo, int ks, uint2 (&g)[2]) {
+  const int k4 = ks >> 2;
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const int idx = threadIdx.x + j * kThreads;
+    g[j] = (idx < R * k4) ? *reinterpret_cast<const uint2*>(gain + k_lo + (idx % k4) * 4) : make_uint2(0u, 0u);
+  }
+}
+__device__ __forceinline__ void planes_fetch(const float* __restrict__ x, int R, int d, int k_lo, int ks, float4 (&v)[2]) {
+  const int k4 = ks >> 2;
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const int idx = threadIdx.x + j * kThreads;
+    v[j] = (idx < R * k4) ? __ldcg(reinterpret_cast<const float4*>(x + (size_t)(idx / k4) * d + k_lo + (idx % k4) * 4))
+                          : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+}
+__device__ __forceinline__ void planes_store(const float4 (&v)[2], const uint2 (&g)[2], int R, int ks, uint8_t* xh, uint8_t* xl, int sx) {
+  const int k4 = ks >> 2;
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const int idx = threadIdx.x + j * kThreads;
+    if (idx < R * k4) {
+      const float w[4] = {v[j].x * __uint_as_float(g[j].x << 16), v[j].y * __uint_as_float(g[j].x & 0xffff0000u),
+                          v[j].z * __uint_as_float(g[j].y << 16), v[j].w * __uint_as_float(g[j].y & 0xffff0000u)};
+      uint32_t hi[4], lo[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) split_bits(w[e], hi[e], lo[e]);
+      const int at = (idx / k4) * sx + (idx % k4) * 8;
+      *reinterpret_cast<uint2*>(xh + at) = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
+      *reinterpret_cast<uint2*>(xl + at) = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
     }
   }
 }
@@ -307,13 +317,18 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
   } else if (tid < nb) {
     s_len[tid] = p.attn.limit_b[tid];
   }
+  uint2 gwords[2];
+  planes_gain(p.gain, p.R, c * ks, ks, gwords);
   __syncthreads();
   // TRACE 1
   pdl_wait();
   // TRACE 2
   const int ended = p.all_done ? *p.all_done : 0;      // the same answer in every CTA
   if (SELF && tid < nb) s_len[tid] = p.attn.st.len[tid];
-  rows_stats_planes(p.x, p.gain, p.R, d, p.eps, c * ks, ks, xh_s, xl_s, L.s_x, s_mean, s_rstd);
+  float4 xrow[2];
+  planes_fetch(p.x, p.R, d, c * ks, ks, xrow);
+  rows_stats(p.x, p.R, d, p.eps, s_mean, s_rstd);
+  planes_store(xrow, gwords, p.R, ks, xh_s, xl_s, L.s_x);
   // TRACE 3
   cp_async_wait_all();
   __syncthreads();
@@ -528,12 +543,17 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) ffn_bl
   for (int i = L.zero_begin / 16 + tid; i < L.zero_end / 16; i += kThreads) reinterpret_cast<uint4*>(fsm)[i] = make_uint4(0, 0, 0, 0);
   // folded layer-norm vectors of the hidden unit this thread finishes (kHS * R <= 256 items, one per thread)
   const float fs = p.fold_s[hid0 + tid % kHS], fc = p.fold_c[hid0 + tid % kHS];
+  uint2 gwords[2];
+  planes_gain(p.gain, p.R, c * ks, ks, gwords);
   __syncthreads();
   // TRACE 1
   pdl_wait();
   // TRACE 2
   const int ended = p.all_done ? *p.all_done : 0;      // the same answer in every CTA
-  rows_stats_planes(p.x, p.gain, p.R, d, p.eps, c * ks, ks, xh_s, xl_s, L.s_x, s_mean, s_rstd);
+  float4 xrow[2];
+  planes_fetch(p.x, p.R, d, c * ks, ks, xrow);
+  rows_stats(p.x, p.R, d, p.eps, s_mean, s_rstd);
+  planes_store(xrow, gwords, p.R, ks, xh_s, xl_s, L.s_x);
   // TRACE 3
   cp_async_wait_all();
   __syncthreads();
@@ -625,7 +645,8 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) ffn_bl
 
 // Shapes this path is built for.
 __host__ inline bool supported(int d, int H, int ff, int rows) {
-  return H > 0 && d == H * kDH && d % (kC * 32) == 0 && ff % (kC * kHS) == 0 && rows >= 1 && rows <= kMaxRows;
+  return H > 0 && d == H * kDH && d % (kC * 32) == 0 && d % 128 == 0 && ff % (kC * kHS) == 0 && rows >= 1 && rows <= kMaxRows &&
+         rows * (d / kC) <= 8 * kThreads;   // planes: at most two groups of four columns per thread
 }
 
 }  // namespace fused

@@ -526,21 +526,22 @@ __device__ __forceinline__ float attention_head(const AttnParams& p, int b, int 
 #pragma unroll
     for (int t = 0; t < DPL; ++t) acc[t] *= corr;
     const CT* vb = V + base + dim0;
-    // value rows are fetched 16 at a time so that their loads overlap; rows beyond the chunk's last key repeat
+    // value rows are fetched VB at a time so that their loads overlap; rows beyond the chunk's last key repeat
     // it with weight 0 (pj is 0 in those lanes), which leaves the sum unchanged
+    constexpr int VB0 = ((sizeof(CT) == 2) ? 64 : 32) / DPL, VB = VB0 > 32 ? 32 : (VB0 < 8 ? 8 : VB0);
 #pragma unroll
-    for (int j0 = 0; j0 < 32; j0 += 16) {
+    for (int j0 = 0; j0 < 32; j0 += VB) {
       if (j0 < nk) {
-        float vv[16][DPL];
+        float vv[VB][DPL];
         if (owns) {
 #pragma unroll
-          for (int jj = 0; jj < 16; ++jj) {
+          for (int jj = 0; jj < VB; ++jj) {
             const int jc = min(j0 + jj, nk - 1);
             if (COHERENT) load_n_cg<DPL>(vb + (size_t)jc * p.ldkv, vv[jj]); else load_n<DPL>(vb + (size_t)jc * p.ldkv, vv[jj]);
           }
         }
 #pragma unroll
-        for (int jj = 0; jj < 16; ++jj) {
+        for (int jj = 0; jj < VB; ++jj) {
           const float pw = __shfl_sync(0xffffffffu, pj, j0 + jj);
           if (owns) {
 #pragma unroll
