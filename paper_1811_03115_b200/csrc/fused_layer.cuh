@@ -9,12 +9,13 @@
 //   attn_block_kernel<SELF>   layer norm -> Q,K,V of one head -> cache write -> attention -> that head's share of
 //                             the output projection -> sum over heads + residual
 //   attn_block_kernel<CROSS>  layer norm -> Q of one head -> attention over the encoder keys -> same tail
-//   ffn_block_kernel          layer norm -> 16 hidden units (ReLU) -> their share of the second projection ->
-//                             sum over all hidden slices + bias + residual
+//   ffn_block_kernel          layer norm -> 16 hidden units (ReLU) -> shared with the cluster -> the cluster's 128
+//                             hidden units times this CTA's slice of the second projection -> sum over clusters
+//                             + bias + residual
 //
-// One thread-block cluster of kC CTAs works on a head (or on kC hidden slices); inside it the reduction length
-// is split over the CTAs and partial sums travel through distributed shared memory, always added in rank
-// order.  Across clusters the partial outputs go through a small workspace and the last cluster to arrive adds
+// One thread-block cluster of kC CTAs works on a head (or on kC * 16 hidden units).  In the attention blocks the
+// reduction length of the input projection is split over the CTAs and partial sums travel through distributed
+// shared memory, always added in rank order; in the feed-forward block the CTAs exchange their hidden units.  Across clusters the partial outputs go through a small workspace and the last cluster to arrive adds
 // them in cluster order, so every element is the same sum in the same order however many rows a pass carries.
 // Weights are static: every CTA starts copying its slice into shared memory before it waits for the previous
 // launch (programmatic dependent launch), which takes HBM latency off the chain.
@@ -39,9 +40,10 @@ constexpr int kDH = 64;          // head width this path is built for
 constexpr int kHS = 16;          // hidden units per CTA in the feed-forward block
 constexpr int kMaxRows = 16;
 
-// Row stride (bytes) of a shared-memory matrix whose rows hold `row_bytes` (a multiple of 64): congruent to 64
-// mod 128, so that the 16-byte fragment loads of eight lanes (two rows x four quarters) cover all 32 banks once.
-__host__ __device__ inline int padded(int row_bytes) { return (row_bytes % 128 == 0) ? row_bytes + 64 : row_bytes; }
+// Byte offset of (row, byte) in a shared-memory matrix with rb bytes per row (a multiple of 64).  When rb is a
+// multiple of 128 the two 64-byte halves of every 128 bytes trade places in odd rows, so that the 16-byte
+// fragment loads of eight lanes (two rows x four quarters) cover all 32 banks once; 64-byte rows do so as they are.
+__host__ __device__ inline int sw(int row, int byte, int rb) { return row * rb + ((rb & 127) ? byte : (byte ^ ((row & 1) << 6))); }
 
 __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(tc::smem_u32(smem)), "l"(gmem) : "memory");
@@ -68,25 +70,28 @@ __device__ __forceinline__ void split_bits(float v, uint32_t& hi, uint32_t& lo) 
   lo = __bfloat16_as_ushort(l);
 }
 
-// acc[nt] += W(16 rows x K) * X(K x 8 tokens of tile nt), X = hi + lo planes.
-// w: first of 16 weight rows in shared memory (row-major, sw bytes apart); xh / xl: planes, one row per token (sx
-// bytes apart).  K is a multiple of 32.  The contraction index is permuted inside each group of 32 so that a
-// lane's fragments are 16 contiguous bytes: lane (g, t) takes k = 8t..8t+7 of rows g and g+8 and of token g, and
-// uses them as slots {2t, 2t+1, 2t+8, 2t+9} of two successive MMAs -- the same permutation on both operands.
+// acc[nt] += W(16 rows x K) * X(K x 8 tokens of tile nt), X = hi + lo planes, over columns [kb0/2, kb0/2 + K).
+// w: first of 16 weight rows (an even row of a matrix laid out by sw() with sw_ bytes per row); xh / xl: planes,
+// one row per token (sx bytes per row, same lay-out).  K is a multiple of 32.  The contraction index is permuted
+// inside each group of 32 so that a lane's fragments are 16 contiguous bytes: lane (g, t) takes k = 8t..8t+7 of
+// rows g and g+8 and of token g, and uses them as slots {2t, 2t+1, 2t+8, 2t+9} of two successive MMAs -- the same
+// permutation on both operands.
 // acc[nt][0..3] = (row g, token 2t), (row g, token 2t+1), (row g+8, token 2t), (row g+8, token 2t+1).
 template <int NT>
-__device__ __forceinline__ void mma_rows16(float (&acc)[NT][4], const uint8_t* w, int sw, const uint8_t* xh, const uint8_t* xl,
-                                           int sx, int K, int lane) {
+__device__ __forceinline__ void mma_rows16(float (&acc)[NT][4], const uint8_t* w, int sw_, const uint8_t* xh, const uint8_t* xl,
+                                           int sx, int K, int lane, int kb0 = 0) {
   const int g = lane >> 2, t = lane & 3;
-  const uint8_t* w0 = w + g * sw + t * 16;
-  const uint8_t* w1 = w0 + 8 * sw;
+  const int flip_w = (sw_ & 127) ? 0 : ((g & 1) << 6), flip_x = (sx & 127) ? 0 : ((g & 1) << 6);
+  const uint8_t* w0 = w + g * sw_;
+  const uint8_t* w1 = w0 + 8 * sw_;
   for (int k0 = 0; k0 < K; k0 += 32) {
-    const uint4 a = *reinterpret_cast<const uint4*>(w0 + k0 * 2);
-    const uint4 b = *reinterpret_cast<const uint4*>(w1 + k0 * 2);
+    const int kb = kb0 + k0 * 2 + t * 16;
+    const uint4 a = *reinterpret_cast<const uint4*>(w0 + (kb ^ flip_w));
+    const uint4 b = *reinterpret_cast<const uint4*>(w1 + (kb ^ flip_w));
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-      const uint4 h = *reinterpret_cast<const uint4*>(xh + (nt * 8 + g) * sx + t * 16 + k0 * 2);
-      const uint4 l = *reinterpret_cast<const uint4*>(xl + (nt * 8 + g) * sx + t * 16 + k0 * 2);
+      const uint4 h = *reinterpret_cast<const uint4*>(xh + (nt * 8 + g) * sx + (kb ^ flip_x));
+      const uint4 l = *reinterpret_cast<const uint4*>(xl + (nt * 8 + g) * sx + (kb ^ flip_x));
       mma_bf16(acc[nt], a.x, b.x, a.y, b.y, h.x, h.y);
       mma_bf16(acc[nt], a.x, b.x, a.y, b.y, l.x, l.y);
       mma_bf16(acc[nt], a.z, b.z, a.w, b.w, h.z, h.w);
@@ -173,7 +178,7 @@ __device__ __forceinline__ void planes_store(const float4 (&v)[2], const uint2 (
       uint32_t hi[4], lo[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) split_bits(w[e], hi[e], lo[e]);
-      const int at = (idx / k4) * sx + (idx % k4) * 8;
+      const int at = sw(idx / k4, (idx % k4) * 8, sx);
       *reinterpret_cast<uint2*>(xh + at) = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
       *reinterpret_cast<uint2*>(xl + at) = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
     }
@@ -237,7 +242,7 @@ template <bool SELF>
 __host__ __device__ inline AttnLayout attn_layout(int d, int NT, int pt_ints) {
   AttnLayout L;
   const int ks = d / kC, rows_in = SELF ? 3 * kDH : kDH;
-  L.s_in = padded(ks * 2); L.s_out = padded(kDH * 2); L.s_x = padded(ks * 2);
+  L.s_in = ks * 2; L.s_out = kDH * 2; L.s_x = ks * 2;
   int off = 0;
   L.w_in = off; off += rows_in * L.s_in;
   L.w_out = off; off += (d / kC) * L.s_out;
@@ -288,7 +293,6 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
 
   // TRACE 0
   pdl_launch_dependents();
-  cluster_arrive();
   // Everything that does not depend on the previous launch starts now.  This CTA's weights: ROWS_IN rows x ks
   // columns of the input projection, `slice` rows x 64 columns of the output projection.
   {
@@ -296,11 +300,11 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
     for (int idx = tid; idx < ROWS_IN * cpr; idx += kThreads) {
       const int row = idx / cpr, c16 = idx % cpr;
       const int grow = (row / kDH) * d + h * kDH + (row % kDH);
-      cp_async16(w_in_s + row * L.s_in + c16 * 16, p.w_in + (size_t)grow * d + c * ks + c16 * 8);
+      cp_async16(w_in_s + sw(row, c16 * 16, L.s_in), p.w_in + (size_t)grow * d + c * ks + c16 * 8);
     }
     for (int idx = tid; idx < slice * 8; idx += kThreads) {
       const int row = idx >> 3, c16 = idx & 7;
-      cp_async16(w_out_s + row * L.s_out + c16 * 16, p.w_out + (size_t)(c * slice + row) * d + h * kDH + c16 * 8);
+      cp_async16(w_out_s + sw(row, c16 * 16, L.s_out), p.w_out + (size_t)(c * slice + row) * d + h * kDH + c16 * 8);
     }
     cp_async_commit();
   }
@@ -320,14 +324,18 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
   uint2 gwords[2];
   planes_gain(p.gain, p.R, c * ks, ks, gwords);
   __syncthreads();
+  cluster_arrive();            // this CTA's shared memory is set up; matched by cluster_wait() below
   // TRACE 1
   pdl_wait();
   // TRACE 2
   const int ended = p.all_done ? *p.all_done : 0;      // the same answer in every CTA
-  if (SELF && tid < nb) s_len[tid] = p.attn.st.len[tid];
+  // a warp issues in order: every load goes out before the first value is used
+  int len_v = 0;
+  if (SELF && tid < nb) len_v = p.attn.st.len[tid];
   float4 xrow[2];
   planes_fetch(p.x, p.R, d, c * ks, ks, xrow);
   rows_stats(p.x, p.R, d, p.eps, s_mean, s_rstd);
+  if (SELF && tid < nb) s_len[tid] = len_v;
   planes_store(xrow, gwords, p.R, ks, xh_s, xl_s, L.s_x);
   // TRACE 3
   cp_async_wait_all();
@@ -403,8 +411,8 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
         split_bits(ov, hi, lo);
 #pragma unroll
         for (int dst = 0; dst < kC; ++dst) {
-          reinterpret_cast<unsigned short*>(cluster.map_shared_rank(oh_s, dst) + token * L.s_out)[tid] = (unsigned short)hi;
-          reinterpret_cast<unsigned short*>(cluster.map_shared_rank(ol_s, dst) + token * L.s_out)[tid] = (unsigned short)lo;
+          *reinterpret_cast<unsigned short*>(cluster.map_shared_rank(oh_s, dst) + sw(token, tid * 2, L.s_out)) = (unsigned short)hi;
+          *reinterpret_cast<unsigned short*>(cluster.map_shared_rank(ol_s, dst) + sw(token, tid * 2, L.s_out)) = (unsigned short)lo;
         }
       }
       __syncthreads();
@@ -456,43 +464,83 @@ struct FfnBlockParams {
   const int* all_done;
 };
 
-// acc[nt] += W(16 rows x 16) * X(16 x 8 tokens of tile nt): the 16-wide version of mma_rows16 (lane (g, t) takes
-// k = 4t..4t+3, eight contiguous bytes, as slots {2t, 2t+1, 2t+8, 2t+9}).
-template <int NT>
-__device__ __forceinline__ void mma_rows16_k16(float (&acc)[NT][4], const uint8_t* w, int sw, const uint8_t* xh,
-                                               const uint8_t* xl, int sx, int lane) {
-  const int g = lane >> 2, t = lane & 3;
-  const uint2 a = *reinterpret_cast<const uint2*>(w + g * sw + t * 8);
-  const uint2 b = *reinterpret_cast<const uint2*>(w + (g + 8) * sw + t * 8);
+// Statistics as in rows_stats, and in the same pass the planes of x * gain for whole rows (lay-out sw(), d * 2
+// bytes per row).  The gain is static; the caller has asked for it to be brought into L1 before the wait.
+__device__ __forceinline__ void rows_stats_full_planes(const float* __restrict__ x, const bf16* __restrict__ gain, int R, int d,
+                                                       float eps, uint8_t* __restrict__ xh, uint8_t* __restrict__ xl,
+                                                       float* s_mean, float* s_rstd) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nv = d >> 2, rb = d * 2;
+  constexpr int kBatch = 8;
+  const float per_lane = (float)(d >> 5), inv_per_lane = 1.0f / per_lane;
+  for (int tk = warp; tk < R; tk += kWarps) {
+    const float4* xr = reinterpret_cast<const float4*>(x + (size_t)tk * d);
+    float shift = 0.f, a1 = 0.f, a2 = 0.f;
+    for (int i0 = lane; i0 < nv; i0 += 32 * kBatch) {
+      float4 buf[kBatch];
+      uint2 gw[kBatch];
 #pragma unroll
-  for (int nt = 0; nt < NT; ++nt) {
-    const uint2 h = *reinterpret_cast<const uint2*>(xh + (nt * 8 + g) * sx + t * 8);
-    const uint2 l = *reinterpret_cast<const uint2*>(xl + (nt * 8 + g) * sx + t * 8);
-    mma_bf16(acc[nt], a.x, b.x, a.y, b.y, h.x, h.y);
-    mma_bf16(acc[nt], a.x, b.x, a.y, b.y, l.x, l.y);
+      for (int u = 0; u < kBatch; ++u) {
+        const bool in = i0 + 32 * u < nv;
+        buf[u] = in ? __ldcg(&xr[i0 + 32 * u]) : make_float4(0.f, 0.f, 0.f, 0.f);
+        gw[u] = in ? *reinterpret_cast<const uint2*>(gain + (i0 + 32 * u) * 4) : make_uint2(0u, 0u);
+      }
+      if (i0 == lane) shift = buf[0].x;
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) {
+        if (i0 + 32 * u < nv) {
+          const float4 a = buf[u];
+          const float d0 = a.x - shift, d1 = a.y - shift, d2 = a.z - shift, d3 = a.w - shift;
+          a1 += (d0 + d1) + (d2 + d3);
+          a2 += (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
+          const float v[4] = {a.x * __uint_as_float(gw[u].x << 16), a.y * __uint_as_float(gw[u].x & 0xffff0000u),
+                              a.z * __uint_as_float(gw[u].y << 16), a.w * __uint_as_float(gw[u].y & 0xffff0000u)};
+          uint32_t hi[4], lo[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) split_bits(v[e], hi[e], lo[e]);
+          const int at = sw(tk, (i0 + 32 * u) * 8, rb);
+          *reinterpret_cast<uint2*>(xh + at) = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
+          *reinterpret_cast<uint2*>(xl + at) = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
+        }
+      }
+    }
+    float mu = shift + a1 * inv_per_lane;
+    float m2 = a2 - a1 * a1 * inv_per_lane;
+    float half_n = 0.5f * per_lane;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const float mb = __shfl_xor_sync(0xffffffffu, mu, off);
+      const float qb = __shfl_xor_sync(0xffffffffu, m2, off);
+      const float delta = mb - mu;
+      m2 = (m2 + qb) + delta * delta * half_n;
+      mu = 0.5f * (mu + mb);
+      half_n *= 2.f;
+    }
+    if (lane == 0) {
+      s_mean[tk] = mu;
+      s_rstd[tk] = rsqrtf(fmaxf(m2, 0.f) / (float)d + eps);
+    }
   }
 }
 
 struct FfnLayout {
-  int s1, s2, s_x, s_h, s_p;      // row strides: bytes, except s_p (floats between the tokens of the partial output)
-  int w1, w2, xh, xl, hh, hl, part1, mean, rstd, flag, total;   // the partial output shares the bytes of w1
+  int s1, s2, s_x, s_h;           // bytes per row
+  int w1, w2, xh, xl, hh, hl, acc, mean, rstd, flag, total;
   int zero_begin, zero_end;
 };
 __host__ __device__ inline FfnLayout ffn_layout(int d, int NT) {
   FfnLayout L;
-  const int ks = d / kC;
-  L.s1 = padded(ks * 2); L.s2 = kHS * 2; L.s_x = padded(ks * 2); L.s_h = kHS * 2; L.s_p = d + 4;
+  L.s1 = d * 2; L.s2 = kC * kHS * 2; L.s_x = d * 2; L.s_h = kC * kHS * 2;
   int off = 0;
-  const int w1_bytes = kC * kHS * L.s1, out_bytes = NT * 8 * L.s_p * 4;
-  L.w1 = off; off += (w1_bytes > out_bytes ? w1_bytes : out_bytes);
-  L.w2 = off; off += d * L.s2;
+  L.w1 = off; off += kHS * L.s1;
+  L.w2 = off; off += (d / kC) * L.s2;
   L.zero_begin = off;
   L.xh = off; off += NT * 8 * L.s_x;
   L.xl = off; off += NT * 8 * L.s_x;
   L.hh = off; off += NT * 8 * L.s_h;
   L.hl = off; off += NT * 8 * L.s_h;
   L.zero_end = off;
-  L.part1 = off; off += kC * kHS * NT * 8 * 4;
+  L.acc = off; off += kWarps * NT * kHS * 8 * 4;
   L.mean = off; off += kMaxRows * 4;
   L.rstd = off; off += kMaxRows * 4;
   L.flag = off; off += 16;
@@ -507,130 +555,107 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) ffn_bl
   const int c = (int)cluster.block_rank(), j = blockIdx.y;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t4 = lane & 3;
-  const int d = p.d, ks = d / kC, slice = d / kC;
-  const int hid_cluster = j * kC * kHS, hid0 = hid_cluster + c * kHS;
+  const int d = p.d, slice = d / kC;
+  constexpr int HC = kC * kHS;                       // hidden units of a cluster
+  const int hid_cluster = j * HC, hid0 = hid_cluster + c * kHS;
   const FfnLayout L = ffn_layout(d, NT);
   uint8_t* w1_s = fsm + L.w1;
-  float* out_s = reinterpret_cast<float*>(fsm + L.w1);
   uint8_t* w2_s = fsm + L.w2;
   uint8_t* xh_s = fsm + L.xh;
   uint8_t* xl_s = fsm + L.xl;
   uint8_t* hh_s = fsm + L.hh;
   uint8_t* hl_s = fsm + L.hl;
-  float* part1_s = reinterpret_cast<float*>(fsm + L.part1);
+  float* acc_s = reinterpret_cast<float*>(fsm + L.acc);
   float* s_mean = reinterpret_cast<float*>(fsm + L.mean);
   float* s_rstd = reinterpret_cast<float*>(fsm + L.rstd);
   volatile int* flag = reinterpret_cast<volatile int*>(fsm + L.flag);
 
   // TRACE 0
   pdl_launch_dependents();
-  cluster_arrive();
-  // Static weights of this CTA: the cluster's kC * kHS rows of the first projection restricted to this rank's ks
-  // columns, and this rank's kHS columns of the second projection (all d rows).
+  // Static weights of this CTA: its kHS rows of the first projection (all d columns) and, of the second
+  // projection, the rows of feature slice c restricted to the cluster's HC hidden units.
   {
-    const int cpr = ks * 2 / 16;
-    for (int idx = tid; idx < kC * kHS * cpr; idx += kThreads) {
+    const int cpr = d * 2 / 16;
+    for (int idx = tid; idx < kHS * cpr; idx += kThreads) {
       const int row = idx / cpr, c16 = idx % cpr;
-      cp_async16(w1_s + row * L.s1 + c16 * 16, p.w1 + (size_t)(hid_cluster + row) * d + c * ks + c16 * 8);
+      cp_async16(w1_s + sw(row, c16 * 16, L.s1), p.w1 + (size_t)(hid0 + row) * d + c16 * 8);
     }
-    constexpr int cpr2 = kHS * 2 / 16;
-    for (int idx = tid; idx < d * cpr2; idx += kThreads) {
+    constexpr int cpr2 = HC * 2 / 16;
+    for (int idx = tid; idx < slice * cpr2; idx += kThreads) {
       const int row = idx / cpr2, c16 = idx % cpr2;
-      cp_async16(w2_s + row * L.s2 + c16 * 16, p.w2 + (size_t)row * p.ff + hid0 + c16 * 8);
+      cp_async16(w2_s + sw(row, c16 * 16, L.s2), p.w2 + (size_t)(c * slice + row) * p.ff + hid_cluster + c16 * 8);
     }
     cp_async_commit();
   }
   for (int i = L.zero_begin / 16 + tid; i < L.zero_end / 16; i += kThreads) reinterpret_cast<uint4*>(fsm)[i] = make_uint4(0, 0, 0, 0);
-  // folded layer-norm vectors of the hidden unit this thread finishes (kHS * R <= 256 items, one per thread)
+  // the folded layer-norm vectors of the hidden unit this thread finishes (kHS * R <= 256 items, one per thread);
+  // the gain is wanted right after the wait: bring it close
   const float fs = p.fold_s[hid0 + tid % kHS], fc = p.fold_c[hid0 + tid % kHS];
-  uint2 gwords[2];
-  planes_gain(p.gain, p.R, c * ks, ks, gwords);
+  if (tid * 64 < d) asm volatile("prefetch.global.L1 [%0];" ::"l"(p.gain + tid * 64));
   __syncthreads();
+  cluster_arrive();            // this CTA's shared memory is set up; matched by cluster_wait() below
   // TRACE 1
   pdl_wait();
   // TRACE 2
   const int ended = p.all_done ? *p.all_done : 0;      // the same answer in every CTA
-  float4 xrow[2];
-  planes_fetch(p.x, p.R, d, c * ks, ks, xrow);
-  rows_stats(p.x, p.R, d, p.eps, s_mean, s_rstd);
-  planes_store(xrow, gwords, p.R, ks, xh_s, xl_s, L.s_x);
+  rows_stats_full_planes(p.x, p.gain, p.R, d, p.eps, xh_s, xl_s, s_mean, s_rstd);
   // TRACE 3
   cp_async_wait_all();
   __syncthreads();
-  cluster_wait();
+  cluster_wait();                                      // every CTA of the cluster is running
   if (ended) return;
   // TRACE 4
 
-  // ---- first projection of the cluster's hidden units over this rank's columns; unit f belongs to rank f / kHS
-  for (int mt = warp; mt < kC * kHS / 16; mt += kWarps) {
+  // ---- first projection: this CTA's kHS hidden units, the reduction split over the warps
+  {
+    const int kr = d / kWarps;
     float acc[NT][4];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
-    mma_rows16<NT>(acc, w1_s + mt * 16 * L.s1, L.s1, xh_s, xl_s, L.s_x, ks, lane);
+    mma_rows16<NT>(acc, w1_s, L.s1, xh_s, xl_s, L.s_x, kr, lane, warp * kr * 2);
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int f = mt * 16 + g + ((e & 2) ? 8 : 0), token = nt * 8 + 2 * t4 + (e & 1);
-        if (token < p.R) {
-          float* remote = cluster.map_shared_rank(part1_s, f / kHS);
-          remote[(c * kHS + f % kHS) * (NT * 8) + token] = acc[nt][e];
-        }
-      }
-  }
-  // TRACE 5
-  cluster.sync();
-  // TRACE 6
-
-  // ---- this rank's hidden units: partials in rank order, layer norm, bias, ReLU, planes
-  for (int idx = tid; idx < kHS * p.R; idx += kThreads) {
-    const int f = idx % kHS, token = idx / kHS;
-    float a = 0.f;
-#pragma unroll
-    for (int src = 0; src < kC; ++src) a += part1_s[(src * kHS + f) * (NT * 8) + token];
-    const float y = fmaxf(s_rstd[token] * (a - s_mean[token] * fs) + fc, 0.f);     // idx == tid: f == tid % kHS
-    uint32_t hi, lo;
-    split_bits(y, hi, lo);
-    reinterpret_cast<unsigned short*>(hh_s + token * L.s_h)[f] = (unsigned short)hi;
-    reinterpret_cast<unsigned short*>(hl_s + token * L.s_h)[f] = (unsigned short)lo;
+      for (int e = 0; e < 4; ++e)
+        acc_s[((warp * NT + nt) * kHS + g + ((e & 2) ? 8 : 0)) * 8 + 2 * t4 + (e & 1)] = acc[nt][e];
   }
   __syncthreads();
+  // TRACE 5
+  // warps in order, layer norm, bias, ReLU; every rank of the cluster gets the planes of these hidden units
+  if (tid < kHS * p.R) {
+    const int f = tid % kHS, token = tid / kHS;
+    float a = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) a += acc_s[((w * NT + token / 8) * kHS + f) * 8 + (token & 7)];
+    const float y = fmaxf(s_rstd[token] * (a - s_mean[token] * fs) + fc, 0.f);
+    uint32_t hi, lo;
+    split_bits(y, hi, lo);
+    const int at = sw(token, (c * kHS + f) * 2, L.s_h);
+#pragma unroll
+    for (int dst = 0; dst < kC; ++dst) {
+      *reinterpret_cast<unsigned short*>(cluster.map_shared_rank(hh_s, dst) + at) = (unsigned short)hi;
+      *reinterpret_cast<unsigned short*>(cluster.map_shared_rank(hl_s, dst) + at) = (unsigned short)lo;
+    }
+  }
+  // TRACE 6
+  cluster.sync();
   // TRACE 7
 
-  // ---- second projection restricted to these kHS hidden units, all d features, kept in this CTA's shared memory
-  // (over the bytes of the first projection's weights, which this CTA no longer reads)
-  for (int mt = warp; mt < d / 16; mt += kWarps) {
+  // ---- second projection: feature slice c, over the cluster's hidden units: the cluster's share of the output
+  float* wsj = p.ws + (size_t)j * p.R * d;
+  for (int mt = warp; mt < slice / 16; mt += kWarps) {
     float acc[NT][4];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
-    mma_rows16_k16<NT>(acc, w2_s + mt * 16 * L.s2, L.s2, hh_s, hl_s, L.s_h, lane);
+    mma_rows16<NT>(acc, w2_s + mt * 16 * L.s2, L.s2, hh_s, hl_s, L.s_h, HC, lane);
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        const int n = mt * 16 + g + ((e & 2) ? 8 : 0), token = nt * 8 + 2 * t4 + (e & 1);
-        out_s[token * L.s_p + n] = acc[nt][e];
+        const int row = mt * 16 + g + ((e & 2) ? 8 : 0), token = nt * 8 + 2 * t4 + (e & 1);
+        if (token < p.R) wsj[(size_t)token * d + c * slice + row] = acc[nt][e];
       }
   }
-  // TRACE 8
-  cluster.sync();
-  // TRACE 9
-
-  // ---- rank c collects feature slice c from all eight ranks (in rank order): the cluster's share of the output
-  float* wsj = p.ws + (size_t)j * p.R * d;
-  const int s4 = slice >> 2;
-  for (int idx = tid; idx < s4 * p.R; idx += kThreads) {
-    const int f4 = idx % s4, token = idx / s4;
-    float4 v[kC];
-#pragma unroll
-    for (int src = 0; src < kC; ++src)
-      v[src] = *reinterpret_cast<const float4*>(cluster.map_shared_rank(out_s, src) + token * L.s_p + c * slice + f4 * 4);
-    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-    for (int src = 0; src < kC; ++src) { a.x += v[src].x; a.y += v[src].y; a.z += v[src].z; a.w += v[src].w; }
-    *reinterpret_cast<float4*>(wsj + (size_t)token * d + c * slice + f4 * 4) = a;
-  }
-  cluster_arrive();          // this CTA has read what it needs from the others
   __syncthreads();
   // TRACE 10
   if (tid == 0) *flag = (tc::atom_add_acq_rel(&p.counters[c], 1u) == (unsigned)p.NJ - 1) ? 1 : 0;
@@ -640,7 +665,6 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) ffn_bl
     merge_slice(p.x, p.ws, p.b2, p.NJ, p.R, d, c * slice, slice);
     if (tid == 0) p.counters[c] = 0;
   }
-  cluster_wait();            // nobody leaves while another rank may still read its shared memory
 }
 
 // Shapes this path is built for.
