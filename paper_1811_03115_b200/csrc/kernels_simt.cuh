@@ -506,16 +506,34 @@ __device__ __forceinline__ float attention_head(const AttnParams& p, int b, int 
     const size_t base = p.paged ? ((size_t)pt[c0 / kPage] * kPage + (c0 % kPage)) * p.ldkv + h * DH
                                 : (size_t)b * p.bstride + (size_t)c0 * p.ldkv + h * DH;
     const int nk = min(32, limit - c0);
-    float sc = -INFINITY;
+    // key row of this lane and the first batch of value rows are fetched together (a warp issues in order: all
+    // loads go out before the first one is used).  Value rows are taken VB at a time; rows beyond the chunk's
+    // last key repeat it with weight 0 (pj is 0 in those lanes), which leaves the sum unchanged.
+    constexpr int VB0 = ((sizeof(CT) == 2) ? 64 : 32) / DPL, VB = VB0 > 32 ? 32 : (VB0 < 8 ? 8 : VB0);
+    const CT* vb = V + base + dim0;
+    float kv[DH / 8][8];
     if (lane < nk) {
       const CT* kr = K + base + (size_t)lane * p.ldkv;
+#pragma unroll
+      for (int c = 0; c < DH; c += 8) {
+        if (COHERENT) load8_cg(kr + c, kv[c / 8]); else load8(kr + c, kv[c / 8]);
+      }
+    }
+    float vv[VB][DPL];
+    if (owns) {
+#pragma unroll
+      for (int jj = 0; jj < VB; ++jj) {
+        const int jc = min(jj, nk - 1);
+        if (COHERENT) load_n_cg<DPL>(vb + (size_t)jc * p.ldkv, vv[jj]); else load_n<DPL>(vb + (size_t)jc * p.ldkv, vv[jj]);
+      }
+    }
+    float sc = -INFINITY;
+    if (lane < nk) {
       float dot = 0.f;
 #pragma unroll
       for (int c = 0; c < DH; c += 8) {
-        float kv[8];
-        if (COHERENT) load8_cg(kr + c, kv); else load8(kr + c, kv);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) dot = fmaf(sm.q[c + e], kv[e], dot);
+        for (int e = 0; e < 8; ++e) dot = fmaf(sm.q[c + e], kv[c / 8][e], dot);
       }
       sc = dot;
     }
@@ -525,15 +543,10 @@ __device__ __forceinline__ float attention_head(const AttnParams& p, int b, int 
     l_run = l_run * corr + warp_sum(pj);
 #pragma unroll
     for (int t = 0; t < DPL; ++t) acc[t] *= corr;
-    const CT* vb = V + base + dim0;
-    // value rows are fetched VB at a time so that their loads overlap; rows beyond the chunk's last key repeat
-    // it with weight 0 (pj is 0 in those lanes), which leaves the sum unchanged
-    constexpr int VB0 = ((sizeof(CT) == 2) ? 64 : 32) / DPL, VB = VB0 > 32 ? 32 : (VB0 < 8 ? 8 : VB0);
 #pragma unroll
     for (int j0 = 0; j0 < 32; j0 += VB) {
       if (j0 < nk) {
-        float vv[VB][DPL];
-        if (owns) {
+        if (j0 > 0 && owns) {
 #pragma unroll
           for (int jj = 0; jj < VB; ++jj) {
             const int jc = min(j0 + jj, nk - 1);
