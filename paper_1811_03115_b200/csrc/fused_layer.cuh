@@ -45,8 +45,9 @@ constexpr int kMaxRows = 16;
 // fragment loads of eight lanes (two rows x four quarters) cover all 32 banks once; 64-byte rows do so as they are.
 __host__ __device__ inline int sw(int row, int byte, int rb) { return row * rb + ((rb & 127) ? byte : (byte ^ ((row & 1) << 6))); }
 
-__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(tc::smem_u32(smem)), "l"(gmem) : "memory");
+// 16 bytes of weights, global -> shared, marked "evict first" in L2 (they are read once per pass).
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem, unsigned long long policy) {
+  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(tc::smem_u32(smem)), "l"(gmem), "l"(policy) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
@@ -293,6 +294,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
 
   // TRACE 0
   pdl_launch_dependents();
+  const unsigned long long stream = tc::l2_evict_first();
   // Everything that does not depend on the previous launch starts now.  This CTA's weights: ROWS_IN rows x ks
   // columns of the input projection, `slice` rows x 64 columns of the output projection.
   {
@@ -300,11 +302,11 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
     for (int idx = tid; idx < ROWS_IN * cpr; idx += kThreads) {
       const int row = idx / cpr, c16 = idx % cpr;
       const int grow = (row / kDH) * d + h * kDH + (row % kDH);
-      cp_async16(w_in_s + sw(row, c16 * 16, L.s_in), p.w_in + (size_t)grow * d + c * ks + c16 * 8);
+      cp_async16(w_in_s + sw(row, c16 * 16, L.s_in), p.w_in + (size_t)grow * d + c * ks + c16 * 8, stream);
     }
     for (int idx = tid; idx < slice * 8; idx += kThreads) {
       const int row = idx >> 3, c16 = idx & 7;
-      cp_async16(w_out_s + sw(row, c16 * 16, L.s_out), p.w_out + (size_t)(c * slice + row) * d + h * kDH + c16 * 8);
+      cp_async16(w_out_s + sw(row, c16 * 16, L.s_out), p.w_out + (size_t)(c * slice + row) * d + h * kDH + c16 * 8, stream);
     }
     cp_async_commit();
   }
@@ -335,6 +337,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
   float4 xrow[2];
   planes_fetch(p.x, p.R, d, c * ks, ks, xrow);
   rows_stats(p.x, p.R, d, p.eps, s_mean, s_rstd);
+  // TRACE 14
   if (SELF && tid < nb) s_len[tid] = len_v;
   planes_store(xrow, gwords, p.R, ks, xh_s, xl_s, L.s_x);
   // TRACE 3
@@ -401,11 +404,13 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
     if (token < p.R) {                   // uniform over the CTA
       if (tid < kDH) sm.q[tid] = q_s[slot * kDH + tid];
       __syncthreads();
+      // TRACE 12
       const int b = token / p.rows_per_b, i = token % p.rows_per_b;
       const int limit = SELF ? (s_len[b] + i + 1) : s_len[b];
       float ov;
       if (SELF) ov = attention_head<bf16, kDH, kWarps, true>(ap, b, h, limit, sm);
       else ov = attention_head<float, kDH, kWarps, false>(ap, b, h, limit, sm);
+      // TRACE 13
       if (tid < kDH) {
         uint32_t hi, lo;
         split_bits(ov, hi, lo);
@@ -572,18 +577,19 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) ffn_bl
 
   // TRACE 0
   pdl_launch_dependents();
+  const unsigned long long stream = tc::l2_evict_first();
   // Static weights of this CTA: its kHS rows of the first projection (all d columns) and, of the second
   // projection, the rows of feature slice c restricted to the cluster's HC hidden units.
   {
     const int cpr = d * 2 / 16;
     for (int idx = tid; idx < kHS * cpr; idx += kThreads) {
       const int row = idx / cpr, c16 = idx % cpr;
-      cp_async16(w1_s + sw(row, c16 * 16, L.s1), p.w1 + (size_t)(hid0 + row) * d + c16 * 8);
+      cp_async16(w1_s + sw(row, c16 * 16, L.s1), p.w1 + (size_t)(hid0 + row) * d + c16 * 8, stream);
     }
     constexpr int cpr2 = HC * 2 / 16;
     for (int idx = tid; idx < slice * cpr2; idx += kThreads) {
       const int row = idx / cpr2, c16 = idx % cpr2;
-      cp_async16(w2_s + sw(row, c16 * 16, L.s2), p.w2 + (size_t)(c * slice + row) * p.ff + hid_cluster + c16 * 8);
+      cp_async16(w2_s + sw(row, c16 * 16, L.s2), p.w2 + (size_t)(c * slice + row) * p.ff + hid_cluster + c16 * 8, stream);
     }
     cp_async_commit();
   }

@@ -67,6 +67,7 @@ struct TcParams {
   const bf16* g_next; bf16* xg_hi; long long xg_plane;
   int* error;                  // device error word
   const int* all_done;
+  int stream_weights;          // 1: the weights are read once per launch (one token tile): load them "evict first"
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -102,6 +103,19 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+// Same with an L2 policy: weights that are read once per pass are marked "evict first", so that streaming
+// hundreds of MB through the 126 MB L2 does not push out what every pass reads again (caches, small vectors).
+__device__ __forceinline__ unsigned long long l2_evict_first() {
+  unsigned long long pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y,
+                                                 unsigned long long policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "l"(policy) : "memory");
 }
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
@@ -519,7 +533,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int npre = min(nchunks, kStages);
     for (int it = 0; it < npre; ++it) {
       mbar_expect_tx(bars + 8 * it, stage_sz);
-      tma_load_2d(base + it * stage_sz, &tmA, bars + 8 * it, (c0 + it) * kBK, a_row);
+      if (p.stream_weights) tma_load_2d_hint(base + it * stage_sz, &tmA, bars + 8 * it, (c0 + it) * kBK, a_row, l2_evict_first());
+      else tma_load_2d(base + it * stage_sz, &tmA, bars + 8 * it, (c0 + it) * kBK, a_row);
     }
     pdl_wait();
     const bool skip = p.all_done && *p.all_done;
@@ -539,7 +554,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const uint32_t sa = base + s * stage_sz;
       mbar_expect_tx(full, stage_sz);
       const int kx = (c0 + it) * kBK;
-      tma_load_2d(sa, &tmA, full, kx, a_row);
+      if (p.stream_weights) tma_load_2d_hint(sa, &tmA, full, kx, a_row, l2_evict_first());
+      else tma_load_2d(sa, &tmA, full, kx, a_row);
       tma_load_2d(sa + kBM * 128, &tmBh, full, slice * b_cols_per_slice + kx, t0);
       tma_load_2d(sa + kBM * 128 + bn * 128, &tmBl, full, slice * b_cols_per_slice + kx, t0);
     }

@@ -158,6 +158,7 @@ int launch(const Operands& op, int N, int K, int T, TcParams p, const Scratch& s
   p.T = T; p.N = N; p.K = K; p.bn = bn; p.splits = pl.splits; p.chunks_per_split = pl.chunks_per_split;
   p.ws = sc.ws; p.tile_counters = sc.tile_counters; p.done_counter = sc.done_counter;
   p.best = sc.best; p.error = sc.error;
+  p.stream_weights = (ttiles == 1 && !getenv("BPD_NO_L2_HINTS")) ? 1 : 0;
   dim3 grid(pl.tiles, pl.splits, ttiles * zslices);
   BPD_CUDA(launch_k(gemm_tc_kernel<EPI>, grid, dim3(kThreads), smem_bytes(bn), st, pdl, ma, mh, ml, p, zslices,
                     a_rows_per_slice, b_cols_per_slice));
