@@ -9,9 +9,10 @@
 //   attn_block_kernel<SELF>   layer norm -> Q,K,V of one head -> cache write -> attention -> that head's share of
 //                             the output projection -> sum over heads + residual
 //   attn_block_kernel<CROSS>  layer norm -> Q of one head -> attention over the encoder keys -> same tail
-//   ffn_block_kernel          layer norm -> 16 hidden units (ReLU) -> shared with the cluster -> the cluster's 128
-//                             hidden units times this CTA's slice of the second projection -> sum over clusters
-//                             + bias + residual
+//   ffn_block_kernel          layer norm -> the cluster's 128 hidden units, each CTA over its part of the reduction
+//                             -> 16 of them finished per CTA (ReLU) and shared with the cluster -> the 128 hidden
+//                             units times this CTA's slice of the second projection -> sum over clusters + bias
+//                             + residual
 //
 // One thread-block cluster of kC CTAs works on a head (or on kC * 16 hidden units).  In the attention blocks the
 // reduction length of the input projection is split over the CTAs and partial sums travel through distributed
@@ -188,9 +189,9 @@ __device__ __forceinline__ void planes_store(const float4 (&v)[2], const uint2 (
 
 // Sum over `np` partial outputs + residual (+ bias) for the feature slice [col0, col0 + width) of all R rows, by
 // the CTA that completed the slice: x[t][f] += bias[f] + ws[0][t][f] + ws[1][t][f] + ... in that order.
+template <int kBatch>
 __device__ __forceinline__ void merge_slice(float* x, const float* ws, const bf16* bias, int np, int R, int d, int col0, int width) {
   const int w4 = width >> 2;
-  constexpr int kBatch = 16;
   for (int idx = threadIdx.x; idx < R * w4; idx += kThreads) {
     const int t = idx / w4, col = col0 + (idx % w4) * 4;
     float4 acc = __ldcg(reinterpret_cast<const float4*>(x + (size_t)t * d + col));
@@ -448,7 +449,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
   __syncthreads();
   // TRACE 11
   if (*flag) {                           // last head to arrive at this slice: heads are added in head order
-    merge_slice(p.x, p.ws, nullptr, p.H, p.R, d, c * slice, slice);
+    merge_slice<16>(p.x, p.ws, nullptr, p.H, p.R, d, c * slice, slice);
     if (tid == 0) p.counters[c] = 0;
   }
 }
@@ -469,83 +470,27 @@ struct FfnBlockParams {
   const int* all_done;
 };
 
-// Statistics as in rows_stats, and in the same pass the planes of x * gain for whole rows (lay-out sw(), d * 2
-// bytes per row).  The gain is static; the caller has asked for it to be brought into L1 before the wait.
-__device__ __forceinline__ void rows_stats_full_planes(const float* __restrict__ x, const bf16* __restrict__ gain, int R, int d,
-                                                       float eps, uint8_t* __restrict__ xh, uint8_t* __restrict__ xl,
-                                                       float* s_mean, float* s_rstd) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int nv = d >> 2, rb = d * 2;
-  constexpr int kBatch = 8;
-  const float per_lane = (float)(d >> 5), inv_per_lane = 1.0f / per_lane;
-  for (int tk = warp; tk < R; tk += kWarps) {
-    const float4* xr = reinterpret_cast<const float4*>(x + (size_t)tk * d);
-    float shift = 0.f, a1 = 0.f, a2 = 0.f;
-    for (int i0 = lane; i0 < nv; i0 += 32 * kBatch) {
-      float4 buf[kBatch];
-      uint2 gw[kBatch];
-#pragma unroll
-      for (int u = 0; u < kBatch; ++u) {
-        const bool in = i0 + 32 * u < nv;
-        buf[u] = in ? __ldcg(&xr[i0 + 32 * u]) : make_float4(0.f, 0.f, 0.f, 0.f);
-        gw[u] = in ? *reinterpret_cast<const uint2*>(gain + (i0 + 32 * u) * 4) : make_uint2(0u, 0u);
-      }
-      if (i0 == lane) shift = buf[0].x;
-#pragma unroll
-      for (int u = 0; u < kBatch; ++u) {
-        if (i0 + 32 * u < nv) {
-          const float4 a = buf[u];
-          const float d0 = a.x - shift, d1 = a.y - shift, d2 = a.z - shift, d3 = a.w - shift;
-          a1 += (d0 + d1) + (d2 + d3);
-          a2 += (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
-          const float v[4] = {a.x * __uint_as_float(gw[u].x << 16), a.y * __uint_as_float(gw[u].x & 0xffff0000u),
-                              a.z * __uint_as_float(gw[u].y << 16), a.w * __uint_as_float(gw[u].y & 0xffff0000u)};
-          uint32_t hi[4], lo[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) split_bits(v[e], hi[e], lo[e]);
-          const int at = sw(tk, (i0 + 32 * u) * 8, rb);
-          *reinterpret_cast<uint2*>(xh + at) = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
-          *reinterpret_cast<uint2*>(xl + at) = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
-        }
-      }
-    }
-    float mu = shift + a1 * inv_per_lane;
-    float m2 = a2 - a1 * a1 * inv_per_lane;
-    float half_n = 0.5f * per_lane;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-      const float mb = __shfl_xor_sync(0xffffffffu, mu, off);
-      const float qb = __shfl_xor_sync(0xffffffffu, m2, off);
-      const float delta = mb - mu;
-      m2 = (m2 + qb) + delta * delta * half_n;
-      mu = 0.5f * (mu + mb);
-      half_n *= 2.f;
-    }
-    if (lane == 0) {
-      s_mean[tk] = mu;
-      s_rstd[tk] = rsqrtf(fmaxf(m2, 0.f) / (float)d + eps);
-    }
-  }
-}
-
 struct FfnLayout {
   int s1, s2, s_x, s_h;           // bytes per row
-  int w1, w2, xh, xl, hh, hl, acc, mean, rstd, flag, total;
+  int w1, w2, xh, xl, hh, hl, part, mean, rstd, flag, total;
   int zero_begin, zero_end;
 };
 __host__ __device__ inline FfnLayout ffn_layout(int d, int NT) {
   FfnLayout L;
-  L.s1 = d * 2; L.s2 = kC * kHS * 2; L.s_x = d * 2; L.s_h = kC * kHS * 2;
+  const int ks = d / kC;
+  L.s1 = ks * 2; L.s2 = kC * kHS * 2; L.s_x = ks * 2; L.s_h = kC * kHS * 2;
   int off = 0;
-  L.w1 = off; off += kHS * L.s1;
+  L.w1 = off; off += kC * kHS * L.s1;
   L.w2 = off; off += (d / kC) * L.s2;
+  // The planes of the hidden units take the place of the planes of x: they are written (by the whole cluster)
+  // only after every rank has finished its first projection.  Rows of tokens beyond R hold left-overs; a token's
+  // column of a product depends on that token's row only, and those columns are never stored.
+  const int x_bytes = NT * 8 * L.s_x, h_bytes = NT * 8 * L.s_h, pl = x_bytes > h_bytes ? x_bytes : h_bytes;
   L.zero_begin = off;
-  L.xh = off; off += NT * 8 * L.s_x;
-  L.xl = off; off += NT * 8 * L.s_x;
-  L.hh = off; off += NT * 8 * L.s_h;
-  L.hl = off; off += NT * 8 * L.s_h;
+  L.xh = off; L.hh = off; off += pl;
+  L.xl = off; L.hl = off; off += pl;
   L.zero_end = off;
-  L.acc = off; off += kWarps * NT * kHS * 8 * 4;
+  L.part = off; off += kC * kHS * NT * 8 * 4;
   L.mean = off; off += kMaxRows * 4;
   L.rstd = off; off += kMaxRows * 4;
   L.flag = off; off += 16;
@@ -554,13 +499,13 @@ __host__ __device__ inline FfnLayout ffn_layout(int d, int NT) {
 }
 
 template <int NT>
-__global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) ffn_block_kernel(FfnBlockParams p) {
+__global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 3) ffn_block_kernel(FfnBlockParams p) {
   extern __shared__ __align__(16) uint8_t fsm[];
   cg::cluster_group cluster = cg::this_cluster();
   const int c = (int)cluster.block_rank(), j = blockIdx.y;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t4 = lane & 3;
-  const int d = p.d, slice = d / kC;
+  const int d = p.d, ks = d / kC, slice = d / kC;
   constexpr int HC = kC * kHS;                       // hidden units of a cluster
   const int hid_cluster = j * HC, hid0 = hid_cluster + c * kHS;
   const FfnLayout L = ffn_layout(d, NT);
@@ -570,7 +515,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) ffn_bl
   uint8_t* xl_s = fsm + L.xl;
   uint8_t* hh_s = fsm + L.hh;
   uint8_t* hl_s = fsm + L.hl;
-  float* acc_s = reinterpret_cast<float*>(fsm + L.acc);
+  float* part_s = reinterpret_cast<float*>(fsm + L.part);
   float* s_mean = reinterpret_cast<float*>(fsm + L.mean);
   float* s_rstd = reinterpret_cast<float*>(fsm + L.rstd);
   volatile int* flag = reinterpret_cast<volatile int*>(fsm + L.flag);
@@ -578,13 +523,13 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) ffn_bl
   // TRACE 0
   pdl_launch_dependents();
   const unsigned long long stream = tc::l2_evict_first();
-  // Static weights of this CTA: its kHS rows of the first projection (all d columns) and, of the second
-  // projection, the rows of feature slice c restricted to the cluster's HC hidden units.
+  // Static weights of this CTA: the cluster's HC rows of the first projection restricted to this rank's ks
+  // columns and, of the second projection, the rows of feature slice c restricted to the cluster's HC hidden units.
   {
-    const int cpr = d * 2 / 16;
-    for (int idx = tid; idx < kHS * cpr; idx += kThreads) {
+    const int cpr = ks * 2 / 16;
+    for (int idx = tid; idx < HC * cpr; idx += kThreads) {
       const int row = idx / cpr, c16 = idx % cpr;
-      cp_async16(w1_s + sw(row, c16 * 16, L.s1), p.w1 + (size_t)(hid0 + row) * d + c16 * 8, stream);
+      cp_async16(w1_s + sw(row, c16 * 16, L.s1), p.w1 + (size_t)(hid_cluster + row) * d + c * ks + c16 * 8, stream);
     }
     constexpr int cpr2 = HC * 2 / 16;
     for (int idx = tid; idx < slice * cpr2; idx += kThreads) {
@@ -594,17 +539,20 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) ffn_bl
     cp_async_commit();
   }
   for (int i = L.zero_begin / 16 + tid; i < L.zero_end / 16; i += kThreads) reinterpret_cast<uint4*>(fsm)[i] = make_uint4(0, 0, 0, 0);
-  // the folded layer-norm vectors of the hidden unit this thread finishes (kHS * R <= 256 items, one per thread);
-  // the gain is wanted right after the wait: bring it close
+  // the folded layer-norm vectors of the hidden unit this thread finishes (kHS * R <= 256 items, one per thread)
   const float fs = p.fold_s[hid0 + tid % kHS], fc = p.fold_c[hid0 + tid % kHS];
-  if (tid * 64 < d) asm volatile("prefetch.global.L1 [%0];" ::"l"(p.gain + tid * 64));
+  uint2 gwords[2];
+  planes_gain(p.gain, p.R, c * ks, ks, gwords);
   __syncthreads();
   cluster_arrive();            // this CTA's shared memory is set up; matched by cluster_wait() below
   // TRACE 1
   pdl_wait();
   // TRACE 2
   const int ended = p.all_done ? *p.all_done : 0;      // the same answer in every CTA
-  rows_stats_full_planes(p.x, p.gain, p.R, d, p.eps, xh_s, xl_s, s_mean, s_rstd);
+  float4 xrow[2];
+  planes_fetch(p.x, p.R, d, c * ks, ks, xrow);
+  rows_stats(p.x, p.R, d, p.eps, s_mean, s_rstd);
+  planes_store(xrow, gwords, p.R, ks, xh_s, xl_s, L.s_x);
   // TRACE 3
   cp_async_wait_all();
   __syncthreads();
@@ -612,27 +560,32 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) ffn_bl
   if (ended) return;
   // TRACE 4
 
-  // ---- first projection: this CTA's kHS hidden units, the reduction split over the warps
-  {
-    const int kr = d / kWarps;
+  // ---- first projection of the cluster's hidden units over this rank's columns; unit f belongs to rank f / kHS
+  for (int mt = warp; mt < HC / 16; mt += kWarps) {
     float acc[NT][4];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
-    mma_rows16<NT>(acc, w1_s, L.s1, xh_s, xl_s, L.s_x, kr, lane, warp * kr * 2);
+    mma_rows16<NT>(acc, w1_s + mt * 16 * L.s1, L.s1, xh_s, xl_s, L.s_x, ks, lane);
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-      for (int e = 0; e < 4; ++e)
-        acc_s[((warp * NT + nt) * kHS + g + ((e & 2) ? 8 : 0)) * 8 + 2 * t4 + (e & 1)] = acc[nt][e];
+      for (int e = 0; e < 4; ++e) {
+        const int f = mt * 16 + g + ((e & 2) ? 8 : 0), token = nt * 8 + 2 * t4 + (e & 1);
+        if (token < p.R) {
+          float* remote = cluster.map_shared_rank(part_s, f / kHS);
+          remote[(c * kHS + f % kHS) * (NT * 8) + token] = acc[nt][e];
+        }
+      }
   }
-  __syncthreads();
   // TRACE 5
-  // warps in order, layer norm, bias, ReLU; every rank of the cluster gets the planes of these hidden units
+  cluster.sync();
+  // TRACE 6
+  // ranks in order, layer norm, bias, ReLU; every rank of the cluster gets the planes of these hidden units
   if (tid < kHS * p.R) {
     const int f = tid % kHS, token = tid / kHS;
     float a = 0.f;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) a += acc_s[((w * NT + token / 8) * kHS + f) * 8 + (token & 7)];
+    for (int src = 0; src < kC; ++src) a += part_s[(src * kHS + f) * (NT * 8) + token];
     const float y = fmaxf(s_rstd[token] * (a - s_mean[token] * fs) + fc, 0.f);
     uint32_t hi, lo;
     split_bits(y, hi, lo);
@@ -643,9 +596,9 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) ffn_bl
       *reinterpret_cast<unsigned short*>(cluster.map_shared_rank(hl_s, dst) + at) = (unsigned short)lo;
     }
   }
-  // TRACE 6
-  cluster.sync();
   // TRACE 7
+  cluster.sync();
+  // TRACE 8
 
   // ---- second projection: feature slice c, over the cluster's hidden units: the cluster's share of the output
   float* wsj = p.ws + (size_t)j * p.R * d;
@@ -668,7 +621,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) ffn_bl
   __syncthreads();
   // TRACE 11
   if (*flag) {               // last cluster to arrive at this slice: clusters are added in cluster order
-    merge_slice(p.x, p.ws, p.b2, p.NJ, p.R, d, c * slice, slice);
+    merge_slice<12>(p.x, p.ws, p.b2, p.NJ, p.R, d, c * slice, slice);
     if (tid == 0) p.counters[c] = 0;
   }
 }
