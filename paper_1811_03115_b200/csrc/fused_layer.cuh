@@ -293,7 +293,6 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
   int* s_len = reinterpret_cast<int*>(fsm + L.len);    // per sequence: tokens in the cache (self) or source length (cross)
   int* s_pt = reinterpret_cast<int*>(fsm + L.pt);      // self: the sequences' page-table rows
 
-  // TRACE 0
   pdl_launch_dependents();
   const unsigned long long stream = tc::l2_evict_first();
   // Everything that does not depend on the previous launch starts now.  This CTA's weights: ROWS_IN rows x ks
@@ -328,9 +327,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
   planes_gain(p.gain, p.R, c * ks, ks, gwords);
   __syncthreads();
   cluster_arrive();            // this CTA's shared memory is set up; matched by cluster_wait() below
-  // TRACE 1
   pdl_wait();
-  // TRACE 2
   const int ended = p.all_done ? *p.all_done : 0;      // the same answer in every CTA
   // a warp issues in order: every load goes out before the first value is used
   int len_v = 0;
@@ -338,15 +335,12 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
   float4 xrow[2];
   planes_fetch(p.x, p.R, d, c * ks, ks, xrow);
   rows_stats(p.x, p.R, d, p.eps, s_mean, s_rstd);
-  // TRACE 14
   if (SELF && tid < nb) s_len[tid] = len_v;
   planes_store(xrow, gwords, p.R, ks, xh_s, xl_s, L.s_x);
-  // TRACE 3
   cp_async_wait_all();
   __syncthreads();
   cluster_wait();                                      // every CTA of the cluster is running: its shared memory may be written
   if (ended) return;
-  // TRACE 4
 
   // ---- input projection over this CTA's part of the reduction; token t's partial goes to rank t % kC
   for (int mt = warp; mt < ROWS_IN / 16; mt += kWarps) {
@@ -365,9 +359,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
         }
       }
   }
-  // TRACE 5
   cluster.sync();
-  // TRACE 6
 
   // ---- this rank's tokens: add the partials in rank order, finish the layer norm, write keys / values
   for (int slot = 0; slot < NT; ++slot) {
@@ -396,7 +388,6 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
     __syncthreads();
   }
 
-  // TRACE 7
   // ---- attention of this rank's rows; the result goes to every rank as planes
   AttnParams ap = p.attn;
   if (SELF) ap.st.page_table = s_pt;
@@ -405,13 +396,11 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
     if (token < p.R) {                   // uniform over the CTA
       if (tid < kDH) sm.q[tid] = q_s[slot * kDH + tid];
       __syncthreads();
-      // TRACE 12
       const int b = token / p.rows_per_b, i = token % p.rows_per_b;
       const int limit = SELF ? (s_len[b] + i + 1) : s_len[b];
       float ov;
       if (SELF) ov = attention_head<bf16, kDH, kWarps, true>(ap, b, h, limit, sm);
       else ov = attention_head<float, kDH, kWarps, false>(ap, b, h, limit, sm);
-      // TRACE 13
       if (tid < kDH) {
         uint32_t hi, lo;
         split_bits(ov, hi, lo);
@@ -424,9 +413,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
       __syncthreads();
     }
   }
-  // TRACE 8
   cluster.sync();
-  // TRACE 9
 
   // ---- this head's share of the output projection for the features of slice c
   float* wsh = p.ws + (size_t)h * p.R * d;
@@ -444,10 +431,8 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
       }
   }
   __syncthreads();
-  // TRACE 10
   if (tid == 0) *flag = (tc::atom_add_acq_rel(&p.counters[c], 1u) == (unsigned)p.H - 1) ? 1 : 0;
   __syncthreads();
-  // TRACE 11
   if (*flag) {                           // last head to arrive at this slice: heads are added in head order
     merge_slice<16>(p.x, p.ws, nullptr, p.H, p.R, d, c * slice, slice);
     if (tid == 0) p.counters[c] = 0;
@@ -520,7 +505,6 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 3) ffn_bl
   float* s_rstd = reinterpret_cast<float*>(fsm + L.rstd);
   volatile int* flag = reinterpret_cast<volatile int*>(fsm + L.flag);
 
-  // TRACE 0
   pdl_launch_dependents();
   const unsigned long long stream = tc::l2_evict_first();
   // Static weights of this CTA: the cluster's HC rows of the first projection restricted to this rank's ks
@@ -545,20 +529,16 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 3) ffn_bl
   planes_gain(p.gain, p.R, c * ks, ks, gwords);
   __syncthreads();
   cluster_arrive();            // this CTA's shared memory is set up; matched by cluster_wait() below
-  // TRACE 1
   pdl_wait();
-  // TRACE 2
   const int ended = p.all_done ? *p.all_done : 0;      // the same answer in every CTA
   float4 xrow[2];
   planes_fetch(p.x, p.R, d, c * ks, ks, xrow);
   rows_stats(p.x, p.R, d, p.eps, s_mean, s_rstd);
   planes_store(xrow, gwords, p.R, ks, xh_s, xl_s, L.s_x);
-  // TRACE 3
   cp_async_wait_all();
   __syncthreads();
   cluster_wait();                                      // every CTA of the cluster is running
   if (ended) return;
-  // TRACE 4
 
   // ---- first projection of the cluster's hidden units over this rank's columns; unit f belongs to rank f / kHS
   for (int mt = warp; mt < HC / 16; mt += kWarps) {
@@ -577,9 +557,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 3) ffn_bl
         }
       }
   }
-  // TRACE 5
   cluster.sync();
-  // TRACE 6
   // ranks in order, layer norm, bias, ReLU; every rank of the cluster gets the planes of these hidden units
   if (tid < kHS * p.R) {
     const int f = tid % kHS, token = tid / kHS;
@@ -596,9 +574,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 3) ffn_bl
       *reinterpret_cast<unsigned short*>(cluster.map_shared_rank(hl_s, dst) + at) = (unsigned short)lo;
     }
   }
-  // TRACE 7
   cluster.sync();
-  // TRACE 8
 
   // ---- second projection: feature slice c, over the cluster's hidden units: the cluster's share of the output
   float* wsj = p.ws + (size_t)j * p.R * d;
@@ -616,10 +592,8 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 3) ffn_bl
       }
   }
   __syncthreads();
-  // TRACE 10
   if (tid == 0) *flag = (tc::atom_add_acq_rel(&p.counters[c], 1u) == (unsigned)p.NJ - 1) ? 1 : 0;
   __syncthreads();
-  // TRACE 11
   if (*flag) {               // last cluster to arrive at this slice: clusters are added in cluster order
     merge_slice<12>(p.x, p.ws, p.b2, p.NJ, p.R, d, c * slice, slice);
     if (tid == 0) p.counters[c] = 0;
