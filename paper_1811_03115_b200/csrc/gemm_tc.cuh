@@ -176,6 +176,18 @@ __device__ __forceinline__ float unpack_value(unsigned long long key) {
   return __uint_as_float((ord & 0x80000000u) ? (ord & 0x7fffffffu) : ~ord);
 }
 
+// Warp-wide (value, index) maximum with ties to the lower index, for lanes whose indices grow with the lane
+// number: one integer max-reduction on the orderable pattern of the value, one ballot for the first lane that
+// holds it -- instead of a five-level shuffle butterfly on two registers.
+__device__ __forceinline__ void warp_argmax_lanes(float& v, int& idx) {
+  const unsigned b = __float_as_uint(v);
+  const unsigned ord = (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+  const unsigned m = __reduce_max_sync(0xffffffffu, ord);
+  const int src = __ffs(__ballot_sync(0xffffffffu, ord == m)) - 1;
+  idx = __shfl_sync(0xffffffffu, idx, src);
+  v = __uint_as_float((m & 0x80000000u) ? (m & 0x7fffffffu) : ~m);
+}
+
 // Arrival on a device-wide counter with release (our earlier writes, and those of the CTA's other threads
 // ordered before us by the barrier, become visible) and acquire (we see what earlier arrivals released).
 __device__ __forceinline__ unsigned atom_add_acq_rel(unsigned* addr, unsigned v) {
@@ -381,7 +393,7 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
             int ix = (n < p.N) ? n : 0x7fffffff;
             if (p.logits && cb + c < nt && n < p.N) p.logits[(size_t)(t0 + cb + c) * p.N + n] = x;
             if (cb + c < nt) count_beats(p, t0 + cb + c, n, x, lane);
-            warp_argmax(x, ix);
+            warp_argmax_lanes(x, ix);
             if (lane == 0) { s_val[q][cb + c] = x; s_idx[q][cb + c] = ix; }
           }
         }
@@ -434,7 +446,7 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
               int ix = (n < p.N) ? n : 0x7fffffff;
               if (p.logits && n < p.N) p.logits[(size_t)(t0 + cg + c) * p.N + n] = x;
               count_beats(p, t0 + cg + c, n, x, lane);
-              warp_argmax(x, ix);
+              warp_argmax_lanes(x, ix);
               if (lane == 0) { s_val[q][cg + c] = x; s_idx[q][cg + c] = ix; }
             }
           }
