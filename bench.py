@@ -53,6 +53,7 @@ DESCRIPTIONS = {
     "C3": "C3: big enc-dec 6+6, d_model 1024, 16 heads, FFN 4096, vocab 32768, k=8 dense heads, batch 1, source 40 ids",
     "C4": "C4: big enc-dec 6+6, d_model 1024, k=10 dense heads, batch 32, source lengths uniform in [10,80]",
     "C5": "C5: super-resolution shape, 6+6, d_model 512, vocab 256, k=10 dense heads, batch 1, 192 source ids",
+    "C5L": "C5L: C5 with 1D local self-attention in the decoder (query blocks of 256, memory 256)",
 }
 
 

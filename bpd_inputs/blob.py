@@ -22,7 +22,10 @@ header (128 bytes)::
     64  uint64   dir_offset       (= 128)
     72  uint64   data_offset
     80  uint64   total_bytes
-    88  zero padding to 128
+    88  int32    local_q          decoder self-attention: 0 = every earlier position; > 0 = 1D local attention
+                                  with query blocks of this length ...
+    92  int32    local_m          ... and this many positions of memory before the query's block
+    96  zero padding to 128
 
 directory: ``n_tensors`` entries of 96 bytes::
 
@@ -64,6 +67,8 @@ class ModelConfig:
     head_layout: int = HEAD_DENSE
     p1_identity: int = 0
     ln_eps: float = 1e-6
+    local_q: int = 0
+    local_m: int = 0
 
     @property
     def elem_bytes(self) -> int:
@@ -141,9 +146,9 @@ def write_blob(cfg: ModelConfig, tensors: Dict[str, np.ndarray]) -> np.ndarray:
     entries, data_offset, total = blob_layout(cfg)
     buf = np.zeros(total, dtype=np.uint8)
     hdr = struct.pack(
-        "<8s12ifiQQQ", BLOB_MAGIC, 1, cfg.dtype, cfg.n_enc, cfg.n_dec, cfg.d_model, cfg.n_heads,
+        "<8s12ifiQQQ2i", BLOB_MAGIC, 1, cfg.dtype, cfg.n_enc, cfg.n_dec, cfg.d_model, cfg.n_heads,
         cfg.d_ff, cfg.vocab, cfg.k_model, cfg.d_hidden, cfg.head_layout, cfg.p1_identity,
-        cfg.ln_eps, len(entries), HEADER_BYTES, data_offset, total)
+        cfg.ln_eps, len(entries), HEADER_BYTES, data_offset, total, cfg.local_q, cfg.local_m)
     buf[:len(hdr)] = np.frombuffer(hdr, dtype=np.uint8)
     pos = HEADER_BYTES
     want = np.float32 if cfg.dtype == DTYPE_F32 else np.uint16

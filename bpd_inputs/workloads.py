@@ -47,6 +47,9 @@ WORKLOADS: Dict[str, Workload] = {
     "C3": _wl("C3", 3, ModelConfig(6, 6, 1024, 16, 4096, 32768, 8, 4096), 0.02, 1, 40, 40, 128),
     "C4": _wl("C4", 4, ModelConfig(6, 6, 1024, 16, 4096, 32768, 10, 4096), 0.02, 32, 10, 80, 128),
     "C5": _wl("C5", 5, ModelConfig(6, 6, 512, 8, 2048, 256, 10, 2048), 0.02, 1, 192, 192, 3072, "sr"),
+    # C5 with 1D local self-attention in the decoder: query blocks of 256 positions, 256 positions of memory
+    "C5L": _wl("C5L", 5, ModelConfig(6, 6, 512, 8, 2048, 256, 10, 2048, local_q=256, local_m=256), 0.02, 1, 192, 192,
+               3072, "sr"),
 }
 
 

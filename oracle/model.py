@@ -37,6 +37,8 @@ class OracleModel:
     p1_identity: int
     eps: float
     w: Dict[str, np.ndarray]   # float64 tensors
+    local_q: int = 0           # decoder self-attention: 0 = full causal, else 1D local attention (query block,
+    local_m: int = 0           # memory length)
 
 
 def parse_blob(blob: np.ndarray) -> OracleModel:
@@ -50,6 +52,7 @@ def parse_blob(blob: np.ndarray) -> OracleModel:
     (eps,) = struct.unpack_from("<f", raw, 56)
     (n_tensors,) = struct.unpack_from("<i", raw, 60)
     dir_off, _data_off, total = struct.unpack_from("<3Q", raw, 64)
+    local_q, local_m = struct.unpack_from("<2i", raw, 88)
     if version != 1 or total != raw.size:
         raise ValueError("bad version or size")
     w: Dict[str, np.ndarray] = {}
@@ -66,7 +69,7 @@ def parse_blob(blob: np.ndarray) -> OracleModel:
             arr = (seg.view(np.uint16).astype(np.uint32) << 16).view(np.float32).astype(F64)
         w[name] = arr.reshape(shape)
     return OracleModel(n_enc, n_dec, d, H, d_ff, V, k_model, d_hidden, dtype, layout, p1id,
-                       float(eps), w)
+                       float(eps), w, int(local_q), int(local_m))
 
 
 # --------------------------------------------------------------------------- primitives
@@ -145,6 +148,22 @@ def encode(m: OracleModel, src_ids, src_len: Optional[int] = None) -> np.ndarray
 
 # --------------------------------------------------------------------------- decoder
 
+def self_attention_allowed(m: OracleModel, query_pos: np.ndarray, n_keys: int) -> np.ndarray:
+    """Which keys (positions 0..n_keys-1) each decoder query may attend to.
+
+    Causal: key j <= query position t.  With 1D local attention (Section 7.3
+    names it for the super-resolution model; the block lengths are this
+    build's choice, carried in the blob header) the target sequence is cut
+    into query blocks of local_q positions, and a query also sees only the
+    local_m positions before its own block: j >= (t // local_q) * local_q - local_m."""
+    t = np.asarray(query_pos)[:, None]
+    j = np.arange(n_keys)[None, :]
+    ok = j <= t
+    if m.local_q > 0:
+        ok &= j >= (t // m.local_q) * m.local_q - m.local_m
+    return ok
+
+
 def decoder_full(m: OracleModel, memory: np.ndarray, src_len: int, dec_inputs) -> np.ndarray:
     """Uncached decoder: final-layer-norm output h [n, d] for decoder inputs
     u_0..u_{n-1} (position of u_t is t).  Causal self-attention, cross-attention
@@ -153,7 +172,7 @@ def decoder_full(m: OracleModel, memory: np.ndarray, src_len: int, dec_inputs) -
     n = len(dec_inputs)
     S = memory.shape[0]
     x = embed(w["tgt_embed"], dec_inputs, 0)
-    causal = np.arange(n)[None, :] <= np.arange(n)[:, None]
+    causal = self_attention_allowed(m, np.arange(n), n)
     cross_ok = np.broadcast_to(np.arange(S)[None, :] < src_len, (n, S))
     for l in range(m.n_dec):
         p = f"dec.{l}"
@@ -190,7 +209,7 @@ class DecoderCache:
         writing their K/V speculatively (length is NOT advanced).  Returns h [n, d]."""
         m, w, T, n = self.m, self.m.w, self.length, len(tokens)
         x = embed(w["tgt_embed"], tokens, T)
-        allowed = np.arange(T + n)[None, :] <= (T + np.arange(n))[:, None]
+        allowed = self_attention_allowed(m, T + np.arange(n), T + n)
         S = self.cross[0][0].shape[0]
         cross_ok = np.broadcast_to(np.arange(S)[None, :] < self.src_len, (n, S))
         for l in range(m.n_dec):

@@ -51,6 +51,10 @@ int parse_blob(const void* blob, size_t n, ParsedBlob* out) {
   Config& c = out->cfg;
   c.dtype = f[1]; c.n_enc = f[2]; c.n_dec = f[3]; c.d = f[4]; c.H = f[5]; c.d_ff = f[6]; c.V = f[7];
   c.k_model = f[8]; c.d_hidden = f[9]; c.head_layout = f[10]; c.p1_identity = f[11]; c.eps = eps;
+  int32_t local[2];
+  memcpy(local, p + 88, sizeof(local));      // 1D local self-attention in the decoder: query block length, memory length
+  c.local_q = local[0]; c.local_m = local[1];
+  if (c.local_q < 0 || c.local_m < 0) return fail(BPD_E_FORMAT, "bad local-attention lengths %d/%d", c.local_q, c.local_m);
   if (c.dtype != 0 && c.dtype != 1) return fail(BPD_E_FORMAT, "unknown dtype %d", c.dtype);
   if (c.n_enc < 1 || c.n_dec < 1 || c.n_enc > 64 || c.n_dec > 64) return fail(BPD_E_FORMAT, "bad layer counts");
   if (c.d < 8 || c.d % 8 || c.H < 1 || c.d % c.H) return fail(BPD_E_FORMAT, "bad d_model/heads %d/%d", c.d, c.H);
@@ -377,7 +381,8 @@ static int run_pass(bpd_session* s, const PassArgs& a) {
     AttnParams ap;
     memset(&ap, 0, sizeof(ap));
     ap.q = s->qbuf; ap.ldq = d; ap.out = s->attn; ap.ldo = d; ap.rows = R; ap.rows_per_b = a.kcur;
-    ap.H = c.H; ap.dh = d / c.H; ap.causal = 1; ap.k = s->kcache[l]; ap.v = s->vcache[l]; ap.ldkv = d;
+    ap.H = c.H; ap.dh = d / c.H; ap.causal = 1; ap.local_q = c.local_q; ap.local_m = c.local_m;
+    ap.k = s->kcache[l]; ap.v = s->vcache[l]; ap.ldkv = d;
     ap.paged = 1; ap.st = s->st; ap.scale = 1.0f / sqrtf((float)ap.dh); ap.by_rows = (s->B >= 8) ? 1 : 0; ap.all_done = done;
     launch_attention<float, WT>(ap, st);
     ++g_launches;
@@ -555,6 +560,7 @@ static int run_layers_fused(bpd_session* s, const PassArgs& a) {
     ps.d = d; ps.H = c.H; ps.R = R; ps.rows_per_b = a.kcur; ps.eps = c.eps;
     ps.kcache = static_cast<bf16*>(s->kcache[l]); ps.vcache = static_cast<bf16*>(s->vcache[l]);
     ps.attn.rows = R; ps.attn.rows_per_b = a.kcur; ps.attn.H = c.H; ps.attn.dh = fused::kDH; ps.attn.causal = 1;
+    ps.attn.local_q = c.local_q; ps.attn.local_m = c.local_m;
     ps.attn.k = s->kcache[l]; ps.attn.v = s->vcache[l]; ps.attn.ldkv = d; ps.attn.paged = 1; ps.attn.st = s->st;
     ps.attn.scale = 1.0f / sqrtf((float)fused::kDH);
     ps.ws = s->fused_ws; ps.counters = s->fused_counters; ps.all_done = done;
@@ -622,7 +628,8 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
     AttnParams ap;
     memset(&ap, 0, sizeof(ap));
     ap.q = s->qbuf; ap.ldq = d; ap.out = s->attn; ap.ldo = d; ap.out_plane = s->pl_attn; ap.rows = R;
-    ap.rows_per_b = a.kcur; ap.H = c.H; ap.dh = d / c.H; ap.causal = 1; ap.k = s->kcache[l]; ap.v = s->vcache[l];
+    ap.rows_per_b = a.kcur; ap.H = c.H; ap.dh = d / c.H; ap.causal = 1; ap.local_q = c.local_q; ap.local_m = c.local_m;
+    ap.k = s->kcache[l]; ap.v = s->vcache[l];
     ap.ldkv = d; ap.paged = 1; ap.st = s->st; ap.scale = 1.0f / sqrtf((float)ap.dh); ap.by_rows = (s->B >= 8) ? 1 : 0; ap.all_done = done;
     PROF(kProfSelfAttn, launch_attention<float, bf16>(ap, st, pdl););
     ++g_launches;

@@ -399,8 +399,8 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
       const int b = token / p.rows_per_b, i = token % p.rows_per_b;
       const int limit = SELF ? (s_len[b] + i + 1) : s_len[b];
       float ov;
-      if (SELF) ov = attention_head<bf16, kDH, kWarps, true>(ap, b, h, limit, sm);
-      else ov = attention_head<float, kDH, kWarps, false>(ap, b, h, limit, sm);
+      if (SELF) ov = attention_head<bf16, kDH, kWarps, true>(ap, b, h, attn_first_key(ap, limit - 1), limit, sm);
+      else ov = attention_head<float, kDH, kWarps, false>(ap, b, h, 0, limit, sm);
       if (tid < kDH) {
         uint32_t hi, lo;
         split_bits(ov, hi, lo);

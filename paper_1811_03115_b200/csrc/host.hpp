@@ -46,6 +46,7 @@ inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
 
 struct Config {
   int dtype, n_enc, n_dec, d, H, d_ff, V, k_model, d_hidden, head_layout, p1_identity;
+  int local_q, local_m;    // decoder self-attention: 0 = all earlier positions; else 1D local attention
   float eps;
   int elem() const { return dtype == 0 ? 4 : 2; }
 };

@@ -335,6 +335,8 @@ struct AttnParams {
   int rows, rows_per_b, H, dh;
   int by_rows;                     // 1: one CTA per (sequence, head) instead of per (row, head)
   int causal;                      // 1: keys 0 .. len[b]+i ; 0: keys 0 .. limit_b[b]-1
+  int local_q, local_m;            // causal only, local_q > 0: 1D local attention -- a query at position t sees keys
+                                   // from (t / local_q) * local_q - local_m (not below 0) to t
   const int* limit_b;
   const void* k; const void* v;    // linear: row s of batch b at base + b*bstride + s*ldkv ; paged: page pool
   long long ldkv, bstride;
@@ -343,6 +345,12 @@ struct AttnParams {
   float scale;
   const int* all_done;
 };
+
+// First key a causal query at position pos may see (0 unless the model uses 1D local attention).
+__device__ __forceinline__ int attn_first_key(const AttnParams& p, int pos) {
+  if (!p.causal || p.local_q <= 0) return 0;
+  return max(0, (pos / p.local_q) * p.local_q - p.local_m);
+}
 
 // Keys are taken in chunks of 32 absolute positions, lane = key; running
 // max / sum are merged chunk by chunk in position order (fixed order).
@@ -359,6 +367,7 @@ __global__ void __launch_bounds__(128) attention_kernel(AttnParams p) {
   const int b = r / p.rows_per_b, i = r % p.rows_per_b;
   const int dh = p.dh;
   const int limit = p.causal ? (p.st.len[b] + i + 1) : p.limit_b[b];
+  const int first = attn_first_key(p, limit - 1);
   const QT* q = reinterpret_cast<const QT*>(p.q) + (long long)r * p.ldq + h * dh;
   for (int c = lane; c < dh; c += 32) qs[warp][c] = to_f(q[c]) * p.scale;
   __syncwarp();
@@ -371,10 +380,10 @@ __global__ void __launch_bounds__(128) attention_kernel(AttnParams p) {
   };
   float m_run = -INFINITY, l_run = 0.f;
   float acc[4] = {0.f, 0.f, 0.f, 0.f};   // output dims lane, lane+32, lane+64, lane+96
-  for (int c0 = 0; c0 < limit; c0 += 32) {
+  for (int c0 = first & ~31; c0 < limit; c0 += 32) {
     const int pos = c0 + lane;
     float s = -INFINITY;
-    if (pos < limit) {
+    if (pos >= first && pos < limit) {
       const CT* kr = K + row_off(pos);
       float dot = 0.f;
       for (int c = 0; c < dh; c += 8) {
@@ -387,7 +396,7 @@ __global__ void __launch_bounds__(128) attention_kernel(AttnParams p) {
     }
     const float m_new = fmaxf(m_run, warp_max(s));
     const float corr = expf(m_run - m_new);      // exp(-inf) = 0 on the first chunk
-    const float pj = (pos < limit) ? expf(s - m_new) : 0.f;
+    const float pj = (pos >= first && pos < limit) ? expf(s - m_new) : 0.f;
     l_run = l_run * corr + warp_sum(pj);
 #pragma unroll
     for (int t = 0; t < 4; ++t) acc[t] *= corr;
@@ -487,7 +496,7 @@ template <> __device__ __forceinline__ void load_n_cg<4>(const bf16* p, float (&
 // COHERENT: keys and values may have been written by other SMs earlier in the same launch, so they are read
 // from L2 rather than through L1.
 template <typename CT, int DH, int NW, bool COHERENT>
-__device__ __forceinline__ float attention_head(const AttnParams& p, int b, int h, int limit, AttnSmem<DH, NW>& sm) {
+__device__ __forceinline__ float attention_head(const AttnParams& p, int b, int h, int first, int limit, AttnSmem<DH, NW>& sm) {
   constexpr int DPL = (DH >= 32) ? DH / 32 : 1;       // output dims per lane (contiguous)
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const CT* K = reinterpret_cast<const CT*>(p.k);
@@ -500,8 +509,9 @@ __device__ __forceinline__ float attention_head(const AttnParams& p, int b, int 
   const int nchunks = (limit + 31) >> 5;
   const bool owns = (DH >= 32) || (lane < DH);
   const int dim0 = (DH >= 32) ? lane * DPL : lane;
-  for (int ch = warp; ch < nchunks; ch += NW) {
+  for (int ch = (first >> 5) + warp; ch < nchunks; ch += NW) {
     const int c0 = ch << 5;
+    const int lo = first - c0;                       // lanes below it hold keys before the first visible one
     // a 32-key chunk never straddles a 64-position page
     const size_t base = p.paged ? ((size_t)pt[c0 / kPage] * kPage + (c0 % kPage)) * p.ldkv + h * DH
                                 : (size_t)b * p.bstride + (size_t)c0 * p.ldkv + h * DH;
@@ -528,7 +538,7 @@ __device__ __forceinline__ float attention_head(const AttnParams& p, int b, int 
       }
     }
     float sc = -INFINITY;
-    if (lane < nk) {
+    if (lane >= lo && lane < nk) {
       float dot = 0.f;
 #pragma unroll
       for (int c = 0; c < DH; c += 8) {
@@ -539,7 +549,7 @@ __device__ __forceinline__ float attention_head(const AttnParams& p, int b, int 
     }
     const float m_new = fmaxf(m_run, warp_max(sc));
     const float corr = expf(m_run - m_new);
-    const float pj = (lane < nk) ? expf(sc - m_new) : 0.f;
+    const float pj = (lane >= lo && lane < nk) ? expf(sc - m_new) : 0.f;
     l_run = l_run * corr + warp_sum(pj);
 #pragma unroll
     for (int t = 0; t < DPL; ++t) acc[t] *= corr;
@@ -598,7 +608,7 @@ __device__ __forceinline__ void attention_item(const AttnParams& p, int item, At
   const QT* q = reinterpret_cast<const QT*>(p.q) + (long long)r * p.ldq + h * DH;
   if (threadIdx.x < DH) sm.q[threadIdx.x] = to_f(q[threadIdx.x]) * p.scale;
   __syncthreads();
-  const float ov = attention_head<CT, DH, NW, false>(p, b, h, limit, sm);
+  const float ov = attention_head<CT, DH, NW, false>(p, b, h, attn_first_key(p, limit - 1), limit, sm);
   if (threadIdx.x < DH) {
     const int c = threadIdx.x;
     if (p.out_plane) {
@@ -641,6 +651,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_rows_kernel(AttnPar
   for (int i = warp; i < p.rows_per_b; i += kAttnWarps) {
     const int r = b * p.rows_per_b + i;
     const int limit = p.causal ? (p.st.len[b] + i + 1) : p.limit_b[b];
+    const int first = attn_first_key(p, limit - 1);
     const QT* q = reinterpret_cast<const QT*>(p.q) + (long long)r * p.ldq + h * DH;
     __syncwarp();
     for (int c = lane; c < DH; c += 32) s_q[warp][c] = to_f(q[c]) * p.scale;
@@ -649,12 +660,13 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_rows_kernel(AttnPar
     float acc[DPL];
 #pragma unroll
     for (int t = 0; t < DPL; ++t) acc[t] = 0.f;
-    for (int c0 = 0; c0 < limit; c0 += 32) {
+    for (int c0 = first & ~31; c0 < limit; c0 += 32) {
       const size_t base = p.paged ? ((size_t)pt[c0 / kPage] * kPage + (c0 % kPage)) * p.ldkv + h * DH
                                   : (size_t)b * p.bstride + (size_t)c0 * p.ldkv + h * DH;
       const int nk = min(32, limit - c0);
+      const int lo = first - c0;
       float sc = -INFINITY;
-      if (lane < nk) {
+      if (lane >= lo && lane < nk) {
         const CT* kr = K + base + (size_t)lane * p.ldkv;
         float dot = 0.f;
 #pragma unroll
@@ -668,7 +680,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_rows_kernel(AttnPar
       }
       const float m_new = fmaxf(m_run, warp_max(sc));
       const float corr = expf(m_run - m_new);
-      const float pj = (lane < nk) ? expf(sc - m_new) : 0.f;
+      const float pj = (lane >= lo && lane < nk) ? expf(sc - m_new) : 0.f;
       l_run = l_run * corr + warp_sum(pj);
 #pragma unroll
       for (int t = 0; t < DPL; ++t) acc[t] *= corr;
@@ -727,6 +739,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_seq_kernel(AttnPara
   const int nrows = p.rows_per_b;
   const int base_limit = p.causal ? p.st.len[b] + 1 : p.limit_b[b];
   const int limit_max = p.causal ? base_limit + nrows - 1 : base_limit;
+  const int first_min = attn_first_key(p, base_limit - 1);   // the first row's window starts earliest
   for (int idx = threadIdx.x; idx < nrows * DH; idx += blockDim.x) {
     const int i = idx / DH, c = idx % DH;
     s_q[i][c] = to_f(reinterpret_cast<const QT*>(p.q)[(long long)(b * nrows + i) * p.ldq + h * DH + c]) * p.scale;
@@ -738,7 +751,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_seq_kernel(AttnPara
 #pragma unroll
     for (int t = 0; t < DPL; ++t) acc[r][t] = 0.f;
   }
-  for (int c0 = 0; c0 < limit_max; c0 += 32) {
+  for (int c0 = first_min & ~31; c0 < limit_max; c0 += 32) {
     const size_t base = p.paged ? ((size_t)pt[c0 / kPage] * kPage + (c0 % kPage)) * p.ldkv + h * DH
                                 : (size_t)b * p.bstride + (size_t)c0 * p.ldkv + h * DH;
     const int nk = min(32, limit_max - c0);
@@ -760,9 +773,10 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_seq_kernel(AttnPara
       if (i >= nrows) continue;                            // uniform over the warp
       const int limit = p.causal ? base_limit + i : base_limit;
       const int live = min(32, limit - c0);                // keys of this chunk the row may see
-      if (live <= 0) continue;
+      const int lo = attn_first_key(p, limit - 1) - c0;    // ... and lanes below lo hold keys before its window
+      if (live <= 0 || lo >= live) continue;
       float sc = -INFINITY;
-      if (lane < live) {
+      if (lane >= lo && lane < live) {
         float dot = 0.f;
 #pragma unroll
         for (int c = 0; c < DH; ++c) dot = fmaf(s_q[i][c], s_k[lane][c], dot);
@@ -770,7 +784,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_seq_kernel(AttnPara
       }
       const float m_new = fmaxf(m_run[r], warp_max(sc));
       const float corr = expf(m_run[r] - m_new);
-      const float pj = (lane < live) ? expf(sc - m_new) : 0.f;
+      const float pj = (lane >= lo && lane < live) ? expf(sc - m_new) : 0.f;
       l_run[r] = l_run[r] * corr + warp_sum(pj);
 #pragma unroll
       for (int t = 0; t < DPL; ++t) acc[r][t] *= corr;

@@ -283,6 +283,35 @@ def test_c5_super_resolution_shape(bpd):
     _full_size(bpd, "C5", iters=3, mean=5.0, free_iters=1)
 
 
+def test_c5_local_attention_deep_into_the_sequence(bpd):
+    """The super-resolution shape with 1D local attention (query blocks of 256, memory 256), followed in lock-step
+    with every proposal accepted until position 1100: by then the window starts at 768 and 24 chunks of 32 keys
+    lie outside it."""
+    from harness import lockstep
+    w = WORKLOADS["C5L"]
+    blob, model, src, src_len, om = _setup(bpd, w)
+    del blob
+    k, N = w.cfg.k_model, w.n_decode
+    s = bpd.Session(model, w.batch, w.max_src, N)
+    s.bpd_encode(src, src_len)
+    g_ids, _, _ = s.bpd_decode_greedy(N)
+    s.bpd_encode(src, src_len)
+    b_ids, _, _ = s.bpd_decode_blockwise(k, N)
+    assert np.array_equal(b_ids, g_ids)
+
+    def all_accepted(b, j, it):
+        return forced_tail(g_ids[b], min(j, N), k, k, 0, w.cfg.vocab)
+    rep = lockstep(s, om, src, src_len, k, N, max_iters=110, tail_fn=all_accepted)
+    assert sum(r[0] for r in rep.khats) == 1100 and rep.emitted[0] == list(g_ids[0][:1100])
+    wf = WORKLOADS["C5"]
+    model_f = bpd.Model(make_weights(wf.cfg, wf.weight_seed, wf.sigma))
+    sf = bpd.Session(model_f, 1, w.max_src, N)
+    sf.bpd_encode(src, src_len)
+    f_ids, _, _ = sf.bpd_decode_greedy(N)
+    assert np.array_equal(f_ids[0][:256], g_ids[0][:256]) and not np.array_equal(f_ids, g_ids)
+    sf.close(); model_f.close(); s.close(); model.close()
+
+
 def test_c4_batch32_ragged(bpd):
     w = WORKLOADS["C4"]
     _, src_len = make_source(w)
@@ -414,6 +443,54 @@ def test_fused_layers_agree_with_kernel_per_projection(bpd, w, monkeypatch):
     for (ha, la), (hb, lb) in zip(a_steps, b_steps):
         assert np.abs(ha - hb).max() <= 2e-3 and np.abs(la - lb).max() <= 2e-3
     model.close()
+
+
+# 1D local attention (query blocks of local_q positions + local_m positions of memory), one model per attention kernel
+_LOC = dict(local_q=8, local_m=20)
+LOCAL_MODELS = [
+    Workload("local-fused", ModelConfig(2, 2, 256, 4, 512, 1000, 4, 256, dtype=DTYPE_BF16, **_LOC), 0.05,
+             61, 62, 63, batch=1, src_lo=9, src_hi=9, n_decode=72),
+    Workload("local-split", ModelConfig(2, 2, 128, 2, 256, 1000, 4, 256, dtype=DTYPE_BF16, **_LOC), 0.05,
+             64, 65, 66, batch=2, src_lo=5, src_hi=9, n_decode=72),
+    Workload("local-generic", ModelConfig(1, 2, 96, 4, 200, 333, 3, 136, dtype=DTYPE_F32, local_q=5, local_m=9), 0.1,
+             67, 68, 69, batch=2, src_lo=2, src_hi=7, n_decode=48),
+    Workload("local-seq", ModelConfig(1, 2, 128, 2, 256, 500, 4, 128, dtype=DTYPE_BF16, **_LOC), 0.05,
+             70, 71, 72, batch=8, src_lo=3, src_hi=8, n_decode=44),
+    Workload("local-rows", ModelConfig(1, 2, 128, 1, 256, 500, 4, 128, dtype=DTYPE_BF16, **_LOC), 0.05,
+             73, 74, 75, batch=8, src_lo=3, src_hi=8, n_decode=44),
+]
+
+
+@pytest.mark.parametrize("w", LOCAL_MODELS, ids=lambda w: w.name)
+def test_local_attention_lockstep(bpd, w):
+    """Section 7.3's model class: decoder self-attention restricted to the query's block and a fixed memory
+    before it.  Every attention kernel (cluster path, split, generic, per-sequence, per-row) against the oracle,
+    decoding far enough that whole 32-key chunks fall out of the window."""
+    from harness import lockstep
+    blob, model, src, src_len, om = _setup(bpd, w)
+    assert om.local_q == w.cfg.local_q and om.local_m == w.cfg.local_m
+    k, N = w.cfg.k_model, w.n_decode
+    s = bpd.Session(model, w.batch, w.max_src, N)
+    s.bpd_encode(src, src_len)
+    g_ids, _, _ = s.bpd_decode_greedy(N)
+    s.bpd_encode(src, src_len)
+    b_ids, _, _ = s.bpd_decode_blockwise(k, N)
+    assert np.array_equal(b_ids, g_ids)
+    fn, sched = _tail_fn(w, g_ids, k, 3.0)
+    rows = sorted({0, w.batch - 1})
+    rep = lockstep(s, om, src, src_len, k, N, max_iters=N, tail_fn=fn, rows=rows)
+    for i, b in enumerate(rows):
+        assert rep.emitted[b] == list(g_ids[b])
+        assert [r[i] for r in rep.khats if r[i] > 0] == _expected_khats(sched[b], k, N)
+    # the window matters: the same weights with full attention decode differently
+    import dataclasses
+    w_full = dataclasses.replace(w, cfg=dataclasses.replace(w.cfg, local_q=0, local_m=0))
+    model_f = bpd.Model(make_weights(w_full.cfg, w.weight_seed, w.sigma))
+    sf = bpd.Session(model_f, w.batch, w.max_src, N)
+    sf.bpd_encode(src, src_len)
+    f_ids, _, _ = sf.bpd_decode_greedy(N)
+    assert not np.array_equal(f_ids, g_ids)
+    sf.close(); model_f.close(); s.close(); model.close()
 
 
 

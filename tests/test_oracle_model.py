@@ -240,3 +240,64 @@ def test_dense_with_block_structure_equals_blockdiag_layout():
     np.testing.assert_allclose(head_logits(md, h, k), head_logits(mb, h, k), atol=1e-12)
     # fewer heads than the model carries: the first k of them
     np.testing.assert_allclose(head_logits(md, h, 2), head_logits(md, h, k)[:, :2], atol=0)
+
+
+# ---------------------------------------------------------------- 1D local attention (Section 7.3's model class)
+
+def test_local_attention_window_by_enumeration():
+    """The visible keys of a query, enumerated from the definition for every (query block, memory) pair and
+    every position: its own block up to itself plus local_m positions before the block's first one."""
+    from dataclasses import replace
+    from oracle.model import self_attention_allowed
+    base = _model()
+    for q_len in (1, 2, 3, 5, 8):
+        for mem in (0, 1, 4, 7):
+            m = replace(base, local_q=q_len, local_m=mem)
+            ok = self_attention_allowed(m, np.arange(20), 20)
+            for t in range(20):
+                block_start = (t // q_len) * q_len
+                want = [j for j in range(20) if block_start - mem <= j <= t]
+                assert list(np.nonzero(ok[t])[0]) == want
+    full = self_attention_allowed(base, np.arange(9), 9)
+    assert np.array_equal(full, np.tril(np.ones((9, 9), dtype=bool)))
+
+
+def test_local_attention_special_cases_and_cache():
+    """(i) memory at least as long as the sequence: identical to full causal attention; (ii) blocks of one
+    position without memory: every query sees only itself, softmax over one key is 1, so a decoder layer's
+    self-attention returns the value row and positions stop influencing each other; (iii) the cached decoder
+    (blocks, rejections) equals the uncached one under local attention."""
+    from dataclasses import replace
+    base = _model()
+    rng = np.random.default_rng(5)
+    src = rng.integers(2, base.V, size=6)
+    memory = encode(base, src, 6)
+    toks = [0] + [int(t) for t in rng.integers(2, base.V, size=11)]
+    full = decoder_full(base, memory, 6, toks)
+    wide = replace(base, local_q=3, local_m=64)
+    np.testing.assert_array_equal(decoder_full(wide, memory, 6, toks), full)
+    alone = replace(base, local_q=1, local_m=0)
+    h_alone = decoder_full(alone, memory, 6, toks)
+    for t in (0, 4, 11):           # a position computed with nothing before it, at its own position: same row
+        solo = replace(base, local_q=1, local_m=0)
+        other = list(toks)
+        for j in range(t):
+            other[j] = 2 + (other[j] + 7) % (base.V - 2)     # change every earlier token
+        np.testing.assert_array_equal(decoder_full(solo, memory, 6, other)[t], h_alone[t])
+    assert not np.allclose(h_alone, full)
+    loc = replace(base, local_q=4, local_m=3)
+    want = decoder_full(loc, memory, 6, toks)
+    assert not np.allclose(want[8:], full[8:])
+    cache = DecoderCache(loc, memory, 6, capacity=32)
+    got = np.zeros_like(want)
+    pos = 0
+    for n, acc in ((1, 1), (4, 2), (3, 3), (4, 1), (5, 5)):
+        n = min(n, len(toks) - pos)
+        h = cache.extend(toks[pos:pos + n])
+        got[pos:pos + n] = h
+        acc = min(acc, n)
+        cache.commit(acc)
+        pos += acc
+        if pos >= len(toks):
+            break
+    np.testing.assert_allclose(got[:pos], want[:pos], rtol=0, atol=1e-12)
