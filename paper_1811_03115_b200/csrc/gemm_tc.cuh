@@ -212,7 +212,7 @@ __device__ __forceinline__ void split_bf16(float v, bf16& hi, bf16& lo) {
 
 // Shared-memory footprint of one CTA.
 __host__ __device__ inline size_t stage_bytes(int bn) { return (size_t)kBM * 128 + 2 * (size_t)bn * 128; }
-__host__ __device__ inline int stages_for(int bn) { return bn <= 32 ? 4 : (bn <= 64 ? 3 : 4); }
+__host__ __device__ inline int stages_for(int bn) { return bn <= 16 ? 5 : (bn <= 32 ? 4 : (bn <= 64 ? 3 : 4)); }
 __host__ __device__ inline size_t smem_bytes(int bn) { return stages_for(bn) * stage_bytes(bn) + 1024 /*alignment*/ + 256; }
 
 // ---------------------------------------------------------------- final epilogue for one (feature, token)
