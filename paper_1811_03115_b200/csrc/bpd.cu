@@ -190,6 +190,7 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
     for (int kh = 1; kh <= km; ++kh) {
       need(kh * fh, dd, Rmax, 1); need(km * fh, dd, Rmax, 1);
       need(kh * dd, km * fh, Rmax, 1);
+      if (wide) ws = std::max(ws, tc::ws_floats(kh * dd, km * fh, B, 1, 1, tc::kSlots));   // stage 2 of the lazy heads
       need(dd, fh, Rmax, kh);
     }
     need(c.V, dd, R2, 1);
@@ -671,15 +672,21 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   BPD_TRY(tc::launch<tc::kTcPlanes>(with_w(xn, m->head_w1, km * fhd), hid, d, R, pu, sc, st, 1, 0, 0, pdl, km * fhd)); ++g_launches;
   prof_mark(s, kProfHeadW1, 1);
   // output layers + shared vocabulary projection with a fused top-1 for T rows and kh heads
+  // Sessions that evaluate the heads lazily never use head 1 of a launch over all heads, so there the output
+  // layers of head 1 alone (greedy passes, stage 1) are planned for their own size, and stage 2 (plan_tt = 1:
+  // one token tile) for its own; everywhere else every launch is planned for the full matrix, so that head 1
+  // is the same sum whether it is evaluated alone or with the others.
+  const bool own_plan = s->lazy_heads != 0 && tc_scratch(s).wide_ttiles > 0;
   auto heads = [&](const void* u_planes, long long u_plane, int u_rows, const float* hres, int T, int kh, int* table_out,
-                   bool rank, float* logits) -> int {
+                   bool rank, float* logits, int plan_tt) -> int {
     prof_mark(s, kProfHeadW2, 0);
     tc::Operands uo{m->head_w2, km * d, u_planes, u_plane, ldu, u_rows, ldu};
     tc::TcParams ph = tc_params(m->head_b2, 0, done);
     ph.out_hi = static_cast<bf16*>(s->o); ph.plane = s->pl_o; ph.ldo = (long long)kh * d;
     ph.h = hres; ph.d = d; ph.head_identity = c.p1_identity;
     if (c.head_layout == 0) {
-      BPD_TRY(tc::launch<tc::kTcHeadOut>(uo, kh * d, km * fhd, T, ph, sc, st, 1, 0, 0, pdl, km * d));
+      BPD_TRY(tc::launch<tc::kTcHeadOut>(uo, kh * d, km * fhd, T, ph, sc, st, 1, 0, 0, pdl, own_plan ? kh * d : km * d,
+                                         own_plan ? plan_tt : 0));
     } else {
       ph.zofs_n = d;
       BPD_TRY(tc::launch<tc::kTcHeadOut>(uo, d, fhd, T, ph, sc, st, kh, d, fhd, pdl));
@@ -703,7 +710,7 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   const bool lazy = pass_is_lazy(s, a);
   if (lazy) {
     // stage 1: p_1 at every block position, verification and commit
-    BPD_TRY(heads(s->u, s->pl_u, s->rows_dec, s->h_f32, R, 1, s->st.table, wants_rank(a), nullptr));
+    BPD_TRY(heads(s->u, s->pl_u, s->rows_dec, s->h_f32, R, 1, s->st.table, wants_rank(a), nullptr, 0));
     PassArgs a1 = a;
     a1.kh = 1; a1.knext = 1;
     VerifyParams v1 = verify_params(s, a1);
@@ -714,7 +721,7 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
                     s->st, s->B, a.kcur, done};
     launch_k(gather_selected_kernel, dim3(s->B), dim3(256), 0, st, pdl, gp);
     ++g_launches;
-    BPD_TRY(heads(s->u2, s->pl_u2, s->B, s->h2, s->B, a.kh, s->table2, false, nullptr));
+    BPD_TRY(heads(s->u2, s->pl_u2, s->B, s->h2, s->B, a.kh, s->table2, false, nullptr, 1));
     SelectParams sp{s->st, s->st.table, s->table2, s->table_full, s->B, a.kcur, a.kh, a.knext, done};
     launch_k(select_next_kernel, dim3(1), dim3(32 * ceil_div(s->B, 32)), 0, st, pdl, sp);
     ++g_launches;
@@ -722,7 +729,7 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
     s->invocations += 1;
     return BPD_OK;
   }
-  BPD_TRY(heads(s->u, s->pl_u, s->rows_dec, s->h_f32, R, a.kh, s->st.table, wants_rank(a), a.logits_dump));
+  BPD_TRY(heads(s->u, s->pl_u, s->rows_dec, s->h_f32, R, a.kh, s->st.table, wants_rank(a), a.logits_dump, 0));
   VerifyParams vp = verify_params(s, a);
   PROF(kProfVerify, launch_k(verify_commit_kernel, dim3(1), dim3(32 * ceil_div(s->B, 32)), 0, st, pdl, vp););
   ++g_launches;

@@ -23,30 +23,43 @@ struct Plan {
 // Depends on (N, K) only -- never on the number of tokens -- so that a position
 // scored alone and the same position scored inside a block add up in the same order.
 // wide_ttiles: 0 for sessions whose passes carry few rows (one token tile, two CTAs per SM, split K finely);
-// otherwise the number of token tiles of the session's widest pass: those launches already have tiles x
-// token tiles CTAs of 128 tokens each (one per SM), so K is split only as far as that leaves SMs idle.
-// It is a property of the session, so greedy and blockwise passes of one session still agree.
-inline Plan plan_splits(int N, int K, int wide_ttiles = 0) {
+// otherwise the number of token tiles the split is planned for (the session's widest pass, unless the launch
+// says otherwise): those launches already have tiles x token tiles CTAs, so K is split only as far as that
+// leaves of the `slots` CTA slots idle.  Both are properties of the session and of the matrix, so greedy and
+// blockwise passes of one session still agree.
+inline Plan plan_splits(int N, int K, int wide_ttiles = 0, int slots = kSlots / 2) {
   Plan pl;
   pl.tiles = (N + kBM - 1) / kBM;
   pl.chunks = (K + kBK - 1) / kBK;
   int splits;
-  if (wide_ttiles > 0) splits = std::max(1, std::min(pl.chunks / 8, (kSlots / 2) / (pl.tiles * wide_ttiles)));
+  if (wide_ttiles > 0) splits = std::max(1, std::min(pl.chunks / 8, slots / (pl.tiles * wide_ttiles)));
   else splits = std::max(1, std::min(pl.chunks / kMinChunksPerSplit, kSlots / pl.tiles));
   pl.chunks_per_split = (pl.chunks + splits - 1) / splits;
   pl.splits = (pl.chunks + pl.chunks_per_split - 1) / pl.chunks_per_split;
   return pl;
 }
+inline int token_bn(int T, int ttiles);
 // Token tiling of a launch: as few tiles of at most 128 tokens as possible, but -- in sessions with many rows --
-// more, narrower ones (not below 32 tokens) while the launch would otherwise leave SMs without a CTA.  The tile
-// width only changes the MMA's N; every output element is still the same sum in the same order.
+// the tiling (tiles of 32 to 128 tokens) that leaves the busiest SM the fewest bytes to stage: with
+// `ctas_per_ttile` CTAs per token tile, a CTA stages 16 KB of weights and bn / 4 KB of activation planes per
+// K chunk, and the busiest SM runs ceil(CTAs / 148) of them.  Ties go to the finer tiling (more loads in
+// flight).  The tile width only changes the MMA's N; every output element is still the same sum in the same order.
 inline int token_tiles(int T, int ctas_per_ttile = 0) {
-  int tt = (T + kMaxBN - 1) / kMaxBN;
+  int tt = std::max(1, (T + kMaxBN - 1) / kMaxBN);
   if (ctas_per_ttile > 0) {
-    const int want = (kSlots / 2 + ctas_per_ttile - 1) / ctas_per_ttile;
-    tt = std::max(tt, std::min(want, (T + 31) / 32));
+    const int hi = std::max(tt, (T + 31) / 32);
+    long best_cost = -1;
+    int best_tt = tt;
+    for (int cand = tt; cand <= hi; ++cand) {
+      const int bn = token_bn(T, cand);
+      if ((long)(cand - 1) * bn >= T) continue;                   // its last tile would be empty
+      const long per_sm = ((long)ctas_per_ttile * cand + 147) / 148;
+      const long cost = per_sm * (64 + bn);                       // quarter KB per K chunk
+      if (best_cost < 0 || cost <= best_cost) { best_cost = cost; best_tt = cand; }
+    }
+    tt = best_tt;
   }
-  return std::max(1, tt);
+  return tt;
 }
 inline int token_bn(int T, int ttiles) {
   const int per = (T + ttiles - 1) / ttiles;
@@ -55,8 +68,8 @@ inline int token_bn(int T, int ttiles) {
 inline int token_bn(int T) { return token_bn(T, token_tiles(T)); }
 inline int max_token_tiles(int T) { return std::max(token_tiles(T), (T + 31) / 32); }
 // fp32 elements of split-K workspace a launch with these sizes needs.
-inline size_t ws_floats(int N, int K, int T, int zslices, int wide_ttiles = 0) {
-  const Plan pl = plan_splits(N, K, wide_ttiles);
+inline size_t ws_floats(int N, int K, int T, int zslices, int wide_ttiles = 0, int slots = kSlots / 2) {
+  const Plan pl = plan_splits(N, K, wide_ttiles, slots);
   if (pl.splits == 1) return 0;
   // upper bound over every token tiling the launch may pick: tiles * bn <= T + 16 per tile
   return (size_t)zslices * pl.tiles * pl.splits * ((size_t)T + 16 * max_token_tiles(T)) * kBM;
@@ -131,7 +144,7 @@ struct Operands {
 
 template <int EPI>
 int launch(const Operands& op, int N, int K, int T, TcParams p, const Scratch& sc, cudaStream_t st, int zslices = 1,
-           int a_rows_per_slice = 0, int b_cols_per_slice = 0, bool pdl = false, int plan_n = 0) {
+           int a_rows_per_slice = 0, int b_cols_per_slice = 0, bool pdl = false, int plan_n = 0, int plan_tt = 0) {
   static bool attr_set = false;
   if (!attr_set) {
     BPD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)std::max(smem_bytes(kMaxBN), smem_bytes(64))));
@@ -139,7 +152,10 @@ int launch(const Operands& op, int N, int K, int T, TcParams p, const Scratch& s
   }
   // plan_n: the feature count the K split is planned for.  A launch that computes only the first features of a
   // matrix (fewer heads) passes the full count so that every feature is summed in the same order either way.
-  Plan pl = plan_splits(plan_n > 0 ? plan_n : N, K, sc.wide_ttiles);
+  // plan_tt: in a session with many rows, a launch whose results need not agree bit for bit with any other
+  // launch (the second stage of the lazy heads) plans its K split for its own token tiles and for two CTAs per SM.
+  Plan pl = (sc.wide_ttiles && plan_tt > 0) ? plan_splits(plan_n > 0 ? plan_n : N, K, plan_tt, kSlots)
+                                            : plan_splits(plan_n > 0 ? plan_n : N, K, sc.wide_ttiles);
   pl.tiles = (N + kBM - 1) / kBM;
   const int ttiles = token_tiles(T, sc.wide_ttiles ? pl.tiles * pl.splits * zslices : 0), bn = token_bn(T, ttiles);
   const size_t need_ws = pl.splits == 1 ? 0 : (size_t)ttiles * zslices * pl.tiles * pl.splits * bn * kBM;
