@@ -298,11 +298,14 @@ static __global__ void wait_probe_kernel(int* error, unsigned long long limit_cy
   }
 }
 
+// Top-1 epilogue: threads that share a token (a power of two, at most 8, with tpt * bn <= 128).
+__host__ __device__ inline int topk_threads_per_token(int bn) { return bn <= 16 ? 8 : (bn <= 32 ? 4 : (bn <= 64 ? 2 : 1)); }
+
 // ---------------------------------------------------------------- epilogue of one (tile, split) unit
 // Shared by the one-shot projection kernel and the persistent layer kernel.  Called by the four epilogue warps
 // (128 threads, named barrier 1).
 struct EpiShared {
-  float (*s_val)[kMaxBN]; int (*s_idx)[kMaxBN];
+  float* s_t;                   // top-1: the tile transposed, [token][128 features], rows of topk_stride() floats
   float* s_mean; float* s_rstd;
   unsigned long long* s_slot;
   volatile uint32_t* ctl;       // [1] reduces the tile, [2] merges the top-1, [3] accumulator arrived
@@ -314,8 +317,7 @@ struct EpiUnit {
 };
 template <int EPI>
 __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& sh, const EpiUnit& u, int warp, int lane) {
-  float (*s_val)[kMaxBN] = sh.s_val;
-  int (*s_idx)[kMaxBN] = sh.s_idx;
+  float* s_t = sh.s_t;
   float* s_mean = sh.s_mean;
   float* s_rstd = sh.s_rstd;
   unsigned long long* s_slot = sh.s_slot;
@@ -327,6 +329,7 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
   const int row = q * 32 + lane;
   const int n = tile * kBM + row;                  // feature index within the slice
   const int et = threadIdx.x - 64;                 // 0..127
+  const int tpt = topk_threads_per_token(bn), tstride = kBM + tpt;   // row stride = tpt mod 32: conflict-free scans
   if (EPI == kTcQkv && !skip && et < nt) {
     const int t = t0 + et;
     const int b = t / p.rows_per_b, i = t % p.rows_per_b;
@@ -389,12 +392,10 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
         } else {
 #pragma unroll
           for (int c = 0; c < 16; ++c) {
-            float x = (n < p.N) ? v[c] : -INFINITY;
-            int ix = (n < p.N) ? n : 0x7fffffff;
+            const float x = (n < p.N) ? v[c] : -INFINITY;
             if (p.logits && cb + c < nt && n < p.N) p.logits[(size_t)(t0 + cb + c) * p.N + n] = x;
             if (cb + c < nt) count_beats(p, t0 + cb + c, n, x, lane);
-            warp_argmax_lanes(x, ix);
-            if (lane == 0) { s_val[q][cb + c] = x; s_idx[q][cb + c] = ix; }
+            s_t[(cb + c) * tstride + row] = x;
           }
         }
       }
@@ -442,12 +443,10 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
               if (cg + c >= nt) break;
-              float x = (n < p.N) ? acc[c] : -INFINITY;
-              int ix = (n < p.N) ? n : 0x7fffffff;
+              const float x = (n < p.N) ? acc[c] : -INFINITY;
               if (p.logits && n < p.N) p.logits[(size_t)(t0 + cg + c) * p.N + n] = x;
               count_beats(p, t0 + cg + c, n, x, lane);
-              warp_argmax_lanes(x, ix);
-              if (lane == 0) { s_val[q][cg + c] = x; s_idx[q][cg + c] = ix; }
+              s_t[(cg + c) * tstride + row] = x;
             }
           }
         }
@@ -455,17 +454,34 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
       }
     }
     if (EPI == kTcArgmax && (direct || ctl[1])) {
-      // tile-level (value, index) per token, then the CTA that completes the last tile merges all tiles
+      // The tile sits in shared memory with one row per token.  tpt threads share a token: each scans every
+      // tpt-th feature in ascending order (a strict comparison keeps the lowest index among equals), then the
+      // tpt partial results are merged with the same ordering.  No shuffle per token, no work for absent tokens.
+      // Then the CTA that completes the last tile merges all tiles.
       asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (et < nt) {
-        float x = s_val[0][et];
-        int ix = s_idx[0][et];
-#pragma unroll
-        for (int w = 1; w < 4; ++w)
-          if (better(s_val[w][et], s_idx[w][et], x, ix)) { x = s_val[w][et]; ix = s_idx[w][et]; }
+      {
+        const int token = et / tpt, part = et % tpt;            // tokens >= bn do not occur: tpt * bn <= 128
+        const float* rowp = s_t + token * tstride;
+        float x = -INFINITY;
+        int ix = 0x7fffffff;
+        if (token < nt) {
+          x = rowp[part];
+          ix = part;
+#pragma unroll 8
+          for (int f = part + tpt; f < kBM; f += tpt) {
+            const float y = rowp[f];
+            if (y > x) { x = y; ix = f; }
+          }
+          ix = (tile * kBM + ix < p.N) ? tile * kBM + ix : 0x7fffffff;
+        }
+        for (int o = 1; o < tpt; o <<= 1) {                     // partners are neighbouring lanes of one warp
+          const float ov = __shfl_xor_sync(0xffffffffu, x, o);
+          const int oi = __shfl_xor_sync(0xffffffffu, ix, o);
+          if (better(ov, oi, x, ix)) { x = ov; ix = oi; }
+        }
         // one 64-bit atomic max per (tile, token): larger value wins, equal values go to the lower index;
         // max is order independent, so the result does not depend on which tile arrives first
-        atomicMax(&p.best[t0 + et], pack_best(x, ix));
+        if (token < nt && part == 0) atomicMax(&p.best[t0 + token], pack_best(x, ix));
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");
       if (et == 0) {
@@ -505,8 +521,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   volatile uint32_t* ctl = reinterpret_cast<volatile uint32_t*>(gen_base + kStages * stage_sz + 128);
   // ctl[0] = tensor-memory base, ctl[1] = "this CTA reduces the tile", ctl[2] = "this CTA merges the top-1",
   // ctl[3] = "the accumulator arrived"
-  __shared__ float s_val[4][kMaxBN];
-  __shared__ int s_idx[4][kMaxBN];
   __shared__ float s_mean[16], s_rstd[16];
   __shared__ unsigned long long s_slot[kMaxBN];   // kTcQkv: cache slot (element offset) of every token of the tile
 
@@ -602,7 +616,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else if (warp >= 2) {
     // ---------------- epilogue: thread = one feature row, registers = tokens
     pdl_wait();
-    const EpiShared sh{s_val, s_idx, s_mean, s_rstd, s_slot, ctl};
+    // the stages are free once the accumulator is complete: the top-1 epilogue transposes the tile into them
+    const EpiShared sh{reinterpret_cast<float*>(gen_base), s_mean, s_rstd, s_slot, ctl};
     const EpiUnit u{tmem, bars + 8 * 2 * kStages, 0u, tile, split, slice, (int)blockIdx.z, (int)gridDim.x,
                     (int)gridDim.z / zslices, t0, nt, bn, nchunks, p.all_done && *p.all_done};
     tc_epilogue<EPI>(p, sh, u, warp, lane);
