@@ -198,7 +198,7 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
   float* tc_ws = a.take<float>(ws);
   unsigned* tc_counters = a.take<unsigned>(ncnt);
   unsigned* tc_done = a.take<unsigned>(1);
-  unsigned long long* tc_best = a.take<unsigned long long>(R2);
+  unsigned long long* tc_best = a.take<unsigned long long>(R2 * tc::kBestStride);
   // fused decoder layers (few rows per pass): per-head / per-cluster shares of the output projections, slice counters
   const bool fused_ok = c.dtype == 1 && fused::supported(c.d, c.H, c.d_ff, (int)Rmax);
   const size_t fused_parts = std::max<size_t>(c.H, c.d_ff / (fused::kC * fused::kHS));
@@ -1237,7 +1237,7 @@ static OpScratch op_scratch_layout(int rows, int in_f, int out_f) {
   o.ws_off = take(o.ws_floats * sizeof(float));
   o.cnt_off = take(o.n_counters * sizeof(unsigned));
   o.done_off = take(sizeof(unsigned));
-  o.pv_off = take(o.part_elems * sizeof(unsigned long long));
+  o.pv_off = take(o.part_elems * tc::kBestStride * sizeof(unsigned long long));
   o.pi_off = o.pv_off;
   o.err_off = take(sizeof(int));
   o.total = off;

@@ -25,6 +25,9 @@ constexpr int kBK = 64;           // K elements per pipeline stage (128 bytes of
 constexpr int kMaxStages = 4;     // pipeline depth is chosen per launch (2..4) so that two CTAs fit on an SM when possible
 constexpr int kThreads = 192;     // warp 0: TMA, warp 1: MMA + tensor-memory allocation, warps 2-5: epilogue
 constexpr int kMaxBN = 128;       // tokens per CTA (MMA N), a multiple of 16
+// Words between the top-1 keys of successive tokens: every key has a 128-byte line of its own.  Hundreds of
+// tiles send one atomic max per token; keys that share a line queue behind one another in L2.
+constexpr int kBestStride = 16;
 constexpr unsigned long long kSpinCycles = 2000000000ull;   // about a second
 
 enum TcEpilogue {
@@ -55,7 +58,8 @@ struct TcParams {
   float* ws;                   // [z][tile][split][bn][128]
   unsigned* tile_counters;     // [z][tiles]
   // top-1
-  unsigned long long* best;         // [T] packed (orderable value, ~index), zero between launches
+  unsigned long long* best;         // [T][kBestStride] packed (orderable value, ~index) in the first word of each
+                                    // token's 128 bytes, zero between launches
   unsigned* done_counter;           // [1]
   int* out_idx; float* out_val; float* logits;
   RankState rank; int rank_kh;      // top-n acceptance: count entries beating each proposal (rank.cnt null = off)
@@ -330,6 +334,8 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
   const int n = tile * kBM + row;                  // feature index within the slice
   const int et = threadIdx.x - 64;                 // 0..127
   const int tpt = topk_threads_per_token(bn), tstride = kBM + tpt;   // row stride = tpt mod 32: conflict-free scans
+  // the debug dump of the logits and the rank counting of top-n acceptance are rare: kept out of the common loops
+  const bool extras = (EPI == kTcArgmax) && (p.logits != nullptr || p.rank.cnt != nullptr);
   if (EPI == kTcQkv && !skip && et < nt) {
     const int t = t0 + et;
     const int b = t / p.rows_per_b, i = t % p.rows_per_b;
@@ -391,11 +397,13 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
           }
         } else {
 #pragma unroll
-          for (int c = 0; c < 16; ++c) {
-            const float x = (n < p.N) ? v[c] : -INFINITY;
-            if (p.logits && cb + c < nt && n < p.N) p.logits[(size_t)(t0 + cb + c) * p.N + n] = x;
-            if (cb + c < nt) count_beats(p, t0 + cb + c, n, x, lane);
-            s_t[(cb + c) * tstride + row] = x;
+          for (int c = 0; c < 16; ++c) s_t[(cb + c) * tstride + row] = (n < p.N) ? v[c] : -INFINITY;
+          if (extras) {
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+              if (p.logits && cb + c < nt && n < p.N) p.logits[(size_t)(t0 + cb + c) * p.N + n] = v[c];
+              if (cb + c < nt) count_beats(p, t0 + cb + c, n, (n < p.N) ? v[c] : -INFINITY, lane);
+            }
           }
         }
       }
@@ -441,12 +449,15 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
             if (n < p.N) tc_store8<EPI>(p, slice, t0 + cg, min(8, nt - cg), n, acc, s_mean, s_rstd, cg, s_slot);
           } else {
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-              if (cg + c >= nt) break;
-              const float x = (n < p.N) ? acc[c] : -INFINITY;
-              if (p.logits && n < p.N) p.logits[(size_t)(t0 + cg + c) * p.N + n] = x;
-              count_beats(p, t0 + cg + c, n, x, lane);
-              s_t[(cg + c) * tstride + row] = x;
+            for (int c = 0; c < 8; ++c)
+              if (cg + c < nt) s_t[(cg + c) * tstride + row] = (n < p.N) ? acc[c] : -INFINITY;
+            if (extras) {
+#pragma unroll
+              for (int c = 0; c < 8; ++c) {
+                if (cg + c >= nt) break;
+                if (p.logits && n < p.N) p.logits[(size_t)(t0 + cg + c) * p.N + n] = acc[c];
+                count_beats(p, t0 + cg + c, n, (n < p.N) ? acc[c] : -INFINITY, lane);
+              }
             }
           }
         }
@@ -465,13 +476,23 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
         float x = -INFINITY;
         int ix = 0x7fffffff;
         if (token < nt) {
-          x = rowp[part];
-          ix = part;
-#pragma unroll 8
-          for (int f = part + tpt; f < kBM; f += tpt) {
-            const float y = rowp[f];
-            if (y > x) { x = y; ix = f; }
+          // four independent running maxima (features part + tpt * (4j + a)), merged by (value, lower index)
+          float xa[4];
+          int ia[4];
+#pragma unroll
+          for (int a = 0; a < 4; ++a) { ia[a] = part + tpt * a; xa[a] = rowp[ia[a]]; }
+          for (int f = part + 4 * tpt; f < kBM; f += 4 * tpt) {
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+              const float y = rowp[f + tpt * a];
+              if (y > xa[a]) { xa[a] = y; ia[a] = f + tpt * a; }
+            }
           }
+          x = xa[0];
+          ix = ia[0];
+#pragma unroll
+          for (int a = 1; a < 4; ++a)
+            if (better(xa[a], ia[a], x, ix)) { x = xa[a]; ix = ia[a]; }
           ix = (tile * kBM + ix < p.N) ? tile * kBM + ix : 0x7fffffff;
         }
         for (int o = 1; o < tpt; o <<= 1) {                     // partners are neighbouring lanes of one warp
@@ -481,7 +502,7 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
         }
         // one 64-bit atomic max per (tile, token): larger value wins, equal values go to the lower index;
         // max is order independent, so the result does not depend on which tile arrives first
-        if (token < nt && part == 0) atomicMax(&p.best[t0 + token], pack_best(x, ix));
+        if (token < nt && part == 0) atomicMax(&p.best[(size_t)(t0 + token) * kBestStride], pack_best(x, ix));
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");
       if (et == 0) {
@@ -491,10 +512,10 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
       asm volatile("bar.sync 1, 128;" ::: "memory");
       if (ctl[2]) {
         for (int t = et; t < p.T; t += 128) {
-          const unsigned long long key = __ldcg(&p.best[t]);
+          const unsigned long long key = __ldcg(&p.best[(size_t)t * kBestStride]);
           p.out_idx[t] = (int)(0xffffffffu - (unsigned)(key & 0xffffffffull));
           if (p.out_val) p.out_val[t] = unpack_value(key);
-          p.best[t] = 0ull;                       // ready for the next launch
+          p.best[(size_t)t * kBestStride] = 0ull;                       // ready for the next launch
         }
         if (et == 0) *p.done_counter = 0;
       }
