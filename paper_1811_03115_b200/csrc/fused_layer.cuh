@@ -40,6 +40,7 @@ constexpr int kWarps = 8;
 constexpr int kDH = 64;          // head width this path is built for
 constexpr int kHS = 16;          // hidden units per CTA in the feed-forward block
 constexpr int kMaxRows = 16;
+constexpr int kPartial = kDH + 2;   // a partial attention state: weighted value sum [kDH], running maximum, weight sum
 
 // Byte offset of (row, byte) in a shared-memory matrix with rb bytes per row (a multiple of 64).  When rb is a
 // multiple of 128 the two 64-byte halves of every 128 bytes trade places in odd rows, so that the 16-byte
@@ -218,6 +219,109 @@ __device__ __forceinline__ void merge_slice(float* x, const float* ws, const bf1
   }
 }
 
+// ------------------------------------------------------------------ self-attention over the paged cache
+// Keys are taken in chunks of 32 absolute positions.  Chunk ch belongs to rank ch % kC and, there, to lump
+// (ch / kC) % 8.  A lump's chunks are folded in position order into one state per query row (running maximum,
+// weight sum, weighted values), the eight lumps of a rank are merged in lump order, the ranks in rank order.
+// The grouping depends on key positions only, so a row's result depends neither on the other rows of the pass
+// nor on which CTA or warp did the arithmetic: the two schedules below (one CTA per row while every rank has at
+// most one chunk; keys shared by all rows of a sequence otherwise) give the same bits.
+
+// One chunk: the 32 key rows and the 32 value rows, 128 contiguous bytes per row and load.  For the keys a lane
+// holds 16 bytes (dimensions 8 seg .. 8 seg + 7, seg = lane % 8) of rows 4 u + lane / 8, u = 0..7; for the
+// values its two output dimensions of every row.  Rows beyond the chunk's last repeat it (their weight is 0).
+// Every load is in flight before the first is used; they go to L2 (other SMs wrote the newest rows in this launch).
+__device__ __forceinline__ void chunk_fetch(const bf16* Kc, const bf16* Vc, size_t base, int nk, long long ldkv, int lane,
+                                            uint4 (&kq)[8], uint32_t (&vq)[32]) {
+  const int grp = lane >> 3, seg = lane & 7;
+#pragma unroll
+  for (int u = 0; u < 8; ++u)
+    kq[u] = __ldcg(reinterpret_cast<const uint4*>(Kc + base + (size_t)min(4 * u + grp, nk - 1) * ldkv) + seg);
+#pragma unroll
+  for (int j = 0; j < 32; ++j)
+    vq[j] = __ldcg(reinterpret_cast<const uint32_t*>(Vc + base + (size_t)min(j, nk - 1) * ldkv) + lane);
+}
+
+// Folds a chunk into the state of one query row (q_row: kDH scaled floats in shared memory; state: kPartial
+// floats in shared memory that only this warp touches; vis: may this lane's key be seen by the row).
+__device__ __forceinline__ void chunk_fold(const uint4 (&kq)[8], const uint32_t (&vq)[32], const float* q_row, bool vis,
+                                           float* state, int lane) {
+  const int seg = lane & 7;
+  const float4* qr = reinterpret_cast<const float4*>(q_row);
+  const float4 qa = qr[2 * seg], qb = qr[2 * seg + 1];
+  // this lane's share (8 dimensions) of the scores of keys 4 u + lane / 8
+  float v[8];
+#pragma unroll
+  for (int u = 0; u < 8; ++u) {
+    float t = qa.x * __uint_as_float(kq[u].x << 16);
+    t = fmaf(qa.y, __uint_as_float(kq[u].x & 0xffff0000u), t);
+    t = fmaf(qa.z, __uint_as_float(kq[u].y << 16), t);
+    t = fmaf(qa.w, __uint_as_float(kq[u].y & 0xffff0000u), t);
+    t = fmaf(qb.x, __uint_as_float(kq[u].z << 16), t);
+    t = fmaf(qb.y, __uint_as_float(kq[u].z & 0xffff0000u), t);
+    t = fmaf(qb.z, __uint_as_float(kq[u].w << 16), t);
+    v[u] = fmaf(qb.w, __uint_as_float(kq[u].w & 0xffff0000u), t);
+  }
+  // sum over the 8 lanes of a group, scattering the 8 sums: lane seg ends with the score of key 4 seg + lane / 8
+  // (a fixed tree over the dimensions)
+  float w4[4], w2[2];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float send = (seg & 4) ? v[j] : v[j + 4], keep = (seg & 4) ? v[j + 4] : v[j];
+    w4[j] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+  }
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const float send = (seg & 2) ? w4[j] : w4[j + 2], keep = (seg & 2) ? w4[j + 2] : w4[j];
+    w2[j] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+  }
+  const float send1 = (seg & 1) ? w2[0] : w2[1], keep1 = (seg & 1) ? w2[1] : w2[0];
+  const float mine = keep1 + __shfl_xor_sync(0xffffffffu, send1, 1);
+  // lane = key: key 4 (lane / 4) + lane % 4 of the chunk sits in group lane % 4, lane lane / 4 of it
+  const float dot = __shfl_sync(0xffffffffu, mine, 8 * (lane & 3) + (lane >> 2));
+  const float sc = vis ? dot : -INFINITY;
+  const float m_old = state[kDH], l_old = state[kDH + 1];
+  const float m_new = fmaxf(m_old, warp_max(sc));
+  if (m_new == -INFINITY) return;                                 // no key of this chunk is visible to the row yet
+  // a row that has seen no key before starts from an empty state (whatever the slot holds)
+  const float corr = (m_old == -INFINITY) ? 0.f : expf(m_old - m_new);
+  const float pj = vis ? expf(sc - m_new) : 0.f;
+  const float l_new = l_old * corr + warp_sum(pj);
+  float2 acc = (m_old == -INFINITY) ? make_float2(0.f, 0.f) : *reinterpret_cast<const float2*>(state + 2 * lane);
+  acc.x *= corr;
+  acc.y *= corr;
+#pragma unroll
+  for (int j = 0; j < 32; ++j) {
+    const float pw = __shfl_sync(0xffffffffu, pj, j);
+    acc.x = fmaf(pw, __uint_as_float(vq[j] << 16), acc.x);
+    acc.y = fmaf(pw, __uint_as_float(vq[j] & 0xffff0000u), acc.y);
+  }
+  __syncwarp();                                                   // every lane has read the old maximum and sum
+  *reinterpret_cast<float2*>(state + 2 * lane) = acc;
+  if (lane == 0) { state[kDH] = m_new; state[kDH + 1] = l_new; }
+  __syncwarp();
+}
+
+// Merges eight states, `stride` floats apart, in order, for output dimension dim: states without a visible key
+// (maximum -inf) weigh nothing.
+__device__ __forceinline__ void states_merge(const float* first, int stride, int dim, float& M, float& num, float& den) {
+  M = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) M = fmaxf(M, first[j * stride + kDH]);
+  num = 0.f;
+  den = 0.f;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const float* src = first + j * stride;
+    const float mj = src[kDH];
+    if (mj > -INFINITY) {
+      const float e = expf(mj - M);
+      num = fmaf(e, src[dim], num);
+      den = fmaf(e, src[kDH + 1], den);
+    }
+  }
+}
+
 // ------------------------------------------------------------------ attention block (self or cross)
 struct AttnBlockParams {
   float* x;                       // residual stream [R, d], updated in place
@@ -238,6 +342,7 @@ struct AttnBlockParams {
 struct AttnLayout {
   int s_in, s_out, s_x;           // row strides (bytes)
   int w_in, w_out, xh, xl, oh, ol, part, q, mean, rstd, attn, flag, len, pt, total;   // offsets (bytes)
+  int qall, lvl1, lvl2;           // self-attention: every row's query, partial attention states (two levels)
   int zero_begin, zero_end;       // planes that must start at zero
 };
 template <bool SELF>
@@ -262,6 +367,16 @@ __host__ __device__ inline AttnLayout attn_layout(int d, int NT, int pt_ints) {
   L.flag = off; off += 16;
   L.len = off; off += kMaxRows * 4;
   L.pt = off; off += (pt_ints * 4 + 15) / 16 * 16;
+  L.qall = L.lvl1 = L.lvl2 = 0;
+  if (SELF) {
+    // Buffers of the attention step reuse what is dead by then where it is large enough: the planes of x (read
+    // by the input projection only) hold every row's query, the input projection's weights hold the partial
+    // attention states.  Other CTAs write into them only after a cluster barrier that follows the projection.
+    const int rp = NT * 8, q_bytes = rp * kDH * 4, lvl_bytes = kC * rp * kPartial * 4;
+    if (2 * NT * 8 * L.s_x >= q_bytes) L.qall = L.xh; else { L.qall = off; off += q_bytes; }
+    if (2 * lvl_bytes <= rows_in * L.s_in) { L.lvl1 = L.w_in; L.lvl2 = L.w_in + lvl_bytes; }
+    else { L.lvl1 = off; off += lvl_bytes; L.lvl2 = off; off += lvl_bytes; }
+  }
   L.total = off;
   return L;
 }
@@ -292,6 +407,9 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
   volatile int* flag = reinterpret_cast<volatile int*>(fsm + L.flag);
   int* s_len = reinterpret_cast<int*>(fsm + L.len);    // per sequence: tokens in the cache (self) or source length (cross)
   int* s_pt = reinterpret_cast<int*>(fsm + L.pt);      // self: the sequences' page-table rows
+  float* q_all = reinterpret_cast<float*>(fsm + L.qall);   // self: scaled query of every row [rows][kDH]
+  float* lvl1 = reinterpret_cast<float*>(fsm + L.lvl1);    // self: [lump][row][kPartial] states of this CTA's key lumps
+  float* lvl2 = reinterpret_cast<float*>(fsm + L.lvl2);    // self: [rank][row][kPartial] states of the cluster's CTAs
 
   pdl_launch_dependents();
   const unsigned long long stream = tc::l2_evict_first();
@@ -361,6 +479,13 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
   }
   cluster.sync();
 
+  // self-attention: does every rank have at most one chunk of keys?  (the same answer in every CTA of the grid)
+  bool one_chunk_per_rank = true;
+  if (SELF) {
+    for (int b = 0; b < nb; ++b)
+      one_chunk_per_rank = one_chunk_per_rank &&
+          ((s_len[b] + p.rows_per_b + 31) >> 5) - (attn_first_key(p.attn, s_len[b]) >> 5) <= kC;
+  }
   // ---- this rank's tokens: add the partials in rank order, finish the layer norm, write keys / values
   for (int slot = 0; slot < NT; ++slot) {
     const int token = slot * kC + c;
@@ -371,7 +496,16 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
       const int sect = tid / kDH, f = tid % kDH;
       const float y = s_rstd[token] * (a - s_mean[token] * fs) + fc;
       if (sect == 0) {
-        q_s[slot * kDH + f] = y * p.attn.scale;
+        if (SELF) {
+          if (one_chunk_per_rank) {
+            q_all[token * kDH + f] = y * p.attn.scale;             // this rank attends for its own rows
+          } else {
+#pragma unroll
+            for (int dst = 0; dst < kC; ++dst) cluster.map_shared_rank(q_all, dst)[token * kDH + f] = y * p.attn.scale;
+          }
+        } else {
+          q_s[slot * kDH + f] = y * p.attn.scale;
+        }
       } else {
         const int b = token / p.rows_per_b, i = token % p.rows_per_b;
         const int pos = s_len[b] + i;
@@ -388,19 +522,121 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
     __syncthreads();
   }
 
-  // ---- attention of this rank's rows; the result goes to every rank as planes
   AttnParams ap = p.attn;
-  if (SELF) ap.st.page_table = s_pt;
+  if (SELF) {
+    // ---- self-attention (see chunk_fetch / chunk_fold / states_merge above)
+    ap.st.page_table = s_pt;
+    constexpr int RP = NT * 8;
+    const bf16* Kc = reinterpret_cast<const bf16*>(ap.k);
+    const bf16* Vc = reinterpret_cast<const bf16*>(ap.v);
+    const int rpb = p.rows_per_b;
+    if (one_chunk_per_rank) {
+      // Short sequences: this rank takes its own rows (as the projection handed them out), warp w stands in for
+      // rank w and folds that rank's only chunk; a rank's single lump is its state (merging one lump multiplies
+      // by exp(0) = 1), so the eight warp states are merged like the ranks' states.  The result goes to every
+      // rank as planes.
+      for (int slot = 0; slot < NT; ++slot) {
+        const int token = slot * kC + c;
+        if (token < p.R) {                                         // uniform over the CTA
+          const int b = token / rpb, i = token % rpb;
+          const int len = s_len[b], lim_max = len + rpb;
+          const int fk = attn_first_key(ap, len + i), ch0 = attn_first_key(ap, len) >> 5;
+          const int ch = ch0 + ((warp - ch0) & (kC - 1));          // chunk of rank `warp` at or after ch0
+          float* state = lvl2 + (warp * RP + token) * kPartial;
+          if (lane == 0) { state[kDH] = -INFINITY; state[kDH + 1] = 0.f; }
+          __syncwarp();
+          if ((ch << 5) <= len + i) {                              // the row sees at least the chunk's first key
+            const int c0 = ch << 5;
+            const size_t base = ((size_t)s_pt[b * ap.st.pages_per_row + c0 / kPage] * kPage + (c0 % kPage)) * ap.ldkv + h * kDH;
+            uint4 kq[8];
+            uint32_t vq[32];
+            chunk_fetch(Kc, Vc, base, min(32, lim_max - c0), ap.ldkv, lane, kq, vq);
+            const int key = c0 + lane;
+            chunk_fold(kq, vq, q_all + token * kDH, key <= len + i && key >= fk, state, lane);
+          }
+          __syncthreads();
+          if (tid < kDH) {
+            float M, num, den;
+            states_merge(lvl2 + token * kPartial, RP * kPartial, tid, M, num, den);
+            uint32_t hi, lo;
+            split_bits(num / den, hi, lo);
+#pragma unroll
+            for (int dst = 0; dst < kC; ++dst) {
+              *reinterpret_cast<unsigned short*>(cluster.map_shared_rank(oh_s, dst) + sw(token, tid * 2, L.s_out)) = (unsigned short)hi;
+              *reinterpret_cast<unsigned short*>(cluster.map_shared_rank(ol_s, dst) + sw(token, tid * 2, L.s_out)) = (unsigned short)lo;
+            }
+          }
+        }
+      }
+      cluster.sync();
+    } else {
+      // Long sequences: rank c folds its own chunks for every row, so that a chunk's keys and values are fetched
+      // once for all rows of the sequence.  Which warp takes which (lump, rows) is free: with few lumps the rows
+      // are spread over the warps, with many a warp takes one lump for all rows.
+      for (int i = tid; i < 8 * RP; i += kThreads) { lvl1[i * kPartial + kDH] = -INFINITY; lvl1[i * kPartial + kDH + 1] = 0.f; }
+      __syncthreads();
+      for (int b = 0; b < nb; ++b) {
+        const int len = s_len[b];
+        const int lim_max = len + rpb;                              // keys in the cache once the block is written
+        const int nch = (lim_max + 31) >> 5, ch0 = attn_first_key(ap, len) >> 5;
+        const int first_my = ch0 + ((c - ch0) & (kC - 1));          // this rank's first chunk at or after ch0
+        const int n_my = first_my < nch ? (nch - first_my + kC - 1) / kC : 0;
+        const int active = min(8, n_my);
+        if (active == 0) continue;                                  // uniform over the CTA
+        const int S = 8 / active;                                   // row subsets per lump
+        const int a = warp / S, sub = warp % S;
+        if (a >= active) continue;                                  // uniform over the warp; no CTA barrier below
+        const int ch_first = first_my + kC * a;
+        const int lump = (ch_first / kC) & 7;
+        const int* pt = s_pt + b * ap.st.pages_per_row;
+        for (int ch = ch_first; ch < nch; ch += 8 * kC) {
+          const int c0 = ch << 5;
+          const size_t base = ((size_t)pt[c0 / kPage] * kPage + (c0 % kPage)) * ap.ldkv + h * kDH;
+          uint4 kq[8];
+          uint32_t vq[32];
+          chunk_fetch(Kc, Vc, base, min(32, lim_max - c0), ap.ldkv, lane, kq, vq);
+          const int key = c0 + lane;
+#pragma unroll 1
+          for (int i = sub; i < rpb; i += S)
+            chunk_fold(kq, vq, q_all + (b * rpb + i) * kDH, key <= len + i && key >= attn_first_key(ap, len + i),
+                       lvl1 + ((size_t)lump * RP + b * rpb + i) * kPartial, lane);
+        }
+      }
+      __syncthreads();
+      // this rank's state per row: its lumps in lump order; sent to every rank
+      for (int idx = tid; idx < p.R * kDH; idx += kThreads) {
+        const int row = idx / kDH, dim = idx % kDH;
+        float M, num, den;
+        states_merge(lvl1 + row * kPartial, RP * kPartial, dim, M, num, den);
+#pragma unroll
+        for (int dst = 0; dst < kC; ++dst) {
+          float* out = cluster.map_shared_rank(lvl2, dst) + (c * RP + row) * kPartial;
+          out[dim] = num;
+          if (dim == 0) { out[kDH] = M; out[kDH + 1] = den; }
+        }
+      }
+      cluster.sync();
+      // every rank merges the ranks' states in rank order and keeps the result as planes for the output projection
+      for (int idx = tid; idx < p.R * kDH; idx += kThreads) {
+        const int row = idx / kDH, dim = idx % kDH;
+        float M, num, den;
+        states_merge(lvl2 + row * kPartial, RP * kPartial, dim, M, num, den);
+        uint32_t hi, lo;
+        split_bits(num / den, hi, lo);
+        *reinterpret_cast<unsigned short*>(oh_s + sw(row, dim * 2, L.s_out)) = (unsigned short)hi;
+        *reinterpret_cast<unsigned short*>(ol_s + sw(row, dim * 2, L.s_out)) = (unsigned short)lo;
+      }
+      __syncthreads();
+    }
+  } else {
+  // ---- attention of this rank's rows; the result goes to every rank as planes
   for (int slot = 0; slot < NT; ++slot) {
     const int token = slot * kC + c;
     if (token < p.R) {                   // uniform over the CTA
       if (tid < kDH) sm.q[tid] = q_s[slot * kDH + tid];
       __syncthreads();
-      const int b = token / p.rows_per_b, i = token % p.rows_per_b;
-      const int limit = SELF ? (s_len[b] + i + 1) : s_len[b];
-      float ov;
-      if (SELF) ov = attention_head<bf16, kDH, kWarps, true>(ap, b, h, attn_first_key(ap, limit - 1), limit, sm);
-      else ov = attention_head<float, kDH, kWarps, false>(ap, b, h, 0, limit, sm);
+      const int b = token / p.rows_per_b;
+      const float ov = attention_head<float, kDH, kWarps, false>(ap, b, h, 0, s_len[b], sm);
       if (tid < kDH) {
         uint32_t hi, lo;
         split_bits(ov, hi, lo);
@@ -414,6 +650,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
     }
   }
   cluster.sync();
+  }
 
   // ---- this head's share of the output projection for the features of slice c
   float* wsh = p.ws + (size_t)h * p.R * d;
