@@ -494,6 +494,42 @@ def test_local_attention_lockstep(bpd, w):
 
 
 
+LONG_MODELS = [
+    Workload("midi-long", MIDI.cfg, 0.05, 41, 42, 43, batch=1, src_lo=9, src_hi=9, n_decode=420),
+    Workload("midi3-long", MIDI.cfg, 0.05, 41, 52, 53, batch=3, src_lo=3, src_hi=11, n_decode=330),
+]
+
+
+@pytest.mark.parametrize("w", LONG_MODELS, ids=lambda w: w.name)
+def test_long_sequences_share_their_keys(bpd, w):
+    """Full causal attention far into a sequence on the cluster path: once a row sees more than eight chunks of
+    32 keys the self-attention block switches from one CTA per row to keys fetched once for all rows of a
+    sequence.  Both schedules must give the same ids (greedy passes carry one row per sequence, blockwise
+    passes k), and the lock-step against the oracle runs across the switch with every proposal accepted."""
+    from harness import lockstep
+    blob, model, src, src_len, om = _setup(bpd, w)
+    k, N = w.cfg.k_model, w.n_decode
+    s = bpd.Session(model, w.batch, w.max_src, N)
+    s.bpd_encode(src, src_len)
+    g_ids, _, _ = s.bpd_decode_greedy(N)
+    s.bpd_encode(src, src_len)
+    b_ids, _, _ = s.bpd_decode_blockwise(k, N)
+    assert np.array_equal(b_ids, g_ids)
+    plan, sched = _plan(w, g_ids, k, 3.0)
+    s.bpd_encode(src, src_len)
+    s.bpd_set_forced_plan(plan, k)
+    p_ids, _, _ = s.bpd_decode_blockwise(k, N)
+    assert np.array_equal(p_ids, g_ids)
+
+    def all_accepted(b, j, it):
+        return forced_tail(g_ids[b], min(j, N), k, k, 0, w.cfg.vocab)
+    rows = sorted({0, w.batch - 1})
+    rep = lockstep(s, om, src, src_len, k, N, max_iters=(N + k - 1) // k, tail_fn=all_accepted, rows=rows)
+    for b in rows:
+        assert rep.emitted[b] == list(g_ids[b])
+    s.close(); model.close()
+
+
 def test_bounded_wait_expires_and_the_context_survives(bpd):
     """Failure detection without a fault: a wait on a barrier nobody signals gives up after its limit,
     the call reports BPD_E_TIMEOUT and the same process keeps computing correctly afterwards."""
