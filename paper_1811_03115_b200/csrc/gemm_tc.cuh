@@ -72,6 +72,8 @@ struct TcParams {
   int* error;                  // device error word
   const int* all_done;
   int stream_weights;          // 1: the weights are read once per launch (one token tile): load them "evict first"
+  int vec;                     // 1: wide token tiles finish through shared memory with 8- and 16-byte stores (the
+                               // host has checked sizes and alignment)
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -289,6 +291,81 @@ __device__ __forceinline__ void tc_store8(const TcParams& p, int z, int t_first,
   }
 }
 
+// ---------------------------------------------------------------- final epilogue of a wide tile
+// The tile lies in shared memory with one row per token (row stride tstride floats, a multiple of 4).  An item is
+// (token, four consecutive features); the 128 epilogue threads take the items in order, so a warp finishes 128
+// consecutive features of a token with one 16-byte (fp32) or 8-byte (bf16) access per lane instead of 32-lane
+// scalar stores per token.  Same arithmetic per element as tc_store8 (no folded layer norm here).
+__device__ __forceinline__ uint2 pack4_bf16(const bf16 (&b)[4]) {
+  return make_uint2((uint32_t)__bfloat16_as_ushort(b[0]) | ((uint32_t)__bfloat16_as_ushort(b[1]) << 16),
+                    (uint32_t)__bfloat16_as_ushort(b[2]) | ((uint32_t)__bfloat16_as_ushort(b[3]) << 16));
+}
+template <int EPI>
+__device__ __forceinline__ void tc_finish_tile(const TcParams& p, int z, int t0, int nt, int tile, const float* s_t, int tstride,
+                                               const unsigned long long* s_slot, int et) {
+  const int g = et & 31;
+  const int n = tile * kBM + g * 4;                 // first of this item's four features (within the slice)
+  if (n >= p.N) return;
+  float bias[4] = {0.f, 0.f, 0.f, 0.f}, gn[4] = {0.f, 0.f, 0.f, 0.f};
+  if (p.bias) {
+    const uint2 bw = *reinterpret_cast<const uint2*>(p.bias + n + p.zofs_n * z);
+    bias[0] = __uint_as_float(bw.x << 16); bias[1] = __uint_as_float(bw.x & 0xffff0000u);
+    bias[2] = __uint_as_float(bw.y << 16); bias[3] = __uint_as_float(bw.y & 0xffff0000u);
+  }
+  if (EPI == kTcResidual && p.g_next) {
+    const uint2 gw = *reinterpret_cast<const uint2*>(p.g_next + n);
+    gn[0] = __uint_as_float(gw.x << 16); gn[1] = __uint_as_float(gw.x & 0xffff0000u);
+    gn[2] = __uint_as_float(gw.y << 16); gn[3] = __uint_as_float(gw.y & 0xffff0000u);
+  }
+  for (int tr = et >> 5; tr < nt; tr += 4) {
+    const int t = t0 + tr;
+    const float4 a = *reinterpret_cast<const float4*>(s_t + tr * tstride + g * 4);
+    float v[4] = {a.x + bias[0], a.y + bias[1], a.z + bias[2], a.w + bias[3]};
+    if (p.relu) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) v[e] = fmaxf(v[e], 0.f);
+    }
+    if (EPI == kTcPlanes || EPI == kTcHeadOut) {
+      const int nz = n + p.zofs_n * z;
+      if (EPI == kTcHeadOut) {
+        const float4 h = __ldg(reinterpret_cast<const float4*>(p.h + (size_t)t * p.d + (n % p.d)));
+        const float pre[4] = {h.x, h.y, h.z, h.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) v[e] = (p.head_identity && nz < p.d) ? pre[e] : v[e] + pre[e];
+      }
+      bf16 hi[4], lo[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) split_bf16(v[e], hi[e], lo[e]);
+      const long long o = (long long)t * p.ldo + nz;
+      *reinterpret_cast<uint2*>(p.out_hi + o) = pack4_bf16(hi);
+      *reinterpret_cast<uint2*>(p.out_hi + o + p.plane) = pack4_bf16(lo);
+    } else if (EPI == kTcF32) {
+      *reinterpret_cast<float4*>(p.out_f32 + (long long)t * p.ldo + n) = make_float4(v[0], v[1], v[2], v[3]);
+    } else if (EPI == kTcResidual) {
+      float4* xp = reinterpret_cast<float4*>(p.out_f32 + (long long)t * p.ldo + n);
+      const float4 old = *xp;                        // one writer per element
+      const float xn[4] = {old.x + v[0], old.y + v[1], old.z + v[2], old.w + v[3]};
+      *xp = make_float4(xn[0], xn[1], xn[2], xn[3]);
+      if (p.g_next) {
+        bf16 hi[4], lo[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) split_bf16(xn[e] * gn[e], hi[e], lo[e]);
+        *reinterpret_cast<uint2*>(p.xg_hi + (long long)t * p.ldo + n) = pack4_bf16(hi);
+        *reinterpret_cast<uint2*>(p.xg_hi + (long long)t * p.ldo + n + p.xg_plane) = pack4_bf16(lo);
+      }
+    } else if (EPI == kTcQkv) {
+      const int d = p.d;
+      if (n < d) {
+        *reinterpret_cast<float4*>(p.out_f32 + (long long)t * p.ldo + n) = make_float4(v[0], v[1], v[2], v[3]);
+      } else {
+        const bf16 b4[4] = {__float2bfloat16_rn(v[0]), __float2bfloat16_rn(v[1]), __float2bfloat16_rn(v[2]), __float2bfloat16_rn(v[3])};
+        bf16* dst = (n < 2 * d) ? p.kcache + s_slot[tr] + (n - d) : p.vcache + s_slot[tr] + (n - 2 * d);
+        *reinterpret_cast<uint2*>(dst) = pack4_bf16(b4);
+      }
+    }
+  }
+}
+
 // ---------------------------------------------------------------- bounded-wait self test
 // One CTA waits on an mbarrier that nothing ever arrives on, gives up after `limit_cycles`, records the same
 // error code the projection kernel would and returns normally: the context stays usable.
@@ -336,6 +413,9 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
   const int tpt = topk_threads_per_token(bn), tstride = kBM + tpt;   // row stride = tpt mod 32: conflict-free scans
   // the debug dump of the logits and the rank counting of top-n acceptance are rare: kept out of the common loops
   const bool extras = (EPI == kTcArgmax) && (p.logits != nullptr || p.rank.cnt != nullptr);
+  // wide tiles of the other epilogues leave through shared memory too (see tc_finish_tile)
+  const bool vec = (EPI != kTcArgmax) && p.vec && bn >= 32 && !p.ln_x;
+  constexpr int vstride = kBM + 4;
   if (EPI == kTcQkv && !skip && et < nt) {
     const int t = t0 + et;
     const int b = t / p.rows_per_b, i = t % p.rows_per_b;
@@ -388,7 +468,10 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
       for (int cb = 0; cb < bn; cb += 16) {
         float v[16];
         tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + cb, v);
-        if (EPI != kTcArgmax) {
+        if (EPI != kTcArgmax && vec) {
+#pragma unroll
+          for (int c = 0; c < 16; ++c) s_t[(cb + c) * vstride + row] = v[c];
+        } else if (EPI != kTcArgmax) {
           if (n < p.N) {
             const float lo8[8] = {v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]};
             const float hi8[8] = {v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15]};
@@ -445,7 +528,11 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
 #pragma unroll
               for (int c = 0; c < 8; ++c) acc[c] += v[ss][c];
           }
-          if (EPI != kTcArgmax) {
+          if (EPI != kTcArgmax && vec) {
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+              if (cg + c < nt) s_t[(cg + c) * vstride + row] = acc[c];
+          } else if (EPI != kTcArgmax) {
             if (n < p.N) tc_store8<EPI>(p, slice, t0 + cg, min(8, nt - cg), n, acc, s_mean, s_rstd, cg, s_slot);
           } else {
 #pragma unroll
@@ -463,6 +550,10 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
         }
         if (et == 0) p.tile_counters[(size_t)u.zidx * ntiles + tile] = 0;   // ready for the next launch
       }
+    }
+    if (EPI != kTcArgmax && vec && (direct || ctl[1])) {
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      tc_finish_tile<EPI>(p, slice, t0, nt, tile, s_t, vstride, s_slot, et);
     }
     if (EPI == kTcArgmax && (direct || ctl[1])) {
       // The tile sits in shared memory with one row per token.  tpt threads share a token: each scans every

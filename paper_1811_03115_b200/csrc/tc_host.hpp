@@ -175,6 +175,13 @@ int launch(const Operands& op, int N, int K, int T, TcParams p, const Scratch& s
   p.ws = sc.ws; p.tile_counters = sc.tile_counters; p.done_counter = sc.done_counter;
   p.best = sc.best; p.error = sc.error;
   p.stream_weights = (ttiles == 1 && !getenv("BPD_NO_L2_HINTS")) ? 1 : 0;
+  {
+    // vector stores in the epilogue of wide tiles: every row offset and pointer involved must allow them
+    auto al = [](const void* q, size_t a) { return q == nullptr || (uintptr_t)q % a == 0; };
+    p.vec = (N % 4 == 0 && p.ldo % 4 == 0 && p.plane % 4 == 0 && p.xg_plane % 4 == 0 && p.zofs_n % 4 == 0 &&
+             (p.d % 4 == 0) && al(p.out_f32, 16) && al(p.out_hi, 8) && al(p.xg_hi, 8) && al(p.h, 16) && al(p.bias, 8) &&
+             al(p.g_next, 8) && al(p.kcache, 8) && al(p.vcache, 8)) ? 1 : 0;
+  }
   dim3 grid(pl.tiles, pl.splits, ttiles * zslices);
   BPD_CUDA(launch_k(gemm_tc_kernel<EPI>, grid, dim3(kThreads), smem_bytes(bn), st, pdl, ma, mh, ml, p, zslices,
                     a_rows_per_slice, b_cols_per_slice));

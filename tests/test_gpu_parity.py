@@ -65,7 +65,8 @@ def _expected_khats(sched_b, k, n):
 # ---------------------------------------------------------------- single operators
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-@pytest.mark.parametrize("rows,in_f,out_f", [(1, 64, 50), (8, 1024, 3072), (13, 520, 77), (64, 256, 129)])
+@pytest.mark.parametrize("rows,in_f,out_f", [(1, 64, 50), (8, 1024, 3072), (13, 520, 77), (64, 256, 129), (64, 256, 384),
+                                             (100, 512, 1024), (40, 2048, 132)])
 def test_op_linear_matches_definition(bpd, dtype, rows, in_f, out_f):
     import torch
     g = torch.Generator().manual_seed(rows * 1000 + in_f)
