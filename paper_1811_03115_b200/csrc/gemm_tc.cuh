@@ -343,10 +343,15 @@ __device__ __forceinline__ void tc_finish_tile(const TcParams& p, int z, int t0,
       *reinterpret_cast<float4*>(p.out_f32 + (long long)t * p.ldo + n) = make_float4(v[0], v[1], v[2], v[3]);
     } else if (EPI == kTcResidual) {
       float4* xp = reinterpret_cast<float4*>(p.out_f32 + (long long)t * p.ldo + n);
-      const float4 old = *xp;                        // one writer per element
+      if (!p.g_next) {
+        // one writer per element: x += v as a 16-byte reduction, nothing to read back
+        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(xp), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]) : "memory");
+        continue;
+      }
+      const float4 old = *xp;
       const float xn[4] = {old.x + v[0], old.y + v[1], old.z + v[2], old.w + v[3]};
       *xp = make_float4(xn[0], xn[1], xn[2], xn[3]);
-      if (p.g_next) {
+      {
         bf16 hi[4], lo[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) split_bf16(xn[e] * gn[e], hi[e], lo[e]);
