@@ -528,7 +528,10 @@ static int run_layers_fused(bpd_session* s, const PassArgs& a) {
   const int* done = s->st.all_done;
   const bool pdl = s->use_pdl != 0;
   const int nt = (R + 7) / 8;
-  const size_t smem_self = fused::attn_layout<true>(d, nt, s->B * s->ppr).total, smem_cross = fused::attn_layout<false>(d, nt, 0).total;
+  // encoder keys / values of a head are staged in shared memory when all sequences' rows fit a small budget
+  const int cross_smax = (s->B * s->max_src * fused::kCrossRowBytes <= fused::kCrossStageMax && !getenv("BPD_NO_CROSS_STAGE")) ? s->max_src : 0;
+  const size_t smem_self = fused::attn_layout<true>(d, nt, s->B * s->ppr).total;
+  const size_t smem_cross = fused::attn_layout<false>(d, nt, 0, s->B * cross_smax).total;
   const size_t smem_ffn = fused::ffn_layout(d, nt).total;
   // the opt-in shared-memory limit of each kernel grows with the widest model seen so far
   static size_t attr_max[3][3] = {{0, 0, 0}, {0, 0, 0}, {0, 0, 0}};
@@ -568,7 +571,7 @@ static int run_layers_fused(bpd_session* s, const PassArgs& a) {
     fused::AttnBlockParams pc = ps;
     pc.gain = static_cast<const bf16*>(L.ln2g); pc.fold_s = L.s_cq; pc.fold_c = L.c_cq;
     pc.w_in = static_cast<const bf16*>(L.cwq); pc.w_out = static_cast<const bf16*>(L.cwo);
-    pc.kcache = nullptr; pc.vcache = nullptr;
+    pc.kcache = nullptr; pc.vcache = nullptr; pc.cross_smax = cross_smax;
     pc.attn.causal = 0; pc.attn.limit_b = s->st.src_len; pc.attn.k = s->crosskv[l];
     pc.attn.v = static_cast<float*>(s->crosskv[l]) + d; pc.attn.ldkv = 2 * d;
     pc.attn.bstride = (long long)s->max_src * 2 * d; pc.attn.paged = 0;

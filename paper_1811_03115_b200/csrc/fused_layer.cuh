@@ -40,6 +40,9 @@ constexpr int kWarps = 8;
 constexpr int kDH = 64;          // head width this path is built for
 constexpr int kHS = 16;          // hidden units per CTA in the feed-forward block
 constexpr int kMaxRows = 16;
+constexpr int kCrossKeyPitch = kDH * 4 + 16;   // bytes per staged encoder key row (fp32): 16-byte reads of 8 lanes hit all banks
+constexpr int kCrossRowBytes = kCrossKeyPitch + kDH * 4;   // key row + value row
+constexpr int kCrossStageMax = 24 * 1024;      // more encoder rows than fit here are read from L2 instead
 constexpr int kPartial = kDH + 2;   // a partial attention state: weighted value sum [kDH], running maximum, weight sum
 
 // Byte offset of (row, byte) in a shared-memory matrix with rb bytes per row (a multiple of 64).  When rb is a
@@ -50,6 +53,9 @@ __host__ __device__ inline int sw(int row, int byte, int rb) { return row * rb +
 // 16 bytes of weights, global -> shared, marked "evict first" in L2 (they are read once per pass).
 __device__ __forceinline__ void cp_async16(void* smem, const void* gmem, unsigned long long policy) {
   asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(tc::smem_u32(smem)), "l"(gmem), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void cp_async16_keep(void* smem, const void* gmem) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(tc::smem_u32(smem)), "l"(gmem) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
@@ -322,6 +328,64 @@ __device__ __forceinline__ void states_merge(const float* first, int stride, int
   }
 }
 
+// ------------------------------------------------------------------ cross-attention over staged encoder rows
+// Attention of one query row (sm.q, scaled) over `limit` encoder positions whose keys and values of this head lie
+// in shared memory (rows of kCrossRowBytes: key, padding, value; fp32).  Warp w folds the chunks w, w + 8, ... of
+// 32 positions in order (lane = key for the scores, lane = two output dimensions for the values); the warps'
+// states are merged in warp order.  Threads c < kDH return output element c.
+__device__ __forceinline__ float cross_attention_staged(const uint8_t* kv, int limit, AttnSmem<kDH, kWarps>& sm) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float m_run = -INFINITY, l_run = 0.f, a0 = 0.f, a1 = 0.f;
+  for (int c0 = warp * 32; c0 < limit; c0 += kWarps * 32) {
+    const int nk = min(32, limit - c0);
+    float sc = -INFINITY;
+    if (lane < nk) {
+      const float4* kr = reinterpret_cast<const float4*>(kv + (size_t)(c0 + lane) * kCrossRowBytes);
+      const float4* qv = reinterpret_cast<const float4*>(sm.q);
+      float dot = 0.f;
+#pragma unroll
+      for (int u = 0; u < kDH / 4; ++u) {
+        const float4 k4 = kr[u], q4 = qv[u];
+        dot = fmaf(q4.x, k4.x, dot); dot = fmaf(q4.y, k4.y, dot); dot = fmaf(q4.z, k4.z, dot); dot = fmaf(q4.w, k4.w, dot);
+      }
+      sc = dot;
+    }
+    const float m_new = fmaxf(m_run, warp_max(sc));
+    const float corr = expf(m_run - m_new);
+    const float pj = (lane < nk) ? expf(sc - m_new) : 0.f;
+    l_run = l_run * corr + warp_sum(pj);
+    a0 *= corr;
+    a1 *= corr;
+    for (int j = 0; j < nk; ++j) {
+      const float pw = __shfl_sync(0xffffffffu, pj, j);
+      const float2 v2 = *reinterpret_cast<const float2*>(kv + (size_t)(c0 + j) * kCrossRowBytes + kCrossKeyPitch + lane * 8);
+      a0 = fmaf(pw, v2.x, a0);
+      a1 = fmaf(pw, v2.y, a1);
+    }
+    m_run = m_new;
+  }
+  if (lane == 0) { sm.m[warp] = m_run; sm.l[warp] = l_run; }
+  sm.acc[warp][2 * lane] = a0;
+  sm.acc[warp][2 * lane + 1] = a1;
+  __syncthreads();
+  float ov = 0.f;
+  if (threadIdx.x < kDH) {
+    const int c = threadIdx.x;
+    float M = sm.m[0];
+#pragma unroll
+    for (int w = 1; w < kWarps; ++w) M = fmaxf(M, sm.m[w]);
+    float num = 0.f, den = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+      const float e = expf(sm.m[w] - M);          // warps without keys hold -inf: weight 0
+      num = fmaf(e, sm.acc[w][c], num);
+      den = fmaf(e, sm.l[w], den);
+    }
+    ov = num / den;
+  }
+  return ov;
+}
+
 // ------------------------------------------------------------------ attention block (self or cross)
 struct AttnBlockParams {
   float* x;                       // residual stream [R, d], updated in place
@@ -334,6 +398,7 @@ struct AttnBlockParams {
   float eps;
   bf16* kcache; bf16* vcache;     // self: paged cache of this layer, new rows are written here
   AttnParams attn;                // keys / values, paging, lengths, scale (q and out are not used)
+  int cross_smax;                 // cross: encoder rows per sequence staged in shared memory (0: read from L2)
   float* ws;                      // [H][R][d] per-head shares of the output projection
   unsigned* counters;             // [kC], zero between launches
   const int* all_done;
@@ -343,10 +408,11 @@ struct AttnLayout {
   int s_in, s_out, s_x;           // row strides (bytes)
   int w_in, w_out, xh, xl, oh, ol, part, q, mean, rstd, attn, flag, len, pt, total;   // offsets (bytes)
   int qall, lvl1, lvl2;           // self-attention: every row's query, partial attention states (two levels)
+  int ckv;                        // cross-attention: the sequences' encoder keys and values of this head
   int zero_begin, zero_end;       // planes that must start at zero
 };
 template <bool SELF>
-__host__ __device__ inline AttnLayout attn_layout(int d, int NT, int pt_ints) {
+__host__ __device__ inline AttnLayout attn_layout(int d, int NT, int pt_ints, int cross_rows = 0) {
   AttnLayout L;
   const int ks = d / kC, rows_in = SELF ? 3 * kDH : kDH;
   L.s_in = ks * 2; L.s_out = kDH * 2; L.s_x = ks * 2;
@@ -368,6 +434,8 @@ __host__ __device__ inline AttnLayout attn_layout(int d, int NT, int pt_ints) {
   L.len = off; off += kMaxRows * 4;
   L.pt = off; off += (pt_ints * 4 + 15) / 16 * 16;
   L.qall = L.lvl1 = L.lvl2 = 0;
+  L.ckv = off;
+  if (!SELF) off += cross_rows * kCrossRowBytes;
   if (SELF) {
     // Buffers of the attention step reuse what is dead by then where it is large enough: the planes of x (read
     // by the input projection only) hold every row's query, the input projection's weights hold the partial
@@ -392,8 +460,9 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
   constexpr int ROWS_IN = SELF ? 3 * kDH : kDH;
   const int nb = p.R / p.rows_per_b;                                   // sequences in this pass
   const int pt_ints = SELF ? nb * p.attn.st.pages_per_row : 0;
-  const AttnLayout L = attn_layout<SELF>(d, NT, pt_ints);
+  const AttnLayout L = attn_layout<SELF>(d, NT, pt_ints, SELF ? 0 : nb * p.cross_smax);
   uint8_t* w_in_s = fsm + L.w_in;
+  uint8_t* ckv_s = fsm + L.ckv;                        // cross: [sequence][row][key | value] of this head
   uint8_t* w_out_s = fsm + L.w_out;
   uint8_t* xh_s = fsm + L.xh;
   uint8_t* xl_s = fsm + L.xl;
@@ -425,6 +494,17 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
     for (int idx = tid; idx < slice * 8; idx += kThreads) {
       const int row = idx >> 3, c16 = idx & 7;
       cp_async16(w_out_s + sw(row, c16 * 16, L.s_out), p.w_out + (size_t)(c * slice + row) * d + h * kDH + c16 * 8, stream);
+    }
+    if (!SELF && p.cross_smax > 0) {
+      // the encoder's keys and values of this head do not change after the encoder ran: they come along
+      const float* Kg = reinterpret_cast<const float*>(p.attn.k);
+      const float* Vg = reinterpret_cast<const float*>(p.attn.v);
+      for (int idx = tid; idx < nb * p.cross_smax * 32; idx += kThreads) {
+        const int row = idx >> 5, piece = idx & 31, b = row / p.cross_smax, sidx = row % p.cross_smax;
+        const size_t at = (size_t)b * p.attn.bstride + (size_t)sidx * p.attn.ldkv + h * kDH + (piece & 15) * 4;
+        if (piece < 16) cp_async16_keep(ckv_s + row * kCrossRowBytes + piece * 16, Kg + at);
+        else cp_async16_keep(ckv_s + row * kCrossRowBytes + kCrossKeyPitch + (piece - 16) * 16, Vg + at);
+      }
     }
     cp_async_commit();
   }
@@ -636,7 +716,8 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
       if (tid < kDH) sm.q[tid] = q_s[slot * kDH + tid];
       __syncthreads();
       const int b = token / p.rows_per_b;
-      const float ov = attention_head<float, kDH, kWarps, false>(ap, b, h, 0, s_len[b], sm);
+      const float ov = p.cross_smax > 0 ? cross_attention_staged(ckv_s + (size_t)b * p.cross_smax * kCrossRowBytes, s_len[b], sm)
+                                        : attention_head<float, kDH, kWarps, false>(ap, b, h, 0, s_len[b], sm);
       if (tid < kDH) {
         uint32_t hi, lo;
         split_bits(ov, hi, lo);
