@@ -648,7 +648,20 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
     PROF(kProfCrossQ, BPD_TRY(tc::launch<tc::kTcF32>(with_w(xn, L.cwq, d), d, d, R, pc, sc, st, 1, 0, 0, pdl)); ++g_launches);
     ap.causal = 0; ap.limit_b = s->st.src_len; ap.k = s->crosskv[l]; ap.v = static_cast<float*>(s->crosskv[l]) + d;
     ap.ldkv = 2 * d; ap.bstride = (long long)s->max_src * 2 * d; ap.paged = 0;
-    PROF(kProfCrossAttn, launch_attention<float, float>(ap, st, pdl););
+    // many sequences, head width 64: the encoder's keys and values are staged before the dependency wait
+    const bool staged_cross = ap.by_rows && ap.dh == 64 && a.kcur <= 16 && cross_staged_smem(s->max_src) <= 160 * 1024 &&
+                              !getenv("BPD_NO_CROSS_STAGE");
+    if (staged_cross) {
+      static size_t attr = 0;
+      const size_t smem = cross_staged_smem(s->max_src);
+      if (smem > attr) {
+        BPD_CUDA(cudaFuncSetAttribute(cross_attention_staged_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        attr = smem;
+      }
+      PROF(kProfCrossAttn, BPD_CUDA(launch_k(cross_attention_staged_kernel<float>, dim3(s->B * c.H), dim3(kAttnWarps * 32), smem, st, pdl, ap, s->max_src)););
+    } else {
+      PROF(kProfCrossAttn, launch_attention<float, float>(ap, st, pdl););
+    }
     ++g_launches;
     if (fold) po.g_next = static_cast<const bf16*>(L.ln3g);
     PROF(kProfCrossO, BPD_TRY(tc::launch<tc::kTcResidual>(with_w(at, L.cwo, d), d, d, R, po, sc, st, 1, 0, 0, pdl)); ++g_launches);

@@ -819,6 +819,94 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_seq_kernel(AttnPara
   }
 }
 
+// Decoder cross-attention for sessions with many sequences: a CTA per (sequence, head), head width 64, fp32 keys
+// and values.  The encoder's keys and values do not change during a decode, so the CTA copies its head's rows
+// (all positions below the source length) into shared memory before it waits for the preceding launch; only the
+// queries depend on that.  Rows of kXKeyPitch + 256 bytes: lane-per-key 16-byte reads of 8 lanes hit all banks.
+// A warp serves query rows warp, warp + 8 and folds the 32-key chunks of a row in position order with a running
+// maximum / sum, the same arithmetic per row as attention_seq_kernel.
+constexpr int kXKeyPitch = 64 * 4 + 16;
+constexpr int kXRowBytes = kXKeyPitch + 64 * 4;
+__host__ __device__ inline size_t cross_staged_smem(int max_src) { return (size_t)max_src * kXRowBytes + 16 * 64 * sizeof(float); }
+template <typename QT>
+__global__ void __launch_bounds__(kAttnWarps * 32) cross_attention_staged_kernel(AttnParams p, int max_src) {
+  extern __shared__ __align__(16) uint8_t xs[];
+  uint8_t* kv = xs;
+  float* s_q = reinterpret_cast<float*>(xs + (size_t)max_src * kXRowBytes);   // [16][64]
+  pdl_launch_dependents();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b = blockIdx.x / p.H, h = blockIdx.x % p.H;
+  const int limit = min(p.limit_b[b], max_src);
+  {
+    const float* Kg = reinterpret_cast<const float*>(p.k) + (size_t)b * p.bstride + h * 64;
+    const float* Vg = reinterpret_cast<const float*>(p.v) + (size_t)b * p.bstride + h * 64;
+    for (int idx = threadIdx.x; idx < limit * 32; idx += blockDim.x) {
+      const int row = idx >> 5, piece = idx & 31;
+      const float* src = (piece < 16 ? Kg : Vg) + (size_t)row * p.ldkv + (piece & 15) * 4;
+      uint8_t* dst = kv + (size_t)row * kXRowBytes + (piece < 16 ? piece * 16 : kXKeyPitch + (piece - 16) * 16);
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  }
+  pdl_wait();
+  const bool ended = p.all_done && *p.all_done;
+  const int nrows = p.rows_per_b;
+  if (!ended) {
+    for (int idx = threadIdx.x; idx < nrows * 64; idx += blockDim.x) {
+      const int i = idx >> 6, c = idx & 63;
+      s_q[idx] = to_f(reinterpret_cast<const QT*>(p.q)[(long long)(b * nrows + i) * p.ldq + h * 64 + c]) * p.scale;
+    }
+  }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();
+  if (ended) return;
+  for (int i = warp; i < nrows; i += kAttnWarps) {
+    float m_run = -INFINITY, l_run = 0.f, a0 = 0.f, a1 = 0.f;
+    const float4* qv = reinterpret_cast<const float4*>(s_q + i * 64);
+    for (int c0 = 0; c0 < limit; c0 += 32) {
+      const int nk = min(32, limit - c0);
+      float sc = -INFINITY;
+      if (lane < nk) {
+        const float4* kr = reinterpret_cast<const float4*>(kv + (size_t)(c0 + lane) * kXRowBytes);
+        float dot = 0.f;
+#pragma unroll
+        for (int u = 0; u < 16; ++u) {
+          const float4 k4 = kr[u], q4 = qv[u];
+          dot = fmaf(q4.x, k4.x, dot); dot = fmaf(q4.y, k4.y, dot); dot = fmaf(q4.z, k4.z, dot); dot = fmaf(q4.w, k4.w, dot);
+        }
+        sc = dot;
+      }
+      const float m_new = fmaxf(m_run, warp_max(sc));
+      const float corr = expf(m_run - m_new);
+      const float pj = (lane < nk) ? expf(sc - m_new) : 0.f;
+      l_run = l_run * corr + warp_sum(pj);
+      a0 *= corr;
+      a1 *= corr;
+      for (int j = 0; j < nk; ++j) {
+        const float pw = __shfl_sync(0xffffffffu, pj, j);
+        const float2 v2 = *reinterpret_cast<const float2*>(kv + (size_t)(c0 + j) * kXRowBytes + kXKeyPitch + lane * 8);
+        a0 = fmaf(pw, v2.x, a0);
+        a1 = fmaf(pw, v2.y, a1);
+      }
+      m_run = m_new;
+    }
+    const float inv = 1.f / l_run;
+    const float o2[2] = {a0 * inv, a1 * inv};
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+      const long long o = (long long)(b * nrows + i) * p.ldo + h * 64 + lane * 2 + t;
+      if (p.out_plane) {
+        bf16* op = reinterpret_cast<bf16*>(p.out) + o;
+        const bf16 hi = __float2bfloat16_rn(o2[t]);
+        op[0] = hi;
+        op[p.out_plane] = __float2bfloat16_rn(o2[t] - __bfloat162float(hi));
+      } else {
+        reinterpret_cast<QT*>(p.out)[o] = from_f<QT>(o2[t]);
+      }
+    }
+  }
+}
+
 // Picks the split kernel for the common head widths, the generic one-warp kernel otherwise.
 template <typename QT, typename CT>
 static void launch_attention(const AttnParams& p, cudaStream_t st, bool pdl = false) {
