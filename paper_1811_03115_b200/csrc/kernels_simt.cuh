@@ -142,13 +142,26 @@ constexpr int kLnMaxD = 1024;   // the row is held in registers: 8 float4 per la
 template <typename WT, typename AT>
 __global__ void __launch_bounds__(128) layernorm_kernel(LnParams p) {
   pdl_launch_dependents();
-  pdl_wait();
-  if (p.all_done && *p.all_done) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = blockIdx.x * 4 + warp;
+  const int nv = p.d >> 2;                 // float4 per row (d is a multiple of 8)
+  // gain and shift do not depend on the preceding launch: they are fetched before the wait
+  const WT* g = reinterpret_cast<const WT*>(p.g);
+  const WT* bb = reinterpret_cast<const WT*>(p.b);
+  float gv[kLnMaxD / 128][4], bv[kLnMaxD / 128][4];
+#pragma unroll
+  for (int i = 0; i < kLnMaxD / 128; ++i) {
+    const int idx = i * 32 + lane;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      gv[i][e] = (idx < nv) ? to_f(g[idx * 4 + e]) : 0.f;
+      bv[i][e] = (idx < nv) ? to_f(bb[idx * 4 + e]) : 0.f;
+    }
+  }
+  pdl_wait();
+  if (p.all_done && *p.all_done) return;
   if (r >= p.rows) return;
   const float4* x4 = reinterpret_cast<const float4*>(p.x + (size_t)r * p.d);
-  const int nv = p.d >> 2;                 // float4 per row (d is a multiple of 8)
   float4 v[kLnMaxD / 128];
   float s = 0.f;
 #pragma unroll
@@ -167,8 +180,6 @@ __global__ void __launch_bounds__(128) layernorm_kernel(LnParams p) {
     }
   }
   const float rstd = rsqrtf(warp_sum(q) / (float)p.d + p.eps);
-  const WT* g = reinterpret_cast<const WT*>(p.g);
-  const WT* bb = reinterpret_cast<const WT*>(p.b);
 #pragma unroll
   for (int i = 0; i < kLnMaxD / 128; ++i) {
     const int idx = i * 32 + lane;
@@ -177,7 +188,7 @@ __global__ void __launch_bounds__(128) layernorm_kernel(LnParams p) {
       const float in[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
       float o[4];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) o[e] = (in[e] - mean) * rstd * to_f(g[c + e]) + to_f(bb[c + e]);
+      for (int e = 0; e < 4; ++e) o[e] = (in[e] - mean) * rstd * gv[i][e] + bv[i][e];
       if (p.plane) {
         bf16* yp = reinterpret_cast<bf16*>(p.y) + (size_t)r * p.d + c;
         bf16 hi[4], lo[4];
