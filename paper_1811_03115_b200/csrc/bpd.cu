@@ -735,7 +735,7 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
     // stage 2: all heads at the last accepted position of every row
     GatherParams gp{static_cast<const bf16*>(s->u), s->pl_u, ldu, static_cast<bf16*>(s->u2), s->pl_u2, s->h_f32, s->h2, d,
                     s->st, s->B, a.kcur, done};
-    launch_k(gather_selected_kernel, dim3(s->B), dim3(256), 0, st, pdl, gp);
+    launch_k(gather_selected_kernel, dim3(s->B, 16), dim3(256), 0, st, pdl, gp);
     ++g_launches;
     BPD_TRY(heads(s->u2, s->pl_u2, s->B, s->h2, s->B, a.kh, s->table2, false, nullptr, 1));
     SelectParams sp{s->st, s->st.table, s->table2, s->table_full, s->B, a.kcur, a.kh, a.knext, done};

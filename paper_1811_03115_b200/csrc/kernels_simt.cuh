@@ -1221,14 +1221,17 @@ static __global__ void __launch_bounds__(256) gather_selected_kernel(GatherParam
   pdl_launch_dependents();
   pdl_wait();
   if (p.all_done && *p.all_done) return;
+  // grid = (sequences, column parts): a row of hidden activations is some hundred KB, one CTA per row copied it
+  // in tens of dependent steps
   const int b = blockIdx.x;
   const int row = b * p.kcur + max(p.st.khat[b], 1) - 1;     // last accepted position (first one for idle rows)
   const uint4* s_hi = reinterpret_cast<const uint4*>(p.u + (size_t)row * p.ldu);
   const uint4* s_lo = reinterpret_cast<const uint4*>(p.u + (size_t)row * p.ldu + p.pl_u);
   uint4* d_hi = reinterpret_cast<uint4*>(p.u2 + (size_t)b * p.ldu);
   uint4* d_lo = reinterpret_cast<uint4*>(p.u2 + (size_t)b * p.ldu + p.pl_u2);
-  for (int i = threadIdx.x; i < p.ldu / 8; i += blockDim.x) { d_hi[i] = s_hi[i]; d_lo[i] = s_lo[i]; }
-  for (int c = threadIdx.x; c < p.d; c += blockDim.x) p.h2[(size_t)b * p.d + c] = p.h[(size_t)row * p.d + c];
+  const int step = blockDim.x * gridDim.y, first = blockIdx.y * blockDim.x + threadIdx.x;
+  for (int i = first; i < p.ldu / 8; i += step) { d_hi[i] = s_hi[i]; d_lo[i] = s_lo[i]; }
+  for (int c = first; c < p.d; c += step) p.h2[(size_t)b * p.d + c] = p.h[(size_t)row * p.d + c];
 }
 
 struct SelectParams {
