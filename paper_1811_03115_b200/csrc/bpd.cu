@@ -1,5 +1,6 @@
 // C ABI of the blockwise-parallel-decoding library: blob parsing, buffer
 // planning, the encoder, the decoder pass and the decode loops.
+#include <chrono>
 #include <math.h>
 #include <stdlib.h>
 #include <string.h>
@@ -160,6 +161,7 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
   st.table = a.take<int>((size_t)B * kMaxK * kMaxK);
   st.out_ids = a.take<int>((size_t)B * max_tgt);
   st.all_done = a.take<int>(1); st.error = a.take<int>(1);
+  st.signal = a.take<int>(2); st.host_flags = nullptr;
   st.stats = a.take<long long>(4 + kMaxK + 1);
   st.page_table = page_table; st.pages_per_row = ppr; st.max_tgt = max_tgt;
   void* u2 = a.take_bytes((size_t)B * c.k_model * c.d_hidden * ea);
@@ -971,6 +973,13 @@ int bpd_session_create(const bpd_model* model, int batch, int max_src, int max_t
       pe[(size_t)pos * model->cfg.d + 2 * i + 1] = (float)cos(ang);
     }
   cudaError_t e = cudaMallocHost(reinterpret_cast<void**>(&s->pinned), (256 + (size_t)batch * kMaxK) * sizeof(int));
+  if (e == cudaSuccess) {
+    memset(s->pinned, 0, (256 + (size_t)batch * kMaxK) * sizeof(int));
+    void* dev_view = nullptr;
+    e = cudaHostGetDevicePointer(&dev_view, s->pinned, 0);
+    s->st.host_flags = static_cast<int*>(dev_view);
+    s->epoch = 0;
+  }
   for (int i = 0; i < 8 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&s->ev_flag[i], cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreate(&s->ev0);
   if (e == cudaSuccess) e = cudaEventCreate(&s->ev1);
@@ -1089,16 +1098,41 @@ static int check_decode_args(bpd_session* s, int max_new, int eos) {
 // Launch passes until the device reports every row finished.  The flag of pass
 // t is read back asynchronously and looked at two passes later, so the host
 // never stalls the stream; passes issued after the end return at once.
+// The verify kernel of pass t writes (epoch, finished?) straight into slot t mod 8 of the pinned flags; nothing is
+// enqueued between two passes.  Returns 1 / 2 (open / all rows finished) once the slot carries this decode's epoch.
+static int wait_pass_flag(bpd_session* s, int slot, int* finished) {
+  volatile int* flags = s->pinned;
+  const auto t0 = std::chrono::steady_clock::now();
+  for (unsigned spins = 0;; ++spins) {
+    const int v = flags[slot];
+    if ((v >> 2) == s->epoch) {
+      flags[slot] = 0;              // the slot's next report (eight passes on) must not be mistaken for this one
+      *finished = (v & 3) == 2;
+      return BPD_OK;
+    }
+    if ((spins & 0x3ff) == 0x3ff) {
+      const cudaError_t q = cudaStreamQuery(s->stream);
+      if (q != cudaSuccess && q != cudaErrorNotReady) return fail(BPD_E_CUDA, "decoder pass failed: %s", cudaGetErrorString(q));
+      if (q == cudaSuccess && (flags[slot] >> 2) != s->epoch) return fail(BPD_E_CUDA, "a pass ended without reporting its state");
+      if (std::chrono::steady_clock::now() - t0 > std::chrono::seconds(30)) return fail(BPD_E_TIMEOUT, "no pass reported its state for 30 s");
+    }
+  }
+}
 static int decode_loop(bpd_session* s, const PassArgs& a, int max_passes) {
+  // a new epoch and pass counter for this decode, ordered on the stream behind whatever the previous one left
+  s->epoch = (s->epoch % 0x0fffffff) + 1;
+  int* stage = &s->pinned[200 + 2 * (s->epoch & 1)];
+  stage[0] = s->epoch; stage[1] = 0;
+  BPD_CUDA(cudaMemcpyAsync(s->st.signal, stage, 2 * sizeof(int), cudaMemcpyHostToDevice, s->stream));
   for (int it = 0; it < max_passes; ++it) {
     if (it >= 2) {
-      BPD_CUDA(cudaEventSynchronize(s->ev_flag[(it - 2) % 8]));
-      if (s->pinned[(it - 2) % 8]) break;
+      int finished = 0;
+      int rc = wait_pass_flag(s, (it - 2) % 8, &finished);
+      if (rc) return rc;
+      if (finished) break;
     }
     int rc = dispatch_pass(s, a);
     if (rc) return rc;
-    BPD_CUDA(cudaMemcpyAsync(&s->pinned[it % 8], s->st.all_done, sizeof(int), cudaMemcpyDeviceToHost, s->stream));
-    BPD_CUDA(cudaEventRecord(s->ev_flag[it % 8], s->stream));
   }
   return BPD_OK;
 }

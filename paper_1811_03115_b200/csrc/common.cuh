@@ -108,6 +108,9 @@ struct RowState {
   int* out_ids;    // [B][max_tgt]
   int* all_done;   // [1]
   int* error;      // [1] first device-side error code
+  int* signal;     // [2] epoch of the running decode, passes verified in it
+  int* host_flags; // [8] pinned host memory (device address): slot (pass number mod 8) = epoch * 4 + 1, + 1 if all
+                   //     rows are finished; the host reads it instead of waiting for a copy between passes
   long long* stats;  // [0] row_iterations, [1] tokens, [2] iterations, [3] priming passes, [4..4+kMaxK] khat histogram
   const int* page_table;  // [B][pages_per_row]
   int pages_per_row;

@@ -133,6 +133,7 @@ struct bpd_session {
   // host side
   int* pinned;             // pinned ring of all_done flags + staging
   cudaEvent_t ev_flag[8];
+  int epoch;               // decodes started on this session (the verify kernel tags its reports with it)
   cudaEvent_t ev0, ev1;
   int64_t invocations;
   int profiling;

@@ -1132,10 +1132,21 @@ struct VerifyParams {
   RankState rank;                             // top-n only
 };
 
+// Tells the host that one more pass has been verified, and whether every row is finished.
+__device__ __forceinline__ void signal_host(const RowState& st, int done) {
+  const int seq = st.signal[1];
+  st.signal[1] = seq + 1;
+  *reinterpret_cast<volatile int*>(st.host_flags + (seq & 7)) = (st.signal[0] << 2) | (done ? 2 : 1);
+  __threadfence_system();
+}
+
 static __global__ void verify_commit_kernel(VerifyParams p) {
   pdl_launch_dependents();
   pdl_wait();
-  if (*p.st.all_done) return;
+  if (*p.st.all_done) {
+    if (threadIdx.x == 0) signal_host(p.st, 1);
+    return;
+  }
   __shared__ int any_open;
   if (threadIdx.x == 0) any_open = 0;
   __syncthreads();
@@ -1202,6 +1213,7 @@ static __global__ void verify_commit_kernel(VerifyParams p) {
   if (threadIdx.x == 0) {
     p.st.stats[p.mode == kModePrime ? 3 : 2] += 1;
     if (!any_open) *p.st.all_done = 1;
+    signal_host(p.st, !any_open);
   }
 }
 
