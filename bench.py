@@ -111,7 +111,7 @@ class ClockSampler:
     def __enter__(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+                                          "-lms", "50", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
         except OSError:
@@ -253,7 +253,12 @@ def run_gpu(args):
     launches0 = bpd.bpd_kernel_launches()
     with ClockSampler(local) as clocks:
         ms_step = max_over_ranks(timed_decodes(args.steps, "block"), dev)
-    launches = bpd.bpd_kernel_launches() - launches0
+        launches = bpd.bpd_kernel_launches() - launches0
+        # the timed region is a fraction of a second: keep the same load running (untimed) until nvidia-smi has
+        # delivered a few samples, so that the clock record describes the GPU under this very workload
+        # (the same count on every rank: ms_step is already the maximum over ranks)
+        for _ in range(int(min(200, max(1, 600.0 / max(ms_step, 1e-3) / max(1, args.steps))))):
+            timed_decodes(args.steps, "block")
     ids, _, st = sess.bpd_fetch_output(N)
     assert np.array_equal(ids, g_ids), "controlled-acceptance decode differs from greedy"
     assert st.row_iterations == len(khats)
