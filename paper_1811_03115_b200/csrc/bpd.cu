@@ -1001,6 +1001,7 @@ int bpd_session_destroy(bpd_session* s) {
   prof_clear(s);
   for (auto& kv : s->graphs)
     if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
+  if (s->enc_graph.exec) cudaGraphExecDestroy(s->enc_graph.exec);
   if (s->pinned) cudaFreeHost(s->pinned);
   for (int i = 0; i < 8; ++i) cudaEventDestroy(s->ev_flag[i]);
   cudaEventDestroy(s->ev0);
@@ -1031,7 +1032,32 @@ int bpd_encode(bpd_session* s, const int32_t* src_ids, const int32_t* src_len) {
   reset_rows_kernel<<<1, 32 * ceil_div(B, 32), 0, s->stream>>>(rp);
   ++g_launches;
   BPD_CUDA(cudaStreamSynchronize(s->stream));   // host vectors go out of scope
-  int rc = s->tc ? run_encoder_tc(s) : ((c.dtype == 0) ? run_encoder<float>(s) : run_encoder<bf16>(s));
+  int rc = BPD_OK;
+  auto eager = [&]() { return s->tc ? run_encoder_tc(s) : ((c.dtype == 0) ? run_encoder<float>(s) : run_encoder<bf16>(s)); };
+  GraphEntry& ge = s->enc_graph;
+  if (s->profiling || !s->use_graphs || !s->tc) {
+    rc = eager();
+  } else if (ge.exec) {
+    BPD_CUDA(cudaGraphLaunch(ge.exec, s->stream));
+    g_launches += ge.launches;
+  } else if (ge.uses++ == 0) {
+    rc = eager();                              // also creates tensor maps and sets kernel attributes
+  } else {
+    const long long before = g_launches.load();
+    BPD_CUDA(cudaStreamBeginCapture(s->stream, cudaStreamCaptureModeThreadLocal));
+    rc = eager();
+    cudaGraph_t graph = nullptr;
+    const cudaError_t e = cudaStreamEndCapture(s->stream, &graph);
+    if (rc) { if (graph) cudaGraphDestroy(graph); return rc; }
+    if (e != cudaSuccess || !graph) return fail(BPD_E_CUDA, "stream capture of the encoder failed: %s", cudaGetErrorString(e));
+    ge.launches = g_launches.load() - before;
+    g_launches -= ge.launches;
+    const cudaError_t e2 = cudaGraphInstantiate(&ge.exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (e2 != cudaSuccess) { ge.exec = nullptr; return fail(BPD_E_CUDA, "cudaGraphInstantiate failed: %s", cudaGetErrorString(e2)); }
+    BPD_CUDA(cudaGraphLaunch(ge.exec, s->stream));
+    g_launches += ge.launches;
+  }
   if (rc) return rc;
   s->phase = kPhaseEncoded; s->plan_len = 0; s->plan_k = 0; s->invocations = 0;
   return BPD_OK;

@@ -147,5 +147,6 @@ struct bpd_session {
   float* fused_ws;
   unsigned* fused_counters;
   std::map<GraphKey, GraphEntry> graphs;
+  GraphEntry enc_graph;    // the encoder's launch sequence (fixed for a session), captured on its second use
   std::vector<cudaEvent_t> prof_begin[kProfSlots], prof_end[kProfSlots];
 };
