@@ -531,7 +531,12 @@ static int run_layers_fused(bpd_session* s, const PassArgs& a) {
   const bool pdl = s->use_pdl != 0;
   const int nt = (R + 7) / 8;
   // encoder keys / values of a head are staged in shared memory when all sequences' rows fit a small budget
-  const int cross_smax = (s->B * s->max_src * fused::kCrossRowBytes <= fused::kCrossStageMax && !getenv("BPD_NO_CROSS_STAGE")) ? s->max_src : 0;
+  // (24 KB keep the three kernels of a big model co-resident on an SM; a model whose attention launches leave half
+  // the SMs free may take up to 160 KB for it)
+  const size_t cross_bytes = (size_t)s->B * s->max_src * fused::kCrossRowBytes;
+  const bool cross_fits = cross_bytes <= (size_t)fused::kCrossStageMax ||
+                          (c.H * fused::kC <= 74 && cross_bytes + fused::attn_layout<false>(d, nt, 0, 0).total <= 160 * 1024);
+  const int cross_smax = (cross_fits && !getenv("BPD_NO_CROSS_STAGE")) ? s->max_src : 0;
   const size_t smem_self = fused::attn_layout<true>(d, nt, s->B * s->ppr).total;
   const size_t smem_cross = fused::attn_layout<false>(d, nt, 0, s->B * cross_smax).total;
   const size_t smem_ffn = fused::ffn_layout(d, nt).total;
