@@ -467,6 +467,7 @@ static int run_encoder_tc(bpd_session* s) {
   cudaStream_t st = s->stream;
   const int E = s->B * s->max_src, d = c.d, f = c.d_ff;
   const tc::Scratch sc = tc_scratch(s);
+  const bool pdl = s->use_pdl != 0;   // every kernel after the first may start while its predecessor ends
   EmbedParams ep;
   memset(&ep, 0, sizeof(ep));
   ep.table = m->src_embed; ep.pe = s->pe; ep.npos = s->npos; ep.x = s->x; ep.rows = E; ep.rows_per_b = s->max_src;
@@ -479,10 +480,10 @@ static int run_encoder_tc(bpd_session* s) {
   auto with_w = [](tc::Operands o, const void* w, int rows) { o.w = w; o.w_rows = rows; return o; };
   for (int l = 0; l < c.n_enc; ++l) {
     const EncLayer& L = m->enc[l];
-    launch_ln<bf16, float>(s->x, L.ln1g, L.ln1b, s->xn, nullptr, E, d, c.eps, nullptr, st, s->pl_xn);
+    launch_ln<bf16, float>(s->x, L.ln1g, L.ln1b, s->xn, nullptr, E, d, c.eps, nullptr, st, s->pl_xn, pdl);
     tc::TcParams pq = tc_params(nullptr, 0, nullptr);
     pq.out_f32 = static_cast<float*>(s->qbuf); pq.ldo = 3 * d;
-    BPD_TRY(tc::launch<tc::kTcF32>(with_w(xn, L.wqkv, 3 * d), 3 * d, d, E, pq, sc, st)); ++g_launches;
+    BPD_TRY(tc::launch<tc::kTcF32>(with_w(xn, L.wqkv, 3 * d), 3 * d, d, E, pq, sc, st, 1, 0, 0, pdl)); ++g_launches;
     AttnParams ap;
     memset(&ap, 0, sizeof(ap));
     ap.q = s->qbuf; ap.ldq = 3 * d; ap.out = s->attn; ap.ldo = d; ap.out_plane = s->pl_attn; ap.rows = E;
@@ -490,24 +491,24 @@ static int run_encoder_tc(bpd_session* s) {
     ap.k = static_cast<float*>(s->qbuf) + d; ap.v = static_cast<float*>(s->qbuf) + 2 * d;
     ap.ldkv = 3 * d; ap.bstride = (long long)s->max_src * 3 * d; ap.paged = 0; ap.st = s->st;
     ap.scale = 1.0f / sqrtf((float)ap.dh); ap.by_rows = (s->B >= 8) ? 1 : 0;
-    launch_attention<float, float>(ap, st);
+    launch_attention<float, float>(ap, st, pdl);
     ++g_launches;
     tc::TcParams po = tc_params(nullptr, 0, nullptr);
     po.out_f32 = s->x; po.ldo = d;
-    BPD_TRY(tc::launch<tc::kTcResidual>(with_w(at, L.wo, d), d, d, E, po, sc, st)); ++g_launches;
-    launch_ln<bf16, float>(s->x, L.ln2g, L.ln2b, s->xn, nullptr, E, d, c.eps, nullptr, st, s->pl_xn);
+    BPD_TRY(tc::launch<tc::kTcResidual>(with_w(at, L.wo, d), d, d, E, po, sc, st, 1, 0, 0, pdl)); ++g_launches;
+    launch_ln<bf16, float>(s->x, L.ln2g, L.ln2b, s->xn, nullptr, E, d, c.eps, nullptr, st, s->pl_xn, pdl);
     tc::TcParams p1 = tc_params(L.b1, 1, nullptr);
     p1.out_hi = static_cast<bf16*>(s->ffh); p1.plane = s->pl_ffh; p1.ldo = f;
-    BPD_TRY(tc::launch<tc::kTcPlanes>(with_w(xn, L.w1, f), f, d, E, p1, sc, st)); ++g_launches;
+    BPD_TRY(tc::launch<tc::kTcPlanes>(with_w(xn, L.w1, f), f, d, E, p1, sc, st, 1, 0, 0, pdl)); ++g_launches;
     tc::TcParams p2 = tc_params(L.b2, 0, nullptr);
     p2.out_f32 = s->x; p2.ldo = d;
-    BPD_TRY(tc::launch<tc::kTcResidual>(with_w(fh, L.w2, d), d, f, E, p2, sc, st)); ++g_launches;
+    BPD_TRY(tc::launch<tc::kTcResidual>(with_w(fh, L.w2, d), d, f, E, p2, sc, st, 1, 0, 0, pdl)); ++g_launches;
   }
-  launch_ln<bf16, float>(s->x, m->enc_lnf_g, m->enc_lnf_b, s->xn, nullptr, E, d, c.eps, nullptr, st, s->pl_xn);
+  launch_ln<bf16, float>(s->x, m->enc_lnf_g, m->enc_lnf_b, s->xn, nullptr, E, d, c.eps, nullptr, st, s->pl_xn, pdl);
   for (int l = 0; l < c.n_dec; ++l) {
     tc::TcParams pk = tc_params(nullptr, 0, nullptr);
     pk.out_f32 = static_cast<float*>(s->crosskv[l]); pk.ldo = 2 * d;
-    BPD_TRY(tc::launch<tc::kTcF32>(with_w(xn, m->dec[l].cwkv, 2 * d), 2 * d, d, E, pk, sc, st)); ++g_launches;
+    BPD_TRY(tc::launch<tc::kTcF32>(with_w(xn, m->dec[l].cwkv, 2 * d), 2 * d, d, E, pk, sc, st, 1, 0, 0, pdl)); ++g_launches;
   }
   BPD_CUDA(cudaGetLastError());
   return BPD_OK;
