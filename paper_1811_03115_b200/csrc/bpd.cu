@@ -461,6 +461,16 @@ static tc::TcParams tc_params(const void* bias, int relu, const int* all_done) {
 
 #define BPD_TRY(expr) do { int rc__ = (expr); if (rc__) return rc__; } while (0)
 
+// The opt-in shared-memory limit of the staged attention kernel grows with the longest source seen so far.
+static int cross_staged_attr(size_t smem) {
+  static size_t most = 0;
+  if (smem > most) {
+    BPD_CUDA(cudaFuncSetAttribute(cross_attention_staged_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    most = smem;
+  }
+  return BPD_OK;
+}
+
 static int run_encoder_tc(bpd_session* s) {
   const bpd_model* m = s->m;
   const Config& c = m->cfg;
@@ -491,7 +501,14 @@ static int run_encoder_tc(bpd_session* s) {
     ap.k = static_cast<float*>(s->qbuf) + d; ap.v = static_cast<float*>(s->qbuf) + 2 * d;
     ap.ldkv = 3 * d; ap.bstride = (long long)s->max_src * 3 * d; ap.paged = 0; ap.st = s->st;
     ap.scale = 1.0f / sqrtf((float)ap.dh); ap.by_rows = (s->B >= 8) ? 1 : 0;
-    launch_attention<float, float>(ap, st, pdl);
+    // many sequences, head width 64: a CTA per (sequence, head) with the sequence's keys and values in shared memory
+    if (ap.by_rows && ap.dh == 64 && cross_staged_smem(s->max_src) <= 160 * 1024 && !getenv("BPD_NO_CROSS_STAGE")) {
+      const size_t smem = cross_staged_smem(s->max_src);
+      BPD_TRY(cross_staged_attr(smem));
+      BPD_CUDA(launch_k(cross_attention_staged_kernel<float>, dim3(s->B * c.H), dim3(kAttnWarps * 32), smem, st, pdl, ap, s->max_src, 0));
+    } else {
+      launch_attention<float, float>(ap, st, pdl);
+    }
     ++g_launches;
     tc::TcParams po = tc_params(nullptr, 0, nullptr);
     po.out_f32 = s->x; po.ldo = d;
@@ -660,13 +677,9 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
     const bool staged_cross = ap.by_rows && ap.dh == 64 && a.kcur <= 16 && cross_staged_smem(s->max_src) <= 160 * 1024 &&
                               !getenv("BPD_NO_CROSS_STAGE");
     if (staged_cross) {
-      static size_t attr = 0;
       const size_t smem = cross_staged_smem(s->max_src);
-      if (smem > attr) {
-        BPD_CUDA(cudaFuncSetAttribute(cross_attention_staged_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        attr = smem;
-      }
-      PROF(kProfCrossAttn, BPD_CUDA(launch_k(cross_attention_staged_kernel<float>, dim3(s->B * c.H), dim3(kAttnWarps * 32), smem, st, pdl, ap, s->max_src)););
+      BPD_TRY(cross_staged_attr(smem));
+      PROF(kProfCrossAttn, BPD_CUDA(launch_k(cross_attention_staged_kernel<float>, dim3(s->B * c.H), dim3(kAttnWarps * 32), smem, st, pdl, ap, s->max_src, 1)););
     } else {
       PROF(kProfCrossAttn, launch_attention<float, float>(ap, st, pdl););
     }

@@ -839,8 +839,10 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_seq_kernel(AttnPara
 constexpr int kXKeyPitch = 64 * 4 + 16;
 constexpr int kXRowBytes = kXKeyPitch + 64 * 4;
 __host__ __device__ inline size_t cross_staged_smem(int max_src) { return (size_t)max_src * kXRowBytes + 16 * 64 * sizeof(float); }
+// kv_static = 0: the keys and values come from the preceding launch (encoder self-attention); they are copied
+// after the wait.  Query rows are taken 16 at a time.
 template <typename QT>
-__global__ void __launch_bounds__(kAttnWarps * 32) cross_attention_staged_kernel(AttnParams p, int max_src) {
+__global__ void __launch_bounds__(kAttnWarps * 32) cross_attention_staged_kernel(AttnParams p, int max_src, int kv_static) {
   extern __shared__ __align__(16) uint8_t xs[];
   uint8_t* kv = xs;
   float* s_q = reinterpret_cast<float*>(xs + (size_t)max_src * kXRowBytes);   // [16][64]
@@ -848,6 +850,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) cross_attention_staged_kernel
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = blockIdx.x / p.H, h = blockIdx.x % p.H;
   const int limit = min(p.limit_b[b], max_src);
+  if (!kv_static) pdl_wait();
   {
     const float* Kg = reinterpret_cast<const float*>(p.k) + (size_t)b * p.bstride + h * 64;
     const float* Vg = reinterpret_cast<const float*>(p.v) + (size_t)b * p.bstride + h * 64;
@@ -859,21 +862,24 @@ __global__ void __launch_bounds__(kAttnWarps * 32) cross_attention_staged_kernel
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
   }
-  pdl_wait();
+  if (kv_static) pdl_wait();
   const bool ended = p.all_done && *p.all_done;
   const int nrows = p.rows_per_b;
+  for (int row0 = 0; row0 < nrows; row0 += 16) {
+  const int ngroup = min(16, nrows - row0);
+  if (row0 > 0) __syncthreads();                       // the previous group's queries have been read
   if (!ended) {
-    for (int idx = threadIdx.x; idx < nrows * 64; idx += blockDim.x) {
-      const int i = idx >> 6, c = idx & 63;
+    for (int idx = threadIdx.x; idx < ngroup * 64; idx += blockDim.x) {
+      const int i = row0 + (idx >> 6), c = idx & 63;
       s_q[idx] = to_f(reinterpret_cast<const QT*>(p.q)[(long long)(b * nrows + i) * p.ldq + h * 64 + c]) * p.scale;
     }
   }
   asm volatile("cp.async.wait_group 0;" ::: "memory");
   __syncthreads();
   if (ended) return;
-  for (int i = warp; i < nrows; i += kAttnWarps) {
+  for (int i = row0 + warp; i < row0 + ngroup; i += kAttnWarps) {
     float m_run = -INFINITY, l_run = 0.f, a0 = 0.f, a1 = 0.f;
-    const float4* qv = reinterpret_cast<const float4*>(s_q + i * 64);
+    const float4* qv = reinterpret_cast<const float4*>(s_q + (i - row0) * 64);
     for (int c0 = 0; c0 < limit; c0 += 32) {
       const int nk = min(32, limit - c0);
       float sc = -INFINITY;
@@ -915,6 +921,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) cross_attention_staged_kernel
         reinterpret_cast<QT*>(p.out)[o] = from_f<QT>(o2[t]);
       }
     }
+  }
   }
 }
 
