@@ -446,6 +446,31 @@ def test_fused_layers_agree_with_kernel_per_projection(bpd, w, monkeypatch):
     model.close()
 
 
+@pytest.mark.parametrize("w", [MIDI, MIDI_BATCH, MINI_BATCH], ids=lambda w: w.name)
+def test_staged_encoder_rows_change_nothing(bpd, w, monkeypatch):
+    """Cross-attention normally reads the encoder's keys and values from shared memory, where they were copied
+    before the dependency wait; sources too long for that are read from L2.  Both routes do the same arithmetic
+    in the same order: same hidden states, logits and ids."""
+    blob, model, src, src_len, om = _setup(bpd, w)
+    k, N = w.cfg.k_model, w.n_decode
+
+    def run():
+        s = bpd.Session(model, w.batch, w.max_src, N)
+        s.bpd_encode(src, src_len)
+        r = s.bpd_iteration(k, N, want_logits=True, want_hidden=True)
+        r = s.bpd_iteration(k, N, want_logits=True, want_hidden=True)
+        hidden, logits = r["hidden"].cpu().numpy().copy(), r["logits"].cpu().numpy().copy()
+        s.bpd_encode(src, src_len)
+        ids, _, _ = s.bpd_decode_blockwise(k, N)
+        s.close()
+        return hidden, logits, ids
+    h_a, l_a, ids_a = run()
+    monkeypatch.setenv("BPD_NO_CROSS_STAGE", "1")
+    h_b, l_b, ids_b = run()
+    assert np.array_equal(h_a, h_b) and np.array_equal(l_a, l_b) and np.array_equal(ids_a, ids_b)
+    model.close()
+
+
 # 1D local attention (query blocks of local_q positions + local_m positions of memory), one model per attention kernel
 _LOC = dict(local_q=8, local_m=20)
 LOCAL_MODELS = [
