@@ -87,7 +87,30 @@ typedef struct {
   int32_t* block;        /* host [B,k]     the proposals this iteration scored                   */
   float*   logits_dev;   /* device [B,k,k,V] fp32 logits of every head at every position, or NULL */
   float*   hidden_dev;   /* device [B,k,d]   fp32 decoder outputs (after the final norm), or NULL  */
+  float*   layers_dev;   /* device [n_dec,B,k,d] fp32 residual stream after every decoder layer
+                            (before the final norm), or NULL; for parity debugging             */
 } bpd_iter_out;
+
+/* Execution strategies a session may use.  They change how the passes are
+ * scheduled on the GPU, never what is computed: every combination decodes the
+ * same tokens (sums are split differently, so hidden states agree to fp32
+ * rounding).  Each field: -1 = the library's choice for this model and batch,
+ * 0 = off, 1 = on where the shapes allow it.  Initialise with
+ * bpd_session_options_init and change what you need. */
+typedef struct {
+  int32_t struct_bytes;       /* sizeof(bpd_session_options), set by bpd_session_options_init              */
+  int32_t tensor_cores;       /* bf16 models: tcgen05 / TMA projection kernels (0: CUDA-core kernels)       */
+  int32_t cuda_graphs;        /* replay each pass as a CUDA graph (needs a non-default stream)              */
+  int32_t dependent_launch;   /* programmatic dependent launch between the kernels of a pass               */
+  int32_t lazy_heads;         /* two-stage heads: p_1 at all k positions, all heads only at the accepted
+                                 one (default: on when batch * k_model >= 64)                              */
+  int32_t fold_layer_norms;   /* decoder layer norms folded into the projections after them (<= 16 rows)   */
+  int32_t cluster_layers;     /* decoder layers as three cluster launches each (<= 16 rows per pass)        */
+  int32_t persistent_layers;  /* all decoder layers of a pass in one persistent kernel (<= 16 rows per
+                                 pass, d_model 256 / 512 / 1024; takes precedence over cluster_layers)     */
+  int32_t stage_encoder_rows; /* encoder keys / values staged in shared memory for cross-attention          */
+  int32_t l2_stream_hints;    /* weights read once per pass are loaded "evict first"                        */
+} bpd_session_options;
 
 /* ---- set-up ------------------------------------------------------------- */
 
@@ -111,6 +134,17 @@ int bpd_load_weights(const void* blob, size_t blob_bytes, void* dev_weight_buf, 
  * length, max_tgt the number of decoded tokens per row. */
 int bpd_session_create(const bpd_model* model, int batch, int max_src, int max_tgt,
                        void* dev_session_buf, size_t dev_bytes, void* cuda_stream, bpd_session** out);
+
+/* The same with explicit options (NULL = all defaults).  A session that runs
+ * its decoder layers in the persistent kernel (persistent_layers) occupies
+ * most of the GPU with CTAs that wait for one another: passes of two such
+ * sessions must not overlap on one GPU (keep them on one stream, or finish
+ * one decode before starting another); if they do, their bounded waits expire
+ * and the calls return BPD_E_TIMEOUT. */
+void bpd_session_options_init(bpd_session_options* options);
+int bpd_session_create_opt(const bpd_model* model, int batch, int max_src, int max_tgt,
+                           void* dev_session_buf, size_t dev_bytes, void* cuda_stream,
+                           const bpd_session_options* options, bpd_session** out);
 
 int bpd_session_destroy(bpd_session* s);
 int bpd_model_destroy(bpd_model* m);

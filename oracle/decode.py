@@ -232,5 +232,12 @@ class TransformerScorer:
         self.last_logits = head_logits(self.m, h, self.k)
         return self.last_logits
 
+    def layer_outputs(self, dec_inputs: Sequence[int], n_new: int) -> np.ndarray:
+        """Residual stream after every decoder layer for the last ``n_new`` inputs, [n_dec, n_new, d]
+        (uncached forward; for comparing intermediates)."""
+        trace: list = []
+        decoder_full(self.m, self.memory, self.src_len, dec_inputs, trace)
+        return np.stack([x[-n_new:] for x in trace])
+
     def __call__(self, dec_inputs: Sequence[int], n_new: int) -> np.ndarray:
         return argmax_lowest(self.logits(dec_inputs, n_new))

@@ -151,7 +151,7 @@ def encode(m: OracleModel, src_ids, src_len: Optional[int] = None) -> np.ndarray
 def self_attention_allowed(m: OracleModel, query_pos: np.ndarray, n_keys: int) -> np.ndarray:
     """Which keys (positions 0..n_keys-1) each decoder query may attend to.
 
-    Causal: key j <= query position t.  With 1D local attention (Section 7.3
+    Causal: key j <= query position t.  With 1D local attention (Section 7.2
     names it for the super-resolution model; the block lengths are this
     build's choice, carried in the blob header) the target sequence is cut
     into query blocks of local_q positions, and a query also sees only the
@@ -164,10 +164,11 @@ def self_attention_allowed(m: OracleModel, query_pos: np.ndarray, n_keys: int) -
     return ok
 
 
-def decoder_full(m: OracleModel, memory: np.ndarray, src_len: int, dec_inputs) -> np.ndarray:
+def decoder_full(m: OracleModel, memory: np.ndarray, src_len: int, dec_inputs, trace: Optional[list] = None) -> np.ndarray:
     """Uncached decoder: final-layer-norm output h [n, d] for decoder inputs
     u_0..u_{n-1} (position of u_t is t).  Causal self-attention, cross-attention
-    over memory rows < src_len."""
+    over memory rows < src_len.  ``trace``, if given, receives a copy of the
+    residual stream [n, d] after every layer (for comparing intermediates)."""
     w = m.w
     n = len(dec_inputs)
     S = memory.shape[0]
@@ -187,6 +188,8 @@ def decoder_full(m: OracleModel, memory: np.ndarray, src_len: int, dec_inputs) -
         x = x + a @ w[p + ".cross.wo"].T
         y = layer_norm(x, w[p + ".ln3.g"], w[p + ".ln3.b"], m.eps)
         x = x + ffn(y, w[p + ".ffn.w1"], w[p + ".ffn.b1"], w[p + ".ffn.w2"], w[p + ".ffn.b2"])
+        if trace is not None:
+            trace.append(x.copy())
     return layer_norm(x, w["dec.lnf.g"], w["dec.lnf.b"], m.eps)
 
 

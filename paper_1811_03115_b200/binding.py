@@ -36,7 +36,15 @@ class bpd_stats(C.Structure):
 class bpd_iter_out(C.Structure):
     _fields_ = [("khat", C.c_void_p), ("accepted", C.c_void_p), ("table", C.c_void_p),
                 ("next_block", C.c_void_p), ("block", C.c_void_p), ("logits_dev", C.c_void_p),
-                ("hidden_dev", C.c_void_p)]
+                ("hidden_dev", C.c_void_p), ("layers_dev", C.c_void_p)]
+
+
+OPTION_FIELDS = ("tensor_cores", "cuda_graphs", "dependent_launch", "lazy_heads", "fold_layer_norms", "cluster_layers",
+                 "persistent_layers", "stage_encoder_rows", "l2_stream_hints")
+
+
+class bpd_session_options(C.Structure):
+    _fields_ = [("struct_bytes", C.c_int32)] + [(name, C.c_int32) for name in OPTION_FIELDS]
 
 
 if not os.path.exists(LIB_PATH):
@@ -51,6 +59,8 @@ _SIGS = {
     "bpd_session_bytes": (_i, [_vp, _i, _i, _i, C.POINTER(_sz)]),
     "bpd_load_weights": (_i, [_vp, _sz, _vp, _sz, _vp, C.POINTER(_vp)]),
     "bpd_session_create": (_i, [_vp, _i, _i, _i, _vp, _sz, _vp, C.POINTER(_vp)]),
+    "bpd_session_options_init": (None, [C.POINTER(bpd_session_options)]),
+    "bpd_session_create_opt": (_i, [_vp, _i, _i, _i, _vp, _sz, _vp, C.POINTER(bpd_session_options), C.POINTER(_vp)]),
     "bpd_session_destroy": (_i, [_vp]),
     "bpd_model_destroy": (_i, [_vp]),
     "bpd_encode": (_i, [_vp, _vp, _vp]),
@@ -156,10 +166,17 @@ class Model:
 
 
 class Session:
-    """bpd_session_create and the calls that take a session."""
+    """bpd_session_create_opt and the calls that take a session.  ``options`` maps the field names of
+    bpd_session_options to 0 / 1 (anything left out keeps the library's default)."""
 
-    def __init__(self, model: Model, batch: int, max_src: int, max_tgt: int):
+    def __init__(self, model: Model, batch: int, max_src: int, max_tgt: int, options: Optional[dict] = None):
         import torch
+        opt = bpd_session_options()
+        lib.bpd_session_options_init(C.byref(opt))
+        for name, value in (options or {}).items():
+            if name not in OPTION_FIELDS:
+                raise ValueError(f"unknown session option {name!r}")
+            setattr(opt, name, int(value))
         self.model, self.B, self.max_src, self.max_tgt = model, batch, max_src, max_tgt
         nb = _sz(0)
         _check(lib.bpd_session_bytes(model.handle, batch, max_src, max_tgt, C.byref(nb)))
@@ -171,8 +188,8 @@ class Session:
             self.stream = torch.cuda.Stream(device=model.device)
             self.stream.wait_stream(torch.cuda.current_stream())
             self.handle = _vp(0)
-            _check(lib.bpd_session_create(model.handle, batch, max_src, max_tgt, self.buf.data_ptr(), sb,
-                                          self.stream.cuda_stream, C.byref(self.handle)))
+            _check(lib.bpd_session_create_opt(model.handle, batch, max_src, max_tgt, self.buf.data_ptr(), sb,
+                                              self.stream.cuda_stream, C.byref(opt), C.byref(self.handle)))
         self.session_bytes = sb
 
     def close(self):
@@ -229,7 +246,7 @@ class Session:
         _check(lib.bpd_set_forced_plan(self.handle, _ptr(p), p.shape[1], k))
 
     def bpd_iteration(self, k: int, max_new: int, eos_id: int = -1, forced_tail=None, accept_mode: int = 0,
-                      want_logits: bool = False, want_hidden: bool = False):
+                      want_logits: bool = False, want_hidden: bool = False, want_layers: bool = False):
         import torch
         B = self.B
         out = bpd_iter_out()
@@ -240,8 +257,11 @@ class Session:
         blk = np.empty((B, k), np.int32)
         out.khat, out.accepted, out.table, out.next_block, out.block = (_ptr(khat), _ptr(acc), _ptr(table),
                                                                         _ptr(nxt), _ptr(blk))
-        logits = hidden = None
+        logits = hidden = layers = None
         V, d = self.vocab, self.d_model
+        if want_layers:
+            layers = torch.empty((self.n_dec, B, k, d), dtype=torch.float32, device=self.model.device)
+            out.layers_dev = layers.data_ptr()
         if want_logits:
             logits = torch.empty((B, k, k, V), dtype=torch.float32, device=self.model.device)
             out.logits_dev = logits.data_ptr()
@@ -255,7 +275,13 @@ class Session:
             res["logits"] = logits
         if hidden is not None:
             res["hidden"] = hidden
+        if layers is not None:
+            res["layers"] = layers
         return res
+
+    @property
+    def n_dec(self) -> int:
+        return int(np.frombuffer(self.model.blob_header[20:24], np.int32)[0])
 
     @property
     def vocab(self) -> int:

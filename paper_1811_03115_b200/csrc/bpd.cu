@@ -7,12 +7,16 @@
 
 #include <algorithm>
 #include <atomic>
+#include <map>
+#include <mutex>
 #include <new>
+#include <utility>
 
 #include "host.hpp"
 #include "kernels_simt.cuh"
 #include "tc_host.hpp"
 #include "fused_layer.cuh"
+#include "layer_stack.cuh"
 
 namespace bpd {
 
@@ -24,6 +28,20 @@ int fail(int code, const char* fmt, ...) {
   vsnprintf(g_err, sizeof(g_err), fmt, ap);
   va_end(ap);
   return code;
+}
+
+int ensure_smem_limit(const void* kernel, size_t bytes) {
+  static std::mutex mu;
+  static std::map<std::pair<int, const void*>, size_t> most;
+  int dev = 0;
+  BPD_CUDA(cudaGetDevice(&dev));
+  std::lock_guard<std::mutex> lock(mu);
+  size_t& cur = most[std::make_pair(dev, kernel)];
+  if (bytes > cur) {
+    BPD_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+    cur = bytes;
+  }
+  return BPD_OK;
 }
 
 static inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
@@ -206,7 +224,13 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
   const size_t fused_parts = std::max<size_t>(c.H, c.d_ff / (fused::kC * fused::kHS));
   float* fused_ws = a.take<float>(fused_ok ? fused_parts * Rmax * d : 0);
   unsigned* fused_counters = a.take<unsigned>(fused::kC);
+  // persistent layer stack: tensor maps, per-layer pointers, the clusters' partial outputs, the join's words
+  void* stack_maps = a.take_bytes(fused_ok ? (size_t)c.n_dec * stack::kMapsPerLayer * sizeof(CUtensorMap) : 0);
+  void* stack_layers = a.take_bytes(fused_ok ? (size_t)c.n_dec * sizeof(stack::LayerPtrs) : 0);
+  float* stack_ws = a.take<float>(fused_ok ? (size_t)2 * c.H * fused::kMaxRows * d : 0);
+  unsigned* stack_bar = a.take<unsigned>(stack::kBarWords);
   if (s) {
+    s->stack_maps = stack_maps; s->stack_layers = stack_layers; s->stack_ws = stack_ws; s->stack_bar = stack_bar;
     s->fused_ws = fused_ws; s->fused_counters = fused_counters;
     s->x = x; s->h_f32 = h_f32; s->xn = xn; s->qbuf = qbuf; s->attn = attn; s->ffh = ffh; s->u = u; s->o = o;
     s->crosskv = crosskv; s->kcache = kc; s->vcache = vc; s->st = st; s->src_dev = src_dev;
@@ -332,6 +356,7 @@ struct PassArgs {
   int accept_kind = kAcceptExact;   // Verify criterion, its parameter (n or eps), forced minimum block size
   int accept_param = 0;
   int min_block = 1;
+  float* layer_dump = nullptr;   // device [n_dec, B*kcur, d] or null: the residual stream after every decoder layer
 };
 
 // accept_mode of the public calls: bits 0-7 parameter, bits 8-15 criterion, bits 16-23 minimum block size
@@ -402,6 +427,8 @@ static int run_pass(bpd_session* s, const PassArgs& a) {
     launch_ln<WT, float>(s->x, L.ln3g, L.ln3b, s->xn, nullptr, R, d, c.eps, done, st);
     launch_linear<WT, float, kEpiStoreAct>(lin(s->xn, d, L.w1, d, c.d_ff, L.b1, R, s->ffh, c.d_ff, 1, done), 1, st);
     launch_linear<WT, float, kEpiResidual>(lin(s->ffh, c.d_ff, L.w2, c.d_ff, d, L.b2, R, s->x, d, 0, done), 1, st);
+    if (a.layer_dump)
+      BPD_CUDA(cudaMemcpyAsync(a.layer_dump + (size_t)l * R * d, s->x, sizeof(float) * R * d, cudaMemcpyDeviceToDevice, st));
   }
   launch_ln<WT, float>(s->x, m->dec_lnf_g, m->dec_lnf_b, s->xn, s->h_f32, R, d, c.eps, done, st);
   prof_mark(s, kProfLayers, 1);
@@ -449,6 +476,7 @@ static tc::Scratch tc_scratch(bpd_session* s) {
   sc.done_counter = s->tc_done; sc.best = s->tc_best; sc.best_elems = s->tc_best_elems;
   sc.error = s->st.error;
   sc.wide_ttiles = session_wide_ttiles(s->m->cfg, s->B);
+  sc.l2_hints = s->opt.l2_stream_hints;
   return sc;
 }
 
@@ -463,12 +491,7 @@ static tc::TcParams tc_params(const void* bias, int relu, const int* all_done) {
 
 // The opt-in shared-memory limit of the staged attention kernel grows with the longest source seen so far.
 static int cross_staged_attr(size_t smem) {
-  static size_t most = 0;
-  if (smem > most) {
-    BPD_CUDA(cudaFuncSetAttribute(cross_attention_staged_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    most = smem;
-  }
-  return BPD_OK;
+  return ensure_smem_limit(reinterpret_cast<const void*>(cross_attention_staged_kernel<float>), smem);
 }
 
 static int run_encoder_tc(bpd_session* s) {
@@ -502,7 +525,7 @@ static int run_encoder_tc(bpd_session* s) {
     ap.ldkv = 3 * d; ap.bstride = (long long)s->max_src * 3 * d; ap.paged = 0; ap.st = s->st;
     ap.scale = 1.0f / sqrtf((float)ap.dh); ap.by_rows = (s->B >= 8) ? 1 : 0;
     // many sequences, head width 64: a CTA per (sequence, head) with the sequence's keys and values in shared memory
-    if (ap.by_rows && ap.dh == 64 && cross_staged_smem(s->max_src) <= 160 * 1024 && !getenv("BPD_NO_CROSS_STAGE")) {
+    if (ap.by_rows && ap.dh == 64 && cross_staged_smem(s->max_src) <= 160 * 1024 && s->opt.stage_encoder_rows) {
       const size_t smem = cross_staged_smem(s->max_src);
       BPD_TRY(cross_staged_attr(smem));
       BPD_CUDA(launch_k(cross_attention_staged_kernel<float>, dim3(s->B * c.H), dim3(kAttnWarps * 32), smem, st, pdl, ap, s->max_src, 0));
@@ -534,8 +557,7 @@ static int run_encoder_tc(bpd_session* s) {
 // ------------------------------------------------------------------ fused decoder layers (few rows per pass)
 template <typename P>
 static int fused_attr(void (*kernel)(P), size_t smem) {
-  BPD_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  return BPD_OK;
+  return ensure_smem_limit(reinterpret_cast<const void*>(kernel), smem);
 }
 
 // Embedding, then three launches per decoder layer (self-attention block, cross-attention block, feed-forward
@@ -554,13 +576,12 @@ static int run_layers_fused(bpd_session* s, const PassArgs& a) {
   const size_t cross_bytes = (size_t)s->B * s->max_src * fused::kCrossRowBytes;
   const bool cross_fits = cross_bytes <= (size_t)fused::kCrossStageMax ||
                           (c.H * fused::kC <= 74 && cross_bytes + fused::attn_layout<false>(d, nt, 0, 0).total <= 160 * 1024);
-  const int cross_smax = (cross_fits && !getenv("BPD_NO_CROSS_STAGE")) ? s->max_src : 0;
+  const int cross_smax = (cross_fits && s->opt.stage_encoder_rows) ? s->max_src : 0;
   const size_t smem_self = fused::attn_layout<true>(d, nt, s->B * s->ppr).total;
   const size_t smem_cross = fused::attn_layout<false>(d, nt, 0, s->B * cross_smax).total;
   const size_t smem_ffn = fused::ffn_layout(d, nt).total;
   // the opt-in shared-memory limit of each kernel grows with the widest model seen so far
-  static size_t attr_max[3][3] = {{0, 0, 0}, {0, 0, 0}, {0, 0, 0}};
-  if (smem_self > attr_max[nt][0] || smem_cross > attr_max[nt][1] || smem_ffn > attr_max[nt][2]) {
+  {
     if (nt == 1) {
       BPD_TRY(fused_attr(fused::attn_block_kernel<true, 1>, smem_self));
       BPD_TRY(fused_attr(fused::attn_block_kernel<false, 1>, smem_cross));
@@ -570,7 +591,6 @@ static int run_layers_fused(bpd_session* s, const PassArgs& a) {
       BPD_TRY(fused_attr(fused::attn_block_kernel<false, 2>, smem_cross));
       BPD_TRY(fused_attr(fused::ffn_block_kernel<2>, smem_ffn));
     }
-    attr_max[nt][0] = smem_self; attr_max[nt][1] = smem_cross; attr_max[nt][2] = smem_ffn;
   }
   EmbedParams ep;
   memset(&ep, 0, sizeof(ep));
@@ -616,7 +636,176 @@ static int run_layers_fused(bpd_session* s, const PassArgs& a) {
       BPD_CUDA(launch_k(fused::ffn_block_kernel<2>, grid_ffn, block, smem_ffn, st, pdl, pf));
     }
     g_launches += 3;
+    if (a.layer_dump)
+      BPD_CUDA(cudaMemcpyAsync(a.layer_dump + (size_t)l * R * d, s->x, sizeof(float) * R * d, cudaMemcpyDeviceToDevice, st));
   }
+  return BPD_OK;
+}
+
+// ------------------------------------------------------------------ persistent layer stack (few rows per pass)
+// Shared-memory plan of the persistent kernel for a session whose widest pass has `rows` rows; `budget` bytes per
+// CTA.  Returns false when the working buffers and a ring that holds at least the two largest tiles do not fit.
+static bool stack_plan(const Config& c, int rows, int nb, int ppr, int cross_rows, bool long_seq, size_t budget,
+                       stack::Layout* out) {
+  const int NT = rows > 8 ? 2 : 1, RP = NT * 8;
+  const stack::Geo g = stack::make_geo(c.d, c.H, c.d_ff, c.n_dec, cross_rows);
+  auto up = [](size_t v, size_t a) { return (v + a - 1) / a * a; };
+  size_t off = 0;
+  stack::Layout L;
+  memset(&L, 0, sizeof(L));
+  auto take = [&](size_t bytes) { const size_t at = off; off = up(off + bytes, 128); return (int)at; };
+  L.x = take((size_t)RP * g.ks * 4);
+  L.xh = take((size_t)RP * g.ks * 2);
+  L.xl = take((size_t)RP * g.ks * 2);
+  L.oh = take((size_t)RP * 128);
+  L.ol = take((size_t)RP * 128);
+  L.hh = take((size_t)g.PH * RP * 128);
+  L.hl = take((size_t)g.PH * RP * 128);
+  L.inbox = take(std::max((size_t)fused::kC * NT * 3 * fused::kDH * 4, (size_t)fused::kC * g.UPR * RP * 4));
+  L.q = take((size_t)RP * fused::kDH * 4);
+  L.stats = take((size_t)fused::kC * fused::kMaxRows * 2 * 4 + 4 * fused::kMaxRows * 4);
+  L.attn = take(sizeof(AttnSmem<fused::kDH, stack::kWarps>));
+  L.wst = take((size_t)stack::kWarps * NT * fused::kPartial * 4);
+  const size_t lvl = long_seq ? (size_t)fused::kC * rows * fused::kPartial * 4 : 0;
+  L.lvl1 = take(lvl);
+  L.lvl2 = take(lvl);
+  L.pt = take((size_t)nb * ppr * 4);
+  L.layers = take((size_t)c.n_dec * sizeof(stack::LayerPtrs));
+  L.misc = take(sizeof(stack::Ctl));
+  const size_t work = off;
+  int largest = 0, second = 0, per_layer = 0;
+  for (int i = 0; i < g.ntl; ++i) {
+    const int b = stack::tile_bytes(g, i, cross_rows);
+    per_layer += b;
+    if (b > largest) { second = largest; largest = b; } else if (b > second) second = b;
+  }
+  if (work + 1024 > budget) return false;
+  size_t ring = std::min((budget - work) / 1024 * 1024, (size_t)per_layer * c.n_dec);
+  if (ring < (size_t)largest + second) return false;
+  L.ring_bytes = (int)ring;
+  int* fields[] = {&L.x, &L.xh, &L.xl, &L.oh, &L.ol, &L.hh, &L.hl, &L.inbox, &L.q, &L.stats, &L.attn, &L.wst, &L.lvl1,
+                   &L.lvl2, &L.pt, &L.layers, &L.misc};
+  for (int* f : fields) *f += (int)ring;
+  L.total = (int)(ring + work);
+  *out = L;
+  return true;
+}
+
+template <int NT>
+static int stack_clusters(size_t smem, int H, int* out) {
+  BPD_TRY(ensure_smem_limit(reinterpret_cast<const void*>(stack::layer_stack_kernel<NT>), smem));
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(fused::kC, H); cfg.blockDim = dim3(stack::kThreads); cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = fused::kC; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  BPD_CUDA(cudaOccupancyMaxActiveClusters(out, stack::layer_stack_kernel<NT>, &cfg));
+  return BPD_OK;
+}
+
+// Shapes the persistent kernel is built for.
+static bool stack_shapes_ok(const Config& c, int rows) {
+  const int d = c.d, H = c.H;
+  if (c.dtype != 1 || H < 1 || d != H * fused::kDH || (d != 256 && d != 512 && d != 1024)) return false;
+  if (c.d_ff % H || (c.d_ff / H) % 64 || c.d_ff / H > 256) return false;
+  if (rows < 1 || rows > fused::kMaxRows || c.n_dec > 64) return false;
+  return true;
+}
+
+// Decides whether the session runs its decoder layers in the persistent kernel and prepares what it needs:
+// a shared-memory plan under which all H clusters are resident at once, tensor maps and per-layer pointers.
+static int stack_setup(bpd_session* s) {
+  const bpd_model* m = s->m;
+  const Config& c = m->cfg;
+  s->stack = 0;
+  const int rows = s->B * c.k_model;
+  if (!s->tc || !s->opt.persistent_layers || !stack_shapes_ok(c, rows)) return BPD_OK;
+  const bool long_seq = s->max_tgt + 1 + c.k_model > 32 * fused::kC;
+  cudaDeviceProp prop;
+  int dev = 0;
+  BPD_CUDA(cudaGetDevice(&dev));
+  BPD_CUDA(cudaGetDeviceProperties(&prop, dev));
+  const size_t optin = prop.sharedMemPerBlockOptin, per_sm = prop.sharedMemPerMultiprocessor;
+  // one CTA per SM, or two (each block also reserves 1 KB of the SM's shared memory)
+  const size_t budgets[2] = {optin, std::min(optin, per_sm / 2 - 1024)};
+  stack::Layout lay;
+  bool ok = false;
+  int cross_rows = 0;
+  for (size_t budget : budgets) {
+    for (int staged = 1; staged >= 0 && !ok; --staged) {
+      cross_rows = (staged && s->B * s->max_src <= 256) ? s->B * s->max_src : 0;
+      if (staged && !cross_rows) continue;
+      if (budget <= 1024 || !stack_plan(c, rows, s->B, s->ppr, cross_rows, long_seq, budget - 1024, &lay)) continue;
+      lay.total += 1024;                       // slack for aligning the ring to 1024 bytes
+      int n1 = 0, n2 = 0;
+      BPD_TRY(stack_clusters<1>((size_t)lay.total, c.H, &n1));
+      BPD_TRY(stack_clusters<2>((size_t)lay.total, c.H, &n2));
+      ok = n1 >= c.H && n2 >= c.H;
+    }
+    if (ok) break;
+  }
+  if (!ok) return BPD_OK;
+  // tensor maps: weight slices as boxes of 64 (32 for d_model 256) reduction columns, encoder keys / values
+  const stack::Geo g = stack::make_geo(c.d, c.H, c.d_ff, c.n_dec, cross_rows);
+  std::vector<CUtensorMap> maps((size_t)c.n_dec * stack::kMapsPerLayer);
+  std::vector<stack::LayerPtrs> lp(c.n_dec);
+  const int d = c.d, f = c.d_ff;
+  for (int l = 0; l < c.n_dec; ++l) {
+    const DecLayer& L = m->dec[l];
+    CUtensorMap* mp = &maps[(size_t)l * stack::kMapsPerLayer];
+    BPD_TRY(tc::make_map_2d(L.wqkv, 2, 3 * d, d, d, g.PW, 64, true, mp + stack::kMapQkv));
+    BPD_TRY(tc::make_map_2d(L.wo, 2, d, d, d, 64, g.ks, true, mp + stack::kMapWo));
+    BPD_TRY(tc::make_map_2d(L.cwq, 2, d, d, d, g.PW, 64, true, mp + stack::kMapCq));
+    BPD_TRY(tc::make_map_2d(L.cwo, 2, d, d, d, 64, g.ks, true, mp + stack::kMapCwo));
+    BPD_TRY(tc::make_map_2d(L.w1, 2, f, d, d, g.PW, g.HCt, true, mp + stack::kMapW1));
+    BPD_TRY(tc::make_map_2d(L.w2, 2, d, f, f, 64, g.ks, true, mp + stack::kMapW2));
+    const int er = std::max(cross_rows, 1);
+    BPD_TRY(tc::make_map_2d(s->crosskv[l], 4, (uint64_t)s->B * s->max_src, 2 * d, 2 * d, 32, er, true, mp + stack::kMapCk));
+    BPD_TRY(tc::make_map_2d(s->crosskv[l], 4, (uint64_t)s->B * s->max_src, 2 * d, 2 * d, 64, er, false, mp + stack::kMapCv));
+    stack::LayerPtrs& P = lp[l];
+    P.g1 = static_cast<const bf16*>(L.ln1g); P.g2 = static_cast<const bf16*>(L.ln2g); P.g3 = static_cast<const bf16*>(L.ln3g);
+    P.s_qkv = L.s_qkv; P.c_qkv = L.c_qkv; P.s_cq = L.s_cq; P.c_cq = L.c_cq; P.s_f1 = L.s_f1; P.c_f1 = L.c_f1;
+    P.b2 = static_cast<const bf16*>(L.b2);
+    P.kcache = static_cast<bf16*>(s->kcache[l]); P.vcache = static_cast<bf16*>(s->vcache[l]);
+    P.crosskv = static_cast<const float*>(s->crosskv[l]);
+  }
+  BPD_CUDA(cudaMemcpyAsync(s->stack_maps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, s->stream));
+  BPD_CUDA(cudaMemcpyAsync(s->stack_layers, lp.data(), lp.size() * sizeof(stack::LayerPtrs), cudaMemcpyHostToDevice, s->stream));
+  BPD_CUDA(cudaStreamSynchronize(s->stream));
+  static_assert(sizeof(stack::Layout) <= sizeof(s->stack_layout), "layout does not fit its opaque copy");
+  memcpy(s->stack_layout, &lay, sizeof(lay));
+  s->stack_cross_rows = cross_rows; s->stack_long = long_seq ? 1 : 0;
+  s->stack = 1;
+  return BPD_OK;
+}
+
+// Embedding, all decoder layers and the final layer norm in one launch; leaves the planes of the decoder output in
+// s->xn and its fp32 copy in s->h_f32 like the layer-by-layer paths followed by the layer-norm kernel.
+static int run_layers_stack(bpd_session* s, const PassArgs& a) {
+  const bpd_model* m = s->m;
+  const Config& c = m->cfg;
+  stack::StackParams p;
+  memset(&p, 0, sizeof(p));
+  p.maps = static_cast<const CUtensorMap*>(s->stack_maps);
+  p.layers = static_cast<const stack::LayerPtrs*>(s->stack_layers);
+  p.L = c.n_dec; p.d = c.d; p.H = c.H; p.ff = c.d_ff; p.R = s->B * a.kcur; p.rows_per_b = a.kcur; p.nb = s->B; p.eps = c.eps;
+  p.tgt_embed = static_cast<const bf16*>(m->tgt_embed); p.pe = s->pe; p.npos = s->npos; p.vocab = c.V;
+  p.st = s->st; p.forced = a.forced; p.forced_rows = a.forced_rows; p.kforced = a.kforced;
+  p.local_q = c.local_q; p.local_m = c.local_m; p.max_src = s->max_src; p.scale = 1.0f / sqrtf((float)fused::kDH);
+  p.cross_rows = s->stack_cross_rows; p.long_seq = s->stack_long;
+  p.lnf_g = static_cast<const bf16*>(m->dec_lnf_g); p.lnf_b = static_cast<const bf16*>(m->dec_lnf_b);
+  p.xn_hi = static_cast<bf16*>(s->xn); p.xn_plane = s->pl_xn; p.h_f32 = s->h_f32;
+  p.layer_dump = a.layer_dump;
+  p.ws = s->stack_ws; p.bar = s->stack_bar; p.error = s->st.error; p.all_done = s->st.all_done;
+  p.spin = stack::kSpin;
+  memcpy(&p.lay, s->stack_layout, sizeof(p.lay));
+  const dim3 grid(fused::kC, c.H), block(stack::kThreads);
+  const bool pdl = s->use_pdl != 0;
+  if (p.R > 8) BPD_CUDA(launch_k(stack::layer_stack_kernel<2>, grid, block, (size_t)p.lay.total, s->stream, pdl, p));
+  else BPD_CUDA(launch_k(stack::layer_stack_kernel<1>, grid, block, (size_t)p.lay.total, s->stream, pdl, p));
+  ++g_launches;
   return BPD_OK;
 }
 
@@ -633,7 +822,8 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   const tc::Operands xn{nullptr, 0, s->xn, s->pl_xn, d, s->rows_all, d};
   auto with_w = [](tc::Operands o, const void* w, int rows) { o.w = w; o.w_rows = rows; return o; };
   prof_mark(s, kProfLayers, 0);
-  if (s->fused) BPD_TRY(run_layers_fused(s, a));
+  if (s->stack) BPD_TRY(run_layers_stack(s, a));
+  else if (s->fused) BPD_TRY(run_layers_fused(s, a));
   else {
   EmbedParams ep;
   memset(&ep, 0, sizeof(ep));
@@ -675,7 +865,7 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
     ap.ldkv = 2 * d; ap.bstride = (long long)s->max_src * 2 * d; ap.paged = 0;
     // many sequences, head width 64: the encoder's keys and values are staged before the dependency wait
     const bool staged_cross = ap.by_rows && ap.dh == 64 && a.kcur <= 16 && cross_staged_smem(s->max_src) <= 160 * 1024 &&
-                              !getenv("BPD_NO_CROSS_STAGE");
+                              s->opt.stage_encoder_rows;
     if (staged_cross) {
       const size_t smem = cross_staged_smem(s->max_src);
       BPD_TRY(cross_staged_attr(smem));
@@ -695,9 +885,11 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
     p2.out_f32 = s->x; p2.ldo = d;
     if (fold && l + 1 < c.n_dec) { p2.g_next = static_cast<const bf16*>(m->dec[l + 1].ln1g); p2.xg_hi = static_cast<bf16*>(s->xn); p2.xg_plane = s->pl_xn; }
     PROF(kProfFfn2, BPD_TRY(tc::launch<tc::kTcResidual>(with_w(fx, L.w2, d), d, f, R, p2, sc, st, 1, 0, 0, pdl)); ++g_launches);
+    if (a.layer_dump)
+      BPD_CUDA(cudaMemcpyAsync(a.layer_dump + (size_t)l * R * d, s->x, sizeof(float) * R * d, cudaMemcpyDeviceToDevice, st));
   }
   }
-  PROF(kProfLn, launch_ln<bf16, float>(s->x, m->dec_lnf_g, m->dec_lnf_b, s->xn, s->h_f32, R, d, c.eps, done, st, s->pl_xn, pdl););
+  if (!s->stack) PROF(kProfLn, launch_ln<bf16, float>(s->x, m->dec_lnf_g, m->dec_lnf_b, s->xn, s->h_f32, R, d, c.eps, done, st, s->pl_xn, pdl););
   prof_mark(s, kProfLayers, 1);
   // proposal heads
   const int fhd = c.d_hidden, km = c.k_model;
@@ -785,7 +977,7 @@ static int dispatch_eager(bpd_session* s, const PassArgs& a) {
 // creates tensor maps and sets kernel attributes), the second captures it into a CUDA graph, later uses replay it.
 static int dispatch_pass(bpd_session* s, const PassArgs& a) {
   s->last_pass_lazy = pass_is_lazy(s, a) ? 1 : 0;
-  if (s->profiling || !s->use_graphs || a.logits_dump) return dispatch_eager(s, a);
+  if (s->profiling || !s->use_graphs || a.logits_dump || a.layer_dump) return dispatch_eager(s, a);
   const GraphKey key(a.mode, a.kcur, a.kh, a.knext, (const void*)a.forced, a.forced_rows, a.kforced, a.max_new, a.eos,
                      (const void*)a.logits_dump, (a.accept_kind << 16) | (a.accept_param << 8) | a.min_block);
   GraphEntry& ge = s->graphs[key];
@@ -822,6 +1014,8 @@ static int check_device_error(bpd_session* s) {
   err = s->pinned[64];
   if (err == 1) return fail(BPD_E_INVALID, "a token id outside the vocabulary reached the decoder");
   if (err >= 101 && err <= 103) return fail(BPD_E_TIMEOUT, "a bounded wait inside the projection kernel expired (code %d)", err);
+  if (err == 104 || err == 105) return fail(BPD_E_TIMEOUT, "a bounded wait inside the persistent layer kernel expired (code %d: %s)", err,
+                                            err == 104 ? "device-wide join" : "weight tile");
   if (err != 0) return fail(BPD_E_CUDA, "device-side error word %d", err);
   return BPD_OK;
 }
@@ -951,9 +1145,30 @@ int bpd_model_destroy(bpd_model* m) {
   return BPD_OK;
 }
 
+void bpd_session_options_init(bpd_session_options* o) {
+  if (!o) return;
+  o->struct_bytes = (int32_t)sizeof(*o);
+  o->tensor_cores = o->cuda_graphs = o->dependent_launch = o->lazy_heads = o->fold_layer_norms = -1;
+  o->cluster_layers = o->persistent_layers = o->stage_encoder_rows = o->l2_stream_hints = -1;
+}
+
 int bpd_session_create(const bpd_model* model, int batch, int max_src, int max_tgt, void* dev_session_buf,
                        size_t dev_bytes, void* cuda_stream, bpd_session** out) {
+  return bpd_session_create_opt(model, batch, max_src, max_tgt, dev_session_buf, dev_bytes, cuda_stream, nullptr, out);
+}
+
+int bpd_session_create_opt(const bpd_model* model, int batch, int max_src, int max_tgt, void* dev_session_buf,
+                           size_t dev_bytes, void* cuda_stream, const bpd_session_options* options, bpd_session** out) {
   if (!out) return fail(BPD_E_INVALID, "out is null");
+  bpd_session_options o;
+  bpd_session_options_init(&o);
+  if (options) {
+    if (options->struct_bytes != (int32_t)sizeof(o)) return fail(BPD_E_INVALID, "bpd_session_options.struct_bytes = %d, this library expects %zu", options->struct_bytes, sizeof(o));
+    o = *options;
+    const int32_t* f = &o.tensor_cores;
+    for (int i = 0; i < 9; ++i)
+      if (f[i] < -1 || f[i] > 1) return fail(BPD_E_INVALID, "session option %d has value %d (want -1, 0 or 1)", i, f[i]);
+  }
   *out = nullptr;
   if (!model || !dev_session_buf) return fail(BPD_E_INVALID, "model or session buffer is null");
   if (batch < 1 || batch > 1024 || max_src < 1 || max_tgt < 1) return fail(BPD_E_INVALID, "batch/max_src/max_tgt out of range");
@@ -965,18 +1180,24 @@ int bpd_session_create(const bpd_model* model, int batch, int max_src, int max_t
   s->m = model; s->B = batch; s->max_src = max_src; s->max_tgt = max_tgt;
   s->base = static_cast<char*>(dev_session_buf); s->bytes = dev_bytes; s->stream = (cudaStream_t)cuda_stream;
   s->profiling = 0;
-  s->tc = (model->cfg.dtype == 1 && !getenv("BPD_DISABLE_TC")) ? 1 : 0;
+  // options: -1 takes the library's choice for this model and batch; 0 / 1 force a strategy off / on (on only
+  // where the shapes allow it)
+  s->tc = (model->cfg.dtype == 1 && o.tensor_cores != 0) ? 1 : 0;
   // the default streams cannot be captured: graphs need a stream of the caller's own
   const bool own_stream = s->stream != nullptr && s->stream != cudaStreamLegacy && s->stream != cudaStreamPerThread;
-  s->use_graphs = (own_stream && !getenv("BPD_DISABLE_GRAPHS")) ? 1 : 0;
-  s->use_pdl = getenv("BPD_DISABLE_PDL") ? 0 : 1;
-  // with at most 16 rows per pass every projection CTA can afford the row statistics itself
-  const char* lz = getenv("BPD_LAZY_HEADS");
-  s->lazy_heads = s->tc && (lz ? atoi(lz) != 0 : batch * model->cfg.k_model >= 64);
+  s->use_graphs = (own_stream && o.cuda_graphs != 0) ? 1 : 0;
+  s->use_pdl = o.dependent_launch != 0 ? 1 : 0;
+  s->lazy_heads = s->tc && (o.lazy_heads >= 0 ? o.lazy_heads != 0 : batch * model->cfg.k_model >= 64);
   s->last_pass_lazy = 0;
-  s->fold_ln = (s->tc && batch * model->cfg.k_model <= 16 && !getenv("BPD_DISABLE_FOLD")) ? 1 : 0;
+  // with at most 16 rows per pass every projection CTA can afford the row statistics itself
+  s->fold_ln = (s->tc && batch * model->cfg.k_model <= 16 && o.fold_layer_norms != 0) ? 1 : 0;
   s->fused = (s->tc && fused::supported(model->cfg.d, model->cfg.H, model->cfg.d_ff, batch * model->cfg.k_model) &&
-              !getenv("BPD_DISABLE_FUSED")) ? 1 : 0;
+              o.cluster_layers != 0) ? 1 : 0;
+  s->opt.persistent_layers = o.persistent_layers != 0 ? 1 : 0;
+  s->opt.stage_encoder_rows = o.stage_encoder_rows != 0 ? 1 : 0;
+  s->opt.l2_stream_hints = o.l2_stream_hints != 0 ? 1 : 0;
+  s->stack = 0; s->stack_dump = nullptr;
+  s->timed = 0;
   s->phase = kPhaseCreated; s->plan_len = 0; s->plan_k = 0; s->invocations = 0; s->pinned = nullptr;
   plan_session(model->cfg, batch, max_src, max_tgt, s->base, s);
   // page table: row b's p-th page is physical page p*B + b (rows interleaved in the pool)
@@ -1010,6 +1231,8 @@ int bpd_session_create(const bpd_model* model, int batch, int max_src, int max_t
     delete s;
     return fail(BPD_E_CUDA, "session set-up failed: %s", cudaGetErrorString(e));
   }
+  const int rc_stack = stack_setup(s);
+  if (rc_stack) { bpd_session_destroy(s); return rc_stack; }
   *out = s;
   return BPD_OK;
 }
@@ -1047,7 +1270,7 @@ int bpd_encode(bpd_session* s, const int32_t* src_ids, const int32_t* src_len) {
   BPD_CUDA(cudaStreamSynchronize(s->stream));
   BPD_CUDA(cudaMemcpyAsync(s->src_dev, ids.data(), ids.size() * sizeof(int), cudaMemcpyHostToDevice, s->stream));
   BPD_CUDA(cudaMemcpyAsync(s->tail_dev, lens.data(), B * sizeof(int), cudaMemcpyHostToDevice, s->stream));
-  ResetParams rp{s->st, B, s->ppr, s->tail_dev};
+  ResetParams rp{s->st, B, s->ppr, s->tail_dev, s->stack_bar};
   reset_rows_kernel<<<1, 32 * ceil_div(B, 32), 0, s->stream>>>(rp);
   ++g_launches;
   BPD_CUDA(cudaStreamSynchronize(s->stream));   // host vectors go out of scope
@@ -1078,18 +1301,18 @@ int bpd_encode(bpd_session* s, const int32_t* src_ids, const int32_t* src_len) {
     g_launches += ge.launches;
   }
   if (rc) return rc;
-  s->phase = kPhaseEncoded; s->plan_len = 0; s->plan_k = 0; s->invocations = 0;
+  s->phase = kPhaseEncoded; s->plan_len = 0; s->plan_k = 0; s->invocations = 0; s->timed = 0;
   return BPD_OK;
 }
 
 int bpd_rewind(bpd_session* s) {
   if (!s) return fail(BPD_E_INVALID, "session is null");
   if (s->phase < kPhaseEncoded) return fail(BPD_E_STATE, "nothing encoded yet");
-  ResetParams rp{s->st, s->B, s->ppr, s->st.src_len};
+  ResetParams rp{s->st, s->B, s->ppr, s->st.src_len, s->stack_bar};
   reset_rows_kernel<<<1, 32 * ceil_div(s->B, 32), 0, s->stream>>>(rp);
   ++g_launches;
   BPD_CUDA(cudaGetLastError());
-  s->phase = kPhaseEncoded; s->invocations = 0;
+  s->phase = kPhaseEncoded; s->invocations = 0; s->timed = 0;
   return BPD_OK;
 }
 
@@ -1184,6 +1407,7 @@ static int decode_loop(bpd_session* s, const PassArgs& a, int max_passes) {
 
 static int finish_decode(bpd_session* s, int max_new, int32_t* out_ids, int32_t* out_len, bpd_stats* stats) {
   BPD_CUDA(cudaEventRecord(s->ev1, s->stream));
+  s->timed = 1;
   if (!out_ids && !out_len && !stats) return BPD_OK;
   BPD_CUDA(cudaEventSynchronize(s->ev1));
   float ms = 0.f;
@@ -1246,7 +1470,7 @@ int bpd_iteration(bpd_session* s, int k, int accept_mode, int max_new, int32_t e
     s->phase = kPhaseBlockwise;
   }
   PassArgs a{kModeBlock, k, k, k, nullptr, 0, 0, max_new, eos_id, out ? out->logits_dev : nullptr,
-             acc.accept_kind, acc.accept_param, acc.min_block};
+             acc.accept_kind, acc.accept_param, acc.min_block, out ? out->layers_dev : nullptr};
   if (forced_tail && k > 1) {
     BPD_CUDA(cudaStreamSynchronize(s->stream));   // the staging slots may still be in flight
     memcpy(&s->pinned[128], forced_tail, sizeof(int) * B * (k - 1));
@@ -1287,7 +1511,7 @@ int bpd_fetch_output(bpd_session* s, int max_new, int32_t* out_ids, int32_t* out
   if (max_new < 1 || max_new > s->max_tgt) return fail(BPD_E_SHAPE, "max_new = %d outside 1..%d", max_new, s->max_tgt);
   if (s->phase < kPhaseEncoded) return fail(BPD_E_STATE, "nothing encoded yet");
   float ms = 0.f;
-  if (s->phase != kPhaseEncoded) {
+  if (s->phase != kPhaseEncoded && s->timed) {   // a decode call bracketed its loop with events; bpd_iteration does not
     BPD_CUDA(cudaEventSynchronize(s->ev1));
     BPD_CUDA(cudaEventElapsedTime(&ms, s->ev0, s->ev1));
   }
@@ -1338,7 +1562,7 @@ static OpScratch op_scratch_layout(int rows, int in_f, int out_f) {
   o.total = off;
   return o;
 }
-static bool op_use_tc(int dtype) { return dtype == 1 && !getenv("BPD_DISABLE_TC"); }
+static bool op_use_tc(int dtype) { return dtype == 1; }
 
 static int op_tc_finish(char* scratch, const OpScratch& L, cudaStream_t st) {
   int err = 0;
@@ -1370,7 +1594,7 @@ int bpd_op_vocab_argmax(const void* x, const void* w, int rows, int d, int vocab
     BPD_CUDA(cudaMemsetAsync(p, 0, L.total, st));
     tc::Scratch sc{reinterpret_cast<float*>(p + L.ws_off), L.ws_floats, reinterpret_cast<unsigned*>(p + L.cnt_off),
                    L.n_counters, reinterpret_cast<unsigned*>(p + L.done_off),
-                   reinterpret_cast<unsigned long long*>(p + L.pv_off), L.part_elems, reinterpret_cast<int*>(p + L.err_off), 0};
+                   reinterpret_cast<unsigned long long*>(p + L.pv_off), L.part_elems, reinterpret_cast<int*>(p + L.err_off), 0, 1};
     const long long plane = (reinterpret_cast<const bf16*>(p + L.zero_off) - static_cast<const bf16*>(x));
     tc::Operands op{w, vocab, x, plane, d, rows, d};
     tc::TcParams tp;
@@ -1415,7 +1639,7 @@ int bpd_op_linear(const void* x, const void* w, const void* bias, int rows, int 
     BPD_CUDA(cudaMemsetAsync(p, 0, L.total, st));
     tc::Scratch sc{reinterpret_cast<float*>(p + L.ws_off), L.ws_floats, reinterpret_cast<unsigned*>(p + L.cnt_off),
                    L.n_counters, reinterpret_cast<unsigned*>(p + L.done_off),
-                   reinterpret_cast<unsigned long long*>(p + L.pv_off), L.part_elems, reinterpret_cast<int*>(p + L.err_off), 0};
+                   reinterpret_cast<unsigned long long*>(p + L.pv_off), L.part_elems, reinterpret_cast<int*>(p + L.err_off), 0, 1};
     const long long plane = (reinterpret_cast<const bf16*>(p + L.zero_off) - static_cast<const bf16*>(x));
     tc::Operands op{w, out_f, x, plane, in_f, rows, in_f};
     tc::TcParams tp;

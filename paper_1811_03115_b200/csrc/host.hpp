@@ -44,6 +44,10 @@ inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// Opt-in dynamic shared-memory limit of a kernel: only ever raised, tracked per (device, kernel), so that
+// sessions of different models and several devices in one process cannot lower or miss each other's limit.
+int ensure_smem_limit(const void* kernel, size_t bytes);
+
 struct Config {
   int dtype, n_enc, n_dec, d, H, d_ff, V, k_model, d_hidden, head_layout, p1_identity;
   int local_q, local_m;    // decoder self-attention: 0 = all earlier positions; else 1D local attention
@@ -135,6 +139,7 @@ struct bpd_session {
   cudaEvent_t ev_flag[8];
   int epoch;               // decodes started on this session (the verify kernel tags its reports with it)
   cudaEvent_t ev0, ev1;
+  int timed;               // ev0 / ev1 bracket a finished decode loop
   int64_t invocations;
   int profiling;
   int use_graphs;
@@ -146,6 +151,17 @@ struct bpd_session {
   int fused;               // decoder layers as three launches each (clusters; at most 16 rows per pass)
   float* fused_ws;
   unsigned* fused_counters;
+  // the whole layer stack as one persistent kernel (see layer_stack.cuh); 0 when the shapes or the device's
+  // cluster occupancy do not allow it
+  struct { int persistent_layers, stage_encoder_rows, l2_stream_hints; } opt;   // resolved session options
+  int stack;
+  void* stack_maps;        // device: CUtensorMap [n_dec][8]
+  void* stack_layers;      // device: stack::LayerPtrs [n_dec]
+  float* stack_ws;         // device: [2][H][16][d] partial outputs of the clusters
+  unsigned* stack_bar;     // device: words of the device-wide join
+  float* stack_dump;       // device: [n_dec][rows][d] residual stream after every layer (debug dump), or null
+  int stack_cross_rows, stack_long;
+  int stack_layout[24];    // stack::Layout, kept opaque here
   std::map<GraphKey, GraphEntry> graphs;
   GraphEntry enc_graph;    // the encoder's launch sequence (fixed for a session), captured on its second use
   std::vector<cudaEvent_t> prof_begin[kProfSlots], prof_end[kProfSlots];

@@ -1283,6 +1283,7 @@ struct ResetParams {
   RowState st;
   int B, ppr;
   const int* src_len;
+  unsigned* join_words;   // words of the persistent layer kernel's device-wide join (64), or null
 };
 static __global__ void reset_rows_kernel(ResetParams p) {
   const int b = threadIdx.x;
@@ -1299,6 +1300,8 @@ static __global__ void reset_rows_kernel(ResetParams p) {
     *p.st.error = 0;
     for (int i = 0; i < 4 + kMaxK + 1; ++i) p.st.stats[i] = 0;
   }
+  if (p.join_words)
+    for (int i = threadIdx.x; i < 64; i += blockDim.x) p.join_words[i] = 0u;
 }
 
 }  // namespace bpd

@@ -88,6 +88,7 @@ struct Scratch {
   unsigned long long* best; size_t best_elems;
   int* error;
   int wide_ttiles;   // see plan_splits
+  int l2_hints;      // 1: weights that a launch reads once are loaded "evict first"
 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -139,6 +140,32 @@ inline int make_map(const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, 
   return BPD_OK;
 }
 
+// A general 2-D map (not cached): `rows` x `cols` elements of `elem_bytes` (2: bf16, 4: fp32) with `ld` elements
+// between rows, boxes of box_cols x box_rows, swizzle chosen by the box's inner extent in bytes (128 -> 128-byte
+// mode, 64 -> 64-byte mode, anything else -> none).
+inline int make_map_2d(const void* ptr, int elem_bytes, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_cols,
+                       uint32_t box_rows, bool swizzle, CUtensorMap* out) {
+  if ((uintptr_t)ptr % 16 || (ld * elem_bytes) % 16) return fail(BPD_E_INVALID, "tensor-map operand is not 16-byte aligned");
+  if (box_rows < 1 || box_rows > 256 || box_cols < 1 || box_cols > 256) return fail(BPD_E_INVALID, "tensor-map box %u x %u", box_cols, box_rows);
+  EncodeTiledFn enc;
+  int rc = get_encode_fn(&enc);
+  if (rc) return rc;
+  const uint32_t inner = box_cols * (uint32_t)elem_bytes;
+  CUtensorMapSwizzle sw = CU_TENSOR_MAP_SWIZZLE_NONE;
+  if (swizzle && inner == 128) sw = CU_TENSOR_MAP_SWIZZLE_128B;
+  else if (swizzle && inner == 64) sw = CU_TENSOR_MAP_SWIZZLE_64B;
+  else if (swizzle) return fail(BPD_E_INVALID, "no swizzle mode for boxes of %u bytes per row", inner);
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {ld * (uint64_t)elem_bytes};
+  const cuuint32_t box[2] = {box_cols, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(out, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                   const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(BPD_E_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+  return BPD_OK;
+}
+
 struct Operands {
   const void* w; int w_rows;            // weights [w_rows, K] (all slices stacked)
   const void* x; long long x_plane;     // activation planes: hi at x, lo at x + x_plane (elements)
@@ -148,10 +175,9 @@ struct Operands {
 template <int EPI>
 int launch(const Operands& op, int N, int K, int T, TcParams p, const Scratch& sc, cudaStream_t st, int zslices = 1,
            int a_rows_per_slice = 0, int b_cols_per_slice = 0, bool pdl = false, int plan_n = 0, int plan_tt = 0) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    BPD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)std::max(smem_bytes(kMaxBN), smem_bytes(64))));
-    attr_set = true;
+  {
+    const int rc0 = ensure_smem_limit(reinterpret_cast<const void*>(gemm_tc_kernel<EPI>), std::max(smem_bytes(kMaxBN), smem_bytes(64)));
+    if (rc0) return rc0;
   }
   // plan_n: the feature count the K split is planned for.  A launch that computes only the first features of a
   // matrix (fewer heads) passes the full count so that every feature is summed in the same order either way.
@@ -177,7 +203,7 @@ int launch(const Operands& op, int N, int K, int T, TcParams p, const Scratch& s
   p.T = T; p.N = N; p.K = K; p.bn = bn; p.splits = pl.splits; p.chunks_per_split = pl.chunks_per_split;
   p.ws = sc.ws; p.tile_counters = sc.tile_counters; p.done_counter = sc.done_counter;
   p.best = sc.best; p.error = sc.error;
-  p.stream_weights = (ttiles == 1 && !getenv("BPD_NO_L2_HINTS")) ? 1 : 0;
+  p.stream_weights = (ttiles == 1 && sc.l2_hints) ? 1 : 0;
   {
     // vector stores in the epilogue of wide tiles: every row offset and pointer involved must allow them
     auto al = [](const void* q, size_t a) { return q == nullptr || (uintptr_t)q % a == 0; };

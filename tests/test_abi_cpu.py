@@ -37,7 +37,15 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_struct_layouts_match_header(lib):
     assert C.sizeof(lib.bpd_stats) == 8 * 4 + 8 * 17 + 8
-    assert C.sizeof(lib.bpd_iter_out) == 7 * C.sizeof(C.c_void_p)
+    assert C.sizeof(lib.bpd_iter_out) == 8 * C.sizeof(C.c_void_p)
+    assert C.sizeof(lib.bpd_session_options) == 10 * 4
+    opt = lib.bpd_session_options()
+    lib.lib.bpd_session_options_init(C.byref(opt))
+    assert opt.struct_bytes == 40 and all(getattr(opt, n) == -1 for n in lib.OPTION_FIELDS)
+    # the header declares the same fields in the same order
+    text = open(os.path.join(ROOT, "include", "bpd.h")).read()
+    body = text[text.index("typedef struct {\n  int32_t struct_bytes"):text.index("} bpd_session_options;")]
+    assert re.findall(r"int32_t (\w+);", body) == ["struct_bytes"] + list(lib.OPTION_FIELDS)
 
 
 def _sizes(lib, blob, batch=1, max_src=8, max_tgt=8):

@@ -388,7 +388,7 @@ def test_minimum_block_lockstep(bpd):
 # ---------------------------------------------------------------- lazy (two-stage) head evaluation
 
 @pytest.mark.parametrize("w", [MINI, MINI_BLOCK, MINI_BATCH], ids=lambda w: w.name)
-def test_lazy_heads_give_the_same_decode(bpd, w, monkeypatch):
+def test_lazy_heads_give_the_same_decode(bpd, w):
     """p_1 at every position first, all heads only at the accepted position: same ids, same accepted
     block sizes, same next blocks as the one-stage evaluation and as the oracle."""
     from harness import lockstep
@@ -402,8 +402,7 @@ def test_lazy_heads_give_the_same_decode(bpd, w, monkeypatch):
     s0.bpd_set_forced_plan(plan, k)
     _, _, st0 = s0.bpd_decode_blockwise(k, N)
     s0.close()
-    monkeypatch.setenv("BPD_LAZY_HEADS", "1")
-    s = bpd.Session(model, w.batch, w.max_src, N)
+    s = bpd.Session(model, w.batch, w.max_src, N, options={"lazy_heads": 1})
     s.bpd_encode(src, src_len)
     ids, _, _ = s.bpd_decode_blockwise(k, N)
     assert np.array_equal(ids, g_ids)
@@ -420,42 +419,78 @@ def test_lazy_heads_give_the_same_decode(bpd, w, monkeypatch):
     s.close()
     model.close()
 
+LAYER_PATHS = {
+    "persistent": {},                                             # one kernel for the whole layer stack (default)
+    "cluster": {"persistent_layers": 0},                          # three cluster launches per layer
+    "per-projection": {"persistent_layers": 0, "cluster_layers": 0},
+}
+
+
 @pytest.mark.parametrize("w", [MIDI, MIDI_BATCH], ids=lambda w: w.name)
-def test_fused_layers_agree_with_kernel_per_projection(bpd, w, monkeypatch):
-    """Sessions with few rows run each decoder layer as three launches (one cluster per head / per group of hidden
-    units).  The sums are split differently from the kernel-per-projection path, so the two agree to fp32
-    rounding of bf16-weight products, far inside the oracle tolerance."""
+def test_layer_paths_agree(bpd, w):
+    """Sessions with few rows run the decoder layers in one persistent kernel (one cluster per head); the same
+    sessions can also run three cluster launches per layer or one kernel per projection.  The sums are split
+    differently, so the three agree to fp32 rounding of bf16-weight products, far inside the oracle tolerance --
+    hidden states after every layer, decoder outputs and logits."""
     blob, model, src, src_len, om = _setup(bpd, w)
     k, N = w.cfg.k_model, w.n_decode
 
-    def run():
-        s = bpd.Session(model, w.batch, w.max_src, N)
+    def run(options):
+        s = bpd.Session(model, w.batch, w.max_src, N, options=options)
         s.bpd_encode(src, src_len)
         steps = []
         for _ in range(4):
-            r = s.bpd_iteration(k, N, want_logits=True, want_hidden=True)
-            steps.append((r["hidden"].cpu().numpy().copy(), r["logits"].cpu().numpy().copy()))
+            r = s.bpd_iteration(k, N, want_logits=True, want_hidden=True, want_layers=True)
+            steps.append((r["hidden"].cpu().numpy().copy(), r["logits"].cpu().numpy().copy(),
+                          r["layers"].cpu().numpy().copy()))
         s.close()
         return steps
 
-    a_steps = run()
-    monkeypatch.setenv("BPD_DISABLE_FUSED", "1")
-    b_steps = run()
-    for (ha, la), (hb, lb) in zip(a_steps, b_steps):
-        assert np.abs(ha - hb).max() <= 2e-3 and np.abs(la - lb).max() <= 2e-3
+    ref = run(LAYER_PATHS["per-projection"])
+    for name in ("persistent", "cluster"):
+        got = run(LAYER_PATHS[name])
+        for it, ((ha, la, xa), (hb, lb, xb)) in enumerate(zip(got, ref)):
+            assert np.abs(xa - xb).max() <= 2e-3, f"{name}, iteration {it}: residual stream differs"
+            assert np.abs(ha - hb).max() <= 2e-3 and np.abs(la - lb).max() <= 2e-3, f"{name}, iteration {it}"
     model.close()
 
 
+def test_layer_dump_matches_the_oracle(bpd):
+    """The residual stream after every decoder layer (the debug dump of bpd_iteration) against the oracle's."""
+    from oracle.decode import TransformerScorer
+    w = MIDI
+    blob, model, src, src_len, om = _setup(bpd, w)
+    k, N = w.cfg.k_model, w.n_decode
+    for name, options in LAYER_PATHS.items():
+        s = bpd.Session(model, 1, w.max_src, N, options=options)
+        s.bpd_encode(src, src_len)
+        s.bpd_iteration(k, N)
+        r = s.bpd_iteration(k, N, want_layers=True)
+        ids, _, _ = s.bpd_fetch_output(N)
+        sc = TransformerScorer(om, src[0, :src_len[0]], k=k)
+        n_prev = int(np.sum(ids[0] >= 0)) - int(r["khat"][0])
+        inputs = [0] + [int(t) for t in ids[0][:n_prev]] + [int(t) for t in r["block"][0]]
+        want = sc.layer_outputs(inputs, k)                                  # [n_dec, k, d]
+        got = r["layers"].cpu().numpy()[:, 0]
+        assert got.shape == want.shape
+        err = np.abs(got - want).max(axis=-1)
+        assert err.max() <= 2e-2, (f"{name}: layer outputs differ, per (layer, row): {err.round(4).tolist()}; inputs {inputs}, "
+                                   f"khat {r['khat']}")
+        s.close()
+    model.close()
+
+
+@pytest.mark.parametrize("path", ["persistent", "cluster"])
 @pytest.mark.parametrize("w", [MIDI, MIDI_BATCH, MINI_BATCH], ids=lambda w: w.name)
-def test_staged_encoder_rows_change_nothing(bpd, w, monkeypatch):
+def test_staged_encoder_rows_change_nothing(bpd, w, path):
     """Cross-attention normally reads the encoder's keys and values from shared memory, where they were copied
-    before the dependency wait; sources too long for that are read from L2.  Both routes do the same arithmetic
-    in the same order: same hidden states, logits and ids."""
+    ahead of time; sources too long for that are read from L2.  Both routes do the same arithmetic in the same
+    order: same hidden states, logits and ids."""
     blob, model, src, src_len, om = _setup(bpd, w)
     k, N = w.cfg.k_model, w.n_decode
 
-    def run():
-        s = bpd.Session(model, w.batch, w.max_src, N)
+    def run(extra):
+        s = bpd.Session(model, w.batch, w.max_src, N, options=dict(LAYER_PATHS[path], **extra))
         s.bpd_encode(src, src_len)
         r = s.bpd_iteration(k, N, want_logits=True, want_hidden=True)
         r = s.bpd_iteration(k, N, want_logits=True, want_hidden=True)
@@ -464,11 +499,31 @@ def test_staged_encoder_rows_change_nothing(bpd, w, monkeypatch):
         ids, _, _ = s.bpd_decode_blockwise(k, N)
         s.close()
         return hidden, logits, ids
-    h_a, l_a, ids_a = run()
-    monkeypatch.setenv("BPD_NO_CROSS_STAGE", "1")
-    h_b, l_b, ids_b = run()
+    h_a, l_a, ids_a = run({})
+    h_b, l_b, ids_b = run({"stage_encoder_rows": 0})
     assert np.array_equal(h_a, h_b) and np.array_equal(l_a, l_b) and np.array_equal(ids_a, ids_b)
     model.close()
+
+
+def test_same_decode_twice_gives_identical_ids(bpd):
+    """Every reduction has a fixed order: decoding the same input twice gives bit-identical hidden states and ids
+    (an order-dependent reduction -- a race between CTAs -- would show up as a difference)."""
+    for w in (MIDI_BATCH, MINI_BATCH):
+        blob, model, src, src_len, om = _setup(bpd, w)
+        k, N = w.cfg.k_model, w.n_decode
+        s = bpd.Session(model, w.batch, w.max_src, N)
+        outs = []
+        for _ in range(3):
+            s.bpd_encode(src, src_len)
+            r = s.bpd_iteration(k, N, want_hidden=True, want_logits=True)
+            hid, lg = r["hidden"].cpu().numpy().copy(), r["logits"].cpu().numpy().copy()
+            s.bpd_encode(src, src_len)
+            ids, _, _ = s.bpd_decode_blockwise(k, N)
+            outs.append((hid, lg, ids))
+        for hid, lg, ids in outs[1:]:
+            assert np.array_equal(hid, outs[0][0]) and np.array_equal(lg, outs[0][1]) and np.array_equal(ids, outs[0][2])
+        s.close()
+        model.close()
 
 
 # 1D local attention (query blocks of local_q positions + local_m positions of memory), one model per attention kernel
@@ -489,7 +544,7 @@ LOCAL_MODELS = [
 
 @pytest.mark.parametrize("w", LOCAL_MODELS, ids=lambda w: w.name)
 def test_local_attention_lockstep(bpd, w):
-    """Section 7.3's model class: decoder self-attention restricted to the query's block and a fixed memory
+    """Section 7.2's model class: decoder self-attention restricted to the query's block and a fixed memory
     before it.  Every attention kernel (cluster path, split, generic, per-sequence, per-row) against the oracle,
     decoding far enough that whole 32-key chunks fall out of the window."""
     from harness import lockstep

@@ -242,7 +242,7 @@ def test_dense_with_block_structure_equals_blockdiag_layout():
     np.testing.assert_allclose(head_logits(md, h, 2), head_logits(md, h, k)[:, :2], atol=0)
 
 
-# ---------------------------------------------------------------- 1D local attention (Section 7.3's model class)
+# ---------------------------------------------------------------- 1D local attention (Section 7.2's model class)
 
 def test_local_attention_window_by_enumeration():
     """The visible keys of a query, enumerated from the definition for every (query block, memory) pair and
