@@ -225,12 +225,11 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
   float* fused_ws = a.take<float>(fused_ok ? fused_parts * Rmax * d : 0);
   unsigned* fused_counters = a.take<unsigned>(fused::kC);
   // persistent layer stack: tensor maps, per-layer pointers, the clusters' partial outputs, the join's words
-  void* stack_maps = a.take_bytes(fused_ok ? (size_t)c.n_dec * stack::kMapsPerLayer * sizeof(CUtensorMap) : 0);
   void* stack_layers = a.take_bytes(fused_ok ? (size_t)c.n_dec * sizeof(stack::LayerPtrs) : 0);
   float* stack_ws = a.take<float>(fused_ok ? (size_t)2 * c.H * fused::kMaxRows * d : 0);
   unsigned* stack_bar = a.take<unsigned>(stack::kBarWords);
   if (s) {
-    s->stack_maps = stack_maps; s->stack_layers = stack_layers; s->stack_ws = stack_ws; s->stack_bar = stack_bar;
+    s->stack_layers = stack_layers; s->stack_ws = stack_ws; s->stack_bar = stack_bar;
     s->fused_ws = fused_ws; s->fused_counters = fused_counters;
     s->x = x; s->h_f32 = h_f32; s->xn = xn; s->qbuf = qbuf; s->attn = attn; s->ffh = ffh; s->u = u; s->o = o;
     s->crosskv = crosskv; s->kcache = kc; s->vcache = vc; s->st = st; s->src_dev = src_dev;
@@ -659,14 +658,15 @@ static bool stack_plan(const Config& c, int rows, int nb, int ppr, int cross_row
   L.xl = take((size_t)RP * g.ks * 2);
   L.oh = take((size_t)RP * 128);
   L.ol = take((size_t)RP * 128);
-  L.hh = take((size_t)g.PH * RP * 128);
-  L.hl = take((size_t)g.PH * RP * 128);
-  L.inbox = take(std::max((size_t)fused::kC * NT * 3 * fused::kDH * 4, (size_t)fused::kC * g.UPR * RP * 4));
-  L.q = take((size_t)RP * fused::kDH * 4);
+  L.hid = take((size_t)fused::kC * 2 * RP * g.UPR * 2);
+  const size_t chunk = std::max((size_t)NT * 3 * fused::kDH * 4, (size_t)g.UPR * RP * 4);
+  L.outbox = take(fused::kC * chunk);
+  L.inbox = take(fused::kC * chunk);
+  L.kvq = take((size_t)RP * 512);
   L.stats = take((size_t)fused::kC * fused::kMaxRows * 2 * 4 + 4 * fused::kMaxRows * 4);
   L.attn = take(sizeof(AttnSmem<fused::kDH, stack::kWarps>));
-  L.wst = take((size_t)stack::kWarps * NT * fused::kPartial * 4);
-  const size_t lvl = long_seq ? (size_t)fused::kC * rows * fused::kPartial * 4 : 0;
+  L.wst = take((size_t)stack::kWarps * NT * stack::kState * 4);
+  const size_t lvl = long_seq ? (size_t)fused::kC * rows * stack::kState * 4 : 0;
   L.lvl1 = take(lvl);
   L.lvl2 = take(lvl);
   L.pt = take((size_t)nb * ppr * 4);
@@ -674,8 +674,9 @@ static bool stack_plan(const Config& c, int rows, int nb, int ppr, int cross_row
   L.misc = take(sizeof(stack::Ctl));
   const size_t work = off;
   int largest = 0, second = 0, per_layer = 0;
+  if (g.ntl > stack::kMaxTiles) return false;
   for (int i = 0; i < g.ntl; ++i) {
-    const int b = stack::tile_bytes(g, i, cross_rows);
+    const int b = stack::make_tile(g, i, cross_rows, c.d, 0, 0).bytes;
     per_layer += b;
     if (b > largest) { second = largest; largest = b; } else if (b > second) second = b;
   }
@@ -683,7 +684,7 @@ static bool stack_plan(const Config& c, int rows, int nb, int ppr, int cross_row
   size_t ring = std::min((budget - work) / 1024 * 1024, (size_t)per_layer * c.n_dec);
   if (ring < (size_t)largest + second) return false;
   L.ring_bytes = (int)ring;
-  int* fields[] = {&L.x, &L.xh, &L.xl, &L.oh, &L.ol, &L.hh, &L.hl, &L.inbox, &L.q, &L.stats, &L.attn, &L.wst, &L.lvl1,
+  int* fields[] = {&L.x, &L.xh, &L.xl, &L.oh, &L.ol, &L.hid, &L.outbox, &L.inbox, &L.kvq, &L.stats, &L.attn, &L.wst, &L.lvl1,
                    &L.lvl2, &L.pt, &L.layers, &L.misc};
   for (int* f : fields) *f += (int)ring;
   L.total = (int)(ring + work);
@@ -691,9 +692,9 @@ static bool stack_plan(const Config& c, int rows, int nb, int ppr, int cross_row
   return true;
 }
 
-template <int NT>
+template <int NT, int KS, int MINB>
 static int stack_clusters(size_t smem, int H, int* out) {
-  BPD_TRY(ensure_smem_limit(reinterpret_cast<const void*>(stack::layer_stack_kernel<NT>), smem));
+  BPD_TRY(ensure_smem_limit(reinterpret_cast<const void*>(stack::layer_stack_kernel<NT, KS, MINB>), smem));
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
   cfg.gridDim = dim3(fused::kC, H); cfg.blockDim = dim3(stack::kThreads); cfg.dynamicSmemBytes = smem;
@@ -701,7 +702,7 @@ static int stack_clusters(size_t smem, int H, int* out) {
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = fused::kC; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
   cfg.attrs = at; cfg.numAttrs = 1;
-  BPD_CUDA(cudaOccupancyMaxActiveClusters(out, stack::layer_stack_kernel<NT>, &cfg));
+  BPD_CUDA(cudaOccupancyMaxActiveClusters(out, stack::layer_stack_kernel<NT, KS, MINB>, &cfg));
   return BPD_OK;
 }
 
@@ -709,7 +710,7 @@ static int stack_clusters(size_t smem, int H, int* out) {
 static bool stack_shapes_ok(const Config& c, int rows) {
   const int d = c.d, H = c.H;
   if (c.dtype != 1 || H < 1 || d != H * fused::kDH || (d != 256 && d != 512 && d != 1024)) return false;
-  if (c.d_ff % H || (c.d_ff / H) % 64 || c.d_ff / H > 256) return false;
+  if (c.d_ff % H || (c.d_ff / H != 128 && c.d_ff / H != 256)) return false;   // hidden units per cluster
   if (rows < 1 || rows > fused::kMaxRows || c.n_dec > 64) return false;
   return true;
 }
@@ -733,37 +734,59 @@ static int stack_setup(bpd_session* s) {
   stack::Layout lay;
   bool ok = false;
   int cross_rows = 0;
+  int minb = 0;
   for (size_t budget : budgets) {
+    ++minb;                                    // first one CTA per SM, then two
     for (int staged = 1; staged >= 0 && !ok; --staged) {
       cross_rows = (staged && s->B * s->max_src <= 256) ? s->B * s->max_src : 0;
       if (staged && !cross_rows) continue;
       if (budget <= 1024 || !stack_plan(c, rows, s->B, s->ppr, cross_rows, long_seq, budget - 1024, &lay)) continue;
       lay.total += 1024;                       // slack for aligning the ring to 1024 bytes
       int n1 = 0, n2 = 0;
-      BPD_TRY(stack_clusters<1>((size_t)lay.total, c.H, &n1));
-      BPD_TRY(stack_clusters<2>((size_t)lay.total, c.H, &n2));
+      const size_t sm = (size_t)lay.total;
+      if (c.d == 256 && minb == 1) { BPD_TRY((stack_clusters<1, 2, 1>(sm, c.H, &n1))); BPD_TRY((stack_clusters<2, 2, 1>(sm, c.H, &n2))); }
+      else if (c.d == 256) { BPD_TRY((stack_clusters<1, 2, 2>(sm, c.H, &n1))); BPD_TRY((stack_clusters<2, 2, 2>(sm, c.H, &n2))); }
+      else if (minb == 1) { BPD_TRY((stack_clusters<1, 4, 1>(sm, c.H, &n1))); BPD_TRY((stack_clusters<2, 4, 1>(sm, c.H, &n2))); }
+      else { BPD_TRY((stack_clusters<1, 4, 2>(sm, c.H, &n1))); BPD_TRY((stack_clusters<2, 4, 2>(sm, c.H, &n2))); }
       ok = n1 >= c.H && n2 >= c.H;
     }
     if (ok) break;
   }
   if (!ok) return BPD_OK;
-  // tensor maps: weight slices as boxes of 64 (32 for d_model 256) reduction columns, encoder keys / values
+  // tensor maps over all layers at once: weight slices as boxes of 64 (32 for d_model 256) reduction columns,
+  // encoder keys / values.  The layers' tensors must lie at a constant stride (they do in a blob written tensor
+  // by tensor, layer after layer; the session's encoder keys / values are laid out the same way).
   const stack::Geo g = stack::make_geo(c.d, c.H, c.d_ff, c.n_dec, cross_rows);
-  std::vector<CUtensorMap> maps((size_t)c.n_dec * stack::kMapsPerLayer);
   std::vector<stack::LayerPtrs> lp(c.n_dec);
-  const int d = c.d, f = c.d_ff;
-  for (int l = 0; l < c.n_dec; ++l) {
-    const DecLayer& L = m->dec[l];
-    CUtensorMap* mp = &maps[(size_t)l * stack::kMapsPerLayer];
-    BPD_TRY(tc::make_map_2d(L.wqkv, 2, 3 * d, d, d, g.PW, 64, true, mp + stack::kMapQkv));
-    BPD_TRY(tc::make_map_2d(L.wo, 2, d, d, d, 64, g.ks, true, mp + stack::kMapWo));
-    BPD_TRY(tc::make_map_2d(L.cwq, 2, d, d, d, g.PW, 64, true, mp + stack::kMapCq));
-    BPD_TRY(tc::make_map_2d(L.cwo, 2, d, d, d, 64, g.ks, true, mp + stack::kMapCwo));
-    BPD_TRY(tc::make_map_2d(L.w1, 2, f, d, d, g.PW, g.HCt, true, mp + stack::kMapW1));
-    BPD_TRY(tc::make_map_2d(L.w2, 2, d, f, f, 64, g.ks, true, mp + stack::kMapW2));
+  const int d = c.d, f = c.d_ff, nl = c.n_dec;
+  auto stride_of = [&](auto get, long long* out) {
+    *out = nl > 1 ? (const char*)get(1) - (const char*)get(0) : 0;
+    for (int l = 1; l + 1 < nl; ++l)
+      if ((const char*)get(l + 1) - (const char*)get(l) != *out) return false;
+    return *out >= 0;
+  };
+  long long st_qkv, st_wo, st_cq, st_cwo, st_w1, st_w2, st_ckv;
+  const bool regular = stride_of([&](int l) { return m->dec[l].wqkv; }, &st_qkv) && stride_of([&](int l) { return m->dec[l].wo; }, &st_wo) &&
+                       stride_of([&](int l) { return m->dec[l].cwq; }, &st_cq) && stride_of([&](int l) { return m->dec[l].cwo; }, &st_cwo) &&
+                       stride_of([&](int l) { return m->dec[l].w1; }, &st_w1) && stride_of([&](int l) { return m->dec[l].w2; }, &st_w2) &&
+                       stride_of([&](int l) { return (const void*)s->crosskv[l]; }, &st_ckv);
+  if (!regular) return BPD_OK;
+  stack::StackMaps maps;
+  memset(&maps, 0, sizeof(maps));
+  {
+    const DecLayer& L0 = m->dec[0];
     const int er = std::max(cross_rows, 1);
-    BPD_TRY(tc::make_map_2d(s->crosskv[l], 4, (uint64_t)s->B * s->max_src, 2 * d, 2 * d, 32, er, true, mp + stack::kMapCk));
-    BPD_TRY(tc::make_map_2d(s->crosskv[l], 4, (uint64_t)s->B * s->max_src, 2 * d, 2 * d, 64, er, false, mp + stack::kMapCv));
+    BPD_TRY(tc::make_map_3d(L0.wqkv, 2, nl, st_qkv, 3 * d, d, d, g.PW, 64, true, &maps.m[stack::kMapQkv]));
+    BPD_TRY(tc::make_map_3d(L0.wo, 2, nl, st_wo, d, d, d, 64, g.ks, true, &maps.m[stack::kMapWo]));
+    BPD_TRY(tc::make_map_3d(L0.cwq, 2, nl, st_cq, d, d, d, g.PW, 64, true, &maps.m[stack::kMapCq]));
+    BPD_TRY(tc::make_map_3d(L0.cwo, 2, nl, st_cwo, d, d, d, 64, g.ks, true, &maps.m[stack::kMapCwo]));
+    BPD_TRY(tc::make_map_3d(L0.w1, 2, nl, st_w1, f, d, d, g.PW, g.HCt, true, &maps.m[stack::kMapW1]));
+    BPD_TRY(tc::make_map_3d(L0.w2, 2, nl, st_w2, d, f, f, 64, g.ks, true, &maps.m[stack::kMapW2]));
+    BPD_TRY(tc::make_map_3d(s->crosskv[0], 4, nl, st_ckv, (uint64_t)s->B * s->max_src, 2 * d, 2 * d, 32, er, true, &maps.m[stack::kMapCk]));
+    BPD_TRY(tc::make_map_3d(s->crosskv[0], 4, nl, st_ckv, (uint64_t)s->B * s->max_src, 2 * d, 2 * d, 64, er, false, &maps.m[stack::kMapCv]));
+  }
+  for (int l = 0; l < nl; ++l) {
+    const DecLayer& L = m->dec[l];
     stack::LayerPtrs& P = lp[l];
     P.g1 = static_cast<const bf16*>(L.ln1g); P.g2 = static_cast<const bf16*>(L.ln2g); P.g3 = static_cast<const bf16*>(L.ln3g);
     P.s_qkv = L.s_qkv; P.c_qkv = L.c_qkv; P.s_cq = L.s_cq; P.c_cq = L.c_cq; P.s_f1 = L.s_f1; P.c_f1 = L.c_f1;
@@ -771,12 +794,13 @@ static int stack_setup(bpd_session* s) {
     P.kcache = static_cast<bf16*>(s->kcache[l]); P.vcache = static_cast<bf16*>(s->vcache[l]);
     P.crosskv = static_cast<const float*>(s->crosskv[l]);
   }
-  BPD_CUDA(cudaMemcpyAsync(s->stack_maps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, s->stream));
+  static_assert(sizeof(stack::StackMaps) == sizeof(s->stack_maps), "tensor maps do not fit their opaque copy");
+  memcpy(s->stack_maps, &maps, sizeof(maps));
   BPD_CUDA(cudaMemcpyAsync(s->stack_layers, lp.data(), lp.size() * sizeof(stack::LayerPtrs), cudaMemcpyHostToDevice, s->stream));
   BPD_CUDA(cudaStreamSynchronize(s->stream));
   static_assert(sizeof(stack::Layout) <= sizeof(s->stack_layout), "layout does not fit its opaque copy");
   memcpy(s->stack_layout, &lay, sizeof(lay));
-  s->stack_cross_rows = cross_rows; s->stack_long = long_seq ? 1 : 0;
+  s->stack_cross_rows = cross_rows; s->stack_long = long_seq ? 1 : 0; s->stack_minb = minb;
   s->stack = 1;
   return BPD_OK;
 }
@@ -788,7 +812,6 @@ static int run_layers_stack(bpd_session* s, const PassArgs& a) {
   const Config& c = m->cfg;
   stack::StackParams p;
   memset(&p, 0, sizeof(p));
-  p.maps = static_cast<const CUtensorMap*>(s->stack_maps);
   p.layers = static_cast<const stack::LayerPtrs*>(s->stack_layers);
   p.L = c.n_dec; p.d = c.d; p.H = c.H; p.ff = c.d_ff; p.R = s->B * a.kcur; p.rows_per_b = a.kcur; p.nb = s->B; p.eps = c.eps;
   p.tgt_embed = static_cast<const bf16*>(m->tgt_embed); p.pe = s->pe; p.npos = s->npos; p.vocab = c.V;
@@ -803,8 +826,20 @@ static int run_layers_stack(bpd_session* s, const PassArgs& a) {
   memcpy(&p.lay, s->stack_layout, sizeof(p.lay));
   const dim3 grid(fused::kC, c.H), block(stack::kThreads);
   const bool pdl = s->use_pdl != 0;
-  if (p.R > 8) BPD_CUDA(launch_k(stack::layer_stack_kernel<2>, grid, block, (size_t)p.lay.total, s->stream, pdl, p));
-  else BPD_CUDA(launch_k(stack::layer_stack_kernel<1>, grid, block, (size_t)p.lay.total, s->stream, pdl, p));
+  stack::StackMaps maps;
+  memcpy(&maps, s->stack_maps, sizeof(maps));
+  const size_t smem = (size_t)p.lay.total;
+  // reduction panels of 32 columns (two steps of 16) for d_model 256, else 64 (four steps); one or two CTAs per SM
+#define BPD_STACK_LAUNCH(NT, KS, MB) BPD_CUDA(launch_k(stack::layer_stack_kernel<NT, KS, MB>, grid, block, smem, s->stream, pdl, maps, p))
+  const int nt = p.R > 8 ? 2 : 1, ksteps = c.d == 256 ? 2 : 4;
+  if (s->stack_minb == 1) {
+    if (ksteps == 2) { if (nt == 2) BPD_STACK_LAUNCH(2, 2, 1); else BPD_STACK_LAUNCH(1, 2, 1); }
+    else { if (nt == 2) BPD_STACK_LAUNCH(2, 4, 1); else BPD_STACK_LAUNCH(1, 4, 1); }
+  } else {
+    if (ksteps == 2) { if (nt == 2) BPD_STACK_LAUNCH(2, 2, 2); else BPD_STACK_LAUNCH(1, 2, 2); }
+    else { if (nt == 2) BPD_STACK_LAUNCH(2, 4, 2); else BPD_STACK_LAUNCH(1, 4, 2); }
+  }
+#undef BPD_STACK_LAUNCH
   ++g_launches;
   return BPD_OK;
 }
@@ -1519,6 +1554,16 @@ int bpd_fetch_output(bpd_session* s, int max_new, int32_t* out_ids, int32_t* out
   if (rc) return rc;
   return fetch(s, max_new, out_ids, out_len, stats, ms);
 }
+
+#ifdef BPD_STACK_TRACE
+// Development builds only: where the persistent layer kernel writes its per-CTA step timestamps (device memory,
+// clusters * 8 * 256 unsigned 64-bit words), or null to stop.
+int bpd_debug_set_stack_trace(void* dev_buffer) {
+  unsigned long long* ptr = static_cast<unsigned long long*>(dev_buffer);
+  BPD_CUDA(cudaMemcpyToSymbol(stack::g_stack_trace, &ptr, sizeof(ptr)));
+  return BPD_OK;
+}
+#endif
 
 // ------------------------------------------------------------------ self test of the bounded waits
 int bpd_debug_wait_timeout(int32_t* dev_word, int limit_us, void* cuda_stream) {

@@ -155,12 +155,12 @@ struct bpd_session {
   // cluster occupancy do not allow it
   struct { int persistent_layers, stage_encoder_rows, l2_stream_hints; } opt;   // resolved session options
   int stack;
-  void* stack_maps;        // device: CUtensorMap [n_dec][8]
+  unsigned char stack_maps[8 * 128] __attribute__((aligned(64)));   // stack::StackMaps (eight tensor maps over all layers)
   void* stack_layers;      // device: stack::LayerPtrs [n_dec]
   float* stack_ws;         // device: [2][H][16][d] partial outputs of the clusters
   unsigned* stack_bar;     // device: words of the device-wide join
   float* stack_dump;       // device: [n_dec][rows][d] residual stream after every layer (debug dump), or null
-  int stack_cross_rows, stack_long;
+  int stack_cross_rows, stack_long, stack_minb;
   int stack_layout[24];    // stack::Layout, kept opaque here
   std::map<GraphKey, GraphEntry> graphs;
   GraphEntry enc_graph;    // the encoder's launch sequence (fixed for a session), captured on its second use

@@ -166,6 +166,32 @@ inline int make_map_2d(const void* ptr, int elem_bytes, uint64_t rows, uint64_t 
   return BPD_OK;
 }
 
+// The same over `layers` tensors that lie `layer_stride_bytes` apart: dimensions (columns, rows, layer), boxes of
+// box_cols x box_rows x 1.
+inline int make_map_3d(const void* ptr, int elem_bytes, uint64_t layers, uint64_t layer_stride_bytes, uint64_t rows, uint64_t cols,
+                       uint64_t ld, uint32_t box_cols, uint32_t box_rows, bool swizzle, CUtensorMap* out) {
+  if ((uintptr_t)ptr % 16 || (ld * elem_bytes) % 16 || layer_stride_bytes % 16)
+    return fail(BPD_E_INVALID, "tensor-map operand is not 16-byte aligned");
+  if (box_rows < 1 || box_rows > 256 || box_cols < 1 || box_cols > 256) return fail(BPD_E_INVALID, "tensor-map box %u x %u", box_cols, box_rows);
+  EncodeTiledFn enc;
+  int rc = get_encode_fn(&enc);
+  if (rc) return rc;
+  const uint32_t inner = box_cols * (uint32_t)elem_bytes;
+  CUtensorMapSwizzle sw = CU_TENSOR_MAP_SWIZZLE_NONE;
+  if (swizzle && inner == 128) sw = CU_TENSOR_MAP_SWIZZLE_128B;
+  else if (swizzle && inner == 64) sw = CU_TENSOR_MAP_SWIZZLE_64B;
+  else if (swizzle) return fail(BPD_E_INVALID, "no swizzle mode for boxes of %u bytes per row", inner);
+  const cuuint64_t dims[3] = {cols, rows, layers};
+  const cuuint64_t strides[2] = {ld * (uint64_t)elem_bytes, layers > 1 ? layer_stride_bytes : ld * (uint64_t)elem_bytes * rows};
+  const cuuint32_t box[3] = {box_cols, box_rows, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = enc(out, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3,
+                   const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(BPD_E_CUDA, "cuTensorMapEncodeTiled (3-D) failed with code %d", (int)r);
+  return BPD_OK;
+}
+
 struct Operands {
   const void* w; int w_rows;            // weights [w_rows, K] (all slices stacked)
   const void* x; long long x_plane;     // activation planes: hi at x, lo at x + x_plane (elements)
