@@ -106,8 +106,9 @@ typedef struct {
                                  one (default: on when batch * k_model >= 64)                              */
   int32_t fold_layer_norms;   /* decoder layer norms folded into the projections after them (<= 16 rows)   */
   int32_t cluster_layers;     /* decoder layers as three cluster launches each (<= 16 rows per pass)        */
-  int32_t persistent_layers;  /* all decoder layers of a pass in one persistent kernel (<= 16 rows per
-                                 pass, d_model 256 / 512 / 1024; takes precedence over cluster_layers)     */
+  int32_t persistent_layers;  /* all decoder layers of a pass in one persistent TMA-fed kernel (<= 16 rows
+                                 per pass, d_model 256 / 512 / 1024; takes precedence over cluster_layers).
+                                 Default off: measured slower than the cluster launches on B200             */
   int32_t stage_encoder_rows; /* encoder keys / values staged in shared memory for cross-attention          */
   int32_t l2_stream_hints;    /* weights read once per pass are loaded "evict first"                        */
 } bpd_session_options;
@@ -245,9 +246,10 @@ int bpd_op_vocab_argmax(const void* x, const void* w, int rows, int d, int vocab
  * that is only allowed to enqueue work.  (The paper has no counterpart; this is
  * a deployment convenience.)  The cross-CTA reduction workspace is a fixed
  * 512 KiB array inside the library image, resident on every GPU that loads the
- * library until the process exits.  Limits: rows <= 256, vocab <= 65536,
- * d <= 1024 and a multiple of 8; larger sizes return BPD_E_NOMEM and leave the
- * outputs untouched.  Arguments as bpd_op_vocab_argmax, minus the scratch.
+ * library until the process exits.  Limits: rows <= 256, vocab <= 65536
+ * (beyond them the call returns BPD_E_NOMEM) and d <= 1024, a multiple of 8
+ * (BPD_E_SHAPE, as for bpd_op_vocab_argmax); a refused call leaves the outputs
+ * untouched.  Arguments as bpd_op_vocab_argmax, minus the scratch.
  * The call performs no cudaMalloc/cudaFree and uses no allocating library.
  * The first call on each device looks the array's device address up (with that
  * device current); make that first call outside any stream capture.  All calls

@@ -249,7 +249,7 @@ static size_t fold_floats(const Config& c) { return c.dtype == 1 ? (size_t)c.n_d
 static size_t weight_bytes_for(const ParsedBlob& pb) { return align_up(pb.total) + align_up(fold_floats(pb.cfg) * sizeof(float)); }
 
 // ------------------------------------------------------------------ launches
-static std::atomic<long long> g_launches{0};
+std::atomic<long long> g_launches{0};
 template <typename WT, typename AT, int EPI>
 static void launch_linear(const LinearParams& p, int zcount, cudaStream_t st) {
   dim3 grid(ceil_div(p.N, kLinWarps * kFPW), ceil_div(p.rows, kRC), zcount);
@@ -737,7 +737,7 @@ static int stack_setup(bpd_session* s) {
   int minb = 0;
   for (size_t budget : budgets) {
     ++minb;                                    // first one CTA per SM, then two
-    for (int staged = 1; staged >= 0 && !ok; --staged) {
+    for (int staged = s->opt.stage_encoder_rows ? 1 : 0; staged >= 0 && !ok; --staged) {
       cross_rows = (staged && s->B * s->max_src <= 256) ? s->B * s->max_src : 0;
       if (staged && !cross_rows) continue;
       if (budget <= 1024 || !stack_plan(c, rows, s->B, s->ppr, cross_rows, long_seq, budget - 1024, &lay)) continue;
@@ -1049,8 +1049,10 @@ static int check_device_error(bpd_session* s) {
   err = s->pinned[64];
   if (err == 1) return fail(BPD_E_INVALID, "a token id outside the vocabulary reached the decoder");
   if (err >= 101 && err <= 103) return fail(BPD_E_TIMEOUT, "a bounded wait inside the projection kernel expired (code %d)", err);
-  if (err == 104 || err == 105) return fail(BPD_E_TIMEOUT, "a bounded wait inside the persistent layer kernel expired (code %d: %s)", err,
-                                            err == 104 ? "device-wide join" : "weight tile");
+  if (err >= 104 && err <= 106) {
+    const char* what[] = {"device-wide join", "weight tile", "exchange inside the cluster"};
+    return fail(BPD_E_TIMEOUT, "a bounded wait inside the persistent layer kernel expired (code %d: %s)", err, what[err - 104]);
+  }
   if (err != 0) return fail(BPD_E_CUDA, "device-side error word %d", err);
   return BPD_OK;
 }
@@ -1228,7 +1230,7 @@ int bpd_session_create_opt(const bpd_model* model, int batch, int max_src, int m
   s->fold_ln = (s->tc && batch * model->cfg.k_model <= 16 && o.fold_layer_norms != 0) ? 1 : 0;
   s->fused = (s->tc && fused::supported(model->cfg.d, model->cfg.H, model->cfg.d_ff, batch * model->cfg.k_model) &&
               o.cluster_layers != 0) ? 1 : 0;
-  s->opt.persistent_layers = o.persistent_layers != 0 ? 1 : 0;
+  s->opt.persistent_layers = o.persistent_layers == 1 ? 1 : 0;   // opt-in: measured slower than the cluster launches
   s->opt.stage_encoder_rows = o.stage_encoder_rows != 0 ? 1 : 0;
   s->opt.l2_stream_hints = o.l2_stream_hints != 0 ? 1 : 0;
   s->stack = 0; s->stack_dump = nullptr;
@@ -1561,6 +1563,7 @@ int bpd_fetch_output(bpd_session* s, int max_new, int32_t* out_ids, int32_t* out
 int bpd_debug_set_stack_trace(void* dev_buffer) {
   unsigned long long* ptr = static_cast<unsigned long long*>(dev_buffer);
   BPD_CUDA(cudaMemcpyToSymbol(stack::g_stack_trace, &ptr, sizeof(ptr)));
+
   return BPD_OK;
 }
 #endif

@@ -6,6 +6,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <atomic>
 #include <map>
 #include <string>
 #include <tuple>
@@ -17,6 +18,7 @@
 namespace bpd {
 
 extern thread_local char g_err[512];
+extern std::atomic<long long> g_launches;   // kernels launched by this library in this process
 int fail(int code, const char* fmt, ...);
 
 #define BPD_CUDA(expr)                                                                   \

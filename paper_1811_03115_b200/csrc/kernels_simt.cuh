@@ -1165,6 +1165,11 @@ static __global__ void verify_commit_kernel(VerifyParams p) {
     const int* A = p.st.table + (size_t)b * p.kcur * p.kh;
     if (p.st.finished[b]) {
       p.st.khat[b] = 0;
+    } else if (p.mode != kModePrime && p.st.j[b] >= p.max_new) {
+      // the caller lowered max_new below what the row already holds (bpd_iteration takes it per call): the row
+      // is complete, nothing is appended or committed
+      p.st.khat[b] = 0;
+      p.st.finished[b] = 1;
     } else if (p.mode == kModePrime) {
       // start token becomes part of the prefix; its row of predictions is the first block
       p.st.len[b] += 1;

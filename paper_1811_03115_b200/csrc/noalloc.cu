@@ -69,6 +69,7 @@ extern "C" int bpd_op_vocab_argmax_noalloc(const void* x, const void* w, int row
   const size_t smem = (size_t)kRC * d * sizeof(float);
   if (dtype == 0) vocab_argmax_kernel<float, float><<<grid, kLinWarps * 32, smem, st>>>(p);
   else vocab_argmax_kernel<bf16, bf16><<<grid, kLinWarps * 32, smem, st>>>(p);
+  ++g_launches;
   BPD_CUDA(cudaGetLastError());
   return BPD_OK;
 }

@@ -19,6 +19,13 @@ MINI_F32 = Workload("minif", ModelConfig(1, 2, 96, 6, 200, 333, 3, 136, dtype=DT
                     31, 32, 33, batch=2, src_lo=2, src_hi=7, n_decode=15)
 
 
+LAYER_PATHS = {
+    "persistent": {"persistent_layers": 1},                       # one kernel for the whole layer stack (opt-in)
+    "cluster": {},                                                # three cluster launches per layer (default)
+    "per-projection": {"cluster_layers": 0},
+}
+
+
 @pytest.fixture(scope="module")
 def bpd():
     import paper_1811_03115_b200 as pkg
@@ -207,6 +214,29 @@ def test_eos_terminates_inside_a_block(bpd):
     model.close()
 
 
+def test_a_smaller_max_new_later_on_finishes_the_row(bpd):
+    """bpd_iteration takes max_new per call.  A later call with max_new at or below what a row already holds must
+    mark the row finished and change nothing else (no negative block size, no writes before the tables)."""
+    w = MINI_BATCH
+    blob, model, src, src_len, om = _setup(bpd, w)
+    k, N = w.cfg.k_model, w.n_decode
+    s = bpd.Session(model, w.batch, w.max_src, N)
+    s.bpd_encode(src, src_len)
+    for _ in range(4):
+        s.bpd_iteration(k, N)
+    ids0, len0, st0 = s.bpd_fetch_output(N)
+    assert np.all(len0 >= 4)
+    r = s.bpd_iteration(k, 2)                      # every row already holds more than 2 tokens
+    assert np.all(r["khat"] == 0)
+    ids1, len1, st1 = s.bpd_fetch_output(N)
+    assert np.array_equal(ids1, ids0) and np.array_equal(len1, len0)
+    assert st1.tokens == st0.tokens and st1.khat_hist == st0.khat_hist
+    r = s.bpd_iteration(k, N)                      # finished rows stay finished
+    assert np.all(r["khat"] == 0)
+    s.close()
+    model.close()
+
+
 def test_state_and_argument_errors(bpd):
     w = MINI
     blob, model, src, src_len, _ = _setup(bpd, w)
@@ -320,6 +350,89 @@ def test_c4_batch32_ragged(bpd):
     _full_size(bpd, "C4", iters=2, rows=rows, mean=2.0, free_iters=1)
 
 
+# ---------------------------------------------------------------- paper-sized configurations, whole decodes
+
+def _whole_decode(bpd, name, mean, rows=None, check_values=True, all_accepted=False):
+    """Lock-step with the oracle from the first iteration to the last token of the configuration's decode, under
+    controlled acceptance (or with every proposal accepted): ids under the margin rule, accepted block sizes and
+    next blocks exact in every iteration, hidden states and logits within tolerance where they are compared."""
+    from harness import lockstep
+    w = WORKLOADS[name]
+    blob, model, src, src_len, om = _setup(bpd, w)
+    del blob
+    k, N = w.cfg.k_model, w.n_decode
+    s = bpd.Session(model, w.batch, w.max_src, N)
+    s.bpd_encode(src, src_len)
+    g_ids, _, _ = s.bpd_decode_greedy(N)
+    if all_accepted:
+        def fn(b, j, it):
+            return forced_tail(g_ids[b], min(j, N), k, k, 0, w.cfg.vocab)
+        want = None
+    else:
+        fn, sched = _tail_fn(w, g_ids, k, mean)
+        want = [_expected_khats(sched[b], k, N) for b in range(w.batch)]
+    sel = list(range(w.batch)) if rows is None else rows
+    rep = lockstep(s, om, src, src_len, k, N, max_iters=N, tail_fn=fn, rows=rows, check_values=check_values)
+    for i, b in enumerate(sel):
+        assert rep.emitted[b] == list(g_ids[b]), f"row {b}: lock-step output differs from the GPU's greedy decode"
+        got = [r[i] for r in rep.khats if r[i] > 0]
+        if want is not None:
+            assert got == want[b]
+        else:
+            assert got == [k] * (N // k) + ([N % k] if N % k else [])
+    s.close()
+    model.close()
+    return rep
+
+
+@pytest.mark.parametrize("mean", [5.0, 2.0])
+def test_c3_whole_decode_in_lockstep(bpd, mean):
+    """The headline configuration, all 128 tokens, every iteration compared with the oracle (values too)."""
+    rep = _whole_decode(bpd, "C3", mean)
+    assert rep.max_logit_err <= 2e-2 and rep.max_hidden_err <= 2e-2
+
+
+def test_c4_whole_decode_in_lockstep(bpd):
+    """Batch 32 with ragged source lengths and per-row acceptance: four rows (shortest and longest source, first and
+    last row) followed through all 128 tokens in the launch configuration the benchmark times (two-stage heads)."""
+    w = WORKLOADS["C4"]
+    _, src_len = make_source(w)
+    rows = sorted({int(np.argmin(src_len)), int(np.argmax(src_len)), 0, w.batch - 1})
+    _whole_decode(bpd, "C4", 5.0, rows=rows, check_values=False)
+
+
+def test_c5_whole_image_in_lockstep(bpd):
+    """The super-resolution shape through all 3072 positions with every proposal accepted: the self-attention
+    schedule switches from one CTA per row to shared keys at 256 visible keys and folds several chunks per lump
+    beyond 2048; hidden states and logits are compared with the oracle in every iteration."""
+    rep = _whole_decode(bpd, "C5", 0.0, all_accepted=True)
+    assert rep.iterations == -(-3072 // 10)
+
+
+def test_full_attention_beyond_2048_keys(bpd):
+    """A small model decoded to 2320 positions with full causal attention: past key 2048 a rank's lumps wrap
+    around and hold several chunks each.  Greedy and blockwise agree, and the lock-step against the oracle (values
+    in every iteration) runs across the wrap."""
+    from harness import lockstep
+    w = Workload("midi-2k", MIDI.cfg, 0.05, 41, 42, 43, batch=1, src_lo=9, src_hi=9, n_decode=2320)
+    blob, model, src, src_len, om = _setup(bpd, w)
+    k, N = w.cfg.k_model, w.n_decode
+    for path in ("cluster", "persistent"):
+        s = bpd.Session(model, w.batch, w.max_src, N, options=LAYER_PATHS[path])
+        s.bpd_encode(src, src_len)
+        g_ids, _, _ = s.bpd_decode_greedy(N)
+        s.bpd_encode(src, src_len)
+        b_ids, _, _ = s.bpd_decode_blockwise(k, N)
+        assert np.array_equal(b_ids, g_ids), path
+
+        def all_accepted(b, j, it):
+            return forced_tail(g_ids[b], min(j, N), k, k, 0, w.cfg.vocab)
+        rep = lockstep(s, om, src, src_len, k, N, max_iters=N, tail_fn=all_accepted)
+        assert rep.emitted[0] == list(g_ids[0]) and rep.iterations == N // k, path
+        s.close()
+    model.close()
+
+
 # ---------------------------------------------------------------- approximate acceptance (Section 5)
 
 @pytest.mark.parametrize("accept", [("topn", 2), ("topn", 3), ("distance", 2)], ids=lambda a: f"{a[0]}{a[1]}")
@@ -419,17 +532,12 @@ def test_lazy_heads_give_the_same_decode(bpd, w):
     s.close()
     model.close()
 
-LAYER_PATHS = {
-    "persistent": {},                                             # one kernel for the whole layer stack (default)
-    "cluster": {"persistent_layers": 0},                          # three cluster launches per layer
-    "per-projection": {"persistent_layers": 0, "cluster_layers": 0},
-}
 
 
 @pytest.mark.parametrize("w", [MIDI, MIDI_BATCH], ids=lambda w: w.name)
 def test_layer_paths_agree(bpd, w):
-    """Sessions with few rows run the decoder layers in one persistent kernel (one cluster per head); the same
-    sessions can also run three cluster launches per layer or one kernel per projection.  The sums are split
+    """Sessions with few rows run each decoder layer as three cluster launches (one cluster per head); the same
+    sessions can also run all layers in one persistent kernel or one kernel per projection.  The sums are split
     differently, so the three agree to fp32 rounding of bf16-weight products, far inside the oracle tolerance --
     hidden states after every layer, decoder outputs and logits."""
     blob, model, src, src_len, om = _setup(bpd, w)
