@@ -100,13 +100,25 @@ def build_plan(w, greedy_ids, k, mean):
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle samples while the timed region runs."""
+    """nvidia-smi clock / throttle samples while the timed region runs.  The GPU is named by its UUID
+    (nvidia-smi numbers physical GPUs and ignores CUDA_VISIBLE_DEVICES, so a CUDA ordinal could
+    describe somebody else's GPU); the id is recorded beside the samples."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index):
-        self.index, self.rows, self.proc = index, [], None
+    def __init__(self, gpu_id):
+        self.index, self.rows, self.proc = str(gpu_id), [], None
+
+    @staticmethod
+    def identity(local: int) -> str:
+        """UUID of CUDA device ``local`` of this process in nvidia-smi's spelling, else its PCI bus id."""
+        import torch
+        props = torch.cuda.get_device_properties(local)
+        uuid = str(getattr(props, "uuid", "") or "")
+        if uuid:
+            return uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+        return f"{props.pci_domain_id:08x}:{props.pci_bus_id:02x}:{props.pci_device_id:02x}.0"
 
     def __enter__(self):
         try:
@@ -140,9 +152,9 @@ class ClockSampler:
                 if v.lower().startswith("active"):
                     reasons.add(n)
         if not sm:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "gpu": self.index}
         return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
-                "samples": len(sm)}
+                "samples": len(sm), "gpu": self.index}
 
 
 # --------------------------------------------------------------------------- oracle legs (CPU)
@@ -180,7 +192,15 @@ def run_reference(args):
     k = w.cfg.k_model
     blob = make_weights(w.cfg, w.weight_seed, w.sigma)
     src, src_len = make_source(w)
-    n_tokens = 32
+    n_tokens = w.n_decode                     # the whole decode: the same configuration as the GPU arm's step
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        # torch's launcher pins OMP_NUM_THREADS to 1 for its children; rank 0 is the only rank that works here,
+        # so it takes the host cores it would have had when started alone
+        try:
+            from threadpoolctl import threadpool_limits
+            threadpool_limits(limits=len(os.sched_getaffinity(0)))
+        except Exception:
+            pass
     tps, times, threads = oracle_sample(w, blob, src, src_len, k, MEAN_ACCEPT, n_tokens,
                                         repeats=args.steps + args.warmup)
     timed = times[args.warmup:]
@@ -189,10 +209,11 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * float(np.mean(timed)),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{HEADLINE}: big enc-dec 6+6, d_model 1024, k=8, batch 1 "
-                               f"(oracle sample: first {n_tokens} tokens, controlled acceptance mean {MEAN_ACCEPT})"},
+        "config": {"workload": f"{DESCRIPTIONS[HEADLINE]}, decode {n_tokens} tokens, controlled acceptance "
+                               f"(geometric mean {MEAN_ACCEPT})"},
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": threads, "kind": "oracle",
-                         "sample": f"first {n_tokens} of {w.n_decode} tokens per step"},
+                         "arithmetic": "numpy float64, matrix products on the BLAS thread pool",
+                         "sample": f"all {n_tokens} tokens of one decode per step"},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -211,6 +232,11 @@ def run_gpu(args):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but the launcher started {world} rank(s)")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py times the CUDA path and needs a GPU; there is no CPU fallback "
+                         "(--impl reference times the oracle)")
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
     torch.cuda.set_device(local)
@@ -251,7 +277,7 @@ def run_gpu(args):
     sess.bpd_set_forced_plan(plan, k)
     timed_decodes(args.warmup, "block")
     launches0 = bpd.bpd_kernel_launches()
-    with ClockSampler(local) as clocks:
+    with ClockSampler(ClockSampler.identity(local)) as clocks:
         ms_step = max_over_ranks(timed_decodes(args.steps, "block"), dev)
         launches = bpd.bpd_kernel_launches() - launches0
         # the timed region is a fraction of a second: keep the same load running (untimed) until nvidia-smi has
@@ -354,7 +380,8 @@ def run_gpu(args):
         n_tok = N
         tps, times, threads = oracle_sample(w, blob, src, src_len, k, MEAN_ACCEPT, n_tok, repeats=2)
         cpu = {"value": tps, "unit": "tokens/s", "cores": threads, "kind": "oracle",
-               "sample": f"first {n_tok} of {N} tokens, 2 decodes, {np.mean(times):.1f} s each"}
+               "arithmetic": "numpy float64, matrix products on the BLAS thread pool",
+               "sample": f"row 0, all {n_tok} tokens of the decode, 2 decodes, {np.mean(times):.1f} s each"}
     line = {
         "metric": METRIC if args.workload == HEADLINE else f"decoded tokens/s ({args.workload})",
         "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
@@ -382,7 +409,21 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
-def main():
+def spawn_replicas(n: int, argv) -> int:
+    """Start ``n`` copies of this script, one process per GPU, under torch's launcher and return its exit
+    code.  The replicas share nothing on the data path; the process group serves the barrier around the
+    timed region and the maximum over ranks."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *argv]
+    return subprocess.call(cmd)
+
+
+def main(argv=None):
+    argv = list(sys.argv[1:] if argv is None else argv)
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
@@ -391,7 +432,12 @@ def main():
     ap.add_argument("--workload", default=HEADLINE, choices=sorted(DESCRIPTIONS), help="configuration to time")
     ap.add_argument("--quick", action="store_true", help="skip the context modes")
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle leg")
-    args = ap.parse_args()
+    args = ap.parse_args(argv)
+    if args.gpus < 1:
+        ap.error("--gpus must be at least 1")
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started by hand rather than by a launcher: become the launcher of N replicas
+        sys.exit(spawn_replicas(args.gpus, argv))
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -173,6 +173,19 @@ int bpd_decode_greedy(bpd_session* s, int max_new, int32_t eos_id,
 int bpd_decode_blockwise(bpd_session* s, int k, int accept_mode, int max_new, int32_t eos_id,
                          int32_t* out_ids, int32_t* out_len, bpd_stats* stats);
 
+/* Blockwise parallel decoding in its two-call form (Section 3: predict,
+ * verify, accept), kept for comparison with the merged form of Section 4:
+ * every iteration is a Verify invocation (p_1 alone at the k block positions,
+ * followed by acceptance and the cache commit) and a Predict invocation (all
+ * k heads at the last accepted token, whose position is recomputed).  The
+ * ids and accepted block sizes are those of bpd_decode_blockwise; the number
+ * of model invocations is 2 per iteration instead of 1 per iteration + 1
+ * (stats->invocations), which is why the merged form is the product path.
+ * Arguments, outputs, forced plans and error behaviour as for
+ * bpd_decode_blockwise. */
+int bpd_decode_blockwise_twocall(bpd_session* s, int k, int accept_mode, int max_new, int32_t eos_id,
+                                 int32_t* out_ids, int32_t* out_len, bpd_stats* stats);
+
 /* One merged score-and-propose iteration (Section 4) on the session's current
  * state; on a freshly encoded session the priming pass runs first.
  * forced_tail: host [batch, k-1] replacing proposals 2..k of every row, or

@@ -66,6 +66,7 @@ _SIGS = {
     "bpd_encode": (_i, [_vp, _vp, _vp]),
     "bpd_decode_greedy": (_i, [_vp, _i, C.c_int32, _vp, _vp, C.POINTER(bpd_stats)]),
     "bpd_decode_blockwise": (_i, [_vp, _i, _i, _i, C.c_int32, _vp, _vp, C.POINTER(bpd_stats)]),
+    "bpd_decode_blockwise_twocall": (_i, [_vp, _i, _i, _i, C.c_int32, _vp, _vp, C.POINTER(bpd_stats)]),
     "bpd_iteration": (_i, [_vp, _i, _i, _i, C.c_int32, _vp, C.POINTER(bpd_iter_out)]),
     "bpd_set_forced_plan": (_i, [_vp, _vp, _i, _i]),
     "bpd_rewind": (_i, [_vp]),
@@ -217,6 +218,9 @@ class Session:
 
     def bpd_decode_blockwise(self, k: int, max_new: int, eos_id: int = -1, accept_mode: int = 0, fetch: bool = True):
         return self._decode(lib.bpd_decode_blockwise, (k, accept_mode, max_new, eos_id), max_new, fetch)
+
+    def bpd_decode_blockwise_twocall(self, k: int, max_new: int, eos_id: int = -1, accept_mode: int = 0, fetch: bool = True):
+        return self._decode(lib.bpd_decode_blockwise_twocall, (k, accept_mode, max_new, eos_id), max_new, fetch)
 
     def bpd_fetch_output(self, max_new: int):
         st = bpd_stats()

@@ -379,7 +379,7 @@ static VerifyParams verify_params(bpd_session* s, const PassArgs& a) {
   return vp;
 }
 static bool pass_is_lazy(const bpd_session* s, const PassArgs& a) {
-  return s->tc && s->lazy_heads && a.mode == kModeBlock && a.kcur > 1 && !a.logits_dump;
+  return s->tc && s->lazy_heads && a.mode == kModeBlock && a.kcur > 1 && a.kh > 1 && !a.logits_dump;
 }
 static bool wants_rank(const PassArgs& a) { return a.mode == kModeBlock && a.accept_kind == kAcceptTopN && a.kcur > 1; }
 
@@ -1004,6 +1004,12 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
 
 #undef PROF
 static int dispatch_eager(bpd_session* s, const PassArgs& a) {
+  if (a.mode == kModePredict) {
+    StepBackParams sp{s->st, s->B};
+    step_back_kernel<<<1, 32 * ceil_div(s->B, 32), 0, s->stream>>>(sp);
+    ++g_launches;
+    BPD_CUDA(cudaGetLastError());
+  }
   if (s->tc) return run_pass_tc(s, a);
   return s->m->cfg.dtype == 0 ? run_pass<float>(s, a) : run_pass<bf16>(s, a);
 }
@@ -1423,7 +1429,7 @@ static int wait_pass_flag(bpd_session* s, int slot, int* finished) {
     }
   }
 }
-static int decode_loop(bpd_session* s, const PassArgs& a, int max_passes) {
+static int decode_loop(bpd_session* s, const PassArgs* cycle, int n_cycle, int max_passes) {
   // a new epoch and pass counter for this decode, ordered on the stream behind whatever the previous one left
   s->epoch = (s->epoch % 0x0fffffff) + 1;
   int* stage = &s->pinned[200 + 2 * (s->epoch & 1)];
@@ -1436,7 +1442,7 @@ static int decode_loop(bpd_session* s, const PassArgs& a, int max_passes) {
       if (rc) return rc;
       if (finished) break;
     }
-    int rc = dispatch_pass(s, a);
+    int rc = dispatch_pass(s, cycle[it % n_cycle]);
     if (rc) return rc;
   }
   return BPD_OK;
@@ -1461,7 +1467,7 @@ int bpd_decode_greedy(bpd_session* s, int max_new, int32_t eos_id, int32_t* out_
   s->phase = kPhaseGreedy;
   BPD_CUDA(cudaEventRecord(s->ev0, s->stream));
   PassArgs a{kModeGreedy, 1, 1, 1, nullptr, 0, 0, max_new, eos_id, nullptr};
-  rc = decode_loop(s, a, max_new);
+  rc = decode_loop(s, &a, 1, max_new);
   if (rc) return rc;
   return finish_decode(s, max_new, out_ids, out_len, stats);
 }
@@ -1482,7 +1488,32 @@ int bpd_decode_blockwise(bpd_session* s, int k, int accept_mode, int max_new, in
   if (rc) return rc;
   PassArgs a{kModeBlock, k, k, k, s->plan_len ? s->plan_dev : nullptr, s->plan_len, k, max_new, eos_id, nullptr,
              acc.accept_kind, acc.accept_param, acc.min_block};
-  rc = decode_loop(s, a, max_new);
+  rc = decode_loop(s, &a, 1, max_new);
+  if (rc) return rc;
+  return finish_decode(s, max_new, out_ids, out_len, stats);
+}
+
+int bpd_decode_blockwise_twocall(bpd_session* s, int k, int accept_mode, int max_new, int32_t eos_id, int32_t* out_ids,
+                                 int32_t* out_len, bpd_stats* stats) {
+  int rc = check_decode_args(s, max_new, eos_id);
+  if (rc) return rc;
+  if (k < 1 || k > s->m->cfg.k_model) return fail(BPD_E_INVALID, "k = %d outside 1..%d", k, s->m->cfg.k_model);
+  PassArgs acc{};
+  if ((rc = decode_accept(accept_mode, k, &acc))) return rc;
+  if (s->phase != kPhaseEncoded) return fail(BPD_E_STATE, "bpd_decode_blockwise_twocall needs a freshly encoded session");
+  if (s->plan_len && s->plan_k != k) return fail(BPD_E_SHAPE, "forced plan was installed for k = %d", s->plan_k);
+  s->phase = kPhaseBlockwise;
+  BPD_CUDA(cudaEventRecord(s->ev0, s->stream));
+  // the first Predict scores the start token: the priming pass
+  PassArgs prime{kModePrime, 1, k, k, nullptr, 0, 0, max_new, eos_id, nullptr};
+  rc = dispatch_pass(s, prime);
+  if (rc) return rc;
+  // Verify: p_1 alone at the k block positions, then accept; Predict: all k heads at the last accepted token
+  PassArgs cycle[2] = {
+      PassArgs{kModeBlock, k, 1, 1, s->plan_len ? s->plan_dev : nullptr, s->plan_len, k, max_new, eos_id, nullptr,
+               acc.accept_kind, acc.accept_param, acc.min_block},
+      PassArgs{kModePredict, 1, k, k, nullptr, 0, 0, max_new, eos_id, nullptr}};
+  rc = decode_loop(s, cycle, 2, 2 * max_new);
   if (rc) return rc;
   return finish_decode(s, max_new, out_ids, out_len, stats);
 }

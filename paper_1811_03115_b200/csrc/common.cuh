@@ -117,7 +117,9 @@ struct RowState {
   int max_tgt;
 };
 
-enum PassMode { kModePrime = 0, kModeBlock = 1, kModeGreedy = 2 };
+// kModePredict: the Predict call of the two-call form -- like the priming pass, one row per sequence with all heads,
+// but at the position of the last accepted token instead of the start token.
+enum PassMode { kModePrime = 0, kModeBlock = 1, kModeGreedy = 2, kModePredict = 3 };
 
 // Acceptance criteria of the Verify substep (values match the public header).
 enum AcceptKind { kAcceptExact = 0, kAcceptTopN = 1, kAcceptDistance = 2 };

@@ -1165,15 +1165,17 @@ static __global__ void verify_commit_kernel(VerifyParams p) {
     const int* A = p.st.table + (size_t)b * p.kcur * p.kh;
     if (p.st.finished[b]) {
       p.st.khat[b] = 0;
-    } else if (p.mode != kModePrime && p.st.j[b] >= p.max_new) {
+    } else if (p.mode != kModePrime && p.mode != kModePredict && p.st.j[b] >= p.max_new) {
       // the caller lowered max_new below what the row already holds (bpd_iteration takes it per call): the row
       // is complete, nothing is appended or committed
       p.st.khat[b] = 0;
       p.st.finished[b] = 1;
-    } else if (p.mode == kModePrime) {
-      // start token becomes part of the prefix; its row of predictions is the first block
+    } else if (p.mode == kModePrime || p.mode == kModePredict) {
+      // priming: the start token becomes part of the prefix; its row of predictions is the first block.
+      // Predict call of the two-call form: the row of the last accepted token (the length was stepped back onto
+      // it) is part of the prefix again; its predictions are the next block.  The accepted count stays.
       p.st.len[b] += 1;
-      p.st.khat[b] = 0;
+      if (p.mode == kModePrime) p.st.khat[b] = 0;
       for (int i = 0; i < p.knext; ++i) blk[i] = A[i];
       atomicOr(&any_open, 1);
     } else if (p.mode == kModeGreedy) {
@@ -1224,10 +1226,24 @@ static __global__ void verify_commit_kernel(VerifyParams p) {
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    p.st.stats[p.mode == kModePrime ? 3 : 2] += 1;
+    p.st.stats[(p.mode == kModePrime || p.mode == kModePredict) ? 3 : 2] += 1;
     if (!any_open) *p.st.all_done = 1;
     signal_host(p.st, !any_open);
   }
+}
+
+// Before a Predict call of the two-call form (Section 3): the single row it scores is the last accepted token, which
+// already sits in the cache at position len - 1.  Step the length back onto it and make it the block's first entry;
+// the pass recomputes that position and the verify kernel (kModePredict) moves the length forward again.
+struct StepBackParams { RowState st; int B; };
+static __global__ void step_back_kernel(StepBackParams p) {
+  if (*p.st.all_done) return;
+  const int b = threadIdx.x;
+  if (b >= p.B || p.st.finished[b]) return;
+  const int khat = p.st.khat[b];
+  if (khat < 1 || p.st.len[b] < 2) return;       // nothing accepted since the last Predict: the block stands
+  p.st.len[b] -= 1;
+  p.st.block[b * kMaxK] = p.st.cur_block[b * kMaxK + khat - 1];
 }
 
 // ------------------------------------------------------------------ lazy heads (two-stage evaluation)

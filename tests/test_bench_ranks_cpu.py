@@ -1,5 +1,6 @@
 """The N > 1 leg of bench.py on CPU: two gloo ranks, replicas only -- the job's time is the slowest rank's,
-its throughput all ranks' tokens over that time, and only rank 0 of the reference arm prints."""
+its throughput all ranks' tokens over that time, and only rank 0 of the reference arm prints.  `bench.py --gpus 2`
+started by hand launches its own two ranks; without a GPU the CUDA arm refuses loudly instead of falling back."""
 import json
 import os
 import socket
@@ -56,3 +57,34 @@ def test_reference_arm_is_silent_on_other_ranks():
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
                         "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=300)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def _run_bench(*argv, timeout=600):
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    return subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), *argv], env=env, capture_output=True,
+                          text=True, timeout=timeout)
+
+
+def test_gpus_2_started_by_hand_launches_two_ranks_and_prints_one_line():
+    """main() itself: --gpus 2 with no launcher around it re-executes under torch's launcher; the reference arm's
+    rank 0 prints the one JSON line (n_gpus 2, the whole 128-token decode), rank 1 exits 0 without work."""
+    r = _run_bench("--gpus", "2", "--impl", "reference", "--steps", "1", "--warmup", "0")
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["steps"] == 1
+    assert "decode 128 tokens" in line["config"]["workload"] and line["cpu_baseline"]["kind"] == "oracle"
+    assert line["e2e"]["value"] == line["value"] and line["gpu_launches"] == 0
+
+
+def test_cuda_arm_refuses_loudly_without_a_gpu():
+    import torch
+    if torch.cuda.is_available():
+        import pytest
+        pytest.skip("a GPU is present")
+    for argv in (("--steps", "1", "--warmup", "0"), ("--gpus", "2", "--steps", "1", "--warmup", "0")):
+        r = _run_bench(*argv)
+        assert r.returncode != 0
+        assert "needs a GPU" in (r.stderr + r.stdout)
+        assert not [ln for ln in r.stdout.splitlines() if ln.startswith("{")]

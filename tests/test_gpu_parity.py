@@ -729,3 +729,56 @@ def test_bounded_wait_expires_and_the_context_survives(bpd):
     w = torch.randn(10, 64).cuda()
     y = bpd.bpd_op_linear(x, w).cpu()
     assert torch.allclose(y, x.cpu() @ w.cpu().T, atol=1e-4)
+
+
+# ---------------------------------------------------------------- the two-call form (Section 3)
+
+@pytest.mark.parametrize("w", [WORKLOADS["C1"], MINI, MINI_BATCH, MIDI], ids=lambda w: w.name)
+def test_two_call_form_gives_the_merged_decode(bpd, w):
+    """Predict and Verify as separate invocations: the same ids and the same accepted block sizes as the
+    merged form and as the oracle's two-call loop, at two invocations per iteration instead of one per
+    iteration plus the priming pass."""
+    from oracle.decode import TransformerScorer, blockwise_twocall
+    blob, model, src, src_len, om = _setup(bpd, w)
+    k, N = w.cfg.k_model, w.n_decode
+    s = bpd.Session(model, w.batch, w.max_src, N)
+    s.bpd_encode(src, src_len)
+    g_ids, _, _ = s.bpd_decode_greedy(N)
+    # free running: whatever the heads propose
+    s.bpd_encode(src, src_len)
+    m_ids, m_len, m_st = s.bpd_decode_blockwise(k, N)
+    s.bpd_encode(src, src_len)
+    t_ids, t_len, t_st = s.bpd_decode_blockwise_twocall(k, N)
+    assert np.array_equal(t_ids, g_ids) and np.array_equal(t_ids, m_ids) and np.array_equal(t_len, m_len)
+    assert t_st.khat_hist == m_st.khat_hist and t_st.row_iterations == m_st.row_iterations
+    assert m_st.invocations == m_st.iterations + 1
+    assert t_st.invocations == 2 * t_st.iterations          # Section 4: 2m/k against m/k + 1
+    # controlled acceptance: the same schedule through both forms, and through the oracle's two-call loop on row 0
+    plan, sched = _plan(w, g_ids, k, 2.0)
+    s.bpd_encode(src, src_len)
+    s.bpd_set_forced_plan(plan, k)
+    _, _, m_st = s.bpd_decode_blockwise(k, N)
+    s.bpd_encode(src, src_len)
+    s.bpd_set_forced_plan(plan, k)
+    t_ids, _, t_st = s.bpd_decode_blockwise_twocall(k, N)
+    assert np.array_equal(t_ids, g_ids) and t_st.khat_hist == m_st.khat_hist
+    assert t_st.invocations == 2 * t_st.iterations and t_st.iterations == m_st.iterations
+    if w.batch == 1:
+        G, R = sched[0]
+        sc = TransformerScorer(om, src[0, :src_len[0]], cached=True, capacity=N + 2 * k + 2)
+        want = blockwise_twocall(sc, k, N, tail_fn=lambda j, it: forced_tail(g_ids[0], j, k, int(G[j]), int(R[j]), w.cfg.vocab))
+        assert want.ids == list(t_ids[0])
+        assert want.invocations == t_st.invocations
+        hist = [0] * 17
+        for kh in want.khats:
+            hist[kh] += 1
+        assert list(t_st.khat_hist) == hist
+    # an end-of-sequence id inside a block ends the row in both forms at the same place
+    eos = int(g_ids[0][min(5, N - 1)])
+    s.bpd_encode(src, src_len)
+    m_ids, m_len, _ = s.bpd_decode_blockwise(k, N, eos_id=eos)
+    s.bpd_encode(src, src_len)
+    t_ids, t_len, _ = s.bpd_decode_blockwise_twocall(k, N, eos_id=eos)
+    assert np.array_equal(t_ids, m_ids) and np.array_equal(t_len, m_len)
+    s.close()
+    model.close()
