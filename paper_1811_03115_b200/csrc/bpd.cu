@@ -1674,8 +1674,7 @@ int bpd_op_vocab_argmax(const void* x, const void* w, int rows, int d, int vocab
     tc::Scratch sc{reinterpret_cast<float*>(p + L.ws_off), L.ws_floats, reinterpret_cast<unsigned*>(p + L.cnt_off),
                    L.n_counters, reinterpret_cast<unsigned*>(p + L.done_off),
                    reinterpret_cast<unsigned long long*>(p + L.pv_off), L.part_elems, reinterpret_cast<int*>(p + L.err_off), 0, 1};
-    const long long plane = (reinterpret_cast<const bf16*>(p + L.zero_off) - static_cast<const bf16*>(x));
-    tc::Operands op{w, vocab, x, plane, d, rows, d};
+    tc::Operands op{w, vocab, x, 0, d, rows, d, p + L.zero_off};   // the lo plane is the scratch's zero block
     tc::TcParams tp;
     memset(&tp, 0, sizeof(tp));
     tp.out_idx = out_idx; tp.out_val = out_val;
@@ -1719,8 +1718,7 @@ int bpd_op_linear(const void* x, const void* w, const void* bias, int rows, int 
     tc::Scratch sc{reinterpret_cast<float*>(p + L.ws_off), L.ws_floats, reinterpret_cast<unsigned*>(p + L.cnt_off),
                    L.n_counters, reinterpret_cast<unsigned*>(p + L.done_off),
                    reinterpret_cast<unsigned long long*>(p + L.pv_off), L.part_elems, reinterpret_cast<int*>(p + L.err_off), 0, 1};
-    const long long plane = (reinterpret_cast<const bf16*>(p + L.zero_off) - static_cast<const bf16*>(x));
-    tc::Operands op{w, out_f, x, plane, in_f, rows, in_f};
+    tc::Operands op{w, out_f, x, 0, in_f, rows, in_f, p + L.zero_off};   // the lo plane is the scratch's zero block
     tc::TcParams tp;
     memset(&tp, 0, sizeof(tp));
     tp.bias = static_cast<const bf16*>(bias); tp.relu = relu; tp.out_f32 = y; tp.ldo = out_f;

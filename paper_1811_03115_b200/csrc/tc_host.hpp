@@ -111,6 +111,8 @@ inline int get_encode_fn(EncodeTiledFn* out) {
   return BPD_OK;
 }
 
+constexpr size_t kMapCacheMax = 4096;   // descriptors kept per process (128 bytes each)
+
 // bf16 matrix [rows, cols] with `ld` elements between rows; boxes of (64 columns, box_rows rows), 128-byte swizzle.
 inline int make_map(const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows, CUtensorMap* out) {
   typedef std::tuple<const void*, uint64_t, uint64_t, uint64_t, uint32_t> Key;
@@ -136,6 +138,10 @@ inline int make_map(const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, 
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return fail(BPD_E_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
   std::lock_guard<std::mutex> lock(mu);
+  // A descriptor is a pure function of its key, so an entry never goes stale (a freed and reused address yields
+  // the same descriptor); the cache only saves the encode call.  Keep it bounded: sessions come and go in a
+  // long-lived process, each with its own activation buffers.
+  if (cache.size() >= kMapCacheMax) cache.clear();
   cache[key] = *out;
   return BPD_OK;
 }
@@ -196,6 +202,7 @@ struct Operands {
   const void* w; int w_rows;            // weights [w_rows, K] (all slices stacked)
   const void* x; long long x_plane;     // activation planes: hi at x, lo at x + x_plane (elements)
   long long ldx; int x_rows; int x_cols;  // allocated rows, total columns per row
+  const void* x_lo = nullptr;           // the lo plane when it lives in another allocation (x_plane unused then)
 };
 
 template <int EPI>
@@ -223,7 +230,7 @@ int launch(const Operands& op, int N, int K, int T, TcParams p, const Scratch& s
   if (rc) return rc;
   rc = make_map(op.x, (uint64_t)op.x_rows, (uint64_t)op.x_cols, (uint64_t)op.ldx, (uint32_t)bn, &mh);
   if (rc) return rc;
-  rc = make_map(static_cast<const bf16*>(op.x) + op.x_plane, (uint64_t)op.x_rows, (uint64_t)op.x_cols, (uint64_t)op.ldx,
+  rc = make_map(op.x_lo ? static_cast<const bf16*>(op.x_lo) : static_cast<const bf16*>(op.x) + op.x_plane, (uint64_t)op.x_rows, (uint64_t)op.x_cols, (uint64_t)op.ldx,
                 (uint32_t)bn, &ml);
   if (rc) return rc;
   p.T = T; p.N = N; p.K = K; p.bn = bn; p.splits = pl.splits; p.chunks_per_split = pl.chunks_per_split;
