@@ -228,7 +228,9 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
   void* stack_layers = a.take_bytes(fused_ok ? (size_t)c.n_dec * sizeof(stack::LayerPtrs) : 0);
   float* stack_ws = a.take<float>(fused_ok ? (size_t)2 * c.H * fused::kMaxRows * d : 0);
   unsigned* stack_bar = a.take<unsigned>(stack::kBarWords);
+  float* ln_stats = a.take<float>((size_t)ceil_div(d, 128) * Rall * 2);
   if (s) {
+    s->ln_stats = ln_stats;
     s->stack_layers = stack_layers; s->stack_ws = stack_ws; s->stack_bar = stack_bar;
     s->fused_ws = fused_ws; s->fused_counters = fused_counters;
     s->x = x; s->h_f32 = h_f32; s->xn = xn; s->qbuf = qbuf; s->attn = attn; s->ffh = ffh; s->u = u; s->o = o;
@@ -866,6 +868,12 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
   ep.d = d; ep.vocab = c.V; ep.st = s->st; ep.forced = a.forced; ep.forced_rows = a.forced_rows;
   ep.kforced = a.kforced; ep.src = nullptr; ep.all_done = done;
   if (fold) { ep.gain = static_cast<const bf16*>(m->dec[0].ln1g); ep.xg_hi = static_cast<bf16*>(s->xn); ep.xg_plane = s->pl_xn; }
+  // passes of more than 16 rows: layer-norm statistics travel as per-tile partial results (see TcParams::stat_out)
+  const bool wide = fold && R > 16;
+  const int parts = d / 128;
+  if (wide) { ep.stat_out = s->ln_stats; ep.stat_T = R; }
+  auto stats_from = [&](tc::TcParams& q) { if (wide) { q.ln_x = nullptr; q.stat_in = s->ln_stats; q.stat_parts = parts; q.stat_T = R; } };
+  auto stats_to = [&](tc::TcParams& q) { if (wide && q.g_next) { q.stat_out = s->ln_stats; q.stat_T = R; } };
   PROF(kProfEmbed, embed_kernel<bf16><<<R, 128, 0, st>>>(ep););
   ++g_launches;
   const tc::Operands at{nullptr, 0, s->attn, s->pl_attn, d, s->rows_all, d};
@@ -877,7 +885,7 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
     pq.out_f32 = static_cast<float*>(s->qbuf); pq.ldo = d; pq.d = d;
     pq.kcache = static_cast<bf16*>(s->kcache[l]); pq.vcache = static_cast<bf16*>(s->vcache[l]);
     pq.st = s->st; pq.rows_per_b = a.kcur;
-    if (fold) { pq.ln_x = s->x; pq.ln_d = d; pq.ln_eps = c.eps; pq.ln_s = L.s_qkv; pq.ln_c = L.c_qkv; }
+    if (fold) { pq.ln_x = s->x; pq.ln_d = d; pq.ln_eps = c.eps; pq.ln_s = L.s_qkv; pq.ln_c = L.c_qkv; stats_from(pq); }
     PROF(kProfQkv, BPD_TRY(tc::launch<tc::kTcQkv>(with_w(xn, L.wqkv, 3 * d), 3 * d, d, R, pq, sc, st, 1, 0, 0, pdl)); ++g_launches);
     AttnParams ap;
     memset(&ap, 0, sizeof(ap));
@@ -889,12 +897,12 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
     ++g_launches;
     tc::TcParams po = tc_params(nullptr, 0, done);
     po.out_f32 = s->x; po.ldo = d;
-    if (fold) { po.g_next = static_cast<const bf16*>(L.ln2g); po.xg_hi = static_cast<bf16*>(s->xn); po.xg_plane = s->pl_xn; }
+    if (fold) { po.g_next = static_cast<const bf16*>(L.ln2g); po.xg_hi = static_cast<bf16*>(s->xn); po.xg_plane = s->pl_xn; stats_to(po); }
     PROF(kProfOproj, BPD_TRY(tc::launch<tc::kTcResidual>(with_w(at, L.wo, d), d, d, R, po, sc, st, 1, 0, 0, pdl)); ++g_launches);
     if (!fold) PROF(kProfLn, launch_ln<bf16, float>(s->x, L.ln2g, L.ln2b, s->xn, nullptr, R, d, c.eps, done, st, s->pl_xn, pdl););
     tc::TcParams pc = tc_params(nullptr, 0, done);
     pc.out_f32 = static_cast<float*>(s->qbuf); pc.ldo = d;
-    if (fold) { pc.ln_x = s->x; pc.ln_d = d; pc.ln_eps = c.eps; pc.ln_s = L.s_cq; pc.ln_c = L.c_cq; }
+    if (fold) { pc.ln_x = s->x; pc.ln_d = d; pc.ln_eps = c.eps; pc.ln_s = L.s_cq; pc.ln_c = L.c_cq; stats_from(pc); }
     PROF(kProfCrossQ, BPD_TRY(tc::launch<tc::kTcF32>(with_w(xn, L.cwq, d), d, d, R, pc, sc, st, 1, 0, 0, pdl)); ++g_launches);
     ap.causal = 0; ap.limit_b = s->st.src_len; ap.k = s->crosskv[l]; ap.v = static_cast<float*>(s->crosskv[l]) + d;
     ap.ldkv = 2 * d; ap.bstride = (long long)s->max_src * 2 * d; ap.paged = 0;
@@ -909,16 +917,16 @@ static int run_pass_tc(bpd_session* s, const PassArgs& a) {
       PROF(kProfCrossAttn, launch_attention<float, float>(ap, st, pdl););
     }
     ++g_launches;
-    if (fold) po.g_next = static_cast<const bf16*>(L.ln3g);
+    if (fold) { po.g_next = static_cast<const bf16*>(L.ln3g); stats_to(po); }
     PROF(kProfCrossO, BPD_TRY(tc::launch<tc::kTcResidual>(with_w(at, L.cwo, d), d, d, R, po, sc, st, 1, 0, 0, pdl)); ++g_launches);
     if (!fold) PROF(kProfLn, launch_ln<bf16, float>(s->x, L.ln3g, L.ln3b, s->xn, nullptr, R, d, c.eps, done, st, s->pl_xn, pdl););
     tc::TcParams p1 = tc_params(L.b1, 1, done);
     p1.out_hi = static_cast<bf16*>(s->ffh); p1.plane = s->pl_ffh; p1.ldo = f;
-    if (fold) { p1.ln_x = s->x; p1.ln_d = d; p1.ln_eps = c.eps; p1.ln_s = L.s_f1; p1.ln_c = L.c_f1; }
+    if (fold) { p1.ln_x = s->x; p1.ln_d = d; p1.ln_eps = c.eps; p1.ln_s = L.s_f1; p1.ln_c = L.c_f1; stats_from(p1); }
     PROF(kProfFfn1, BPD_TRY(tc::launch<tc::kTcPlanes>(with_w(xn, L.w1, f), f, d, R, p1, sc, st, 1, 0, 0, pdl)); ++g_launches);
     tc::TcParams p2 = tc_params(L.b2, 0, done);
     p2.out_f32 = s->x; p2.ldo = d;
-    if (fold && l + 1 < c.n_dec) { p2.g_next = static_cast<const bf16*>(m->dec[l + 1].ln1g); p2.xg_hi = static_cast<bf16*>(s->xn); p2.xg_plane = s->pl_xn; }
+    if (fold && l + 1 < c.n_dec) { p2.g_next = static_cast<const bf16*>(m->dec[l + 1].ln1g); p2.xg_hi = static_cast<bf16*>(s->xn); p2.xg_plane = s->pl_xn; stats_to(p2); }
     PROF(kProfFfn2, BPD_TRY(tc::launch<tc::kTcResidual>(with_w(fx, L.w2, d), d, f, R, p2, sc, st, 1, 0, 0, pdl)); ++g_launches);
     if (a.layer_dump)
       BPD_CUDA(cudaMemcpyAsync(a.layer_dump + (size_t)l * R * d, s->x, sizeof(float) * R * d, cudaMemcpyDeviceToDevice, st));
@@ -1233,7 +1241,9 @@ int bpd_session_create_opt(const bpd_model* model, int batch, int max_src, int m
   s->lazy_heads = s->tc && (o.lazy_heads >= 0 ? o.lazy_heads != 0 : batch * model->cfg.k_model >= 64);
   s->last_pass_lazy = 0;
   // with at most 16 rows per pass every projection CTA can afford the row statistics itself
-  s->fold_ln = (s->tc && batch * model->cfg.k_model <= 16 && o.fold_layer_norms != 0) ? 1 : 0;
+  // passes of at most 16 rows take the statistics from the stream itself; wider ones need whole 128-feature tiles (and
+  // the embedding kernel whole warps: d_model a multiple of 256)
+  s->fold_ln = (s->tc && o.fold_layer_norms != 0 && (batch * model->cfg.k_model <= 16 || model->cfg.d % 256 == 0)) ? 1 : 0;
   s->fused = (s->tc && fused::supported(model->cfg.d, model->cfg.H, model->cfg.d_ff, batch * model->cfg.k_model) &&
               o.cluster_layers != 0) ? 1 : 0;
   s->opt.persistent_layers = o.persistent_layers == 1 ? 1 : 0;   // opt-in: measured slower than the cluster launches
@@ -1595,6 +1605,16 @@ int bpd_debug_set_stack_trace(void* dev_buffer) {
   unsigned long long* ptr = static_cast<unsigned long long*>(dev_buffer);
   BPD_CUDA(cudaMemcpyToSymbol(stack::g_stack_trace, &ptr, sizeof(ptr)));
 
+  return BPD_OK;
+}
+#endif
+
+#ifdef BPD_TC_TRACE
+// Development builds only: where the projection kernel writes its per-CTA step timestamps (4096 * 16 unsigned 64-bit
+// words of device memory), or null to stop.
+int bpd_debug_set_tc_trace(void* dev_buffer) {
+  unsigned long long* ptr = static_cast<unsigned long long*>(dev_buffer);
+  BPD_CUDA(cudaMemcpyToSymbol(tc::g_tc_trace, &ptr, sizeof(ptr)));
   return BPD_OK;
 }
 #endif

@@ -13,12 +13,30 @@
 // skips its remaining work, waits (bounded) for copies in flight, frees its
 // tensor memory and returns.
 #pragma once
+#include <type_traits>
 #include <cuda.h>
 
 #include "common.cuh"
 
 namespace bpd {
 namespace tc {
+
+#ifdef BPD_TC_TRACE
+// Development builds only: per-CTA step timestamps of the projection kernel (16 words per CTA, up to 4096 CTAs of
+// the launches that run while the pointer is set; 128 regions chosen by the host's launch counter).
+__device__ unsigned long long* g_tc_trace = nullptr;
+__device__ __forceinline__ void tc_stamp(int region, int slot) {
+  if (!g_tc_trace) return;
+  const unsigned cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+  if (cta >= 2047) return;
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  g_tc_trace[((size_t)region * 2048 + cta) * 16 + slot] = t;
+}
+#define BPD_TC_STAMP(slot) tc_stamp(p.trace_id, slot)
+#else
+#define BPD_TC_STAMP(slot) do { } while (0)
+#endif
 
 constexpr int kBM = 128;          // features per tile (MMA M)
 constexpr int kBK = 64;           // K elements per pipeline stage (128 bytes of bf16: one swizzle row)
@@ -69,6 +87,14 @@ struct TcParams {
   const float* ln_s; const float* ln_c;        // [N]: sum_c gain_c w[n][c]  and  sum_c shift_c w[n][c] + bias[n]
   // kTcResidual: also write planes of the updated stream times the next layer norm's gain
   const bf16* g_next; bf16* xg_hi; long long xg_plane;
+  // Wide token tiles (more than 16 tokens) cannot afford to read whole rows of the residual stream for the folded
+  // layer norm.  There the kernel that updates the stream also writes, per (128-feature tile, token), the mean and
+  // the sum of squared deviations of its 128 new values (stat_out, [tiles][stat_T][2]); the projection that
+  // consumes the normalised stream merges the stat_parts tiles of a token in tile order (stat_in).
+  float* stat_out; const float* stat_in; int stat_parts; int stat_T;
+#ifdef BPD_TC_TRACE
+  int trace_id;
+#endif
   int* error;                  // device error word
   const int* all_done;
   int stream_weights;          // 1: the weights are read once per launch (one token tile): load them "evict first"
@@ -300,75 +326,215 @@ __device__ __forceinline__ uint2 pack4_bf16(const bf16 (&b)[4]) {
   return make_uint2((uint32_t)__bfloat16_as_ushort(b[0]) | ((uint32_t)__bfloat16_as_ushort(b[1]) << 16),
                     (uint32_t)__bfloat16_as_ushort(b[2]) | ((uint32_t)__bfloat16_as_ushort(b[3]) << 16));
 }
+// A 16-byte load from L2 that stays where it is written: the compiler otherwise sinks such loads to their first use,
+// which turns a batch of independent loads into a chain of round trips.
+__device__ __forceinline__ float4 ld_cg_v4_here(const float* ptr) {
+  float4 v;
+  asm volatile("ld.global.cg.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(ptr) : "memory");
+  return v;
+}
+
+// Per-thread constants of an item's four features.
+struct FinishCtx {
+  float bias[4], gn[4], lns[4];
+  bool folded;     // y = rstd * (acc - mean * ln_s) + ln_c; ln_c holds the bias
+  int n, g;
+};
 template <int EPI>
-__device__ __forceinline__ void tc_finish_tile(const TcParams& p, int z, int t0, int nt, int tile, const float* s_t, int tstride,
-                                               const unsigned long long* s_slot, int et) {
-  const int g = et & 31;
-  const int n = tile * kBM + g * 4;                 // first of this item's four features (within the slice)
-  if (n >= p.N) return;
-  float bias[4] = {0.f, 0.f, 0.f, 0.f}, gn[4] = {0.f, 0.f, 0.f, 0.f};
-  if (p.bias) {
-    const uint2 bw = *reinterpret_cast<const uint2*>(p.bias + n + p.zofs_n * z);
-    bias[0] = __uint_as_float(bw.x << 16); bias[1] = __uint_as_float(bw.x & 0xffff0000u);
-    bias[2] = __uint_as_float(bw.y << 16); bias[3] = __uint_as_float(bw.y & 0xffff0000u);
+__device__ __forceinline__ bool tc_finish_setup(const TcParams& p, int z, int tile, int et, FinishCtx& c) {
+  c.g = et & 31;
+  c.n = tile * kBM + c.g * 4;                       // first of this item's four features (within the slice)
+  if (c.n >= p.N) return false;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) { c.bias[e] = 0.f; c.gn[e] = 0.f; c.lns[e] = 0.f; }
+  c.folded = (p.stat_in != nullptr);
+  if (c.folded) {
+    const float4 s4 = *reinterpret_cast<const float4*>(p.ln_s + c.n), c4 = *reinterpret_cast<const float4*>(p.ln_c + c.n);
+    c.lns[0] = s4.x; c.lns[1] = s4.y; c.lns[2] = s4.z; c.lns[3] = s4.w;
+    c.bias[0] = c4.x; c.bias[1] = c4.y; c.bias[2] = c4.z; c.bias[3] = c4.w;
+  } else if (p.bias) {
+    const uint2 bw = *reinterpret_cast<const uint2*>(p.bias + c.n + p.zofs_n * z);
+    c.bias[0] = __uint_as_float(bw.x << 16); c.bias[1] = __uint_as_float(bw.x & 0xffff0000u);
+    c.bias[2] = __uint_as_float(bw.y << 16); c.bias[3] = __uint_as_float(bw.y & 0xffff0000u);
   }
   if (EPI == kTcResidual && p.g_next) {
-    const uint2 gw = *reinterpret_cast<const uint2*>(p.g_next + n);
-    gn[0] = __uint_as_float(gw.x << 16); gn[1] = __uint_as_float(gw.x & 0xffff0000u);
-    gn[2] = __uint_as_float(gw.y << 16); gn[3] = __uint_as_float(gw.y & 0xffff0000u);
+    const uint2 gw = *reinterpret_cast<const uint2*>(p.g_next + c.n);
+    c.gn[0] = __uint_as_float(gw.x << 16); c.gn[1] = __uint_as_float(gw.x & 0xffff0000u);
+    c.gn[2] = __uint_as_float(gw.y << 16); c.gn[3] = __uint_as_float(gw.y & 0xffff0000u);
   }
-  for (int tr = et >> 5; tr < nt; tr += 4) {
-    const int t = t0 + tr;
-    const float4 a = *reinterpret_cast<const float4*>(s_t + tr * tstride + g * 4);
-    float v[4] = {a.x + bias[0], a.y + bias[1], a.z + bias[2], a.w + bias[3]};
-    if (p.relu) {
+  return true;
+}
+// Finishes one item: token t (row tr of the tile), features c.n .. c.n + 3, accumulated values a; `old` is the
+// residual stream's current content (only read by the caller when the new value is needed: residual with g_next).
+template <int EPI>
+__device__ __forceinline__ void tc_finish_item(const TcParams& p, const FinishCtx& c, int z, int t, int tr, const float4& a,
+                                               float4& old, const unsigned long long* s_slot, const float* s_mean,
+                                               const float* s_rstd) {
+  const int n = c.n;
+  float v[4] = {a.x + c.bias[0], a.y + c.bias[1], a.z + c.bias[2], a.w + c.bias[3]};
+  if (c.folded) {
+    const float mu = s_mean[tr], rs = s_rstd[tr];
+    v[0] = rs * (a.x - mu * c.lns[0]) + c.bias[0]; v[1] = rs * (a.y - mu * c.lns[1]) + c.bias[1];
+    v[2] = rs * (a.z - mu * c.lns[2]) + c.bias[2]; v[3] = rs * (a.w - mu * c.lns[3]) + c.bias[3];
+  }
+  if (p.relu) {
 #pragma unroll
-      for (int e = 0; e < 4; ++e) v[e] = fmaxf(v[e], 0.f);
+    for (int e = 0; e < 4; ++e) v[e] = fmaxf(v[e], 0.f);
+  }
+  if (EPI == kTcPlanes || EPI == kTcHeadOut) {
+    const int nz = n + p.zofs_n * z;
+    if (EPI == kTcHeadOut) {
+      const float4 h = __ldg(reinterpret_cast<const float4*>(p.h + (size_t)t * p.d + (n % p.d)));
+      const float pre[4] = {h.x, h.y, h.z, h.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) v[e] = (p.head_identity && nz < p.d) ? pre[e] : v[e] + pre[e];
     }
-    if (EPI == kTcPlanes || EPI == kTcHeadOut) {
-      const int nz = n + p.zofs_n * z;
-      if (EPI == kTcHeadOut) {
-        const float4 h = __ldg(reinterpret_cast<const float4*>(p.h + (size_t)t * p.d + (n % p.d)));
-        const float pre[4] = {h.x, h.y, h.z, h.w};
+    bf16 hi[4], lo[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) v[e] = (p.head_identity && nz < p.d) ? pre[e] : v[e] + pre[e];
-      }
+    for (int e = 0; e < 4; ++e) split_bf16(v[e], hi[e], lo[e]);
+    const long long o = (long long)t * p.ldo + nz;
+    *reinterpret_cast<uint2*>(p.out_hi + o) = pack4_bf16(hi);
+    *reinterpret_cast<uint2*>(p.out_hi + o + p.plane) = pack4_bf16(lo);
+  } else if (EPI == kTcF32) {
+    *reinterpret_cast<float4*>(p.out_f32 + (long long)t * p.ldo + n) = make_float4(v[0], v[1], v[2], v[3]);
+  } else if (EPI == kTcResidual) {
+    float4* xp = reinterpret_cast<float4*>(p.out_f32 + (long long)t * p.ldo + n);
+    if (!p.g_next) {
+      // one writer per element: x += v as a 16-byte reduction, nothing to read back
+      asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(xp), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]) : "memory");
+      return;
+    }
+    const float xn[4] = {old.x + v[0], old.y + v[1], old.z + v[2], old.w + v[3]};
+    *xp = make_float4(xn[0], xn[1], xn[2], xn[3]);
+    {
       bf16 hi[4], lo[4];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) split_bf16(v[e], hi[e], lo[e]);
-      const long long o = (long long)t * p.ldo + nz;
-      *reinterpret_cast<uint2*>(p.out_hi + o) = pack4_bf16(hi);
-      *reinterpret_cast<uint2*>(p.out_hi + o + p.plane) = pack4_bf16(lo);
-    } else if (EPI == kTcF32) {
+      for (int e = 0; e < 4; ++e) split_bf16(xn[e] * c.gn[e], hi[e], lo[e]);
+      *reinterpret_cast<uint2*>(p.xg_hi + (long long)t * p.ldo + n) = pack4_bf16(hi);
+      *reinterpret_cast<uint2*>(p.xg_hi + (long long)t * p.ldo + n + p.xg_plane) = pack4_bf16(lo);
+    }
+    old = make_float4(xn[0], xn[1], xn[2], xn[3]);   // handed back for the per-tile statistics
+  } else if (EPI == kTcQkv) {
+    const int d = p.d;
+    if (n < d) {
       *reinterpret_cast<float4*>(p.out_f32 + (long long)t * p.ldo + n) = make_float4(v[0], v[1], v[2], v[3]);
-    } else if (EPI == kTcResidual) {
-      float4* xp = reinterpret_cast<float4*>(p.out_f32 + (long long)t * p.ldo + n);
-      if (!p.g_next) {
-        // one writer per element: x += v as a 16-byte reduction, nothing to read back
-        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(xp), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]) : "memory");
-        continue;
-      }
-      const float4 old = *xp;
-      const float xn[4] = {old.x + v[0], old.y + v[1], old.z + v[2], old.w + v[3]};
-      *xp = make_float4(xn[0], xn[1], xn[2], xn[3]);
-      {
-        bf16 hi[4], lo[4];
+    } else {
+      const bf16 b4[4] = {__float2bfloat16_rn(v[0]), __float2bfloat16_rn(v[1]), __float2bfloat16_rn(v[2]), __float2bfloat16_rn(v[3])};
+      bf16* dst = (n < 2 * d) ? p.kcache + s_slot[tr] + (n - d) : p.vcache + s_slot[tr] + (n - 2 * d);
+      *reinterpret_cast<uint2*>(dst) = pack4_bf16(b4);
+    }
+  }
+}
+// Per-tile statistics of TB tokens at once (kTcResidual with stat_out): the warp holds the tile's 128 new values of
+// each token, four per lane (N is a multiple of 128 here: every lane is live).  Sums of deviations from the token's
+// first value in the tile, and of their squares, are reduced for all TB tokens together so that the shuffles of one
+// token hide behind those of the others; mean and squared deviations about the mean follow exactly from the two.
+template <int TB>
+__device__ __forceinline__ void tc_tile_stats(const TcParams& p, const FinishCtx& c, int t0, int tb, int nt, const float4 (&xn)[TB]) {
+  float s1[TB], s2[TB], pivot[TB];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) split_bf16(xn[e] * gn[e], hi[e], lo[e]);
-        *reinterpret_cast<uint2*>(p.xg_hi + (long long)t * p.ldo + n) = pack4_bf16(hi);
-        *reinterpret_cast<uint2*>(p.xg_hi + (long long)t * p.ldo + n + p.xg_plane) = pack4_bf16(lo);
-      }
-    } else if (EPI == kTcQkv) {
-      const int d = p.d;
-      if (n < d) {
-        *reinterpret_cast<float4*>(p.out_f32 + (long long)t * p.ldo + n) = make_float4(v[0], v[1], v[2], v[3]);
-      } else {
-        const bf16 b4[4] = {__float2bfloat16_rn(v[0]), __float2bfloat16_rn(v[1]), __float2bfloat16_rn(v[2]), __float2bfloat16_rn(v[3])};
-        bf16* dst = (n < 2 * d) ? p.kcache + s_slot[tr] + (n - d) : p.vcache + s_slot[tr] + (n - 2 * d);
-        *reinterpret_cast<uint2*>(dst) = pack4_bf16(b4);
+  for (int i = 0; i < TB; ++i) {
+    pivot[i] = __shfl_sync(0xffffffffu, xn[i].x, 0);
+    const float d0 = xn[i].x - pivot[i], d1 = xn[i].y - pivot[i], d2 = xn[i].z - pivot[i], d3 = xn[i].w - pivot[i];
+    s1[i] = (d0 + d1) + (d2 + d3);
+    s2[i] = (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+    for (int i = 0; i < TB; ++i) {
+      s1[i] += __shfl_xor_sync(0xffffffffu, s1[i], o);
+      s2[i] += __shfl_xor_sync(0xffffffffu, s2[i], o);
+    }
+  }
+  if (c.g == 0) {
+#pragma unroll
+    for (int i = 0; i < TB; ++i) {
+      const int tr = tb + 4 * i;
+      if (tr < nt) {
+        const float dm = s1[i] * (1.0f / kBM);              // mean - pivot
+        reinterpret_cast<float2*>(p.stat_out)[(size_t)(c.n / kBM) * p.stat_T + t0 + tr] =
+            make_float2(pivot[i] + dm, fmaxf(s2[i] - s1[i] * dm, 0.f));
       }
     }
   }
+}
+
+// The complete tile lies in shared memory (one row per token).  Warp w of the four takes tokens w, w + 4, ...; four
+// tokens are in flight per lane so that the loads of the old residual values overlap.
+template <int EPI>
+__device__ __forceinline__ void tc_finish_tile(const TcParams& p, int z, int t0, int nt, int tile, const float* s_t, int tstride,
+                                               const unsigned long long* s_slot, int et, const float* s_mean,
+                                               const float* s_rstd) {
+  FinishCtx c;
+  if (!tc_finish_setup<EPI>(p, z, tile, et, c)) return;
+  const bool need_old = (EPI == kTcResidual) && p.g_next != nullptr;
+  constexpr int TB = 4;
+  for (int tb = et >> 5; tb < nt; tb += 4 * TB) {
+    float4 old[TB];
+#pragma unroll
+    for (int i = 0; i < TB; ++i) {
+      const int tr = tb + 4 * i;
+      old[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (need_old && tr < nt) old[i] = ld_cg_v4_here(p.out_f32 + (long long)(t0 + tr) * p.ldo + c.n);
+    }
+#pragma unroll
+    for (int i = 0; i < TB; ++i) {
+      const int tr = tb + 4 * i;
+      if (tr < nt) {
+        const float4 a = *reinterpret_cast<const float4*>(s_t + tr * tstride + c.g * 4);
+        tc_finish_item<EPI>(p, c, z, t0 + tr, tr, a, old[i], s_slot, s_mean, s_rstd);
+      }
+    }
+    if (EPI == kTcResidual && p.stat_out) tc_tile_stats<TB>(p, c, t0, tb, nt, old);
+  }
+}
+// The tile is the sum of `splits` partial tiles in the workspace ([split][token][128 features]): the CTA that
+// arrived last adds them in split order and finishes the items straight from registers -- TB tokens x up to four
+// splits of 16-byte loads (and the old residual values) are in flight per lane.
+template <int EPI, int TB>
+__device__ __forceinline__ void tc_merge_finish_tile(const TcParams& p, int z, int t0, int nt, int tile, const float* wsz, int bn,
+                                                     const unsigned long long* s_slot, int et, const float* s_mean,
+                                                     const float* s_rstd) {
+  FinishCtx c;
+  if (!tc_finish_setup<EPI>(p, z, tile, et, c)) return;
+  const bool need_old = (EPI == kTcResidual) && p.g_next != nullptr;
+  constexpr int SB = 16 / TB;                       // 16 partial loads in flight
+  if (et == 0) BPD_TC_STAMP(8);
+  for (int tb = et >> 5; tb < nt; tb += 4 * TB) {
+    float4 old[TB], acc[TB];
+#pragma unroll
+    for (int i = 0; i < TB; ++i) {
+      const int tr = tb + 4 * i;
+      old[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (need_old && tr < nt) old[i] = ld_cg_v4_here(p.out_f32 + (long long)(t0 + tr) * p.ldo + c.n);
+    }
+    for (int s0 = 0; s0 < p.splits; s0 += SB) {
+      float4 v[SB][TB];
+#pragma unroll
+      for (int ss = 0; ss < SB; ++ss)
+#pragma unroll
+        for (int i = 0; i < TB; ++i) {
+          const int tr = tb + 4 * i;
+          v[ss][i] = (s0 + ss < p.splits && tr < nt) ? ld_cg_v4_here(wsz + ((size_t)(s0 + ss) * bn + tr) * kBM + c.g * 4)
+                                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+      for (int ss = 0; ss < SB; ++ss)
+#pragma unroll
+        for (int i = 0; i < TB; ++i) {
+          acc[i].x += v[ss][i].x; acc[i].y += v[ss][i].y; acc[i].z += v[ss][i].z; acc[i].w += v[ss][i].w;
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < TB; ++i) {
+      const int tr = tb + 4 * i;
+      if (tr < nt) tc_finish_item<EPI>(p, c, z, t0 + tr, tr, acc[i], old[i], s_slot, s_mean, s_rstd);
+    }
+    if (EPI == kTcResidual && p.stat_out) tc_tile_stats<TB>(p, c, t0, tb, nt, old);
+  }
+  if (et == 0) BPD_TC_STAMP(12);
 }
 
 // ---------------------------------------------------------------- bounded-wait self test
@@ -401,7 +567,10 @@ struct EpiUnit {
   int tile, split, slice, zidx, ntiles, zcount, t0, nt, bn, nchunks;
   bool skip;
 };
-template <int EPI>
+// WIDE: the launch has token tiles of 32 or more tokens.  Everything that only such tiles use (the way out through
+// shared memory, per-tile statistics, the merge that finishes items from registers) is compiled into that variant
+// alone, so that the few-row launches of the weight-streaming kernels carry none of it.
+template <int EPI, bool WIDE>
 __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& sh, const EpiUnit& u, int warp, int lane) {
   float* s_t = sh.s_t;
   float* s_mean = sh.s_mean;
@@ -419,7 +588,7 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
   // the debug dump of the logits and the rank counting of top-n acceptance are rare: kept out of the common loops
   const bool extras = (EPI == kTcArgmax) && (p.logits != nullptr || p.rank.cnt != nullptr);
   // wide tiles of the other epilogues leave through shared memory too (see tc_finish_tile)
-  const bool vec = (EPI != kTcArgmax) && p.vec && bn >= 32 && !p.ln_x;
+  const bool vec = WIDE && (EPI != kTcArgmax) && p.vec && bn >= 32 && !p.ln_x;   // a folded layer norm on wide tiles comes with stat_in
   constexpr int vstride = kBM + 4;
   if (EPI == kTcQkv && !skip && et < nt) {
     const int t = t0 + et;
@@ -427,6 +596,30 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
     const int pos = p.st.len[b] + i;
     const int page = p.st.page_table[b * p.st.pages_per_row + pos / kPage];
     s_slot[et] = ((unsigned long long)page * kPage + (pos % kPage)) * p.d;
+  }
+  if (WIDE && p.stat_in && !skip && et < nt) {
+    // per-token statistics from the per-tile partial results of the kernel that wrote the stream: merged in
+    // tile order (pairwise update of mean and sum of squared deviations), the same for every consumer
+    const float2* sp = reinterpret_cast<const float2*>(p.stat_in) + (t0 + et);
+    float2 part[8];
+    float mean = 0.f, m2 = 0.f, cnt = 0.f;
+    for (int i0 = 0; i0 < p.stat_parts; i0 += 8) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        if (i0 + i < p.stat_parts) part[i] = __ldcg(sp + (size_t)(i0 + i) * p.stat_T);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        if (i0 + i < p.stat_parts) {
+          const float nb = (float)kBM, tot = cnt + nb;
+          const float delta = part[i].x - mean;
+          mean += delta * (nb / tot);
+          m2 += part[i].y + delta * delta * (cnt * nb / tot);
+          cnt = tot;
+        }
+      }
+    }
+    s_mean[et] = mean;
+    s_rstd[et] = rsqrtf(m2 / cnt + p.ln_eps);
   }
   if (p.ln_x && !skip) {
     // per-token mean and 1/std of the residual stream, computed while the main loop runs: 8 threads per
@@ -461,6 +654,7 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
     if (nchunks > 0 && !skip) done = mbar_wait(u.acc_bar, u.acc_parity);
     if (!done && !skip) atomicCAS(p.error, 0, 103);
     ctl[3] = done ? 1u : 0u;
+    BPD_TC_STAMP(5);
   }
   asm volatile("bar.sync 1, 128;" ::: "memory");
   const bool ok = (ctl[3] != 0);
@@ -510,29 +704,16 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");
       if (et == 0) {
+        BPD_TC_STAMP(6);
         const unsigned prev = atom_add_acq_rel(&p.tile_counters[(size_t)u.zidx * ntiles + tile], 1u);
         ctl[1] = (prev == (unsigned)p.splits - 1) ? 1u : 0u;
+        BPD_TC_STAMP(7);
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");
       if (ctl[1]) {
-        // splits are added in split order; the loads of eight splits x eight tokens are issued together
-        for (int cg = 0; cg < nt; cg += 8) {
-          float acc[8];
-#pragma unroll
-          for (int c = 0; c < 8; ++c) acc[c] = 0.f;
-          for (int s0 = 0; s0 < p.splits; s0 += 8) {
-            float v[8][8];
-#pragma unroll
-            for (int ss = 0; ss < 8; ++ss)
-#pragma unroll
-              for (int c = 0; c < 8; ++c)
-                v[ss][c] = (s0 + ss < p.splits && cg + c < nt)
-                               ? __ldcg(&wsz[((size_t)(s0 + ss) * bn + cg + c) * kBM + row]) : 0.f;
-#pragma unroll
-            for (int ss = 0; ss < 8; ++ss)
-#pragma unroll
-              for (int c = 0; c < 8; ++c) acc[c] += v[ss][c];
-          }
+        // Splits are added in split order.  The partial tiles sit in L2 and every load is a round trip of about a
+        // microsecond, so as many as the registers hold are issued together: G tokens x SB splits = 64 per thread.
+        auto emit8 = [&](const float (&acc)[8], int cg) {
           if (EPI != kTcArgmax && vec) {
 #pragma unroll
             for (int c = 0; c < 8; ++c)
@@ -552,13 +733,48 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
               }
             }
           }
-        }
+        };
+        auto merge = [&](auto g_tag, auto sb_tag) {
+          constexpr int G = decltype(g_tag)::value, SB = decltype(sb_tag)::value;
+          for (int cg = 0; cg < nt; cg += G) {
+            float acc[G];
+#pragma unroll
+            for (int c = 0; c < G; ++c) acc[c] = 0.f;
+            for (int s0 = 0; s0 < p.splits; s0 += SB) {
+              float v[SB][G];
+#pragma unroll
+              for (int ss = 0; ss < SB; ++ss)
+#pragma unroll
+                for (int c = 0; c < G; ++c)
+                  v[ss][c] = (s0 + ss < p.splits && cg + c < nt)
+                                 ? __ldcg(&wsz[((size_t)(s0 + ss) * bn + cg + c) * kBM + row]) : 0.f;
+#pragma unroll
+              for (int ss = 0; ss < SB; ++ss)
+#pragma unroll
+                for (int c = 0; c < G; ++c) acc[c] += v[ss][c];
+            }
+#pragma unroll
+            for (int g8 = 0; g8 < G; g8 += 8) {
+              if (cg + g8 < nt) {
+                const float a8[8] = {acc[g8], acc[g8 + 1], acc[g8 + 2], acc[g8 + 3], acc[g8 + 4], acc[g8 + 5], acc[g8 + 6], acc[g8 + 7]};
+                emit8(a8, cg + g8);
+              }
+            }
+          }
+        };
+        if (WIDE && EPI != kTcArgmax && vec) {
+          tc_merge_finish_tile<EPI, 4>(p, slice, t0, nt, tile, wsz, bn, s_slot, et, s_mean, s_rstd);
+        } else if (!WIDE || nt <= 8) merge(std::integral_constant<int, 8>{}, std::integral_constant<int, 8>{});
+        else if (p.splits <= 2) merge(std::integral_constant<int, 32>{}, std::integral_constant<int, 2>{});
+        else if (p.splits <= 4) merge(std::integral_constant<int, 16>{}, std::integral_constant<int, 4>{});
+        else merge(std::integral_constant<int, 8>{}, std::integral_constant<int, 8>{});
         if (et == 0) p.tile_counters[(size_t)u.zidx * ntiles + tile] = 0;   // ready for the next launch
       }
     }
-    if (EPI != kTcArgmax && vec && (direct || ctl[1])) {
+    if (WIDE && EPI != kTcArgmax && vec && direct) {
       asm volatile("bar.sync 1, 128;" ::: "memory");
-      tc_finish_tile<EPI>(p, slice, t0, nt, tile, s_t, vstride, s_slot, et);
+      if (et == 0) BPD_TC_STAMP(8);
+      tc_finish_tile<EPI>(p, slice, t0, nt, tile, s_t, vstride, s_slot, et, s_mean, s_rstd);
     }
     if (EPI == kTcArgmax && (direct || ctl[1])) {
       // The tile sits in shared memory with one row per token.  tpt threads share a token: each scans every
@@ -622,12 +838,22 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const EpiShared& 
 // ---------------------------------------------------------------- the kernel
 // grid = (feature tiles, K splits, z), z = token tile * zslices + slice (slices: block-diagonal heads).
 // tmA: weights [N, K]; tmBh / tmBl: activation planes [rows, K]; box = (64, 128) and (64, bn).
-template <int EPI>
+template <int EPI, bool WIDE>
 __global__ void __launch_bounds__(kThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmBh,
                const __grid_constant__ CUtensorMap tmBl, TcParams p, int zslices, int a_rows_per_slice,
                int b_cols_per_slice) {
   pdl_launch_dependents();
+  if (threadIdx.x == 0) {
+    BPD_TC_STAMP(0);
+#ifdef BPD_TC_TRACE
+    if (g_tc_trace && blockIdx.x + blockIdx.y + blockIdx.z == 0) {
+      unsigned long long* h = g_tc_trace + ((size_t)p.trace_id * 2048 + 2047) * 16;
+      h[10] = EPI; h[11] = p.N; h[12] = p.K; h[13] = p.T; h[14] = p.splits;
+      h[15] = gridDim.x | (gridDim.y << 12) | ((unsigned long long)gridDim.z << 24) | ((unsigned long long)p.bn << 40);
+    }
+#endif
+  }
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;      // swizzled tiles need 1024-byte alignment
   uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
@@ -638,7 +864,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   volatile uint32_t* ctl = reinterpret_cast<volatile uint32_t*>(gen_base + kStages * stage_sz + 128);
   // ctl[0] = tensor-memory base, ctl[1] = "this CTA reduces the tile", ctl[2] = "this CTA merges the top-1",
   // ctl[3] = "the accumulator arrived"
-  __shared__ float s_mean[16], s_rstd[16];
+  __shared__ float s_mean[WIDE ? kMaxBN : 16], s_rstd[WIDE ? kMaxBN : 16];
   __shared__ unsigned long long s_slot[kMaxBN];   // kTcQkv: cache slot (element offset) of every token of the tile
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -668,6 +894,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   tc_fence_after();
   const uint32_t tmem = ctl[0];
   bool ok = true;
+  if (threadIdx.x == 0) BPD_TC_STAMP(1);
 
   if (warp == 0 && lane == 0) {
     // ---------------- TMA producer.  Weights do not depend on the preceding kernel: the first stages'
@@ -680,6 +907,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       else tma_load_2d(base + it * stage_sz, &tmA, bars + 8 * it, (c0 + it) * kBK, a_row);
     }
     pdl_wait();
+    BPD_TC_STAMP(2);
     const bool skip = p.all_done && *p.all_done;
     for (int it = 0; it < npre; ++it) {
       const uint32_t sa = base + it * stage_sz;
@@ -717,6 +945,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const uint32_t ph = (it / kStages) & 1;
       if (!mbar_wait(bars + 8 * s, ph)) { ok = false; break; }
       tc_fence_after();
+      if (it == 0) BPD_TC_STAMP(3);
       const uint32_t sa = base + s * stage_sz;
 #pragma unroll
       for (int kk = 0; kk < kBK / 16; ++kk) {
@@ -729,6 +958,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       umma_commit(bars + 8 * (kStages + s));       // frees the stage once these MMAs have read it
     }
     if (!skip) umma_commit(bars + 8 * 2 * kStages);            // accumulator complete
+    BPD_TC_STAMP(4);
     if (!ok) atomicCAS(p.error, 0, 102);
   } else if (warp >= 2) {
     // ---------------- epilogue: thread = one feature row, registers = tokens
@@ -737,10 +967,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const EpiShared sh{reinterpret_cast<float*>(gen_base), s_mean, s_rstd, s_slot, ctl};
     const EpiUnit u{tmem, bars + 8 * 2 * kStages, 0u, tile, split, slice, (int)blockIdx.z, (int)gridDim.x,
                     (int)gridDim.z / zslices, t0, nt, bn, nchunks, p.all_done && *p.all_done};
-    tc_epilogue<EPI>(p, sh, u, warp, lane);
+    tc_epilogue<EPI, WIDE>(p, sh, u, warp, lane);
   }
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0) BPD_TC_STAMP(9);
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem, ncols);

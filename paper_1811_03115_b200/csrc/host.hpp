@@ -149,7 +149,8 @@ struct bpd_session {
   int lazy_heads;          // two-stage head evaluation (p_1 everywhere, all heads only at the accepted position)
   int last_pass_lazy;
   void* u2; long long pl_u2; float* h2; int *table2, *table_full;
-  int fold_ln;             // decoder layer norms are folded into the projections (few rows only)
+  int fold_ln;             // decoder layer norms are folded into the projections that follow them
+  float* ln_stats;         // [d / 128][rows][2]: per-tile mean and squared deviations of the residual stream (passes of more than 16 rows)
   int fused;               // decoder layers as three launches each (clusters; at most 16 rows per pass)
   float* fused_ws;
   unsigned* fused_counters;

@@ -26,6 +26,7 @@ struct EmbedParams {
   const int* src;          // [B][rows_per_b] or null (decoder mode)
   const bf16* gain;        // optional: also write planes (hi, lo) of x * gain for a projection with a folded layer norm
   bf16* xg_hi; long long xg_plane;
+  float* stat_out; int stat_T;   // optional: mean and squared deviations of every 128 consecutive features of a row, [d / 128][stat_T][2]
   const int* all_done;
 };
 
@@ -67,6 +68,19 @@ __device__ __forceinline__ void embed_row(const EmbedParams& p, int r) {
     for (int i = 0; i < 8; ++i) v[i] = w[i] * scale + e[i];
     out[0] = make_float4(v[0], v[1], v[2], v[3]);
     out[1] = make_float4(v[4], v[5], v[6], v[7]);
+    if (p.stat_out) {
+      // 16 consecutive lanes hold 128 consecutive features (d is a multiple of 128 here, so half-warps are whole)
+      float sum = ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
+#pragma unroll
+      for (int o = 8; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      const float mean = sum * (1.0f / 128.0f);
+      float sq = 0.f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) sq += (v[i] - mean) * (v[i] - mean);
+#pragma unroll
+      for (int o = 8; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+      if ((threadIdx.x & 15) == 0) reinterpret_cast<float2*>(p.stat_out)[(size_t)(c >> 7) * p.stat_T + r] = make_float2(mean, sq);
+    }
     if (p.gain) {
       float g[8];
       load8(p.gain + c, g);

@@ -209,7 +209,8 @@ template <int EPI>
 int launch(const Operands& op, int N, int K, int T, TcParams p, const Scratch& sc, cudaStream_t st, int zslices = 1,
            int a_rows_per_slice = 0, int b_cols_per_slice = 0, bool pdl = false, int plan_n = 0, int plan_tt = 0) {
   {
-    const int rc0 = ensure_smem_limit(reinterpret_cast<const void*>(gemm_tc_kernel<EPI>), std::max(smem_bytes(kMaxBN), smem_bytes(64)));
+    int rc0 = ensure_smem_limit(reinterpret_cast<const void*>(gemm_tc_kernel<EPI, false>), smem_bytes(16));
+    if (!rc0) rc0 = ensure_smem_limit(reinterpret_cast<const void*>(gemm_tc_kernel<EPI, true>), std::max(smem_bytes(kMaxBN), smem_bytes(64)));
     if (rc0) return rc0;
   }
   // plan_n: the feature count the K split is planned for.  A launch that computes only the first features of a
@@ -234,6 +235,9 @@ int launch(const Operands& op, int N, int K, int T, TcParams p, const Scratch& s
                 (uint32_t)bn, &ml);
   if (rc) return rc;
   p.T = T; p.N = N; p.K = K; p.bn = bn; p.splits = pl.splits; p.chunks_per_split = pl.chunks_per_split;
+#ifdef BPD_TC_TRACE
+  { static int next_trace_id = 0; p.trace_id = next_trace_id++ & 127; }
+#endif
   p.ws = sc.ws; p.tile_counters = sc.tile_counters; p.done_counter = sc.done_counter;
   p.best = sc.best; p.error = sc.error;
   p.stream_weights = (ttiles == 1 && sc.l2_hints) ? 1 : 0;
@@ -244,9 +248,15 @@ int launch(const Operands& op, int N, int K, int T, TcParams p, const Scratch& s
              (p.d % 4 == 0) && al(p.out_f32, 16) && al(p.out_hi, 8) && al(p.xg_hi, 8) && al(p.h, 16) && al(p.bias, 8) &&
              al(p.g_next, 8) && al(p.kcache, 8) && al(p.vcache, 8)) ? 1 : 0;
   }
+  if ((p.stat_in || p.stat_out) && !(p.vec && bn >= 32 && N % kBM == 0 && EPI != kTcArgmax && !p.ln_x))
+    return fail(BPD_E_UNSUPPORTED, "per-tile layer-norm statistics need wide, vectorisable tiles (N = %d, %d tokens per tile)", N, bn);
   dim3 grid(pl.tiles, pl.splits, ttiles * zslices);
-  BPD_CUDA(launch_k(gemm_tc_kernel<EPI>, grid, dim3(kThreads), smem_bytes(bn), st, pdl, ma, mh, ml, p, zslices,
-                    a_rows_per_slice, b_cols_per_slice));
+  if (bn >= 32)
+    BPD_CUDA(launch_k(gemm_tc_kernel<EPI, true>, grid, dim3(kThreads), smem_bytes(bn), st, pdl, ma, mh, ml, p, zslices,
+                      a_rows_per_slice, b_cols_per_slice));
+  else
+    BPD_CUDA(launch_k(gemm_tc_kernel<EPI, false>, grid, dim3(kThreads), smem_bytes(bn), st, pdl, ma, mh, ml, p, zslices,
+                      a_rows_per_slice, b_cols_per_slice));
   return BPD_OK;
 }
 
