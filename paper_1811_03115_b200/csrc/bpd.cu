@@ -583,12 +583,18 @@ static int run_layers_fused(bpd_session* s, const PassArgs& a) {
   const size_t smem_ffn = fused::ffn_layout(d, nt).total;
   // the opt-in shared-memory limit of each kernel grows with the widest model seen so far
   {
+    BPD_TRY(fused_attr(fused::attn_block_kernel<true, 1, 1>, smem_self));
+    BPD_TRY(fused_attr(fused::attn_block_kernel<true, 2, 1>, smem_self));
+    BPD_TRY(fused_attr(fused::attn_block_kernel<true, 1, 2>, smem_self));
+    BPD_TRY(fused_attr(fused::attn_block_kernel<true, 2, 2>, smem_self));
+    BPD_TRY(fused_attr(fused::attn_block_kernel<true, 1, 2, 1>, smem_self));
+    BPD_TRY(fused_attr(fused::attn_block_kernel<true, 2, 2, 1>, smem_self));
+    BPD_TRY(fused_attr(fused::attn_block_kernel<false, 1, 1>, smem_cross));
+    BPD_TRY(fused_attr(fused::attn_block_kernel<false, 2, 1>, smem_cross));
     if (nt == 1) {
-      BPD_TRY(fused_attr(fused::attn_block_kernel<true, 1>, smem_self));
       BPD_TRY(fused_attr(fused::attn_block_kernel<false, 1>, smem_cross));
       BPD_TRY(fused_attr(fused::ffn_block_kernel<1>, smem_ffn));
     } else {
-      BPD_TRY(fused_attr(fused::attn_block_kernel<true, 2>, smem_self));
       BPD_TRY(fused_attr(fused::attn_block_kernel<false, 2>, smem_cross));
       BPD_TRY(fused_attr(fused::ffn_block_kernel<2>, smem_ffn));
     }
@@ -627,12 +633,23 @@ static int run_layers_fused(bpd_session* s, const PassArgs& a) {
     pf.w1 = static_cast<const bf16*>(L.w1); pf.w2 = static_cast<const bf16*>(L.w2); pf.b2 = static_cast<const bf16*>(L.b2);
     pf.d = d; pf.ff = c.d_ff; pf.R = R; pf.NJ = (int)grid_ffn.y; pf.eps = c.eps;
     pf.ws = s->fused_ws; pf.counters = s->fused_counters; pf.all_done = done;
+    // every position the cache can hold (max_tgt + k + 1 of them) within kC chunks of 32: the short schedule only
+    const bool short_only = s->max_tgt + c.k_model + 1 <= fused::kC * 32;
+    const bool roomy = c.H * fused::kC <= 74;      // an attention launch leaves half the SMs free
     if (nt == 1) {
-      BPD_CUDA(launch_k(fused::attn_block_kernel<true, 1>, grid_attn, block, smem_self, st, pdl, ps));
+      if (short_only) BPD_CUDA(launch_k(fused::attn_block_kernel<true, 1, 1>, grid_attn, block, smem_self, st, pdl, ps));
+      else if (roomy) BPD_CUDA(launch_k(fused::attn_block_kernel<true, 1, 2, 1>, grid_attn, block, smem_self, st, pdl, ps));
+      else BPD_CUDA(launch_k(fused::attn_block_kernel<true, 1, 2>, grid_attn, block, smem_self, st, pdl, ps));
+      if (cross_smax > 0) BPD_CUDA(launch_k(fused::attn_block_kernel<false, 1, 1>, grid_attn, block, smem_cross, st, pdl, pc));
+      else
       BPD_CUDA(launch_k(fused::attn_block_kernel<false, 1>, grid_attn, block, smem_cross, st, pdl, pc));
       BPD_CUDA(launch_k(fused::ffn_block_kernel<1>, grid_ffn, block, smem_ffn, st, pdl, pf));
     } else {
-      BPD_CUDA(launch_k(fused::attn_block_kernel<true, 2>, grid_attn, block, smem_self, st, pdl, ps));
+      if (short_only) BPD_CUDA(launch_k(fused::attn_block_kernel<true, 2, 1>, grid_attn, block, smem_self, st, pdl, ps));
+      else if (roomy) BPD_CUDA(launch_k(fused::attn_block_kernel<true, 2, 2, 1>, grid_attn, block, smem_self, st, pdl, ps));
+      else BPD_CUDA(launch_k(fused::attn_block_kernel<true, 2, 2>, grid_attn, block, smem_self, st, pdl, ps));
+      if (cross_smax > 0) BPD_CUDA(launch_k(fused::attn_block_kernel<false, 2, 1>, grid_attn, block, smem_cross, st, pdl, pc));
+      else
       BPD_CUDA(launch_k(fused::attn_block_kernel<false, 2>, grid_attn, block, smem_cross, st, pdl, pc));
       BPD_CUDA(launch_k(fused::ffn_block_kernel<2>, grid_ffn, block, smem_ffn, st, pdl, pf));
     }

@@ -449,8 +449,17 @@ __host__ __device__ inline AttnLayout attn_layout(int d, int NT, int pt_ints, in
   return L;
 }
 
-template <bool SELF, int NT>
-__global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_block_kernel(AttnBlockParams p) {
+// LEAN variants carry only the path their session takes -- the general kernels run out of registers under the
+// 128-per-thread budget that keeps two CTAs on an SM (ptxas: 184 bytes of spills in the self-attention block) and
+// are 1.5-2 us per launch slower.  Self-attention: the cache never holds more than kC chunks of keys per row, so
+// only the short schedule is compiled in (sessions of up to 256 positions: the machine-translation shapes).
+// Cross-attention: the encoder's rows are staged in shared memory (cross_smax > 0).
+// Self-attention, LEAN = 2: only the long schedule (rank c folds its own chunks for all rows), which is correct at
+// any length and the same arithmetic; sessions whose cache can exceed 256 positions use it from the start.
+// MINB = 1 lifts the register budget to 255 per thread for models whose attention launches occupy at most half the
+// SMs (the next launch's CTAs find free SMs anyway): the long schedule then keeps its chunk in registers.
+template <bool SELF, int NT, int LEAN = 0, int MINB = 2>
+__global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, MINB) attn_block_kernel(AttnBlockParams p) {
   extern __shared__ __align__(16) uint8_t fsm[];
   cg::cluster_group cluster = cg::this_cluster();
   const int c = (int)cluster.block_rank(), h = blockIdx.y;
@@ -495,7 +504,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
       const int row = idx >> 3, c16 = idx & 7;
       cp_async16(w_out_s + sw(row, c16 * 16, L.s_out), p.w_out + (size_t)(c * slice + row) * d + h * kDH + c16 * 8, stream);
     }
-    if (!SELF && p.cross_smax > 0) {
+    if (!SELF && (LEAN != 0 || p.cross_smax > 0)) {
       // the encoder's keys and values of this head do not change after the encoder ran: they come along
       const float* Kg = reinterpret_cast<const float*>(p.attn.k);
       const float* Vg = reinterpret_cast<const float*>(p.attn.v);
@@ -561,7 +570,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
 
   // self-attention: does every rank have at most one chunk of keys?  (the same answer in every CTA of the grid)
   bool one_chunk_per_rank = true;
-  if (SELF) {
+  if (SELF && LEAN == 0) {
     for (int b = 0; b < nb; ++b)
       one_chunk_per_rank = one_chunk_per_rank &&
           ((s_len[b] + p.rows_per_b + 31) >> 5) - (attn_first_key(p.attn, s_len[b]) >> 5) <= kC;
@@ -577,7 +586,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
       const float y = s_rstd[token] * (a - s_mean[token] * fs) + fc;
       if (sect == 0) {
         if (SELF) {
-          if (one_chunk_per_rank) {
+          if (LEAN == 1 || (LEAN == 0 && one_chunk_per_rank)) {
             q_all[token * kDH + f] = y * p.attn.scale;             // this rank attends for its own rows
           } else {
 #pragma unroll
@@ -610,7 +619,7 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
     const bf16* Kc = reinterpret_cast<const bf16*>(ap.k);
     const bf16* Vc = reinterpret_cast<const bf16*>(ap.v);
     const int rpb = p.rows_per_b;
-    if (one_chunk_per_rank) {
+    if (LEAN == 1 || (LEAN == 0 && one_chunk_per_rank)) {
       // Short sequences: this rank takes its own rows (as the projection handed them out), warp w stands in for
       // rank w and folds that rank's only chunk; a rank's single lump is its state (merging one lump multiplies
       // by exp(0) = 1), so the eight warp states are merged like the ranks' states.  The result goes to every
@@ -716,8 +725,9 @@ __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 2) attn_b
       if (tid < kDH) sm.q[tid] = q_s[slot * kDH + tid];
       __syncthreads();
       const int b = token / p.rows_per_b;
-      const float ov = p.cross_smax > 0 ? cross_attention_staged(ckv_s + (size_t)b * p.cross_smax * kCrossRowBytes, s_len[b], sm)
-                                        : attention_head<float, kDH, kWarps, false>(ap, b, h, 0, s_len[b], sm);
+      float ov;
+      if (LEAN != 0 || p.cross_smax > 0) ov = cross_attention_staged(ckv_s + (size_t)b * p.cross_smax * kCrossRowBytes, s_len[b], sm);
+      else ov = attention_head<float, kDH, kWarps, false>(ap, b, h, 0, s_len[b], sm);
       if (tid < kDH) {
         uint32_t hi, lo;
         split_bits(ov, hi, lo);
