@@ -594,9 +594,11 @@ static int run_layers_fused(bpd_session* s, const PassArgs& a) {
     if (nt == 1) {
       BPD_TRY(fused_attr(fused::attn_block_kernel<false, 1>, smem_cross));
       BPD_TRY(fused_attr(fused::ffn_block_kernel<1>, smem_ffn));
+      BPD_TRY(fused_attr(fused::ffn_block_kernel<1, 2>, smem_ffn));
     } else {
       BPD_TRY(fused_attr(fused::attn_block_kernel<false, 2>, smem_cross));
       BPD_TRY(fused_attr(fused::ffn_block_kernel<2>, smem_ffn));
+      BPD_TRY(fused_attr(fused::ffn_block_kernel<2, 2>, smem_ffn));
     }
   }
   EmbedParams ep;
@@ -636,6 +638,7 @@ static int run_layers_fused(bpd_session* s, const PassArgs& a) {
     // every position the cache can hold (max_tgt + k + 1 of them) within kC chunks of 32: the short schedule only
     const bool short_only = s->max_tgt + c.k_model + 1 <= fused::kC * 32;
     const bool roomy = c.H * fused::kC <= 74;      // an attention launch leaves half the SMs free
+    const bool ffn_small = grid_ffn.x * grid_ffn.y <= 148;   // one CTA per SM is enough for the feed-forward launch
     if (nt == 1) {
       if (short_only) BPD_CUDA(launch_k(fused::attn_block_kernel<true, 1, 1>, grid_attn, block, smem_self, st, pdl, ps));
       else if (roomy) BPD_CUDA(launch_k(fused::attn_block_kernel<true, 1, 2, 1>, grid_attn, block, smem_self, st, pdl, ps));
@@ -643,7 +646,8 @@ static int run_layers_fused(bpd_session* s, const PassArgs& a) {
       if (cross_smax > 0) BPD_CUDA(launch_k(fused::attn_block_kernel<false, 1, 1>, grid_attn, block, smem_cross, st, pdl, pc));
       else
       BPD_CUDA(launch_k(fused::attn_block_kernel<false, 1>, grid_attn, block, smem_cross, st, pdl, pc));
-      BPD_CUDA(launch_k(fused::ffn_block_kernel<1>, grid_ffn, block, smem_ffn, st, pdl, pf));
+      if (ffn_small) BPD_CUDA(launch_k(fused::ffn_block_kernel<1, 2>, grid_ffn, block, smem_ffn, st, pdl, pf));
+      else BPD_CUDA(launch_k(fused::ffn_block_kernel<1>, grid_ffn, block, smem_ffn, st, pdl, pf));
     } else {
       if (short_only) BPD_CUDA(launch_k(fused::attn_block_kernel<true, 2, 1>, grid_attn, block, smem_self, st, pdl, ps));
       else if (roomy) BPD_CUDA(launch_k(fused::attn_block_kernel<true, 2, 2, 1>, grid_attn, block, smem_self, st, pdl, ps));
@@ -651,7 +655,8 @@ static int run_layers_fused(bpd_session* s, const PassArgs& a) {
       if (cross_smax > 0) BPD_CUDA(launch_k(fused::attn_block_kernel<false, 2, 1>, grid_attn, block, smem_cross, st, pdl, pc));
       else
       BPD_CUDA(launch_k(fused::attn_block_kernel<false, 2>, grid_attn, block, smem_cross, st, pdl, pc));
-      BPD_CUDA(launch_k(fused::ffn_block_kernel<2>, grid_ffn, block, smem_ffn, st, pdl, pf));
+      if (ffn_small) BPD_CUDA(launch_k(fused::ffn_block_kernel<2, 2>, grid_ffn, block, smem_ffn, st, pdl, pf));
+      else BPD_CUDA(launch_k(fused::ffn_block_kernel<2>, grid_ffn, block, smem_ffn, st, pdl, pf));
     }
     g_launches += 3;
     if (a.layer_dump)
@@ -711,9 +716,22 @@ static bool stack_plan(const Config& c, int rows, int nb, int ppr, int cross_row
   return true;
 }
 
-template <int NT, int KS, int MINB>
-static int stack_clusters(size_t smem, int H, int* out) {
-  BPD_TRY(ensure_smem_limit(reinterpret_cast<const void*>(stack::layer_stack_kernel<NT, KS, MINB>), smem));
+// The persistent kernel's instantiations: token tiles (1 or 2 of 8 rows), reduction steps per panel (2: d_model 256,
+// else 4), CTAs per SM (1 or 2), lean (short sequences and staged encoder rows only).  `f` gets the kernel.
+template <typename F>
+static int stack_variant(int nt, int ksteps, int minb, bool lean, F&& f) {
+#define BPD_V(NT, KS, MB, LN) if (nt == NT && ksteps == KS && minb == MB && lean == LN) return f(stack::layer_stack_kernel<NT, KS, MB, LN>)
+  BPD_V(1, 2, 1, false); BPD_V(2, 2, 1, false); BPD_V(1, 4, 1, false); BPD_V(2, 4, 1, false);
+  BPD_V(1, 2, 2, false); BPD_V(2, 2, 2, false); BPD_V(1, 4, 2, false); BPD_V(2, 4, 2, false);
+  BPD_V(1, 2, 1, true); BPD_V(2, 2, 1, true); BPD_V(1, 4, 1, true); BPD_V(2, 4, 1, true);
+  BPD_V(1, 2, 2, true); BPD_V(2, 2, 2, true); BPD_V(1, 4, 2, true); BPD_V(2, 4, 2, true);
+#undef BPD_V
+  return fail(BPD_E_UNSUPPORTED, "no persistent layer kernel for %d token tiles, %d steps, %d CTAs per SM", nt, ksteps, minb);
+}
+
+template <typename K>
+static int stack_clusters(K kernel, size_t smem, int H, int* out) {
+  BPD_TRY(ensure_smem_limit(reinterpret_cast<const void*>(kernel), smem));
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
   cfg.gridDim = dim3(fused::kC, H); cfg.blockDim = dim3(stack::kThreads); cfg.dynamicSmemBytes = smem;
@@ -721,7 +739,7 @@ static int stack_clusters(size_t smem, int H, int* out) {
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = fused::kC; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
   cfg.attrs = at; cfg.numAttrs = 1;
-  BPD_CUDA(cudaOccupancyMaxActiveClusters(out, stack::layer_stack_kernel<NT, KS, MINB>, &cfg));
+  BPD_CUDA(cudaOccupancyMaxActiveClusters(out, kernel, &cfg));
   return BPD_OK;
 }
 
@@ -763,10 +781,10 @@ static int stack_setup(bpd_session* s) {
       lay.total += 1024;                       // slack for aligning the ring to 1024 bytes
       int n1 = 0, n2 = 0;
       const size_t sm = (size_t)lay.total;
-      if (c.d == 256 && minb == 1) { BPD_TRY((stack_clusters<1, 2, 1>(sm, c.H, &n1))); BPD_TRY((stack_clusters<2, 2, 1>(sm, c.H, &n2))); }
-      else if (c.d == 256) { BPD_TRY((stack_clusters<1, 2, 2>(sm, c.H, &n1))); BPD_TRY((stack_clusters<2, 2, 2>(sm, c.H, &n2))); }
-      else if (minb == 1) { BPD_TRY((stack_clusters<1, 4, 1>(sm, c.H, &n1))); BPD_TRY((stack_clusters<2, 4, 1>(sm, c.H, &n2))); }
-      else { BPD_TRY((stack_clusters<1, 4, 2>(sm, c.H, &n1))); BPD_TRY((stack_clusters<2, 4, 2>(sm, c.H, &n2))); }
+      const bool lean = !long_seq && cross_rows > 0;
+      const int ksteps = c.d == 256 ? 2 : 4, H = c.H;
+      BPD_TRY(stack_variant(1, ksteps, minb, lean, [&](auto kernel) { return stack_clusters(kernel, sm, H, &n1); }));
+      BPD_TRY(stack_variant(2, ksteps, minb, lean, [&](auto kernel) { return stack_clusters(kernel, sm, H, &n2); }));
       ok = n1 >= c.H && n2 >= c.H;
     }
     if (ok) break;
@@ -849,16 +867,13 @@ static int run_layers_stack(bpd_session* s, const PassArgs& a) {
   memcpy(&maps, s->stack_maps, sizeof(maps));
   const size_t smem = (size_t)p.lay.total;
   // reduction panels of 32 columns (two steps of 16) for d_model 256, else 64 (four steps); one or two CTAs per SM
-#define BPD_STACK_LAUNCH(NT, KS, MB) BPD_CUDA(launch_k(stack::layer_stack_kernel<NT, KS, MB>, grid, block, smem, s->stream, pdl, maps, p))
   const int nt = p.R > 8 ? 2 : 1, ksteps = c.d == 256 ? 2 : 4;
-  if (s->stack_minb == 1) {
-    if (ksteps == 2) { if (nt == 2) BPD_STACK_LAUNCH(2, 2, 1); else BPD_STACK_LAUNCH(1, 2, 1); }
-    else { if (nt == 2) BPD_STACK_LAUNCH(2, 4, 1); else BPD_STACK_LAUNCH(1, 4, 1); }
-  } else {
-    if (ksteps == 2) { if (nt == 2) BPD_STACK_LAUNCH(2, 2, 2); else BPD_STACK_LAUNCH(1, 2, 2); }
-    else { if (nt == 2) BPD_STACK_LAUNCH(2, 4, 2); else BPD_STACK_LAUNCH(1, 4, 2); }
-  }
-#undef BPD_STACK_LAUNCH
+  const bool lean = !s->stack_long && s->stack_cross_rows > 0;
+  cudaStream_t stream = s->stream;
+  BPD_TRY(stack_variant(nt, ksteps, s->stack_minb, lean, [&](auto kernel) {
+    BPD_CUDA(launch_k(kernel, grid, block, smem, stream, pdl, maps, p));
+    return (int)BPD_OK;
+  }));
   ++g_launches;
   return BPD_OK;
 }

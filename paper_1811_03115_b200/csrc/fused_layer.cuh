@@ -811,8 +811,10 @@ __host__ __device__ inline FfnLayout ffn_layout(int d, int NT) {
   return L;
 }
 
-template <int NT>
-__global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, 3) ffn_block_kernel(FfnBlockParams p) {
+// MINB = 3 (80 registers) lets all 32 clusters of a wide feed-forward layer be resident at once; launches of at
+// most 148 CTAs take MINB = 2 (128 registers).
+template <int NT, int MINB = 3>
+__global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, MINB) ffn_block_kernel(FfnBlockParams p) {
   extern __shared__ __align__(16) uint8_t fsm[];
   cg::cluster_group cluster = cg::this_cluster();
   const int c = (int)cluster.block_rank(), j = blockIdx.y;

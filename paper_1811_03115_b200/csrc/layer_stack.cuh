@@ -615,7 +615,10 @@ constexpr int kTracePts = 256;
 // grid = (8, H), clusters of 8 along x.  All clusters must be resident at once (the host checks the occupancy).
 // MINB: CTAs per SM the kernel is compiled for.  Models with at most 15 heads have an SM to themselves per CTA (no
 // register limit to speak of); 16 clusters only fit with two CTAs on some SMs, which caps the registers at 128.
-template <int NT, int KS, int MINB>
+// LEAN: sessions whose cache holds at most 256 positions and whose encoder rows are staged by TMA carry only that
+// path (the short self-attention schedule, the staged cross-attention); the general kernel needs far more than the
+// 128 registers a thread has when two CTAs share an SM.
+template <int NT, int KS, int MINB, bool LEAN>
 __global__ void __cluster_dims__(kC, 1, 1) __launch_bounds__(kThreads, MINB)
 layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant__ StackParams p) {
   extern __shared__ __align__(1024) uint8_t ssm_raw[];
@@ -738,8 +741,10 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
   ap.rows = R; ap.rows_per_b = rpb; ap.H = p.H; ap.dh = kDH; ap.causal = 1; ap.local_q = p.local_q; ap.local_m = p.local_m;
   ap.ldkv = d; ap.paged = 1; ap.st = p.st; ap.st.page_table = s_pt; ap.scale = p.scale;
   bool one_chunk_per_rank = true;
-  for (int b = 0; b < nb; ++b)
-    one_chunk_per_rank = one_chunk_per_rank && ((s_len[b] + rpb + 31) >> 5) - (attn_first_key(ap, s_len[b]) >> 5) <= kC;
+  if (!LEAN) {
+    for (int b = 0; b < nb; ++b)
+      one_chunk_per_rank = one_chunk_per_rank && ((s_len[b] + rpb + 31) >> 5) - (attn_first_key(ap, s_len[b]) >> 5) <= kC;
+  }
 
   unsigned nbar = 0;                        // joins passed so far in this launch
   int seq = 0;                              // next tile to consume
@@ -847,7 +852,7 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
       ap.k = LP.kcache; ap.v = LP.vcache;
       const bf16* Kc = LP.kcache;
       const bf16* Vc = LP.vcache;
-      if (one_chunk_per_rank) {
+      if (LEAN || one_chunk_per_rank) {
         // this rank attends for its own rows; warp w folds the chunk that belongs to rank w
         for (int slot = 0; slot < NT; ++slot) {
           const int token = slot * kC + c;
@@ -1013,8 +1018,9 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
           }
           __syncthreads();
           const int b = token / rpb;
-          const float ov = g.staged ? cross_attention_tile(ckv_g, ckv_g + kb, ckv_g + 2 * kb, b * p.max_src, s_src[b], sm)
-                                    : attention_head<float, kDH, kWarps, false>(ap, b, j, 0, s_src[b], sm);
+          float ov;
+          if (LEAN || g.staged) ov = cross_attention_tile(ckv_g, ckv_g + kb, ckv_g + 2 * kb, b * p.max_src, s_src[b], sm);
+          else ov = attention_head<float, kDH, kWarps, false>(ap, b, j, 0, s_src[b], sm);
           if (tid < kDH) store_attn_out(oh, ol, token, tid, ov);
           __syncthreads();
         }
