@@ -124,6 +124,11 @@ int bpd_query_sizes(const void* blob, size_t blob_bytes, int batch, int max_src,
 /* session_bytes for an already loaded model (same value bpd_query_sizes gives). */
 int bpd_session_bytes(const bpd_model* model, int batch, int max_src, int max_tgt, size_t* session_bytes);
 
+/* Which form the session's decoder layers take: 0 = one kernel per projection, 1 = three cluster launches per
+ * layer, 2 = one persistent kernel per pass.  The options of bpd_session_create_opt are requests: a shape or a
+ * device that a form does not take falls back to the next one, and this call tells.  Negative on a null handle. */
+int bpd_session_layer_path(const bpd_session* s);
+
 /* Copy the blob's tensors into dev_weight_buf (device, 256-byte aligned,
  * >= weight_bytes) and return a model handle.  The blob may be freed after the
  * call returns (the call synchronises the stream). */

@@ -57,6 +57,7 @@ _SIGS = {
     "bpd_last_error": (C.c_char_p, []),
     "bpd_query_sizes": (_i, [_vp, _sz, _i, _i, _i, C.POINTER(_sz), C.POINTER(_sz)]),
     "bpd_session_bytes": (_i, [_vp, _i, _i, _i, C.POINTER(_sz)]),
+    "bpd_session_layer_path": (_i, [_vp]),
     "bpd_load_weights": (_i, [_vp, _sz, _vp, _sz, _vp, C.POINTER(_vp)]),
     "bpd_session_create": (_i, [_vp, _i, _i, _i, _vp, _sz, _vp, C.POINTER(_vp)]),
     "bpd_session_options_init": (None, [C.POINTER(bpd_session_options)]),
@@ -282,6 +283,11 @@ class Session:
         if layers is not None:
             res["layers"] = layers
         return res
+
+    @property
+    def layer_path(self) -> int:
+        """0: one kernel per projection, 1: three cluster launches per layer, 2: one persistent kernel per pass."""
+        return int(lib.bpd_session_layer_path(self.handle))
 
     @property
     def n_dec(self) -> int:

@@ -226,7 +226,7 @@ static size_t plan_session(const Config& c, int B, int max_src, int max_tgt, cha
   unsigned* fused_counters = a.take<unsigned>(fused::kC);
   // persistent layer stack: tensor maps, per-layer pointers, the clusters' partial outputs, the join's words
   void* stack_layers = a.take_bytes(fused_ok ? (size_t)c.n_dec * sizeof(stack::LayerPtrs) : 0);
-  float* stack_ws = a.take<float>(fused_ok ? (size_t)2 * c.H * fused::kMaxRows * d : 0);
+  unsigned long long* stack_ws = a.take<unsigned long long>(fused_ok ? (size_t)2 * (c.H + 1) * fused::kMaxRows * d : 0);
   unsigned* stack_bar = a.take<unsigned>(stack::kBarWords);
   float* ln_stats = a.take<float>((size_t)ceil_div(d, 128) * Rall * 2);
   if (s) {
@@ -682,7 +682,8 @@ static bool stack_plan(const Config& c, int rows, int nb, int ppr, int cross_row
   L.xl = take((size_t)RP * g.ks * 2);
   L.oh = take((size_t)RP * 128);
   L.ol = take((size_t)RP * 128);
-  L.hid = take((size_t)fused::kC * 2 * RP * g.UPR * 2);
+  // hidden-unit planes; the same bytes are the scratch of the two-hop reduction (2 * rows * H float4)
+  L.hid = take(std::max((size_t)fused::kC * 2 * RP * g.UPR * 2, c.H >= 16 ? (size_t)2 * rows * c.H * 16 : (size_t)0));
   const size_t chunk = std::max((size_t)NT * 3 * fused::kDH * 4, (size_t)g.UPR * RP * 4);
   L.outbox = take(fused::kC * chunk);
   L.inbox = take(fused::kC * chunk);
@@ -858,7 +859,7 @@ static int run_layers_stack(bpd_session* s, const PassArgs& a) {
   p.lnf_g = static_cast<const bf16*>(m->dec_lnf_g); p.lnf_b = static_cast<const bf16*>(m->dec_lnf_b);
   p.xn_hi = static_cast<bf16*>(s->xn); p.xn_plane = s->pl_xn; p.h_f32 = s->h_f32;
   p.layer_dump = a.layer_dump;
-  p.ws = s->stack_ws; p.bar = s->stack_bar; p.error = s->st.error; p.all_done = s->st.all_done;
+  p.ws = s->stack_ws; p.gather = s->stack_ws + (size_t)2 * c.H * fused::kMaxRows * c.d; p.bar = s->stack_bar; p.error = s->st.error; p.all_done = s->st.all_done;
   p.spin = stack::kSpin;
   memcpy(&p.lay, s->stack_layout, sizeof(p.lay));
   const dim3 grid(fused::kC, c.H), block(stack::kThreads);
@@ -1149,6 +1150,11 @@ int bpd_query_sizes(const void* blob, size_t blob_bytes, int batch, int max_src,
   if (weight_bytes) *weight_bytes = weight_bytes_for(pb);
   if (session_bytes) *session_bytes = plan_session(pb.cfg, batch, max_src, max_tgt, nullptr, nullptr);
   return BPD_OK;
+}
+
+int bpd_session_layer_path(const bpd_session* s) {
+  if (!s) return fail(BPD_E_INVALID, "session is null");
+  return s->stack ? 2 : (s->fused ? 1 : 0);
 }
 
 int bpd_session_bytes(const bpd_model* model, int batch, int max_src, int max_tgt, size_t* session_bytes) {

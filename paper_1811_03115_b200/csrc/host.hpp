@@ -160,7 +160,7 @@ struct bpd_session {
   int stack;
   unsigned char stack_maps[8 * 128] __attribute__((aligned(64)));   // stack::StackMaps (eight tensor maps over all layers)
   void* stack_layers;      // device: stack::LayerPtrs [n_dec]
-  float* stack_ws;         // device: [2][H][16][d] partial outputs of the clusters
+  unsigned long long* stack_ws;   // device: [2][H][16][d] words (value, tag): the clusters' shares of the projection outputs
   unsigned* stack_bar;     // device: words of the device-wide join
   float* stack_dump;       // device: [n_dec][rows][d] residual stream after every layer (debug dump), or null
   int stack_cross_rows, stack_long, stack_minb;

@@ -1318,7 +1318,7 @@ struct ResetParams {
   RowState st;
   int B, ppr;
   const int* src_len;
-  unsigned* join_words;   // words of the persistent layer kernel's device-wide join (64), or null
+  unsigned* join_words;   // control words of the persistent layer kernel (64), or null
 };
 static __global__ void reset_rows_kernel(ResetParams p) {
   const int b = threadIdx.x;
@@ -1335,8 +1335,11 @@ static __global__ void reset_rows_kernel(ResetParams p) {
     *p.st.error = 0;
     for (int i = 0; i < 4 + kMaxK + 1; ++i) p.st.stats[i] = 0;
   }
+  // the abort word is cleared; word 32 numbers the kernel's reductions over the whole life of the session (its
+  // workspace keeps the tags of earlier decodes) and stays
   if (p.join_words)
-    for (int i = threadIdx.x; i < 64; i += blockDim.x) p.join_words[i] = 0u;
+    for (int i = threadIdx.x; i < 64; i += blockDim.x)
+      if (i != 32) p.join_words[i] = 0u;
 }
 
 }  // namespace bpd

@@ -63,9 +63,8 @@ constexpr int kState = 68;                 // floats per partial attention state
                                            // padding to a multiple of 16 bytes
 constexpr unsigned long long kSpin = 2000000000ull;   // about a second
 // words of the device-wide join
-constexpr int kBarCount = 0;               // arrivals, never reset while the session decodes
 constexpr int kBarAbort = 1;               // non-zero: some wait expired, nobody waits any more
-constexpr int kBarBase = 32;               // arrivals at the start of the next launch
+constexpr int kBarBase = 32;               // reductions done so far in this session: the next launch's tags go on from here (never reset)
 constexpr int kBarWords = 64;
 
 // Tensor maps over all decoder layers at once (the layers' tensors lie at a constant stride): dimensions
@@ -104,7 +103,8 @@ struct StackParams {
   bf16* xn_hi; long long xn_plane; float* h_f32;
   float* layer_dump;                       // optional [L][R][d]: the residual stream after every layer
   // exchange between clusters
-  float* ws;                               // [2][H][kMaxRows][d]
+  unsigned long long* ws;                  // [2][H][kMaxRows][d] words of (value bits, tag): the clusters' shares of a projection output
+  unsigned long long* gather;              // [2][kMaxRows][d] words of (value bits, tag): the summed shares, models with 16 or more heads
   unsigned* bar;                           // [kBarWords]
   int* error;
   const int* all_done;
@@ -113,14 +113,6 @@ struct StackParams {
 };
 
 // ------------------------------------------------------------------ small PTX helpers
-__device__ __forceinline__ unsigned long long ld_acquire_u64(const void* p) {
-  unsigned long long v;
-  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ void red_release_add(unsigned* p, unsigned v) {
-  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
@@ -341,27 +333,14 @@ __device__ __forceinline__ void xchg_wait(const Cta& k, int n) {
   }
 }
 
-// All threads: the device-wide join.  Arrive (our workspace writes are released), release `nfree` consumed tiles,
-// wait until `target` arrivals have been counted.
-__device__ __forceinline__ void grid_join(const Cta& k, unsigned target, int nfree) {
-  __syncthreads();
-  if (k.tid == kPumpThread && nfree) release_tiles(k, nfree);
-  if (k.tid == 0) {
-    red_release_add(k.p->bar + kBarCount, 1u);
-    if (!is_zombie(k)) {
-      const unsigned long long t0 = clock64();
-      for (unsigned spins = 0;; ++spins) {
-        const unsigned long long v = ld_acquire_u64(k.p->bar + kBarCount);
-        if ((int)((unsigned)v - target) >= 0) break;
-        if ((unsigned)(v >> 32) != 0u) { *reinterpret_cast<volatile int*>(&k.ctl->zombie) = 1; break; }
-        if ((spins & 63u) == 63u && (unsigned long long)(clock64() - t0) > k.p->spin) { raise_abort(k, 104); break; }
-      }
-#ifdef BPD_STACK_TRACE
-      k.ctl->cyc_poll += clock64() - t0;
-#endif
-    }
-  }
-  __syncthreads();
+// A cluster's share of a projection output travels to the other clusters as 64-bit words (value bits, tag): the tag
+// is the number of the reduction in this session (never reused), and an aligned 64-bit store is indivisible, so a
+// reader that sees the tag has the value -- no fence, no counter, one trip through L2 instead of three.
+__device__ __forceinline__ void ll_store(unsigned long long* at, float v, unsigned tag) {
+  asm volatile("st.volatile.global.u64 [%0], %1;" ::"l"(at), "l"(((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(v)) : "memory");
+}
+__device__ __forceinline__ void ll_load2(const unsigned long long* at, unsigned long long& a, unsigned long long& b) {
+  asm volatile("ld.volatile.global.v2.u64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "l"(at) : "memory");
 }
 
 // ------------------------------------------------------------------ x slice: reduce, planes, statistics
@@ -380,30 +359,121 @@ __device__ __forceinline__ Words load_words(const Cta& k, const bf16* v) {
 // After a join: x[t][col] += bias[col] + sum over the H clusters' partial outputs, in cluster order, for this
 // rank's columns.  Item = (row, four columns); rows are aligned to groups of lanes.  The loads of up to 16
 // partials are all in flight before the first is added.
-__device__ __forceinline__ void reduce_slice(const Cta& k, float* x_s, const float* ws, const Words& bias) {
+__device__ __forceinline__ void reduce_slice(const Cta& k, float* x_s, const unsigned long long* ws, const Words& bias,
+                                             unsigned tag, int nfree) {
   const StackParams& p = *k.p;
   const int ks = k.g.ks, n4 = ks >> 2, R = p.R, d = p.d, H = p.H;
+  __syncthreads();                                             // every warp is done with the tiles released here
+  if (k.tid == kPumpThread && nfree) release_tiles(k, nfree);
 #pragma unroll
   for (int it = 0; it < 2; ++it) {
     const int idx = k.tid + it * kThreads;
     if (idx >= R * n4) break;
     const int t = idx >> k.g.lg_n4, c4 = idx & (n4 - 1);
-    const float4* src = reinterpret_cast<const float4*>(ws + (size_t)t * d + k.c * ks) + c4;
-    const size_t step = (size_t)kMaxRows * d / 4;
+    const unsigned long long* src = ws + (size_t)t * d + k.c * ks + c4 * 4;
+    const size_t step = (size_t)kMaxRows * d;
     float4 acc = *reinterpret_cast<const float4*>(x_s + t * ks + c4 * 4);
     {
       const uint2 bw = bias.w[it];
       acc.x += __uint_as_float(bw.x << 16); acc.y += __uint_as_float(bw.x & 0xffff0000u);
       acc.z += __uint_as_float(bw.y << 16); acc.w += __uint_as_float(bw.y & 0xffff0000u);
     }
-    for (int p0 = 0; p0 < H; p0 += 16) {
-      float4 v[16];
+    for (int p0 = 0; p0 < H; p0 += 8) {
+      // eight producers per round; a round is repeated as a whole until every word carries this reduction's tag
+      unsigned long long v[8][4];
+      const unsigned long long t0 = clock64();
+      for (unsigned spins = 0;; ++spins) {
 #pragma unroll
-      for (int u = 0; u < 16; ++u) v[u] = (p0 + u < H) ? __ldcg(src + (size_t)(p0 + u) * step) : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int u = 0; u < 8; ++u) {
+          const unsigned long long* at = src + (size_t)min(p0 + u, H - 1) * step;
+          ll_load2(at, v[u][0], v[u][1]);
+          ll_load2(at + 2, v[u][2], v[u][3]);
+        }
+        bool ready = true;
 #pragma unroll
-      for (int u = 0; u < 16; ++u)
-        if (p0 + u < H) { acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w; }
+        for (int u = 0; u < 8; ++u)
+          ready = ready && (unsigned)(v[u][0] >> 32) == tag && (unsigned)(v[u][1] >> 32) == tag &&
+                  (unsigned)(v[u][2] >> 32) == tag && (unsigned)(v[u][3] >> 32) == tag;
+        if (ready || is_zombie(k)) break;
+        if ((spins & 15u) == 15u) {
+          if (__ldcg(p.bar + kBarAbort) != 0u) { *reinterpret_cast<volatile int*>(&k.ctl->zombie) = 1; break; }
+          if ((unsigned long long)(clock64() - t0) > p.spin) { raise_abort(k, 104); break; }
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (p0 + u < H) {
+          acc.x += __uint_as_float((unsigned)v[u][0]); acc.y += __uint_as_float((unsigned)v[u][1]);
+          acc.z += __uint_as_float((unsigned)v[u][2]); acc.w += __uint_as_float((unsigned)v[u][3]);
+        }
     }
+    *reinterpret_cast<float4*>(x_s + t * ks + c4 * 4) = acc;
+  }
+}
+
+// The same for models with many heads, where every CTA pulling all H shares of its slice (H * 8 KB through L2, H-fold
+// redundant over the clusters) is what takes the time: cluster j sums only part j of the slice (2R of the slice's
+// R * ks / 4 four-value items; one (item, producer) load per thread, summed in producer order through shared memory)
+// and publishes the sums, again as tagged words; every cluster then gathers the H parts.  Two trips through L2 but
+// 16 KB per CTA instead of 128.
+__device__ __forceinline__ bool ll_wait4(const Cta& k, const unsigned long long* at, unsigned tag, float4& out) {
+  const StackParams& p = *k.p;
+  unsigned long long a0, a1, a2, a3;
+  const unsigned long long t0 = clock64();
+  for (unsigned spins = 0;; ++spins) {
+    ll_load2(at, a0, a1);
+    ll_load2(at + 2, a2, a3);
+    if (((unsigned)(a0 >> 32) == tag && (unsigned)(a1 >> 32) == tag && (unsigned)(a2 >> 32) == tag && (unsigned)(a3 >> 32) == tag) ||
+        is_zombie(k))
+      break;
+    if ((spins & 15u) == 15u) {
+      if (__ldcg(p.bar + kBarAbort) != 0u) { *reinterpret_cast<volatile int*>(&k.ctl->zombie) = 1; break; }
+      if ((unsigned long long)(clock64() - t0) > p.spin) { raise_abort(k, 104); break; }
+    }
+  }
+  out = make_float4(__uint_as_float((unsigned)a0), __uint_as_float((unsigned)a1), __uint_as_float((unsigned)a2), __uint_as_float((unsigned)a3));
+  return true;
+}
+__device__ __forceinline__ void reduce_slice_2hop(const Cta& k, float* x_s, const unsigned long long* ws, unsigned long long* gather,
+                                                  float4* red, const Words& bias, unsigned tag, int nfree) {
+  const StackParams& p = *k.p;
+  const int ks = k.g.ks, n4 = ks >> 2, R = p.R, d = p.d, H = p.H, j = blockIdx.y;
+  __syncthreads();                                             // every warp is done with the tiles released here
+  if (k.tid == kPumpThread && nfree) release_tiles(k, nfree);
+  const int ipp = (R * n4) / H;                                // items of a part: n4 = 2H, so 2R
+  const size_t step = (size_t)kMaxRows * d;
+  // hop 1: (item q of part j, producer h) per thread
+  for (int w = k.tid; w < ipp * H; w += kThreads) {
+    const int q = w / H, h = w - q * H;
+    const int item = j * ipp + q, t = item >> k.g.lg_n4, c4 = item & (n4 - 1);
+    float4 v;
+    ll_wait4(k, ws + (size_t)h * step + (size_t)t * d + k.c * ks + c4 * 4, tag, v);
+    red[q * H + h] = v;
+  }
+  __syncthreads();
+  if (k.tid < ipp) {
+    const int q = k.tid;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int h = 0; h < H; ++h) { const float4 v = red[q * H + h]; acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w; }
+    const int item = j * ipp + q, t = item >> k.g.lg_n4, c4 = item & (n4 - 1);
+    unsigned long long* at = gather + (size_t)t * d + k.c * ks + c4 * 4;
+    ll_store(at, acc.x, tag); ll_store(at + 1, acc.y, tag); ll_store(at + 2, acc.z, tag); ll_store(at + 3, acc.w, tag);
+  }
+  // hop 2: every cluster gathers the whole slice
+#pragma unroll
+  for (int it = 0; it < 2; ++it) {
+    const int idx = k.tid + it * kThreads;
+    if (idx >= R * n4) break;
+    const int t = idx >> k.g.lg_n4, c4 = idx & (n4 - 1);
+    float4 acc = *reinterpret_cast<const float4*>(x_s + t * ks + c4 * 4);
+    {
+      const uint2 bw = bias.w[it];
+      acc.x += __uint_as_float(bw.x << 16); acc.y += __uint_as_float(bw.x & 0xffff0000u);
+      acc.z += __uint_as_float(bw.y << 16); acc.w += __uint_as_float(bw.y & 0xffff0000u);
+    }
+    float4 v;
+    ll_wait4(k, gather + (size_t)t * d + k.c * ks + c4 * 4, tag, v);
+    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
     *reinterpret_cast<float4*>(x_s + t * ks + c4 * 4) = acc;
   }
 }
@@ -644,6 +714,9 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
   const int d = p.d, ks = g.ks, R = p.R, nb = p.nb, rpb = p.rows_per_b;
   const int lg = lane >> 2, t4 = lane & 3;
   float* x_s = reinterpret_cast<float*>(ssm + p.lay.x);
+  // scratch of the two-hop reduction, [item of the part][producer] (2 R H float4): the hidden-unit planes are idle during
+  // every reduction -- a rank only writes another rank's planes two cluster-wide exchanges after its own reduction
+  float4* red_s = reinterpret_cast<float4*>(ssm + p.lay.hid);
   uint8_t* xh = ssm + p.lay.xh;
   uint8_t* xl = ssm + p.lay.xl;
   uint8_t* oh = ssm + p.lay.oh;
@@ -664,7 +737,6 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
   int* s_pt = reinterpret_cast<int*>(ssm + p.lay.pt);
   LayerPtrs* layers_s = reinterpret_cast<LayerPtrs*>(ssm + p.lay.layers);
   float* stats_mine = stats_in + c * kMaxRows * 2;
-  const unsigned G = gridDim.x * gridDim.y;
   const int hrow = g.UPR * 2;                                             // bytes per row of a rank's hidden planes
   const int hblock = 2 * RP * hrow;                                       // bytes of a rank's hidden planes (hi, lo)
 
@@ -783,9 +855,10 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
     }
     if (l > 0) {
       const Words bw = load_words(k, layers_s[l - 1].b2);
-      grid_join(k, base + (++nbar) * G, g.PH);
+      ++nbar;
       BPD_TR();
-      reduce_slice(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, bw);
+      if (p.H >= 16) reduce_slice_2hop(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, p.gather + (size_t)((nbar - 1) & 1) * kMaxRows * d, red_s, bw, base + nbar, g.PH);
+      else reduce_slice(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, bw, base + nbar, g.PH);
       BPD_TR();
       if (p.layer_dump && j == 0) {
         __syncthreads();
@@ -944,7 +1017,8 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
     BPD_TR();
     // this head's share of the output projection for feature slice c
     {
-      float* wsj = p.ws + ((size_t)(nbar & 1) * p.H + j) * kMaxRows * d;
+      unsigned long long* wsj = p.ws + ((size_t)(nbar & 1) * p.H + j) * kMaxRows * d;
+      const unsigned tag_out = base + nbar + 1;            // the reduction that consumes these shares
       for (int mt = warp; mt < ks / 16; mt += kWarps) {
         float acc[NT][4];
 #pragma unroll
@@ -957,7 +1031,7 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int row = mt * 16 + lg + ((e & 2) ? 8 : 0), token = nt * 8 + 2 * t4 + (e & 1);
-            if (token < R) wsj[(size_t)token * d + c * ks + row] = acc[nt][e];
+            if (token < R) ll_store(wsj + (size_t)token * d + c * ks + row, acc[nt][e], tag_out);
           }
       }
       seq += 1;
@@ -968,9 +1042,10 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
     gw = load_words(k, LP.g2);
     const Words nobias = load_words(k, nullptr);
     if (tid < kDH) { fs = LP.s_cq[j * kDH + tid]; fc = LP.c_cq[j * kDH + tid]; }
-    grid_join(k, base + (++nbar) * G, 1);
+    ++nbar;
     BPD_TR();
-    reduce_slice(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, nobias);
+    if (p.H >= 16) reduce_slice_2hop(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, p.gather + (size_t)((nbar - 1) & 1) * kMaxRows * d, red_s, nobias, base + nbar, 1);
+      else reduce_slice(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, nobias, base + nbar, 1);
     BPD_TR();
     planes_and_stats<NT>(k, x_s, gw, xh, xl, stats_mine);
     __syncthreads();
@@ -1032,7 +1107,8 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
     ++xn;
     BPD_TR();
     {
-      float* wsj = p.ws + ((size_t)(nbar & 1) * p.H + j) * kMaxRows * d;
+      unsigned long long* wsj = p.ws + ((size_t)(nbar & 1) * p.H + j) * kMaxRows * d;
+      const unsigned tag_out = base + nbar + 1;            // the reduction that consumes these shares
       for (int mt = warp; mt < ks / 16; mt += kWarps) {
         float acc[NT][4];
 #pragma unroll
@@ -1045,7 +1121,7 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int row = mt * 16 + lg + ((e & 2) ? 8 : 0), token = nt * 8 + 2 * t4 + (e & 1);
-            if (token < R) wsj[(size_t)token * d + c * ks + row] = acc[nt][e];
+            if (token < R) ll_store(wsj + (size_t)token * d + c * ks + row, acc[nt][e], tag_out);
           }
       }
       seq += 1;
@@ -1062,9 +1138,10 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
       fs1[u] = idx < g.UPR * R ? LP.s_f1[unit] : 0.f;
       fc1[u] = idx < g.UPR * R ? LP.c_f1[unit] : 0.f;
     }
-    grid_join(k, base + (++nbar) * G, 1);
+    ++nbar;
     BPD_TR();
-    reduce_slice(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, nobias);
+    if (p.H >= 16) reduce_slice_2hop(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, p.gather + (size_t)((nbar - 1) & 1) * kMaxRows * d, red_s, nobias, base + nbar, 1);
+      else reduce_slice(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, nobias, base + nbar, 1);
     BPD_TR();
     planes_and_stats<NT>(k, x_s, gw, xh, xl, stats_mine);
     __syncthreads();
@@ -1122,7 +1199,8 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
     BPD_TR();
     // the hidden units times slice c of the second projection: this cluster's share of the block's output
     {
-      float* wsj = p.ws + ((size_t)(nbar & 1) * p.H + j) * kMaxRows * d;
+      unsigned long long* wsj = p.ws + ((size_t)(nbar & 1) * p.H + j) * kMaxRows * d;
+      const unsigned tag_out = base + nbar + 1;            // the reduction that consumes these shares
       for (int mt = warp; mt < ks / 16; mt += kWarps) {
         float acc[NT][4];
 #pragma unroll
@@ -1146,7 +1224,7 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int row = mt * 16 + lg + ((e & 2) ? 8 : 0), token = nt * 8 + 2 * t4 + (e & 1);
-            if (token < R) wsj[(size_t)token * d + c * ks + row] = acc[nt][e];
+            if (token < R) ll_store(wsj + (size_t)token * d + c * ks + row, acc[nt][e], tag_out);
           }
       }
       seq += g.PH;
@@ -1156,10 +1234,11 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
   // =================================================================== final layer norm
   {
     const Words bw = load_words(k, layers_s[p.L - 1].b2), gw = load_words(k, p.lnf_g);
-    grid_join(k, base + (++nbar) * G, g.PH);
+    ++nbar;
     BPD_TR();
     pdl_launch_dependents();
-    reduce_slice(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, bw);
+    if (p.H >= 16) reduce_slice_2hop(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, p.gather + (size_t)((nbar - 1) & 1) * kMaxRows * d, red_s, bw, base + nbar, g.PH);
+      else reduce_slice(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, bw, base + nbar, g.PH);
     BPD_TR();
     if (p.layer_dump && j == 0) {
       __syncthreads();
@@ -1198,7 +1277,7 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
       *reinterpret_cast<uint2*>(yp + p.xn_plane) = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
       *reinterpret_cast<float4*>(p.h_f32 + (size_t)t * d + col) = make_float4(o[0], o[1], o[2], o[3]);
     }
-    if (c == 0 && tid == 0) p.bar[kBarBase] = base + nbar * G;     // where the next launch starts counting
+    if (c == 0 && tid == 0) p.bar[kBarBase] = base + nbar;         // tags of the next launch go on from here
   }
 #ifdef BPD_STACK_TRACE
   if (g_stack_trace && tid == 0) {

@@ -419,6 +419,7 @@ def test_full_attention_beyond_2048_keys(bpd):
     k, N = w.cfg.k_model, w.n_decode
     for path in ("cluster", "persistent"):
         s = bpd.Session(model, w.batch, w.max_src, N, options=LAYER_PATHS[path])
+        assert s.layer_path == (2 if path == "persistent" else 1)
         s.bpd_encode(src, src_len)
         g_ids, _, _ = s.bpd_decode_greedy(N)
         s.bpd_encode(src, src_len)
@@ -543,8 +544,9 @@ def test_layer_paths_agree(bpd, w):
     blob, model, src, src_len, om = _setup(bpd, w)
     k, N = w.cfg.k_model, w.n_decode
 
-    def run(options):
+    def run(options, path):
         s = bpd.Session(model, w.batch, w.max_src, N, options=options)
+        assert s.layer_path == path, f"asked for {options}, got layer path {s.layer_path}"
         s.bpd_encode(src, src_len)
         steps = []
         for _ in range(4):
@@ -554,9 +556,9 @@ def test_layer_paths_agree(bpd, w):
         s.close()
         return steps
 
-    ref = run(LAYER_PATHS["per-projection"])
-    for name in ("persistent", "cluster"):
-        got = run(LAYER_PATHS[name])
+    ref = run(LAYER_PATHS["per-projection"], 0)
+    for name, path in (("persistent", 2), ("cluster", 1)):
+        got = run(LAYER_PATHS[name], path)
         for it, ((ha, la, xa), (hb, lb, xb)) in enumerate(zip(got, ref)):
             assert np.abs(xa - xb).max() <= 2e-3, f"{name}, iteration {it}: residual stream differs"
             assert np.abs(ha - hb).max() <= 2e-3 and np.abs(la - lb).max() <= 2e-3, f"{name}, iteration {it}"
@@ -571,6 +573,7 @@ def test_layer_dump_matches_the_oracle(bpd):
     k, N = w.cfg.k_model, w.n_decode
     for name, options in LAYER_PATHS.items():
         s = bpd.Session(model, 1, w.max_src, N, options=options)
+        assert s.layer_path == {"persistent": 2, "cluster": 1, "per-projection": 0}[name]
         s.bpd_encode(src, src_len)
         s.bpd_iteration(k, N)
         r = s.bpd_iteration(k, N, want_layers=True)
