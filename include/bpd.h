@@ -108,7 +108,9 @@ typedef struct {
   int32_t cluster_layers;     /* decoder layers as three cluster launches each (<= 16 rows per pass)        */
   int32_t persistent_layers;  /* all decoder layers of a pass in one persistent TMA-fed kernel (<= 16 rows
                                  per pass, d_model 256 / 512 / 1024; takes precedence over cluster_layers).
-                                 Default off: measured slower than the cluster launches on B200             */
+                                 Default: on for sessions of at most 256 positions whose encoder rows fit
+                                 the staging tile (measured faster there), off elsewhere; 1 asks for it
+                                 wherever it runs.  See bpd_session_create_opt for what it needs          */
   int32_t stage_encoder_rows; /* encoder keys / values staged in shared memory for cross-attention          */
   int32_t l2_stream_hints;    /* weights read once per pass are loaded "evict first"                        */
 } bpd_session_options;
@@ -142,11 +144,13 @@ int bpd_session_create(const bpd_model* model, int batch, int max_src, int max_t
                        void* dev_session_buf, size_t dev_bytes, void* cuda_stream, bpd_session** out);
 
 /* The same with explicit options (NULL = all defaults).  A session that runs
- * its decoder layers in the persistent kernel (persistent_layers) occupies
- * most of the GPU with CTAs that wait for one another: passes of two such
- * sessions must not overlap on one GPU (keep them on one stream, or finish
- * one decode before starting another); if they do, their bounded waits expire
- * and the calls return BPD_E_TIMEOUT. */
+ * its decoder layers in the persistent kernel (persistent_layers; see
+ * bpd_session_layer_path) occupies most of the GPU with CTAs that wait for
+ * one another: passes of two such sessions must not overlap on one GPU (keep
+ * them on one stream, or finish one decode before starting another); if they
+ * do, their bounded waits expire after about a second and the calls return
+ * BPD_E_TIMEOUT.  Programs that decode on several streams of one GPU at the
+ * same time set persistent_layers = 0. */
 void bpd_session_options_init(bpd_session_options* options);
 int bpd_session_create_opt(const bpd_model* model, int batch, int max_src, int max_tgt,
                            void* dev_session_buf, size_t dev_bytes, void* cuda_stream,

@@ -762,6 +762,8 @@ static int stack_setup(bpd_session* s) {
   const int rows = s->B * c.k_model;
   if (!s->tc || !s->opt.persistent_layers || !stack_shapes_ok(c, rows)) return BPD_OK;
   const bool long_seq = s->max_tgt + 1 + c.k_model > 32 * fused::kC;
+  const bool only_lean = s->opt.persistent_layers < 0;   // the library's own choice: sessions the lean kernel takes
+  if (only_lean && (long_seq || !s->opt.stage_encoder_rows || s->B * s->max_src > 256)) return BPD_OK;
   cudaDeviceProp prop;
   int dev = 0;
   BPD_CUDA(cudaGetDevice(&dev));
@@ -775,7 +777,7 @@ static int stack_setup(bpd_session* s) {
   int minb = 0;
   for (size_t budget : budgets) {
     ++minb;                                    // first one CTA per SM, then two
-    for (int staged = s->opt.stage_encoder_rows ? 1 : 0; staged >= 0 && !ok; --staged) {
+    for (int staged = s->opt.stage_encoder_rows ? 1 : 0; staged >= (only_lean ? 1 : 0) && !ok; --staged) {
       cross_rows = (staged && s->B * s->max_src <= 256) ? s->B * s->max_src : 0;
       if (staged && !cross_rows) continue;
       if (budget <= 1024 || !stack_plan(c, rows, s->B, s->ppr, cross_rows, long_seq, budget - 1024, &lay)) continue;
@@ -1284,7 +1286,7 @@ int bpd_session_create_opt(const bpd_model* model, int batch, int max_src, int m
   s->fold_ln = (s->tc && o.fold_layer_norms != 0 && (batch * model->cfg.k_model <= 16 || model->cfg.d % 256 == 0)) ? 1 : 0;
   s->fused = (s->tc && fused::supported(model->cfg.d, model->cfg.H, model->cfg.d_ff, batch * model->cfg.k_model) &&
               o.cluster_layers != 0) ? 1 : 0;
-  s->opt.persistent_layers = o.persistent_layers == 1 ? 1 : 0;   // opt-in: measured slower than the cluster launches
+  s->opt.persistent_layers = o.persistent_layers;   // -1: where its lean variant applies (measured faster there), 0: never, 1: wherever it runs
   s->opt.stage_encoder_rows = o.stage_encoder_rows != 0 ? 1 : 0;
   s->opt.l2_stream_hints = o.l2_stream_hints != 0 ? 1 : 0;
   s->stack = 0; s->stack_dump = nullptr;

@@ -20,9 +20,9 @@ MINI_F32 = Workload("minif", ModelConfig(1, 2, 96, 6, 200, 333, 3, 136, dtype=DT
 
 
 LAYER_PATHS = {
-    "persistent": {"persistent_layers": 1},                       # one kernel for the whole layer stack (opt-in)
-    "cluster": {},                                                # three cluster launches per layer (default)
-    "per-projection": {"cluster_layers": 0},
+    "persistent": {"persistent_layers": 1},                       # one kernel for the whole layer stack
+    "cluster": {"persistent_layers": 0},                          # three cluster launches per layer
+    "per-projection": {"persistent_layers": 0, "cluster_layers": 0},
 }
 
 
