@@ -36,6 +36,7 @@ NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu capture
 # summarised under profiles/ (None until a capture of the current kernel exists)
 TRAFFIC = {"C3": 538161152 + 3223296}     # profiles/head_output_gemm_tc_c3.txt
+TRAFFIC_LAYERS = {"C3": 179013120 + 4276224}   # profiles/layer_stack_kernel_c3.txt
 
 
 def _peaks():
@@ -302,12 +303,29 @@ def run_gpu(args):
     n_w2, ms_w2 = phases[2]
     # the priming pass evaluates the same k heads on one row per sequence: same weight bytes per launch
     w2_us = 1e3 * ms_w2 / max(1, n_w2)
+    roofline_head_output = None
     if w.batch < 16:
         achieved = w2_bytes / (w2_us * 1e-6) / 1e9
         roofline = {"bound": "hbm", "kernel": "head output layers (k*d_model x k*d_hidden weights, + residual)",
                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "peak_kind": f"of {peak_kind}", "traffic": TRAFFIC.get(args.workload),
                     "bytes_per_launch": w2_bytes, "us_per_launch": w2_us, "launches_timed": n_w2}
+        if sess.layer_path == 2:
+            # the whole decoder-layer stack is one launch here and the longest kernel of the pass: it is the one the
+            # roofline line reports (bytes it must move: every layer's weights once, the cache once); the head output
+            # projection, the kernel that moves most of the pass's bytes, keeps a line of its own
+            roofline_head_output = roofline
+            e = cfg.elem_bytes
+            layer_bytes = e * cfg.n_dec * (6 * cfg.d_model * cfg.d_model + 2 * cfg.d_model * cfg.d_ff) + \
+                w.batch * cfg.n_dec * 2 * e * cfg.d_model * (mean_T + float(src_len.mean()))
+            n_l, ms_l = phases[0]
+            l_us = 1e3 * ms_l / max(1, n_l)
+            achieved = layer_bytes / (l_us * 1e-6) / 1e9
+            roofline = {"bound": "hbm", "kernel": "decoder layer stack (persistent kernel: embedding, 6 layers, final layer norm)",
+                        "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                        "peak_kind": f"of {peak_kind}", "traffic": TRAFFIC_LAYERS.get(args.workload),
+                        "bytes_per_launch": layer_bytes, "us_per_launch": l_us, "launches_timed": n_l,
+                        "note": "latency-bound: a chain of 19 dependent reductions across all SMs and 42 exchanges inside the clusters"}
     else:
         # batched: the same kernel is a dense contraction.  Sessions this wide evaluate the heads lazily: one launch
         # for head 1 at all batch*k positions, one for all k heads at the accepted position of each row; the
@@ -402,6 +420,8 @@ def run_gpu(args):
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
         "gpu_launches": int(launches),
         "roofline": roofline,
+        "roofline_head_output": roofline_head_output,
+        "layer_path": sess.layer_path,
         "cpu_baseline": cpu,
     }
     print(json.dumps(line))
