@@ -240,10 +240,12 @@ int bpd_profile(bpd_session* s, int enable);
 int bpd_profile_read(bpd_session* s, int phase, int64_t* launches, double* total_ms);
 
 /* Self test of the bounded device-side waits: launches one CTA that waits on a
- * barrier nothing ever arrives on, with a limit of about limit_us microseconds.
- * The wait gives up, the kernel records the error word and returns normally, and
- * the call reports BPD_E_TIMEOUT -- the status a real decode call returns if one
- * of its kernels' waits ever expires.  BPD_OK would mean the wait did not expire.
+ * barrier nothing ever arrives on, then one that waits for tagged words nobody
+ * writes (the two kinds of wait the kernels have), each with a limit of about
+ * limit_us microseconds.  The waits give up, the kernels record their error words
+ * and return normally, and the call reports BPD_E_TIMEOUT -- the status a real
+ * decode call returns if one of its kernels' waits ever expires.  BPD_OK or
+ * BPD_E_CUDA would mean that a wait did not expire the way it should.
  * dev_word: device int32 used as the error word.  Synchronises the stream. */
 int bpd_debug_wait_timeout(int32_t* dev_word, int limit_us, void* cuda_stream);
 

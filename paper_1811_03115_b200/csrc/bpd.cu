@@ -1673,8 +1673,17 @@ int bpd_debug_wait_timeout(int32_t* dev_word, int limit_us, void* cuda_stream) {
   int word = 0;
   BPD_CUDA(cudaMemcpyAsync(&word, dev_word, sizeof(int), cudaMemcpyDeviceToHost, st));
   BPD_CUDA(cudaStreamSynchronize(st));
-  if (word) return fail(BPD_E_TIMEOUT, "a bounded wait inside the probe kernel expired (code %d), as it should", word);
-  return BPD_OK;
+  if (!word) return BPD_OK;
+  // the same for the tagged words the persistent layer kernel's reductions wait on
+  const int first = word;
+  BPD_CUDA(cudaMemsetAsync(dev_word, 0, sizeof(int), st));
+  stack::tagged_wait_probe_kernel<<<1, 32, 0, st>>>(dev_word, (unsigned long long)limit_us * (unsigned long long)khz / 1000ull);
+  ++g_launches;
+  BPD_CUDA(cudaGetLastError());
+  BPD_CUDA(cudaMemcpyAsync(&word, dev_word, sizeof(int), cudaMemcpyDeviceToHost, st));
+  BPD_CUDA(cudaStreamSynchronize(st));
+  if (word != 104) return fail(BPD_E_CUDA, "the wait on tagged words did not expire as it should (word %d)", word);
+  return fail(BPD_E_TIMEOUT, "the bounded waits inside the probe kernels expired (codes %d and %d), as they should", first, word);
 }
 
 // ------------------------------------------------------------------ single operators

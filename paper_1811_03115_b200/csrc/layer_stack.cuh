@@ -478,6 +478,29 @@ __device__ __forceinline__ void reduce_slice_2hop(const Cta& k, float* x_s, cons
   }
 }
 
+// Self test of the bounded wait on tagged words: one warp waits for a tag that nobody writes, gives up after
+// `limit_cycles`, records the error code a real pass would (104) and raises the abort word; the kernel returns
+// normally and the context stays usable.
+static __device__ unsigned long long g_probe_words[4];
+static __device__ unsigned g_probe_bar[kBarWords];
+static __global__ void tagged_wait_probe_kernel(int* error, unsigned long long limit_cycles) {
+  __shared__ Ctl ctl;
+  __shared__ StackParams sp;
+  if (threadIdx.x == 0) {
+    ctl.zombie = 0;
+    sp.error = error; sp.bar = g_probe_bar; sp.spin = limit_cycles;
+    g_probe_bar[kBarAbort] = 0u;
+    for (int i = 0; i < 4; ++i) g_probe_words[i] = 0ull;          // tag 0: never the tag of a reduction
+  }
+  __syncthreads();
+  Cta k;
+  k.p = &sp; k.ctl = &ctl; k.tid = threadIdx.x;
+  float4 v;
+  ll_wait4(k, g_probe_words, 1u, v);
+  __syncthreads();
+  if (threadIdx.x == 0 && (ctl.zombie == 0 || g_probe_bar[kBarAbort] == 0u)) atomicExch(error, -1);   // the wait ended some other way
+}
+
 // Planes (hi, lo) of x * gain for this rank's columns, and the slice's per-row (mean, sum of squared deviations)
 // into this rank's block of the statistics table (sent to the other ranks with the next exchange).  A thread
 // reads back the items it wrote itself in reduce_slice / the embedding (same idx -> thread mapping): no barrier

@@ -723,11 +723,13 @@ def test_long_sequences_share_their_keys(bpd, w):
 
 
 def test_bounded_wait_expires_and_the_context_survives(bpd):
-    """Failure detection without a fault: a wait on a barrier nobody signals gives up after its limit,
-    the call reports BPD_E_TIMEOUT and the same process keeps computing correctly afterwards."""
+    """Failure detection without a fault: a wait on a barrier nobody signals, and a wait for tagged words nobody
+    writes, give up after their limit; the call reports BPD_E_TIMEOUT and the same process keeps computing
+    correctly afterwards."""
     import torch
     assert bpd.bpd_debug_wait_timeout(2000) == -7
-    assert "expired" in bpd.lib.bpd_last_error().decode()
+    msg = bpd.lib.bpd_last_error().decode()
+    assert "expired" in msg and "104" in msg          # both kinds of wait: the mbarrier and the tagged words
     x = torch.randn(4, 64).cuda()
     w = torch.randn(10, 64).cuda()
     y = bpd.bpd_op_linear(x, w).cpu()
