@@ -682,8 +682,7 @@ static bool stack_plan(const Config& c, int rows, int nb, int ppr, int cross_row
   L.xl = take((size_t)RP * g.ks * 2);
   L.oh = take((size_t)RP * 128);
   L.ol = take((size_t)RP * 128);
-  // hidden-unit planes; the same bytes are the scratch of the two-hop reduction (2 * rows * H float4)
-  L.hid = take(std::max((size_t)fused::kC * 2 * RP * g.UPR * 2, c.H >= 16 ? (size_t)2 * rows * c.H * 16 : (size_t)0));
+  L.hid = take((size_t)fused::kC * 2 * RP * g.UPR * 2);
   const size_t chunk = std::max((size_t)NT * 3 * fused::kDH * 4, (size_t)g.UPR * RP * 4);
   L.outbox = take(fused::kC * chunk);
   L.inbox = take(fused::kC * chunk);

@@ -413,7 +413,7 @@ __device__ __forceinline__ void reduce_slice(const Cta& k, float* x_s, const uns
 
 // The same for models with many heads, where every CTA pulling all H shares of its slice (H * 8 KB through L2, H-fold
 // redundant over the clusters) is what takes the time: cluster j sums only part j of the slice (2R of the slice's
-// R * ks / 4 four-value items; one (item, producer) load per thread, summed in producer order through shared memory)
+// R * ks / 4 four-value items; one (item, producer) load per thread, the 16 producers added by a fixed butterfly)
 // and publishes the sums, again as tagged words; every cluster then gathers the H parts.  Two trips through L2 but
 // 16 KB per CTA instead of 128.
 __device__ __forceinline__ bool ll_wait4(const Cta& k, const unsigned long long* at, unsigned tag, float4& out) {
@@ -435,29 +435,29 @@ __device__ __forceinline__ bool ll_wait4(const Cta& k, const unsigned long long*
   return true;
 }
 __device__ __forceinline__ void reduce_slice_2hop(const Cta& k, float* x_s, const unsigned long long* ws, unsigned long long* gather,
-                                                  float4* red, const Words& bias, unsigned tag, int nfree) {
+                                                  const Words& bias, unsigned tag, int nfree) {
   const StackParams& p = *k.p;
   const int ks = k.g.ks, n4 = ks >> 2, R = p.R, d = p.d, H = p.H, j = blockIdx.y;
   __syncthreads();                                             // every warp is done with the tiles released here
   if (k.tid == kPumpThread && nfree) release_tiles(k, nfree);
   const int ipp = (R * n4) / H;                                // items of a part: n4 = 2H, so 2R
   const size_t step = (size_t)kMaxRows * d;
-  // hop 1: (item q of part j, producer h) per thread
+  // hop 1: (item q of part j, producer h) per thread; H = 16, so the 16 producers of an item sit in one half-warp
+  // and are added by a fixed butterfly (ipp * H = 32 R pairs: whole warps are in or out); lane 0's order is the sum
   for (int w = k.tid; w < ipp * H; w += kThreads) {
-    const int q = w / H, h = w - q * H;
+    const int q = w >> 4, h = w & 15;
     const int item = j * ipp + q, t = item >> k.g.lg_n4, c4 = item & (n4 - 1);
     float4 v;
     ll_wait4(k, ws + (size_t)h * step + (size_t)t * d + k.c * ks + c4 * 4, tag, v);
-    red[q * H + h] = v;
-  }
-  __syncthreads();
-  if (k.tid < ipp) {
-    const int q = k.tid;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int h = 0; h < H; ++h) { const float4 v = red[q * H + h]; acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w; }
-    const int item = j * ipp + q, t = item >> k.g.lg_n4, c4 = item & (n4 - 1);
-    unsigned long long* at = gather + (size_t)t * d + k.c * ks + c4 * 4;
-    ll_store(at, acc.x, tag); ll_store(at + 1, acc.y, tag); ll_store(at + 2, acc.z, tag); ll_store(at + 3, acc.w, tag);
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) {
+      v.x += __shfl_xor_sync(0xffffffffu, v.x, o); v.y += __shfl_xor_sync(0xffffffffu, v.y, o);
+      v.z += __shfl_xor_sync(0xffffffffu, v.z, o); v.w += __shfl_xor_sync(0xffffffffu, v.w, o);
+    }
+    if (h == 0) {
+      unsigned long long* at = gather + (size_t)t * d + k.c * ks + c4 * 4;
+      ll_store(at, v.x, tag); ll_store(at + 1, v.y, tag); ll_store(at + 2, v.z, tag); ll_store(at + 3, v.w, tag);
+    }
   }
   // hop 2: every cluster gathers the whole slice
 #pragma unroll
@@ -737,9 +737,6 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
   const int d = p.d, ks = g.ks, R = p.R, nb = p.nb, rpb = p.rows_per_b;
   const int lg = lane >> 2, t4 = lane & 3;
   float* x_s = reinterpret_cast<float*>(ssm + p.lay.x);
-  // scratch of the two-hop reduction, [item of the part][producer] (2 R H float4): the hidden-unit planes are idle during
-  // every reduction -- a rank only writes another rank's planes two cluster-wide exchanges after its own reduction
-  float4* red_s = reinterpret_cast<float4*>(ssm + p.lay.hid);
   uint8_t* xh = ssm + p.lay.xh;
   uint8_t* xl = ssm + p.lay.xl;
   uint8_t* oh = ssm + p.lay.oh;
@@ -880,7 +877,7 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
       const Words bw = load_words(k, layers_s[l - 1].b2);
       ++nbar;
       BPD_TR();
-      if (p.H >= 16) reduce_slice_2hop(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, p.gather + (size_t)((nbar - 1) & 1) * kMaxRows * d, red_s, bw, base + nbar, g.PH);
+      if (p.H == 16) reduce_slice_2hop(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, p.gather + (size_t)((nbar - 1) & 1) * kMaxRows * d, bw, base + nbar, g.PH);
       else reduce_slice(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, bw, base + nbar, g.PH);
       BPD_TR();
       if (p.layer_dump && j == 0) {
@@ -1067,7 +1064,7 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
     if (tid < kDH) { fs = LP.s_cq[j * kDH + tid]; fc = LP.c_cq[j * kDH + tid]; }
     ++nbar;
     BPD_TR();
-    if (p.H >= 16) reduce_slice_2hop(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, p.gather + (size_t)((nbar - 1) & 1) * kMaxRows * d, red_s, nobias, base + nbar, 1);
+    if (p.H == 16) reduce_slice_2hop(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, p.gather + (size_t)((nbar - 1) & 1) * kMaxRows * d, nobias, base + nbar, 1);
       else reduce_slice(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, nobias, base + nbar, 1);
     BPD_TR();
     planes_and_stats<NT>(k, x_s, gw, xh, xl, stats_mine);
@@ -1163,7 +1160,7 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
     }
     ++nbar;
     BPD_TR();
-    if (p.H >= 16) reduce_slice_2hop(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, p.gather + (size_t)((nbar - 1) & 1) * kMaxRows * d, red_s, nobias, base + nbar, 1);
+    if (p.H == 16) reduce_slice_2hop(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, p.gather + (size_t)((nbar - 1) & 1) * kMaxRows * d, nobias, base + nbar, 1);
       else reduce_slice(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, nobias, base + nbar, 1);
     BPD_TR();
     planes_and_stats<NT>(k, x_s, gw, xh, xl, stats_mine);
@@ -1260,7 +1257,7 @@ layer_stack_kernel(const __grid_constant__ StackMaps maps, const __grid_constant
     ++nbar;
     BPD_TR();
     pdl_launch_dependents();
-    if (p.H >= 16) reduce_slice_2hop(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, p.gather + (size_t)((nbar - 1) & 1) * kMaxRows * d, red_s, bw, base + nbar, g.PH);
+    if (p.H == 16) reduce_slice_2hop(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, p.gather + (size_t)((nbar - 1) & 1) * kMaxRows * d, bw, base + nbar, g.PH);
       else reduce_slice(k, x_s, p.ws + (size_t)((nbar - 1) & 1) * p.H * kMaxRows * d, bw, base + nbar, g.PH);
     BPD_TR();
     if (p.layer_dump && j == 0) {
