@@ -267,13 +267,15 @@ def test_state_and_argument_errors(bpd):
 
 # ---------------------------------------------------------------- paper-sized configurations
 
-def _full_size(bpd, name, iters, rows=None, layout=HEAD_DENSE, mean=2.0, free_iters=2):
+def _full_size(bpd, name, iters, rows=None, layout=HEAD_DENSE, mean=2.0, free_iters=2, layer_path=None):
     from harness import lockstep
-    w = WORKLOADS[name].with_layout(layout)
+    w = (WORKLOADS[name] if isinstance(name, str) else name).with_layout(layout)
     blob, model, src, src_len, om = _setup(bpd, w)
     del blob
     k, N = w.cfg.k_model, w.n_decode
     s = bpd.Session(model, w.batch, w.max_src, N)
+    if layer_path is not None:
+        assert s.layer_path == layer_path, f"expected layer path {layer_path}, got {s.layer_path}"
     s.bpd_encode(src, src_len)
     g_ids, _, _ = s.bpd_decode_greedy(N)
     s.bpd_encode(src, src_len)
@@ -308,6 +310,15 @@ def test_c2_base_model_blockdiag(bpd):
 
 def test_c3_big_model(bpd):
     _full_size(bpd, "C3", iters=3, mean=5.0, free_iters=1)
+
+
+def test_c3_model_two_sequences_sixteen_rows(bpd):
+    """The big model with two sequences of different source lengths: 16 rows per pass, the widest pass of the
+    few-row layer paths (two token tiles of 8 rows, 16 heads; the working buffers of two token tiles leave the
+    persistent kernel no room beside a second CTA on the SM, so such a session runs the cluster launches)."""
+    c3 = WORKLOADS["C3"]
+    w = Workload("c3x2", c3.cfg, c3.sigma, c3.weight_seed, 2103, 3103, batch=2, src_lo=23, src_hi=40, n_decode=40)
+    _full_size(bpd, w, iters=4, mean=5.0, free_iters=1, layer_path=1)
 
 
 def test_c5_super_resolution_shape(bpd):
