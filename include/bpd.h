@@ -109,8 +109,9 @@ typedef struct {
   int32_t persistent_layers;  /* all decoder layers of a pass in one persistent TMA-fed kernel (<= 16 rows
                                  per pass, d_model 256 / 512 / 1024; takes precedence over cluster_layers).
                                  Default: on for sessions of at most 256 positions whose encoder rows fit
-                                 the staging tile (measured faster there), off elsewhere; 1 asks for it
-                                 wherever it runs.  See bpd_session_create_opt for what it needs          */
+                                 the staging tile (measured faster there) while no other live session of
+                                 the device has it, off elsewhere; 1 asks for it wherever it runs.  See
+                                 bpd_session_create_opt for what it needs                                  */
   int32_t stage_encoder_rows; /* encoder keys / values staged in shared memory for cross-attention          */
   int32_t l2_stream_hints;    /* weights read once per pass are loaded "evict first"                        */
 } bpd_session_options;
@@ -149,8 +150,10 @@ int bpd_session_create(const bpd_model* model, int batch, int max_src, int max_t
  * one another: passes of two such sessions must not overlap on one GPU (keep
  * them on one stream, or finish one decode before starting another); if they
  * do, their bounded waits expire after about a second and the calls return
- * BPD_E_TIMEOUT.  Programs that decode on several streams of one GPU at the
- * same time set persistent_layers = 0. */
+ * BPD_E_TIMEOUT.  Left to the library (the default), at most one live session
+ * per device gets the persistent kernel -- a session created while another
+ * holds it runs the cluster launches, which may overlap with anything -- so
+ * only sessions that ask for it with persistent_layers = 1 can meet this. */
 void bpd_session_options_init(bpd_session_options* options);
 int bpd_session_create_opt(const bpd_model* model, int batch, int max_src, int max_tgt,
                            void* dev_session_buf, size_t dev_bytes, void* cuda_stream,

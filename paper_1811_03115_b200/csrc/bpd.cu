@@ -752,6 +752,19 @@ static bool stack_shapes_ok(const Config& c, int rows) {
   return true;
 }
 
+// Live sessions per device whose decoder layers run in the persistent kernel.  Two such kernels on one GPU at the
+// same time can starve each other of SMs (each waits for clusters the other keeps from being scheduled) until their
+// bounded waits expire, so the library's own choice gives the persistent kernel to one session per device at a time;
+// a session that asks for it explicitly (persistent_layers = 1) gets it regardless.
+static std::mutex g_stack_mu;
+static std::map<int, int> g_stack_live;
+static int stack_live(int dev, int delta) {
+  std::lock_guard<std::mutex> lock(g_stack_mu);
+  int& n = g_stack_live[dev];
+  n += delta;
+  return n;
+}
+
 // Decides whether the session runs its decoder layers in the persistent kernel and prepares what it needs:
 // a shared-memory plan under which all H clusters are resident at once, tensor maps and per-layer pointers.
 static int stack_setup(bpd_session* s) {
@@ -766,6 +779,7 @@ static int stack_setup(bpd_session* s) {
   cudaDeviceProp prop;
   int dev = 0;
   BPD_CUDA(cudaGetDevice(&dev));
+  if (only_lean && stack_live(dev, 0) > 0) return BPD_OK;   // another session of this device has it: see stack_live
   BPD_CUDA(cudaGetDeviceProperties(&prop, dev));
   const size_t optin = prop.sharedMemPerBlockOptin, per_sm = prop.sharedMemPerMultiprocessor;
   // one CTA per SM, or two (each block also reserves 1 KB of the SM's shared memory)
@@ -841,6 +855,8 @@ static int stack_setup(bpd_session* s) {
   memcpy(s->stack_layout, &lay, sizeof(lay));
   s->stack_cross_rows = cross_rows; s->stack_long = long_seq ? 1 : 0; s->stack_minb = minb;
   s->stack = 1;
+  s->stack_dev = dev;
+  stack_live(dev, +1);
   return BPD_OK;
 }
 
@@ -1332,6 +1348,7 @@ int bpd_session_create_opt(const bpd_model* model, int batch, int max_src, int m
 int bpd_session_destroy(bpd_session* s) {
   if (!s) return BPD_OK;
   cudaStreamSynchronize(s->stream);
+  if (s->stack) { stack_live(s->stack_dev, -1); s->stack = 0; }
   prof_clear(s);
   for (auto& kv : s->graphs)
     if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);

@@ -163,7 +163,7 @@ struct bpd_session {
   unsigned long long* stack_ws;   // device: [2][H][16][d] words (value, tag): the clusters' shares of the projection outputs
   unsigned* stack_bar;     // device: words of the device-wide join
   float* stack_dump;       // device: [n_dec][rows][d] residual stream after every layer (debug dump), or null
-  int stack_cross_rows, stack_long, stack_minb;
+  int stack_cross_rows, stack_long, stack_minb, stack_dev;
   int stack_layout[24];    // stack::Layout, kept opaque here
   std::map<GraphKey, GraphEntry> graphs;
   GraphEntry enc_graph;    // the encoder's launch sequence (fixed for a session), captured on its second use

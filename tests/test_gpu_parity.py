@@ -627,6 +627,32 @@ def test_staged_encoder_rows_change_nothing(bpd, w, path):
     model.close()
 
 
+def test_one_session_per_device_takes_the_persistent_kernel(bpd):
+    """Two persistent layer kernels running at once could keep each other's clusters off the SMs, so the library
+    gives that kernel to one live session per device: a second session created meanwhile runs the cluster launches,
+    decodes the same ids, and the kernel is free again once its holder is closed."""
+    w = MIDI
+    blob, model, src, src_len, om = _setup(bpd, w)
+    k, N = w.cfg.k_model, w.n_decode
+    a = bpd.Session(model, w.batch, w.max_src, N)
+    b = bpd.Session(model, w.batch, w.max_src, N)
+    assert (a.layer_path, b.layer_path) == (2, 1)
+    forced = bpd.Session(model, w.batch, w.max_src, N, options=LAYER_PATHS["persistent"])
+    assert forced.layer_path == 2                 # an explicit request is honoured
+    forced.close()
+    ids = []
+    for s in (a, b, a, b):                        # decodes of the two sessions follow one another on one stream
+        s.bpd_encode(src, src_len)
+        ids.append(s.bpd_decode_blockwise(k, N)[0])
+    assert np.array_equal(ids[0], ids[2]) and np.array_equal(ids[1], ids[3])
+    b.bpd_encode(src, src_len)
+    assert np.array_equal(b.bpd_decode_greedy(N)[0], ids[1])
+    a.close()
+    c = bpd.Session(model, w.batch, w.max_src, N)
+    assert c.layer_path == 2
+    c.close(); b.close(); model.close()
+
+
 def test_same_decode_twice_gives_identical_ids(bpd):
     """Every reduction has a fixed order: decoding the same input twice gives bit-identical hidden states and ids
     (an order-dependent reduction -- a race between CTAs -- would show up as a difference)."""
