@@ -37,6 +37,8 @@ NOMINAL_HBM_GBS = 8000.0
 # summarised under profiles/ (None until a capture of the current kernel exists)
 TRAFFIC = {"C3": 538161152 + 3223296}     # profiles/head_output_gemm_tc_c3.txt
 TRAFFIC_LAYERS = {"C3": 178899200 + 4904448}   # profiles/layer_stack_kernel_c3.txt
+# both lazy stages of the head output layers, per pass (profiles/projection_kernels_c4_batch32_tensor_pipe.txt)
+TRAFFIC_PAIR = {"C4": int((138.4 + 3.7 + 844.4 + 3.2) * 1e6)}
 
 
 def _peaks():
@@ -338,7 +340,7 @@ def run_gpu(args):
         achieved = flops / (pair_us * 1e-6) / 1e12
         roofline = {"bound": "tensor", "kernel": "head output layers, both lazy stages (k*d_model x k*d_hidden weights)",
                     "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf,
-                    "peak_kind": f"of {peak_kind} (sustained bf16)", "traffic": None,
+                    "peak_kind": f"of {peak_kind} (sustained bf16)", "traffic": TRAFFIC_PAIR.get(args.workload),
                     "flops_per_pass": flops, "us_per_pass": pair_us, "launches_timed": n_w2}
     phase_us = {name: (1e3 * ms / max(1, n)) for name, (n, ms) in
                 zip(["layers", "head_hidden", "head_output", "vocab_top1"], phases)}
