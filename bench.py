@@ -36,7 +36,7 @@ NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu capture
 # summarised under profiles/ (None until a capture of the current kernel exists)
 TRAFFIC = {"C3": 538161152 + 3223296}     # profiles/head_output_gemm_tc_c3.txt
-TRAFFIC_LAYERS = {"C3": 178899200 + 4904448}   # profiles/layer_stack_kernel_c3.txt
+TRAFFIC_LAYERS = {"C3": 178907648 + 4899328}   # profiles/layer_stack_kernel_c3.txt
 # both lazy stages of the head output layers, per pass (profiles/projection_kernels_c4_batch32_tensor_pipe.txt)
 TRAFFIC_PAIR = {"C4": int((138.4 + 3.7 + 844.4 + 3.2) * 1e6)}
 
