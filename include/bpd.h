@@ -278,8 +278,12 @@ int bpd_op_vocab_argmax(const void* x, const void* w, int rows, int d, int vocab
  * (BPD_E_SHAPE, as for bpd_op_vocab_argmax); a refused call leaves the outputs
  * untouched.  Arguments as bpd_op_vocab_argmax, minus the scratch.
  * The call performs no cudaMalloc/cudaFree and uses no allocating library.
- * The first call on each device looks the array's device address up (with that
- * device current); make that first call outside any stream capture.  All calls
+ * The first call on each device is a set-up call: it looks the array's device
+ * address up (with that device current), and, as with any kernel, the CUDA
+ * driver loads the kernel's code when a data type is first launched (memory of
+ * the driver's own: about 2 MiB in a fresh process) -- make one call per device
+ * and data type at start-up, outside any stream capture; from then on the
+ * device's free memory stays exactly as it is across calls.  All calls
  * share the one array: the call clears the arrival counters it needs, but two
  * calls whose kernels may overlap on the GPU (different streams, or different
  * host threads) race on it -- keep them on one stream or serialise them. */

@@ -42,6 +42,14 @@ def test_noalloc_matches_definition_and_workspace_variant_twice(dtype):
     w = w.cuda()
     out_idx = torch.empty(64, dtype=torch.int32, device="cuda")
     out_val = torch.empty(64, dtype=torch.float32, device="cuda")
+    # The first call on a device is the set-up call: the library looks up its array's address, and the CUDA driver
+    # loads the kernel's code when it is first launched (the driver's own memory, 2 MiB in a fresh process; nothing
+    # when other tests have launched that kernel before).  Embedders make it once at start-up; the calls after it
+    # must leave the device's free memory exactly as it was.
+    x0 = torch.randn(1, 512, generator=g).to(td).cuda()
+    bpd.bpd_op_vocab_argmax_noalloc(x0, w, out_idx[:1], out_val[:1])
+    torch.cuda.synchronize()
+    _check_against_definition(x0, w, out_idx[:1], out_val[:1], "set-up call")
     for call, rows in enumerate((64, 37)):          # second call: fewer rows over the used workspace
         x = torch.randn(rows, 512, generator=g).to(td)
         x[0] = (w[3].float().cpu() * 50).to(td)
